@@ -1,0 +1,199 @@
+/*
+ * paac.h -- C boundary of the B200 parallel advantage actor-critic (PAAC) library.
+ *
+ * One context holds one learner: the parameters theta of a CNN with a softmax
+ * policy head and a scalar value head (Section 5.1 of the paper), n_e synthetic
+ * environments, and the RMSProp state.  paac_rollout() and paac_update() are the
+ * two halves of one pass of Algorithm 1; everything they compute runs in CUDA
+ * kernels on the device of the context.  There is no CPU fallback: every entry
+ * point that needs the GPU fails with PAAC_ERR_CUDA when it is not there.
+ *
+ * Conventions
+ *   - All functions return an int status (PAAC_OK = 0) unless stated; nothing is
+ *     printed, nothing aborts.  paac_strerror() names a status.
+ *   - "host" / "device" on a pointer says where the memory lives.
+ *   - A context is not thread-safe.  Calls must follow init -> (rollout -> update)*.
+ *   - Work is enqueued on the stream given at init; calls that return data to the
+ *     host synchronise that stream, the others do not.
+ *   - Indices: t in [0, t_max) is the step inside the current rollout, e in [0, n_e)
+ *     the environment, i = t*n_e + e the experience inside the update batch of
+ *     B = n_e*t_max.  Frames are uint8 [84][84][4] (row, column, channel).
+ *   - Canonical parameter vector (float): layers conv1, conv2, [conv3], fc, policy
+ *     head, value head; each layer W then b; conv W as [c_out][k_h][k_w][c_in];
+ *     fc W as [out][in] with in enumerated (row, column, channel).
+ */
+#ifndef PAAC_H_
+#define PAAC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct paac_ctx paac_ctx;   /* opaque, owned by the library */
+
+/* The two networks of Section 5.1 (layer sizes from the papers it cites):
+ * NIPS:   conv 16@8x8/4, conv 32@4x4/2, fc 256
+ * NATURE: conv 32@8x8/4, conv 64@4x4/2, conv 64@3x3/1, fc 512      (ReLU, VALID) */
+enum { PAAC_ARCH_NIPS = 0, PAAC_ARCH_NATURE = 1 };
+
+/* PAAC_FP32: float storage and arithmetic.
+ * PAAC_BF16: bfloat16 weights copies, activations and activation gradients,
+ *            float accumulation, float master parameters and optimiser. */
+enum { PAAC_FP32 = 0, PAAC_BF16 = 1 };
+
+enum {
+  PAAC_OK = 0,
+  PAAC_ERR_ARG = 1,        /* null pointer, size or enum out of range */
+  PAAC_ERR_WORKSPACE = 2,  /* caller's workspace too small or misaligned */
+  PAAC_ERR_CUDA = 3,       /* a CUDA call failed (no device, launch error, ...) */
+  PAAC_ERR_NONFINITE = 4,  /* gradient norm was inf/nan: the update was skipped */
+  PAAC_ERR_TIMEOUT = 5,    /* a bounded device-side wait gave up */
+  PAAC_ERR_STATE = 6       /* call out of order (update without a fresh rollout, ...) */
+};
+
+/* Hyper-parameters.  paac_default_hparams() fills in the values of Section 5.1:
+ * gamma 0.99, RMSProp learning rate 0.0224 (= 0.0007 * 32), decay 0.99, epsilon 0.1,
+ * clipping threshold 40, entropy weight beta 0.01. */
+typedef struct {
+  float gamma;          /* discount of the n-step return */
+  float lr;             /* RMSProp step size alpha */
+  float rms_decay;      /* RMSProp decay of the squared-gradient average */
+  float rms_eps;        /* RMSProp epsilon, inside the square root */
+  float clip_norm;      /* global L2-norm threshold; <= 0 disables clipping */
+  float entropy_beta;   /* weight of the entropy bonus */
+  float value_coef;     /* weight of (R - V)^2; Algorithm 1 has no 1/2, so 1 */
+  uint32_t term_denom;  /* synthetic environment: a transition is terminal with probability 1/term_denom */
+  int precision;        /* PAAC_FP32 or PAAC_BF16 */
+  void* workspace;      /* device; caller-owned scratch of >= paac_workspace_bytes(), 256-byte aligned;
+                           NULL: the library allocates and owns it */
+  size_t workspace_bytes;
+  void* stream;         /* cudaStream_t the work is enqueued on; NULL: the default stream */
+} paac_hparams;
+
+void paac_default_hparams(paac_hparams* hp /* host, out */);
+
+/* Bytes of device scratch a context of this shape needs (0 on bad arguments). */
+size_t paac_workspace_bytes(int arch, int n_e, int t_max, int n_actions, const paac_hparams* hp /* host */);
+
+/* Algorithm 1, first two lines: N = 0, theta Xavier-uniform from `seed` (biases and
+ * RMSProp state zero), n_e environments put in their start states.
+ * n_e in [1, 65536], t_max in [1, 64], n_actions in [2, 32].  *out is set only on PAAC_OK. */
+int paac_init(paac_ctx** out /* host */, int arch, int n_e, int t_max, int n_actions,
+              const paac_hparams* hp /* host */, uint64_t seed);
+
+/* Device pointers into the context's buffers, valid until the next paac_rollout()
+ * or paac_destroy() on the same context.  Borrowed: never free them. */
+typedef struct {
+  const uint8_t* frames;      /* device [t_max][n_e][84][84][4]: s_t for t = 0..t_max-1 */
+  const uint8_t* next_frames; /* device [n_e][84][84][4]: s_{t_max}, the state the next rollout starts from */
+  const int32_t* actions;     /* device [t_max][n_e] */
+  const int8_t* rewards;      /* device [t_max][n_e], in {-1, 0, 1}: reward for a_t taken in s_t */
+  const uint8_t* terminals;   /* device [t_max][n_e]: 1 if that transition ended an episode */
+  const float* values;        /* device [t_max+1][n_e]: V(s_t); row t_max is the bootstrap value */
+  const float* logits;        /* device [t_max][n_e][n_actions] */
+  const float* uniforms;      /* device [t_max][n_e]: the uniform that picked a_t */
+} paac_rollout_view;
+
+/* Algorithm 1, the inner loop and the bootstrap: for t = 0..t_max-1 evaluate the
+ * network on s_t for all environments, sample a_t from the softmax policy by
+ * inverse CDF with a Philox4x32-10 uniform, step every environment; then evaluate
+ * V on the final states.  Asynchronous.  view may be NULL. */
+int paac_rollout(paac_ctx* ctx, paac_rollout_view* view /* host, out, nullable */);
+
+typedef struct {
+  float policy_loss;   /* -(1/B) sum adv_i log pi(a_i | s_i) */
+  float value_loss;    /* (value_coef/B) sum (R_i - V_i)^2 */
+  float entropy;       /* (1/B) sum H(pi(. | s_i)) */
+  float grad_norm;     /* global L2 norm before clipping */
+  float clip_scale;    /* factor applied to the gradient (1 when not clipped) */
+  int32_t status;      /* PAAC_OK or PAAC_ERR_NONFINITE */
+  uint64_t timesteps;  /* N after this update */
+} paac_update_stats;
+
+/* Algorithm 1 after the inner loop: returns R_t = r_t + gamma (1 - terminal_t) R_{t+1}
+ * from the bootstrap value, advantages R_t - V(s_t) (constants), the batch-mean
+ * gradient of  -adv log pi - beta H + value_coef (R - V)^2  (Eqs. 9-10) through the
+ * whole network, global-norm clipping, RMSProp, N += n_e * t_max.
+ * stats == NULL: asynchronous.  stats != NULL: synchronises and fills it; returns
+ * PAAC_ERR_NONFINITE if the update was skipped. */
+int paac_update(paac_ctx* ctx, paac_update_stats* stats /* host, out, nullable */);
+
+size_t paac_param_count(const paac_ctx* ctx);
+
+/* Copy the float master parameters (canonical layout) to the host; n must equal
+ * paac_param_count().  Synchronises. */
+int paac_params(paac_ctx* ctx, float* dst /* host */, size_t n);
+
+/* Release the context and what it owns (never the caller's workspace). */
+int paac_destroy(paac_ctx* ctx);
+
+const char* paac_strerror(int status);
+
+/* ---- external-environment mode: the emulators of Algorithm 1's parallel-for live on
+ * the host (as in the paper's set-up); frames come in, actions go out ---- */
+
+/* Step t of a rollout with host frames s_t [n_e][84][84][4] (pinned memory advised):
+ * copies them in, evaluates the network, samples a_t, copies actions (and values, if
+ * values != NULL) out.  t == t_max evaluates the bootstrap value only (actions may be
+ * NULL).  Synchronises.  t must run 0, 1, ..., t_max in order. */
+int paac_act_host(paac_ctx* ctx, int t, const uint8_t* frames /* host */, int32_t* actions /* host, out */,
+                  float* values /* host, out, nullable */);
+
+/* Outcome of the actions of step t, observed on the host: rewards in {-1,0,1} and
+ * terminal flags, [n_e] each.  After step t_max-1 and the bootstrap paac_act_host(t_max),
+ * paac_update() may be called. */
+int paac_observe_host(paac_ctx* ctx, int t, const int8_t* rewards /* host */, const uint8_t* terminals /* host */);
+
+/* ---- test and resume hooks ---- */
+
+/* Overwrite the master parameters (and their bf16 copies) from the host. Synchronises. */
+int paac_set_params(paac_ctx* ctx, const float* src /* host */, size_t n);
+
+/* Actions to take instead of sampling in the following rollouts: host int32
+ * [t_max][n_e], -1 = sample as usual.  NULL clears.  Lets a checker walk in lock
+ * step when a uniform falls within rounding of a CDF boundary. */
+int paac_force_actions(paac_ctx* ctx, const int32_t* actions /* host, nullable */);
+
+/* Internal tensors readable through paac_debug_read (storage type in brackets;
+ * "T" is float in PAAC_FP32 and bfloat16 in PAAC_BF16). */
+enum {
+  PAAC_DBG_FRAMES = 0,     /* u8  [t_max][n_e][84][84][4] */
+  PAAC_DBG_NEXT_FRAMES,    /* u8  [n_e][84][84][4] */
+  PAAC_DBG_ACTIONS,        /* i32 [t_max][n_e] */
+  PAAC_DBG_REWARDS,        /* i8  [t_max][n_e] */
+  PAAC_DBG_TERMINALS,      /* u8  [t_max][n_e] */
+  PAAC_DBG_VALUES,         /* f32 [t_max+1][n_e] */
+  PAAC_DBG_LOGITS,         /* f32 [t_max][n_e][A] */
+  PAAC_DBG_UNIFORMS,       /* f32 [t_max][n_e] */
+  PAAC_DBG_COUNTERS,       /* i32 [3][n_e]: episode length, episode return, episodes finished */
+  PAAC_DBG_RETURNS,        /* f32 [B] */
+  PAAC_DBG_ADVANTAGES,     /* f32 [B] */
+  PAAC_DBG_DLOGITS,        /* f32 [B][A] */
+  PAAC_DBG_DVALUES,        /* f32 [B] */
+  PAAC_DBG_GRAD,           /* f32 [P] gradient of the last update, before clipping */
+  PAAC_DBG_RMS,            /* f32 [P] RMSProp state */
+  PAAC_DBG_SAMPLED,        /* i32 [t_max][n_e]: the action inverse-CDF sampling gave, before any forcing */
+  PAAC_DBG_ACT0 = 32,      /* T [B][...] stored activation of layer l = which - PAAC_DBG_ACT0
+                              (conv layers, then fc) */
+  PAAC_DBG_GACT0 = 48      /* T [B][...] gradient w.r.t. the pre-activation of layer l */
+};
+
+/* Bytes of tensor `which` (0 if unknown). */
+size_t paac_debug_bytes(const paac_ctx* ctx, int which);
+/* Copy tensor `which` to the host; bytes must equal paac_debug_bytes(). Synchronises. */
+int paac_debug_read(paac_ctx* ctx, int which, void* dst /* host */, size_t bytes);
+/* Overwrite tensor `which` from the host (fault injection from the host side, e.g. a
+ * poisoned gradient is not possible here since the gradient is recomputed; used for
+ * PAAC_DBG_RMS and PAAC_DBG_COUNTERS on resume). Synchronises. */
+int paac_debug_write(paac_ctx* ctx, int which, const void* src /* host */, size_t bytes);
+
+/* Number of kernels the library has launched on this context since init. */
+uint64_t paac_launch_count(const paac_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PAAC_H_ */

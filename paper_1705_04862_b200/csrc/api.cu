@@ -1,0 +1,379 @@
+// C boundary of the PAAC library: context, workspace carving, and the order in which the
+// kernels of one pass of Algorithm 1 are enqueued.
+#include <new>
+#include <string.h>
+
+#include "kernels.h"
+
+using namespace paac;
+
+struct paac_ctx {
+  int arch, n_e, t_max, A, prec, B;
+  paac_hparams hp;
+  uint64_t seed;
+  NetDims nd;
+  cudaStream_t st;
+  int device;
+  bool owns_workspace;
+  char* ws;
+  size_t ws_bytes;
+  uint64_t launches;
+  uint64_t N;              // timesteps consumed by updates
+  uint64_t env_step;       // global step index of the environments (same for all)
+  bool rollout_fresh;      // a rollout has completed since the last update
+  int host_t;              // external-environment mode: next expected step
+  bool forced_on;
+
+  // device buffers (all inside the workspace)
+  float *theta, *grad, *rms;
+  bf16* theta16;
+  uint8_t* frames[2];      // [t_max][n_e][FRAME_BYTES] each; rollouts alternate, the bootstrap state of one
+                           // rollout is written straight into slot 0 of the other
+  int cur;                 // buffer the last / current rollout used
+  void* act[MAX_LAYERS];   // [(t_max+1)*n_e][out_size], slot t_max is bootstrap scratch
+  void* gact[MAX_LAYERS];  // [B][out_size]
+  float *logits, *values, *uniforms, *R, *adv, *dz, *dV, *loss_terms, *scratch, *norm_partials;
+  int32_t *actions, *sampled, *forced, *counters;
+  int8_t* rewards;
+  uint8_t* terminals;
+  DeviceStats* stats;
+  size_t elt;              // bytes of one stored activation element
+};
+
+namespace {
+
+struct Carver {
+  char* base; size_t off;
+  template <class T> T* take(size_t count) {
+    off = (off + 255) & ~(size_t)255;
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += count * sizeof(T);
+    return p;
+  }
+};
+
+bool valid_shape(int arch, int n_e, int t_max, int A, const paac_hparams* hp) {
+  if (hp == nullptr) return false;
+  if (arch != PAAC_ARCH_NIPS && arch != PAAC_ARCH_NATURE) return false;
+  if (hp->precision != PAAC_FP32 && hp->precision != PAAC_BF16) return false;
+  if (n_e < 1 || n_e > 65536 || t_max < 1 || t_max > 64 || A < 2 || A > 32) return false;
+  if ((long long)n_e * (t_max + 1) > 131072) return false;   // keeps every row index below 2^31
+  if (hp->term_denom == 0) return false;
+  return true;
+}
+
+// lays the buffers out; with base == nullptr only measures
+size_t carve(paac_ctx* c, char* base) {
+  Carver k{base, 0};
+  const NetDims& nd = c->nd;
+  const size_t n_e = c->n_e, T = c->t_max, B = c->B, A = c->A;
+  c->theta = k.take<float>(nd.P);
+  c->grad = k.take<float>(nd.P);
+  c->rms = k.take<float>(nd.P);
+  c->theta16 = k.take<bf16>(nd.P);
+  c->frames[0] = k.take<uint8_t>(T * n_e * FRAME_BYTES);
+  c->frames[1] = k.take<uint8_t>(T * n_e * FRAME_BYTES);
+  for (int l = 0; l <= nd.n_conv; ++l) {
+    c->act[l] = k.take<char>((T + 1) * n_e * nd.layer[l].out_size * c->elt);
+    c->gact[l] = k.take<char>(B * nd.layer[l].out_size * c->elt);
+  }
+  c->logits = k.take<float>((T + 1) * n_e * A);
+  c->values = k.take<float>((T + 1) * n_e);
+  c->uniforms = k.take<float>(B);
+  c->R = k.take<float>(B);
+  c->adv = k.take<float>(B);
+  c->dz = k.take<float>(B * A);
+  c->dV = k.take<float>(B);
+  c->loss_terms = k.take<float>(3 * B);
+  c->scratch = k.take<float>(simt_scratch_floats(c->arch, nd, (int)B));
+  c->norm_partials = k.take<float>(NORM_BLOCKS);
+  c->actions = k.take<int32_t>(B);
+  c->sampled = k.take<int32_t>(B);
+  c->forced = k.take<int32_t>(B);
+  c->counters = k.take<int32_t>(3 * n_e);
+  c->rewards = k.take<int8_t>(B);
+  c->terminals = k.take<uint8_t>(B);
+  c->stats = k.take<DeviceStats>(1);
+  return (k.off + 255) & ~(size_t)255;
+}
+
+void fill_shape(paac_ctx* c, int arch, int n_e, int t_max, int A, const paac_hparams* hp) {
+  c->arch = arch; c->n_e = n_e; c->t_max = t_max; c->A = A; c->B = n_e * t_max;
+  c->hp = *hp; c->prec = hp->precision;
+  c->nd = make_net(arch, A);
+  c->elt = hp->precision == PAAC_BF16 ? 2 : 4;
+}
+
+int cuda_status(paac_ctx* c) {
+  (void)c;
+  return cudaGetLastError() == cudaSuccess ? PAAC_OK : PAAC_ERR_CUDA;
+}
+
+// network + heads on the n_e states of `frames`, activations into slot `slot`
+void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, uint64_t step) {
+  void* act[MAX_LAYERS];
+  for (int l = 0; l <= c->nd.n_conv; ++l)
+    act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
+  simt_forward(c->st, &c->launches, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
+  const size_t row = (size_t)slot * c->n_e;
+  launch_heads(c->st, &c->launches, c->prec, c->nd, c->theta, c->theta16, act[c->nd.n_conv], c->n_e,
+               c->logits + row * c->A, c->values + row, c->seed, step,
+               sample && c->forced_on ? c->forced + row : nullptr, sample ? c->actions + row : nullptr,
+               sample ? c->sampled + row : nullptr, sample ? c->uniforms + row : nullptr);
+}
+
+}  // namespace
+
+extern "C" {
+
+void paac_default_hparams(paac_hparams* hp) {
+  if (!hp) return;
+  memset(hp, 0, sizeof(*hp));
+  hp->gamma = 0.99f; hp->lr = 0.0224f; hp->rms_decay = 0.99f; hp->rms_eps = 0.1f;
+  hp->clip_norm = 40.f; hp->entropy_beta = 0.01f; hp->value_coef = 1.f;
+  hp->term_denom = 200; hp->precision = PAAC_FP32;
+}
+
+size_t paac_workspace_bytes(int arch, int n_e, int t_max, int n_actions, const paac_hparams* hp) {
+  if (!valid_shape(arch, n_e, t_max, n_actions, hp)) return 0;
+  paac_ctx tmp{};
+  fill_shape(&tmp, arch, n_e, t_max, n_actions, hp);
+  return carve(&tmp, nullptr);
+}
+
+int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const paac_hparams* hp, uint64_t seed) {
+  if (!out || !valid_shape(arch, n_e, t_max, n_actions, hp)) return PAAC_ERR_ARG;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  paac_ctx* c = new (std::nothrow) paac_ctx{};
+  if (!c) return PAAC_ERR_CUDA;
+  fill_shape(c, arch, n_e, t_max, n_actions, hp);
+  c->seed = seed; c->device = dev; c->st = (cudaStream_t)hp->stream;
+  const size_t need = carve(c, nullptr);
+  if (hp->workspace) {
+    if (hp->workspace_bytes < need || ((uintptr_t)hp->workspace & 255)) { delete c; return PAAC_ERR_WORKSPACE; }
+    c->ws = (char*)hp->workspace; c->owns_workspace = false;
+  } else {
+    if (cudaMalloc((void**)&c->ws, need) != cudaSuccess) { cudaGetLastError(); delete c; return PAAC_ERR_CUDA; }
+    c->owns_workspace = true;
+  }
+  c->ws_bytes = need;
+  carve(c, c->ws);
+  cudaMemsetAsync(c->ws, 0, need, c->st);
+  cudaMemsetAsync(c->forced, 0xFF, (size_t)c->B * sizeof(int32_t), c->st);
+  launch_init_params(c->st, &c->launches, c->nd, seed, c->theta);
+  launch_cast_bf16(c->st, &c->launches, c->theta, c->theta16, c->nd.P);
+  c->cur = 1;   // the first rollout flips to buffer 0; its start states are written there now
+  launch_env_step(c->st, &c->launches, seed, n_e, 0u, nullptr, hp->term_denom, c->frames[0], nullptr, nullptr, nullptr);
+  if (cudaStreamSynchronize(c->st) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
+    if (c->owns_workspace) cudaFree(c->ws);
+    delete c;
+    return PAAC_ERR_CUDA;
+  }
+  *out = c;
+  return PAAC_OK;
+}
+
+int paac_rollout(paac_ctx* c, paac_rollout_view* view) {
+  if (!c) return PAAC_ERR_ARG;
+  if (c->host_t != 0) return PAAC_ERR_STATE;
+  c->cur ^= 1;
+  uint8_t* fr = c->frames[c->cur];
+  uint8_t* nxt = c->frames[c->cur ^ 1];
+  const size_t fstep = (size_t)c->n_e * FRAME_BYTES;
+  for (int t = 0; t < c->t_max; ++t) {
+    forward_slot(c, fr + t * fstep, t, true, c->env_step + t);
+    uint8_t* dst = t + 1 < c->t_max ? fr + (t + 1) * fstep : nxt;
+    const size_t row = (size_t)t * c->n_e;
+    launch_env_step(c->st, &c->launches, c->seed, c->n_e, (uint32_t)(c->env_step + t), c->actions + row,
+                    c->hp.term_denom, dst, c->rewards + row, c->terminals + row, c->counters);
+  }
+  forward_slot(c, nxt, c->t_max, false, 0);
+  c->env_step += c->t_max;
+  c->rollout_fresh = true;
+  if (view) {
+    view->frames = fr; view->next_frames = nxt; view->actions = c->actions; view->rewards = c->rewards;
+    view->terminals = c->terminals; view->values = c->values; view->logits = c->logits; view->uniforms = c->uniforms;
+  }
+  return cuda_status(c);
+}
+
+int paac_update(paac_ctx* c, paac_update_stats* stats) {
+  if (!c) return PAAC_ERR_ARG;
+  if (!c->rollout_fresh) return PAAC_ERR_STATE;
+  const paac_hparams& hp = c->hp;
+  launch_returns(c->st, &c->launches, c->n_e, c->t_max, hp.gamma, c->rewards, c->terminals, c->values, c->R, c->adv);
+  launch_head_grad(c->st, &c->launches, c->B, c->A, hp.entropy_beta, hp.value_coef, c->logits, c->values, c->actions,
+                   c->R, c->adv, c->dz, c->dV, c->loss_terms, c->stats);
+  const int L = c->nd.n_conv;
+  heads_backward(c->st, &c->launches, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
+                 c->grad, c->scratch);
+  simt_backward(c->st, &c->launches, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
+                c->gact, c->grad, c->scratch);
+  launch_clip_rmsprop(c->st, &c->launches, c->nd.P, c->theta, c->rms, c->grad,
+                      c->prec == PAAC_BF16 ? c->theta16 : nullptr, hp.lr, hp.rms_decay, hp.rms_eps, hp.clip_norm,
+                      c->norm_partials, c->stats);
+  c->N += (uint64_t)c->B;
+  c->rollout_fresh = false;
+  if (cuda_status(c) != PAAC_OK) return PAAC_ERR_CUDA;
+  if (stats) {
+    DeviceStats ds;
+    if (cudaMemcpyAsync(&ds, c->stats, sizeof(ds), cudaMemcpyDeviceToHost, c->st) != cudaSuccess ||
+        cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+    stats->policy_loss = ds.policy_loss; stats->value_loss = ds.value_loss; stats->entropy = ds.entropy;
+    stats->grad_norm = ds.grad_norm; stats->clip_scale = ds.clip_scale; stats->status = ds.status;
+    stats->timesteps = c->N;
+    if (ds.error_word) return PAAC_ERR_TIMEOUT;
+    if (ds.status != PAAC_OK) return ds.status;
+  }
+  return PAAC_OK;
+}
+
+size_t paac_param_count(const paac_ctx* c) { return c ? c->nd.P : 0; }
+
+int paac_params(paac_ctx* c, float* dst, size_t n) {
+  if (!c || !dst || n != c->nd.P) return PAAC_ERR_ARG;
+  if (cudaMemcpyAsync(dst, c->theta, n * sizeof(float), cudaMemcpyDeviceToHost, c->st) != cudaSuccess ||
+      cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  return PAAC_OK;
+}
+
+int paac_set_params(paac_ctx* c, const float* src, size_t n) {
+  if (!c || !src || n != c->nd.P) return PAAC_ERR_ARG;
+  if (cudaMemcpyAsync(c->theta, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
+    cudaGetLastError(); return PAAC_ERR_CUDA;
+  }
+  launch_cast_bf16(c->st, &c->launches, c->theta, c->theta16, n);
+  if (cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  return cuda_status(c);
+}
+
+int paac_force_actions(paac_ctx* c, const int32_t* actions) {
+  if (!c) return PAAC_ERR_ARG;
+  if (!actions) { c->forced_on = false; return PAAC_OK; }
+  for (int i = 0; i < c->B; ++i)
+    if (actions[i] < -1 || actions[i] >= c->A) return PAAC_ERR_ARG;
+  if (cudaMemcpyAsync(c->forced, actions, (size_t)c->B * sizeof(int32_t), cudaMemcpyHostToDevice, c->st) != cudaSuccess ||
+      cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  c->forced_on = true;
+  return PAAC_OK;
+}
+
+int paac_destroy(paac_ctx* c) {
+  if (!c) return PAAC_ERR_ARG;
+  cudaStreamSynchronize(c->st);
+  if (c->owns_workspace) cudaFree(c->ws);
+  cudaGetLastError();
+  delete c;
+  return PAAC_OK;
+}
+
+const char* paac_strerror(int s) {
+  switch (s) {
+    case PAAC_OK: return "ok";
+    case PAAC_ERR_ARG: return "bad argument";
+    case PAAC_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case PAAC_ERR_CUDA: return "CUDA error (no device, allocation or launch failure)";
+    case PAAC_ERR_NONFINITE: return "gradient norm not finite: update skipped";
+    case PAAC_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case PAAC_ERR_STATE: return "call out of order";
+    default: return "unknown status";
+  }
+}
+
+uint64_t paac_launch_count(const paac_ctx* c) { return c ? c->launches : 0; }
+
+// ---- external-environment mode ------------------------------------------------------------------
+int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, float* values) {
+  if (!c || !frames || t < 0 || t > c->t_max || (t < c->t_max && !actions)) return PAAC_ERR_ARG;
+  if (t != c->host_t) return PAAC_ERR_STATE;
+  const size_t fstep = (size_t)c->n_e * FRAME_BYTES;
+  if (t == 0) c->cur ^= 1;
+  uint8_t* dst = t < c->t_max ? c->frames[c->cur] + t * fstep : c->frames[c->cur ^ 1];
+  if (cudaMemcpyAsync(dst, frames, fstep, cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
+    cudaGetLastError(); return PAAC_ERR_CUDA;
+  }
+  const bool sample = t < c->t_max;
+  forward_slot(c, dst, t, sample, c->env_step + t);
+  const size_t row = (size_t)t * c->n_e;
+  if (sample) cudaMemcpyAsync(actions, c->actions + row, c->n_e * sizeof(int32_t), cudaMemcpyDeviceToHost, c->st);
+  if (values) cudaMemcpyAsync(values, c->values + row, c->n_e * sizeof(float), cudaMemcpyDeviceToHost, c->st);
+  if (cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  if (t == c->t_max) { c->host_t = 0; c->env_step += c->t_max; c->rollout_fresh = true; }
+  else c->host_t = t + 1;
+  return cuda_status(c);
+}
+
+int paac_observe_host(paac_ctx* c, int t, const int8_t* rewards, const uint8_t* terminals) {
+  if (!c || !rewards || !terminals || t < 0 || t >= c->t_max) return PAAC_ERR_ARG;
+  if (t + 1 != c->host_t) return PAAC_ERR_STATE;
+  const size_t row = (size_t)t * c->n_e;
+  if (cudaMemcpyAsync(c->rewards + row, rewards, c->n_e, cudaMemcpyHostToDevice, c->st) != cudaSuccess ||
+      cudaMemcpyAsync(c->terminals + row, terminals, c->n_e, cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
+    cudaGetLastError(); return PAAC_ERR_CUDA;
+  }
+  return PAAC_OK;
+}
+
+// ---- debug access -----------------------------------------------------------------------------------
+static void* debug_ptr(const paac_ctx* c, int which, size_t* bytes) {
+  const size_t n_e = c->n_e, T = c->t_max, B = c->B, A = c->A, P = c->nd.P;
+  switch (which) {
+    case PAAC_DBG_FRAMES: *bytes = T * n_e * FRAME_BYTES; return c->frames[c->cur];
+    case PAAC_DBG_NEXT_FRAMES: *bytes = n_e * FRAME_BYTES; return c->frames[c->cur ^ 1];
+    case PAAC_DBG_ACTIONS: *bytes = B * 4; return c->actions;
+    case PAAC_DBG_REWARDS: *bytes = B; return c->rewards;
+    case PAAC_DBG_TERMINALS: *bytes = B; return c->terminals;
+    case PAAC_DBG_VALUES: *bytes = (T + 1) * n_e * 4; return c->values;
+    case PAAC_DBG_LOGITS: *bytes = B * A * 4; return c->logits;
+    case PAAC_DBG_UNIFORMS: *bytes = B * 4; return c->uniforms;
+    case PAAC_DBG_COUNTERS: *bytes = 3 * n_e * 4; return c->counters;
+    case PAAC_DBG_RETURNS: *bytes = B * 4; return c->R;
+    case PAAC_DBG_ADVANTAGES: *bytes = B * 4; return c->adv;
+    case PAAC_DBG_DLOGITS: *bytes = B * A * 4; return c->dz;
+    case PAAC_DBG_DVALUES: *bytes = B * 4; return c->dV;
+    case PAAC_DBG_GRAD: *bytes = P * 4; return c->grad;
+    case PAAC_DBG_RMS: *bytes = P * 4; return c->rms;
+    case PAAC_DBG_SAMPLED: *bytes = B * 4; return c->sampled;
+    default: break;
+  }
+  if (which >= PAAC_DBG_ACT0 && which <= PAAC_DBG_ACT0 + c->nd.n_conv) {
+    const int l = which - PAAC_DBG_ACT0;
+    *bytes = B * c->nd.layer[l].out_size * c->elt; return c->act[l];
+  }
+  if (which >= PAAC_DBG_GACT0 && which <= PAAC_DBG_GACT0 + c->nd.n_conv) {
+    const int l = which - PAAC_DBG_GACT0;
+    *bytes = B * c->nd.layer[l].out_size * c->elt; return c->gact[l];
+  }
+  *bytes = 0;
+  return nullptr;
+}
+
+size_t paac_debug_bytes(const paac_ctx* c, int which) {
+  if (!c) return 0;
+  size_t b = 0;
+  debug_ptr(c, which, &b);
+  return b;
+}
+
+int paac_debug_read(paac_ctx* c, int which, void* dst, size_t bytes) {
+  if (!c || !dst) return PAAC_ERR_ARG;
+  size_t b = 0;
+  void* p = debug_ptr(c, which, &b);
+  if (!p || b != bytes) return PAAC_ERR_ARG;
+  if (cudaMemcpyAsync(dst, p, b, cudaMemcpyDeviceToHost, c->st) != cudaSuccess ||
+      cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  return PAAC_OK;
+}
+
+int paac_debug_write(paac_ctx* c, int which, const void* src, size_t bytes) {
+  if (!c || !src) return PAAC_ERR_ARG;
+  size_t b = 0;
+  void* p = debug_ptr(c, which, &b);
+  if (!p || b != bytes) return PAAC_ERR_ARG;
+  if (cudaMemcpyAsync(p, src, b, cudaMemcpyHostToDevice, c->st) != cudaSuccess ||
+      cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  return PAAC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,133 @@
+// Shared device helpers and the context layout of the PAAC library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/paac.h"
+
+namespace paac {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int FRAME_H = 84, FRAME_W = 84, FRAME_C = 4;
+constexpr int FRAME_BYTES = FRAME_H * FRAME_W * FRAME_C;   // 28,224
+constexpr int MAX_LAYERS = 4;                              // conv layers + fc
+
+// ---- storage type helpers ---------------------------------------------------
+__device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(bf16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ float to_f(uint8_t x) { return (float)x; }
+template <class T> __device__ __forceinline__ T from_f(float x);
+template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float x) { return __float2bfloat16_rn(x); }
+
+// ---- Philox4x32-10 (Salmon et al., SC'11) -------------------------------------
+__host__ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                       uint32_t k0, uint32_t k1, uint32_t out[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    c0 = n0; c1 = (uint32_t)p1; c2 = n2; c3 = (uint32_t)p0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+constexpr uint32_t RNG_STREAM_INIT = 1u, RNG_STREAM_ACTION = 2u;
+
+// 24-bit uniform in [0,1) from the first output word
+__host__ __device__ __forceinline__ float philox_uniform(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t stream,
+                                                         uint64_t seed) {
+  uint32_t o[4];
+  philox4x32_10(c0, c1, c2, stream, (uint32_t)seed, (uint32_t)(seed >> 32), o);
+  return (float)(o[0] >> 8) * (1.0f / 16777216.0f);
+}
+
+// ---- environment hash -----------------------------------------------------------
+constexpr uint32_t HASH_K0 = 0x9E3779B9u, HASH_K1 = 0xBB67AE85u, HASH_K2 = 0x6A09E667u;
+constexpr uint32_t HASH_TAG_REWARD = 0x52455744u, HASH_TAG_TERMINAL = 0x5445524Du;
+
+__host__ __device__ __forceinline__ uint32_t hash_mix(uint32_t x) {
+  x ^= x >> 16; x *= HASH_K0; x ^= x >> 15; x *= HASH_K1; x ^= x >> 16;
+  return x;
+}
+__host__ __device__ __forceinline__ uint32_t env_hash_base(uint64_t seed, uint32_t env, uint32_t step, uint32_t tag) {
+  uint32_t h = hash_mix((uint32_t)seed ^ HASH_K2);
+  h = hash_mix(h ^ (uint32_t)(seed >> 32));
+  h = hash_mix(h ^ env);
+  h = hash_mix(h ^ step);
+  return hash_mix(h ^ tag);
+}
+
+// ---- network geometry (compile time) ----------------------------------------------
+template <int H_, int W_, int C_, int K_, int S_, int CO_>
+struct ConvGeom {
+  static constexpr int H = H_, W = W_, C = C_, K = K_, S = S_, CO = CO_;
+  static constexpr int OH = (H - K) / S + 1, OW = (W - K) / S + 1;
+  static constexpr int KK = K * K * C;          // reduction length of the forward contraction
+  static constexpr int IN_SIZE = H * W * C, OUT_SIZE = OH * OW * CO;
+};
+typedef ConvGeom<84, 84, 4, 8, 4, 16> NipsConv1;
+typedef ConvGeom<20, 20, 16, 4, 2, 32> NipsConv2;
+typedef ConvGeom<84, 84, 4, 8, 4, 32> NatConv1;
+typedef ConvGeom<20, 20, 32, 4, 2, 64> NatConv2;
+typedef ConvGeom<9, 9, 64, 3, 1, 64> NatConv3;
+
+// run-time copy of the same numbers for host-side sizing
+struct LayerDims {
+  int H, W, C, K, S, CO, OH, OW;   // fc: K = S = 0, H*W*C = inputs, CO = outputs, OH = OW = 1
+  size_t w_off, b_off;             // offsets into the canonical parameter vector
+  size_t out_size;                 // elements per state of the stored activation
+};
+
+struct NetDims {
+  int n_conv;
+  LayerDims layer[MAX_LAYERS];     // conv layers then fc
+  int F, A;
+  size_t pi_w, pi_b, v_w, v_b, P;
+};
+
+inline NetDims make_net(int arch, int A) {
+  NetDims n{};
+  const int nips[2][3] = {{16, 8, 4}, {32, 4, 2}};
+  const int nat[3][3] = {{32, 8, 4}, {64, 4, 2}, {64, 3, 1}};
+  n.n_conv = arch == PAAC_ARCH_NIPS ? 2 : 3;
+  n.F = arch == PAAC_ARCH_NIPS ? 256 : 512;
+  n.A = A;
+  int H = FRAME_H, W = FRAME_W, C = FRAME_C;
+  size_t off = 0;
+  for (int l = 0; l < n.n_conv; ++l) {
+    const int* s = arch == PAAC_ARCH_NIPS ? nips[l] : nat[l];
+    LayerDims& d = n.layer[l];
+    d.H = H; d.W = W; d.C = C; d.CO = s[0]; d.K = s[1]; d.S = s[2];
+    d.OH = (H - d.K) / d.S + 1; d.OW = (W - d.K) / d.S + 1;
+    d.w_off = off; off += (size_t)d.CO * d.K * d.K * C;
+    d.b_off = off; off += d.CO;
+    d.out_size = (size_t)d.OH * d.OW * d.CO;
+    H = d.OH; W = d.OW; C = d.CO;
+  }
+  LayerDims& f = n.layer[n.n_conv];
+  f.H = H; f.W = W; f.C = C; f.K = 0; f.S = 0; f.CO = n.F; f.OH = f.OW = 1;
+  f.w_off = off; off += (size_t)H * W * C * n.F;
+  f.b_off = off; off += n.F;
+  f.out_size = n.F;
+  n.pi_w = off; off += (size_t)A * n.F;
+  n.pi_b = off; off += A;
+  n.v_w = off; off += n.F;
+  n.v_b = off; off += 1;
+  n.P = off;
+  return n;
+}
+
+// device-side statistics block written by the update kernels
+struct DeviceStats {
+  float policy_loss, value_loss, entropy, grad_norm, clip_scale;
+  int32_t status;
+  uint32_t error_word;   // bit set by a kernel whose bounded wait or bounds check gave up
+  uint32_t pad;
+};
+
+}  // namespace paac

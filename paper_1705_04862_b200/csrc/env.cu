@@ -1,0 +1,105 @@
+// Parameter initialisation and the synthetic hashed environment.
+#include "kernels.h"
+
+namespace paac {
+
+// Xavier-uniform: element i of weight tensor `layer` is (2u-1)*bound with u the 24-bit
+// Philox uniform of counter (i, layer, 0, RNG_STREAM_INIT).  2u-1 is exact in float, so the
+// single rounding of the product is the same on any IEEE machine.
+__global__ void xavier_kernel(float* w, uint32_t count, float bound, uint32_t layer, uint64_t seed) {
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < count; i += gridDim.x * blockDim.x) {
+    const float u = philox_uniform(i, layer, 0u, RNG_STREAM_INIT, seed);
+    w[i] = __fmul_rn(__fsub_rn(__fmul_rn(2.0f, u), 1.0f), bound);
+  }
+}
+
+static void xavier(cudaStream_t st, uint64_t* launches, float* w, size_t count, double fan_in, double fan_out,
+                   uint32_t layer, uint64_t seed) {
+  const float bound = (float)sqrt(6.0 / (fan_in + fan_out));
+  int blocks = (int)((count + 255) / 256);
+  if (blocks > 1184) blocks = 1184;
+  xavier_kernel<<<blocks, 256, 0, st>>>(w, (uint32_t)count, bound, layer, seed);
+  ++*launches;
+}
+
+void launch_init_params(cudaStream_t st, uint64_t* launches, const NetDims& nd, uint64_t seed, float* theta) {
+  cudaMemsetAsync(theta, 0, nd.P * sizeof(float), st);
+  uint32_t id = 0;
+  for (int l = 0; l < nd.n_conv; ++l, ++id) {
+    const LayerDims& d = nd.layer[l];
+    const double kk = (double)d.K * d.K;
+    xavier(st, launches, theta + d.w_off, (size_t)d.CO * d.K * d.K * d.C, kk * d.C, kk * d.CO, id, seed);
+  }
+  const LayerDims& f = nd.layer[nd.n_conv];
+  const size_t in = (size_t)f.H * f.W * f.C;
+  xavier(st, launches, theta + f.w_off, in * nd.F, (double)in, (double)nd.F, id++, seed);
+  xavier(st, launches, theta + nd.pi_w, (size_t)nd.A * nd.F, (double)nd.F, (double)nd.A, id++, seed);
+  xavier(st, launches, theta + nd.v_w, (size_t)nd.F, (double)nd.F, 1.0, id++, seed);
+}
+
+__global__ void cast_bf16_kernel(const float* src, bf16* dst, size_t n) {
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+    dst[i] = __float2bfloat16_rn(src[i]);
+}
+void launch_cast_bf16(cudaStream_t st, uint64_t* launches, const float* src, bf16* dst, size_t n) {
+  int blocks = (int)((n + 255) / 256);
+  if (blocks > 1184) blocks = 1184;
+  cast_bf16_kernel<<<blocks, 256, 0, st>>>(src, dst, n);
+  ++*launches;
+}
+
+// One block per environment.  The block's first thread decides reward and terminal flag of
+// the transition (seed, env, step, action) and keeps the episode counters; all threads then
+// write the 84x84x4 frame of the state reached, one hashed 32-bit word per pixel (its bytes,
+// little endian, are the four channels), as 16-byte stores.
+constexpr int ENV_THREADS = 256;
+constexpr int FRAME_WORDS = FRAME_H * FRAME_W;   // 7056, a multiple of 4
+
+__global__ void __launch_bounds__(ENV_THREADS)
+env_step_kernel(uint64_t seed, int n_e, uint32_t step, const int32_t* __restrict__ actions, uint32_t term_denom,
+                uint8_t* __restrict__ next_frames, int8_t* __restrict__ rewards, uint8_t* __restrict__ terminals,
+                int32_t* __restrict__ counters) {
+  __shared__ uint32_t s_base;
+  const uint32_t e = blockIdx.x;
+  if (threadIdx.x == 0) {
+    uint32_t tag = 0u, frame_step = 0u;
+    if (actions != nullptr) {
+      const int32_t a = actions[e];
+      const uint32_t base = env_hash_base(seed, e, step, (uint32_t)a + 1u);
+      const uint32_t hr = hash_mix(base ^ HASH_TAG_REWARD) & 15u;
+      const int r = hr == 0u ? 1 : (hr == 1u ? -1 : 0);
+      const uint32_t ht = hash_mix(base ^ HASH_TAG_TERMINAL);
+      const bool term = (uint32_t)(((uint64_t)ht * term_denom) >> 32) == 0u;
+      rewards[e] = (int8_t)r;
+      terminals[e] = term ? 1 : 0;
+      int32_t len = counters[e] + 1, ret = counters[n_e + e] + r;
+      if (term) { counters[2 * n_e + e] += 1; len = 0; ret = 0; }
+      counters[e] = len; counters[n_e + e] = ret;
+      tag = term ? 0u : (uint32_t)a + 1u;
+      frame_step = step + 1u;
+    }
+    s_base = env_hash_base(seed, e, frame_step, tag);
+  }
+  __syncthreads();
+  const uint32_t base = s_base;
+  uint4* out = reinterpret_cast<uint4*>(next_frames + (size_t)e * FRAME_BYTES);
+  for (int q = threadIdx.x; q < FRAME_WORDS / 4; q += ENV_THREADS) {
+    const uint32_t p = (uint32_t)q * 4u + 1u;
+    uint4 v;
+    v.x = hash_mix(base + HASH_K0 * p);
+    v.y = hash_mix(base + HASH_K0 * (p + 1u));
+    v.z = hash_mix(base + HASH_K0 * (p + 2u));
+    v.w = hash_mix(base + HASH_K0 * (p + 3u));
+    out[q] = v;
+  }
+}
+
+void launch_env_step(cudaStream_t st, uint64_t* launches, uint64_t seed, int n_e, uint32_t step,
+                     const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
+                     uint8_t* terminals, int32_t* counters) {
+  env_step_kernel<<<n_e, ENV_THREADS, 0, st>>>(seed, n_e, step, actions, term_denom, next_frames, rewards, terminals,
+                                               counters);
+  ++*launches;
+}
+
+}  // namespace paac

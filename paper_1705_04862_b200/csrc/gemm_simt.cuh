@@ -1,0 +1,194 @@
+// Generic float-accumulating contraction on the CUDA cores:
+//   C(m, n) = sum_k A(m, k) * B(n, k),  k in the split's range,
+// with A, B given as index functors (so convolution windows, transposes and
+// validity masks need no materialised matrix) and the result handed to an
+// epilogue functor.  Used for the fp32 configurations, for the small head
+// layers, and as the portable path every tensor-core kernel is checked against.
+#pragma once
+#include "common.cuh"
+
+namespace paac {
+
+constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16, SG_THREADS = 256;
+
+template <class LA, class LB, class EP>
+__global__ void __launch_bounds__(SG_THREADS)
+gemm_simt_kernel(int M, int N, int K, int k_per_split, LA la, LB lb, EP ep) {
+  __shared__ float As[SG_BK][SG_BM + 4];
+  __shared__ float Bs[SG_BK][SG_BN + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int m0 = blockIdx.x * SG_BM, n0 = blockIdx.y * SG_BN, split = blockIdx.z;
+  const int k_begin = split * k_per_split;
+  const int k_end = min(K, k_begin + k_per_split);
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = k_begin; k0 < k_end; k0 += SG_BK) {
+#pragma unroll
+    for (int i = 0; i < SG_BM * SG_BK / SG_THREADS; ++i) {
+      const int idx = tid + i * SG_THREADS;
+      int kk, mm;
+      if (LA::K_CONTIG) { kk = idx % SG_BK; mm = idx / SG_BK; } else { mm = idx % SG_BM; kk = idx / SG_BM; }
+      const int m = m0 + mm, k = k0 + kk;
+      As[kk][mm] = (m < M && k < k_end) ? la(m, k) : 0.f;
+    }
+#pragma unroll
+    for (int i = 0; i < SG_BN * SG_BK / SG_THREADS; ++i) {
+      const int idx = tid + i * SG_THREADS;
+      int kk, nn;
+      if (LB::K_CONTIG) { kk = idx % SG_BK; nn = idx / SG_BK; } else { nn = idx % SG_BN; kk = idx / SG_BN; }
+      const int n = n0 + nn, k = k0 + kk;
+      Bs[kk][nn] = (n < N && k < k_end) ? lb(n, k) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < SG_BK; ++kk) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
+      if (m < M && n < N) ep(m, n, acc[i][j], split);
+    }
+}
+
+template <class LA, class LB, class EP>
+inline void gemm_simt(cudaStream_t st, uint64_t* launches, int M, int N, int K, int splits, LA la, LB lb, EP ep) {
+  if (M <= 0 || N <= 0 || K <= 0) return;
+  int kps = (K + splits - 1) / splits;
+  kps = (kps + SG_BK - 1) / SG_BK * SG_BK;
+  dim3 grid((M + SG_BM - 1) / SG_BM, (N + SG_BN - 1) / SG_BN, (K + kps - 1) / kps);
+  gemm_simt_kernel<<<grid, SG_THREADS, 0, st>>>(M, N, K, kps, la, lb, ep);
+  ++*launches;
+}
+// number of k-splits gemm_simt will really launch for a requested count
+inline int gemm_simt_splits(int K, int splits) {
+  int kps = (K + splits - 1) / splits;
+  kps = (kps + SG_BK - 1) / SG_BK * SG_BK;
+  return (K + kps - 1) / kps;
+}
+
+// ---- operand functors ----------------------------------------------------------------
+// x[row][k], rows ld apart
+template <class T> struct RowMajorOp {
+  static constexpr bool K_CONTIG = true;
+  const T* p; int ld;
+  __device__ __forceinline__ float operator()(int r, int k) const { return to_f(p[(size_t)r * ld + k]); }
+};
+// x[k][row]
+template <class T> struct ColMajorOp {
+  static constexpr bool K_CONTIG = false;
+  const T* p; int ld;
+  __device__ __forceinline__ float operator()(int r, int k) const { return to_f(p[(size_t)k * ld + r]); }
+};
+// x[k][row] with one extra row index == n_rows that reads as 1 (folds the bias gradient
+// into a weight-gradient contraction)
+template <class T> struct ColMajorOnesOp {
+  static constexpr bool K_CONTIG = false;
+  const T* p; int ld; int n_rows;
+  __device__ __forceinline__ float operator()(int r, int k) const {
+    return r < n_rows ? to_f(p[(size_t)k * ld + r]) : 1.f;
+  }
+};
+
+// convolution window: row m = (state, oh, ow), k = (r, s, ci)
+template <class G, class T> struct ConvWindowOp {
+  static constexpr bool K_CONTIG = true;
+  const T* x;
+  __device__ __forceinline__ float operator()(int m, int k) const {
+    const int b = m / (G::OH * G::OW), rem = m % (G::OH * G::OW), oh = rem / G::OW, ow = rem % G::OW;
+    const int r = k / (G::K * G::C), s = (k / G::C) % G::K, ci = k % G::C;
+    return to_f(x[((size_t)(b * G::H + oh * G::S + r) * G::W + (ow * G::S + s)) * G::C + ci]);
+  }
+};
+// the same window seen from the weight gradient: row j = (r, s, ci) or the ones row, k = (state, oh, ow)
+template <class G, class T> struct ConvWindowTOp {
+  static constexpr bool K_CONTIG = false;
+  const T* x;
+  __device__ __forceinline__ float operator()(int j, int m) const {
+    if (j >= G::KK) return 1.f;
+    const int b = m / (G::OH * G::OW), rem = m % (G::OH * G::OW), oh = rem / G::OW, ow = rem % G::OW;
+    const int r = j / (G::K * G::C), s = (j / G::C) % G::K, ci = j % G::C;
+    return to_f(x[((size_t)(b * G::H + oh * G::S + r) * G::W + (ow * G::S + s)) * G::C + ci]);
+  }
+};
+// data gradient: row m = (state, y, x) of the layer input, k = (r, s, co); zero where the
+// window (oh, ow) = ((y-r)/S, (x-s)/S) does not exist
+template <class G, class T> struct ConvDgradOp {
+  static constexpr bool K_CONTIG = true;
+  const T* g;
+  __device__ __forceinline__ float operator()(int m, int k) const {
+    const int b = m / (G::H * G::W), rem = m % (G::H * G::W), y = rem / G::W, x = rem % G::W;
+    const int r = k / (G::K * G::CO), s = (k / G::CO) % G::K, co = k % G::CO;
+    const int t = y - r, u = x - s;
+    if (t < 0 || u < 0 || t % G::S || u % G::S) return 0.f;
+    const int oh = t / G::S, ow = u / G::S;
+    if (oh >= G::OH || ow >= G::OW) return 0.f;
+    return to_f(g[((size_t)(b * G::OH + oh) * G::OW + ow) * G::CO + co]);
+  }
+};
+// weights seen from the data gradient: row ci, k = (r, s, co)
+template <class G, class T> struct ConvWeightTOp {
+  static constexpr bool K_CONTIG = true;
+  const T* w;
+  __device__ __forceinline__ float operator()(int ci, int k) const {
+    const int r = k / (G::K * G::CO), s = (k / G::CO) % G::K, co = k % G::CO;
+    return to_f(w[((size_t)(co * G::K + r) * G::K + s) * G::C + ci]);
+  }
+};
+
+// ---- epilogues ------------------------------------------------------------------------
+// out[m][n] = relu(acc * scale + bias[n])
+template <class T> struct BiasReluEp {
+  T* out; const float* bias; int ld; float scale;
+  __device__ __forceinline__ void operator()(int m, int n, float acc, int) const {
+    const float z = fmaf(acc, scale, bias[n]);
+    out[(size_t)m * ld + n] = from_f<T>(fmaxf(z, 0.f));
+  }
+};
+// out[m][n] = act[m][n] > 0 ? acc : 0   (gradient through the ReLU of the layer below)
+template <class T> struct ReluMaskEp {
+  T* out; const T* act; int ld;
+  __device__ __forceinline__ void operator()(int m, int n, float acc, int) const {
+    const size_t i = (size_t)m * ld + n;
+    out[i] = to_f(act[i]) > 0.f ? from_f<T>(acc) : from_f<T>(0.f);
+  }
+};
+// split-k partial: part[split][m][n]
+struct PartialEp {
+  float* part; int M, N;
+  __device__ __forceinline__ void operator()(int m, int n, float acc, int split) const {
+    part[((size_t)split * M + m) * N + n] = acc;
+  }
+};
+
+// fixed-order sum of the split-k partials part[split][part_rows][cols+1] (last column = bias
+// gradient) for rows row0 .. row0+rows-1 into the canonical gradient vector
+static __global__ void wgrad_reduce_kernel(const float* part, int splits, int part_rows, int row0, int rows, int cols,
+                                           float scale, float* gw, float* gb) {
+  const size_t total = (size_t)rows * (cols + 1), stride = (size_t)part_rows * (cols + 1);
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const float* src = part + (size_t)row0 * (cols + 1) + i;
+    float s = 0.f;
+    for (int p = 0; p < splits; ++p) s += src[(size_t)p * stride];
+    const int r = (int)(i / (cols + 1)), c = (int)(i % (cols + 1));
+    if (c < cols) gw[(size_t)r * cols + c] = s * scale; else gb[r] = s;
+  }
+}
+
+}  // namespace paac

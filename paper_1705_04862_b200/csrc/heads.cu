@@ -1,0 +1,167 @@
+// Policy / value heads with softmax, entropy and Philox inverse-CDF sampling; the reverse
+// scan for n-step returns; the loss gradient at the heads.
+#include "kernels.h"
+
+namespace paac {
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// One warp per state.  Lane k ends up holding logit k (A <= 32).  If `actions` is given,
+// the warp also draws a_t: u from Philox counter (env, step_lo, step_hi, ACTION stream), then the
+// smallest k with u < p_0 + ... + p_k, the running sum taken serially in float in index order.
+template <class T, class TW>
+__global__ void __launch_bounds__(128)
+heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* __restrict__ bpi,
+             const TW* __restrict__ wv, const float* __restrict__ bv, int n, int F, int A,
+             float* __restrict__ logits, float* __restrict__ values, uint64_t seed, uint64_t step,
+             const int32_t* __restrict__ forced, int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
+             float* __restrict__ uniforms) {
+  const int lane = threadIdx.x & 31;
+  const int e = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (e >= n) return;
+  const T* x = h + (size_t)e * F;
+  float z = -INFINITY;
+  for (int k = 0; k < A; ++k) {
+    float acc = 0.f;
+    for (int i = lane; i < F; i += 32) acc = fmaf(to_f(wpi[(size_t)k * F + i]), to_f(x[i]), acc);
+    acc = warp_sum(acc) + bpi[k];
+    if (lane == k) z = acc;
+  }
+  float v = 0.f;
+  for (int i = lane; i < F; i += 32) v = fmaf(to_f(wv[i]), to_f(x[i]), v);
+  v = warp_sum(v) + bv[0];
+  if (lane < A) logits[(size_t)e * A + lane] = z;
+  if (lane == 0) values[e] = v;
+  if (actions == nullptr) return;
+
+  const float m = warp_max(z);
+  const float ex = lane < A ? expf(z - m) : 0.f;
+  const float lse = m + logf(warp_sum(ex));
+  const float p = lane < A ? expf(z - lse) : 0.f;
+  const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
+  float c = 0.f;
+  int a = A - 1;
+  bool found = false;
+  for (int k = 0; k < A; ++k) {
+    c += __shfl_sync(0xffffffffu, p, k);
+    if (!found && u < c) { a = k; found = true; }
+  }
+  if (lane == 0) {
+    sampled[e] = a;
+    if (forced != nullptr && forced[e] >= 0) a = forced[e];
+    actions[e] = a;
+    uniforms[e] = u;
+  }
+}
+
+void launch_heads(cudaStream_t st, uint64_t* launches, int prec, const NetDims& nd, const float* theta,
+                  const bf16* theta16, const void* h, int n, float* logits, float* values, uint64_t seed,
+                  uint64_t step, const int32_t* forced, int32_t* actions, int32_t* sampled, float* uniforms) {
+  const int blocks = (n + 3) / 4;
+  if (prec == PAAC_BF16)
+    heads_kernel<bf16, bf16><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, theta + nd.pi_b,
+                                                     theta16 + nd.v_w, theta + nd.v_b, n, nd.F, nd.A, logits, values,
+                                                     seed, step, forced, actions, sampled, uniforms);
+  else
+    heads_kernel<float, float><<<blocks, 128, 0, st>>>((const float*)h, theta + nd.pi_w, theta + nd.pi_b,
+                                                       theta + nd.v_w, theta + nd.v_b, n, nd.F, nd.A, logits, values,
+                                                       seed, step, forced, actions, sampled, uniforms);
+  ++*launches;
+}
+
+// One thread per environment walks its t_max transitions backwards:
+// R_t = r_t + gamma * (1 - terminal_t) * R_{t+1}, starting from the bootstrap value.
+__global__ void returns_kernel(int n_e, int t_max, float gamma, const int8_t* __restrict__ rewards,
+                               const uint8_t* __restrict__ terminals, const float* __restrict__ values,
+                               float* __restrict__ R, float* __restrict__ adv) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n_e) return;
+  float next = values[(size_t)t_max * n_e + e];
+  for (int t = t_max - 1; t >= 0; --t) {
+    const size_t i = (size_t)t * n_e + e;
+    const float keep = terminals[i] ? 0.f : 1.f;
+    next = __fadd_rn((float)rewards[i], __fmul_rn(__fmul_rn(gamma, keep), next));
+    R[i] = next;
+    adv[i] = __fsub_rn(next, values[i]);
+  }
+}
+
+void launch_returns(cudaStream_t st, uint64_t* launches, int n_e, int t_max, float gamma, const int8_t* rewards,
+                    const uint8_t* terminals, const float* values, float* R, float* adv) {
+  returns_kernel<<<(n_e + 127) / 128, 128, 0, st>>>(n_e, t_max, gamma, rewards, terminals, values, R, adv);
+  ++*launches;
+}
+
+// One warp per experience: d/dz and d/dV of
+//   (1/B) [ -adv log pi(a) - beta H + c_v (R - V)^2 ]
+// with adv and R constants; also the three per-sample loss terms for the statistics.
+__global__ void __launch_bounds__(128)
+head_grad_kernel(int B, int A, float beta, float value_coef, const float* __restrict__ logits,
+                 const float* __restrict__ values, const int32_t* __restrict__ actions, const float* __restrict__ R,
+                 const float* __restrict__ adv, float* __restrict__ dz, float* __restrict__ dV,
+                 float* __restrict__ loss_terms) {
+  const int lane = threadIdx.x & 31;
+  const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (i >= B) return;
+  const float z = lane < A ? logits[(size_t)i * A + lane] : -INFINITY;
+  const float m = warp_max(z);
+  const float ex = lane < A ? expf(z - m) : 0.f;
+  const float lse = m + logf(warp_sum(ex));
+  const float lp = z - lse;
+  const float p = lane < A ? expf(lp) : 0.f;
+  const float H = -warp_sum(lane < A ? p * lp : 0.f);
+  const int a = actions[i];
+  const float ad = adv[i], invB = 1.0f / (float)B;
+  if (lane < A) {
+    const float g = -ad * ((lane == a ? 1.f : 0.f) - p) + beta * p * (lp + H);
+    dz[(size_t)i * A + lane] = g * invB;
+  }
+  const float lp_a = __shfl_sync(0xffffffffu, lp, a);
+  if (lane == 0) {
+    const float d = values[i] - R[i];
+    dV[i] = 2.f * value_coef * d * invB;
+    loss_terms[i] = -ad * lp_a;
+    loss_terms[(size_t)B + i] = value_coef * d * d;
+    loss_terms[2 * (size_t)B + i] = H;
+  }
+}
+
+// single block: fixed-order (hence reproducible) means of the three loss terms
+__global__ void __launch_bounds__(256) loss_stats_kernel(int B, const float* __restrict__ loss_terms, DeviceStats* stats) {
+  __shared__ float sh[3][256];
+  float acc[3] = {0.f, 0.f, 0.f};
+  for (int i = threadIdx.x; i < B; i += 256)
+    for (int j = 0; j < 3; ++j) acc[j] += loss_terms[(size_t)j * B + i];
+  for (int j = 0; j < 3; ++j) sh[j][threadIdx.x] = acc[j];
+  __syncthreads();
+  for (int s = 128; s > 0; s >>= 1) {
+    if (threadIdx.x < s)
+      for (int j = 0; j < 3; ++j) sh[j][threadIdx.x] += sh[j][threadIdx.x + s];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    stats->policy_loss = sh[0][0] / B;
+    stats->value_loss = sh[1][0] / B;
+    stats->entropy = sh[2][0] / B;
+  }
+}
+
+void launch_head_grad(cudaStream_t st, uint64_t* launches, int B, int A, float beta, float value_coef,
+                      const float* logits, const float* values, const int32_t* actions, const float* R,
+                      const float* adv, float* dz, float* dV, float* loss_terms, DeviceStats* stats) {
+  head_grad_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, A, beta, value_coef, logits, values, actions, R, adv, dz, dV,
+                                                loss_terms);
+  loss_stats_kernel<<<1, 256, 0, st>>>(B, loss_terms, stats);
+  *launches += 2;
+}
+
+}  // namespace paac

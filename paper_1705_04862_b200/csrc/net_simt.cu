@@ -1,0 +1,174 @@
+// The network's layers as contractions on the CUDA cores (float accumulate):
+// forward with fused bias + ReLU, data gradients with the ReLU mask of the layer
+// below fused, weight gradients as split-k partial sums reduced in a fixed order.
+#include "gemm_simt.cuh"
+#include "kernels.h"
+
+namespace paac {
+
+static int pick_splits(int M, int N, int K) {
+  const int blocks = ((M + SG_BM - 1) / SG_BM) * ((N + SG_BN - 1) / SG_BN);
+  int s = (592 + blocks - 1) / blocks;
+  const int by_k = (K + 127) / 128;
+  if (s > by_k) s = by_k;
+  if (s > 512) s = 512;
+  if (s < 1) s = 1;
+  return gemm_simt_splits(K, s);
+}
+
+static void reduce_wgrad(cudaStream_t st, uint64_t* launches, const float* part, int splits, int part_rows, int row0,
+                         int rows, int cols, float scale, float* gw, float* gb) {
+  const size_t total = (size_t)rows * (cols + 1);
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > 2368) blocks = 2368;
+  wgrad_reduce_kernel<<<blocks, 256, 0, st>>>(part, splits, part_rows, row0, rows, cols, scale, gw, gb);
+  ++*launches;
+}
+
+template <class G, class TIn, class T, class TW>
+static void conv_fwd(cudaStream_t st, uint64_t* launches, const TIn* x, const TW* w, const float* bias, T* out, int n,
+                     float scale) {
+  gemm_simt(st, launches, n * G::OH * G::OW, G::CO, G::KK, 1, ConvWindowOp<G, TIn>{x}, RowMajorOp<TW>{w, G::KK},
+            BiasReluEp<T>{out, bias, G::CO, scale});
+}
+template <class T, class TW>
+static void fc_fwd(cudaStream_t st, uint64_t* launches, const T* x, const TW* w, const float* bias, T* out, int n,
+                   int IN, int F) {
+  gemm_simt(st, launches, n, F, IN, 1, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, BiasReluEp<T>{out, bias, F, 1.f});
+}
+template <class G, class T, class TW>
+static void conv_dgrad(cudaStream_t st, uint64_t* launches, const T* g, const TW* w, const T* act_in, T* gin, int n) {
+  gemm_simt(st, launches, n * G::H * G::W, G::C, G::K * G::K * G::CO, 1, ConvDgradOp<G, T>{g}, ConvWeightTOp<G, TW>{w},
+            ReluMaskEp<T>{gin, act_in, G::C});
+}
+template <class G, class TIn, class T>
+static void conv_wgrad(cudaStream_t st, uint64_t* launches, const T* g, const TIn* x, int n, float scale, float* gw,
+                       float* gb, float* scratch) {
+  const int M = G::CO, N = G::KK + 1, K = n * G::OH * G::OW;
+  const int splits = pick_splits(M, N, K);
+  gemm_simt(st, launches, M, N, K, splits, ColMajorOp<T>{g, G::CO}, ConvWindowTOp<G, TIn>{x}, PartialEp{scratch, M, N});
+  reduce_wgrad(st, launches, scratch, splits, M, 0, M, G::KK, scale, gw, gb);
+}
+template <class T, class TW>
+static void fc_dgrad(cudaStream_t st, uint64_t* launches, const T* g, const TW* w, const T* act_in, T* gin, int n,
+                     int IN, int F) {
+  gemm_simt(st, launches, n, IN, F, 1, RowMajorOp<T>{g, F}, ColMajorOp<TW>{w, IN}, ReluMaskEp<T>{gin, act_in, IN});
+}
+template <class T>
+static void fc_wgrad(cudaStream_t st, uint64_t* launches, const T* g, const T* x, int n, int IN, int F, float* gw,
+                     float* gb, float* scratch) {
+  const int M = F, N = IN + 1, K = n;
+  const int splits = pick_splits(M, N, K);
+  gemm_simt(st, launches, M, N, K, splits, ColMajorOp<T>{g, F}, ColMajorOnesOp<T>{x, IN, IN}, PartialEp{scratch, M, N});
+  reduce_wgrad(st, launches, scratch, splits, M, 0, M, IN, 1.f, gw, gb);
+}
+
+template <class T, class TW>
+static void forward_t(cudaStream_t st, uint64_t* L, int arch, const NetDims& nd, const float* theta, const TW* w,
+                      const uint8_t* frames, int n, void* const act[]) {
+  const LayerDims* d = nd.layer;
+  const float s255 = 1.0f / 255.0f;
+  if (arch == PAAC_ARCH_NIPS) {
+    conv_fwd<NipsConv1, uint8_t, T, TW>(st, L, frames, w + d[0].w_off, theta + d[0].b_off, (T*)act[0], n, s255);
+    conv_fwd<NipsConv2, T, T, TW>(st, L, (const T*)act[0], w + d[1].w_off, theta + d[1].b_off, (T*)act[1], n, 1.f);
+    fc_fwd<T, TW>(st, L, (const T*)act[1], w + d[2].w_off, theta + d[2].b_off, (T*)act[2], n, 2592, 256);
+  } else {
+    conv_fwd<NatConv1, uint8_t, T, TW>(st, L, frames, w + d[0].w_off, theta + d[0].b_off, (T*)act[0], n, s255);
+    conv_fwd<NatConv2, T, T, TW>(st, L, (const T*)act[0], w + d[1].w_off, theta + d[1].b_off, (T*)act[1], n, 1.f);
+    conv_fwd<NatConv3, T, T, TW>(st, L, (const T*)act[1], w + d[2].w_off, theta + d[2].b_off, (T*)act[2], n, 1.f);
+    fc_fwd<T, TW>(st, L, (const T*)act[2], w + d[3].w_off, theta + d[3].b_off, (T*)act[3], n, 3136, 512);
+  }
+}
+
+template <class T, class TW>
+static void backward_t(cudaStream_t st, uint64_t* L, int arch, const NetDims& nd, const TW* w, const uint8_t* frames,
+                       int n, void* const act[], void* const gact[], float* grad, float* scratch) {
+  const LayerDims* d = nd.layer;
+  const float s255 = 1.0f / 255.0f;
+  if (arch == PAAC_ARCH_NIPS) {
+    fc_wgrad<T>(st, L, (const T*)gact[2], (const T*)act[1], n, 2592, 256, grad + d[2].w_off, grad + d[2].b_off, scratch);
+    fc_dgrad<T, TW>(st, L, (const T*)gact[2], w + d[2].w_off, (const T*)act[1], (T*)gact[1], n, 2592, 256);
+    conv_wgrad<NipsConv2, T, T>(st, L, (const T*)gact[1], (const T*)act[0], n, 1.f, grad + d[1].w_off, grad + d[1].b_off, scratch);
+    conv_dgrad<NipsConv2, T, TW>(st, L, (const T*)gact[1], w + d[1].w_off, (const T*)act[0], (T*)gact[0], n);
+    conv_wgrad<NipsConv1, uint8_t, T>(st, L, (const T*)gact[0], frames, n, s255, grad + d[0].w_off, grad + d[0].b_off, scratch);
+  } else {
+    fc_wgrad<T>(st, L, (const T*)gact[3], (const T*)act[2], n, 3136, 512, grad + d[3].w_off, grad + d[3].b_off, scratch);
+    fc_dgrad<T, TW>(st, L, (const T*)gact[3], w + d[3].w_off, (const T*)act[2], (T*)gact[2], n, 3136, 512);
+    conv_wgrad<NatConv3, T, T>(st, L, (const T*)gact[2], (const T*)act[1], n, 1.f, grad + d[2].w_off, grad + d[2].b_off, scratch);
+    conv_dgrad<NatConv3, T, TW>(st, L, (const T*)gact[2], w + d[2].w_off, (const T*)act[1], (T*)gact[1], n);
+    conv_wgrad<NatConv2, T, T>(st, L, (const T*)gact[1], (const T*)act[0], n, 1.f, grad + d[1].w_off, grad + d[1].b_off, scratch);
+    conv_dgrad<NatConv2, T, TW>(st, L, (const T*)gact[1], w + d[1].w_off, (const T*)act[0], (T*)gact[0], n);
+    conv_wgrad<NatConv1, uint8_t, T>(st, L, (const T*)gact[0], frames, n, s255, grad + d[0].w_off, grad + d[0].b_off, scratch);
+  }
+}
+
+void simt_forward(cudaStream_t st, uint64_t* launches, int arch, int prec, const NetDims& nd, const float* theta,
+                  const bf16* theta16, const uint8_t* frames, int n, void* const act[]) {
+  if (prec == PAAC_BF16) forward_t<bf16, bf16>(st, launches, arch, nd, theta, theta16, frames, n, act);
+  else forward_t<float, float>(st, launches, arch, nd, theta, theta, frames, n, act);
+}
+
+void simt_backward(cudaStream_t st, uint64_t* launches, int arch, int prec, const NetDims& nd, const float* theta,
+                   const bf16* theta16, const uint8_t* frames, int n, void* const act[], void* const gact[],
+                   float* grad, float* scratch) {
+  if (prec == PAAC_BF16) backward_t<bf16, bf16>(st, launches, arch, nd, theta16, frames, n, act, gact, grad, scratch);
+  else backward_t<float, float>(st, launches, arch, nd, theta, frames, n, act, gact, grad, scratch);
+}
+
+size_t simt_scratch_floats(int arch, const NetDims& nd, int n) {
+  size_t best = 0;
+  for (int l = 0; l <= nd.n_conv; ++l) {
+    const LayerDims& d = nd.layer[l];
+    const int M = d.CO;
+    const int N = (l < nd.n_conv ? d.K * d.K * d.C : d.H * d.W * d.C) + 1;
+    const int K = n * d.OH * d.OW;
+    const size_t need = (size_t)pick_splits(M, N, K) * M * N;
+    if (need > best) best = need;
+  }
+  const size_t heads = (size_t)pick_splits(nd.A + 1, nd.F + 1, n) * (nd.A + 1) * (nd.F + 1);
+  (void)arch;
+  return best > heads ? best : heads;
+}
+
+// ---- heads backward (tiny contractions over the A+1 head units) ------------------------------
+struct HeadGradOp {          // row = sample, k = head unit (policy logits then value)
+  static constexpr bool K_CONTIG = true;
+  const float* dz; const float* dV; int A;
+  __device__ __forceinline__ float operator()(int m, int k) const { return k < A ? dz[(size_t)m * A + k] : dV[m]; }
+};
+struct HeadGradTOp {         // row = head unit, k = sample
+  static constexpr bool K_CONTIG = false;
+  const float* dz; const float* dV; int A;
+  __device__ __forceinline__ float operator()(int u, int b) const { return u < A ? dz[(size_t)b * A + u] : dV[b]; }
+};
+template <class TW> struct HeadWeightOp {   // row = fc unit i, k = head unit
+  static constexpr bool K_CONTIG = false;
+  const TW* wpi; const TW* wv; int F, A;
+  __device__ __forceinline__ float operator()(int i, int k) const {
+    return k < A ? to_f(wpi[(size_t)k * F + i]) : to_f(wv[i]);
+  }
+};
+
+template <class T, class TW>
+static void heads_backward_t(cudaStream_t st, uint64_t* L, const NetDims& nd, const TW* w, const T* h, int n,
+                             const float* dz, const float* dV, T* gact_fc, float* grad, float* scratch) {
+  const int A = nd.A, F = nd.F;
+  gemm_simt(st, L, n, F, A + 1, 1, HeadGradOp{dz, dV, A}, HeadWeightOp<TW>{w + nd.pi_w, w + nd.v_w, F, A},
+            ReluMaskEp<T>{gact_fc, h, F});
+  const int splits = pick_splits(A + 1, F + 1, n);
+  gemm_simt(st, L, A + 1, F + 1, n, splits, HeadGradTOp{dz, dV, A}, ColMajorOnesOp<T>{h, F, F},
+            PartialEp{scratch, A + 1, F + 1});
+  reduce_wgrad(st, L, scratch, splits, A + 1, 0, A, F, 1.f, grad + nd.pi_w, grad + nd.pi_b);
+  reduce_wgrad(st, L, scratch, splits, A + 1, A, 1, F, 1.f, grad + nd.v_w, grad + nd.v_b);
+}
+
+void heads_backward(cudaStream_t st, uint64_t* launches, int prec, const NetDims& nd, const float* theta,
+                    const bf16* theta16, const void* h, int n, const float* dz, const float* dV, void* gact_fc,
+                    float* grad, float* scratch) {
+  if (prec == PAAC_BF16)
+    heads_backward_t<bf16, bf16>(st, launches, nd, theta16, (const bf16*)h, n, dz, dV, (bf16*)gact_fc, grad, scratch);
+  else
+    heads_backward_t<float, float>(st, launches, nd, theta, (const float*)h, n, dz, dV, (float*)gact_fc, grad, scratch);
+}
+
+}  // namespace paac

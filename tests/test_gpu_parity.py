@@ -1,0 +1,192 @@
+"""Parity of the CUDA library with the CPU oracle, element by element, through the C-ABI."""
+import numpy as np
+import pytest
+
+from paper_1705_04862_b200 import binding as pb
+from paper_1705_04862_b200.configs import CONFIGS
+
+from parity_util import TOL, TOL_PARAMS_10, check_rollout, check_update, make_pair, rel
+
+pytestmark = pytest.mark.gpu
+
+
+def test_init_is_bit_exact(orc):
+    for cfg in (CONFIGS[0], CONFIGS[2]):
+        o, g = make_pair(orc, cfg)
+        assert np.array_equal(g.params(), o.theta)
+        g.close()
+    o, g = make_pair(orc, CONFIGS[0], seed=(5 << 32) | 9)
+    assert np.array_equal(g.params(), o.theta)
+    g.close()
+
+
+def test_config1_nips_fp32_three_updates(orc):
+    cfg = CONFIGS[0]
+    o, g = make_pair(orc, cfg)
+    for it in range(cfg["updates"]):
+        ro, r1 = check_rollout(orc, o, g, TOL["fp32"])
+        up, st, r2 = check_update(orc, o, g, TOL["fp32"])
+        assert r1["action_mismatches"] == 0
+        assert r2["theta"] <= TOL_PARAMS_10
+    g.close()
+
+
+def test_config2_nips_fp32_params_after_10_updates(orc):
+    cfg = CONFIGS[1]
+    o, g = make_pair(orc, cfg)
+    mism = 0
+    for it in range(10):
+        ro, r1 = check_rollout(orc, o, g, TOL["fp32"])
+        up, st, r2 = check_update(orc, o, g, TOL["fp32"], check_acts=(it < 2))
+        mism += r1["action_mismatches"]
+    assert rel(g.params(), o.theta) <= TOL_PARAMS_10
+    assert rel(g.debug_read(pb.DBG_RMS), o.m) <= TOL_PARAMS_10
+    assert mism <= 1
+    g.close()
+
+
+def test_config2_free_running_actions_agree(orc):
+    """Without forcing: both sides sample for themselves; with float parameters the draws agree."""
+    cfg = CONFIGS[1]
+    o, g = make_pair(orc, cfg)
+    for it in range(3):
+        ro, r1 = check_rollout(orc, o, g, TOL["fp32"], lockstep=False)
+        check_update(orc, o, g, TOL["fp32"], check_acts=False)
+    g.close()
+
+
+def test_config3_nature_bf16_lockstep(orc):
+    cfg = CONFIGS[2]
+    o, g = make_pair(orc, cfg)
+    th0 = o.theta.copy()
+    for it in range(10):
+        ro, r1 = check_rollout(orc, o, g, TOL["bf16"])
+        up, st, r2 = check_update(orc, o, g, TOL["bf16"], check_acts=(it < 2))
+    assert rel(g.params(), o.theta) <= TOL_PARAMS_10
+    assert rel(g.params() - th0, o.theta - th0) <= TOL["bf16"]
+    g.close()
+
+
+def test_config4_nature_bf16_terminals(orc):
+    cfg = CONFIGS[3]
+    o, g = make_pair(orc, cfg)
+    terms = 0
+    for it in range(2):
+        ro, r1 = check_rollout(orc, o, g, TOL["bf16"])
+        terms += int(ro["terminals"].sum())
+        check_update(orc, o, g, TOL["bf16"], check_acts=(it == 0))
+    assert terms > 0          # return resets were exercised
+    g.close()
+
+
+def test_ragged_sizes_and_action_counts(orc):
+    """n_e that is no multiple of any tile, every action-set size of the configs."""
+    for arch, prec, n_e, t_max, A in (("nips", "fp32", 5, 3, 18), ("nips", "bf16", 3, 2, 4),
+                                      ("nature", "fp32", 7, 2, 6), ("nature", "bf16", 13, 1, 2),
+                                      ("nips", "fp32", 1, 1, 32)):
+        cfg = dict(arch=arch, precision=prec, n_e=n_e, t_max=t_max, n_actions=A, lr=0.01, term_denom=3)
+        o, g = make_pair(orc, cfg, seed=77)
+        for it in range(2):
+            check_rollout(orc, o, g, TOL[prec])
+            check_update(orc, o, g, TOL[prec])
+        g.close()
+
+
+def test_resync_after_many_updates(orc):
+    """Free-run the library for 60 updates (config 2), copy its parameters and RMSProp state into
+    the oracle and compare one more iteration from there."""
+    cfg = CONFIGS[1]
+    o, g = make_pair(orc, cfg)
+    for it in range(60):
+        g.rollout()
+        st = g.update()
+        assert st["status"] == 0 and np.isfinite(st["grad_norm"])
+    o.theta = g.params()
+    o.m = g.debug_read(pb.DBG_RMS).copy()
+    o.N = 60 * cfg["n_e"] * cfg["t_max"]
+    o.state = g.debug_read(pb.DBG_NEXT_FRAMES).reshape(cfg["n_e"], 84, 84, 4).copy()
+    for j, c in enumerate(g.debug_read(pb.DBG_COUNTERS).reshape(3, -1)):
+        o.counters[j][:] = c
+    check_rollout(orc, o, g, TOL["fp32"])
+    check_update(orc, o, g, TOL["fp32"], check_acts=False)
+    g.close()
+
+
+def test_determinism_bitwise(orc):
+    cfg = CONFIGS[2]
+    outs = []
+    for rep in range(2):
+        _, g = make_pair(orc, cfg)
+        for it in range(3):
+            g.rollout()
+            g.update()
+        outs.append((g.params(), g.debug_read(pb.DBG_GRAD).copy()))
+        g.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+def test_error_paths(orc):
+    import ctypes as C
+    L = pb.lib()
+    hp = pb.default_hparams()
+    h = C.c_void_p()
+    assert L.paac_init(C.byref(h), 7, 4, 5, 4, C.byref(hp), 1) == pb.ERR_ARG
+    assert L.paac_init(C.byref(h), 0, 0, 5, 4, C.byref(hp), 1) == pb.ERR_ARG
+    assert L.paac_init(C.byref(h), 0, 4, 5, 1, C.byref(hp), 1) == pb.ERR_ARG
+    assert L.paac_init(None, 0, 4, 5, 4, C.byref(hp), 1) == pb.ERR_ARG
+    assert L.paac_rollout(None, None) == pb.ERR_ARG
+    import torch
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    hp2 = pb.default_hparams(workspace=small.data_ptr(), workspace_bytes=1024)
+    assert L.paac_init(C.byref(h), 0, 4, 5, 4, C.byref(hp2), 1) == pb.ERR_WORKSPACE
+    g = pb.Paac("nips", 4, 2, 4, 3)
+    assert L.paac_update(g._h, None) == pb.ERR_STATE          # no rollout yet
+    buf = np.zeros(3, np.float32)
+    assert L.paac_params(g._h, buf.ctypes.data, 3) == pb.ERR_ARG
+    bad = np.full(g.B, 9, np.int32)
+    assert L.paac_force_actions(g._h, bad.ctypes.data) == pb.ERR_ARG
+    # a NaN parameter makes the gradient norm non-finite: the update is skipped and says so
+    th = g.params()
+    th_bad = th.copy()
+    th_bad[10] = np.nan
+    g.set_params(th_bad)
+    g.rollout()
+    rms0 = g.debug_read(pb.DBG_RMS).copy()
+    st = g.update()
+    assert st["status"] == pb.ERR_NONFINITE
+    assert np.array_equal(g.debug_read(pb.DBG_RMS), rms0)
+    after = g.params()
+    assert np.array_equal(after[np.isfinite(th_bad)], th_bad[np.isfinite(th_bad)])
+    g.set_params(th)
+    g.rollout()
+    assert g.update()["status"] == 0
+    g.close()
+
+
+def test_external_environment_mode_matches_device_environment(orc):
+    """Frames, rewards and terminals fed from the host (the oracle's environment) give the same
+    actions, values and update as the on-device environment."""
+    cfg = CONFIGS[0]
+    o, g = make_pair(orc, cfg)
+    _, g2 = make_pair(orc, cfg)
+    n_e, T = cfg["n_e"], cfg["t_max"]
+    g.rollout()
+    g.update()
+    # replay the same iteration on g2 through the host entry points
+    frames = g.debug_read(pb.DBG_FRAMES).reshape(T, n_e, 84, 84, 4)
+    nxt = g.debug_read(pb.DBG_NEXT_FRAMES).reshape(n_e, 84, 84, 4)
+    rewards = g.debug_read(pb.DBG_REWARDS).reshape(T, n_e)
+    terms = g.debug_read(pb.DBG_TERMINALS).reshape(T, n_e)
+    acts_dev = g.debug_read(pb.DBG_ACTIONS).reshape(T, n_e)
+    for t in range(T):
+        a = np.zeros(n_e, np.int32)
+        v = np.zeros(n_e, np.float32)
+        g2.act_host(t, np.ascontiguousarray(frames[t]), a, v)
+        assert np.array_equal(a, acts_dev[t])
+        g2.observe_host(t, np.ascontiguousarray(rewards[t]), np.ascontiguousarray(terms[t]))
+    vb = np.zeros(n_e, np.float32)
+    g2.act_host(T, np.ascontiguousarray(nxt), None, vb)
+    g2.update()
+    assert np.array_equal(g2.params(), g.params())
+    g.close()
+    g2.close()
