@@ -201,6 +201,16 @@ class Paac:
         arr = np.ascontiguousarray(arr)
         _check(lib().paac_debug_write(self._h, which, arr.ctypes.data, arr.nbytes))
 
+    def debug_write_act(self, layer, arr):
+        """Overwrite stored activation `layer` from float32 values (which, with bf16 storage, must
+        already be bf16-representable)."""
+        arr = np.ascontiguousarray(arr, np.float32)
+        if self.precision == BF16:
+            bits = arr.view(np.uint32)
+            assert not np.any(bits & 0xFFFF), "not bf16 values"
+            arr = (bits >> 16).astype(np.uint16)
+        self.debug_write(DBG_ACT0 + layer, arr)
+
     def launch_count(self):
         return int(lib().paac_launch_count(self._h))
 

@@ -43,6 +43,15 @@ def layer_slices(orc, net):
     return out
 
 
+def resync(o, g):
+    """Give the library the oracle's parameters and RMSProp state.  With bf16 storage two correct
+    implementations drift apart within a few updates (a parameter difference far below one bf16
+    unit still flips the rounding of many weights and activations, and the differences grow about
+    tenfold per update), so the bf16 cases compare one iteration at a time from a common start."""
+    g.set_params(o.theta)
+    g.debug_write(pb.DBG_RMS, o.m)
+
+
 def check_rollout(orc, o, g, tol, lockstep=True):
     """Oracle rolls out with its own sampling; the library is forced onto the oracle's actions so
     that a tolerated near-boundary difference cannot cascade, and its own draw is compared."""
@@ -78,31 +87,74 @@ def check_rollout(orc, o, g, tol, lockstep=True):
     return ro, rep
 
 
-def check_update(orc, o, g, tol, check_acts=True):
+FLIP_L2 = 5e-2
+
+
+def check_update(orc, o, g, tol, check_acts=True, inject=False):
+    """One update on both sides, compared tensor by tensor (max norm relative to the tensor's
+    largest magnitude, `rel`).
+
+    inject=True: the oracle's stored activations, logits and values are first written into the
+    library, so both backward passes start from identical tensors and ReLU masks; every tensor
+    must then meet the tolerance.
+
+    inject=False: the library updates from its own rollout.  A unit whose pre-activation is within
+    rounding of zero can be switched on on one side and off on the other; both are valid, but such
+    a flip moves gradient elements below it by a whole term of their sums.  If no unit flipped,
+    every tensor must meet the tolerance; if some did (they must be rare and sit at numerically
+    zero activation), the activation gradients are compared where the masks agree and the
+    parameter gradients in the L2 sense against FLIP_L2, and the caller should re-synchronise.
+    Returns (oracle update, library stats, report); report["flips"] counts flipped units."""
     L = o.net.n_conv
-    B = o.n_e * o.t_max
     up = o.update()
-    st = g.update()
-    rep = {}
-    assert st["status"] == 0 and st["timesteps"] == o.N
-    rep["R"] = rel(g.debug_read(pb.DBG_RETURNS), up["R"])
-    rep["adv"] = rel(g.debug_read(pb.DBG_ADVANTAGES), up["adv"])
-    rep["dz"] = rel(g.debug_read(pb.DBG_DLOGITS), up["dz"])
-    rep["dV"] = rel(g.debug_read(pb.DBG_DVALUES), up["dV"])
-    if check_acts:
+    if inject:
         for l in range(L + 1):
-            rep["act%d" % l] = rel(g.debug_read(pb.DBG_ACT0 + l), up["acts"][l])
-            rep["gact%d" % l] = rel(g.debug_read(pb.DBG_GACT0 + l), up["gacts"][l])
+            g.debug_write_act(l, up["acts"][l])
+        g.debug_write(pb.DBG_LOGITS, up["logits"])
+        g.debug_write(pb.DBG_VALUES, o.ro["values"])
+    st = g.update()
+    rep, loose = {}, {}
+    assert st["status"] == 0 and st["timesteps"] == o.N
+    for k, w in (("R", pb.DBG_RETURNS), ("adv", pb.DBG_ADVANTAGES), ("dz", pb.DBG_DLOGITS), ("dV", pb.DBG_DVALUES)):
+        rep[k] = rel(g.debug_read(w), up[k])
+    acts_g = [g.debug_read(pb.DBG_ACT0 + l) for l in range(L + 1)]
+    acts_o = [up["acts"][l].reshape(-1) for l in range(L + 1)]
+    agree = [(a > 0) == (b > 0) for a, b in zip(acts_g, acts_o)]
+    flips = int(sum((~m).sum() for m in agree))
+    rep["flips"] = 0.0
+    for l in range(L + 1):
+        rep["act%d" % l] = rel(acts_g[l], acts_o[l])
+        if inject:
+            assert np.array_equal(acts_g[l], acts_o[l])
+        bad = ~agree[l]
+        assert bad.mean() <= 5e-3, (l, bad.mean())
+        if bad.any():
+            assert max(acts_g[l][bad].max(), acts_o[l][bad].max()) <= tol * np.abs(acts_o[l]).max(), l
+        if check_acts or flips:
+            ga_g, ga_o = g.debug_read(pb.DBG_GACT0 + l), up["gacts"][l].reshape(-1)
+            if flips == 0:
+                rep["gact%d" % l] = rel(ga_g, ga_o)
+            else:
+                d = (ga_g.astype(np.float64) - ga_o)[agree[l]]
+                loose["gact%d" % l] = float(np.linalg.norm(d) / (np.linalg.norm(ga_o[agree[l]]) + 1e-30))
     grad = g.debug_read(pb.DBG_GRAD)
-    for name, sl in layer_slices(orc, o.net):
-        rep["g." + name] = rel(grad[sl], up["grad"][sl])
-    rep["grad"] = rel(grad, up["grad"])
+    for name, sl in layer_slices(orc, o.net) + [("all", slice(None))]:
+        gg, go = grad[sl].astype(np.float64), up["grad"][sl].astype(np.float64)
+        if flips == 0:
+            rep["g." + name] = rel(gg, go)
+        else:
+            loose["g." + name] = float(np.linalg.norm(gg - go) / (np.linalg.norm(go) + 1e-30))
     for k, v in rep.items():
-        assert v <= tol, (k, v, rep)
+        assert v <= tol, (k, v, rep, loose)
+    for k, v in loose.items():
+        assert v <= FLIP_L2, (k, v, rep, loose)
+    stat_tol = tol if flips == 0 else FLIP_L2
     for k in ("policy_loss", "value_loss", "entropy"):
         assert abs(st[k] - up[k]) <= tol * max(1.0, abs(up[k])), (k, st[k], up[k])
-    assert abs(st["grad_norm"] - up["grad_norm"]) <= tol * up["grad_norm"]
-    assert abs(st["clip_scale"] - up["clip_scale"]) <= tol
+    assert abs(st["grad_norm"] - up["grad_norm"]) <= stat_tol * up["grad_norm"]
+    assert abs(st["clip_scale"] - up["clip_scale"]) <= stat_tol
+    rep.update(loose)
+    rep["flips"] = flips
     rep["theta"] = rel(g.params(), o.theta)
     rep["rms"] = rel(g.debug_read(pb.DBG_RMS), o.m)
     return up, st, rep
