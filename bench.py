@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Throughput of one PAAC iteration (rollout of t_max steps for n_e environments + one update)
+on B200, reported as environment steps per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl ours|reference]
+
+One "step" is one whole iteration of Algorithm 1 on the synthetic hashed environment.  The line
+printed by rank 0 carries the device-timed value, an end-to-end figure through the
+external-environment entry points (host frames in, actions out), a per-kernel CUDA-event breakdown
+with a roofline entry for the kernel that takes the most time, and the CPU oracle timed on a
+bounded sample of the same workload.  With --gpus N > 1 every rank runs an independent replica
+(the path is single-GPU: environments are not sharded and nothing is exchanged).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1705_04862_b200.configs import COMMON, CONFIGS  # noqa: E402
+
+FRAME_BYTES = 84 * 84 * 4
+
+
+# ----------------------------------------------------------------------------- workload arithmetic
+def net_layers(arch):
+    """(name, rows per state, N, K) of each forward contraction."""
+    if arch == "nips":
+        return [("conv1", 400, 16, 256), ("conv2", 81, 32, 256), ("fc", 1, 256, 2592)], 256
+    return [("conv1", 400, 32, 256), ("conv2", 81, 64, 512), ("conv3", 49, 64, 576), ("fc", 1, 512, 3136)], 512
+
+
+def kernel_work(cfg):
+    """Algorithmic FLOPs (2 x MAC, unpadded) or bytes of ONE launch of each kernel family, and the
+    roofline that bounds it.  n = n_e for rollout kernels, B = n_e * t_max for update kernels."""
+    layers, F = net_layers(cfg["arch"])
+    n_e, T, A = cfg["n_e"], cfg["t_max"], cfg["n_actions"]
+    B = n_e * T
+    elt = 2 if cfg["precision"] == "bf16" else 4
+    P = sum(N * K + N for _, _, N, K in layers) + (A + 1) * (F + 1)
+    w = {}
+    for name, rows, N, K in layers:
+        mac = rows * N * K
+        w[name + "_fwd"] = ("tensor", 2.0 * mac * n_e)
+        w[name + "_wgrad"] = ("tensor", 2.0 * mac * B)
+        if name != "conv1":
+            w[name + "_dgrad"] = ("tensor", 2.0 * mac * B)
+    w["heads_fwd_sample"] = ("tensor", 2.0 * (A + 1) * F * n_e)
+    w["heads_bwd"] = ("tensor", 2.0 * (A + 1) * F * B)          # per launch (dgrad or wgrad)
+    w["env_step"] = ("hbm", n_e * (FRAME_BYTES + 6.0))
+    w["clip_rmsprop"] = ("hbm", P * (22.0 if elt == 2 else 20.0))
+    w["grad_sumsq"] = ("hbm", P * 4.0)
+    return w, P
+
+
+def iteration_flops(cfg):
+    layers, F = net_layers(cfg["arch"])
+    A = cfg["n_actions"]
+    fwd = sum(2.0 * r * N * K for _, r, N, K in layers) + 2.0 * (A + 1) * F
+    bwd = 2.0 * fwd - 2.0 * layers[0][1] * layers[0][2] * layers[0][3]      # no data gradient for conv1
+    n_e, T = cfg["n_e"], cfg["t_max"]
+    return fwd * n_e * (T + 1), bwd * n_e * T
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d.get("bf16_tflops_sustained"),
+                    src="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, src="fallback")
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc = [], None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for ts, r in self.rows if t0 - 0.05 <= ts <= t1 + 0.15 and len(r) >= 7] or \
+               [r for _, r in self.rows if len(r) >= 7]
+        sm = sorted(float(r[0]) for r in rows if r[0].replace(".", "").isdigit())
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for j, n in enumerate(names) if any(r[3 + j].lower().startswith("active") for r in rows)]
+        mx = [float(r[1]) for r in rows if r[1].replace(".", "").isdigit()]
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx[0] if mx else None,
+                "reasons": reasons, "samples": len(rows)}
+
+
+# ----------------------------------------------------------------------------- oracle legs
+def oracle_time(cfg, n_e_sample, iters, warm=0):
+    """Seconds per iteration of the CPU oracle on the first n_e_sample environments of cfg."""
+    from oracle import oracle as orc
+    orc.build()
+    hp = dict(gamma=COMMON["gamma"], lr=cfg["lr"], rms_decay=COMMON["rms_decay"], rms_eps=COMMON["rms_eps"],
+              clip_norm=COMMON["clip_norm"], entropy_beta=COMMON["entropy_beta"], value_coef=COMMON["value_coef"],
+              term_denom=cfg["term_denom"])
+    o = orc.OraclePAAC(cfg["arch"], n_e_sample, cfg["t_max"], cfg["n_actions"], COMMON["seed"],
+                       bf16=cfg["precision"] == "bf16", hp=hp)
+    for _ in range(warm):
+        o.rollout()
+        o.update()
+    t0 = time.time()
+    for _ in range(iters):
+        o.rollout()
+        o.update()
+    return (time.time() - t0) / iters
+
+
+def run_reference(args, cfg):
+    """The oracle as it stands on the host cores; each step is one iteration on a bounded sample."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    cores = os.cpu_count() or 1
+    total = max(1, args.steps + args.warmup)
+    n_s = 1
+    while n_s * 2 <= min(cfg["n_e"], 256) and 0.7 * n_s * 2 * total / max(cores, 1) <= 150:
+        n_s *= 2
+    sec = oracle_time(cfg, n_s, args.steps, warm=args.warmup)
+    val = n_s * cfg["t_max"] / sec
+    sample = "one iteration per step on the first %d of %d environments" % (n_s, cfg["n_e"])
+    print(json.dumps({
+        "impl": "reference", "metric": "env_steps_per_sec", "value": val, "unit": "env-steps/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg),
+        "cpu_baseline": {"value": val, "unit": "env-steps/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "env-steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def workload_config(cfg):
+    return {"workload": cfg["name"], "arch": cfg["arch"], "precision": cfg["precision"], "n_e": cfg["n_e"],
+            "t_max": cfg["t_max"], "n_actions": cfg["n_actions"], "update_batch": cfg["n_e"] * cfg["t_max"],
+            "l2": "per-step working set (frames + stored activations) exceeds the 126 MB L2"
+                  if cfg["n_e"] >= 256 else "working set fits L2; an L2-sized buffer is rewritten between steps"}
+
+
+# ----------------------------------------------------------------------------- our arm
+def run_ours(args, cfg):
+    import torch
+    from paper_1705_04862_b200 import binding as pb
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    hp = dict(gamma=COMMON["gamma"], lr=cfg["lr"], rms_decay=COMMON["rms_decay"], rms_eps=COMMON["rms_eps"],
+              clip_norm=COMMON["clip_norm"], entropy_beta=COMMON["entropy_beta"], value_coef=COMMON["value_coef"],
+              term_denom=cfg["term_denom"])
+    prec = pb.BF16 if cfg["precision"] == "bf16" else pb.FP32
+    g = pb.Paac(cfg["arch"], cfg["n_e"], cfg["t_max"], cfg["n_actions"], COMMON["seed"] + rank, precision=prec,
+                device="cuda:%d" % local, **hp)
+    n_e, T = cfg["n_e"], cfg["t_max"]
+    small = cfg["n_e"] < 256
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if small else None
+
+    def step(sync_stats=False):
+        if flush is not None:
+            flush.zero_()
+        g.rollout()
+        return g.update(sync=sync_stats)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    # ---- timed region: K whole iterations, device time, max over ranks
+    K = args.steps
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K + 1)]
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    l0, t0 = g.launch_count(), time.time()
+    ev[0].record()
+    for k in range(K):
+        if flush is not None:
+            flush.zero_()
+        g.rollout()
+        ev[2 * k + 1].record()
+        g.update(sync=False)
+        ev[2 * k + 2].record()
+    barrier()
+    t1 = time.time()
+    launches = g.launch_count() - l0
+    clocks = sampler.stop(t0, t1) if sampler else None
+    total_ms = ev[0].elapsed_time(ev[2 * K])
+    roll_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(K)) / K
+    upd_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(K)) / K
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / K
+    value = world * n_e * T / (ms_per_step * 1e-3)
+
+    # ---- per-kernel CUDA-event breakdown over another K steps (same kernels, event pairs around each)
+    g.profile(True)
+    for _ in range(K):
+        step()
+    prof = g.profile_read()
+    g.profile(False)
+
+    # ---- end to end through the external-environment entry points (host frames in, actions out)
+    frames_dev = torch.empty(0)
+    e2e = None
+    if rank == 0 or world > 1:
+        g.rollout()
+        import numpy as np
+        fr = g.debug_read(pb.DBG_FRAMES).reshape(T, n_e, FRAME_BYTES)
+        nx = g.debug_read(pb.DBG_NEXT_FRAMES).reshape(1, n_e, FRAME_BYTES)
+        host_frames = torch.from_numpy(np.concatenate([fr, nx])).pin_memory()
+        host_r = torch.from_numpy(g.debug_read(pb.DBG_REWARDS).reshape(T, n_e).copy()).pin_memory()
+        host_t = torch.from_numpy(g.debug_read(pb.DBG_TERMINALS).reshape(T, n_e).copy()).pin_memory()
+        host_a = torch.zeros(n_e, dtype=torch.int32).pin_memory()
+        host_v = torch.zeros(n_e, dtype=torch.float32).pin_memory()
+        g.update()
+
+        def e2e_step():
+            for t in range(T):
+                g.act_host(t, host_frames[t], host_a, host_v)
+                g.observe_host(t, host_r[t], host_t[t])
+            g.act_host(T, host_frames[T], None, host_v)
+            return g.update(sync=True)
+
+        Ke = max(3, min(K, 10))
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        w0 = time.time()
+        for _ in range(Ke):
+            e2e_step()
+        barrier()
+        e_sec = (time.time() - w0) / Ke
+        if dist is not None:
+            t = torch.tensor([e_sec], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_sec = float(t.item())
+        e2e = {"value": world * n_e * T / e_sec, "unit": "env-steps/s", "ms_per_step": e_sec * 1e3,
+               "h2d_bytes_per_step": (T + 1) * n_e * FRAME_BYTES + 2 * T * n_e,
+               "d2h_bytes_per_step": T * n_e * 4 + (T + 1) * n_e * 4 + 32,
+               "api": "paac_act_host / paac_observe_host / paac_update, pinned host buffers, wall clock"}
+    del frames_dev
+    g.close()
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the kernel family that takes the most time
+    pk = peaks()
+    work, P = kernel_work(cfg)
+    tot = sum(ms for ms, _ in prof.values())
+    shares = {k: {"ms_per_step": ms / K, "launches_per_step": n / K, "share": ms / tot} for k, (ms, n) in prof.items()}
+    dom = max(prof, key=lambda k: prof[k][0])
+    dom_ms = prof[dom][0] / prof[dom][1]
+    bound, amount = work.get(dom, ("hbm", 0.0))
+    if bound == "tensor":
+        ach, peak, unit = amount / (dom_ms * 1e-3) / 1e12, pk["bf16"], "TFLOP/s"
+    else:
+        ach, peak, unit = amount / (dom_ms * 1e-3) / 1e9, pk["hbm"], "GB/s"
+    roofline = {"kernel": dom, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
+                "traffic": None, "peak_source": pk["src"], "avg_launch_ms": dom_ms,
+                "algorithmic_per_launch": amount}
+    side = {}
+    for k in ("env_step", "clip_rmsprop", "grad_sumsq"):
+        if k in prof and prof[k][1]:
+            gbs = work[k][1] / (prof[k][0] / prof[k][1] * 1e-3) / 1e9
+            side[k] = {"GB/s": gbs, "frac_of_%s_hbm" % pk["src"]: gbs / pk["hbm"]}
+    roll_flops, upd_flops = iteration_flops(cfg)
+
+    # ---- CPU oracle on a bounded sample (rank 0, one GPU only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cores = os.cpu_count() or 1
+        n_s = min(cfg["n_e"], 128 if cfg["arch"] == "nature" else 512)
+        sec = oracle_time(cfg, n_s, 1)
+        cpu = {"value": n_s * T / sec, "unit": "env-steps/s", "cores": cores, "kind": "oracle",
+               "sample": "one iteration on the first %d of %d environments (%.1f s)" % (n_s, cfg["n_e"], sec)}
+
+    out = {
+        "metric": "env_steps_per_sec", "value": value, "unit": "env-steps/s", "n_gpus": world, "steps": K,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": cfg["precision"], "data": "synthetic", "config": workload_config(cfg),
+        "updates_per_sec": world * 1e3 / ms_per_step, "rollout_ms": roll_ms, "update_ms": upd_ms,
+        "update_tflops": upd_flops / (upd_ms * 1e-3) / 1e12,
+        "update_frac_of_bf16_peak": upd_flops / (upd_ms * 1e-3) / 1e12 / pk["bf16"],
+        "rollout_tflops": roll_flops / (roll_ms * 1e-3) / 1e12,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "hbm_kernels": side,
+        "kernels": shares, "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=4, help="index into the five workloads (4 = n_e 1024, Nature CNN, bf16)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -193,6 +193,17 @@ int paac_debug_write(paac_ctx* ctx, int which, const void* src /* host */, size_
 /* Number of kernels the library has launched on this context since init. */
 uint64_t paac_launch_count(const paac_ctx* ctx);
 
+/* Per-kernel timing for the time-usage breakdown (the paper's Fig. 2 splits an iteration into
+ * environment interaction, action selection and learning).  enable != 0: zero the totals and
+ * bracket every following kernel launch with a CUDA event pair on the context's stream;
+ * enable == 0: stop.  Synchronises.  Timed runs launch the same kernels, slightly spaced out. */
+int paac_profile(paac_ctx* ctx, int enable);
+/* Totals since profiling was enabled, one entry per kernel family that ran: names[i] (static
+ * strings owned by the library), ms[i] device milliseconds, launches[i].  Arrays are host, sized
+ * max_entries.  Returns the number of entries written, or -1 on bad arguments.  Synchronises. */
+int paac_profile_read(paac_ctx* ctx, int max_entries, const char** names /* out */, double* ms /* out */,
+                      uint64_t* launches /* out */);
+
 #ifdef __cplusplus
 }
 #endif

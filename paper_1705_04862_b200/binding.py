@@ -45,7 +45,7 @@ class UpdateStats(C.Structure):
 EXPORTS = ["paac_default_hparams", "paac_workspace_bytes", "paac_init", "paac_rollout", "paac_update",
            "paac_param_count", "paac_params", "paac_destroy", "paac_strerror", "paac_act_host",
            "paac_observe_host", "paac_set_params", "paac_force_actions", "paac_debug_bytes", "paac_debug_read",
-           "paac_debug_write", "paac_launch_count"]
+           "paac_debug_write", "paac_launch_count", "paac_profile", "paac_profile_read"]
 
 _lib = None
 
@@ -82,6 +82,8 @@ def lib():
         L.paac_debug_write.argtypes = [vp, i, vp, sz]
         L.paac_launch_count.argtypes = [vp]
         L.paac_launch_count.restype = u64
+        L.paac_profile.argtypes = [vp, i]
+        L.paac_profile_read.argtypes = [vp, i, C.POINTER(C.c_char_p), C.POINTER(C.c_double), C.POINTER(u64)]
         _lib = L
     return _lib
 
@@ -213,6 +215,18 @@ class Paac:
 
     def launch_count(self):
         return int(lib().paac_launch_count(self._h))
+
+    def profile(self, enable):
+        _check(lib().paac_profile(self._h, 1 if enable else 0))
+
+    def profile_read(self):
+        """{kernel family: (device ms, launches)} since profiling was enabled."""
+        n = 64
+        names, ms, cnt = (C.c_char_p * n)(), (C.c_double * n)(), (C.c_uint64 * n)()
+        k = lib().paac_profile_read(self._h, n, names, ms, cnt)
+        if k < 0:
+            raise PaacError(ERR_ARG)
+        return {names[j].decode(): (ms[j], int(cnt[j])) for j in range(k)}
 
     def close(self):
         if getattr(self, "_h", None):

@@ -12,12 +12,12 @@ struct paac_ctx {
   paac_hparams hp;
   uint64_t seed;
   NetDims nd;
+  LaunchCtx lc;            // stream, launch counter, optional per-kernel timing
   cudaStream_t st;
   int device;
   bool owns_workspace;
   char* ws;
   size_t ws_bytes;
-  uint64_t launches;
   uint64_t N;              // timesteps consumed by updates
   uint64_t env_step;       // global step index of the environments (same for all)
   bool rollout_fresh;      // a rollout has completed since the last update
@@ -114,9 +114,9 @@ void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, uin
   void* act[MAX_LAYERS];
   for (int l = 0; l <= c->nd.n_conv; ++l)
     act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
-  simt_forward(c->st, &c->launches, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
+  simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
   const size_t row = (size_t)slot * c->n_e;
-  launch_heads(c->st, &c->launches, c->prec, c->nd, c->theta, c->theta16, act[c->nd.n_conv], c->n_e,
+  launch_heads(c->lc, c->prec, c->nd, c->theta, c->theta16, act[c->nd.n_conv], c->n_e,
                c->logits + row * c->A, c->values + row, c->seed, step,
                sample && c->forced_on ? c->forced + row : nullptr, sample ? c->actions + row : nullptr,
                sample ? c->sampled + row : nullptr, sample ? c->uniforms + row : nullptr);
@@ -148,7 +148,7 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   paac_ctx* c = new (std::nothrow) paac_ctx{};
   if (!c) return PAAC_ERR_CUDA;
   fill_shape(c, arch, n_e, t_max, n_actions, hp);
-  c->seed = seed; c->device = dev; c->st = (cudaStream_t)hp->stream;
+  c->seed = seed; c->device = dev; c->st = (cudaStream_t)hp->stream; c->lc.st = c->st;
   const size_t need = carve(c, nullptr);
   if (hp->workspace) {
     if (hp->workspace_bytes < need || ((uintptr_t)hp->workspace & 255)) { delete c; return PAAC_ERR_WORKSPACE; }
@@ -161,10 +161,10 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   carve(c, c->ws);
   cudaMemsetAsync(c->ws, 0, need, c->st);
   cudaMemsetAsync(c->forced, 0xFF, (size_t)c->B * sizeof(int32_t), c->st);
-  launch_init_params(c->st, &c->launches, c->nd, seed, c->theta);
-  launch_cast_bf16(c->st, &c->launches, c->theta, c->theta16, c->nd.P);
+  launch_init_params(c->lc, c->nd, seed, c->theta);
+  launch_cast_bf16(c->lc, c->theta, c->theta16, c->nd.P);
   c->cur = 1;   // the first rollout flips to buffer 0; its start states are written there now
-  launch_env_step(c->st, &c->launches, seed, n_e, 0u, nullptr, hp->term_denom, c->frames[0], nullptr, nullptr, nullptr);
+  launch_env_step(c->lc, seed, n_e, 0u, nullptr, hp->term_denom, c->frames[0], nullptr, nullptr, nullptr);
   if (cudaStreamSynchronize(c->st) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
     if (c->owns_workspace) cudaFree(c->ws);
     delete c;
@@ -185,7 +185,7 @@ int paac_rollout(paac_ctx* c, paac_rollout_view* view) {
     forward_slot(c, fr + t * fstep, t, true, c->env_step + t);
     uint8_t* dst = t + 1 < c->t_max ? fr + (t + 1) * fstep : nxt;
     const size_t row = (size_t)t * c->n_e;
-    launch_env_step(c->st, &c->launches, c->seed, c->n_e, (uint32_t)(c->env_step + t), c->actions + row,
+    launch_env_step(c->lc, c->seed, c->n_e, (uint32_t)(c->env_step + t), c->actions + row,
                     c->hp.term_denom, dst, c->rewards + row, c->terminals + row, c->counters);
   }
   forward_slot(c, nxt, c->t_max, false, 0);
@@ -202,15 +202,15 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
   if (!c) return PAAC_ERR_ARG;
   if (!c->rollout_fresh) return PAAC_ERR_STATE;
   const paac_hparams& hp = c->hp;
-  launch_returns(c->st, &c->launches, c->n_e, c->t_max, hp.gamma, c->rewards, c->terminals, c->values, c->R, c->adv);
-  launch_head_grad(c->st, &c->launches, c->B, c->A, hp.entropy_beta, hp.value_coef, c->logits, c->values, c->actions,
+  launch_returns(c->lc, c->n_e, c->t_max, hp.gamma, c->rewards, c->terminals, c->values, c->R, c->adv);
+  launch_head_grad(c->lc, c->B, c->A, hp.entropy_beta, hp.value_coef, c->logits, c->values, c->actions,
                    c->R, c->adv, c->dz, c->dV, c->loss_terms, c->stats);
   const int L = c->nd.n_conv;
-  heads_backward(c->st, &c->launches, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
+  heads_backward(c->lc, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
                  c->grad, c->scratch);
-  simt_backward(c->st, &c->launches, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
+  simt_backward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
                 c->gact, c->grad, c->scratch);
-  launch_clip_rmsprop(c->st, &c->launches, c->nd.P, c->theta, c->rms, c->grad,
+  launch_clip_rmsprop(c->lc, c->nd.P, c->theta, c->rms, c->grad,
                       c->prec == PAAC_BF16 ? c->theta16 : nullptr, hp.lr, hp.rms_decay, hp.rms_eps, hp.clip_norm,
                       c->norm_partials, c->stats);
   c->N += (uint64_t)c->B;
@@ -243,7 +243,7 @@ int paac_set_params(paac_ctx* c, const float* src, size_t n) {
   if (cudaMemcpyAsync(c->theta, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
     cudaGetLastError(); return PAAC_ERR_CUDA;
   }
-  launch_cast_bf16(c->st, &c->launches, c->theta, c->theta16, n);
+  launch_cast_bf16(c->lc, c->theta, c->theta16, n);
   if (cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
   return cuda_status(c);
 }
@@ -262,6 +262,7 @@ int paac_force_actions(paac_ctx* c, const int32_t* actions) {
 int paac_destroy(paac_ctx* c) {
   if (!c) return PAAC_ERR_ARG;
   cudaStreamSynchronize(c->st);
+  c->lc.release();
   if (c->owns_workspace) cudaFree(c->ws);
   cudaGetLastError();
   delete c;
@@ -281,7 +282,29 @@ const char* paac_strerror(int s) {
   }
 }
 
-uint64_t paac_launch_count(const paac_ctx* c) { return c ? c->launches : 0; }
+uint64_t paac_launch_count(const paac_ctx* c) { return c ? c->lc.count : 0; }
+
+int paac_profile(paac_ctx* c, int enable) {
+  if (!c) return PAAC_ERR_ARG;
+  if (cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  c->lc.collect();
+  if (enable) { for (int i = 0; i < KID_COUNT; ++i) { c->lc.ms[i] = 0.0; c->lc.calls[i] = 0; } }
+  c->lc.profiling = enable != 0;
+  return PAAC_OK;
+}
+
+int paac_profile_read(paac_ctx* c, int max_entries, const char** names, double* ms, uint64_t* launches) {
+  if (!c || max_entries < 0 || !names || !ms || !launches) return -1;
+  if (cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return -1; }
+  c->lc.collect();
+  int n = 0;
+  for (int i = 0; i < KID_COUNT && n < max_entries; ++i) {
+    if (c->lc.calls[i] == 0) continue;
+    names[n] = kernel_name(i); ms[n] = c->lc.ms[i]; launches[n] = c->lc.calls[i];
+    ++n;
+  }
+  return n;
+}
 
 // ---- external-environment mode ------------------------------------------------------------------
 int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, float* values) {

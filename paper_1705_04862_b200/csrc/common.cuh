@@ -122,6 +122,65 @@ inline NetDims make_net(int arch, int A) {
   return n;
 }
 
+// ---- launch bookkeeping ----------------------------------------------------------------------
+// Kernel families, for the launch counter and the optional per-kernel CUDA-event timing.
+enum KernelId {
+  KID_INIT = 0, KID_ENV_STEP, KID_CONV1_FWD, KID_CONV2_FWD, KID_CONV3_FWD, KID_FC_FWD, KID_HEADS_FWD,
+  KID_RETURNS, KID_HEAD_GRAD, KID_HEADS_BWD, KID_FC_WGRAD, KID_FC_DGRAD, KID_CONV3_WGRAD, KID_CONV3_DGRAD,
+  KID_CONV2_WGRAD, KID_CONV2_DGRAD, KID_CONV1_WGRAD, KID_WGRAD_REDUCE, KID_SUMSQ, KID_CLIP_RMSPROP, KID_CAST,
+  KID_COUNT
+};
+inline const char* kernel_name(int id) {
+  static const char* names[KID_COUNT] = {
+      "init_params", "env_step", "conv1_fwd", "conv2_fwd", "conv3_fwd", "fc_fwd", "heads_fwd_sample", "returns",
+      "head_grad", "heads_bwd", "fc_wgrad", "fc_dgrad", "conv3_wgrad", "conv3_dgrad", "conv2_wgrad", "conv2_dgrad",
+      "conv1_wgrad", "wgrad_reduce", "grad_sumsq", "clip_rmsprop", "cast_bf16"};
+  return id >= 0 && id < KID_COUNT ? names[id] : "?";
+}
+
+struct LaunchCtx {
+  cudaStream_t st = nullptr;
+  uint64_t count = 0;                 // kernels launched so far
+  bool profiling = false;             // record a CUDA event pair around every launch
+  static constexpr int MAX_PENDING = 512;
+  cudaEvent_t ev[MAX_PENDING][2];
+  int ev_kid[MAX_PENDING];
+  int n_events = 0, n_created = 0;
+  double ms[KID_COUNT] = {};          // accumulated device time per family
+  uint64_t calls[KID_COUNT] = {};
+
+  // fold the pending event pairs into ms[]; the stream must be idle
+  void collect() {
+    for (int i = 0; i < n_events; ++i) {
+      float t = 0.f;
+      if (cudaEventElapsedTime(&t, ev[i][0], ev[i][1]) == cudaSuccess) { ms[ev_kid[i]] += t; calls[ev_kid[i]] += 1; }
+    }
+    n_events = 0;
+  }
+  void release() {
+    for (int i = 0; i < n_created; ++i) { cudaEventDestroy(ev[i][0]); cudaEventDestroy(ev[i][1]); }
+    n_created = n_events = 0;
+  }
+};
+
+// Brackets one kernel launch: counts it and, when profiling, times it with an event pair.
+struct KernelScope {
+  LaunchCtx& lc; int slot;
+  KernelScope(LaunchCtx& l, int kid) : lc(l), slot(-1) {
+    ++lc.count;
+    if (!lc.profiling) return;
+    if (lc.n_events == LaunchCtx::MAX_PENDING) { cudaStreamSynchronize(lc.st); lc.collect(); }
+    slot = lc.n_events++;
+    if (slot >= lc.n_created) {
+      cudaEventCreate(&lc.ev[slot][0]); cudaEventCreate(&lc.ev[slot][1]);
+      lc.n_created = slot + 1;
+    }
+    lc.ev_kid[slot] = kid;
+    cudaEventRecord(lc.ev[slot][0], lc.st);
+  }
+  ~KernelScope() { if (slot >= 0) cudaEventRecord(lc.ev[slot][1], lc.st); }
+};
+
 // device-side statistics block written by the update kernels
 struct DeviceStats {
   float policy_loss, value_loss, entropy, grad_norm, clip_scale;

@@ -13,39 +13,39 @@ __global__ void xavier_kernel(float* w, uint32_t count, float bound, uint32_t la
   }
 }
 
-static void xavier(cudaStream_t st, uint64_t* launches, float* w, size_t count, double fan_in, double fan_out,
+static void xavier(LaunchCtx& lc, float* w, size_t count, double fan_in, double fan_out,
                    uint32_t layer, uint64_t seed) {
   const float bound = (float)sqrt(6.0 / (fan_in + fan_out));
   int blocks = (int)((count + 255) / 256);
   if (blocks > 1184) blocks = 1184;
-  xavier_kernel<<<blocks, 256, 0, st>>>(w, (uint32_t)count, bound, layer, seed);
-  ++*launches;
+  KernelScope scope(lc, KID_INIT);
+  xavier_kernel<<<blocks, 256, 0, lc.st>>>(w, (uint32_t)count, bound, layer, seed);
 }
 
-void launch_init_params(cudaStream_t st, uint64_t* launches, const NetDims& nd, uint64_t seed, float* theta) {
-  cudaMemsetAsync(theta, 0, nd.P * sizeof(float), st);
+void launch_init_params(LaunchCtx& lc, const NetDims& nd, uint64_t seed, float* theta) {
+  cudaMemsetAsync(theta, 0, nd.P * sizeof(float), lc.st);
   uint32_t id = 0;
   for (int l = 0; l < nd.n_conv; ++l, ++id) {
     const LayerDims& d = nd.layer[l];
     const double kk = (double)d.K * d.K;
-    xavier(st, launches, theta + d.w_off, (size_t)d.CO * d.K * d.K * d.C, kk * d.C, kk * d.CO, id, seed);
+    xavier(lc, theta + d.w_off, (size_t)d.CO * d.K * d.K * d.C, kk * d.C, kk * d.CO, id, seed);
   }
   const LayerDims& f = nd.layer[nd.n_conv];
   const size_t in = (size_t)f.H * f.W * f.C;
-  xavier(st, launches, theta + f.w_off, in * nd.F, (double)in, (double)nd.F, id++, seed);
-  xavier(st, launches, theta + nd.pi_w, (size_t)nd.A * nd.F, (double)nd.F, (double)nd.A, id++, seed);
-  xavier(st, launches, theta + nd.v_w, (size_t)nd.F, (double)nd.F, 1.0, id++, seed);
+  xavier(lc, theta + f.w_off, in * nd.F, (double)in, (double)nd.F, id++, seed);
+  xavier(lc, theta + nd.pi_w, (size_t)nd.A * nd.F, (double)nd.F, (double)nd.A, id++, seed);
+  xavier(lc, theta + nd.v_w, (size_t)nd.F, (double)nd.F, 1.0, id++, seed);
 }
 
 __global__ void cast_bf16_kernel(const float* src, bf16* dst, size_t n) {
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     dst[i] = __float2bfloat16_rn(src[i]);
 }
-void launch_cast_bf16(cudaStream_t st, uint64_t* launches, const float* src, bf16* dst, size_t n) {
+void launch_cast_bf16(LaunchCtx& lc, const float* src, bf16* dst, size_t n) {
   int blocks = (int)((n + 255) / 256);
   if (blocks > 1184) blocks = 1184;
-  cast_bf16_kernel<<<blocks, 256, 0, st>>>(src, dst, n);
-  ++*launches;
+  KernelScope scope(lc, KID_CAST);
+  cast_bf16_kernel<<<blocks, 256, 0, lc.st>>>(src, dst, n);
 }
 
 // One block per environment.  The block's first thread decides reward and terminal flag of
@@ -94,12 +94,12 @@ env_step_kernel(uint64_t seed, int n_e, uint32_t step, const int32_t* __restrict
   }
 }
 
-void launch_env_step(cudaStream_t st, uint64_t* launches, uint64_t seed, int n_e, uint32_t step,
+void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, uint32_t step,
                      const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
                      uint8_t* terminals, int32_t* counters) {
-  env_step_kernel<<<n_e, ENV_THREADS, 0, st>>>(seed, n_e, step, actions, term_denom, next_frames, rewards, terminals,
-                                               counters);
-  ++*launches;
+  KernelScope scope(lc, KID_ENV_STEP);
+  env_step_kernel<<<n_e, ENV_THREADS, 0, lc.st>>>(seed, n_e, step, actions, term_denom, next_frames, rewards,
+                                                  terminals, counters);
 }
 
 }  // namespace paac

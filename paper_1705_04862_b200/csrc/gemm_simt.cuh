@@ -68,13 +68,13 @@ gemm_simt_kernel(int M, int N, int K, int k_per_split, LA la, LB lb, EP ep) {
 }
 
 template <class LA, class LB, class EP>
-inline void gemm_simt(cudaStream_t st, uint64_t* launches, int M, int N, int K, int splits, LA la, LB lb, EP ep) {
+inline void gemm_simt(LaunchCtx& lc, int kid, int M, int N, int K, int splits, LA la, LB lb, EP ep) {
   if (M <= 0 || N <= 0 || K <= 0) return;
+  KernelScope scope(lc, kid);
   int kps = (K + splits - 1) / splits;
   kps = (kps + SG_BK - 1) / SG_BK * SG_BK;
   dim3 grid((M + SG_BM - 1) / SG_BM, (N + SG_BN - 1) / SG_BN, (K + kps - 1) / kps);
-  gemm_simt_kernel<<<grid, SG_THREADS, 0, st>>>(M, N, K, kps, la, lb, ep);
-  ++*launches;
+  gemm_simt_kernel<<<grid, SG_THREADS, 0, lc.st>>>(M, N, K, kps, la, lb, ep);
 }
 // number of k-splits gemm_simt will really launch for a requested count
 inline int gemm_simt_splits(int K, int splits) {

@@ -63,10 +63,12 @@ heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* _
   }
 }
 
-void launch_heads(cudaStream_t st, uint64_t* launches, int prec, const NetDims& nd, const float* theta,
+void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
                   const bf16* theta16, const void* h, int n, float* logits, float* values, uint64_t seed,
                   uint64_t step, const int32_t* forced, int32_t* actions, int32_t* sampled, float* uniforms) {
   const int blocks = (n + 3) / 4;
+  KernelScope scope(lc, KID_HEADS_FWD);
+  cudaStream_t st = lc.st;
   if (prec == PAAC_BF16)
     heads_kernel<bf16, bf16><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, theta + nd.pi_b,
                                                      theta16 + nd.v_w, theta + nd.v_b, n, nd.F, nd.A, logits, values,
@@ -75,7 +77,6 @@ void launch_heads(cudaStream_t st, uint64_t* launches, int prec, const NetDims& 
     heads_kernel<float, float><<<blocks, 128, 0, st>>>((const float*)h, theta + nd.pi_w, theta + nd.pi_b,
                                                        theta + nd.v_w, theta + nd.v_b, n, nd.F, nd.A, logits, values,
                                                        seed, step, forced, actions, sampled, uniforms);
-  ++*launches;
 }
 
 // One thread per environment walks its t_max transitions backwards:
@@ -95,10 +96,10 @@ __global__ void returns_kernel(int n_e, int t_max, float gamma, const int8_t* __
   }
 }
 
-void launch_returns(cudaStream_t st, uint64_t* launches, int n_e, int t_max, float gamma, const int8_t* rewards,
+void launch_returns(LaunchCtx& lc, int n_e, int t_max, float gamma, const int8_t* rewards,
                     const uint8_t* terminals, const float* values, float* R, float* adv) {
-  returns_kernel<<<(n_e + 127) / 128, 128, 0, st>>>(n_e, t_max, gamma, rewards, terminals, values, R, adv);
-  ++*launches;
+  KernelScope scope(lc, KID_RETURNS);
+  returns_kernel<<<(n_e + 127) / 128, 128, 0, lc.st>>>(n_e, t_max, gamma, rewards, terminals, values, R, adv);
 }
 
 // One warp per experience: d/dz and d/dV of
@@ -155,13 +156,16 @@ __global__ void __launch_bounds__(256) loss_stats_kernel(int B, const float* __r
   }
 }
 
-void launch_head_grad(cudaStream_t st, uint64_t* launches, int B, int A, float beta, float value_coef,
+void launch_head_grad(LaunchCtx& lc, int B, int A, float beta, float value_coef,
                       const float* logits, const float* values, const int32_t* actions, const float* R,
                       const float* adv, float* dz, float* dV, float* loss_terms, DeviceStats* stats) {
-  head_grad_kernel<<<(B + 3) / 4, 128, 0, st>>>(B, A, beta, value_coef, logits, values, actions, R, adv, dz, dV,
-                                                loss_terms);
-  loss_stats_kernel<<<1, 256, 0, st>>>(B, loss_terms, stats);
-  *launches += 2;
+  {
+    KernelScope scope(lc, KID_HEAD_GRAD);
+    head_grad_kernel<<<(B + 3) / 4, 128, 0, lc.st>>>(B, A, beta, value_coef, logits, values, actions, R, adv, dz, dV,
+                                                     loss_terms);
+  }
+  KernelScope scope(lc, KID_HEAD_GRAD);
+  loss_stats_kernel<<<1, 256, 0, lc.st>>>(B, loss_terms, stats);
 }
 
 }  // namespace paac

@@ -1,24 +1,24 @@
-// Host-side launchers of the PAAC kernels.  Every function enqueues work on `st`
-// and bumps *launches once per kernel launch; none synchronises.
+// Host-side launchers of the PAAC kernels.  Every function enqueues work on lc.st and
+// counts (and optionally times) each kernel launch through lc; none synchronises.
 #pragma once
 #include "common.cuh"
 
 namespace paac {
 
 // ---- initialisation and environment (env.cu) -----------------------------------------
-void launch_init_params(cudaStream_t st, uint64_t* launches, const NetDims& nd, uint64_t seed, float* theta);
-void launch_cast_bf16(cudaStream_t st, uint64_t* launches, const float* src, bf16* dst, size_t n);
+void launch_init_params(LaunchCtx& lc, const NetDims& nd, uint64_t seed, float* theta);
+void launch_cast_bf16(LaunchCtx& lc, const float* src, bf16* dst, size_t n);
 // actions == nullptr: start states (step index 0) for every environment
-void launch_env_step(cudaStream_t st, uint64_t* launches, uint64_t seed, int n_e, uint32_t step,
+void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, uint32_t step,
                      const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
                      uint8_t* terminals, int32_t* counters /* [3][n_e] */);
 
 // ---- network on the CUDA cores (net_simt.cu) --------------------------------------------
 // act[l]: stored activation of layer l for the n states, storage float (PAAC_FP32) or bf16
-void simt_forward(cudaStream_t st, uint64_t* launches, int arch, int prec, const NetDims& nd, const float* theta,
+void simt_forward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
                   const bf16* theta16, const uint8_t* frames, int n, void* const act[]);
 // from gact[fc] (gradient at the fc pre-activation) down to conv1; fills grad for conv and fc layers
-void simt_backward(cudaStream_t st, uint64_t* launches, int arch, int prec, const NetDims& nd, const float* theta,
+void simt_backward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
                    const bf16* theta16, const uint8_t* frames, int n, void* const act[], void* const gact[],
                    float* grad, float* scratch);
 // scratch floats simt_backward / heads_backward need for split-k partials
@@ -26,23 +26,23 @@ size_t simt_scratch_floats(int arch, const NetDims& nd, int n);
 
 // ---- heads, sampling, returns, loss gradient (heads.cu) -----------------------------------
 // logits/values of n states from the fc activation; if actions != nullptr also samples
-void launch_heads(cudaStream_t st, uint64_t* launches, int prec, const NetDims& nd, const float* theta,
+void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
                   const bf16* theta16, const void* h, int n, float* logits, float* values, uint64_t seed,
                   uint64_t step, const int32_t* forced, int32_t* actions, int32_t* sampled /* action before forcing */,
                   float* uniforms);
-void launch_returns(cudaStream_t st, uint64_t* launches, int n_e, int t_max, float gamma, const int8_t* rewards,
+void launch_returns(LaunchCtx& lc, int n_e, int t_max, float gamma, const int8_t* rewards,
                     const uint8_t* terminals, const float* values, float* R, float* adv);
-void launch_head_grad(cudaStream_t st, uint64_t* launches, int B, int A, float beta, float value_coef,
+void launch_head_grad(LaunchCtx& lc, int B, int A, float beta, float value_coef,
                       const float* logits, const float* values, const int32_t* actions, const float* R,
                       const float* adv, float* dz, float* dV, float* loss_terms /* [3][B] */, DeviceStats* stats);
 // gradient of the two heads' parameters and of the fc pre-activation
-void heads_backward(cudaStream_t st, uint64_t* launches, int prec, const NetDims& nd, const float* theta,
+void heads_backward(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
                     const bf16* theta16, const void* h, int n, const float* dz, const float* dV, void* gact_fc,
                     float* grad, float* scratch);
 
 // ---- optimiser (optim.cu) -------------------------------------------------------------------
 constexpr int NORM_BLOCKS = 592;
-void launch_clip_rmsprop(cudaStream_t st, uint64_t* launches, size_t P, float* theta, float* rms, const float* grad,
+void launch_clip_rmsprop(LaunchCtx& lc, size_t P, float* theta, float* rms, const float* grad,
                          bf16* theta16 /* nullable */, float lr, float rho, float eps, float clip,
                          float* norm_partials /* [NORM_BLOCKS] */, DeviceStats* stats);
 

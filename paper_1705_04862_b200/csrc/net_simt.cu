@@ -16,103 +16,103 @@ static int pick_splits(int M, int N, int K) {
   return gemm_simt_splits(K, s);
 }
 
-static void reduce_wgrad(cudaStream_t st, uint64_t* launches, const float* part, int splits, int part_rows, int row0,
+static void reduce_wgrad(LaunchCtx& lc, const float* part, int splits, int part_rows, int row0,
                          int rows, int cols, float scale, float* gw, float* gb) {
   const size_t total = (size_t)rows * (cols + 1);
   int blocks = (int)((total + 255) / 256);
   if (blocks > 2368) blocks = 2368;
-  wgrad_reduce_kernel<<<blocks, 256, 0, st>>>(part, splits, part_rows, row0, rows, cols, scale, gw, gb);
-  ++*launches;
+  KernelScope scope(lc, KID_WGRAD_REDUCE);
+  wgrad_reduce_kernel<<<blocks, 256, 0, lc.st>>>(part, splits, part_rows, row0, rows, cols, scale, gw, gb);
 }
 
 template <class G, class TIn, class T, class TW>
-static void conv_fwd(cudaStream_t st, uint64_t* launches, const TIn* x, const TW* w, const float* bias, T* out, int n,
+static void conv_fwd(LaunchCtx& lc, int kid, const TIn* x, const TW* w, const float* bias, T* out, int n,
                      float scale) {
-  gemm_simt(st, launches, n * G::OH * G::OW, G::CO, G::KK, 1, ConvWindowOp<G, TIn>{x}, RowMajorOp<TW>{w, G::KK},
+  gemm_simt(lc, kid, n * G::OH * G::OW, G::CO, G::KK, 1, ConvWindowOp<G, TIn>{x}, RowMajorOp<TW>{w, G::KK},
             BiasReluEp<T>{out, bias, G::CO, scale});
 }
 template <class T, class TW>
-static void fc_fwd(cudaStream_t st, uint64_t* launches, const T* x, const TW* w, const float* bias, T* out, int n,
+static void fc_fwd(LaunchCtx& lc, int kid, const T* x, const TW* w, const float* bias, T* out, int n,
                    int IN, int F) {
-  gemm_simt(st, launches, n, F, IN, 1, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, BiasReluEp<T>{out, bias, F, 1.f});
+  gemm_simt(lc, kid, n, F, IN, 1, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, BiasReluEp<T>{out, bias, F, 1.f});
 }
 template <class G, class T, class TW>
-static void conv_dgrad(cudaStream_t st, uint64_t* launches, const T* g, const TW* w, const T* act_in, T* gin, int n) {
-  gemm_simt(st, launches, n * G::H * G::W, G::C, G::K * G::K * G::CO, 1, ConvDgradOp<G, T>{g}, ConvWeightTOp<G, TW>{w},
+static void conv_dgrad(LaunchCtx& lc, int kid, const T* g, const TW* w, const T* act_in, T* gin, int n) {
+  gemm_simt(lc, kid, n * G::H * G::W, G::C, G::K * G::K * G::CO, 1, ConvDgradOp<G, T>{g}, ConvWeightTOp<G, TW>{w},
             ReluMaskEp<T>{gin, act_in, G::C});
 }
 template <class G, class TIn, class T>
-static void conv_wgrad(cudaStream_t st, uint64_t* launches, const T* g, const TIn* x, int n, float scale, float* gw,
+static void conv_wgrad(LaunchCtx& lc, int kid, const T* g, const TIn* x, int n, float scale, float* gw,
                        float* gb, float* scratch) {
   const int M = G::CO, N = G::KK + 1, K = n * G::OH * G::OW;
   const int splits = pick_splits(M, N, K);
-  gemm_simt(st, launches, M, N, K, splits, ColMajorOp<T>{g, G::CO}, ConvWindowTOp<G, TIn>{x}, PartialEp{scratch, M, N});
-  reduce_wgrad(st, launches, scratch, splits, M, 0, M, G::KK, scale, gw, gb);
+  gemm_simt(lc, kid, M, N, K, splits, ColMajorOp<T>{g, G::CO}, ConvWindowTOp<G, TIn>{x}, PartialEp{scratch, M, N});
+  reduce_wgrad(lc, scratch, splits, M, 0, M, G::KK, scale, gw, gb);
 }
 template <class T, class TW>
-static void fc_dgrad(cudaStream_t st, uint64_t* launches, const T* g, const TW* w, const T* act_in, T* gin, int n,
+static void fc_dgrad(LaunchCtx& lc, int kid, const T* g, const TW* w, const T* act_in, T* gin, int n,
                      int IN, int F) {
-  gemm_simt(st, launches, n, IN, F, 1, RowMajorOp<T>{g, F}, ColMajorOp<TW>{w, IN}, ReluMaskEp<T>{gin, act_in, IN});
+  gemm_simt(lc, kid, n, IN, F, 1, RowMajorOp<T>{g, F}, ColMajorOp<TW>{w, IN}, ReluMaskEp<T>{gin, act_in, IN});
 }
 template <class T>
-static void fc_wgrad(cudaStream_t st, uint64_t* launches, const T* g, const T* x, int n, int IN, int F, float* gw,
+static void fc_wgrad(LaunchCtx& lc, int kid, const T* g, const T* x, int n, int IN, int F, float* gw,
                      float* gb, float* scratch) {
   const int M = F, N = IN + 1, K = n;
   const int splits = pick_splits(M, N, K);
-  gemm_simt(st, launches, M, N, K, splits, ColMajorOp<T>{g, F}, ColMajorOnesOp<T>{x, IN, IN}, PartialEp{scratch, M, N});
-  reduce_wgrad(st, launches, scratch, splits, M, 0, M, IN, 1.f, gw, gb);
+  gemm_simt(lc, kid, M, N, K, splits, ColMajorOp<T>{g, F}, ColMajorOnesOp<T>{x, IN, IN}, PartialEp{scratch, M, N});
+  reduce_wgrad(lc, scratch, splits, M, 0, M, IN, 1.f, gw, gb);
 }
 
 template <class T, class TW>
-static void forward_t(cudaStream_t st, uint64_t* L, int arch, const NetDims& nd, const float* theta, const TW* w,
+static void forward_t(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const TW* w,
                       const uint8_t* frames, int n, void* const act[]) {
   const LayerDims* d = nd.layer;
   const float s255 = 1.0f / 255.0f;
   if (arch == PAAC_ARCH_NIPS) {
-    conv_fwd<NipsConv1, uint8_t, T, TW>(st, L, frames, w + d[0].w_off, theta + d[0].b_off, (T*)act[0], n, s255);
-    conv_fwd<NipsConv2, T, T, TW>(st, L, (const T*)act[0], w + d[1].w_off, theta + d[1].b_off, (T*)act[1], n, 1.f);
-    fc_fwd<T, TW>(st, L, (const T*)act[1], w + d[2].w_off, theta + d[2].b_off, (T*)act[2], n, 2592, 256);
+    conv_fwd<NipsConv1, uint8_t, T, TW>(lc, KID_CONV1_FWD, frames, w + d[0].w_off, theta + d[0].b_off, (T*)act[0], n, s255);
+    conv_fwd<NipsConv2, T, T, TW>(lc, KID_CONV2_FWD, (const T*)act[0], w + d[1].w_off, theta + d[1].b_off, (T*)act[1], n, 1.f);
+    fc_fwd<T, TW>(lc, KID_FC_FWD, (const T*)act[1], w + d[2].w_off, theta + d[2].b_off, (T*)act[2], n, 2592, 256);
   } else {
-    conv_fwd<NatConv1, uint8_t, T, TW>(st, L, frames, w + d[0].w_off, theta + d[0].b_off, (T*)act[0], n, s255);
-    conv_fwd<NatConv2, T, T, TW>(st, L, (const T*)act[0], w + d[1].w_off, theta + d[1].b_off, (T*)act[1], n, 1.f);
-    conv_fwd<NatConv3, T, T, TW>(st, L, (const T*)act[1], w + d[2].w_off, theta + d[2].b_off, (T*)act[2], n, 1.f);
-    fc_fwd<T, TW>(st, L, (const T*)act[2], w + d[3].w_off, theta + d[3].b_off, (T*)act[3], n, 3136, 512);
+    conv_fwd<NatConv1, uint8_t, T, TW>(lc, KID_CONV1_FWD, frames, w + d[0].w_off, theta + d[0].b_off, (T*)act[0], n, s255);
+    conv_fwd<NatConv2, T, T, TW>(lc, KID_CONV2_FWD, (const T*)act[0], w + d[1].w_off, theta + d[1].b_off, (T*)act[1], n, 1.f);
+    conv_fwd<NatConv3, T, T, TW>(lc, KID_CONV3_FWD, (const T*)act[1], w + d[2].w_off, theta + d[2].b_off, (T*)act[2], n, 1.f);
+    fc_fwd<T, TW>(lc, KID_FC_FWD, (const T*)act[2], w + d[3].w_off, theta + d[3].b_off, (T*)act[3], n, 3136, 512);
   }
 }
 
 template <class T, class TW>
-static void backward_t(cudaStream_t st, uint64_t* L, int arch, const NetDims& nd, const TW* w, const uint8_t* frames,
+static void backward_t(LaunchCtx& lc, int arch, const NetDims& nd, const TW* w, const uint8_t* frames,
                        int n, void* const act[], void* const gact[], float* grad, float* scratch) {
   const LayerDims* d = nd.layer;
   const float s255 = 1.0f / 255.0f;
   if (arch == PAAC_ARCH_NIPS) {
-    fc_wgrad<T>(st, L, (const T*)gact[2], (const T*)act[1], n, 2592, 256, grad + d[2].w_off, grad + d[2].b_off, scratch);
-    fc_dgrad<T, TW>(st, L, (const T*)gact[2], w + d[2].w_off, (const T*)act[1], (T*)gact[1], n, 2592, 256);
-    conv_wgrad<NipsConv2, T, T>(st, L, (const T*)gact[1], (const T*)act[0], n, 1.f, grad + d[1].w_off, grad + d[1].b_off, scratch);
-    conv_dgrad<NipsConv2, T, TW>(st, L, (const T*)gact[1], w + d[1].w_off, (const T*)act[0], (T*)gact[0], n);
-    conv_wgrad<NipsConv1, uint8_t, T>(st, L, (const T*)gact[0], frames, n, s255, grad + d[0].w_off, grad + d[0].b_off, scratch);
+    fc_wgrad<T>(lc, KID_FC_WGRAD, (const T*)gact[2], (const T*)act[1], n, 2592, 256, grad + d[2].w_off, grad + d[2].b_off, scratch);
+    fc_dgrad<T, TW>(lc, KID_FC_DGRAD, (const T*)gact[2], w + d[2].w_off, (const T*)act[1], (T*)gact[1], n, 2592, 256);
+    conv_wgrad<NipsConv2, T, T>(lc, KID_CONV2_WGRAD, (const T*)gact[1], (const T*)act[0], n, 1.f, grad + d[1].w_off, grad + d[1].b_off, scratch);
+    conv_dgrad<NipsConv2, T, TW>(lc, KID_CONV2_DGRAD, (const T*)gact[1], w + d[1].w_off, (const T*)act[0], (T*)gact[0], n);
+    conv_wgrad<NipsConv1, uint8_t, T>(lc, KID_CONV1_WGRAD, (const T*)gact[0], frames, n, s255, grad + d[0].w_off, grad + d[0].b_off, scratch);
   } else {
-    fc_wgrad<T>(st, L, (const T*)gact[3], (const T*)act[2], n, 3136, 512, grad + d[3].w_off, grad + d[3].b_off, scratch);
-    fc_dgrad<T, TW>(st, L, (const T*)gact[3], w + d[3].w_off, (const T*)act[2], (T*)gact[2], n, 3136, 512);
-    conv_wgrad<NatConv3, T, T>(st, L, (const T*)gact[2], (const T*)act[1], n, 1.f, grad + d[2].w_off, grad + d[2].b_off, scratch);
-    conv_dgrad<NatConv3, T, TW>(st, L, (const T*)gact[2], w + d[2].w_off, (const T*)act[1], (T*)gact[1], n);
-    conv_wgrad<NatConv2, T, T>(st, L, (const T*)gact[1], (const T*)act[0], n, 1.f, grad + d[1].w_off, grad + d[1].b_off, scratch);
-    conv_dgrad<NatConv2, T, TW>(st, L, (const T*)gact[1], w + d[1].w_off, (const T*)act[0], (T*)gact[0], n);
-    conv_wgrad<NatConv1, uint8_t, T>(st, L, (const T*)gact[0], frames, n, s255, grad + d[0].w_off, grad + d[0].b_off, scratch);
+    fc_wgrad<T>(lc, KID_FC_WGRAD, (const T*)gact[3], (const T*)act[2], n, 3136, 512, grad + d[3].w_off, grad + d[3].b_off, scratch);
+    fc_dgrad<T, TW>(lc, KID_FC_DGRAD, (const T*)gact[3], w + d[3].w_off, (const T*)act[2], (T*)gact[2], n, 3136, 512);
+    conv_wgrad<NatConv3, T, T>(lc, KID_CONV3_WGRAD, (const T*)gact[2], (const T*)act[1], n, 1.f, grad + d[2].w_off, grad + d[2].b_off, scratch);
+    conv_dgrad<NatConv3, T, TW>(lc, KID_CONV3_DGRAD, (const T*)gact[2], w + d[2].w_off, (const T*)act[1], (T*)gact[1], n);
+    conv_wgrad<NatConv2, T, T>(lc, KID_CONV2_WGRAD, (const T*)gact[1], (const T*)act[0], n, 1.f, grad + d[1].w_off, grad + d[1].b_off, scratch);
+    conv_dgrad<NatConv2, T, TW>(lc, KID_CONV2_DGRAD, (const T*)gact[1], w + d[1].w_off, (const T*)act[0], (T*)gact[0], n);
+    conv_wgrad<NatConv1, uint8_t, T>(lc, KID_CONV1_WGRAD, (const T*)gact[0], frames, n, s255, grad + d[0].w_off, grad + d[0].b_off, scratch);
   }
 }
 
-void simt_forward(cudaStream_t st, uint64_t* launches, int arch, int prec, const NetDims& nd, const float* theta,
+void simt_forward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
                   const bf16* theta16, const uint8_t* frames, int n, void* const act[]) {
-  if (prec == PAAC_BF16) forward_t<bf16, bf16>(st, launches, arch, nd, theta, theta16, frames, n, act);
-  else forward_t<float, float>(st, launches, arch, nd, theta, theta, frames, n, act);
+  if (prec == PAAC_BF16) forward_t<bf16, bf16>(lc, arch, nd, theta, theta16, frames, n, act);
+  else forward_t<float, float>(lc, arch, nd, theta, theta, frames, n, act);
 }
 
-void simt_backward(cudaStream_t st, uint64_t* launches, int arch, int prec, const NetDims& nd, const float* theta,
+void simt_backward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
                    const bf16* theta16, const uint8_t* frames, int n, void* const act[], void* const gact[],
                    float* grad, float* scratch) {
-  if (prec == PAAC_BF16) backward_t<bf16, bf16>(st, launches, arch, nd, theta16, frames, n, act, gact, grad, scratch);
-  else backward_t<float, float>(st, launches, arch, nd, theta, frames, n, act, gact, grad, scratch);
+  if (prec == PAAC_BF16) backward_t<bf16, bf16>(lc, arch, nd, theta16, frames, n, act, gact, grad, scratch);
+  else backward_t<float, float>(lc, arch, nd, theta, frames, n, act, gact, grad, scratch);
 }
 
 size_t simt_scratch_floats(int arch, const NetDims& nd, int n) {
@@ -150,25 +150,25 @@ template <class TW> struct HeadWeightOp {   // row = fc unit i, k = head unit
 };
 
 template <class T, class TW>
-static void heads_backward_t(cudaStream_t st, uint64_t* L, const NetDims& nd, const TW* w, const T* h, int n,
+static void heads_backward_t(LaunchCtx& lc, const NetDims& nd, const TW* w, const T* h, int n,
                              const float* dz, const float* dV, T* gact_fc, float* grad, float* scratch) {
   const int A = nd.A, F = nd.F;
-  gemm_simt(st, L, n, F, A + 1, 1, HeadGradOp{dz, dV, A}, HeadWeightOp<TW>{w + nd.pi_w, w + nd.v_w, F, A},
+  gemm_simt(lc, KID_HEADS_BWD, n, F, A + 1, 1, HeadGradOp{dz, dV, A}, HeadWeightOp<TW>{w + nd.pi_w, w + nd.v_w, F, A},
             ReluMaskEp<T>{gact_fc, h, F});
   const int splits = pick_splits(A + 1, F + 1, n);
-  gemm_simt(st, L, A + 1, F + 1, n, splits, HeadGradTOp{dz, dV, A}, ColMajorOnesOp<T>{h, F, F},
+  gemm_simt(lc, KID_HEADS_BWD, A + 1, F + 1, n, splits, HeadGradTOp{dz, dV, A}, ColMajorOnesOp<T>{h, F, F},
             PartialEp{scratch, A + 1, F + 1});
-  reduce_wgrad(st, L, scratch, splits, A + 1, 0, A, F, 1.f, grad + nd.pi_w, grad + nd.pi_b);
-  reduce_wgrad(st, L, scratch, splits, A + 1, A, 1, F, 1.f, grad + nd.v_w, grad + nd.v_b);
+  reduce_wgrad(lc, scratch, splits, A + 1, 0, A, F, 1.f, grad + nd.pi_w, grad + nd.pi_b);
+  reduce_wgrad(lc, scratch, splits, A + 1, A, 1, F, 1.f, grad + nd.v_w, grad + nd.v_b);
 }
 
-void heads_backward(cudaStream_t st, uint64_t* launches, int prec, const NetDims& nd, const float* theta,
+void heads_backward(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
                     const bf16* theta16, const void* h, int n, const float* dz, const float* dV, void* gact_fc,
                     float* grad, float* scratch) {
   if (prec == PAAC_BF16)
-    heads_backward_t<bf16, bf16>(st, launches, nd, theta16, (const bf16*)h, n, dz, dV, (bf16*)gact_fc, grad, scratch);
+    heads_backward_t<bf16, bf16>(lc, nd, theta16, (const bf16*)h, n, dz, dV, (bf16*)gact_fc, grad, scratch);
   else
-    heads_backward_t<float, float>(st, launches, nd, theta, (const float*)h, n, dz, dV, (float*)gact_fc, grad, scratch);
+    heads_backward_t<float, float>(lc, nd, theta, (const float*)h, n, dz, dV, (float*)gact_fc, grad, scratch);
 }
 
 }  // namespace paac

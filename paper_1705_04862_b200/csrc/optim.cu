@@ -98,13 +98,16 @@ clip_rmsprop_kernel(size_t P, float* __restrict__ theta, float* __restrict__ rms
   }
 }
 
-void launch_clip_rmsprop(cudaStream_t st, uint64_t* launches, size_t P, float* theta, float* rms, const float* grad,
+void launch_clip_rmsprop(LaunchCtx& lc, size_t P, float* theta, float* rms, const float* grad,
                          bf16* theta16, float lr, float rho, float eps, float clip, float* norm_partials,
                          DeviceStats* stats) {
-  sumsq_kernel<<<NORM_BLOCKS, OPT_THREADS, 0, st>>>(grad, P, norm_partials);
-  clip_rmsprop_kernel<<<NORM_BLOCKS, OPT_THREADS, 0, st>>>(P, theta, rms, grad, theta16, lr, rho, eps, clip,
-                                                           norm_partials, NORM_BLOCKS, stats);
-  *launches += 2;
+  {
+    KernelScope scope(lc, KID_SUMSQ);
+    sumsq_kernel<<<NORM_BLOCKS, OPT_THREADS, 0, lc.st>>>(grad, P, norm_partials);
+  }
+  KernelScope scope(lc, KID_CLIP_RMSPROP);
+  clip_rmsprop_kernel<<<NORM_BLOCKS, OPT_THREADS, 0, lc.st>>>(P, theta, rms, grad, theta16, lr, rho, eps, clip,
+                                                              norm_partials, NORM_BLOCKS, stats);
 }
 
 }  // namespace paac
