@@ -190,6 +190,11 @@ int paac_debug_read(paac_ctx* ctx, int which, void* dst /* host */, size_t bytes
  * PAAC_DBG_RMS and PAAC_DBG_COUNTERS on resume). Synchronises. */
 int paac_debug_write(paac_ctx* ctx, int which, const void* src /* host */, size_t bytes);
 
+/* Run-time options.  PAAC_OPT_CUDA_CORES_ONLY != 0 keeps the bf16 network off the tensor cores
+ * (same rounding points, CUDA-core contractions): a second implementation to compare against. */
+enum { PAAC_OPT_CUDA_CORES_ONLY = 1 };
+int paac_set_option(paac_ctx* ctx, int option, int value);
+
 /* Number of kernels the library has launched on this context since init. */
 uint64_t paac_launch_count(const paac_ctx* ctx);
 

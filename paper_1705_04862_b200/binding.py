@@ -19,6 +19,7 @@ OK, ERR_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_STATE = ra
 (DBG_FRAMES, DBG_NEXT_FRAMES, DBG_ACTIONS, DBG_REWARDS, DBG_TERMINALS, DBG_VALUES, DBG_LOGITS, DBG_UNIFORMS,
  DBG_COUNTERS, DBG_RETURNS, DBG_ADVANTAGES, DBG_DLOGITS, DBG_DVALUES, DBG_GRAD, DBG_RMS, DBG_SAMPLED) = range(16)
 DBG_ACT0, DBG_GACT0 = 32, 48
+OPT_CUDA_CORES_ONLY = 1
 
 _DBG_DTYPE = {DBG_FRAMES: np.uint8, DBG_NEXT_FRAMES: np.uint8, DBG_ACTIONS: np.int32, DBG_REWARDS: np.int8,
               DBG_TERMINALS: np.uint8, DBG_COUNTERS: np.int32, DBG_SAMPLED: np.int32}
@@ -45,7 +46,7 @@ class UpdateStats(C.Structure):
 EXPORTS = ["paac_default_hparams", "paac_workspace_bytes", "paac_init", "paac_rollout", "paac_update",
            "paac_param_count", "paac_params", "paac_destroy", "paac_strerror", "paac_act_host",
            "paac_observe_host", "paac_set_params", "paac_force_actions", "paac_debug_bytes", "paac_debug_read",
-           "paac_debug_write", "paac_launch_count", "paac_profile", "paac_profile_read"]
+           "paac_debug_write", "paac_launch_count", "paac_profile", "paac_profile_read", "paac_set_option"]
 
 _lib = None
 
@@ -83,6 +84,7 @@ def lib():
         L.paac_launch_count.argtypes = [vp]
         L.paac_launch_count.restype = u64
         L.paac_profile.argtypes = [vp, i]
+        L.paac_set_option.argtypes = [vp, i, i]
         L.paac_profile_read.argtypes = [vp, i, C.POINTER(C.c_char_p), C.POINTER(C.c_double), C.POINTER(u64)]
         _lib = L
     return _lib
@@ -215,6 +217,9 @@ class Paac:
 
     def launch_count(self):
         return int(lib().paac_launch_count(self._h))
+
+    def set_option(self, option, value):
+        _check(lib().paac_set_option(self._h, option, value))
 
     def profile(self, enable):
         _check(lib().paac_profile(self._h, 1 if enable else 0))

@@ -23,6 +23,7 @@ struct paac_ctx {
   bool rollout_fresh;      // a rollout has completed since the last update
   int host_t;              // external-environment mode: next expected step
   bool forced_on;
+  bool simt_only;          // keep the bf16 network on the CUDA cores (cross-check of the tensor-core path)
 
   // device buffers (all inside the workspace)
   float *theta, *grad, *rms;
@@ -114,7 +115,10 @@ void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, uin
   void* act[MAX_LAYERS];
   for (int l = 0; l <= c->nd.n_conv; ++l)
     act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
-  simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
+  if (tc_supported(c->arch, c->prec) && !c->simt_only)
+    tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, frames, c->n_e, act, &c->stats->error_word);
+  else
+    simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
   const size_t row = (size_t)slot * c->n_e;
   launch_heads(c->lc, c->prec, c->nd, c->theta, c->theta16, act[c->nd.n_conv], c->n_e,
                c->logits + row * c->A, c->values + row, c->seed, step,
@@ -231,11 +235,19 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
 
 size_t paac_param_count(const paac_ctx* c) { return c ? c->nd.P : 0; }
 
+// a kernel whose bounded wait gave up leaves a bit in the device error word
+static int device_error(paac_ctx* c) {
+  uint32_t w = 0;
+  if (cudaMemcpyAsync(&w, &c->stats->error_word, sizeof(w), cudaMemcpyDeviceToHost, c->st) != cudaSuccess ||
+      cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  return w ? PAAC_ERR_TIMEOUT : PAAC_OK;
+}
+
 int paac_params(paac_ctx* c, float* dst, size_t n) {
   if (!c || !dst || n != c->nd.P) return PAAC_ERR_ARG;
   if (cudaMemcpyAsync(dst, c->theta, n * sizeof(float), cudaMemcpyDeviceToHost, c->st) != cudaSuccess ||
       cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
-  return PAAC_OK;
+  return device_error(c);
 }
 
 int paac_set_params(paac_ctx* c, const float* src, size_t n) {
@@ -283,6 +295,12 @@ const char* paac_strerror(int s) {
 }
 
 uint64_t paac_launch_count(const paac_ctx* c) { return c ? c->lc.count : 0; }
+
+int paac_set_option(paac_ctx* c, int option, int value) {
+  if (!c) return PAAC_ERR_ARG;
+  if (option == PAAC_OPT_CUDA_CORES_ONLY) { c->simt_only = value != 0; return PAAC_OK; }
+  return PAAC_ERR_ARG;
+}
 
 int paac_profile(paac_ctx* c, int enable) {
   if (!c) return PAAC_ERR_ARG;
@@ -386,7 +404,7 @@ int paac_debug_read(paac_ctx* c, int which, void* dst, size_t bytes) {
   if (!p || b != bytes) return PAAC_ERR_ARG;
   if (cudaMemcpyAsync(dst, p, b, cudaMemcpyDeviceToHost, c->st) != cudaSuccess ||
       cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
-  return PAAC_OK;
+  return device_error(c);
 }
 
 int paac_debug_write(paac_ctx* c, int which, const void* src, size_t bytes) {

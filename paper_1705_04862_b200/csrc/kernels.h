@@ -24,6 +24,11 @@ void simt_backward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const f
 // scratch floats simt_backward / heads_backward need for split-k partials
 size_t simt_scratch_floats(int arch, const NetDims& nd, int n);
 
+// ---- network on the tensor cores (net_tc.cu): Nature CNN, bf16 ------------------------------
+bool tc_supported(int arch, int prec);
+void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* theta16,
+                const uint8_t* frames, int n, void* const act[], uint32_t* error_word);
+
 // ---- heads, sampling, returns, loss gradient (heads.cu) -----------------------------------
 // logits/values of n states from the fc activation; if actions != nullptr also samples
 void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
