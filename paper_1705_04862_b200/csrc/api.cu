@@ -28,6 +28,7 @@ struct paac_ctx {
   // device buffers (all inside the workspace)
   float *theta, *grad, *rms;
   bf16* theta16;
+  bf16* w_images;          // regrouped bf16 weights read by the tensor-core backward kernels
   uint8_t* frames[2];      // [t_max][n_e][FRAME_BYTES] each; rollouts alternate, the bootstrap state of one
                            // rollout is written straight into slot 0 of the other
   int cur;                 // buffer the last / current rollout used
@@ -72,6 +73,7 @@ size_t carve(paac_ctx* c, char* base) {
   c->grad = k.take<float>(nd.P);
   c->rms = k.take<float>(nd.P);
   c->theta16 = k.take<bf16>(nd.P);
+  c->w_images = k.take<bf16>(tc_supported(c->arch, c->prec) ? tc_weight_image_elems() : 0);
   c->frames[0] = k.take<uint8_t>(T * n_e * FRAME_BYTES);
   c->frames[1] = k.take<uint8_t>(T * n_e * FRAME_BYTES);
   for (int l = 0; l <= nd.n_conv; ++l) {
@@ -110,12 +112,20 @@ int cuda_status(paac_ctx* c) {
   return cudaGetLastError() == cudaSuccess ? PAAC_OK : PAAC_ERR_CUDA;
 }
 
+bool use_tc(const paac_ctx* c) { return tc_supported(c->arch, c->prec) && !c->simt_only; }
+
+// bf16 copies of the master parameters, in the canonical layout and regrouped for the backward kernels
+void refresh_weight_copies(paac_ctx* c, bool cast) {
+  if (cast) launch_cast_bf16(c->lc, c->theta, c->theta16, c->nd.P);
+  if (tc_supported(c->arch, c->prec)) tc_relayout_weights(c->lc, c->nd, c->theta16, c->w_images);
+}
+
 // network + heads on the n_e states of `frames`, activations into slot `slot`
 void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, uint64_t step) {
   void* act[MAX_LAYERS];
   for (int l = 0; l <= c->nd.n_conv; ++l)
     act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
-  if (tc_supported(c->arch, c->prec) && !c->simt_only)
+  if (use_tc(c))
     tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, frames, c->n_e, act, &c->stats->error_word);
   else
     simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
@@ -166,7 +176,7 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   cudaMemsetAsync(c->ws, 0, need, c->st);
   cudaMemsetAsync(c->forced, 0xFF, (size_t)c->B * sizeof(int32_t), c->st);
   launch_init_params(c->lc, c->nd, seed, c->theta);
-  launch_cast_bf16(c->lc, c->theta, c->theta16, c->nd.P);
+  refresh_weight_copies(c, true);
   c->cur = 1;   // the first rollout flips to buffer 0; its start states are written there now
   launch_env_step(c->lc, seed, n_e, 0u, nullptr, hp->term_denom, c->frames[0], nullptr, nullptr, nullptr);
   if (cudaStreamSynchronize(c->st) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
@@ -212,11 +222,22 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
   const int L = c->nd.n_conv;
   heads_backward(c->lc, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
                  c->grad, c->scratch);
-  simt_backward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
-                c->gact, c->grad, c->scratch);
+  uint32_t* err = &c->stats->error_word;
+  for (int l = L; l >= 0; --l) {
+    // tensor-core kernels where they exist, the CUDA-core contraction otherwise
+    bool dgrad_done = false;
+    if (use_tc(c)) {
+      if (l == 3) { tc_backward_dgrad_fc(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
+      if (l == 2) { tc_backward_dgrad_conv3(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
+      if (l == 1) { tc_backward_dgrad_conv2(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
+    }
+    simt_backward_layer(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act, c->gact,
+                        c->grad, c->scratch, l, true, l > 0 && !dgrad_done);
+  }
   launch_clip_rmsprop(c->lc, c->nd.P, c->theta, c->rms, c->grad,
                       c->prec == PAAC_BF16 ? c->theta16 : nullptr, hp.lr, hp.rms_decay, hp.rms_eps, hp.clip_norm,
                       c->norm_partials, c->stats);
+  if (c->prec == PAAC_BF16) refresh_weight_copies(c, false);
   c->N += (uint64_t)c->B;
   c->rollout_fresh = false;
   if (cuda_status(c) != PAAC_OK) return PAAC_ERR_CUDA;
@@ -255,7 +276,7 @@ int paac_set_params(paac_ctx* c, const float* src, size_t n) {
   if (cudaMemcpyAsync(c->theta, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
     cudaGetLastError(); return PAAC_ERR_CUDA;
   }
-  launch_cast_bf16(c->lc, c->theta, c->theta16, n);
+  refresh_weight_copies(c, true);
   if (cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
   return cuda_status(c);
 }

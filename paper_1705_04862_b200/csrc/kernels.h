@@ -28,6 +28,18 @@ size_t simt_scratch_floats(int arch, const NetDims& nd, int n);
 bool tc_supported(int arch, int prec);
 void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* theta16,
                 const uint8_t* frames, int n, void* const act[], uint32_t* error_word);
+// transposed / regrouped bf16 weight images the backward contractions read (refreshed after every
+// parameter change), and the data-gradient kernels that use them
+size_t tc_weight_image_elems();
+void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, bf16* images);
+void tc_backward_dgrad_fc(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err);
+void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err);
+void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err);
+// single layers of the CUDA-core backward pass (the tensor-core update mixes them in where it has no
+// kernel of its own yet)
+void simt_backward_layer(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta, const bf16* theta16,
+                         const uint8_t* frames, int n, void* const act[], void* const gact[], float* grad,
+                         float* scratch, int layer, bool wgrad, bool dgrad);
 
 // ---- heads, sampling, returns, loss gradient (heads.cu) -----------------------------------
 // logits/values of n states from the fc activation; if actions != nullptr also samples

@@ -80,26 +80,51 @@ static void forward_t(LaunchCtx& lc, int arch, const NetDims& nd, const float* t
   }
 }
 
+// one layer of the backward pass: its weight gradient and/or the data gradient handed to the layer below
 template <class T, class TW>
-static void backward_t(LaunchCtx& lc, int arch, const NetDims& nd, const TW* w, const uint8_t* frames,
-                       int n, void* const act[], void* const gact[], float* grad, float* scratch) {
+static void backward_layer_t(LaunchCtx& lc, int arch, const NetDims& nd, const TW* w, const uint8_t* frames, int n,
+                             void* const act[], void* const gact[], float* grad, float* scratch, int l, bool wg,
+                             bool dg) {
   const LayerDims* d = nd.layer;
   const float s255 = 1.0f / 255.0f;
+  const T* g = (const T*)gact[l];
+  const T* x = l > 0 ? (const T*)act[l - 1] : nullptr;
+  T* gin = l > 0 ? (T*)gact[l - 1] : nullptr;
+  float* gw = grad + d[l].w_off; float* gb = grad + d[l].b_off;
+  const TW* wl = w + d[l].w_off;
   if (arch == PAAC_ARCH_NIPS) {
-    fc_wgrad<T>(lc, KID_FC_WGRAD, (const T*)gact[2], (const T*)act[1], n, 2592, 256, grad + d[2].w_off, grad + d[2].b_off, scratch);
-    fc_dgrad<T, TW>(lc, KID_FC_DGRAD, (const T*)gact[2], w + d[2].w_off, (const T*)act[1], (T*)gact[1], n, 2592, 256);
-    conv_wgrad<NipsConv2, T, T>(lc, KID_CONV2_WGRAD, (const T*)gact[1], (const T*)act[0], n, 1.f, grad + d[1].w_off, grad + d[1].b_off, scratch);
-    conv_dgrad<NipsConv2, T, TW>(lc, KID_CONV2_DGRAD, (const T*)gact[1], w + d[1].w_off, (const T*)act[0], (T*)gact[0], n);
-    conv_wgrad<NipsConv1, uint8_t, T>(lc, KID_CONV1_WGRAD, (const T*)gact[0], frames, n, s255, grad + d[0].w_off, grad + d[0].b_off, scratch);
+    if (l == 2) {
+      if (wg) fc_wgrad<T>(lc, KID_FC_WGRAD, g, x, n, 2592, 256, gw, gb, scratch);
+      if (dg) fc_dgrad<T, TW>(lc, KID_FC_DGRAD, g, wl, x, gin, n, 2592, 256);
+    } else if (l == 1) {
+      if (wg) conv_wgrad<NipsConv2, T, T>(lc, KID_CONV2_WGRAD, g, x, n, 1.f, gw, gb, scratch);
+      if (dg) conv_dgrad<NipsConv2, T, TW>(lc, KID_CONV2_DGRAD, g, wl, x, gin, n);
+    } else if (wg) {
+      conv_wgrad<NipsConv1, uint8_t, T>(lc, KID_CONV1_WGRAD, g, frames, n, s255, gw, gb, scratch);
+    }
   } else {
-    fc_wgrad<T>(lc, KID_FC_WGRAD, (const T*)gact[3], (const T*)act[2], n, 3136, 512, grad + d[3].w_off, grad + d[3].b_off, scratch);
-    fc_dgrad<T, TW>(lc, KID_FC_DGRAD, (const T*)gact[3], w + d[3].w_off, (const T*)act[2], (T*)gact[2], n, 3136, 512);
-    conv_wgrad<NatConv3, T, T>(lc, KID_CONV3_WGRAD, (const T*)gact[2], (const T*)act[1], n, 1.f, grad + d[2].w_off, grad + d[2].b_off, scratch);
-    conv_dgrad<NatConv3, T, TW>(lc, KID_CONV3_DGRAD, (const T*)gact[2], w + d[2].w_off, (const T*)act[1], (T*)gact[1], n);
-    conv_wgrad<NatConv2, T, T>(lc, KID_CONV2_WGRAD, (const T*)gact[1], (const T*)act[0], n, 1.f, grad + d[1].w_off, grad + d[1].b_off, scratch);
-    conv_dgrad<NatConv2, T, TW>(lc, KID_CONV2_DGRAD, (const T*)gact[1], w + d[1].w_off, (const T*)act[0], (T*)gact[0], n);
-    conv_wgrad<NatConv1, uint8_t, T>(lc, KID_CONV1_WGRAD, (const T*)gact[0], frames, n, s255, grad + d[0].w_off, grad + d[0].b_off, scratch);
+    if (l == 3) {
+      if (wg) fc_wgrad<T>(lc, KID_FC_WGRAD, g, x, n, 3136, 512, gw, gb, scratch);
+      if (dg) fc_dgrad<T, TW>(lc, KID_FC_DGRAD, g, wl, x, gin, n, 3136, 512);
+    } else if (l == 2) {
+      if (wg) conv_wgrad<NatConv3, T, T>(lc, KID_CONV3_WGRAD, g, x, n, 1.f, gw, gb, scratch);
+      if (dg) conv_dgrad<NatConv3, T, TW>(lc, KID_CONV3_DGRAD, g, wl, x, gin, n);
+    } else if (l == 1) {
+      if (wg) conv_wgrad<NatConv2, T, T>(lc, KID_CONV2_WGRAD, g, x, n, 1.f, gw, gb, scratch);
+      if (dg) conv_dgrad<NatConv2, T, TW>(lc, KID_CONV2_DGRAD, g, wl, x, gin, n);
+    } else if (wg) {
+      conv_wgrad<NatConv1, uint8_t, T>(lc, KID_CONV1_WGRAD, g, frames, n, s255, gw, gb, scratch);
+    }
   }
+}
+
+void simt_backward_layer(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta, const bf16* theta16,
+                         const uint8_t* frames, int n, void* const act[], void* const gact[], float* grad,
+                         float* scratch, int layer, bool wgrad, bool dgrad) {
+  if (prec == PAAC_BF16)
+    backward_layer_t<bf16, bf16>(lc, arch, nd, theta16, frames, n, act, gact, grad, scratch, layer, wgrad, dgrad);
+  else
+    backward_layer_t<float, float>(lc, arch, nd, theta, frames, n, act, gact, grad, scratch, layer, wgrad, dgrad);
 }
 
 void simt_forward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
@@ -111,8 +136,8 @@ void simt_forward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const fl
 void simt_backward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
                    const bf16* theta16, const uint8_t* frames, int n, void* const act[], void* const gact[],
                    float* grad, float* scratch) {
-  if (prec == PAAC_BF16) backward_t<bf16, bf16>(lc, arch, nd, theta16, frames, n, act, gact, grad, scratch);
-  else backward_t<float, float>(lc, arch, nd, theta, frames, n, act, gact, grad, scratch);
+  for (int l = nd.n_conv; l >= 0; --l)
+    simt_backward_layer(lc, arch, prec, nd, theta, theta16, frames, n, act, gact, grad, scratch, l, true, l > 0);
 }
 
 size_t simt_scratch_floats(int arch, const NetDims& nd, int n) {

@@ -121,6 +121,95 @@ struct BiasReluEpiTc {
   }
 };
 
+// ---- data-gradient sources: rows of the layer INPUT, k = (tap, co) -------------------------------------
+// stride-1 convolution with CO = 64: K block kb is tap (r, s); the row for input pixel (y, x) is the
+// 64 output-channel gradients of window (y - r, x - s), or zeros where that window does not exist.
+template <class G> struct DgradSrcS1 {
+  const bf16* g; int M;
+  __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
+    static_assert(G::S == 1 && G::CO == 64, "one tap per K block");
+    m = min(m, M - 1);
+    const int b = m / (G::H * G::W), rem = m % (G::H * G::W), y = rem / G::W, x = rem % G::W;
+    const int oh = y - kb / G::K, ow = x - kb % G::K;
+    if (oh < 0 || oh >= G::OH || ow < 0 || ow >= G::OW) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = make_uint4(0u, 0u, 0u, 0u);
+      return;
+    }
+    const uint4* p = reinterpret_cast<const uint4*>(g + ((size_t)(b * G::OH + oh) * G::OW + ow) * G::CO);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __ldg(p + i);
+  }
+};
+// stride-2, 4x4 kernel, CO = 64.  Input pixels are split into four parity classes z = (y&1, x&1); a
+// pixel of class z is touched only by the four taps (r, s) = (py + 2i, px + 2j), so each class is its
+// own dense contraction with K = 4 taps x 64 and no structural zeros.  Row m = (state, y>>1, x>>1).
+template <class G> struct DgradSrcS2 {
+  const bf16* g; int M;
+  __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
+    static_assert(G::S == 2 && G::K == 4 && G::CO == 64 && G::H % 2 == 0 && G::W % 2 == 0, "parity split");
+    constexpr int HH = G::H / 2, WW = G::W / 2;
+    m = min(m, M - 1);
+    const int b = m / (HH * WW), rem = m % (HH * WW), yy = rem / WW, xx = rem % WW;
+    const int oh = yy - (kb >> 1), ow = xx - (kb & 1);
+    if (oh < 0 || oh >= G::OH || ow < 0 || ow >= G::OW) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = make_uint4(0u, 0u, 0u, 0u);
+      return;
+    }
+    const uint4* p = reinterpret_cast<const uint4*>(g + ((size_t)(b * G::OH + oh) * G::OW + ow) * G::CO);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __ldg(p + i);
+  }
+};
+// per-class K-major weights w[z][n][k]
+struct ClassWeightSrc {
+  const bf16* w; int ld; int class_stride;
+  __device__ __forceinline__ void load(int n, int kb, int z, uint4 (&v)[8]) const {
+    const uint4* p = reinterpret_cast<const uint4*>(w + (size_t)z * class_stride + (size_t)n * ld + kb * TC_BK);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __ldg(p + i);
+  }
+};
+
+// out[m][n] = act[m][n] > 0 ? bf16(acc) : 0     (gradient through the ReLU of the layer below)
+__device__ __forceinline__ void relu_mask_store(bf16* out, const bf16* act, size_t idx, const uint32_t (&r)[32]) {
+  const uint4* a4 = reinterpret_cast<const uint4*>(act + idx);
+  uint4* dst = reinterpret_cast<uint4*>(out + idx);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint4 a = __ldg(a4 + j);
+    const uint32_t aw[4] = {a.x, a.y, a.z, a.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      // stored activations are >= 0, so "positive" is "non-zero bit pattern other than -0"
+      const float lo = (aw[q] & 0x7FFFu) ? __uint_as_float(r[8 * j + 2 * q]) : 0.f;
+      const float hi = (aw[q] & 0x7FFF0000u) ? __uint_as_float(r[8 * j + 2 * q + 1]) : 0.f;
+      o[q] = pack_bf16x2(lo, hi);
+    }
+    dst[j] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+struct ReluMaskEpiTc {
+  bf16* out; const bf16* act; int ld; int M;
+  __device__ __forceinline__ void operator()(int m, int n0, int, const uint32_t (&r)[32]) const {
+    if (m >= M) return;
+    relu_mask_store(out, act, (size_t)m * ld + n0, r);
+  }
+};
+// same, scattering parity class z of a stride-2 layer back to its input pixels
+template <class G> struct ReluMaskEpiS2 {
+  bf16* out; const bf16* act; int M;
+  __device__ __forceinline__ void operator()(int m, int n0, int z, const uint32_t (&r)[32]) const {
+    if (m >= M) return;
+    constexpr int HH = G::H / 2, WW = G::W / 2;
+    const int b = m / (HH * WW), rem = m % (HH * WW), yy = rem / WW, xx = rem % WW;
+    const int y = 2 * yy + (z >> 1), x = 2 * xx + (z & 1);
+    relu_mask_store(out, act, ((size_t)(b * G::H + y) * G::W + x) * G::C + n0, r);
+  }
+};
+
 // ---- the kernel ----------------------------------------------------------------------------------------
 template <class ASrc, class BSrc, class Epi, int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS)
@@ -247,6 +336,59 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
         lc, KID_FC_FWD, PlainSrc{(const bf16*)act[2], 3136, n}, WeightSrc{w + d[3].w_off, 3136},
         BiasReluEpiTc{(bf16*)act[3], theta + d[3].b_off, 512, 1.f, n}, n, 512, 3136 / 64, 1, err);
   }
+}
+
+// ---- weight images for the backward contractions ------------------------------------------------------
+// From the canonical bf16 copy: wfc_t[i][o] = Wfc[o][i];  w3_d[ci][r][s][co] = W3[co][r][s][ci];
+// w2_d[z][ci][i][j][co] = W2[co][py + 2i][px + 2j][ci] with z = 2 py + px.
+__global__ void relayout_weights_kernel(const bf16* __restrict__ w2, const bf16* __restrict__ w3,
+                                        const bf16* __restrict__ wfc, bf16* __restrict__ w2_d,
+                                        bf16* __restrict__ w3_d, bf16* __restrict__ wfc_t) {
+  typedef NatConv2 C2; typedef NatConv3 C3;
+  constexpr int N2 = 4 * C2::C * 4 * C2::CO, N3 = C3::C * 9 * C3::CO, NF = 3136 * 512;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N2 + N3 + NF; i += gridDim.x * blockDim.x) {
+    if (i < N2) {
+      const int co = i % 64, t = (i / 64) % 4, ci = (i / 256) % 32, z = i / (256 * 32);
+      const int r = (z >> 1) + 2 * (t >> 1), s = (z & 1) + 2 * (t & 1);
+      w2_d[i] = w2[((co * 4 + r) * 4 + s) * 32 + ci];
+    } else if (i < N2 + N3) {
+      const int j = i - N2, co = j % 64, tap = (j / 64) % 9, ci = j / 576;
+      w3_d[j] = w3[(co * 9 + tap) * 64 + ci];
+    } else {
+      const int j = i - N2 - N3, o = j % 512, in = j / 512;
+      wfc_t[j] = wfc[(size_t)o * 3136 + in];
+    }
+  }
+}
+size_t tc_weight_image_elems() { return 4 * 32 * 256 + 64 * 576 + (size_t)3136 * 512; }
+
+void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, bf16* images) {
+  const LayerDims* d = nd.layer;
+  KernelScope scope(lc, KID_CAST);
+  relayout_weights_kernel<<<592, 256, 0, lc.st>>>(theta16 + d[1].w_off, theta16 + d[2].w_off, theta16 + d[3].w_off,
+                                                  images, images + 4 * 32 * 256, images + 4 * 32 * 256 + 64 * 576);
+}
+
+// ---- backward: data gradients ---------------------------------------------------------------------------
+void tc_backward_dgrad_fc(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
+  const bf16* wfc_t = images + 4 * 32 * 256 + 64 * 576;
+  tc_gemm<PlainSrc, WeightSrc, ReluMaskEpiTc, 64, 4>(
+      lc, KID_FC_DGRAD, PlainSrc{(const bf16*)gact[3], 512, n}, WeightSrc{wfc_t, 512},
+      ReluMaskEpiTc{(bf16*)gact[2], (const bf16*)act[2], 3136, n}, n, 3136, 512 / 64, 1, err);
+}
+void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
+  typedef NatConv3 C3;
+  const int M = n * C3::H * C3::W;
+  tc_gemm<DgradSrcS1<C3>, WeightSrc, ReluMaskEpiTc, 64, 4>(
+      lc, KID_CONV3_DGRAD, DgradSrcS1<C3>{(const bf16*)gact[2], M}, WeightSrc{images + 4 * 32 * 256, 576},
+      ReluMaskEpiTc{(bf16*)gact[1], (const bf16*)act[1], 64, M}, M, 64, 9, 1, err);
+}
+void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
+  typedef NatConv2 C2;
+  const int M = n * (C2::H / 2) * (C2::W / 2);
+  tc_gemm<DgradSrcS2<C2>, ClassWeightSrc, ReluMaskEpiS2<C2>, 32, 4>(
+      lc, KID_CONV2_DGRAD, DgradSrcS2<C2>{(const bf16*)gact[1], M}, ClassWeightSrc{images, 256, 32 * 256},
+      ReluMaskEpiS2<C2>{(bf16*)gact[0], (const bf16*)act[0], M}, M, 32, 4, 4, err);
 }
 
 }  // namespace paac
