@@ -191,8 +191,10 @@ int paac_debug_read(paac_ctx* ctx, int which, void* dst /* host */, size_t bytes
 int paac_debug_write(paac_ctx* ctx, int which, const void* src /* host */, size_t bytes);
 
 /* Run-time options.  PAAC_OPT_CUDA_CORES_ONLY != 0 keeps the bf16 network off the tensor cores
- * (same rounding points, CUDA-core contractions): a second implementation to compare against. */
-enum { PAAC_OPT_CUDA_CORES_ONLY = 1 };
+ * (same rounding points, CUDA-core contractions): a second implementation to compare against.
+ * PAAC_OPT_TC_WGRAD_LAYERS: bit mask (bit l = layer l, conv1 = 0) of the layers whose weight gradient
+ * runs on the tensor cores; the others use the CUDA-core contraction.  Default: all. */
+enum { PAAC_OPT_CUDA_CORES_ONLY = 1, PAAC_OPT_TC_WGRAD_LAYERS = 2 };
 int paac_set_option(paac_ctx* ctx, int option, int value);
 
 /* Number of kernels the library has launched on this context since init. */

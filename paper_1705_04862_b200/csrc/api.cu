@@ -23,6 +23,7 @@ struct paac_ctx {
   bool rollout_fresh;      // a rollout has completed since the last update
   int host_t;              // external-environment mode: next expected step
   bool forced_on;
+  int tc_wgrad_mask;       // bit l: layer l's weight gradient runs on the tensor cores
   bool simt_only;          // keep the bf16 network on the CUDA cores (cross-check of the tensor-core path)
 
   // device buffers (all inside the workspace)
@@ -88,7 +89,11 @@ size_t carve(paac_ctx* c, char* base) {
   c->dz = k.take<float>(B * A);
   c->dV = k.take<float>(B);
   c->loss_terms = k.take<float>(3 * B);
-  c->scratch = k.take<float>(simt_scratch_floats(c->arch, nd, (int)B));
+  {
+    size_t sc = simt_scratch_floats(c->arch, nd, (int)B);
+    if (tc_supported(c->arch, c->prec) && tc_scratch_floats((int)B) > sc) sc = tc_scratch_floats((int)B);
+    c->scratch = k.take<float>(sc);
+  }
   c->norm_partials = k.take<float>(NORM_BLOCKS);
   c->actions = k.take<int32_t>(B);
   c->sampled = k.take<int32_t>(B);
@@ -162,6 +167,7 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   paac_ctx* c = new (std::nothrow) paac_ctx{};
   if (!c) return PAAC_ERR_CUDA;
   fill_shape(c, arch, n_e, t_max, n_actions, hp);
+  c->tc_wgrad_mask = 0xF;
   c->seed = seed; c->device = dev; c->st = (cudaStream_t)hp->stream; c->lc.st = c->st;
   const size_t need = carve(c, nullptr);
   if (hp->workspace) {
@@ -231,8 +237,14 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
       if (l == 2) { tc_backward_dgrad_conv3(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
       if (l == 1) { tc_backward_dgrad_conv2(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
     }
-    simt_backward_layer(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act, c->gact,
-                        c->grad, c->scratch, l, true, l > 0 && !dgrad_done);
+    bool wgrad_done = false;
+    if (use_tc(c) && (c->tc_wgrad_mask >> l) & 1) {
+      tc_backward_wgrad(c->lc, c->nd, c->frames[c->cur], c->B, c->act, c->gact, c->grad, c->scratch, l, err);
+      wgrad_done = true;
+    }
+    if (!wgrad_done || (l > 0 && !dgrad_done))
+      simt_backward_layer(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
+                          c->gact, c->grad, c->scratch, l, !wgrad_done, l > 0 && !dgrad_done);
   }
   launch_clip_rmsprop(c->lc, c->nd.P, c->theta, c->rms, c->grad,
                       c->prec == PAAC_BF16 ? c->theta16 : nullptr, hp.lr, hp.rms_decay, hp.rms_eps, hp.clip_norm,
@@ -320,6 +332,7 @@ uint64_t paac_launch_count(const paac_ctx* c) { return c ? c->lc.count : 0; }
 int paac_set_option(paac_ctx* c, int option, int value) {
   if (!c) return PAAC_ERR_ARG;
   if (option == PAAC_OPT_CUDA_CORES_ONLY) { c->simt_only = value != 0; return PAAC_OK; }
+  if (option == PAAC_OPT_TC_WGRAD_LAYERS) { c->tc_wgrad_mask = value & 0xF; return PAAC_OK; }
   return PAAC_ERR_ARG;
 }
 

@@ -127,14 +127,14 @@ inline NetDims make_net(int arch, int A) {
 enum KernelId {
   KID_INIT = 0, KID_ENV_STEP, KID_CONV1_FWD, KID_CONV2_FWD, KID_CONV3_FWD, KID_FC_FWD, KID_HEADS_FWD,
   KID_RETURNS, KID_HEAD_GRAD, KID_HEADS_BWD, KID_FC_WGRAD, KID_FC_DGRAD, KID_CONV3_WGRAD, KID_CONV3_DGRAD,
-  KID_CONV2_WGRAD, KID_CONV2_DGRAD, KID_CONV1_WGRAD, KID_WGRAD_REDUCE, KID_SUMSQ, KID_CLIP_RMSPROP, KID_CAST,
+  KID_CONV2_WGRAD, KID_CONV2_DGRAD, KID_CONV1_WGRAD, KID_WGRAD_REDUCE, KID_SUMSQ, KID_CLIP_RMSPROP, KID_CAST, KID_BIAS_GRAD,
   KID_COUNT
 };
 inline const char* kernel_name(int id) {
   static const char* names[KID_COUNT] = {
       "init_params", "env_step", "conv1_fwd", "conv2_fwd", "conv3_fwd", "fc_fwd", "heads_fwd_sample", "returns",
       "head_grad", "heads_bwd", "fc_wgrad", "fc_dgrad", "conv3_wgrad", "conv3_dgrad", "conv2_wgrad", "conv2_dgrad",
-      "conv1_wgrad", "wgrad_reduce", "grad_sumsq", "clip_rmsprop", "cast_bf16"};
+      "conv1_wgrad", "wgrad_reduce", "grad_sumsq", "clip_rmsprop", "cast_bf16", "bias_grad"};
   return id >= 0 && id < KID_COUNT ? names[id] : "?";
 }
 

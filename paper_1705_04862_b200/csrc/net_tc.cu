@@ -338,6 +338,277 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
   }
 }
 
+// ---- weight gradients ------------------------------------------------------------------------------------
+// dW^T[j][co] = sum_m X[m][j] * G[m][co]: the reduction runs over the rows m = (state, oh, ow), so both
+// operands are "MN-major": a shared-memory row holds 64 consecutive j (or co) of ONE m, exactly the 128
+// bytes the forward sources deliver (an atom = K block of the forward pass).  Image of one stage (64 rows
+// of m): atom column a -> 8 groups of 8 rows -> 128-byte swizzled rows; leading (atom-column) stride 8 KB,
+// stride between 8-row groups 1 KB; a K=16 MMA step covers two groups.
+// A CTA owns JT row tiles of 128 j each and a contiguous range of 64-row blocks of m (split-k); it writes
+// its float partial tile to scratch, and a second kernel adds the partials in a fixed order.
+constexpr int WG_ROWS = 64;
+
+// G rows: BN (64 or 128) bf16 starting at column n0; rows past M read as zero so that the tail of the last
+// block adds nothing.  VALID < 64 pads a narrower matrix (conv1: 32 channels) with zero columns.
+template <int VALID> struct GradSrc {
+  const bf16* g; int ld; int M;
+  __device__ __forceinline__ void load(int m, int n0, uint4 (&v)[8]) const {
+    if (m >= M) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = make_uint4(0u, 0u, 0u, 0u);
+      return;
+    }
+    const uint4* p = reinterpret_cast<const uint4*>(g + (size_t)m * ld + n0);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = i < VALID / 8 ? __ldg(p + i) : make_uint4(0u, 0u, 0u, 0u);
+  }
+};
+
+template <class XSrc, class GSrc, int JT, int BN, int STAGES>
+__global__ void __launch_bounds__(TC_THREADS)
+tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, int n_atoms, int J, int CO, int num_blocks,
+                int blocks_per_split, uint32_t* error_word) {
+  static_assert(BN == 64 || BN == 128, "tile width");
+  static_assert(JT == 1 || JT == 2, "row tiles per CTA");
+  constexpr uint32_t ATOM_COL = WG_ROWS * 128;                      // 8 KB: one atom column of a stage
+  constexpr uint32_t A_BYTES = 2 * JT * ATOM_COL, B_BYTES = (BN / 64) * ATOM_COL, STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int A_PER_HALF = JT, B_COLS = BN / 64;
+  extern __shared__ uint8_t dyn_smem[];
+  __shared__ TcShared sh;
+  const uint32_t tiles = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, atom0 = blockIdx.y * 2 * JT, n0 = blockIdx.z * BN;
+  const int kb0 = split * blocks_per_split, kb1 = min(num_blocks, kb0 + blocks_per_split);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    mbar_init(&sh.acc, 1);
+    sh.abort = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 4) tmem_alloc(&sh.tmem_base, JT * BN);
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp < 4) {
+    // ---------------- producers: thread = (row of the block, half) ----------------
+    const int row = threadIdx.x & 63, half = threadIdx.x >> 6;
+    const uint32_t row_off = (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u;
+    for (int kb = kb0; kb < kb1; ++kb) {
+      const int it = kb - kb0, s = it % STAGES;
+      const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const uint32_t a_base = tiles + s * STAGE_BYTES, b_base = a_base + A_BYTES;
+      const int m = kb * WG_ROWS + row;
+      uint4 v[8];
+#pragma unroll
+      for (int q = 0; q < A_PER_HALF; ++q) {
+        const int col = half * A_PER_HALF + q;                      // atom column inside the stage
+        const int atom = atom0 + col;
+        if (atom < n_atoms) x_src.load(m, atom, 0, v);
+        else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_base + col * ATOM_COL + row_off +
+                       ((uint32_t)(c ^ (row & 7)) << 4)), "r"(v[c].x), "r"(v[c].y), "r"(v[c].z), "r"(v[c].w) : "memory");
+      }
+      if (half < B_COLS) {
+        g_src.load(m, n0 + half * 64, v);
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_base + half * ATOM_COL + row_off +
+                       ((uint32_t)(c ^ (row & 7)) << 4)), "r"(v[c].x), "r"(v[c].y), "r"(v[c].z), "r"(v[c].w) : "memory");
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.full[s]);
+    }
+    // ---------------- epilogue: float partial tile to scratch ----------------
+    if (kb1 > kb0 && mbar_wait(&sh.acc, 0, &sh.abort, error_word, ERR_WAIT_ACC)) {
+      tcgen05_fence_after();
+#pragma unroll 1
+      for (int jt = 0; jt < JT; ++jt) {
+        const int j = (atom0 / 2 + jt) * 128 + threadIdx.x;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + jt * BN + c * 32, r);
+          if (j < J && n0 + c * 32 < CO) {
+            float4* dst = reinterpret_cast<float4*>(partial + ((size_t)split * J + j) * CO + n0 + c * 32);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                   __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+          }
+        }
+      }
+    }
+  } else if (lane == 0) {
+    // ---------------- MMA issuer ----------------
+    constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 1, 1);
+    bool ok = true;
+    for (int kb = kb0; kb < kb1 && ok; ++kb) {
+      const int it = kb - kb0, s = it % STAGES;
+      ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      if (!ok) break;
+      tcgen05_fence_after();
+      const uint32_t a_base = tiles + s * STAGE_BYTES, b_base = a_base + A_BYTES;
+#pragma unroll
+      for (int jt = 0; jt < JT; ++jt) {
+#pragma unroll
+        for (int t = 0; t < WG_ROWS / 16; ++t) {
+          const uint64_t ad = make_smem_desc(a_base + jt * 2 * ATOM_COL + t * 2048, ATOM_COL, 1024, SWIZZLE_128B);
+          const uint64_t bd = make_smem_desc(b_base + t * 2048, ATOM_COL, 1024, SWIZZLE_128B);
+          mma_bf16(tmem + jt * BN, ad, bd, idesc, (it | t) != 0 ? 1u : 0u);
+        }
+      }
+      mma_commit(&sh.empty[s]);
+    }
+    if (ok && kb1 > kb0) mma_commit(&sh.acc);
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    __syncwarp();
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, JT * BN);
+  }
+}
+
+// dW[co][j] = scale * sum over splits of partial[split][j][co]   (fixed order)
+__global__ void tc_wgrad_reduce_kernel(const float* __restrict__ partial, int splits, int J, int CO, float scale,
+                                       float* __restrict__ gw) {
+  const int total = J * CO;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    float s = 0.f;
+    for (int p = 0; p < splits; ++p) s += partial[(size_t)p * total + i];
+    const int j = i / CO, co = i % CO;
+    gw[(size_t)co * J + j] = s * scale;
+  }
+}
+
+// bias gradient: column sums of G[rows][CO]; block b adds its slice of rows in a fixed order, then the
+// last stage adds the per-block results in block order
+template <int CO>
+__global__ void __launch_bounds__(256) tc_bias_partial_kernel(const bf16* __restrict__ g, int rows, float* __restrict__ part) {
+  constexpr int TPR = CO / 8, RPB = 256 / TPR;          // threads per row (8 channels each), rows per pass
+  __shared__ float sh[256][9];
+  const int c8 = threadIdx.x % TPR, r0 = threadIdx.x / TPR;
+  const int per = (rows + gridDim.x - 1) / gridDim.x;
+  const int lo = blockIdx.x * per, hi = min(rows, lo + per);
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  for (int r = lo + r0; r < hi; r += RPB) {
+    const uint4 q = __ldg(reinterpret_cast<const uint4*>(g + (size_t)r * CO) + c8);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      acc[2 * i] += __uint_as_float(w[i] << 16);
+      acc[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) sh[threadIdx.x][i] = acc[i];
+  __syncthreads();
+  for (int c = threadIdx.x; c < CO; c += 256) {
+    float s = 0.f;
+    for (int r = 0; r < RPB; ++r) s += sh[r * TPR + c / 8][c % 8];
+    part[(size_t)blockIdx.x * CO + c] = s;
+  }
+}
+__global__ void tc_bias_final_kernel(const float* __restrict__ part, int blocks, int CO, float* __restrict__ gb) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= CO) return;
+  float s = 0.f;
+  for (int b = 0; b < blocks; ++b) s += part[(size_t)b * CO + c];
+  gb[c] = s;
+}
+
+constexpr int WG_BIAS_BLOCKS = 296;
+static int wg_splits(int num_blocks, int tiles_yz) {
+  int s = (296 + tiles_yz - 1) / tiles_yz;           // about two CTAs per SM in total
+  if (s > num_blocks) s = num_blocks;
+  if (s < 1) s = 1;
+  return s;
+}
+static size_t wg_scratch_floats(int rows, int J, int CO, int tiles_yz) {
+  const int num_blocks = (rows + WG_ROWS - 1) / WG_ROWS;
+  const int bps = (num_blocks + wg_splits(num_blocks, tiles_yz) - 1) / wg_splits(num_blocks, tiles_yz);
+  const int splits = (num_blocks + bps - 1) / bps;
+  return (size_t)splits * J * CO + (size_t)WG_BIAS_BLOCKS * CO;
+}
+
+template <class XSrc, class GSrc, int JT, int BN, int STAGES, int CO>
+static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, const bf16* g, int rows, int n_atoms, float scale,
+                     float* gw, float* gb, float* scratch, uint32_t* err) {
+  constexpr int smem = STAGES * ((2 * JT + BN / 64) * WG_ROWS * 128) + 1024;
+  auto kern = tc_wgrad_kernel<XSrc, GSrc, JT, BN, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  const int J = n_atoms * 64;
+  const int gy = (n_atoms + 2 * JT - 1) / (2 * JT), gz = (CO + BN - 1) / BN;
+  const int num_blocks = (rows + WG_ROWS - 1) / WG_ROWS;
+  const int bps = (num_blocks + wg_splits(num_blocks, gy * gz) - 1) / wg_splits(num_blocks, gy * gz);
+  const int splits = (num_blocks + bps - 1) / bps;
+  float* bias_part = scratch + (size_t)splits * J * CO;
+  {
+    KernelScope scope(lc, kid);
+    kern<<<dim3(splits, gy, gz), TC_THREADS, smem, lc.st>>>(xs, gs, scratch, n_atoms, J, CO, num_blocks, bps, err);
+  }
+  {
+    KernelScope scope(lc, KID_WGRAD_REDUCE);
+    tc_wgrad_reduce_kernel<<<(J * CO + 255) / 256, 256, 0, lc.st>>>(scratch, splits, J, CO, scale, gw);
+  }
+  {
+    KernelScope scope(lc, KID_BIAS_GRAD);
+    tc_bias_partial_kernel<CO><<<WG_BIAS_BLOCKS, 256, 0, lc.st>>>(g, rows, bias_part);
+  }
+  KernelScope scope(lc, KID_BIAS_GRAD);
+  tc_bias_final_kernel<<<(CO + 127) / 128, 128, 0, lc.st>>>(bias_part, WG_BIAS_BLOCKS, CO, gb);
+}
+
+size_t tc_scratch_floats(int n) {
+  size_t best = wg_scratch_floats(n * 400, 256, 32, 1);
+  size_t v = wg_scratch_floats(n * 81, 512, 64, 2); if (v > best) best = v;
+  v = wg_scratch_floats(n * 49, 576, 64, 3); if (v > best) best = v;
+  v = wg_scratch_floats(n, 3136, 512, 25 * 4); if (v > best) best = v;
+  return best;
+}
+
+void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, int n, void* const act[],
+                       void* const gact[], float* grad, float* scratch, int layer, uint32_t* err) {
+  const LayerDims* d = nd.layer;
+  float* gw = grad + d[layer].w_off; float* gb = grad + d[layer].b_off;
+  const bf16* g = (const bf16*)gact[layer];
+  if (layer == 0) {
+    typedef NatConv1 C1;
+    const int rows = n * C1::OH * C1::OW;
+    tc_wgrad<FrameSrc<C1>, GradSrc<32>, 2, 64, 3, 32>(lc, KID_CONV1_WGRAD, FrameSrc<C1>{frames, rows},
+                                                      GradSrc<32>{g, 32, rows}, g, rows, 4, 1.0f / 255.0f, gw, gb,
+                                                      scratch, err);
+  } else if (layer == 1) {
+    typedef NatConv2 C2;
+    const int rows = n * C2::OH * C2::OW;
+    tc_wgrad<ConvSrc<C2>, GradSrc<64>, 2, 64, 3, 64>(lc, KID_CONV2_WGRAD, ConvSrc<C2>{(const bf16*)act[0], rows},
+                                                     GradSrc<64>{g, 64, rows}, g, rows, 8, 1.f, gw, gb, scratch, err);
+  } else if (layer == 2) {
+    typedef NatConv3 C3;
+    const int rows = n * C3::OH * C3::OW;
+    tc_wgrad<ConvSrc<C3>, GradSrc<64>, 2, 64, 3, 64>(lc, KID_CONV3_WGRAD, ConvSrc<C3>{(const bf16*)act[1], rows},
+                                                     GradSrc<64>{g, 64, rows}, g, rows, 9, 1.f, gw, gb, scratch, err);
+  } else {
+    tc_wgrad<PlainSrc, GradSrc<64>, 1, 128, 4, 512>(lc, KID_FC_WGRAD, PlainSrc{(const bf16*)act[2], 3136, n},
+                                                    GradSrc<64>{g, 512, n}, g, n, 49, 1.f, gw, gb, scratch, err);
+  }
+}
+
 // ---- weight images for the backward contractions ------------------------------------------------------
 // From the canonical bf16 copy: wfc_t[i][o] = Wfc[o][i];  w3_d[ci][r][s][co] = W3[co][r][s][ci];
 // w2_d[z][ci][i][j][co] = W2[co][py + 2i][px + 2j][ci] with z = 2 py + px.
