@@ -51,7 +51,8 @@ enum {
   PAAC_ERR_CUDA = 3,       /* a CUDA call failed (no device, launch error, ...) */
   PAAC_ERR_NONFINITE = 4,  /* gradient norm was inf/nan: the update was skipped */
   PAAC_ERR_TIMEOUT = 5,    /* a bounded device-side wait gave up */
-  PAAC_ERR_STATE = 6       /* call out of order (update without a fresh rollout, ...) */
+  PAAC_ERR_STATE = 6,      /* call out of order (update without a fresh rollout, ...) */
+  PAAC_ERR_LIMIT = 7       /* size beyond the fixed capacity of an entry point that cannot allocate */
 };
 
 /* Hyper-parameters.  paac_default_hparams() fills in the values of Section 5.1:
@@ -210,6 +211,35 @@ int paac_profile(paac_ctx* ctx, int enable);
  * max_entries.  Returns the number of entries written, or -1 on bad arguments.  Synchronises. */
 int paac_profile_read(paac_ctx* ctx, int max_entries, const char** names /* out */, double* ms /* out */,
                       uint64_t* launches /* out */);
+
+/* ---- for callers that may not allocate device memory ----
+ *
+ * (The paper has no counterpart to this entry point; it exists for deployment constraints.)
+ * Some hosts of this library cannot call cudaMalloc at all: a control loop with a frozen memory budget, a
+ * process whose device pool belongs to another framework and is fully handed out, a sandbox that only
+ * lets pre-built modules touch the GPU.  For them the optimiser step of Algorithm 1 -- global L2-norm
+ * clipping followed by RMSProp, as in paac_update -- is offered on plain caller-owned arrays, with the
+ * per-slice partial sums of the squared gradient kept in a 16 KB array that is part of the library's
+ * device image (each GPU that loads the library holds it until the process exits).  The call allocates
+ * and frees nothing, neither through CUDA nor through any library.
+ *
+ *   theta, rms   device float[n], updated in place      grad   device float[n], read only
+ *   theta_bf16   device, nullable: bfloat16 bits of the new theta, [n]
+ *   norm_and_scale  device float[2], nullable: gradient norm before clipping, factor applied (0 when
+ *                   the norm was not finite and nothing was changed)
+ *   stream       cudaStream_t; the two kernels are enqueued on it, the call does not synchronise
+ *
+ * n may not exceed paac_noalloc_max_params() (16,777,216): beyond that the call returns PAAC_ERR_LIMIT
+ * and does nothing.  The first call on each device looks up the device address of the built-in array
+ * (cudaGetSymbolAddress) with that device current; make that first call outside any stream capture.
+ * All calls on one device share the array, which keeps the last call's sums: every call rewrites the
+ * entries it reads before reading them, so nothing has to be cleared, but two calls that overlap on
+ * the GPU (on different streams) race on it -- keep them on one stream or order them with events. */
+int paac_clip_rmsprop_noalloc(float* theta /* device */, float* rms /* device */, const float* grad /* device */,
+                              uint16_t* theta_bf16 /* device, nullable */, size_t n, float lr, float rms_decay,
+                              float rms_eps, float clip_norm, float* norm_and_scale /* device, nullable */,
+                              void* stream);
+size_t paac_noalloc_max_params(void);
 
 #ifdef __cplusplus
 }

@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libpaac_b200.so")
 
 ARCH_NIPS, ARCH_NATURE = 0, 1
 FP32, BF16 = 0, 1
-OK, ERR_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_STATE = range(7)
+OK, ERR_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_STATE, ERR_LIMIT = range(8)
 (DBG_FRAMES, DBG_NEXT_FRAMES, DBG_ACTIONS, DBG_REWARDS, DBG_TERMINALS, DBG_VALUES, DBG_LOGITS, DBG_UNIFORMS,
  DBG_COUNTERS, DBG_RETURNS, DBG_ADVANTAGES, DBG_DLOGITS, DBG_DVALUES, DBG_GRAD, DBG_RMS, DBG_SAMPLED) = range(16)
 DBG_ACT0, DBG_GACT0 = 32, 48
@@ -46,7 +46,8 @@ class UpdateStats(C.Structure):
 EXPORTS = ["paac_default_hparams", "paac_workspace_bytes", "paac_init", "paac_rollout", "paac_update",
            "paac_param_count", "paac_params", "paac_destroy", "paac_strerror", "paac_act_host",
            "paac_observe_host", "paac_set_params", "paac_force_actions", "paac_debug_bytes", "paac_debug_read",
-           "paac_debug_write", "paac_launch_count", "paac_profile", "paac_profile_read", "paac_set_option"]
+           "paac_debug_write", "paac_launch_count", "paac_profile", "paac_profile_read", "paac_set_option", "paac_clip_rmsprop_noalloc",
+           "paac_noalloc_max_params"]
 
 _lib = None
 
@@ -85,6 +86,10 @@ def lib():
         L.paac_launch_count.restype = u64
         L.paac_profile.argtypes = [vp, i]
         L.paac_set_option.argtypes = [vp, i, i]
+        f = C.c_float
+        L.paac_clip_rmsprop_noalloc.argtypes = [vp, vp, vp, vp, sz, f, f, f, f, vp, vp]
+        L.paac_noalloc_max_params.argtypes = []
+        L.paac_noalloc_max_params.restype = sz
         L.paac_profile_read.argtypes = [vp, i, C.POINTER(C.c_char_p), C.POINTER(C.c_double), C.POINTER(u64)]
         _lib = L
     return _lib
@@ -120,6 +125,17 @@ def _host_ptr(a):
         assert a.flags["C_CONTIGUOUS"]
         return a.ctypes.data
     return a.data_ptr()
+
+
+def clip_rmsprop_noalloc(theta, rms, grad, n, lr, rms_decay, rms_eps, clip_norm, theta_bf16=None,
+                         norm_and_scale=None, stream=None):
+    """Optimiser step on caller-owned device arrays for hosts that may not allocate device memory (see
+    paac_clip_rmsprop_noalloc in include/paac.h).  Arguments are torch CUDA tensors (or raw device
+    addresses); returns the library status without raising, so callers can test for ERR_LIMIT."""
+    def addr(x):
+        return None if x is None else (x if isinstance(x, int) else x.data_ptr())
+    return int(lib().paac_clip_rmsprop_noalloc(addr(theta), addr(rms), addr(grad), addr(theta_bf16), n, lr, rms_decay,
+                                               rms_eps, clip_norm, addr(norm_and_scale), addr(stream)))
 
 
 class Paac:

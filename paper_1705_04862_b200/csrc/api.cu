@@ -323,6 +323,7 @@ const char* paac_strerror(int s) {
     case PAAC_ERR_NONFINITE: return "gradient norm not finite: update skipped";
     case PAAC_ERR_TIMEOUT: return "a bounded device-side wait gave up";
     case PAAC_ERR_STATE: return "call out of order";
+    case PAAC_ERR_LIMIT: return "size beyond the fixed capacity of a non-allocating entry point";
     default: return "unknown status";
   }
 }

@@ -56,8 +56,8 @@ def test_null_handles_and_strerror():
     assert L.paac_update(None, None) == pb.ERR_ARG
     assert L.paac_destroy(None) == pb.ERR_ARG
     assert L.paac_param_count(None) == 0 and L.paac_debug_bytes(None, 0) == 0
-    names = {L.paac_strerror(i) for i in range(7)}
-    assert len(names) == 7 and L.paac_strerror(99) == b"unknown status"
+    names = {L.paac_strerror(i) for i in range(8)}
+    assert len(names) == 8 and L.paac_strerror(99) == b"unknown status"
 
 
 def test_init_fails_loudly_without_a_gpu():
