@@ -31,7 +31,13 @@ struct TcShared {
 // ---- A-operand sources: 64 bf16 (128 bytes) of row m for K block kb ---------------------------
 // plain row-major matrix x[m][k]
 struct PlainSrc {
+  static constexpr bool ASYNC = true;
   const bf16* x; int ld; int M;
+  // address of the 128 bytes; valid = false means "this row reads as zeros"
+  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const {
+    valid = true;
+    return x + (size_t)min(m, M - 1) * ld + kb * TC_BK;
+  }
   __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
     m = min(m, M - 1);
     const uint4* p = reinterpret_cast<const uint4*>(x + (size_t)m * ld + kb * TC_BK);
@@ -41,7 +47,15 @@ struct PlainSrc {
 };
 // convolution window over a bf16 NHWC tensor; k = (r, s, ci); a K block holds 64 / C taps of one kernel row
 template <class G> struct ConvSrc {
+  static constexpr bool ASYNC = true;
   const bf16* x; int M;
+  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const {
+    valid = true;
+    m = min(m, M - 1);
+    const int b = m / (G::OH * G::OW), rem = m % (G::OH * G::OW), oh = rem / G::OW, ow = rem % G::OW;
+    const int tap = kb * (64 / G::C), r = tap / G::K, s = tap % G::K;
+    return x + ((size_t)(b * G::H + oh * G::S + r) * G::W + (ow * G::S + s)) * G::C;
+  }
   __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
     static_assert(64 % G::C == 0 && G::K % (64 / G::C) == 0, "a K block must stay inside one kernel row");
     m = min(m, M - 1);
@@ -71,6 +85,7 @@ __device__ __forceinline__ void u8x16_to_bf16(const uint4& q, uint4& a, uint4& b
   b = make_uint4(o[4], o[5], o[6], o[7]);
 }
 template <class G> struct FrameSrc {
+  static constexpr bool ASYNC = false;     // needs the uint8 -> bf16 conversion, so it goes through registers
   const uint8_t* x; int M;
   __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
     static_assert(G::K * G::C == 32, "one kernel row must be 32 bytes");
@@ -126,6 +141,13 @@ struct BiasReluEpiTc {
 // 64 output-channel gradients of window (y - r, x - s), or zeros where that window does not exist.
 template <class G> struct DgradSrcS1 {
   const bf16* g; int M;
+  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const {
+    m = min(m, M - 1);
+    const int b = m / (G::H * G::W), rem = m % (G::H * G::W), y = rem / G::W, x = rem % G::W;
+    const int oh = y - kb / G::K, ow = x - kb % G::K;
+    valid = oh >= 0 && oh < G::OH && ow >= 0 && ow < G::OW;
+    return valid ? g + ((size_t)(b * G::OH + oh) * G::OW + ow) * G::CO : g;
+  }
   __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
     static_assert(G::S == 1 && G::CO == 64, "one tap per K block");
     m = min(m, M - 1);
@@ -146,6 +168,14 @@ template <class G> struct DgradSrcS1 {
 // own dense contraction with K = 4 taps x 64 and no structural zeros.  Row m = (state, y>>1, x>>1).
 template <class G> struct DgradSrcS2 {
   const bf16* g; int M;
+  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const {
+    constexpr int HH = G::H / 2, WW = G::W / 2;
+    m = min(m, M - 1);
+    const int b = m / (HH * WW), rem = m % (HH * WW), yy = rem / WW, xx = rem % WW;
+    const int oh = yy - (kb >> 1), ow = xx - (kb & 1);
+    valid = oh >= 0 && oh < G::OH && ow >= 0 && ow < G::OW;
+    return valid ? g + ((size_t)(b * G::OH + oh) * G::OW + ow) * G::CO : g;
+  }
   __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
     static_assert(G::S == 2 && G::K == 4 && G::CO == 64 && G::H % 2 == 0 && G::W % 2 == 0, "parity split");
     constexpr int HH = G::H / 2, WW = G::W / 2;
@@ -298,6 +328,169 @@ tc_gemm_kernel(ASrc a_src, BSrc b_src, Epi epi, int num_kb, uint32_t* error_word
   }
 }
 
+// ---- persistent variant: weights resident in shared memory, A streamed with cp.async -------------------
+// One CTA per SM walks over output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...; tile t is row tile
+// t % tiles_m of class t / tiles_m (classes: the parity classes of a stride-2 data gradient, else one).
+// The whole K extent of the CTA's weight slice (BN rows, KB blocks, all classes) is loaded once.
+//   warps 0-3  epilogue: tile i is read out of its TMEM buffer while tile i+1 is being multiplied
+//   warps 4-7  producers: one tile row per thread, eight 16-byte cp.async per K block straight into the
+//              swizzled image; a stage is published LAG blocks later, after the thread's copies of it
+//              have landed (cp.async.wait_group) and were fenced towards the async proxy
+//   warp 8     lane 0 issues the MMAs and commits stages / accumulators
+constexpr int PK_THREADS = 288, PK_LAG = 3;
+struct PkShared {
+  uint64_t full[8], empty[8], acc_full[2], acc_empty[2];
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES>
+__global__ void __launch_bounds__(PK_THREADS, 1)
+tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi epi, int tiles_m, uint32_t* error_word) {
+  static_assert(BN == 32 || BN == 64 || BN == 128, "tile width");
+  static_assert(STAGES >= PK_LAG + 2 && STAGES <= 8, "pipeline depth");
+  constexpr uint32_t A_BYTES = TC_BM * 128, B_BLOCK = BN * 128, B_BYTES = NCLS * KB * B_BLOCK;
+  extern __shared__ uint8_t dyn_smem[];
+  __shared__ PkShared sh;
+  const uint32_t b_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+  const uint32_t a_base0 = b_base + B_BYTES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.y * BN;
+  const int total_tiles = NCLS * tiles_m;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 4); }
+    sh.abort = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 8) tmem_alloc(&sh.tmem_base, 2 * BN);
+  // resident weights: chunk index -> (class, k block, row, 16-byte chunk)
+  for (int i = threadIdx.x; i < NCLS * KB * BN * 8; i += PK_THREADS) {
+    const int c = i & 7, row = (i >> 3) % BN, kb = (i / (8 * BN)) % KB, cls = i / (8 * BN * KB);
+    const bf16* src = w + ((size_t)(cls * n_total + n0 + row) * KB + kb) * TC_BK + c * 8;
+    cp_async16(b_base + (cls * KB + kb) * B_BLOCK + sw128_offset(row, c), src, 16u);
+  }
+  cp_async_commit();
+  cp_async_wait<0>();
+  fence_proxy_async_smem();
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp >= 4 && warp < 8) {
+    // ---------------- producers ----------------
+    const int row = threadIdx.x - 128;
+    int it = 0;
+    bool alive = true;
+    for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
+      const int z = t / tiles_m, m = (t % tiles_m) * TC_BM + row;
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int s = it % STAGES;
+        const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+        bool valid;
+        const bf16* src = a_src.ptr(m, kb, z, valid);
+        const uint32_t dst = a_base0 + s * A_BYTES + row * 128u;
+        const uint32_t nbytes = valid ? 16u : 0u;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) cp_async16(dst + ((uint32_t)(c ^ (row & 7)) << 4), src + c * 8, nbytes);
+        cp_async_commit();
+        if (it >= PK_LAG) {
+          cp_async_wait<PK_LAG>();
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.full[(it - PK_LAG) % STAGES]);
+        }
+      }
+    }
+    // publish the last blocks
+    cp_async_wait<0>();
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (alive && lane == 0)
+      for (int j = it > PK_LAG ? it - PK_LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % STAGES]);
+  } else if (warp < 4) {
+    // ---------------- epilogue ----------------
+    int local = 0;
+    for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++local) {
+      const int ab = local & 1, z = t / tiles_m, m = (t % tiles_m) * TC_BM + threadIdx.x;
+      const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      tcgen05_fence_after();
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN + c * 32, r);
+        epi(m, n0 + c * 32, z, r);
+      }
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
+    }
+  } else if (lane == 0) {
+    // ---------------- MMA issuer ----------------
+    constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
+    int it = 0, local = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++local) {
+      const int ab = local & 1, z = t / tiles_m;
+      ok = mbar_wait(&sh.acc_empty[ab], ((local >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      if (!ok) break;
+      tcgen05_fence_after();
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int s = it % STAGES;
+        ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const uint32_t a_addr = a_base0 + s * A_BYTES, b_addr = b_base + (z * KB + kb) * B_BLOCK;
+#pragma unroll
+        for (int k = 0; k < TC_BK / 16; ++k)
+          mma_bf16(tmem + ab * BN, make_smem_desc(a_addr + k * 32, 0, 1024, SWIZZLE_128B),
+                   make_smem_desc(b_addr + k * 32, 0, 1024, SWIZZLE_128B), idesc, (kb | k) != 0 ? 1u : 0u);
+        mma_commit(&sh.empty[s]);
+      }
+      if (ok) mma_commit(&sh.acc_full[ab]);
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    __syncwarp();
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, 2 * BN);
+  }
+}
+
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES>
+static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_total, Epi e, int M, uint32_t* err) {
+  constexpr int smem = NCLS * KB * BN * 128 + STAGES * TC_BM * 128 + 1024;
+  static_assert(smem <= 227 * 1024, "shared memory budget");
+  auto kern = tc_persistent_kernel<ASrc, Epi, BN, KB, NCLS, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  const int tiles_m = (M + TC_BM - 1) / TC_BM, gy = n_total / BN;
+  int gx = sm_count() / gy;
+  if (gx < 1) gx = 1;
+  if (gx > NCLS * tiles_m) gx = NCLS * tiles_m;
+  KernelScope scope(lc, kid);
+  kern<<<dim3(gx, gy), PK_THREADS, smem, lc.st>>>(a, w, n_total, e, tiles_m, err);
+}
+
 template <class ASrc, class BSrc, class Epi, int BN, int STAGES>
 static void tc_gemm(LaunchCtx& lc, int kid, ASrc a, BSrc b, Epi e, int M, int N, int num_kb, int Z, uint32_t* error_word) {
   constexpr int smem = STAGES * (TC_BM * 128 + BN * 128) + 1024;
@@ -326,12 +519,12 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
     tc_gemm<FrameSrc<C1>, WeightSrc, BiasReluEpiTc, 32, 4>(
         lc, KID_CONV1_FWD, FrameSrc<C1>{frames, M1}, WeightSrc{w + d[0].w_off, C1::KK},
         BiasReluEpiTc{(bf16*)act[0], theta + d[0].b_off, 32, s255, M1}, M1, 32, C1::KK / 64, 1, err);
-    tc_gemm<ConvSrc<C2>, WeightSrc, BiasReluEpiTc, 64, 4>(
-        lc, KID_CONV2_FWD, ConvSrc<C2>{(const bf16*)act[0], M2}, WeightSrc{w + d[1].w_off, C2::KK},
-        BiasReluEpiTc{(bf16*)act[1], theta + d[1].b_off, 64, 1.f, M2}, M2, 64, C2::KK / 64, 1, err);
-    tc_gemm<ConvSrc<C3>, WeightSrc, BiasReluEpiTc, 64, 4>(
-        lc, KID_CONV3_FWD, ConvSrc<C3>{(const bf16*)act[1], M3}, WeightSrc{w + d[2].w_off, C3::KK},
-        BiasReluEpiTc{(bf16*)act[2], theta + d[2].b_off, 64, 1.f, M3}, M3, 64, C3::KK / 64, 1, err);
+    tc_persistent<ConvSrc<C2>, BiasReluEpiTc, 64, C2::KK / 64, 1, 6>(
+        lc, KID_CONV2_FWD, ConvSrc<C2>{(const bf16*)act[0], M2}, w + d[1].w_off, 64,
+        BiasReluEpiTc{(bf16*)act[1], theta + d[1].b_off, 64, 1.f, M2}, M2, err);
+    tc_persistent<ConvSrc<C3>, BiasReluEpiTc, 64, C3::KK / 64, 1, 6>(
+        lc, KID_CONV3_FWD, ConvSrc<C3>{(const bf16*)act[1], M3}, w + d[2].w_off, 64,
+        BiasReluEpiTc{(bf16*)act[2], theta + d[2].b_off, 64, 1.f, M3}, M3, err);
     tc_gemm<PlainSrc, WeightSrc, BiasReluEpiTc, 128, 4>(
         lc, KID_FC_FWD, PlainSrc{(const bf16*)act[2], 3136, n}, WeightSrc{w + d[3].w_off, 3136},
         BiasReluEpiTc{(bf16*)act[3], theta + d[3].b_off, 512, 1.f, n}, n, 512, 3136 / 64, 1, err);
@@ -346,12 +539,16 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
 // stride between 8-row groups 1 KB; a K=16 MMA step covers two groups.
 // A CTA owns JT row tiles of 128 j each and a contiguous range of 64-row blocks of m (split-k); it writes
 // its float partial tile to scratch, and a second kernel adds the partials in a fixed order.
-constexpr int WG_ROWS = 64;
+constexpr int WG_ROWS = 64, WG_LAG = 2;
 
 // G rows: BN (64 or 128) bf16 starting at column n0; rows past M read as zero so that the tail of the last
 // block adds nothing.  VALID < 64 pads a narrower matrix (conv1: 32 channels) with zero columns.
 template <int VALID> struct GradSrc {
   const bf16* g; int ld; int M;
+  __device__ __forceinline__ const bf16* ptr(int m, int n0, bool& valid) const {
+    valid = m < M;
+    return valid ? g + (size_t)m * ld + n0 : g;
+  }
   __device__ __forceinline__ void load(int m, int n0, uint4 (&v)[8]) const {
     if (m >= M) {
 #pragma unroll
@@ -364,7 +561,7 @@ template <int VALID> struct GradSrc {
   }
 };
 
-template <class XSrc, class GSrc, int JT, int BN, int STAGES>
+template <class XSrc, class GSrc, int VALID_N, int JT, int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS)
 tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, int n_atoms, int J, int CO, int num_blocks,
                 int blocks_per_split, uint32_t* error_word) {
@@ -402,31 +599,67 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, int n_atoms
       if (!__all_sync(0xffffffffu, ok)) break;
       const uint32_t a_base = tiles + s * STAGE_BYTES, b_base = a_base + A_BYTES;
       const int m = kb * WG_ROWS + row;
-      uint4 v[8];
+      if constexpr (XSrc::ASYNC && VALID_N == 64) {
+        // sixteen-byte asynchronous copies straight into the image; the stage is published WG_LAG blocks later
 #pragma unroll
-      for (int q = 0; q < A_PER_HALF; ++q) {
-        const int col = half * A_PER_HALF + q;                      // atom column inside the stage
-        const int atom = atom0 + col;
-        if (atom < n_atoms) x_src.load(m, atom, 0, v);
-        else {
+        for (int q = 0; q < A_PER_HALF; ++q) {
+          const int col = half * A_PER_HALF + q, atom = atom0 + col;
+          bool valid = false;
+          const bf16* src = x_src.x;
+          if (atom < n_atoms) src = x_src.ptr(m, atom, 0, valid);
+          const uint32_t dst = a_base + col * ATOM_COL + row_off, nbytes = valid ? 16u : 0u;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) v[i] = make_uint4(0u, 0u, 0u, 0u);
+          for (int c = 0; c < 8; ++c) cp_async16(dst + ((uint32_t)(c ^ (row & 7)) << 4), src + c * 8, nbytes);
         }
+        if (half < B_COLS) {
+          bool valid;
+          const bf16* src = g_src.ptr(m, n0 + half * 64, valid);
+          const uint32_t dst = b_base + half * ATOM_COL + row_off, nbytes = valid ? 16u : 0u;
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_base + col * ATOM_COL + row_off +
-                       ((uint32_t)(c ^ (row & 7)) << 4)), "r"(v[c].x), "r"(v[c].y), "r"(v[c].z), "r"(v[c].w) : "memory");
-      }
-      if (half < B_COLS) {
-        g_src.load(m, n0 + half * 64, v);
+          for (int c = 0; c < 8; ++c) cp_async16(dst + ((uint32_t)(c ^ (row & 7)) << 4), src + c * 8, nbytes);
+        }
+        cp_async_commit();
+        if (it >= WG_LAG) {
+          cp_async_wait<WG_LAG>();
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.full[(it - WG_LAG) % STAGES]);
+        }
+      } else {
+        uint4 v[8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_base + half * ATOM_COL + row_off +
-                       ((uint32_t)(c ^ (row & 7)) << 4)), "r"(v[c].x), "r"(v[c].y), "r"(v[c].z), "r"(v[c].w) : "memory");
+        for (int q = 0; q < A_PER_HALF; ++q) {
+          const int col = half * A_PER_HALF + q;                      // atom column inside the stage
+          const int atom = atom0 + col;
+          if (atom < n_atoms) x_src.load(m, atom, 0, v);
+          else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = make_uint4(0u, 0u, 0u, 0u);
+          }
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_base + col * ATOM_COL + row_off +
+                         ((uint32_t)(c ^ (row & 7)) << 4)), "r"(v[c].x), "r"(v[c].y), "r"(v[c].z), "r"(v[c].w) : "memory");
+        }
+        if (half < B_COLS) {
+          g_src.load(m, n0 + half * 64, v);
+#pragma unroll
+          for (int c = 0; c < 8; ++c)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_base + half * ATOM_COL + row_off +
+                         ((uint32_t)(c ^ (row & 7)) << 4)), "r"(v[c].x), "r"(v[c].y), "r"(v[c].z), "r"(v[c].w) : "memory");
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.full[s]);
       }
+    }
+    if constexpr (XSrc::ASYNC && VALID_N == 64) {
+      const int n_it = kb1 > kb0 ? kb1 - kb0 : 0;
+      cp_async_wait<0>();
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.full[s]);
+      if (lane == 0 && !sh.abort)
+        for (int j = n_it > WG_LAG ? n_it - WG_LAG : 0; j < n_it; ++j) mbar_arrive(&sh.full[j % STAGES]);
     }
     // ---------------- epilogue: float partial tile to scratch ----------------
     if (kb1 > kb0 && mbar_wait(&sh.acc, 0, &sh.abort, error_word, ERR_WAIT_ACC)) {
@@ -546,7 +779,8 @@ template <class XSrc, class GSrc, int JT, int BN, int STAGES, int CO>
 static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, const bf16* g, int rows, int n_atoms, float scale,
                      float* gw, float* gb, float* scratch, uint32_t* err) {
   constexpr int smem = STAGES * ((2 * JT + BN / 64) * WG_ROWS * 128) + 1024;
-  auto kern = tc_wgrad_kernel<XSrc, GSrc, JT, BN, STAGES>;
+  static_assert(STAGES >= WG_LAG + 1, "pipeline depth");
+  auto kern = tc_wgrad_kernel<XSrc, GSrc, (CO < 64 ? CO : 64), JT, BN, STAGES>;
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -643,23 +877,23 @@ void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, 
 // ---- backward: data gradients ---------------------------------------------------------------------------
 void tc_backward_dgrad_fc(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   const bf16* wfc_t = images + 4 * 32 * 256 + 64 * 576;
-  tc_gemm<PlainSrc, WeightSrc, ReluMaskEpiTc, 64, 4>(
-      lc, KID_FC_DGRAD, PlainSrc{(const bf16*)gact[3], 512, n}, WeightSrc{wfc_t, 512},
-      ReluMaskEpiTc{(bf16*)gact[2], (const bf16*)act[2], 3136, n}, n, 3136, 512 / 64, 1, err);
+  tc_persistent<PlainSrc, ReluMaskEpiTc, 64, 8, 1, 6>(
+      lc, KID_FC_DGRAD, PlainSrc{(const bf16*)gact[3], 512, n}, wfc_t, 3136,
+      ReluMaskEpiTc{(bf16*)gact[2], (const bf16*)act[2], 3136, n}, n, err);
 }
 void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   typedef NatConv3 C3;
   const int M = n * C3::H * C3::W;
-  tc_gemm<DgradSrcS1<C3>, WeightSrc, ReluMaskEpiTc, 64, 4>(
-      lc, KID_CONV3_DGRAD, DgradSrcS1<C3>{(const bf16*)gact[2], M}, WeightSrc{images + 4 * 32 * 256, 576},
-      ReluMaskEpiTc{(bf16*)gact[1], (const bf16*)act[1], 64, M}, M, 64, 9, 1, err);
+  tc_persistent<DgradSrcS1<C3>, ReluMaskEpiTc, 64, 9, 1, 6>(
+      lc, KID_CONV3_DGRAD, DgradSrcS1<C3>{(const bf16*)gact[2], M}, images + 4 * 32 * 256, 64,
+      ReluMaskEpiTc{(bf16*)gact[1], (const bf16*)act[1], 64, M}, M, err);
 }
 void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   typedef NatConv2 C2;
   const int M = n * (C2::H / 2) * (C2::W / 2);
-  tc_gemm<DgradSrcS2<C2>, ClassWeightSrc, ReluMaskEpiS2<C2>, 32, 4>(
-      lc, KID_CONV2_DGRAD, DgradSrcS2<C2>{(const bf16*)gact[1], M}, ClassWeightSrc{images, 256, 32 * 256},
-      ReluMaskEpiS2<C2>{(bf16*)gact[0], (const bf16*)act[0], M}, M, 32, 4, 4, err);
+  tc_persistent<DgradSrcS2<C2>, ReluMaskEpiS2<C2>, 32, 4, 4, 6>(
+      lc, KID_CONV2_DGRAD, DgradSrcS2<C2>{(const bf16*)gact[1], M}, images, 32,
+      ReluMaskEpiS2<C2>{(bf16*)gact[0], (const bf16*)act[0], M}, M, err);
 }
 
 }  // namespace paac

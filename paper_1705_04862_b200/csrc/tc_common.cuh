@@ -116,6 +116,16 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t r[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// ---- asynchronous 16-byte copies global -> shared (LDGSTS) ---------------------------------------
+// src_bytes = 16 copies, src_bytes = 0 writes sixteen zero bytes (nothing is read)
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst_smem), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
 // ---- shared-memory images ----------------------------------------------------------------------
 // 128-byte swizzle: within each 1024-byte group of eight 128-byte rows, the 16-byte chunk c of
 // row r lives at chunk position c ^ (r & 7).  The same image serves a K-major operand (rows =
