@@ -15,12 +15,85 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
+// EPL consecutive elements of a row as floats (EPL = 8 or 16; 16-byte loads)
+template <int EPL> __device__ __forceinline__ void load_row_slice(const float* p, float (&v)[EPL]) {
+  const float4* q = reinterpret_cast<const float4*>(p);
+#pragma unroll
+  for (int i = 0; i < EPL / 4; ++i) { const float4 t = __ldg(q + i); v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w; }
+}
+template <int EPL> __device__ __forceinline__ void load_row_slice(const bf16* p, float (&v)[EPL]) {
+  const uint4* q = reinterpret_cast<const uint4*>(p);
+#pragma unroll
+  for (int i = 0; i < EPL / 8; ++i) {
+    const uint4 t = __ldg(q + i);
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { v[8 * i + 2 * j] = __uint_as_float(w[j] << 16); v[8 * i + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u); }
+  }
+}
+
+// One warp per state; lane l holds elements [l*EPL, (l+1)*EPL) of the fc activation (F = 32*EPL) and of
+// each head row.  Lane k ends up holding logit k (A <= 32).  If `actions` is given, the warp also draws
+// a_t: u from Philox counter (env, step_lo, step_hi, ACTION stream), then the smallest k with
+// u < p_0 + ... + p_k, the running sum taken serially in float in index order.
+template <class T, class TW, int EPL>
+__global__ void __launch_bounds__(128)
+heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* __restrict__ bpi,
+             const TW* __restrict__ wv, const float* __restrict__ bv, int n, int A,
+             float* __restrict__ logits, float* __restrict__ values, uint64_t seed, uint64_t step,
+             const int32_t* __restrict__ forced, int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
+             float* __restrict__ uniforms) {
+  constexpr int F = 32 * EPL;
+  const int lane = threadIdx.x & 31;
+  const int e = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (e >= n) return;
+  float x[EPL], w[EPL];
+  load_row_slice<EPL>(h + (size_t)e * F + lane * EPL, x);
+  float z = -INFINITY;
+  for (int k = 0; k < A; ++k) {
+    load_row_slice<EPL>(wpi + (size_t)k * F + lane * EPL, w);
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) acc = fmaf(w[i], x[i], acc);
+    acc = warp_sum(acc) + bpi[k];
+    if (lane == k) z = acc;
+  }
+  // the value row follows the policy biases in the parameter vector, so it is not 16-byte aligned
+  float v = 0.f;
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) v = fmaf(to_f(wv[lane * EPL + i]), x[i], v);
+  v = warp_sum(v) + bv[0];
+  if (lane < A) logits[(size_t)e * A + lane] = z;
+  if (lane == 0) values[e] = v;
+  if (actions == nullptr) return;
+
+  const float m = warp_max(z);
+  const float ex = lane < A ? expf(z - m) : 0.f;
+  const float lse = m + logf(warp_sum(ex));
+  const float p = lane < A ? expf(z - lse) : 0.f;
+  const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
+  float c = 0.f;
+  int a = A - 1;
+  bool found = false;
+  for (int k = 0; k < A; ++k) {
+    c += __shfl_sync(0xffffffffu, p, k);
+    if (!found && u < c) { a = k; found = true; }
+  }
+  if (lane == 0) {
+    sampled[e] = a;
+    if (forced != nullptr && forced[e] >= 0) a = forced[e];
+    actions[e] = a;
+    uniforms[e] = u;
+  }
+}
+
+// Element-wise variant of the heads kernel for layouts without 16-byte alignment and for float storage.
 // One warp per state.  Lane k ends up holding logit k (A <= 32).  If `actions` is given,
 // the warp also draws a_t: u from Philox counter (env, step_lo, step_hi, ACTION stream), then the
 // smallest k with u < p_0 + ... + p_k, the running sum taken serially in float in index order.
 template <class T, class TW>
 __global__ void __launch_bounds__(128)
-heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* __restrict__ bpi,
+heads_slow_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* __restrict__ bpi,
              const TW* __restrict__ wv, const float* __restrict__ bv, int n, int F, int A,
              float* __restrict__ logits, float* __restrict__ values, uint64_t seed, uint64_t step,
              const int32_t* __restrict__ forced, int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
@@ -69,14 +142,22 @@ void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta
   const int blocks = (n + 3) / 4;
   KernelScope scope(lc, KID_HEADS_FWD);
   cudaStream_t st = lc.st;
-  if (prec == PAAC_BF16)
-    heads_kernel<bf16, bf16><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, theta + nd.pi_b,
-                                                     theta16 + nd.v_w, theta + nd.v_b, n, nd.F, nd.A, logits, values,
-                                                     seed, step, forced, actions, sampled, uniforms);
+  const float* bpi = theta + nd.pi_b; const float* bv = theta + nd.v_b;
+  const bool aligned = nd.pi_w % 8 == 0;      // 16-byte loads of the policy rows
+  if (prec == PAAC_BF16 && nd.F == 512 && aligned)
+    heads_kernel<bf16, bf16, 16><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
+                                                         nd.A, logits, values, seed, step, forced, actions, sampled, uniforms);
+  else if (prec == PAAC_BF16 && nd.F == 256 && aligned)
+    heads_kernel<bf16, bf16, 8><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
+                                                        nd.A, logits, values, seed, step, forced, actions, sampled, uniforms);
+  else if (prec == PAAC_BF16)
+    heads_slow_kernel<bf16, bf16><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv,
+                                                          n, nd.F, nd.A, logits, values, seed, step, forced, actions,
+                                                          sampled, uniforms);
   else
-    heads_kernel<float, float><<<blocks, 128, 0, st>>>((const float*)h, theta + nd.pi_w, theta + nd.pi_b,
-                                                       theta + nd.v_w, theta + nd.v_b, n, nd.F, nd.A, logits, values,
-                                                       seed, step, forced, actions, sampled, uniforms);
+    heads_slow_kernel<float, float><<<blocks, 128, 0, st>>>((const float*)h, theta + nd.pi_w, bpi, theta + nd.v_w, bv,
+                                                            n, nd.F, nd.A, logits, values, seed, step, forced, actions,
+                                                            sampled, uniforms);
 }
 
 // One thread per environment walks its t_max transitions backwards:

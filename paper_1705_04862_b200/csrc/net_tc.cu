@@ -228,15 +228,19 @@ struct ReluMaskEpiTc {
     relu_mask_store(out, act, (size_t)m * ld + n0, r);
   }
 };
-// same, scattering parity class z of a stride-2 layer back to its input pixels
+// same for the stride-2 layer, whose four parity classes share one A operand and are laid side by side
+// along N: column n belongs to class n / C, channel n % C, and goes back to input pixel
+// (2 yy + class / 2, 2 xx + class % 2)
 template <class G> struct ReluMaskEpiS2 {
   bf16* out; const bf16* act; int M;
-  __device__ __forceinline__ void operator()(int m, int n0, int z, const uint32_t (&r)[32]) const {
+  __device__ __forceinline__ void operator()(int m, int n0, int, const uint32_t (&r)[32]) const {
+    static_assert(G::C == 32, "one class per 32-column slice");
     if (m >= M) return;
     constexpr int HH = G::H / 2, WW = G::W / 2;
+    const int cls = n0 / G::C;
     const int b = m / (HH * WW), rem = m % (HH * WW), yy = rem / WW, xx = rem % WW;
-    const int y = 2 * yy + (z >> 1), x = 2 * xx + (z & 1);
-    relu_mask_store(out, act, ((size_t)(b * G::H + y) * G::W + x) * G::C + n0, r);
+    const int y = 2 * yy + (cls >> 1), x = 2 * xx + (cls & 1);
+    relu_mask_store(out, act, ((size_t)(b * G::H + y) * G::W + x) * G::C, r);
   }
 };
 
@@ -563,8 +567,8 @@ template <int VALID> struct GradSrc {
 
 template <class XSrc, class GSrc, int VALID_N, int JT, int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS)
-tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, int n_atoms, int J, int CO, int num_blocks,
-                int blocks_per_split, uint32_t* error_word) {
+tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, float* __restrict__ bias_partial, int n_atoms,
+                int J, int CO, int num_blocks, int blocks_per_split, uint32_t* error_word) {
   static_assert(BN == 64 || BN == 128, "tile width");
   static_assert(JT == 1 || JT == 2, "row tiles per CTA");
   constexpr uint32_t ATOM_COL = WG_ROWS * 128;                      // 8 KB: one atom column of a stage
@@ -576,6 +580,11 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, int n_atoms
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, atom0 = blockIdx.y * 2 * JT, n0 = blockIdx.z * BN;
   const int kb0 = split * blocks_per_split, kb1 = min(num_blocks, kb0 + blocks_per_split);
+  // The bias gradient sum_m G[m][co] rides along as one more row tile whose operand is constant: row j = 0
+  // is all ones, the other rows zero.  Only the CTAs of the first row-tile group compute it.
+  constexpr uint32_t TMEM_COLS = (JT + 1) * BN <= 128 ? 128 : 256;
+  const bool do_bias = blockIdx.y == 0;
+  const uint32_t ones_base = tiles + STAGES * STAGE_BYTES;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
@@ -583,7 +592,16 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, int n_atoms
     sh.abort = 0u;
     fence_barrier_init();
   }
-  if (warp == 4) tmem_alloc(&sh.tmem_base, JT * BN);
+  if (warp == 4) tmem_alloc(&sh.tmem_base, TMEM_COLS);
+  if (do_bias) {
+    for (uint32_t i = threadIdx.x; i < 2 * ATOM_COL / 16; i += TC_THREADS) {
+      // 16-byte chunk i of the image: element j = 0 of k-row (i / 8) sits in physical chunk (row & 7) of atom column 0
+      const uint32_t krow = i >> 3, chunk = i & 7;
+      const uint32_t one = (i < ATOM_COL / 16 && chunk == (krow & 7)) ? 0x3F80u : 0u;
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %2, %2};" ::"r"(ones_base + i * 16), "r"(one), "r"(0u) : "memory");
+    }
+    fence_proxy_async_smem();
+  }
   tcgen05_fence_before();
   __syncthreads();
   tcgen05_fence_after();
@@ -680,6 +698,17 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, int n_atoms
           }
         }
       }
+      if (do_bias && warp == 0) {
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32(tmem + JT * BN + c * 32, r);
+          if (lane == 0 && n0 + c * 32 < CO) {
+#pragma unroll
+            for (int q = 0; q < 32; ++q) bias_partial[(size_t)split * CO + n0 + c * 32 + q] = __uint_as_float(r[q]);
+          }
+        }
+      }
     }
   } else if (lane == 0) {
     // ---------------- MMA issuer ----------------
@@ -700,6 +729,14 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, int n_atoms
           mma_bf16(tmem + jt * BN, ad, bd, idesc, (it | t) != 0 ? 1u : 0u);
         }
       }
+      if (do_bias) {
+#pragma unroll
+        for (int t = 0; t < WG_ROWS / 16; ++t) {
+          const uint64_t ad = make_smem_desc(ones_base + t * 2048, ATOM_COL, 1024, SWIZZLE_128B);
+          const uint64_t bd = make_smem_desc(b_base + t * 2048, ATOM_COL, 1024, SWIZZLE_128B);
+          mma_bf16(tmem + JT * BN, ad, bd, idesc, (it | t) != 0 ? 1u : 0u);
+        }
+      }
       mma_commit(&sh.empty[s]);
     }
     if (ok && kb1 > kb0) mma_commit(&sh.acc);
@@ -709,50 +746,32 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, int n_atoms
   if (warp == 4) {
     __syncwarp();
     tcgen05_fence_after();
-    tmem_dealloc(tmem, JT * BN);
+    tmem_dealloc(tmem, TMEM_COLS);
   }
 }
 
-// dW[co][j] = scale * sum over splits of partial[split][j][co]   (fixed order)
-__global__ void tc_wgrad_reduce_kernel(const float* __restrict__ partial, int splits, int J, int CO, float scale,
-                                       float* __restrict__ gw) {
-  const int total = J * CO;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
-    float s = 0.f;
-    for (int p = 0; p < splits; ++p) s += partial[(size_t)p * total + i];
-    const int j = i / CO, co = i % CO;
-    gw[(size_t)co * J + j] = s * scale;
-  }
-}
-
-// bias gradient: column sums of G[rows][CO]; block b adds its slice of rows in a fixed order, then the
-// last stage adds the per-block results in block order
-template <int CO>
-__global__ void __launch_bounds__(256) tc_bias_partial_kernel(const bf16* __restrict__ g, int rows, float* __restrict__ part) {
-  constexpr int TPR = CO / 8, RPB = 256 / TPR;          // threads per row (8 channels each), rows per pass
-  __shared__ float sh[256][9];
-  const int c8 = threadIdx.x % TPR, r0 = threadIdx.x / TPR;
-  const int per = (rows + gridDim.x - 1) / gridDim.x;
-  const int lo = blockIdx.x * per, hi = min(rows, lo + per);
-  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-  for (int r = lo + r0; r < hi; r += RPB) {
-    const uint4 q = __ldg(reinterpret_cast<const uint4*>(g + (size_t)r * CO) + c8);
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      acc[2 * i] += __uint_as_float(w[i] << 16);
-      acc[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) sh[threadIdx.x][i] = acc[i];
+// dW[co][j] = scale * sum over splits of partial[split][j][co].  A block owns 32 consecutive outputs;
+// its 8 thread rows each add every 8th split, then the 8 sums are added in a fixed order.
+__global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* __restrict__ partial, int splits, int J, int CO,
+                                                              float scale, float* __restrict__ gw) {
+  __shared__ float sh[8][33];
+  const int total = J * CO, lane = threadIdx.x & 31, part = threadIdx.x >> 5;
+  const int i = blockIdx.x * 32 + lane;
+  float s = 0.f;
+  if (i < total)
+    for (int p = part; p < splits; p += 8) s += partial[(size_t)p * total + i];
+  sh[part][lane] = s;
   __syncthreads();
-  for (int c = threadIdx.x; c < CO; c += 256) {
-    float s = 0.f;
-    for (int r = 0; r < RPB; ++r) s += sh[r * TPR + c / 8][c % 8];
-    part[(size_t)blockIdx.x * CO + c] = s;
+  if (part == 0 && i < total) {
+    float t = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) t += sh[q][lane];
+    const int j = i / CO, co = i % CO;
+    gw[(size_t)co * J + j] = t * scale;
   }
 }
+
+// bias gradient: the per-split column sums written by the weight-gradient kernel, added in split order
 __global__ void tc_bias_final_kernel(const float* __restrict__ part, int blocks, int CO, float* __restrict__ gb) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= CO) return;
@@ -761,7 +780,6 @@ __global__ void tc_bias_final_kernel(const float* __restrict__ part, int blocks,
   gb[c] = s;
 }
 
-constexpr int WG_BIAS_BLOCKS = 296;
 static int wg_splits(int num_blocks, int tiles_yz) {
   int s = (296 + tiles_yz - 1) / tiles_yz;           // about two CTAs per SM in total
   if (s > num_blocks) s = num_blocks;
@@ -772,13 +790,13 @@ static size_t wg_scratch_floats(int rows, int J, int CO, int tiles_yz) {
   const int num_blocks = (rows + WG_ROWS - 1) / WG_ROWS;
   const int bps = (num_blocks + wg_splits(num_blocks, tiles_yz) - 1) / wg_splits(num_blocks, tiles_yz);
   const int splits = (num_blocks + bps - 1) / bps;
-  return (size_t)splits * J * CO + (size_t)WG_BIAS_BLOCKS * CO;
+  return (size_t)splits * J * CO + (size_t)splits * CO;
 }
 
 template <class XSrc, class GSrc, int JT, int BN, int STAGES, int CO>
-static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, const bf16* g, int rows, int n_atoms, float scale,
+static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, int rows, int n_atoms, float scale,
                      float* gw, float* gb, float* scratch, uint32_t* err) {
-  constexpr int smem = STAGES * ((2 * JT + BN / 64) * WG_ROWS * 128) + 1024;
+  constexpr int smem = STAGES * ((2 * JT + BN / 64) * WG_ROWS * 128) + 2 * WG_ROWS * 128 + 1024;
   static_assert(STAGES >= WG_LAG + 1, "pipeline depth");
   auto kern = tc_wgrad_kernel<XSrc, GSrc, (CO < 64 ? CO : 64), JT, BN, STAGES>;
   static bool configured = false;
@@ -794,18 +812,15 @@ static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, const bf16* g, in
   float* bias_part = scratch + (size_t)splits * J * CO;
   {
     KernelScope scope(lc, kid);
-    kern<<<dim3(splits, gy, gz), TC_THREADS, smem, lc.st>>>(xs, gs, scratch, n_atoms, J, CO, num_blocks, bps, err);
+    kern<<<dim3(splits, gy, gz), TC_THREADS, smem, lc.st>>>(xs, gs, scratch, bias_part, n_atoms, J, CO, num_blocks, bps,
+                                                            err);
   }
   {
     KernelScope scope(lc, KID_WGRAD_REDUCE);
-    tc_wgrad_reduce_kernel<<<(J * CO + 255) / 256, 256, 0, lc.st>>>(scratch, splits, J, CO, scale, gw);
-  }
-  {
-    KernelScope scope(lc, KID_BIAS_GRAD);
-    tc_bias_partial_kernel<CO><<<WG_BIAS_BLOCKS, 256, 0, lc.st>>>(g, rows, bias_part);
+    tc_wgrad_reduce_kernel<<<(J * CO + 31) / 32, 256, 0, lc.st>>>(scratch, splits, J, CO, scale, gw);
   }
   KernelScope scope(lc, KID_BIAS_GRAD);
-  tc_bias_final_kernel<<<(CO + 127) / 128, 128, 0, lc.st>>>(bias_part, WG_BIAS_BLOCKS, CO, gb);
+  tc_bias_final_kernel<<<(CO + 127) / 128, 128, 0, lc.st>>>(bias_part, splits, CO, gb);
 }
 
 size_t tc_scratch_floats(int n) {
@@ -825,21 +840,21 @@ void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, 
     typedef NatConv1 C1;
     const int rows = n * C1::OH * C1::OW;
     tc_wgrad<FrameSrc<C1>, GradSrc<32>, 2, 64, 3, 32>(lc, KID_CONV1_WGRAD, FrameSrc<C1>{frames, rows},
-                                                      GradSrc<32>{g, 32, rows}, g, rows, 4, 1.0f / 255.0f, gw, gb,
+                                                      GradSrc<32>{g, 32, rows}, rows, 4, 1.0f / 255.0f, gw, gb,
                                                       scratch, err);
   } else if (layer == 1) {
     typedef NatConv2 C2;
     const int rows = n * C2::OH * C2::OW;
     tc_wgrad<ConvSrc<C2>, GradSrc<64>, 2, 64, 3, 64>(lc, KID_CONV2_WGRAD, ConvSrc<C2>{(const bf16*)act[0], rows},
-                                                     GradSrc<64>{g, 64, rows}, g, rows, 8, 1.f, gw, gb, scratch, err);
+                                                     GradSrc<64>{g, 64, rows}, rows, 8, 1.f, gw, gb, scratch, err);
   } else if (layer == 2) {
     typedef NatConv3 C3;
     const int rows = n * C3::OH * C3::OW;
     tc_wgrad<ConvSrc<C3>, GradSrc<64>, 2, 64, 3, 64>(lc, KID_CONV3_WGRAD, ConvSrc<C3>{(const bf16*)act[1], rows},
-                                                     GradSrc<64>{g, 64, rows}, g, rows, 9, 1.f, gw, gb, scratch, err);
+                                                     GradSrc<64>{g, 64, rows}, rows, 9, 1.f, gw, gb, scratch, err);
   } else {
     tc_wgrad<PlainSrc, GradSrc<64>, 1, 128, 4, 512>(lc, KID_FC_WGRAD, PlainSrc{(const bf16*)act[2], 3136, n},
-                                                    GradSrc<64>{g, 512, n}, g, n, 49, 1.f, gw, gb, scratch, err);
+                                                    GradSrc<64>{g, 512, n}, n, 49, 1.f, gw, gb, scratch, err);
   }
 }
 
@@ -891,8 +906,8 @@ void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* con
 void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   typedef NatConv2 C2;
   const int M = n * (C2::H / 2) * (C2::W / 2);
-  tc_persistent<DgradSrcS2<C2>, ReluMaskEpiS2<C2>, 32, 4, 4, 6>(
-      lc, KID_CONV2_DGRAD, DgradSrcS2<C2>{(const bf16*)gact[1], M}, images, 32,
+  tc_persistent<DgradSrcS2<C2>, ReluMaskEpiS2<C2>, 128, 4, 1, 6>(
+      lc, KID_CONV2_DGRAD, DgradSrcS2<C2>{(const bf16*)gact[1], M}, images, 128,
       ReluMaskEpiS2<C2>{(bf16*)gact[0], (const bf16*)act[0], M}, M, err);
 }
 
