@@ -30,14 +30,19 @@ struct TcShared {
 
 // ---- A-operand sources: 64 bf16 (128 bytes) of row m for K block kb ---------------------------
 // plain row-major matrix x[m][k]
+// Asynchronous sources split the address of (row m, K block kb) into a per-row part, computed once per tile
+// row, and a cheap per-block part: row(m) -> RowRef, at(ref, kb, valid) -> address of the 128 bytes, with
+// valid = false meaning "reads as zeros".
+struct RowRef { uint32_t base; int32_t yx; };
 struct PlainSrc {
   static constexpr bool ASYNC = true;
   const bf16* x; int ld; int M;
-  // address of the 128 bytes; valid = false means "this row reads as zeros"
-  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const {
+  __device__ __forceinline__ RowRef row(int m) const { return RowRef{(uint32_t)min(m, M - 1) * (uint32_t)ld, 0}; }
+  __device__ __forceinline__ const bf16* at(const RowRef& r, int kb, bool& valid) const {
     valid = true;
-    return x + (size_t)min(m, M - 1) * ld + kb * TC_BK;
+    return x + r.base + kb * TC_BK;
   }
+  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const { return at(row(m), kb, valid); }
   __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
     m = min(m, M - 1);
     const uint4* p = reinterpret_cast<const uint4*>(x + (size_t)m * ld + kb * TC_BK);
@@ -49,13 +54,17 @@ struct PlainSrc {
 template <class G> struct ConvSrc {
   static constexpr bool ASYNC = true;
   const bf16* x; int M;
-  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const {
-    valid = true;
+  __device__ __forceinline__ RowRef row(int m) const {
     m = min(m, M - 1);
     const int b = m / (G::OH * G::OW), rem = m % (G::OH * G::OW), oh = rem / G::OW, ow = rem % G::OW;
-    const int tap = kb * (64 / G::C), r = tap / G::K, s = tap % G::K;
-    return x + ((size_t)(b * G::H + oh * G::S + r) * G::W + (ow * G::S + s)) * G::C;
+    return RowRef{(uint32_t)(((b * G::H + oh * G::S) * G::W + ow * G::S) * G::C), 0};
   }
+  __device__ __forceinline__ const bf16* at(const RowRef& rr, int kb, bool& valid) const {
+    valid = true;
+    const int tap = kb * (64 / G::C), r = tap / G::K, s = tap % G::K;
+    return x + rr.base + (r * G::W + s) * G::C;
+  }
+  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const { return at(row(m), kb, valid); }
   __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
     static_assert(64 % G::C == 0 && G::K % (64 / G::C) == 0, "a K block must stay inside one kernel row");
     m = min(m, M - 1);
@@ -141,13 +150,17 @@ struct BiasReluEpiTc {
 // 64 output-channel gradients of window (y - r, x - s), or zeros where that window does not exist.
 template <class G> struct DgradSrcS1 {
   const bf16* g; int M;
-  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const {
+  __device__ __forceinline__ RowRef row(int m) const {
     m = min(m, M - 1);
     const int b = m / (G::H * G::W), rem = m % (G::H * G::W), y = rem / G::W, x = rem % G::W;
-    const int oh = y - kb / G::K, ow = x - kb % G::K;
-    valid = oh >= 0 && oh < G::OH && ow >= 0 && ow < G::OW;
-    return valid ? g + ((size_t)(b * G::OH + oh) * G::OW + ow) * G::CO : g;
+    return RowRef{(uint32_t)(b * G::OH * G::OW * G::CO), (y << 8) | x};
   }
+  __device__ __forceinline__ const bf16* at(const RowRef& rr, int kb, bool& valid) const {
+    const int oh = (rr.yx >> 8) - kb / G::K, ow = (rr.yx & 255) - kb % G::K;
+    valid = oh >= 0 && oh < G::OH && ow >= 0 && ow < G::OW;
+    return valid ? g + rr.base + (oh * G::OW + ow) * G::CO : g;
+  }
+  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const { return at(row(m), kb, valid); }
   __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
     static_assert(G::S == 1 && G::CO == 64, "one tap per K block");
     m = min(m, M - 1);
@@ -168,14 +181,18 @@ template <class G> struct DgradSrcS1 {
 // own dense contraction with K = 4 taps x 64 and no structural zeros.  Row m = (state, y>>1, x>>1).
 template <class G> struct DgradSrcS2 {
   const bf16* g; int M;
-  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const {
+  __device__ __forceinline__ RowRef row(int m) const {
     constexpr int HH = G::H / 2, WW = G::W / 2;
     m = min(m, M - 1);
     const int b = m / (HH * WW), rem = m % (HH * WW), yy = rem / WW, xx = rem % WW;
-    const int oh = yy - (kb >> 1), ow = xx - (kb & 1);
-    valid = oh >= 0 && oh < G::OH && ow >= 0 && ow < G::OW;
-    return valid ? g + ((size_t)(b * G::OH + oh) * G::OW + ow) * G::CO : g;
+    return RowRef{(uint32_t)(b * G::OH * G::OW * G::CO), (yy << 8) | xx};
   }
+  __device__ __forceinline__ const bf16* at(const RowRef& rr, int kb, bool& valid) const {
+    const int oh = (rr.yx >> 8) - (kb >> 1), ow = (rr.yx & 255) - (kb & 1);
+    valid = oh >= 0 && oh < G::OH && ow >= 0 && ow < G::OW;
+    return valid ? g + rr.base + (oh * G::OW + ow) * G::CO : g;
+  }
+  __device__ __forceinline__ const bf16* ptr(int m, int kb, int, bool& valid) const { return at(row(m), kb, valid); }
   __device__ __forceinline__ void load(int m, int kb, int, uint4 (&v)[8]) const {
     static_assert(G::S == 2 && G::K == 4 && G::CO == 64 && G::H % 2 == 0 && G::W % 2 == 0, "parity split");
     constexpr int HH = G::H / 2, WW = G::W / 2;
@@ -341,7 +358,7 @@ tc_gemm_kernel(ASrc a_src, BSrc b_src, Epi epi, int num_kb, uint32_t* error_word
 //              swizzled image; a stage is published LAG blocks later, after the thread's copies of it
 //              have landed (cp.async.wait_group) and were fenced towards the async proxy
 //   warp 8     lane 0 issues the MMAs and commits stages / accumulators
-constexpr int PK_THREADS = 288, PK_LAG = 3;
+constexpr int PK_THREADS = 288, PK_LAG = 5;
 struct PkShared {
   uint64_t full[8], empty[8], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
@@ -385,21 +402,28 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
 
   if (warp >= 4 && warp < 8) {
     // ---------------- producers ----------------
-    const int row = threadIdx.x - 128;
+    // Eight lanes cover the 128 bytes of one row, so every warp-wide copy instruction moves four whole
+    // rows; lane l handles chunk l & 7 of rows 32 pw + 4 p + (l >> 3), p = 0..7.
+    const int pw = warp - 4, c = lane & 7, r4 = lane >> 3;
     int it = 0;
     bool alive = true;
     for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
-      const int z = t / tiles_m, m = (t % tiles_m) * TC_BM + row;
+      const int m0 = (t % tiles_m) * TC_BM + 32 * pw + r4;
+      RowRef ref[8];
+#pragma unroll
+      for (int p = 0; p < 8; ++p) ref[p] = a_src.row(m0 + 4 * p);
       for (int kb = 0; kb < KB; ++kb, ++it) {
         const int s = it % STAGES;
         const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
         if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
-        bool valid;
-        const bf16* src = a_src.ptr(m, kb, z, valid);
-        const uint32_t dst = a_base0 + s * A_BYTES + row * 128u;
-        const uint32_t nbytes = valid ? 16u : 0u;
+        const uint32_t stage = a_base0 + s * A_BYTES + (uint32_t)(32 * pw) * 128u;
 #pragma unroll
-        for (int c = 0; c < 8; ++c) cp_async16(dst + ((uint32_t)(c ^ (row & 7)) << 4), src + c * 8, nbytes);
+        for (int p = 0; p < 8; ++p) {
+          bool valid;
+          const bf16* src = a_src.at(ref[p], kb, valid);
+          const uint32_t row = 4 * p + r4;                       // row inside the warp's 32-row slice
+          cp_async16(stage + row * 128u + ((uint32_t)(c ^ (row & 7)) << 4), src + c * 8, valid ? 16u : 0u);
+        }
         cp_async_commit();
         if (it >= PK_LAG) {
           cp_async_wait<PK_LAG>();
@@ -467,6 +491,152 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
   }
 }
 
+// ---- first layer, forward: uint8 frames -> bf16 operand on the fly --------------------------------------
+// Same persistent skeleton, with eight producer warps: thread (row, half) stages the raw 128 bytes of its
+// output pixel's window rows 4*half .. 4*half+3 with cp.async into a private slot (one tile ahead), then
+// expands them to bf16 into the two K blocks it owns.  Integers 0..255 are exact in bf16: the bytes are
+// spliced into floats 2^23 + n, 2^23 is subtracted, and the upper halves of two results are packed.
+__device__ __forceinline__ void u8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  const float f0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7440)) - 8388608.f;
+  const float f1 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7441)) - 8388608.f;
+  const float f2 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7442)) - 8388608.f;
+  const float f3 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7443)) - 8388608.f;
+  lo = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632);
+  hi = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
+}
+
+constexpr int C1_THREADS = 416;      // warps 0-3 epilogue, 4-11 producers, 12 MMA
+
+template <class G, class Epi, int STAGES>
+__global__ void __launch_bounds__(C1_THREADS, 1)
+tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, Epi epi, int M, int tiles_m,
+                uint32_t* error_word) {
+  static_assert(G::K * G::C == 32 && G::K == 8 && G::CO == 32, "window rows of 32 bytes, 32 output channels");
+  constexpr int BN = 32, KB = 4;
+  constexpr uint32_t A_BYTES = TC_BM * 128, B_BLOCK = BN * 128, B_BYTES = KB * B_BLOCK, RAW_BYTES = 2 * TC_BM * 128;
+  extern __shared__ uint8_t dyn_smem[];
+  __shared__ PkShared sh;
+  const uint32_t b_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+  const uint32_t a_base0 = b_base + B_BYTES;
+  const uint32_t raw_base = a_base0 + STAGES * A_BYTES;       // [2 buffers][2 halves][128 rows][128 bytes]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 4); }
+    sh.abort = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 12) tmem_alloc(&sh.tmem_base, 2 * BN);
+  for (int i = threadIdx.x; i < KB * BN * 8; i += C1_THREADS) {
+    const int c = i & 7, row = (i >> 3) % BN, kb = i / (8 * BN);
+    cp_async16(b_base + kb * B_BLOCK + sw128_offset(row, c), w + ((size_t)row * KB + kb) * TC_BK + c * 8, 16u);
+  }
+  cp_async_commit();
+  cp_async_wait<0>();
+  fence_proxy_async_smem();
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp >= 4 && warp < 12) {
+    // ---------------- producers ----------------
+    const int p = threadIdx.x - 128, row = p & 127, half = p >> 7;
+    const uint32_t my_raw = raw_base + (uint32_t)(half * TC_BM + row) * 128u;
+    // raw chunk c of the slot sits at position c ^ (row & 7), so the reads of a warp spread over the banks
+    auto stage_raw = [&](int t, int buf) {
+      const int m = min((t % tiles_m) * TC_BM + row, M - 1);
+      const int b = m / (G::OH * G::OW), rem = m % (G::OH * G::OW), oh = rem / G::OW, ow = rem % G::OW;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint8_t* src = frames + ((size_t)(b * G::H + oh * G::S + 4 * half + j) * G::W + ow * G::S) * G::C;
+        cp_async16(my_raw + buf * RAW_BYTES + ((uint32_t)((2 * j) ^ (row & 7)) << 4), src, 16u);
+        cp_async16(my_raw + buf * RAW_BYTES + ((uint32_t)((2 * j + 1) ^ (row & 7)) << 4), src + 16, 16u);
+      }
+      cp_async_commit();
+    };
+    int local = 0;
+    bool alive = true;
+    if (blockIdx.x < tiles_m) stage_raw(blockIdx.x, 0);
+    for (int t = blockIdx.x; t < tiles_m && alive; t += gridDim.x, ++local) {
+      const int buf = local & 1;
+      if (t + (int)gridDim.x < tiles_m) { stage_raw(t + gridDim.x, buf ^ 1); cp_async_wait<1>(); }
+      else cp_async_wait<0>();
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        const int kb = 2 * half + q, it = local * KB + kb, s = it % STAGES;
+        const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+        const uint32_t dst = a_base0 + s * A_BYTES + row * 128u;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {            // raw chunk 4q + c -> operand chunks 2c, 2c + 1 of this K block
+          uint32_t r0, r1, r2, r3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                       : "r"(my_raw + buf * RAW_BYTES + ((uint32_t)((4 * q + c) ^ (row & 7)) << 4)) : "memory");
+          uint32_t o[8];
+          u8x4_to_bf16x4(r0, o[0], o[1]); u8x4_to_bf16x4(r1, o[2], o[3]);
+          u8x4_to_bf16x4(r2, o[4], o[5]); u8x4_to_bf16x4(r3, o[6], o[7]);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * c) ^ (row & 7)) << 4)),
+                       "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * c + 1) ^ (row & 7)) << 4)),
+                       "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.full[s]);
+      }
+    }
+    cp_async_wait<0>();
+  } else if (warp < 4) {
+    // ---------------- epilogue ----------------
+    int local = 0;
+    for (int t = blockIdx.x; t < tiles_m; t += gridDim.x, ++local) {
+      const int ab = local & 1, m = t * TC_BM + threadIdx.x;
+      const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      tcgen05_fence_after();
+      uint32_t r[32];
+      tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN, r);
+      epi(m, 0, 0, r);
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
+    }
+  } else if (warp == 12 && lane == 0) {
+    // ---------------- MMA issuer ----------------
+    constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
+    int it = 0, local = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < tiles_m && ok; t += gridDim.x, ++local) {
+      const int ab = local & 1;
+      ok = mbar_wait(&sh.acc_empty[ab], ((local >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      if (!ok) break;
+      tcgen05_fence_after();
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int s = it % STAGES;
+        ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const uint32_t a_addr = a_base0 + s * A_BYTES, b_addr = b_base + kb * B_BLOCK;
+#pragma unroll
+        for (int k = 0; k < TC_BK / 16; ++k)
+          mma_bf16(tmem + ab * BN, make_smem_desc(a_addr + k * 32, 0, 1024, SWIZZLE_128B),
+                   make_smem_desc(b_addr + k * 32, 0, 1024, SWIZZLE_128B), idesc, (kb | k) != 0 ? 1u : 0u);
+        mma_commit(&sh.empty[s]);
+      }
+      if (ok) mma_commit(&sh.acc_full[ab]);
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 12) {
+    __syncwarp();
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, 2 * BN);
+  }
+}
+
 static int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -495,6 +665,22 @@ static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_t
   kern<<<dim3(gx, gy), PK_THREADS, smem, lc.st>>>(a, w, n_total, e, tiles_m, err);
 }
 
+template <class G, class Epi>
+static void tc_conv1(LaunchCtx& lc, const uint8_t* frames, const bf16* w, Epi e, int M, uint32_t* err) {
+  constexpr int STAGES = 4;
+  constexpr int smem = 4 * 32 * 128 + STAGES * TC_BM * 128 + 2 * 2 * TC_BM * 128 + 1024;
+  auto kern = tc_conv1_kernel<G, Epi, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  const int tiles_m = (M + TC_BM - 1) / TC_BM;
+  const int gx = tiles_m < sm_count() ? tiles_m : sm_count();
+  KernelScope scope(lc, KID_CONV1_FWD);
+  kern<<<gx, C1_THREADS, smem, lc.st>>>(frames, w, e, M, tiles_m, err);
+}
+
 template <class ASrc, class BSrc, class Epi, int BN, int STAGES>
 static void tc_gemm(LaunchCtx& lc, int kid, ASrc a, BSrc b, Epi e, int M, int N, int num_kb, int Z, uint32_t* error_word) {
   constexpr int smem = STAGES * (TC_BM * 128 + BN * 128) + 1024;
@@ -520,13 +706,12 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
   {
     typedef NatConv1 C1; typedef NatConv2 C2; typedef NatConv3 C3;
     const int M1 = n * C1::OH * C1::OW, M2 = n * C2::OH * C2::OW, M3 = n * C3::OH * C3::OW;
-    tc_gemm<FrameSrc<C1>, WeightSrc, BiasReluEpiTc, 32, 4>(
-        lc, KID_CONV1_FWD, FrameSrc<C1>{frames, M1}, WeightSrc{w + d[0].w_off, C1::KK},
-        BiasReluEpiTc{(bf16*)act[0], theta + d[0].b_off, 32, s255, M1}, M1, 32, C1::KK / 64, 1, err);
-    tc_persistent<ConvSrc<C2>, BiasReluEpiTc, 64, C2::KK / 64, 1, 6>(
+    tc_conv1<C1, BiasReluEpiTc>(lc, frames, w + d[0].w_off, BiasReluEpiTc{(bf16*)act[0], theta + d[0].b_off, 32, s255, M1},
+                                M1, err);
+    tc_persistent<ConvSrc<C2>, BiasReluEpiTc, 64, C2::KK / 64, 1, 8>(
         lc, KID_CONV2_FWD, ConvSrc<C2>{(const bf16*)act[0], M2}, w + d[1].w_off, 64,
         BiasReluEpiTc{(bf16*)act[1], theta + d[1].b_off, 64, 1.f, M2}, M2, err);
-    tc_persistent<ConvSrc<C3>, BiasReluEpiTc, 64, C3::KK / 64, 1, 6>(
+    tc_persistent<ConvSrc<C3>, BiasReluEpiTc, 64, C3::KK / 64, 1, 8>(
         lc, KID_CONV3_FWD, ConvSrc<C3>{(const bf16*)act[1], M3}, w + d[2].w_off, 64,
         BiasReluEpiTc{(bf16*)act[2], theta + d[2].b_off, 64, 1.f, M3}, M3, err);
     tc_gemm<PlainSrc, WeightSrc, BiasReluEpiTc, 128, 4>(
@@ -543,7 +728,7 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
 // stride between 8-row groups 1 KB; a K=16 MMA step covers two groups.
 // A CTA owns JT row tiles of 128 j each and a contiguous range of 64-row blocks of m (split-k); it writes
 // its float partial tile to scratch, and a second kernel adds the partials in a fixed order.
-constexpr int WG_ROWS = 64, WG_LAG = 2;
+constexpr int WG_ROWS = 64, WG_LAG = 3;
 
 // G rows: BN (64 or 128) bf16 starting at column n0; rows past M read as zero so that the tail of the last
 // block adds nothing.  VALID < 64 pads a narrower matrix (conv1: 32 channels) with zero columns.
@@ -618,23 +803,27 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, float* __re
       const uint32_t a_base = tiles + s * STAGE_BYTES, b_base = a_base + A_BYTES;
       const int m = kb * WG_ROWS + row;
       if constexpr (XSrc::ASYNC && VALID_N == 64) {
-        // sixteen-byte asynchronous copies straight into the image; the stage is published WG_LAG blocks later
+        // Eight lanes cover the 128 bytes of one row: lane l copies chunk l & 7 of rows 16 w + 4 p + (l >> 3),
+        // p = 0..3, for every atom column; the stage is published WG_LAG blocks later.
+        const int c = lane & 7, r4 = lane >> 3;
 #pragma unroll
-        for (int q = 0; q < A_PER_HALF; ++q) {
-          const int col = half * A_PER_HALF + q, atom = atom0 + col;
-          bool valid = false;
-          const bf16* src = x_src.x;
-          if (atom < n_atoms) src = x_src.ptr(m, atom, 0, valid);
-          const uint32_t dst = a_base + col * ATOM_COL + row_off, nbytes = valid ? 16u : 0u;
+        for (int p = 0; p < 4; ++p) {
+          const int rw = 16 * warp + 4 * p + r4, mm = kb * WG_ROWS + rw;
+          const uint32_t off = (uint32_t)(rw >> 3) * 1024u + (uint32_t)(rw & 7) * 128u + ((uint32_t)(c ^ (rw & 7)) << 4);
+          const RowRef ref = x_src.row(mm);
 #pragma unroll
-          for (int c = 0; c < 8; ++c) cp_async16(dst + ((uint32_t)(c ^ (row & 7)) << 4), src + c * 8, nbytes);
-        }
-        if (half < B_COLS) {
-          bool valid;
-          const bf16* src = g_src.ptr(m, n0 + half * 64, valid);
-          const uint32_t dst = b_base + half * ATOM_COL + row_off, nbytes = valid ? 16u : 0u;
+          for (int col = 0; col < 2 * JT; ++col) {
+            bool valid = false;
+            const bf16* src = x_src.x;
+            if (atom0 + col < n_atoms) src = x_src.at(ref, atom0 + col, valid);
+            cp_async16(a_base + col * ATOM_COL + off, src + c * 8, valid ? 16u : 0u);
+          }
 #pragma unroll
-          for (int c = 0; c < 8; ++c) cp_async16(dst + ((uint32_t)(c ^ (row & 7)) << 4), src + c * 8, nbytes);
+          for (int gc = 0; gc < B_COLS; ++gc) {
+            bool valid;
+            const bf16* src = g_src.ptr(mm, n0 + gc * 64, valid);
+            cp_async16(b_base + gc * ATOM_COL + off, src + c * 8, valid ? 16u : 0u);
+          }
         }
         cp_async_commit();
         if (it >= WG_LAG) {
@@ -797,7 +986,7 @@ template <class XSrc, class GSrc, int JT, int BN, int STAGES, int CO>
 static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, int rows, int n_atoms, float scale,
                      float* gw, float* gb, float* scratch, uint32_t* err) {
   constexpr int smem = STAGES * ((2 * JT + BN / 64) * WG_ROWS * 128) + 2 * WG_ROWS * 128 + 1024;
-  static_assert(STAGES >= WG_LAG + 1, "pipeline depth");
+  static_assert(STAGES >= WG_LAG || !XSrc::ASYNC, "pipeline depth");
   auto kern = tc_wgrad_kernel<XSrc, GSrc, (CO < 64 ? CO : 64), JT, BN, STAGES>;
   static bool configured = false;
   if (!configured) {
@@ -845,15 +1034,15 @@ void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, 
   } else if (layer == 1) {
     typedef NatConv2 C2;
     const int rows = n * C2::OH * C2::OW;
-    tc_wgrad<ConvSrc<C2>, GradSrc<64>, 2, 64, 3, 64>(lc, KID_CONV2_WGRAD, ConvSrc<C2>{(const bf16*)act[0], rows},
+    tc_wgrad<ConvSrc<C2>, GradSrc<64>, 2, 64, 5, 64>(lc, KID_CONV2_WGRAD, ConvSrc<C2>{(const bf16*)act[0], rows},
                                                      GradSrc<64>{g, 64, rows}, rows, 8, 1.f, gw, gb, scratch, err);
   } else if (layer == 2) {
     typedef NatConv3 C3;
     const int rows = n * C3::OH * C3::OW;
-    tc_wgrad<ConvSrc<C3>, GradSrc<64>, 2, 64, 3, 64>(lc, KID_CONV3_WGRAD, ConvSrc<C3>{(const bf16*)act[1], rows},
+    tc_wgrad<ConvSrc<C3>, GradSrc<64>, 2, 64, 5, 64>(lc, KID_CONV3_WGRAD, ConvSrc<C3>{(const bf16*)act[1], rows},
                                                      GradSrc<64>{g, 64, rows}, rows, 9, 1.f, gw, gb, scratch, err);
   } else {
-    tc_wgrad<PlainSrc, GradSrc<64>, 1, 128, 4, 512>(lc, KID_FC_WGRAD, PlainSrc{(const bf16*)act[2], 3136, n},
+    tc_wgrad<PlainSrc, GradSrc<64>, 1, 128, 6, 512>(lc, KID_FC_WGRAD, PlainSrc{(const bf16*)act[2], 3136, n},
                                                     GradSrc<64>{g, 512, n}, n, 49, 1.f, gw, gb, scratch, err);
   }
 }
@@ -892,21 +1081,21 @@ void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, 
 // ---- backward: data gradients ---------------------------------------------------------------------------
 void tc_backward_dgrad_fc(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   const bf16* wfc_t = images + 4 * 32 * 256 + 64 * 576;
-  tc_persistent<PlainSrc, ReluMaskEpiTc, 64, 8, 1, 6>(
+  tc_persistent<PlainSrc, ReluMaskEpiTc, 64, 8, 1, 8>(
       lc, KID_FC_DGRAD, PlainSrc{(const bf16*)gact[3], 512, n}, wfc_t, 3136,
       ReluMaskEpiTc{(bf16*)gact[2], (const bf16*)act[2], 3136, n}, n, err);
 }
 void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   typedef NatConv3 C3;
   const int M = n * C3::H * C3::W;
-  tc_persistent<DgradSrcS1<C3>, ReluMaskEpiTc, 64, 9, 1, 6>(
+  tc_persistent<DgradSrcS1<C3>, ReluMaskEpiTc, 64, 9, 1, 8>(
       lc, KID_CONV3_DGRAD, DgradSrcS1<C3>{(const bf16*)gact[2], M}, images + 4 * 32 * 256, 64,
       ReluMaskEpiTc{(bf16*)gact[1], (const bf16*)act[1], 64, M}, M, err);
 }
 void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   typedef NatConv2 C2;
   const int M = n * (C2::H / 2) * (C2::W / 2);
-  tc_persistent<DgradSrcS2<C2>, ReluMaskEpiS2<C2>, 128, 4, 1, 6>(
+  tc_persistent<DgradSrcS2<C2>, ReluMaskEpiS2<C2>, 128, 4, 1, 8>(
       lc, KID_CONV2_DGRAD, DgradSrcS2<C2>{(const bf16*)gact[1], M}, images, 128,
       ReluMaskEpiS2<C2>{(bf16*)gact[0], (const bf16*)act[0], M}, M, err);
 }
