@@ -1012,6 +1012,203 @@ static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, int rows, int n_a
   tc_bias_final_kernel<<<(CO + 127) / 128, 128, 0, lc.st>>>(bias_part, splits, CO, gb);
 }
 
+// ---- first layer, weight gradient: one state at a time ----------------------------------------------------
+// dW1^T[j][co] = sum over (state, oh, ow) of window[j] * G[co].  A CTA walks over its share of the states;
+// each state's raw uint8 frame (28,224 bytes) and its 400 x 32 gradient rows are brought into shared memory
+// once by cp.async (one state ahead), so no byte is fetched twice, and the 400 rows are consumed as five
+// blocks of 80: thread (row, q) expands kernel rows 2q, 2q+1 of its window (64 bytes) to bf16 into atom
+// column q of the MN-major image, and thread t copies 16 bytes of G, adding them to its bias sums on the way.
+constexpr int W1_PRODUCERS = 320, W1_THREADS = 352, W1_ROWS = 80, W1_STAGES = 2;
+
+template <class G>
+__global__ void __launch_bounds__(W1_THREADS, 1)
+tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ g, float* __restrict__ partial,
+                      float* __restrict__ bias_partial, int n_states, uint32_t* error_word) {
+  static_assert(G::OH * G::OW == 5 * W1_ROWS && G::CO == 32 && G::K == 8 && G::C == 4 && G::S == 4, "geometry");
+  constexpr uint32_t ATOM_COL = W1_ROWS * 128, A_BYTES = 4 * ATOM_COL, STAGE_BYTES = A_BYTES + ATOM_COL;
+  constexpr uint32_t FRAME_PAD = 28672, GRAW_BYTES = G::OH * G::OW * 64;           // 28,224 rounded up; 25,600
+  constexpr int ROW_BYTES = G::W * G::C;                                          // 336
+  extern __shared__ uint8_t dyn_smem[];
+  __shared__ TcShared sh;
+  const uint32_t tiles = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+  const uint32_t frame_base = tiles + W1_STAGES * STAGE_BYTES;                     // [2][FRAME_PAD]
+  const uint32_t graw_base = frame_base + 2 * FRAME_PAD;                           // [2][GRAW_BYTES]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
+  const int per = (n_states + gridDim.x - 1) / gridDim.x;
+  const int s0 = blockIdx.x * per, s1 = min(n_states, s0 + per);
+
+  if (tid == 0) {
+    for (int s = 0; s < W1_STAGES; ++s) { mbar_init(&sh.full[s], W1_PRODUCERS / 32); mbar_init(&sh.empty[s], 1); }
+    mbar_init(&sh.acc, 1);
+    sh.abort = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 10) tmem_alloc(&sh.tmem_base, 128);
+  // the G image has 128-byte rows of which only 64 bytes carry data: clear both stages once
+  for (uint32_t i = tid; i < W1_STAGES * ATOM_COL / 16; i += W1_THREADS) {
+    const uint32_t st = i / (ATOM_COL / 16), o = i % (ATOM_COL / 16);
+    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(tiles + st * STAGE_BYTES + A_BYTES + o * 16), "r"(0u) : "memory");
+  }
+  fence_proxy_async_smem();
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+  float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+
+  if (warp < 10) {
+    // ---------------- producers ----------------
+    auto prefetch = [&](int st, int buf) {
+      const uint8_t* fsrc = frames + (size_t)st * G::IN_SIZE;
+      for (int i = tid; i < G::IN_SIZE / 16; i += W1_PRODUCERS) cp_async16(frame_base + buf * FRAME_PAD + i * 16, fsrc + i * 16, 16u);
+      const bf16* gsrc = g + (size_t)st * G::OH * G::OW * G::CO;
+      for (int i = tid; i < (int)GRAW_BYTES / 16; i += W1_PRODUCERS) cp_async16(graw_base + buf * GRAW_BYTES + i * 16, gsrc + i * 8, 16u);
+      cp_async_commit();
+    };
+    const int row = tid % W1_ROWS, q = tid / W1_ROWS;       // X work item: row of the block, kernel-row pair
+    const int grow = tid >> 2, gc = tid & 3;                 // G work item: row of the block, 16-byte chunk
+    const uint32_t x_off = (uint32_t)q * ATOM_COL + (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u;
+    const uint32_t g_off = A_BYTES + (uint32_t)(grow >> 3) * 1024u + (uint32_t)(grow & 7) * 128u +
+                           ((uint32_t)(gc ^ (grow & 7)) << 4);
+    int it = 0;
+    bool alive = true;
+    if (s0 < s1) prefetch(s0, 0);
+    for (int st = s0; st < s1 && alive; ++st) {
+      const int buf = (st - s0) & 1;
+      cp_async_wait<0>();
+      asm volatile("bar.sync 1, %0;" ::"n"(W1_PRODUCERS) : "memory");   // this state's bytes are in; the other buffer is free
+      if (st + 1 < s1) prefetch(st + 1, buf ^ 1);
+      const uint32_t fb = frame_base + buf * FRAME_PAD, gb = graw_base + buf * GRAW_BYTES;
+      for (int blk = 0; blk < 5; ++blk, ++it) {
+        const int s = it % W1_STAGES;
+        const bool ok = mbar_wait(&sh.empty[s], ((it / W1_STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+        const uint32_t stage = tiles + s * STAGE_BYTES;
+        const int ml = blk * W1_ROWS + row, oh = ml / G::OW, ow = ml % G::OW;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const uint32_t src = fb + (uint32_t)((oh * G::S + 2 * q + j) * ROW_BYTES + ow * G::S * G::C);
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            uint32_t r0, r1, r2, r3, o[8];
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(src + h * 16) : "memory");
+            u8x4_to_bf16x4(r0, o[0], o[1]); u8x4_to_bf16x4(r1, o[2], o[3]);
+            u8x4_to_bf16x4(r2, o[4], o[5]); u8x4_to_bf16x4(r3, o[6], o[7]);
+            const int c0 = 4 * j + 2 * h;                     // 16 pixels-channels -> two operand chunks
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + x_off + ((uint32_t)(c0 ^ (row & 7)) << 4)),
+                         "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + x_off + ((uint32_t)((c0 + 1) ^ (row & 7)) << 4)),
+                         "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+          }
+        }
+        {
+          uint32_t r0, r1, r2, r3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                       : "r"(gb + (uint32_t)((blk * W1_ROWS + grow) * 64 + gc * 16)) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + g_off), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
+          const uint32_t w[4] = {r0, r1, r2, r3};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            bias[2 * i] += __uint_as_float(w[i] << 16);
+            bias[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
+          }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.full[s]);
+      }
+    }
+    cp_async_wait<0>();
+  } else if (lane == 0) {
+    // ---------------- MMA issuer ----------------
+    constexpr uint32_t idesc = make_idesc_bf16(TC_BM, 64, 1, 1);
+    const int n_it = (s1 > s0 ? s1 - s0 : 0) * 5;
+    bool ok = true;
+    for (int it = 0; it < n_it && ok; ++it) {
+      const int s = it % W1_STAGES;
+      ok = mbar_wait(&sh.full[s], (it / W1_STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      if (!ok) break;
+      tcgen05_fence_after();
+      const uint32_t a_base = tiles + s * STAGE_BYTES, b_base = a_base + A_BYTES;
+#pragma unroll
+      for (int jt = 0; jt < 2; ++jt) {
+#pragma unroll
+        for (int t = 0; t < W1_ROWS / 16; ++t)
+          mma_bf16(tmem + jt * 64, make_smem_desc(a_base + jt * 2 * ATOM_COL + t * 2048, ATOM_COL, 1024, SWIZZLE_128B),
+                   make_smem_desc(b_base + t * 2048, ATOM_COL, 1024, SWIZZLE_128B), idesc, (it | t) != 0 ? 1u : 0u);
+      }
+      mma_commit(&sh.empty[s]);
+    }
+    if (ok && n_it > 0) mma_commit(&sh.acc);
+  }
+  __syncthreads();
+  // bias: channel (gc, i) summed over the 80 threads that carried it, in thread order
+  {
+    float* red = reinterpret_cast<float*>(dyn_smem + (frame_base - smem_u32(dyn_smem)));
+    if (warp < 10) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) red[tid * 8 + i] = bias[i];
+    }
+    __syncthreads();
+    if (tid < 32) {
+      const int gcc = tid >> 3, i = tid & 7;
+      float sum = 0.f;
+      for (int r = 0; r < W1_ROWS; ++r) sum += red[(r * 4 + gcc) * 8 + i];
+      bias_partial[(size_t)blockIdx.x * 32 + tid] = s1 > s0 ? sum : 0.f;
+    }
+  }
+  if (warp < 4) {
+    if (s1 > s0 && mbar_wait(&sh.acc, 0, &sh.abort, error_word, ERR_WAIT_ACC)) {
+      tcgen05_fence_after();
+#pragma unroll 1
+      for (int jt = 0; jt < 2; ++jt) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + jt * 64, r);
+        float4* dst = reinterpret_cast<float4*>(partial + ((size_t)blockIdx.x * 256 + jt * 128 + tid) * 32);
+#pragma unroll
+        for (int v = 0; v < 8; ++v)
+          dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                               __uint_as_float(r[4 * v + 3]));
+      }
+    } else if (s1 <= s0) {
+      for (int jt = 0; jt < 2; ++jt)
+        for (int v = 0; v < 32; ++v) partial[((size_t)blockIdx.x * 256 + jt * 128 + tid) * 32 + v] = 0.f;
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 10) {
+    __syncwarp();
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, 128);
+  }
+}
+
+template <class G>
+static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, int n_states, float* gw, float* gb,
+                           float* scratch, uint32_t* err) {
+  constexpr int smem = W1_STAGES * 5 * W1_ROWS * 128 + 2 * 28672 + 2 * 25600 + 1024;
+  static_assert(smem <= 227 * 1024, "shared memory budget");
+  auto kern = tc_conv1_wgrad_kernel<G>;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  const int splits = n_states < sm_count() ? n_states : sm_count();
+  float* bias_part = scratch + (size_t)splits * 256 * 32;
+  {
+    KernelScope scope(lc, KID_CONV1_WGRAD);
+    kern<<<splits, W1_THREADS, smem, lc.st>>>(frames, g, scratch, bias_part, n_states, err);
+  }
+  {
+    KernelScope scope(lc, KID_WGRAD_REDUCE);
+    tc_wgrad_reduce_kernel<<<(256 * 32 + 31) / 32, 256, 0, lc.st>>>(scratch, splits, 256, 32, 1.0f / 255.0f, gw);
+  }
+  KernelScope scope(lc, KID_BIAS_GRAD);
+  tc_bias_final_kernel<<<1, 128, 0, lc.st>>>(bias_part, splits, 32, gb);
+}
+
 size_t tc_scratch_floats(int n) {
   size_t best = wg_scratch_floats(n * 400, 256, 32, 1);
   size_t v = wg_scratch_floats(n * 81, 512, 64, 2); if (v > best) best = v;
@@ -1028,9 +1225,8 @@ void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, 
   if (layer == 0) {
     typedef NatConv1 C1;
     const int rows = n * C1::OH * C1::OW;
-    tc_wgrad<FrameSrc<C1>, GradSrc<32>, 2, 64, 3, 32>(lc, KID_CONV1_WGRAD, FrameSrc<C1>{frames, rows},
-                                                      GradSrc<32>{g, 32, rows}, rows, 4, 1.0f / 255.0f, gw, gb,
-                                                      scratch, err);
+    tc_conv1_wgrad<C1>(lc, frames, g, n, gw, gb, scratch, err);
+    (void)rows;
   } else if (layer == 1) {
     typedef NatConv2 C2;
     const int rows = n * C2::OH * C2::OW;
