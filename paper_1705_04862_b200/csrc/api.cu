@@ -92,6 +92,7 @@ size_t carve(paac_ctx* c, char* base) {
   {
     size_t sc = simt_scratch_floats(c->arch, nd, (int)B);
     if (tc_supported(c->arch, c->prec) && tc_scratch_floats((int)B) > sc) sc = tc_scratch_floats((int)B);
+    if (tc_supported(c->arch, c->prec) && tc_fc_scratch_floats((int)n_e) > sc) sc = tc_fc_scratch_floats((int)n_e);
     c->scratch = k.take<float>(sc);
   }
   c->norm_partials = k.take<float>(NORM_BLOCKS);
@@ -131,7 +132,7 @@ void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, uin
   for (int l = 0; l <= c->nd.n_conv; ++l)
     act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
   if (use_tc(c))
-    tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, frames, c->n_e, act, &c->stats->error_word);
+    tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, frames, c->n_e, act, c->scratch, &c->stats->error_word);
   else
     simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
   const size_t row = (size_t)slot * c->n_e;

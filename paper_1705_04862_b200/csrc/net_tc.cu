@@ -491,6 +491,152 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
   }
 }
 
+// ---- plain split-k GEMM with both operands streamed (the fully connected layer, forward) ----------------
+// C[m][n] = sum_k A[m][k] W[n][k] for A[M][K], W[N][K] row-major bf16.  Same persistent skeleton; a work item
+// is (row tile, 128-column tile, k split), the stage holds the A and the W tile of one K block, and the
+// epilogue stores float partial sums part[split][m][n].  fc_finish_kernel adds the splits in order, then
+// bias, ReLU and the bf16 rounding.
+constexpr int SK_BN = 128, SK_STAGES = 6, SK_LAG = 4;
+
+__global__ void __launch_bounds__(PK_THREADS, 1)
+tc_splitk_kernel(const bf16* __restrict__ a, const bf16* __restrict__ w, float* __restrict__ part, int M, int N, int K,
+                 int tiles_m, int tiles_n, int splits, int kb_per, uint32_t* error_word) {
+  constexpr uint32_t A_BYTES = TC_BM * 128, STAGE_BYTES = A_BYTES + SK_BN * 128;
+  extern __shared__ uint8_t dyn_smem[];
+  __shared__ PkShared sh;
+  const uint32_t base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total = tiles_m * tiles_n * splits, kb_total = K / TC_BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < SK_STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 4); }
+    sh.abort = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 8) tmem_alloc(&sh.tmem_base, 2 * SK_BN);
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp >= 4 && warp < 8) {
+    // ---------------- producers: lane l copies chunk l & 7 of rows 32 pw + 4 p + (l >> 3) of both tiles ----------------
+    const int pw = warp - 4, c = lane & 7, r4 = lane >> 3;
+    int it = 0;
+    bool alive = true;
+    for (int t = blockIdx.x; t < total && alive; t += gridDim.x) {
+      const int split = t % splits, nt = (t / splits) % tiles_n, mt = t / (splits * tiles_n);
+      const int kb0 = split * kb_per, kb1 = min(kb_total, kb0 + kb_per);
+      for (int kb = kb0; kb < kb1; ++kb, ++it) {
+        const int s = it % SK_STAGES;
+        const bool ok = mbar_wait(&sh.empty[s], ((it / SK_STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+        const uint32_t stage = base + s * STAGE_BYTES + (uint32_t)(32 * pw) * 128u;
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+          const uint32_t row = 4 * p + r4, off = row * 128u + ((uint32_t)(c ^ (row & 7)) << 4);
+          const int m = min(mt * TC_BM + 32 * pw + (int)row, M - 1), n = nt * SK_BN + 32 * pw + (int)row;
+          cp_async16(stage + off, a + (size_t)m * K + kb * TC_BK + c * 8, 16u);
+          cp_async16(stage + A_BYTES + off, w + (size_t)n * K + kb * TC_BK + c * 8, 16u);
+        }
+        cp_async_commit();
+        if (it >= SK_LAG) {
+          cp_async_wait<SK_LAG>();
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sh.full[(it - SK_LAG) % SK_STAGES]);
+        }
+      }
+    }
+    cp_async_wait<0>();
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (alive && lane == 0)
+      for (int j = it > SK_LAG ? it - SK_LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % SK_STAGES]);
+  } else if (warp < 4) {
+    // ---------------- epilogue ----------------
+    int local = 0;
+    for (int t = blockIdx.x; t < total; t += gridDim.x, ++local) {
+      const int ab = local & 1, split = t % splits, nt = (t / splits) % tiles_n, mt = t / (splits * tiles_n);
+      const int m = mt * TC_BM + threadIdx.x;
+      const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      tcgen05_fence_after();
+#pragma unroll 1
+      for (int cc = 0; cc < SK_BN / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * SK_BN + cc * 32, r);
+        if (m < M) {
+          float4* dst = reinterpret_cast<float4*>(part + ((size_t)split * M + m) * N + nt * SK_BN + cc * 32);
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
+                                 __uint_as_float(r[4 * q + 3]));
+        }
+      }
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
+    }
+  } else if (lane == 0) {
+    // ---------------- MMA issuer ----------------
+    constexpr uint32_t idesc = make_idesc_bf16(TC_BM, SK_BN, 0, 0);
+    int it = 0, local = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++local) {
+      const int ab = local & 1, split = t % splits;
+      const int kb0 = split * kb_per, kb1 = min(kb_total, kb0 + kb_per);
+      ok = mbar_wait(&sh.acc_empty[ab], ((local >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      if (!ok) break;
+      tcgen05_fence_after();
+      for (int kb = kb0; kb < kb1; ++kb, ++it) {
+        const int s = it % SK_STAGES;
+        ok = mbar_wait(&sh.full[s], (it / SK_STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const uint32_t a_addr = base + s * STAGE_BYTES, b_addr = a_addr + A_BYTES;
+#pragma unroll
+        for (int k = 0; k < TC_BK / 16; ++k)
+          mma_bf16(tmem + ab * SK_BN, make_smem_desc(a_addr + k * 32, 0, 1024, SWIZZLE_128B),
+                   make_smem_desc(b_addr + k * 32, 0, 1024, SWIZZLE_128B), idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+        mma_commit(&sh.empty[s]);
+      }
+      if (ok) mma_commit(&sh.acc_full[ab]);
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    __syncwarp();
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, 2 * SK_BN);
+  }
+}
+
+// out[m][n..n+7] = bf16(relu(sum_s part[s][m][n] + bias[n]))
+__global__ void __launch_bounds__(256) fc_finish_kernel(const float* __restrict__ part, int splits, int M, int N,
+                                                        const float* __restrict__ bias, bf16* __restrict__ out) {
+  const size_t total = (size_t)M * N / 8;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    const size_t e = i * 8;
+    const int n = (int)(e % N);
+    float v[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) v[q] = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      const float4* p = reinterpret_cast<const float4*>(part + (size_t)s * M * N + e);
+      const float4 lo = __ldg(p), hi = __ldg(p + 1);
+      v[0] += lo.x; v[1] += lo.y; v[2] += lo.z; v[3] += lo.w; v[4] += hi.x; v[5] += hi.y; v[6] += hi.z; v[7] += hi.w;
+    }
+    uint32_t o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      o[q] = pack_bf16x2(fmaxf(v[2 * q] + __ldg(bias + n + 2 * q), 0.f), fmaxf(v[2 * q + 1] + __ldg(bias + n + 2 * q + 1), 0.f));
+    *reinterpret_cast<uint4*>(out + e) = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 // ---- first layer, forward: uint8 frames -> bf16 operand on the fly --------------------------------------
 // Same persistent skeleton, with eight producer warps: thread (row, half) stages the raw 128 bytes of its
 // output pixel's window rows 4*half .. 4*half+3 with cp.async into a private slot (one tile ahead), then
@@ -695,11 +841,35 @@ static void tc_gemm(LaunchCtx& lc, int kid, ASrc a, BSrc b, Epi e, int M, int N,
   kern<<<grid, TC_THREADS, smem, lc.st>>>(a, b, e, num_kb, error_word);
 }
 
+constexpr int FC_SPLITS = 7;
+size_t tc_fc_scratch_floats(int n) { return (size_t)FC_SPLITS * n * 512; }
+
+static void tc_fc_forward(LaunchCtx& lc, const bf16* a, const bf16* w, const float* bias, bf16* out, int M, int N, int K,
+                          float* part, uint32_t* err) {
+  constexpr int smem = SK_STAGES * (TC_BM * 128 + SK_BN * 128) + 1024;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(tc_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  const int tiles_m = (M + TC_BM - 1) / TC_BM, tiles_n = N / SK_BN, kb_total = K / TC_BK;
+  const int kb_per = (kb_total + FC_SPLITS - 1) / FC_SPLITS, splits = (kb_total + kb_per - 1) / kb_per;
+  const int total = tiles_m * tiles_n * splits;
+  {
+    KernelScope scope(lc, KID_FC_FWD);
+    tc_splitk_kernel<<<total < sm_count() ? total : sm_count(), PK_THREADS, smem, lc.st>>>(a, w, part, M, N, K, tiles_m,
+                                                                                         tiles_n, splits, kb_per, err);
+  }
+  KernelScope scope(lc, KID_FC_FWD);
+  const int blocks = (M * N / 8 + 255) / 256;
+  fc_finish_kernel<<<blocks < 1184 ? blocks : 1184, 256, 0, lc.st>>>(part, splits, M, N, bias, out);
+}
+
 // ---- forward ---------------------------------------------------------------------------------------------
 bool tc_supported(int arch, int prec) { return arch == PAAC_ARCH_NATURE && prec == PAAC_BF16; }
 
 void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* w, const uint8_t* frames,
-                int n, void* const act[], uint32_t* err) {
+                int n, void* const act[], float* fc_scratch, uint32_t* err) {
   const LayerDims* d = nd.layer;
   const float s255 = 1.0f / 255.0f;
   if (arch != PAAC_ARCH_NATURE) return;   // the caller routes the smaller network to the CUDA-core path
@@ -714,9 +884,7 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
     tc_persistent<ConvSrc<C3>, BiasReluEpiTc, 64, C3::KK / 64, 1, 8>(
         lc, KID_CONV3_FWD, ConvSrc<C3>{(const bf16*)act[1], M3}, w + d[2].w_off, 64,
         BiasReluEpiTc{(bf16*)act[2], theta + d[2].b_off, 64, 1.f, M3}, M3, err);
-    tc_gemm<PlainSrc, WeightSrc, BiasReluEpiTc, 128, 4>(
-        lc, KID_FC_FWD, PlainSrc{(const bf16*)act[2], 3136, n}, WeightSrc{w + d[3].w_off, 3136},
-        BiasReluEpiTc{(bf16*)act[3], theta + d[3].b_off, 512, 1.f, n}, n, 512, 3136 / 64, 1, err);
+    tc_fc_forward(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, (bf16*)act[3], n, 512, 3136, fc_scratch, err);
   }
 }
 
