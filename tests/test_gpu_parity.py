@@ -82,6 +82,86 @@ def test_config4_nature_bf16_terminals(orc):
     assert _bf16_iterations(orc, CONFIGS[3], 2) > 0          # return resets were exercised
 
 
+def test_config5_full_size_first_environments(orc):
+    """The throughput configuration in the launch shape the bench times (n_e = 1024): environments are
+    independent and the network acts per state, so the first 16 environments of the library must walk
+    exactly like a 16-environment oracle with the same seed; then one full-size update is checked
+    through quantities the oracle can compute from small inputs and properties that hold at any size."""
+    cfg = CONFIGS[4]
+    sub = dict(cfg, n_e=16)
+    o, _g = make_pair(orc, sub)
+    _g.close()
+    g = pb.Paac(cfg["arch"], cfg["n_e"], cfg["t_max"], cfg["n_actions"], 1, precision=pb.BF16,
+                lr=cfg["lr"], term_denom=cfg["term_denom"])
+    T, n_e, A, k = cfg["t_max"], cfg["n_e"], cfg["n_actions"], 16
+    ro = o.rollout()
+    forced = np.full((T, n_e), -1, np.int32)
+    forced[:, :k] = ro["actions"]
+    g.force_actions(forced)
+    g.rollout()
+    fr = g.debug_read(pb.DBG_FRAMES).reshape(T, n_e, -1)
+    assert np.array_equal(fr[:, :k], ro["frames"][:T].reshape(T, k, -1))
+    assert np.array_equal(g.debug_read(pb.DBG_NEXT_FRAMES).reshape(n_e, -1)[:k], ro["frames"][T].reshape(k, -1))
+    assert np.array_equal(g.debug_read(pb.DBG_REWARDS).reshape(T, n_e)[:, :k], ro["rewards"])
+    assert np.array_equal(g.debug_read(pb.DBG_TERMINALS).reshape(T, n_e)[:, :k], ro["terminals"])
+    assert np.array_equal(g.debug_read(pb.DBG_UNIFORMS).reshape(T, n_e)[:, :k], ro["uniforms"])
+    logits = g.debug_read(pb.DBG_LOGITS).reshape(T, n_e, A)
+    values = g.debug_read(pb.DBG_VALUES).reshape(T + 1, n_e)
+    assert rel(logits[:, :k], ro["logits"]) <= TOL["bf16"] and rel(values[:, :k], ro["values"]) <= TOL["bf16"]
+    sampled = g.debug_read(pb.DBG_SAMPLED).reshape(T, n_e)[:, :k]
+    pg, _, _ = orc.softmax(np.ascontiguousarray(logits[:, :k]))
+    for t, e in zip(*np.nonzero(sampled != ro["actions"])):
+        band = 1e-5 + float(np.abs(pg[t, e] - ro["probs"][t, e]).sum())
+        assert orc.cdf_margin(ro["probs"][t, e], float(ro["uniforms"][t, e])) <= band
+    # every environment's frames are the hash of its own (seed, env, step, action): spot-check far ones
+    acts = g.debug_read(pb.DBG_ACTIONS).reshape(T, n_e)
+    terms = g.debug_read(pb.DBG_TERMINALS).reshape(T, n_e)
+    rewards = g.debug_read(pb.DBG_REWARDS).reshape(T, n_e)
+    for e in (17, 500, 1023):
+        for t in range(1, T):
+            tag = 0 if terms[t - 1, e] else int(acts[t - 1, e]) + 1
+            assert np.array_equal(fr[t, e].reshape(84, 84, 4), orc.env_frame(1, e, t, tag))
+            assert (int(rewards[t, e]), int(terms[t, e])) == orc.env_outcome(1, e, t, int(acts[t, e]), cfg["term_denom"])
+    # full-size update: returns, advantages and head gradients recomputed by the oracle from the small
+    # tensors; row sums; the reported norm against the gradient vector
+    st = g.update()
+    assert st["status"] == 0 and st["timesteps"] == n_e * T and np.isfinite(st["grad_norm"])
+    R, adv = orc.returns(0.99, rewards, terms, values)
+    assert rel(g.debug_read(pb.DBG_RETURNS), R) <= 1e-6 and rel(g.debug_read(pb.DBG_ADVANTAGES), adv) <= 1e-5
+    dz = g.debug_read(pb.DBG_DLOGITS).reshape(-1, A)
+    assert np.abs(dz.sum(1)).max() <= 1e-7
+    dz_o, dV_o, stats_o = orc.head_grad(0.01, 1.0, logits.reshape(-1, A), values[:T].reshape(-1), acts.reshape(-1),
+                                        R.reshape(-1), adv.reshape(-1))
+    assert rel(dz, dz_o) <= 1e-4 and rel(g.debug_read(pb.DBG_DVALUES), dV_o) <= 1e-4
+    assert abs(st["entropy"] - stats_o["entropy"]) <= 1e-4 and abs(st["value_loss"] - stats_o["value_loss"]) <= 1e-4
+    grad = g.debug_read(pb.DBG_GRAD)
+    assert abs(np.linalg.norm(grad.astype(np.float64)) - st["grad_norm"]) <= 1e-4 * st["grad_norm"]
+    g.close()
+
+
+def test_tensor_core_path_matches_cuda_core_path(orc):
+    """Two implementations of the bf16 network inside the library (tcgen05 tiles vs CUDA-core
+    contractions, same rounding points) agree within the bf16 tolerance on a ragged batch."""
+    outs = []
+    for cores_only in (0, 1):
+        g = pb.Paac("nature", 37, 3, 18, seed=5, precision=pb.BF16, lr=0.0224, term_denom=50)
+        g.set_option(pb.OPT_CUDA_CORES_ONLY, cores_only)
+        if outs:
+            g.force_actions(outs[0]["actions"])
+        g.rollout()
+        acts = g.debug_read(pb.DBG_ACTIONS).copy()
+        st = g.update()
+        outs.append(dict(actions=acts, sampled=g.debug_read(pb.DBG_SAMPLED).copy(),
+                         logits=g.debug_read(pb.DBG_LOGITS).copy(), grad=g.debug_read(pb.DBG_GRAD).copy(),
+                         norm=st["grad_norm"]))
+        g.close()
+    assert np.mean(outs[0]["sampled"] != outs[1]["sampled"]) <= 0.02
+    assert rel(outs[0]["logits"], outs[1]["logits"]) <= TOL["bf16"]
+    d = outs[0]["grad"].astype(np.float64) - outs[1]["grad"]
+    assert np.linalg.norm(d) / np.linalg.norm(outs[1]["grad"]) <= TOL["bf16"]
+    assert abs(outs[0]["norm"] - outs[1]["norm"]) <= TOL["bf16"] * outs[1]["norm"]
+
+
 def test_ragged_sizes_and_action_counts(orc):
     """n_e that is no multiple of any tile, every action-set size of the configs."""
     for arch, prec, n_e, t_max, A in (("nips", "fp32", 5, 3, 18), ("nips", "bf16", 3, 2, 4),
