@@ -638,9 +638,9 @@ __global__ void __launch_bounds__(256) fc_finish_kernel(const float* __restrict_
 }
 
 // ---- first layer, forward: uint8 frames -> bf16 operand on the fly --------------------------------------
-// Same persistent skeleton, with eight producer warps: thread (row, half) stages the raw 128 bytes of its
-// output pixel's window rows 4*half .. 4*half+3 with cp.async into a private slot (one tile ahead), then
-// expands them to bf16 into the two K blocks it owns.  Integers 0..255 are exact in bf16: the bytes are
+// Same persistent skeleton, with eight producer warps: the frame rows a tile needs are copied once into
+// shared memory with cp.async (two tiles ahead); thread (row, half) then expands window rows
+// 4*half .. 4*half+3 of its output pixel to bf16 into the two K blocks it owns.  Integers 0..255 are exact in bf16: the bytes are
 // spliced into floats 2^23 + n, 2^23 is subtracted, and the upper halves of two results are packed.
 __device__ __forceinline__ void u8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
   const float f0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7440)) - 8388608.f;
@@ -652,6 +652,7 @@ __device__ __forceinline__ void u8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_
 }
 
 constexpr int C1_THREADS = 416;      // warps 0-3 epilogue, 4-11 producers, 12 MMA
+constexpr int C1_RAW_BYTES = 14336;  // >= 40 frame rows of 336 bytes
 
 template <class G, class Epi, int STAGES>
 __global__ void __launch_bounds__(C1_THREADS, 1)
@@ -659,12 +660,12 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
                 uint32_t* error_word) {
   static_assert(G::K * G::C == 32 && G::K == 8 && G::CO == 32, "window rows of 32 bytes, 32 output channels");
   constexpr int BN = 32, KB = 4;
-  constexpr uint32_t A_BYTES = TC_BM * 128, B_BLOCK = BN * 128, B_BYTES = KB * B_BLOCK, RAW_BYTES = 2 * TC_BM * 128;
+  constexpr uint32_t A_BYTES = TC_BM * 128, B_BLOCK = BN * 128, B_BYTES = KB * B_BLOCK, RAW_BYTES = C1_RAW_BYTES;
   extern __shared__ uint8_t dyn_smem[];
   __shared__ PkShared sh;
   const uint32_t b_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
   const uint32_t a_base0 = b_base + B_BYTES;
-  const uint32_t raw_base = a_base0 + STAGES * A_BYTES;       // [2 buffers][2 halves][128 rows][128 bytes]
+  const uint32_t raw_base = a_base0 + STAGES * A_BYTES;       // ring of three slots of up to 40 frame rows
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -688,27 +689,47 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
 
   if (warp >= 4 && warp < 12) {
     // ---------------- producers ----------------
+    // The 128 output pixels of a tile lie in at most two states and at most eight output rows, so their
+    // windows cover at most 40 whole frame rows, which are contiguous in memory per state: two plain byte
+    // ranges are copied into a ring slot two tiles ahead, and every window row is then read from there.
+    constexpr int ROW_BYTES = G::W * G::C, POS = G::OH * G::OW, NPROD = 256;
     const int p = threadIdx.x - 128, row = p & 127, half = p >> 7;
-    const uint32_t my_raw = raw_base + (uint32_t)(half * TC_BM + row) * 128u;
-    // raw chunk c of the slot sits at position c ^ (row & 7), so the reads of a warp spread over the banks
-    auto stage_raw = [&](int t, int buf) {
-      const int m = min((t % tiles_m) * TC_BM + row, M - 1);
-      const int b = m / (G::OH * G::OW), rem = m % (G::OH * G::OW), oh = rem / G::OW, ow = rem % G::OW;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const uint8_t* src = frames + ((size_t)(b * G::H + oh * G::S + 4 * half + j) * G::W + ow * G::S) * G::C;
-        cp_async16(my_raw + buf * RAW_BYTES + ((uint32_t)((2 * j) ^ (row & 7)) << 4), src, 16u);
-        cp_async16(my_raw + buf * RAW_BYTES + ((uint32_t)((2 * j + 1) ^ (row & 7)) << 4), src + 16, 16u);
+    auto tile_ranges = [&](int t, int& b0, int& r0, int& n0, int& n1) {
+      const int mf = t * TC_BM, ml = min(mf + TC_BM - 1, M - 1);
+      b0 = mf / POS;
+      const int b1 = ml / POS, ohf = (mf % POS) / G::OW, ohl = (ml % POS) / G::OW;
+      r0 = ohf * G::S;
+      if (b1 == b0) { n0 = (ohl - ohf) * G::S + G::K; n1 = 0; }
+      else { n0 = G::H - r0; n1 = ohl * G::S + G::K; }
+    };
+    auto stage_rows = [&](int t, int slot) {
+      if (t < tiles_m) {
+        int b0, r0, n0, n1;
+        tile_ranges(t, b0, r0, n0, n1);
+        const uint8_t* src0 = frames + ((size_t)b0 * G::H + r0) * ROW_BYTES;
+        const uint8_t* src1 = frames + (size_t)(b0 + 1) * G::H * ROW_BYTES;
+        const int c0 = n0 * (ROW_BYTES / 16), c1 = n1 * (ROW_BYTES / 16);
+        const uint32_t dst = raw_base + slot * RAW_BYTES;
+        for (int i = p; i < c0 + c1; i += NPROD)
+          cp_async16(dst + i * 16, i < c0 ? src0 + (size_t)i * 16 : src1 + (size_t)(i - c0) * 16, 16u);
       }
-      cp_async_commit();
+      cp_async_commit();        // always one group per call, so the wait counts stay uniform
     };
     int local = 0;
     bool alive = true;
-    if (blockIdx.x < tiles_m) stage_raw(blockIdx.x, 0);
+    stage_rows(blockIdx.x, 0);
+    stage_rows(blockIdx.x + gridDim.x, 1);
     for (int t = blockIdx.x; t < tiles_m && alive; t += gridDim.x, ++local) {
-      const int buf = local & 1;
-      if (t + (int)gridDim.x < tiles_m) { stage_raw(t + gridDim.x, buf ^ 1); cp_async_wait<1>(); }
-      else cp_async_wait<0>();
+      cp_async_wait<1>();                                              // this tile's rows (my share) have landed
+      asm volatile("bar.sync 1, %0;" ::"n"(NPROD) : "memory");        // everyone's share has; the slot of tile-1 is free
+      stage_rows(t + 2 * gridDim.x, (local + 2) % 3);
+      int b0, r0, n0, n1;
+      tile_ranges(t, b0, r0, n0, n1);
+      const int m = min(t * TC_BM + row, M - 1);
+      const int b = m / POS, rem = m % POS, oh = rem / G::OW, ow = rem % G::OW;
+      const int first = b == b0 ? oh * G::S - r0 : n0 + oh * G::S;     // slot row of this pixel's window top
+      const uint32_t my_raw = raw_base + (local % 3) * RAW_BYTES +
+                              (uint32_t)((first + 4 * half) * ROW_BYTES + ow * G::S * G::C);
 #pragma unroll
       for (int q = 0; q < 2; ++q) {
         const int kb = 2 * half + q, it = local * KB + kb, s = it % STAGES;
@@ -716,13 +737,13 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
         if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
         const uint32_t dst = a_base0 + s * A_BYTES + row * 128u;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {            // raw chunk 4q + c -> operand chunks 2c, 2c + 1 of this K block
-          uint32_t r0, r1, r2, r3;
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                       : "r"(my_raw + buf * RAW_BYTES + ((uint32_t)((4 * q + c) ^ (row & 7)) << 4)) : "memory");
+        for (int c = 0; c < 4; ++c) {            // window row 2q + c/2, half c&1 -> operand chunks 2c, 2c + 1 of this K block
+          uint32_t r0w, r1w, r2w, r3w;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0w), "=r"(r1w), "=r"(r2w), "=r"(r3w)
+                       : "r"(my_raw + (uint32_t)((2 * q + (c >> 1)) * ROW_BYTES + (c & 1) * 16)) : "memory");
           uint32_t o[8];
-          u8x4_to_bf16x4(r0, o[0], o[1]); u8x4_to_bf16x4(r1, o[2], o[3]);
-          u8x4_to_bf16x4(r2, o[4], o[5]); u8x4_to_bf16x4(r3, o[6], o[7]);
+          u8x4_to_bf16x4(r0w, o[0], o[1]); u8x4_to_bf16x4(r1w, o[2], o[3]);
+          u8x4_to_bf16x4(r2w, o[4], o[5]); u8x4_to_bf16x4(r3w, o[6], o[7]);
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * c) ^ (row & 7)) << 4)),
                        "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * c + 1) ^ (row & 7)) << 4)),
@@ -813,8 +834,8 @@ static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_t
 
 template <class G, class Epi>
 static void tc_conv1(LaunchCtx& lc, const uint8_t* frames, const bf16* w, Epi e, int M, uint32_t* err) {
-  constexpr int STAGES = 4;
-  constexpr int smem = 4 * 32 * 128 + STAGES * TC_BM * 128 + 2 * 2 * TC_BM * 128 + 1024;
+  constexpr int STAGES = 8;
+  constexpr int smem = 4 * 32 * 128 + STAGES * TC_BM * 128 + 3 * C1_RAW_BYTES + 1024;
   auto kern = tc_conv1_kernel<G, Epi, STAGES>;
   static bool configured = false;
   if (!configured) {
