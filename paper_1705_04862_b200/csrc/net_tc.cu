@@ -491,6 +491,228 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
   }
 }
 
+// ---- convolutions without im2col: shifted views of one staged row block ----------------------------------
+// A 128-byte-swizzled operand image may be entered at any 128-byte row (the swizzle is a function of the
+// shared-memory address, not of the descriptor), so when the rows of an image are the pixels of a feature
+// map in raster order, the A operand of filter tap (r, s) is simply the same image entered (r * width + s)
+// rows further down.  A tile therefore stages its 128 + max-shift rows ONCE and issues one group of MMAs
+// per tap, instead of gathering a fresh 128 x 64 block per tap.  The tile rows run over every position of
+// the (padded or full-width) raster, including positions that are not outputs (right / bottom margins):
+// those accumulate finite garbage that the epilogue drops.
+//
+// Cfg supplies: PLANES (row blocks staged per tile), NT (taps), STAGE_ROWS (multiple of 8, >= 128 + largest
+// shift), src(plane, g, valid) -> address of the 128 bytes of raster row g (valid = false: zeros),
+// tap_plane(t), tap_shift(t).  The weights are [BN][NT * 64] K-major, block t belonging to tap t.
+constexpr int SH_LAG = 2;
+
+template <class Cfg, class Epi, int BN, int STAGES>
+__global__ void __launch_bounds__(PK_THREADS, 1)
+tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_t* error_word) {
+  static_assert(BN == 64 || BN == 128, "tile width");
+  static_assert(STAGES >= SH_LAG + 2 && STAGES <= 8 && Cfg::STAGE_ROWS % 8 == 0, "pipeline shape");
+  constexpr int NT = Cfg::NT, SR = Cfg::STAGE_ROWS, PLANES = Cfg::PLANES;
+  constexpr uint32_t PLANE_BYTES = SR * 128, STAGE_BYTES = PLANES * PLANE_BYTES, B_BLOCK = BN * 128, B_BYTES = NT * B_BLOCK;
+  extern __shared__ uint8_t dyn_smem[];
+  __shared__ PkShared sh;
+  const uint32_t b_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+  const uint32_t a_base0 = b_base + B_BYTES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 4); }
+    sh.abort = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 8) tmem_alloc(&sh.tmem_base, 2 * BN);
+  for (int i = threadIdx.x; i < NT * BN * 8; i += PK_THREADS) {
+    const int c = i & 7, row = (i >> 3) % BN, t = i / (8 * BN);
+    cp_async16(b_base + t * B_BLOCK + sw128_offset(row, c), w + ((size_t)row * NT + t) * TC_BK + c * 8, 16u);
+  }
+  cp_async_commit();
+  cp_async_wait<0>();
+  fence_proxy_async_smem();
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp >= 4 && warp < 8) {
+    // ---------------- producers: eight lanes per 128-byte row, 16 rows per pass ----------------
+    const int c = lane & 7, sub = (warp - 4) * 4 + (lane >> 3);
+    int it = 0;
+    bool alive = true;
+    for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x, ++it) {
+      const int s = it % STAGES;
+      const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+      if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+      const uint32_t stage = a_base0 + s * STAGE_BYTES;
+      for (int idx = sub; idx < PLANES * SR; idx += 16) {
+        const int plane = idx / SR, ri = idx % SR;
+        bool valid;
+        const bf16* src = cfg.src(plane, t * TC_BM + ri, valid);
+        cp_async16(stage + plane * PLANE_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), src + c * 8, valid ? 16u : 0u);
+      }
+      cp_async_commit();
+      if (it >= SH_LAG) {
+        cp_async_wait<SH_LAG>();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.full[(it - SH_LAG) % STAGES]);
+      }
+    }
+    cp_async_wait<0>();
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (alive && lane == 0)
+      for (int j = it > SH_LAG ? it - SH_LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % STAGES]);
+  } else if (warp < 4) {
+    // ---------------- epilogue ----------------
+    int local = 0;
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
+      const int ab = local & 1, pos = t * TC_BM + threadIdx.x;
+      const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      tcgen05_fence_after();
+#pragma unroll 1
+      for (int cc = 0; cc < BN / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN + cc * 32, r);
+        epi(pos, cc * 32, r);
+      }
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
+    }
+  } else if (lane == 0) {
+    // ---------------- MMA issuer ----------------
+    constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
+    int it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
+      const int ab = it & 1, s = it % STAGES;
+      ok = mbar_wait(&sh.acc_empty[ab], ((it >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      if (!ok) break;
+      ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      if (!ok) break;
+      tcgen05_fence_after();
+      // descriptor low words: (address >> 4); every operand slice is a compile-time offset from the stage
+      const uint32_t a_lo = ((a_base0 + s * STAGE_BYTES) >> 4) & 0x3FFFu, b_lo = (b_base >> 4) & 0x3FFFu;
+      const uint32_t hi = desc_hi_kmajor_sw128(), d = tmem + ab * BN;
+#pragma unroll
+      for (int tap = 0; tap < NT; ++tap) {
+        constexpr uint32_t K_STEP = 32 >> 4;
+        const uint32_t a_off = (Cfg::tap_plane(tap) * PLANE_BYTES + Cfg::tap_shift(tap) * 128u) >> 4;
+        const uint32_t b_off = (tap * B_BLOCK) >> 4;
+#pragma unroll
+        for (int k = 0; k < TC_BK / 16; ++k) {
+          if (tap == 0 && k == 0) mma_bf16_lo<false>(d, a_lo + a_off, b_lo + b_off, hi, idesc);
+          else mma_bf16_lo<true>(d, a_lo + a_off + k * K_STEP, b_lo + b_off + k * K_STEP, hi, idesc);
+        }
+      }
+      mma_commit(&sh.empty[s]);
+      mma_commit(&sh.acc_full[ab]);
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    __syncwarp();
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, 2 * BN);
+  }
+}
+
+// conv3 forward: rows = the 9 x 9 x 64 input pixels in memory order; tap (r, s) is 9 r + s rows down
+struct C3FwdCfg {
+  static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152;
+  const bf16* x; int rows;                                   // rows = states * 81
+  __device__ __forceinline__ const bf16* src(int, int g, bool& valid) const {
+    valid = g < rows;
+    return valid ? x + (size_t)g * 64 : x;
+  }
+  __host__ __device__ static constexpr int tap_plane(int) { return 0; }
+  __host__ __device__ static constexpr int tap_shift(int t) { return (t / 3) * 9 + t % 3; }
+};
+// conv2 forward: rows = pairs of horizontally adjacent 32-channel pixels (128 bytes), i.e. the input in memory
+// order seen as [state][y][10 pairs]; even and odd image rows go to separate planes, so that tap row r
+// lives in plane r & 1, 10 (r >> 1) + (pair offset) rows down, and tile rows run over a 10 x 10 raster
+struct C2FwdCfg {
+  static constexpr int PLANES = 2, NT = 8, STAGE_ROWS = 144;
+  const bf16* x; int states;
+  __device__ __forceinline__ const bf16* src(int plane, int g, bool& valid) const {
+    // plane row g = (b, oh, X) is pair row 2 g - X + 10 plane of the input in memory order
+    valid = g < states * 100;
+    return valid ? x + (size_t)(2 * g - g % 10 + 10 * plane) * 64 : x;
+  }
+  __host__ __device__ static constexpr int tap_plane(int t) { return (t >> 1) & 1; }
+  __host__ __device__ static constexpr int tap_shift(int t) { return 10 * (t >> 2) + (t & 1); }
+};
+// conv3 data gradient: the 7 x 7 x 64 output gradient on a zero-padded 11 x 11 raster; input pixel (y, x) is
+// raster position 11 y + x and tap (r, s) reads (2 - r) * 11 + (2 - s) rows down
+struct C3DgradCfg {
+  static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152;
+  const bf16* g3; int states;
+  __device__ __forceinline__ const bf16* src(int, int g, bool& valid) const {
+    const int b = g / 121, rem = g % 121, Y = rem / 11, X = rem % 11;
+    valid = b < states && Y >= 2 && Y <= 8 && X >= 2 && X <= 8;
+    return valid ? g3 + ((size_t)b * 49 + (Y - 2) * 7 + (X - 2)) * 64 : g3;
+  }
+  __host__ __device__ static constexpr int tap_plane(int) { return 0; }
+  __host__ __device__ static constexpr int tap_shift(int t) { return (2 - t / 3) * 11 + (2 - t % 3); }
+};
+// conv2 data gradient (all four parity classes along N): the 9 x 9 x 64 gradient on a zero-padded 11 x 11
+// raster; class pixel (yy, xx) is position 11 yy + xx and tap (i, j) reads (1 - i) * 11 + (1 - j) rows down
+struct C2DgradCfg {
+  static constexpr int PLANES = 1, NT = 4, STAGE_ROWS = 144;
+  const bf16* g2; int states;
+  __device__ __forceinline__ const bf16* src(int, int g, bool& valid) const {
+    const int b = g / 121, rem = g % 121, Y = rem / 11, X = rem % 11;
+    valid = b < states && Y >= 1 && Y <= 9 && X >= 1 && X <= 9;
+    return valid ? g2 + ((size_t)b * 81 + (Y - 1) * 9 + (X - 1)) * 64 : g2;
+  }
+  __host__ __device__ static constexpr int tap_plane(int) { return 0; }
+  __host__ __device__ static constexpr int tap_shift(int t) { return (1 - (t >> 1)) * 11 + (1 - (t & 1)); }
+};
+
+// epilogues of the shifted kernels: raster position -> output row, or nothing for a margin position
+template <int RASTER, int WIDTH, int OUT_H, int OUT_W> struct RasterMap {
+  int states;
+  __device__ __forceinline__ bool operator()(int pos, int& b, int& y, int& x) const {
+    b = pos / RASTER;
+    const int rem = pos % RASTER;
+    y = rem / WIDTH; x = rem % WIDTH;
+    return b < states && y < OUT_H && x < OUT_W;
+  }
+};
+template <class Map, int OUT_H, int OUT_W> struct ShiftBiasReluEpi {
+  Map map; bf16* out; const float* bias;
+  __device__ __forceinline__ void operator()(int pos, int n0, const uint32_t (&r)[32]) const {
+    int b, y, x;
+    if (!map(pos, b, y, x)) return;
+    BiasReluEpiTc e{out, bias, 64, 1.f, 0x7fffffff};
+    e((b * OUT_H + y) * OUT_W + x, n0, 0, r);
+  }
+};
+template <class Map, int OUT_H, int OUT_W> struct ShiftReluMaskEpi {
+  Map map; bf16* out; const bf16* act;
+  __device__ __forceinline__ void operator()(int pos, int n0, const uint32_t (&r)[32]) const {
+    int b, y, x;
+    if (!map(pos, b, y, x)) return;
+    relu_mask_store(out, act, ((size_t)(b * OUT_H + y) * OUT_W + x) * 64 + n0, r);
+  }
+};
+// stride-2 data gradient: column slice n0 is parity class n0 / 32 of raster pixel (yy, xx)
+template <class Map> struct ShiftReluMaskEpiS2 {
+  Map map; bf16* out; const bf16* act;
+  __device__ __forceinline__ void operator()(int pos, int n0, const uint32_t (&r)[32]) const {
+    int b, yy, xx;
+    if (!map(pos, b, yy, xx)) return;
+    const int cls = n0 >> 5, y = 2 * yy + (cls >> 1), x = 2 * xx + (cls & 1);
+    relu_mask_store(out, act, ((size_t)(b * 20 + y) * 20 + x) * 32, r);
+  }
+};
+
 // ---- plain split-k GEMM with both operands streamed (the fully connected layer, forward) ----------------
 // C[m][n] = sum_k A[m][k] W[n][k] for A[M][K], W[N][K] row-major bf16.  Same persistent skeleton; a work item
 // is (row tile, 128-column tile, k split), the stage holds the A and the W tile of one K block, and the
@@ -832,6 +1054,21 @@ static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_t
   kern<<<dim3(gx, gy), PK_THREADS, smem, lc.st>>>(a, w, n_total, e, tiles_m, err);
 }
 
+template <class Cfg, class Epi, int BN, int STAGES>
+static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int positions, uint32_t* err) {
+  constexpr int smem = Cfg::NT * BN * 128 + STAGES * Cfg::PLANES * Cfg::STAGE_ROWS * 128 + 1024;
+  static_assert(smem <= 227 * 1024, "shared memory budget");
+  auto kern = tc_shift_kernel<Cfg, Epi, BN, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  const int tiles = (positions + TC_BM - 1) / TC_BM;
+  KernelScope scope(lc, kid);
+  kern<<<tiles < sm_count() ? tiles : sm_count(), PK_THREADS, smem, lc.st>>>(cfg, w, e, tiles, err);
+}
+
 template <class G, class Epi>
 static void tc_conv1(LaunchCtx& lc, const uint8_t* frames, const bf16* w, Epi e, int M, uint32_t* err) {
   constexpr int STAGES = 8;
@@ -899,12 +1136,19 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
     const int M1 = n * C1::OH * C1::OW, M2 = n * C2::OH * C2::OW, M3 = n * C3::OH * C3::OW;
     tc_conv1<C1, BiasReluEpiTc>(lc, frames, w + d[0].w_off, BiasReluEpiTc{(bf16*)act[0], theta + d[0].b_off, 32, s255, M1},
                                 M1, err);
-    tc_persistent<ConvSrc<C2>, BiasReluEpiTc, 64, C2::KK / 64, 1, 8>(
-        lc, KID_CONV2_FWD, ConvSrc<C2>{(const bf16*)act[0], M2}, w + d[1].w_off, 64,
-        BiasReluEpiTc{(bf16*)act[1], theta + d[1].b_off, 64, 1.f, M2}, M2, err);
-    tc_persistent<ConvSrc<C3>, BiasReluEpiTc, 64, C3::KK / 64, 1, 8>(
-        lc, KID_CONV3_FWD, ConvSrc<C3>{(const bf16*)act[1], M3}, w + d[2].w_off, 64,
-        BiasReluEpiTc{(bf16*)act[2], theta + d[2].b_off, 64, 1.f, M3}, M3, err);
+    {
+      typedef RasterMap<100, 10, 9, 9> Map;
+      tc_shift<C2FwdCfg, ShiftBiasReluEpi<Map, 9, 9>, 64, 4>(
+          lc, KID_CONV2_FWD, C2FwdCfg{(const bf16*)act[0], n}, w + d[1].w_off,
+          ShiftBiasReluEpi<Map, 9, 9>{Map{n}, (bf16*)act[1], theta + d[1].b_off}, n * 100, err);
+    }
+    {
+      typedef RasterMap<81, 9, 7, 7> Map;
+      tc_shift<C3FwdCfg, ShiftBiasReluEpi<Map, 7, 7>, 64, 6>(
+          lc, KID_CONV3_FWD, C3FwdCfg{(const bf16*)act[1], n * 81}, w + d[2].w_off,
+          ShiftBiasReluEpi<Map, 7, 7>{Map{n}, (bf16*)act[2], theta + d[2].b_off}, n * 81, err);
+    }
+    (void)M2; (void)M3;
     tc_fc_forward(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, (bf16*)act[3], n, 512, 3136, fc_scratch, err);
   }
 }
@@ -1473,16 +1717,20 @@ void tc_backward_dgrad_fc(LaunchCtx& lc, const bf16* images, int n, void* const 
 void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   typedef NatConv3 C3;
   const int M = n * C3::H * C3::W;
-  tc_persistent<DgradSrcS1<C3>, ReluMaskEpiTc, 64, 9, 1, 8>(
-      lc, KID_CONV3_DGRAD, DgradSrcS1<C3>{(const bf16*)gact[2], M}, images + 4 * 32 * 256, 64,
-      ReluMaskEpiTc{(bf16*)gact[1], (const bf16*)act[1], 64, M}, M, err);
+  typedef RasterMap<121, 11, 9, 9> Map;
+  tc_shift<C3DgradCfg, ShiftReluMaskEpi<Map, 9, 9>, 64, 6>(
+      lc, KID_CONV3_DGRAD, C3DgradCfg{(const bf16*)gact[2], n}, images + 4 * 32 * 256,
+      ShiftReluMaskEpi<Map, 9, 9>{Map{n}, (bf16*)gact[1], (const bf16*)act[1]}, n * 121, err);
+  (void)M;
 }
 void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   typedef NatConv2 C2;
   const int M = n * (C2::H / 2) * (C2::W / 2);
-  tc_persistent<DgradSrcS2<C2>, ReluMaskEpiS2<C2>, 128, 4, 1, 8>(
-      lc, KID_CONV2_DGRAD, DgradSrcS2<C2>{(const bf16*)gact[1], M}, images, 128,
-      ReluMaskEpiS2<C2>{(bf16*)gact[0], (const bf16*)act[0], M}, M, err);
+  typedef RasterMap<121, 11, 10, 10> Map;
+  tc_shift<C2DgradCfg, ShiftReluMaskEpiS2<Map>, 128, 6>(
+      lc, KID_CONV2_DGRAD, C2DgradCfg{(const bf16*)gact[1], n}, images,
+      ShiftReluMaskEpiS2<Map>{Map{n}, (bf16*)gact[0], (const bf16*)act[0]}, n * 121, err);
+  (void)M;
 }
 
 }  // namespace paac
