@@ -238,11 +238,40 @@ __device__ __forceinline__ void relu_mask_store(bf16* out, const bf16* act, size
     dst[j] = make_uint4(o[0], o[1], o[2], o[3]);
   }
 }
+// the same with the 32 activations of the slice already in registers (four 16-byte words)
+__device__ __forceinline__ void relu_mask_store_pre(bf16* out, size_t idx, const uint32_t (&r)[32], const uint4* a4) {
+  uint4* dst = reinterpret_cast<uint4*>(out + idx);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t aw[4] = {a4[j].x, a4[j].y, a4[j].z, a4[j].w};
+    uint32_t o[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float lo = (aw[q] & 0x7FFFu) ? __uint_as_float(r[8 * j + 2 * q]) : 0.f;
+      const float hi = (aw[q] & 0x7FFF0000u) ? __uint_as_float(r[8 * j + 2 * q + 1]) : 0.f;
+      o[q] = pack_bf16x2(lo, hi);
+    }
+    dst[j] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+template <int BN> struct MaskPre { uint4 m[BN / 8]; size_t idx; bool valid; };
 struct ReluMaskEpiTc {
   bf16* out; const bf16* act; int ld; int M;
   __device__ __forceinline__ void operator()(int m, int n0, int, const uint32_t (&r)[32]) const {
     if (m >= M) return;
     relu_mask_store(out, act, (size_t)m * ld + n0, r);
+  }
+  // two-step form: fetch the BN activations of row m starting at column n0 early, use them later
+  template <class P> __device__ __forceinline__ void prefetch(int m, int n0, P& p) const {
+    p.valid = m < M;
+    p.idx = (size_t)m * ld + n0;
+    if (!p.valid) return;
+    const uint4* a4 = reinterpret_cast<const uint4*>(act + p.idx);
+#pragma unroll
+    for (int j = 0; j < (int)(sizeof(p.m) / sizeof(uint4)); ++j) p.m[j] = __ldg(a4 + j);
+  }
+  template <class P> __device__ __forceinline__ void store(int col, const uint32_t (&r)[32], const P& p) const {
+    if (p.valid) relu_mask_store_pre(out, p.idx + col, r, &p.m[col / 8]);
   }
 };
 // same for the stride-2 layer, whose four parity classes share one A operand and are laid side by side
@@ -444,14 +473,17 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
     int local = 0;
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++local) {
       const int ab = local & 1, z = t / tiles_m, m = (t % tiles_m) * TC_BM + threadIdx.x;
+      MaskPre<BN> pre;
+      epi.prefetch(m, n0, pre);
+      (void)z;
       const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
-#pragma unroll 1
+#pragma unroll
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
         tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN + c * 32, r);
-        epi(m, n0 + c * 32, z, r);
+        epi.store(c * 32, r, pre);
       }
       tcgen05_fence_before();
       __syncwarp();
@@ -571,14 +603,16 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
     int local = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
       const int ab = local & 1, pos = t * TC_BM + threadIdx.x;
+      typename Epi::template Pre<BN>::type pre;
+      epi.prefetch(pos, pre);
       const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
-#pragma unroll 1
+#pragma unroll
       for (int cc = 0; cc < BN / 32; ++cc) {
         uint32_t r[32];
         tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN + cc * 32, r);
-        epi(pos, cc * 32, r);
+        epi(pos, cc * 32, r, pre);
       }
       tcgen05_fence_before();
       __syncwarp();
@@ -685,9 +719,14 @@ template <int RASTER, int WIDTH, int OUT_H, int OUT_W> struct RasterMap {
     return b < states && y < OUT_H && x < OUT_W;
   }
 };
+// An epilogue may fetch what it needs from global memory (the ReLU mask of the layer below) into `Pre`
+// before the accumulator is ready, so that the latency hides behind the tile's MMAs.
+struct NoPre {};
 template <class Map, int OUT_H, int OUT_W> struct ShiftBiasReluEpi {
+  template <int BN> struct Pre { typedef NoPre type; };
   Map map; bf16* out; const float* bias;
-  __device__ __forceinline__ void operator()(int pos, int n0, const uint32_t (&r)[32]) const {
+  template <class P> __device__ __forceinline__ void prefetch(int, P&) const {}
+  template <class P> __device__ __forceinline__ void operator()(int pos, int n0, const uint32_t (&r)[32], const P&) const {
     int b, y, x;
     if (!map(pos, b, y, x)) return;
     BiasReluEpiTc e{out, bias, 64, 1.f, 0x7fffffff};
@@ -695,21 +734,42 @@ template <class Map, int OUT_H, int OUT_W> struct ShiftBiasReluEpi {
   }
 };
 template <class Map, int OUT_H, int OUT_W> struct ShiftReluMaskEpi {
+  template <int BN> struct Pre { typedef MaskPre<BN> type; };
   Map map; bf16* out; const bf16* act;
-  __device__ __forceinline__ void operator()(int pos, int n0, const uint32_t (&r)[32]) const {
+  template <class P> __device__ __forceinline__ void prefetch(int pos, P& p) const {
     int b, y, x;
-    if (!map(pos, b, y, x)) return;
-    relu_mask_store(out, act, ((size_t)(b * OUT_H + y) * OUT_W + x) * 64 + n0, r);
+    p.valid = map(pos, b, y, x);
+    p.idx = ((size_t)(b * OUT_H + y) * OUT_W + x) * 64;
+    if (!p.valid) return;
+    const uint4* a4 = reinterpret_cast<const uint4*>(act + p.idx);
+#pragma unroll
+    for (int j = 0; j < (int)(sizeof(p.m) / sizeof(uint4)); ++j) p.m[j] = __ldg(a4 + j);
+  }
+  template <class P> __device__ __forceinline__ void operator()(int, int n0, const uint32_t (&r)[32], const P& p) const {
+    if (p.valid) relu_mask_store_pre(out, p.idx + n0, r, &p.m[n0 / 8]);
   }
 };
 // stride-2 data gradient: column slice n0 is parity class n0 / 32 of raster pixel (yy, xx)
 template <class Map> struct ShiftReluMaskEpiS2 {
+  template <int BN> struct Pre { typedef MaskPre<BN> type; };
   Map map; bf16* out; const bf16* act;
-  __device__ __forceinline__ void operator()(int pos, int n0, const uint32_t (&r)[32]) const {
+  __device__ __forceinline__ size_t class_idx(size_t base, int cls) const {      // base = pixel (2 yy, 2 xx)
+    return base + (size_t)((cls >> 1) * 20 + (cls & 1)) * 32;
+  }
+  template <class P> __device__ __forceinline__ void prefetch(int pos, P& p) const {
     int b, yy, xx;
-    if (!map(pos, b, yy, xx)) return;
-    const int cls = n0 >> 5, y = 2 * yy + (cls >> 1), x = 2 * xx + (cls & 1);
-    relu_mask_store(out, act, ((size_t)(b * 20 + y) * 20 + x) * 32, r);
+    p.valid = map(pos, b, yy, xx);
+    p.idx = ((size_t)(b * 20 + 2 * yy) * 20 + 2 * xx) * 32;
+    if (!p.valid) return;
+#pragma unroll
+    for (int cls = 0; cls < 4; ++cls) {
+      const uint4* a4 = reinterpret_cast<const uint4*>(act + class_idx(p.idx, cls));
+#pragma unroll
+      for (int j = 0; j < 4; ++j) p.m[4 * cls + j] = __ldg(a4 + j);
+    }
+  }
+  template <class P> __device__ __forceinline__ void operator()(int, int n0, const uint32_t (&r)[32], const P& p) const {
+    if (p.valid) relu_mask_store_pre(out, class_idx(p.idx, n0 >> 5), r, &p.m[n0 / 8]);
   }
 };
 
