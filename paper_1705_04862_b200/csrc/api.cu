@@ -24,6 +24,7 @@ struct paac_ctx {
   int host_t;              // external-environment mode: next expected step
   bool forced_on;
   int tc_wgrad_mask;       // bit l: layer l's weight gradient runs on the tensor cores
+  GradSegments grad_segs;  // partial-sum regions of the update in flight
   bool simt_only;          // keep the bf16 network on the CUDA cores (cross-check of the tensor-core path)
 
   // device buffers (all inside the workspace)
@@ -240,13 +241,14 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
     }
     bool wgrad_done = false;
     if (use_tc(c) && (c->tc_wgrad_mask >> l) & 1) {
-      tc_backward_wgrad(c->lc, c->nd, c->frames[c->cur], c->B, c->act, c->gact, c->grad, c->scratch, l, err);
+      tc_backward_wgrad(c->lc, c->nd, c->frames[c->cur], c->B, c->act, c->gact, c->grad, c->scratch, l, &c->grad_segs, err);
       wgrad_done = true;
     }
     if (!wgrad_done || (l > 0 && !dgrad_done))
       simt_backward_layer(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
                           c->gact, c->grad, c->scratch, l, !wgrad_done, l > 0 && !dgrad_done);
   }
+  if (use_tc(c)) tc_backward_finish(c->lc, &c->grad_segs);
   launch_clip_rmsprop(c->lc, c->nd.P, c->theta, c->rms, c->grad,
                       c->prec == PAAC_BF16 ? c->theta16 : nullptr, hp.lr, hp.rms_decay, hp.rms_eps, hp.clip_norm,
                       c->norm_partials, c->stats);

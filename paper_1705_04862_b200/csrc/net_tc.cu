@@ -1462,6 +1462,52 @@ __global__ void tc_bias_final_kernel(const float* __restrict__ part, int blocks,
   gb[c] = s;
 }
 
+// One launch finishes every tensor-core weight gradient of an update: for each segment (a layer's weights, or
+// its bias with J = 1) dst[co * J + j] = scale * sum over splits of part[split][j][co], the splits added in a
+// fixed order.  Segments with many splits give eight threads to every output (each adds every 8th split,
+// the eight sums are then added in order); segments with few splits give one thread to every output.
+__global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments segs) {
+  __shared__ float sh[8][33];
+  const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
+  for (int grp = blockIdx.x; grp < segs.total_groups; grp += gridDim.x) {
+    int si = 0;
+    while (si + 1 < segs.n && grp >= segs.seg[si + 1].first_group) ++si;
+    const GradSegment& sg = segs.seg[si];
+    const int total = sg.J * sg.CO, local = grp - sg.first_group;
+    if (sg.wide) {
+      const int i = local * 32 + lane;
+      float s = 0.f;
+      if (i < total)
+        for (int p = part; p < sg.splits; p += 8) s += sg.part[(size_t)p * total + i];
+      sh[part][lane] = s;
+      __syncthreads();
+      if (part == 0 && i < total) {
+        float t = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) t += sh[q][lane];
+        sg.dst[(size_t)(i % sg.CO) * sg.J + i / sg.CO] = t * sg.scale;
+      }
+      __syncthreads();
+    } else {
+      const int i = local * 256 + threadIdx.x;
+      if (i < total) {
+        float s = 0.f;
+        for (int p = 0; p < sg.splits; ++p) s += sg.part[(size_t)p * total + i];
+        sg.dst[(size_t)(i % sg.CO) * sg.J + i / sg.CO] = s * sg.scale;
+      }
+    }
+  }
+}
+
+static void add_segment(GradSegments* segs, const float* part, float* dst, int splits, int J, int CO, float scale) {
+  GradSegment& g = segs->seg[segs->n++];
+  g.part = part; g.dst = dst; g.splits = splits; g.J = J; g.CO = CO; g.scale = scale;
+  g.wide = splits > 8;
+  g.first_group = segs->total_groups;
+  g.groups = (J * CO + (g.wide ? 32 : 256) - 1) / (g.wide ? 32 : 256);
+  segs->total_groups += g.groups;
+}
+
 static int wg_splits(int num_blocks, int tiles_yz) {
   int s = (296 + tiles_yz - 1) / tiles_yz;           // about two CTAs per SM in total
   if (s > num_blocks) s = num_blocks;
@@ -1477,7 +1523,7 @@ static size_t wg_scratch_floats(int rows, int J, int CO, int tiles_yz) {
 
 template <class XSrc, class GSrc, int JT, int BN, int STAGES, int CO>
 static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, int rows, int n_atoms, float scale,
-                     float* gw, float* gb, float* scratch, uint32_t* err) {
+                     float* gw, float* gb, float* scratch, GradSegments* segs, uint32_t* err) {
   constexpr int smem = STAGES * ((2 * JT + BN / 64) * WG_ROWS * 128) + 2 * WG_ROWS * 128 + 1024;
   static_assert(STAGES >= WG_LAG || !XSrc::ASYNC, "pipeline depth");
   auto kern = tc_wgrad_kernel<XSrc, GSrc, (CO < 64 ? CO : 64), JT, BN, STAGES>;
@@ -1492,17 +1538,10 @@ static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, int rows, int n_a
   const int bps = (num_blocks + wg_splits(num_blocks, gy * gz) - 1) / wg_splits(num_blocks, gy * gz);
   const int splits = (num_blocks + bps - 1) / bps;
   float* bias_part = scratch + (size_t)splits * J * CO;
-  {
-    KernelScope scope(lc, kid);
-    kern<<<dim3(splits, gy, gz), TC_THREADS, smem, lc.st>>>(xs, gs, scratch, bias_part, n_atoms, J, CO, num_blocks, bps,
-                                                            err);
-  }
-  {
-    KernelScope scope(lc, KID_WGRAD_REDUCE);
-    tc_wgrad_reduce_kernel<<<(J * CO + 31) / 32, 256, 0, lc.st>>>(scratch, splits, J, CO, scale, gw);
-  }
-  KernelScope scope(lc, KID_BIAS_GRAD);
-  tc_bias_final_kernel<<<(CO + 127) / 128, 128, 0, lc.st>>>(bias_part, splits, CO, gb);
+  KernelScope scope(lc, kid);
+  kern<<<dim3(splits, gy, gz), TC_THREADS, smem, lc.st>>>(xs, gs, scratch, bias_part, n_atoms, J, CO, num_blocks, bps, err);
+  add_segment(segs, scratch, gw, splits, J, CO, scale);
+  add_segment(segs, bias_part, gb, splits, 1, CO, 1.f);
 }
 
 // ---- first layer, weight gradient: one state at a time ----------------------------------------------------
@@ -1679,7 +1718,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
 
 template <class G>
 static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, int n_states, float* gw, float* gb,
-                           float* scratch, uint32_t* err) {
+                           float* scratch, GradSegments* segs, uint32_t* err) {
   constexpr int smem = W1_STAGES * 5 * W1_ROWS * 128 + 2 * 28672 + 2 * 25600 + 1024;
   static_assert(smem <= 227 * 1024, "shared memory budget");
   auto kern = tc_conv1_wgrad_kernel<G>;
@@ -1690,49 +1729,63 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
   }
   const int splits = n_states < sm_count() ? n_states : sm_count();
   float* bias_part = scratch + (size_t)splits * 256 * 32;
-  {
-    KernelScope scope(lc, KID_CONV1_WGRAD);
-    kern<<<splits, W1_THREADS, smem, lc.st>>>(frames, g, scratch, bias_part, n_states, err);
-  }
-  {
-    KernelScope scope(lc, KID_WGRAD_REDUCE);
-    tc_wgrad_reduce_kernel<<<(256 * 32 + 31) / 32, 256, 0, lc.st>>>(scratch, splits, 256, 32, 1.0f / 255.0f, gw);
-  }
-  KernelScope scope(lc, KID_BIAS_GRAD);
-  tc_bias_final_kernel<<<1, 128, 0, lc.st>>>(bias_part, splits, 32, gb);
+  KernelScope scope(lc, KID_CONV1_WGRAD);
+  kern<<<splits, W1_THREADS, smem, lc.st>>>(frames, g, scratch, bias_part, n_states, err);
+  add_segment(segs, scratch, gw, splits, 256, 32, 1.0f / 255.0f);
+  add_segment(segs, bias_part, gb, splits, 1, 32, 1.f);
 }
 
-size_t tc_scratch_floats(int n) {
-  size_t best = wg_scratch_floats(n * 400, 256, 32, 1);
-  size_t v = wg_scratch_floats(n * 81, 512, 64, 2); if (v > best) best = v;
-  v = wg_scratch_floats(n * 49, 576, 64, 3); if (v > best) best = v;
-  v = wg_scratch_floats(n, 3136, 512, 25 * 4); if (v > best) best = v;
-  return best;
+// every layer keeps its own partial-sum region until the finishing kernel has run
+static size_t tc_layer_scratch_floats(int n, int layer) {
+  switch (layer) {
+    case 0: return wg_scratch_floats(n * 400, 256, 32, 1);
+    case 1: return wg_scratch_floats(n * 81, 512, 64, 2);
+    case 2: return wg_scratch_floats(n * 49, 576, 64, 3);
+    default: return wg_scratch_floats(n, 3136, 512, 25 * 4);
+  }
+}
+static size_t tc_layer_scratch_offset(int n, int layer) {
+  size_t off = 0;
+  for (int l = 0; l < layer; ++l) off += (tc_layer_scratch_floats(n, l) + 63) / 64 * 64;
+  return off;
+}
+
+size_t tc_scratch_floats(int n) { return tc_layer_scratch_offset(n, 4); }
+
+// Enqueues the weight-gradient kernel of `layer` (0 = conv1 .. 3 = fc) and notes in *segs where its partial
+// sums are; tc_backward_finish() then turns all noted partial sums into the gradient vector in one launch.
+void tc_backward_finish(LaunchCtx& lc, GradSegments* segs) {
+  if (segs->n > 0) {
+    KernelScope scope(lc, KID_WGRAD_REDUCE);
+    const int blocks = segs->total_groups < 8 * sm_count() ? segs->total_groups : 8 * sm_count();
+    tc_finalize_grads_kernel<<<blocks, 256, 0, lc.st>>>(*segs);
+  }
+  segs->n = 0; segs->total_groups = 0;
 }
 
 void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, int n, void* const act[],
-                       void* const gact[], float* grad, float* scratch, int layer, uint32_t* err) {
+                       void* const gact[], float* grad, float* scratch, int layer, GradSegments* segsp, uint32_t* err) {
+  GradSegments& segs = *segsp;
   const LayerDims* d = nd.layer;
   float* gw = grad + d[layer].w_off; float* gb = grad + d[layer].b_off;
   const bf16* g = (const bf16*)gact[layer];
+  float* sc = scratch + tc_layer_scratch_offset(n, layer);
   if (layer == 0) {
     typedef NatConv1 C1;
-    const int rows = n * C1::OH * C1::OW;
-    tc_conv1_wgrad<C1>(lc, frames, g, n, gw, gb, scratch, err);
-    (void)rows;
+    tc_conv1_wgrad<C1>(lc, frames, g, n, gw, gb, sc, &segs, err);
   } else if (layer == 1) {
     typedef NatConv2 C2;
     const int rows = n * C2::OH * C2::OW;
     tc_wgrad<ConvSrc<C2>, GradSrc<64>, 2, 64, 5, 64>(lc, KID_CONV2_WGRAD, ConvSrc<C2>{(const bf16*)act[0], rows},
-                                                     GradSrc<64>{g, 64, rows}, rows, 8, 1.f, gw, gb, scratch, err);
+                                                     GradSrc<64>{g, 64, rows}, rows, 8, 1.f, gw, gb, sc, &segs, err);
   } else if (layer == 2) {
     typedef NatConv3 C3;
     const int rows = n * C3::OH * C3::OW;
     tc_wgrad<ConvSrc<C3>, GradSrc<64>, 2, 64, 5, 64>(lc, KID_CONV3_WGRAD, ConvSrc<C3>{(const bf16*)act[1], rows},
-                                                     GradSrc<64>{g, 64, rows}, rows, 9, 1.f, gw, gb, scratch, err);
+                                                     GradSrc<64>{g, 64, rows}, rows, 9, 1.f, gw, gb, sc, &segs, err);
   } else {
     tc_wgrad<PlainSrc, GradSrc<64>, 1, 128, 6, 512>(lc, KID_FC_WGRAD, PlainSrc{(const bf16*)act[2], 3136, n},
-                                                    GradSrc<64>{g, 512, n}, n, 49, 1.f, gw, gb, scratch, err);
+                                                    GradSrc<64>{g, 512, n}, n, 49, 1.f, gw, gb, sc, &segs, err);
   }
 }
 
