@@ -25,6 +25,9 @@ sys.path.insert(0, ROOT)
 from paper_1705_04862_b200.configs import COMMON, CONFIGS  # noqa: E402
 
 FRAME_BYTES = 84 * 84 * 4
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of a kernel family from the ncu capture summarised
+# under profiles/ (bytes); an entry is dropped when its kernel changes after the capture
+NCU_TRAFFIC = {}
 
 
 # ----------------------------------------------------------------------------- workload arithmetic
@@ -36,8 +39,10 @@ def net_layers(arch):
 
 
 def kernel_work(cfg):
-    """Algorithmic FLOPs (2 x MAC, unpadded) or bytes of ONE launch of each kernel family, and the
-    roofline that bounds it.  n = n_e for rollout kernels, B = n_e * t_max for update kernels."""
+    """Per kernel family: (roofline that bounds it, algorithmic FLOPs (2 x MAC, unpadded) or bytes of ONE logical
+    launch, logical launches per iteration).  A logical launch may be more than one kernel (the fully
+    connected forward is a split-k GEMM plus its finishing kernel).  Rollout kernels see n_e states per launch,
+    update kernels B = n_e * t_max."""
     layers, F = net_layers(cfg["arch"])
     n_e, T, A = cfg["n_e"], cfg["t_max"], cfg["n_actions"]
     B = n_e * T
@@ -46,15 +51,15 @@ def kernel_work(cfg):
     w = {}
     for name, rows, N, K in layers:
         mac = rows * N * K
-        w[name + "_fwd"] = ("tensor", 2.0 * mac * n_e)
-        w[name + "_wgrad"] = ("tensor", 2.0 * mac * B)
+        w[name + "_fwd"] = ("tensor", 2.0 * mac * n_e, T + 1)
+        w[name + "_wgrad"] = ("tensor", 2.0 * mac * B, 1)
         if name != "conv1":
-            w[name + "_dgrad"] = ("tensor", 2.0 * mac * B)
-    w["heads_fwd_sample"] = ("tensor", 2.0 * (A + 1) * F * n_e)
-    w["heads_bwd"] = ("tensor", 2.0 * (A + 1) * F * B)          # per launch (dgrad or wgrad)
-    w["env_step"] = ("hbm", n_e * (FRAME_BYTES + 6.0))
-    w["clip_rmsprop"] = ("hbm", P * (22.0 if elt == 2 else 20.0))
-    w["grad_sumsq"] = ("hbm", P * 4.0)
+            w[name + "_dgrad"] = ("tensor", 2.0 * mac * B, 1)
+    w["heads_fwd_sample"] = ("tensor", 2.0 * (A + 1) * F * n_e, T + 1)
+    w["heads_bwd"] = ("tensor", 4.0 * (A + 1) * F * B, 1)
+    w["env_step"] = ("hbm", n_e * (FRAME_BYTES + 6.0), T)
+    w["clip_rmsprop"] = ("hbm", P * (22.0 if elt == 2 else 20.0), 1)
+    w["grad_sumsq"] = ("hbm", P * 4.0, 1)
     return w, P
 
 
@@ -74,6 +79,22 @@ def peaks():
         return dict(hbm=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d.get("bf16_tflops_sustained"),
                     src="measured")
     return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, src="fallback")
+
+
+# ----------------------------------------------------------------------------- ranks
+def max_over_ranks(x, dist=None, device="cpu"):
+    """Largest value of x over the ranks of the job (x itself without a process group)."""
+    if dist is None:
+        return float(x)
+    import torch
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank, world, ms_per_step):
+    """Units all ranks processed per second, given the slowest rank's time per step (replicas: weak scaling)."""
+    return world * units_per_rank / (ms_per_step * 1e-3)
 
 
 # ----------------------------------------------------------------------------- clocks
@@ -222,12 +243,9 @@ def run_ours(args, cfg):
     total_ms = ev[0].elapsed_time(ev[2 * K])
     roll_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(K)) / K
     upd_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(K)) / K
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, "cuda")
     ms_per_step = total_ms / K
-    value = world * n_e * T / (ms_per_step * 1e-3)
+    value = whole_job_value(n_e * T, world, ms_per_step)
 
     # ---- per-kernel CUDA-event breakdown over another K steps (same kernels, event pairs around each)
     g.profile(True)
@@ -267,11 +285,8 @@ def run_ours(args, cfg):
             e2e_step()
         barrier()
         e_sec = (time.time() - w0) / Ke
-        if dist is not None:
-            t = torch.tensor([e_sec], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_sec = float(t.item())
-        e2e = {"value": world * n_e * T / e_sec, "unit": "env-steps/s", "ms_per_step": e_sec * 1e3,
+        e_sec = max_over_ranks(e_sec, dist, "cuda")
+        e2e = {"value": whole_job_value(n_e * T, world, e_sec * 1e3), "unit": "env-steps/s", "ms_per_step": e_sec * 1e3,
                "h2d_bytes_per_step": (T + 1) * n_e * FRAME_BYTES + 2 * T * n_e,
                "d2h_bytes_per_step": T * n_e * 4 + (T + 1) * n_e * 4 + 32,
                "api": "paac_act_host / paac_observe_host / paac_update, pinned host buffers, wall clock"}
@@ -288,20 +303,24 @@ def run_ours(args, cfg):
     tot = sum(ms for ms, _ in prof.values())
     shares = {k: {"ms_per_step": ms / K, "launches_per_step": n / K, "share": ms / tot} for k, (ms, n) in prof.items()}
     dom = max(prof, key=lambda k: prof[k][0])
-    dom_ms = prof[dom][0] / prof[dom][1]
-    bound, amount = work.get(dom, ("hbm", 0.0))
+    bound, amount, logical = work.get(dom, ("hbm", 0.0, 1))
+    dom_ms = prof[dom][0] / K / logical                    # device time of one logical launch
     if bound == "tensor":
         ach, peak, unit = amount / (dom_ms * 1e-3) / 1e12, pk["bf16"], "TFLOP/s"
     else:
         ach, peak, unit = amount / (dom_ms * 1e-3) / 1e9, pk["hbm"], "GB/s"
     roofline = {"kernel": dom, "bound": bound, "achieved": ach, "peak": peak, "unit": unit, "frac": ach / peak,
-                "traffic": None, "peak_source": pk["src"], "avg_launch_ms": dom_ms,
+                "traffic": NCU_TRAFFIC.get((cfg["name"], dom)), "peak_source": pk["src"], "avg_launch_ms": dom_ms,
                 "algorithmic_per_launch": amount}
     side = {}
     for k in ("env_step", "clip_rmsprop", "grad_sumsq"):
         if k in prof and prof[k][1]:
-            gbs = work[k][1] / (prof[k][0] / prof[k][1] * 1e-3) / 1e9
+            gbs = work[k][1] / (prof[k][0] / K / work[k][2] * 1e-3) / 1e9
             side[k] = {"GB/s": gbs, "frac_of_%s_hbm" % pk["src"]: gbs / pk["hbm"]}
+    per_family = {}
+    for k, (ms, n) in prof.items():
+        if k in work and work[k][0] == "tensor":
+            per_family[k] = work[k][1] * work[k][2] / (ms / K * 1e-3) / 1e12
     roll_flops, upd_flops = iteration_flops(cfg)
 
     # ---- CPU oracle on a bounded sample (rank 0, one GPU only)
@@ -320,7 +339,10 @@ def run_ours(args, cfg):
         "updates_per_sec": world * 1e3 / ms_per_step, "rollout_ms": roll_ms, "update_ms": upd_ms,
         "update_tflops": upd_flops / (upd_ms * 1e-3) / 1e12,
         "update_frac_of_bf16_peak": upd_flops / (upd_ms * 1e-3) / 1e12 / pk["bf16"],
+        "update_frac_of_bf16_sustained": (upd_flops / (upd_ms * 1e-3) / 1e12 / pk["bf16_sustained"]
+                                          if pk.get("bf16_sustained") else None),
         "rollout_tflops": roll_flops / (roll_ms * 1e-3) / 1e12,
+        "kernel_tflops": per_family,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "hbm_kernels": side,
         "kernels": shares, "cpu_baseline": cpu,
     }
