@@ -133,7 +133,8 @@ void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, uin
   for (int l = 0; l <= c->nd.n_conv; ++l)
     act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
   if (use_tc(c))
-    tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, frames, c->n_e, act, c->scratch, &c->stats->error_word);
+    tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, c->w_images, frames, c->n_e, act, c->scratch,
+               &c->stats->error_word);
   else
     simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
   const size_t row = (size_t)slot * c->n_e;

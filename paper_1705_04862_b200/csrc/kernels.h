@@ -28,7 +28,7 @@ size_t simt_scratch_floats(int arch, const NetDims& nd, int n);
 bool tc_supported(int arch, int prec);
 // fc_scratch: tc_fc_scratch_floats(n) floats for the split-k partial sums of the fully connected layer
 size_t tc_fc_scratch_floats(int n);
-void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* theta16,
+void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* theta16, const bf16* images,
                 const uint8_t* frames, int n, void* const act[], float* fc_scratch, uint32_t* error_word);
 // transposed / regrouped bf16 weight images the backward contractions read (refreshed after every
 // parameter change), and the data-gradient kernels that use them

@@ -21,6 +21,10 @@ namespace paac {
 using namespace tc;
 
 constexpr int TC_BM = 128, TC_BK = 64, TC_THREADS = 160;
+// element offsets of the regrouped weight images (see relayout_weights_kernel)
+constexpr size_t TC_IMG_W2 = 0, TC_IMG_W3 = 4 * 32 * 256, TC_IMG_WFC = TC_IMG_W3 + 64 * 576,
+                 TC_IMG_W1 = TC_IMG_WFC + (size_t)3136 * 512, TC_IMG_END = TC_IMG_W1 + 32 * 256;
+
 
 struct TcShared {
   uint64_t full[8], empty[8], acc;
@@ -933,33 +937,40 @@ __device__ __forceinline__ void u8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_
   hi = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
 }
 
+// Space-to-depth view: with stride 4 and an 8 x 8 kernel, the window of output (oh, ow) is the 2 x 2 group of
+// 4 x 4-pixel blocks (oh + i, ow + j), i, j in {0, 1}.  A block is 4 x 4 x 4 channels = 64 values = one 128-byte
+// bf16 operand row, so the layer is a 2 x 2, stride-1 convolution over the 21 x 21 raster of blocks and runs
+// as four shifted views (0, 1, 21, 22 rows) of one staged row block, like the other convolutions.  Every input
+// byte is expanded to bf16 once per tile instead of once per window that contains it.
 constexpr int C1_THREADS = 416;      // warps 0-3 epilogue, 4-11 producers, 12 MMA
-constexpr int C1_RAW_BYTES = 14336;  // >= 40 frame rows of 336 bytes
+constexpr int C1_RAW_BYTES = 12288;  // >= 36 frame rows of 336 bytes
+constexpr int C1_STAGE_ROWS = 152, C1_USED_ROWS = 150, C1_RASTER = 21;
 
 template <class G, class Epi, int STAGES>
 __global__ void __launch_bounds__(C1_THREADS, 1)
-tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, Epi epi, int M, int tiles_m,
+tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, Epi epi, int n_states, int tiles,
                 uint32_t* error_word) {
-  static_assert(G::K * G::C == 32 && G::K == 8 && G::CO == 32, "window rows of 32 bytes, 32 output channels");
-  constexpr int BN = 32, KB = 4;
-  constexpr uint32_t A_BYTES = TC_BM * 128, B_BLOCK = BN * 128, B_BYTES = KB * B_BLOCK, RAW_BYTES = C1_RAW_BYTES;
+  static_assert(G::K == 8 && G::S == 4 && G::C == 4 && G::CO == 32 && G::H == 84 && G::W == 84, "geometry");
+  constexpr int BN = 32, NT = 4, NPROD = 256, POS = C1_RASTER * C1_RASTER, ROW_BYTES = G::W * G::C;
+  constexpr uint32_t A_BYTES = C1_STAGE_ROWS * 128, B_BLOCK = BN * 128, B_BYTES = NT * B_BLOCK, RAW_BYTES = C1_RAW_BYTES;
   extern __shared__ uint8_t dyn_smem[];
   __shared__ PkShared sh;
   const uint32_t b_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
   const uint32_t a_base0 = b_base + B_BYTES;
-  const uint32_t raw_base = a_base0 + STAGES * A_BYTES;       // ring of three slots of up to 40 frame rows
+  const uint32_t raw_base = a_base0 + STAGES * A_BYTES;       // ring of three slots of up to 36 frame rows
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_pos = n_states * POS;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], NPROD / 32); mbar_init(&sh.empty[s], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 4); }
     sh.abort = 0u;
     fence_barrier_init();
   }
   if (warp == 12) tmem_alloc(&sh.tmem_base, 2 * BN);
-  for (int i = threadIdx.x; i < KB * BN * 8; i += C1_THREADS) {
-    const int c = i & 7, row = (i >> 3) % BN, kb = i / (8 * BN);
-    cp_async16(b_base + kb * B_BLOCK + sw128_offset(row, c), w + ((size_t)row * KB + kb) * TC_BK + c * 8, 16u);
+  for (int i = threadIdx.x; i < NT * BN * 8; i += C1_THREADS) {     // weights regrouped per block tap: [32][4 * 64]
+    const int c = i & 7, row = (i >> 3) % BN, t = i / (8 * BN);
+    cp_async16(b_base + t * B_BLOCK + sw128_offset(row, c), w + ((size_t)row * NT + t) * TC_BK + c * 8, 16u);
   }
   cp_async_commit();
   cp_async_wait<0>();
@@ -971,21 +982,19 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
 
   if (warp >= 4 && warp < 12) {
     // ---------------- producers ----------------
-    // The 128 output pixels of a tile lie in at most two states and at most eight output rows, so their
-    // windows cover at most 40 whole frame rows, which are contiguous in memory per state: two plain byte
-    // ranges are copied into a ring slot two tiles ahead, and every window row is then read from there.
-    constexpr int ROW_BYTES = G::W * G::C, POS = G::OH * G::OW, NPROD = 256;
-    const int p = threadIdx.x - 128, row = p & 127, half = p >> 7;
+    const int p = threadIdx.x - 128;
+    // block rows of a tile: raster positions q0 .. q0 + 149 (clamped to the last one), at most nine block rows in
+    // at most two states, i.e. at most 36 whole frame rows, contiguous per state
     auto tile_ranges = [&](int t, int& b0, int& r0, int& n0, int& n1) {
-      const int mf = t * TC_BM, ml = min(mf + TC_BM - 1, M - 1);
-      b0 = mf / POS;
-      const int b1 = ml / POS, ohf = (mf % POS) / G::OW, ohl = (ml % POS) / G::OW;
-      r0 = ohf * G::S;
-      if (b1 == b0) { n0 = (ohl - ohf) * G::S + G::K; n1 = 0; }
-      else { n0 = G::H - r0; n1 = ohl * G::S + G::K; }
+      const int qf = t * TC_BM, ql = min(qf + C1_USED_ROWS - 1, total_pos - 1);
+      b0 = qf / POS;
+      const int b1 = ql / POS, yf = (qf % POS) / C1_RASTER, yl = (ql % POS) / C1_RASTER;
+      r0 = 4 * yf;
+      if (b1 == b0) { n0 = 4 * (yl - yf + 1); n1 = 0; }
+      else { n0 = G::H - r0; n1 = 4 * (yl + 1); }
     };
     auto stage_rows = [&](int t, int slot) {
-      if (t < tiles_m) {
+      if (t < tiles) {
         int b0, r0, n0, n1;
         tile_ranges(t, b0, r0, n0, n1);
         const uint8_t* src0 = frames + ((size_t)b0 * G::H + r0) * ROW_BYTES;
@@ -1001,53 +1010,50 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
     bool alive = true;
     stage_rows(blockIdx.x, 0);
     stage_rows(blockIdx.x + gridDim.x, 1);
-    for (int t = blockIdx.x; t < tiles_m && alive; t += gridDim.x, ++local) {
+    for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x, ++local) {
       cp_async_wait<1>();                                              // this tile's rows (my share) have landed
       asm volatile("bar.sync 1, %0;" ::"n"(NPROD) : "memory");        // everyone's share has; the slot of tile-1 is free
       stage_rows(t + 2 * gridDim.x, (local + 2) % 3);
       int b0, r0, n0, n1;
       tile_ranges(t, b0, r0, n0, n1);
-      const int m = min(t * TC_BM + row, M - 1);
-      const int b = m / POS, rem = m % POS, oh = rem / G::OW, ow = rem % G::OW;
-      const int first = b == b0 ? oh * G::S - r0 : n0 + oh * G::S;     // slot row of this pixel's window top
-      const uint32_t my_raw = raw_base + (local % 3) * RAW_BYTES +
-                              (uint32_t)((first + 4 * half) * ROW_BYTES + ow * G::S * G::C);
-#pragma unroll
-      for (int q = 0; q < 2; ++q) {
-        const int kb = 2 * half + q, it = local * KB + kb, s = it % STAGES;
-        const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
-        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
-        const uint32_t dst = a_base0 + s * A_BYTES + row * 128u;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {            // window row 2q + c/2, half c&1 -> operand chunks 2c, 2c + 1 of this K block
-          uint32_t r0w, r1w, r2w, r3w;
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0w), "=r"(r1w), "=r"(r2w), "=r"(r3w)
-                       : "r"(my_raw + (uint32_t)((2 * q + (c >> 1)) * ROW_BYTES + (c & 1) * 16)) : "memory");
-          uint32_t o[8];
-          u8x4_to_bf16x4(r0w, o[0], o[1]); u8x4_to_bf16x4(r1w, o[2], o[3]);
-          u8x4_to_bf16x4(r2w, o[4], o[5]); u8x4_to_bf16x4(r3w, o[6], o[7]);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * c) ^ (row & 7)) << 4)),
-                       "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * c + 1) ^ (row & 7)) << 4)),
-                       "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.full[s]);
+      const int s = local % STAGES;
+      const bool ok = mbar_wait(&sh.empty[s], ((local / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+      if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+      const uint32_t stage = a_base0 + s * A_BYTES, raw = raw_base + (local % 3) * RAW_BYTES;
+      // work item = (block row ri of the stage, pixel row py of the block): 16 raw bytes -> two operand chunks
+      for (int item = p; item < C1_USED_ROWS * 4; item += NPROD) {
+        const int ri = item >> 2, py = item & 3;
+        const int q = min(t * TC_BM + ri, total_pos - 1);
+        const int b = q / POS, rem = q % POS, Y = rem / C1_RASTER, X = rem % C1_RASTER;
+        const int slot_row = (b == b0 ? 4 * Y - r0 : n0 + 4 * Y) + py;
+        uint32_t r0w, r1w, r2w, r3w, o[8];
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0w), "=r"(r1w), "=r"(r2w), "=r"(r3w)
+                     : "r"(raw + (uint32_t)(slot_row * ROW_BYTES + X * 16)) : "memory");
+        u8x4_to_bf16x4(r0w, o[0], o[1]); u8x4_to_bf16x4(r1w, o[2], o[3]);
+        u8x4_to_bf16x4(r2w, o[4], o[5]); u8x4_to_bf16x4(r3w, o[6], o[7]);
+        const uint32_t dst = stage + (uint32_t)ri * 128u;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py) ^ (ri & 7)) << 4)),
+                     "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py + 1) ^ (ri & 7)) << 4)),
+                     "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
       }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.full[s]);
     }
     cp_async_wait<0>();
   } else if (warp < 4) {
     // ---------------- epilogue ----------------
     int local = 0;
-    for (int t = blockIdx.x; t < tiles_m; t += gridDim.x, ++local) {
-      const int ab = local & 1, m = t * TC_BM + threadIdx.x;
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
+      const int ab = local & 1, pos = t * TC_BM + threadIdx.x;
       const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
       uint32_t r[32];
       tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN, r);
-      epi(m, 0, 0, r);
+      const int b = pos / POS, rem = pos % POS, Y = rem / C1_RASTER, X = rem % C1_RASTER;
+      if (b < n_states && Y < G::OH && X < G::OW) epi((b * G::OH + Y) * G::OW + X, 0, 0, r);
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
@@ -1055,26 +1061,28 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
   } else if (warp == 12 && lane == 0) {
     // ---------------- MMA issuer ----------------
     constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
-    int it = 0, local = 0;
+    const uint32_t hi = desc_hi_kmajor_sw128(), b_lo = (b_base >> 4) & 0x3FFFu;
+    int local = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < tiles_m && ok; t += gridDim.x, ++local) {
-      const int ab = local & 1;
+    for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++local) {
+      const int ab = local & 1, s = local % STAGES;
       ok = mbar_wait(&sh.acc_empty[ab], ((local >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!ok) break;
+      ok = mbar_wait(&sh.full[s], (local / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      if (!ok) break;
       tcgen05_fence_after();
-      for (int kb = 0; kb < KB; ++kb, ++it) {
-        const int s = it % STAGES;
-        ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
-        if (!ok) break;
-        tcgen05_fence_after();
-        const uint32_t a_addr = a_base0 + s * A_BYTES, b_addr = b_base + kb * B_BLOCK;
+      const uint32_t a_lo = ((a_base0 + s * A_BYTES) >> 4) & 0x3FFFu, d = tmem + ab * BN;
 #pragma unroll
-        for (int k = 0; k < TC_BK / 16; ++k)
-          mma_bf16(tmem + ab * BN, make_smem_desc(a_addr + k * 32, 0, 1024, SWIZZLE_128B),
-                   make_smem_desc(b_addr + k * 32, 0, 1024, SWIZZLE_128B), idesc, (kb | k) != 0 ? 1u : 0u);
-        mma_commit(&sh.empty[s]);
+      for (int tap = 0; tap < NT; ++tap) {
+        const uint32_t a_off = (((tap >> 1) * C1_RASTER + (tap & 1)) * 128u) >> 4, b_off = (tap * B_BLOCK) >> 4;
+#pragma unroll
+        for (int k = 0; k < TC_BK / 16; ++k) {
+          if (tap == 0 && k == 0) mma_bf16_lo<false>(d, a_lo + a_off, b_lo + b_off, hi, idesc);
+          else mma_bf16_lo<true>(d, a_lo + a_off + k * 2, b_lo + b_off + k * 2, hi, idesc);
+        }
       }
-      if (ok) mma_commit(&sh.acc_full[ab]);
+      mma_commit(&sh.empty[s]);
+      mma_commit(&sh.acc_full[ab]);
     }
   }
   tcgen05_fence_before();
@@ -1130,19 +1138,19 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
 }
 
 template <class G, class Epi>
-static void tc_conv1(LaunchCtx& lc, const uint8_t* frames, const bf16* w, Epi e, int M, uint32_t* err) {
-  constexpr int STAGES = 8;
-  constexpr int smem = 4 * 32 * 128 + STAGES * TC_BM * 128 + 3 * C1_RAW_BYTES + 1024;
+static void tc_conv1(LaunchCtx& lc, const uint8_t* frames, const bf16* w_blocks, Epi e, int n_states, uint32_t* err) {
+  constexpr int STAGES = 6;
+  constexpr int smem = 4 * 32 * 128 + STAGES * C1_STAGE_ROWS * 128 + 3 * C1_RAW_BYTES + 1024;
   auto kern = tc_conv1_kernel<G, Epi, STAGES>;
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     configured = true;
   }
-  const int tiles_m = (M + TC_BM - 1) / TC_BM;
-  const int gx = tiles_m < sm_count() ? tiles_m : sm_count();
+  const int tiles = (n_states * C1_RASTER * C1_RASTER + TC_BM - 1) / TC_BM;
+  const int gx = tiles < sm_count() ? tiles : sm_count();
   KernelScope scope(lc, KID_CONV1_FWD);
-  kern<<<gx, C1_THREADS, smem, lc.st>>>(frames, w, e, M, tiles_m, err);
+  kern<<<gx, C1_THREADS, smem, lc.st>>>(frames, w_blocks, e, n_states, tiles, err);
 }
 
 template <class ASrc, class BSrc, class Epi, int BN, int STAGES>
@@ -1186,16 +1194,16 @@ static void tc_fc_forward(LaunchCtx& lc, const bf16* a, const bf16* w, const flo
 // ---- forward ---------------------------------------------------------------------------------------------
 bool tc_supported(int arch, int prec) { return arch == PAAC_ARCH_NATURE && prec == PAAC_BF16; }
 
-void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* w, const uint8_t* frames,
-                int n, void* const act[], float* fc_scratch, uint32_t* err) {
+void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* w, const bf16* images,
+                const uint8_t* frames, int n, void* const act[], float* fc_scratch, uint32_t* err) {
   const LayerDims* d = nd.layer;
   const float s255 = 1.0f / 255.0f;
   if (arch != PAAC_ARCH_NATURE) return;   // the caller routes the smaller network to the CUDA-core path
   {
     typedef NatConv1 C1; typedef NatConv2 C2; typedef NatConv3 C3;
     const int M1 = n * C1::OH * C1::OW, M2 = n * C2::OH * C2::OW, M3 = n * C3::OH * C3::OW;
-    tc_conv1<C1, BiasReluEpiTc>(lc, frames, w + d[0].w_off, BiasReluEpiTc{(bf16*)act[0], theta + d[0].b_off, 32, s255, M1},
-                                M1, err);
+    tc_conv1<C1, BiasReluEpiTc>(lc, frames, images + TC_IMG_W1, BiasReluEpiTc{(bf16*)act[0], theta + d[0].b_off, 32, s255, M1},
+                                n, err);
     {
       typedef RasterMap<100, 10, 9, 9> Map;
       tc_shift<C2FwdCfg, ShiftBiasReluEpi<Map, 9, 9>, 64, 4>(
@@ -1791,13 +1799,21 @@ void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, 
 
 // ---- weight images for the backward contractions ------------------------------------------------------
 // From the canonical bf16 copy: wfc_t[i][o] = Wfc[o][i];  w3_d[ci][r][s][co] = W3[co][r][s][ci];
-// w2_d[z][ci][i][j][co] = W2[co][py + 2i][px + 2j][ci] with z = 2 py + px.
-__global__ void relayout_weights_kernel(const bf16* __restrict__ w2, const bf16* __restrict__ w3,
-                                        const bf16* __restrict__ wfc, bf16* __restrict__ w2_d,
-                                        bf16* __restrict__ w3_d, bf16* __restrict__ wfc_t) {
+// w2_d[z][ci][i][j][co] = W2[co][py + 2i][px + 2j][ci] with z = 2 py + px;
+// w1_b[co][2i + j][py][px][ci] = W1[co][4i + py][4j + px][ci] (the first layer's weights per 4 x 4 block tap).
+__global__ void relayout_weights_kernel(const bf16* __restrict__ w1, const bf16* __restrict__ w2,
+                                        const bf16* __restrict__ w3, const bf16* __restrict__ wfc,
+                                        bf16* __restrict__ w2_d, bf16* __restrict__ w3_d, bf16* __restrict__ wfc_t,
+                                        bf16* __restrict__ w1_b) {
   typedef NatConv2 C2; typedef NatConv3 C3;
-  constexpr int N2 = 4 * C2::C * 4 * C2::CO, N3 = C3::C * 9 * C3::CO, NF = 3136 * 512;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N2 + N3 + NF; i += gridDim.x * blockDim.x) {
+  constexpr int N2 = 4 * C2::C * 4 * C2::CO, N3 = C3::C * 9 * C3::CO, NF = 3136 * 512, N1 = 32 * 256;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N2 + N3 + NF + N1; i += gridDim.x * blockDim.x) {
+    if (i >= N2 + N3 + NF) {
+      const int j = i - N2 - N3 - NF, ci = j & 3, px = (j >> 2) & 3, py = (j >> 4) & 3, tap = (j >> 6) & 3, co = j >> 8;
+      const int r = 4 * (tap >> 1) + py, sx = 4 * (tap & 1) + px;
+      w1_b[j] = w1[((co * 8 + r) * 8 + sx) * 4 + ci];
+      continue;
+    }
     if (i < N2) {
       const int co = i % 64, t = (i / 64) % 4, ci = (i / 256) % 32, z = i / (256 * 32);
       const int r = (z >> 1) + 2 * (t >> 1), s = (z & 1) + 2 * (t & 1);
@@ -1811,13 +1827,14 @@ __global__ void relayout_weights_kernel(const bf16* __restrict__ w2, const bf16*
     }
   }
 }
-size_t tc_weight_image_elems() { return 4 * 32 * 256 + 64 * 576 + (size_t)3136 * 512; }
+size_t tc_weight_image_elems() { return TC_IMG_END; }
 
 void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, bf16* images) {
   const LayerDims* d = nd.layer;
   KernelScope scope(lc, KID_CAST);
-  relayout_weights_kernel<<<592, 256, 0, lc.st>>>(theta16 + d[1].w_off, theta16 + d[2].w_off, theta16 + d[3].w_off,
-                                                  images, images + 4 * 32 * 256, images + 4 * 32 * 256 + 64 * 576);
+  relayout_weights_kernel<<<592, 256, 0, lc.st>>>(theta16 + d[0].w_off, theta16 + d[1].w_off, theta16 + d[2].w_off,
+                                                  theta16 + d[3].w_off, images + TC_IMG_W2, images + TC_IMG_W3,
+                                                  images + TC_IMG_WFC, images + TC_IMG_W1);
 }
 
 // ---- backward: data gradients ---------------------------------------------------------------------------
