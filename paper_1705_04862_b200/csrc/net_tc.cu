@@ -539,12 +539,15 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
 // Cfg supplies: PLANES (row blocks staged per tile), NT (taps), STAGE_ROWS (multiple of 8, >= 128 + largest
 // shift), src(plane, g, valid) -> address of the 128 bytes of raster row g (valid = false: zeros),
 // tap_plane(t), tap_shift(t).  The weights are [BN][NT * 64] K-major, block t belonging to tap t.
-constexpr int SH_LAG = 2;
+constexpr int SH_LAG = 2, SH_THREADS = 416;     // warps 0-7 epilogue, 8-11 producers, 12 MMA
 
-template <class Cfg, class Epi, int BN, int STAGES>
-__global__ void __launch_bounds__(PK_THREADS, 1)
+// Consecutive MMAs go to NACC different accumulators in turn (any partition of the tap x k products sums to the
+// same result), so that an MMA does not have to wait for the one before it; the epilogue adds the NACC pieces.
+template <class Cfg, class Epi, int BN, int STAGES, int NACC>
+__global__ void __launch_bounds__(SH_THREADS, 1)
 tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_t* error_word) {
   static_assert(BN == 64 || BN == 128, "tile width");
+  static_assert(2 * NACC * BN <= 512 && (NACC == 1 || NACC == 2 || NACC == 4), "tensor memory budget");
   static_assert(STAGES >= SH_LAG + 2 && STAGES <= 8 && Cfg::STAGE_ROWS % 8 == 0, "pipeline shape");
   constexpr int NT = Cfg::NT, SR = Cfg::STAGE_ROWS, PLANES = Cfg::PLANES;
   constexpr uint32_t PLANE_BYTES = SR * 128, STAGE_BYTES = PLANES * PLANE_BYTES, B_BLOCK = BN * 128, B_BYTES = NT * B_BLOCK;
@@ -556,12 +559,12 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 8); }
     sh.abort = 0u;
     fence_barrier_init();
   }
-  if (warp == 8) tmem_alloc(&sh.tmem_base, 2 * BN);
-  for (int i = threadIdx.x; i < NT * BN * 8; i += PK_THREADS) {
+  if (warp == 12) tmem_alloc(&sh.tmem_base, 2 * NACC * BN);
+  for (int i = threadIdx.x; i < NT * BN * 8; i += SH_THREADS) {
     const int c = i & 7, row = (i >> 3) % BN, t = i / (8 * BN);
     cp_async16(b_base + t * B_BLOCK + sw128_offset(row, c), w + ((size_t)row * NT + t) * TC_BK + c * 8, 16u);
   }
@@ -573,9 +576,9 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
 
-  if (warp >= 4 && warp < 8) {
+  if (warp >= 8 && warp < 12) {
     // ---------------- producers: eight lanes per 128-byte row, 16 rows per pass ----------------
-    const int c = lane & 7, sub = (warp - 4) * 4 + (lane >> 3);
+    const int c = lane & 7, sub = (warp - 8) * 4 + (lane >> 3);
     int it = 0;
     bool alive = true;
     for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x, ++it) {
@@ -602,27 +605,36 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
     __syncwarp();
     if (alive && lane == 0)
       for (int j = it > SH_LAG ? it - SH_LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % STAGES]);
-  } else if (warp < 4) {
-    // ---------------- epilogue ----------------
+  } else if (warp < 8) {
+    // ---------------- epilogue: warps e and e + 4 share TMEM lane quarter e & 3 and split the columns ----------------
+    constexpr int COLS = BN / 2;
+    const int quarter = warp & 3, col0 = (warp >> 2) * COLS, rowi = quarter * 32 + lane;
     int local = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
-      const int ab = local & 1, pos = t * TC_BM + threadIdx.x;
-      typename Epi::template Pre<BN>::type pre;
-      epi.prefetch(pos, pre);
+      const int ab = local & 1, pos = t * TC_BM + rowi;
+      typename Epi::template Pre<COLS>::type pre;
+      epi.prefetch(pos, col0, pre);
       const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
 #pragma unroll
-      for (int cc = 0; cc < BN / 32; ++cc) {
+      for (int cc = 0; cc < COLS / 32; ++cc) {
         uint32_t r[32];
-        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN + cc * 32, r);
-        epi(pos, cc * 32, r, pre);
+        tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + ab * NACC * BN + col0 + cc * 32, r);
+#pragma unroll
+        for (int a = 1; a < NACC; ++a) {
+          uint32_t r2[32];
+          tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + (ab * NACC + a) * BN + col0 + cc * 32, r2);
+#pragma unroll
+          for (int q = 0; q < 32; ++q) r[q] = __float_as_uint(__uint_as_float(r[q]) + __uint_as_float(r2[q]));
+        }
+        epi(col0, cc * 32, r, pre);
       }
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
     }
-  } else if (lane == 0) {
+  } else if (warp == 12 && lane == 0) {
     // ---------------- MMA issuer ----------------
     constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
     int it = 0;
@@ -636,7 +648,7 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
       tcgen05_fence_after();
       // descriptor low words: (address >> 4); every operand slice is a compile-time offset from the stage
       const uint32_t a_lo = ((a_base0 + s * STAGE_BYTES) >> 4) & 0x3FFFu, b_lo = (b_base >> 4) & 0x3FFFu;
-      const uint32_t hi = desc_hi_kmajor_sw128(), d = tmem + ab * BN;
+      const uint32_t hi = desc_hi_kmajor_sw128(), d = tmem + ab * NACC * BN;
 #pragma unroll
       for (int tap = 0; tap < NT; ++tap) {
         constexpr uint32_t K_STEP = 32 >> 4;
@@ -644,8 +656,10 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
         const uint32_t b_off = (tap * B_BLOCK) >> 4;
 #pragma unroll
         for (int k = 0; k < TC_BK / 16; ++k) {
-          if (tap == 0 && k == 0) mma_bf16_lo<false>(d, a_lo + a_off, b_lo + b_off, hi, idesc);
-          else mma_bf16_lo<true>(d, a_lo + a_off + k * K_STEP, b_lo + b_off + k * K_STEP, hi, idesc);
+          constexpr int KS = TC_BK / 16;
+          const int m = tap * KS + k;                       // m-th MMA of the tile -> accumulator m % NACC
+          if (m < NACC) mma_bf16_lo<false>(d + (m % NACC) * BN, a_lo + a_off + k * K_STEP, b_lo + b_off + k * K_STEP, hi, idesc);
+          else mma_bf16_lo<true>(d + (m % NACC) * BN, a_lo + a_off + k * K_STEP, b_lo + b_off + k * K_STEP, hi, idesc);
         }
       }
       mma_commit(&sh.empty[s]);
@@ -654,10 +668,10 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
   }
   tcgen05_fence_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == 12) {
     __syncwarp();
     tcgen05_fence_after();
-    tmem_dealloc(tmem, 2 * BN);
+    tmem_dealloc(tmem, 2 * NACC * BN);
   }
 }
 
@@ -723,57 +737,74 @@ template <int RASTER, int WIDTH, int OUT_H, int OUT_W> struct RasterMap {
     return b < states && y < OUT_H && x < OUT_W;
   }
 };
-// An epilogue may fetch what it needs from global memory (the ReLU mask of the layer below) into `Pre`
-// before the accumulator is ready, so that the latency hides behind the tile's MMAs.
-struct NoPre {};
+// An epilogue thread finishes COLS consecutive columns (starting at col0) of its tile row.  It may fetch what
+// it needs from global memory (bias, the ReLU mask of the layer below) into `Pre` before the accumulator is
+// ready, so that the latency hides behind the tile's MMAs.
+template <int COLS> struct BiasPre { float b[COLS]; int row; bool valid; };
 template <class Map, int OUT_H, int OUT_W> struct ShiftBiasReluEpi {
-  template <int BN> struct Pre { typedef NoPre type; };
+  template <int COLS> struct Pre { typedef BiasPre<COLS> type; };
   Map map; bf16* out; const float* bias;
-  template <class P> __device__ __forceinline__ void prefetch(int, P&) const {}
-  template <class P> __device__ __forceinline__ void operator()(int pos, int n0, const uint32_t (&r)[32], const P&) const {
+  template <class P> __device__ __forceinline__ void prefetch(int pos, int col0, P& p) const {
     int b, y, x;
-    if (!map(pos, b, y, x)) return;
-    BiasReluEpiTc e{out, bias, 64, 1.f, 0x7fffffff};
-    e((b * OUT_H + y) * OUT_W + x, n0, 0, r);
+    p.valid = map(pos, b, y, x);
+    p.row = (b * OUT_H + y) * OUT_W + x;
+    const float4* b4 = reinterpret_cast<const float4*>(bias + col0);
+#pragma unroll
+    for (int j = 0; j < (int)(sizeof(p.b) / 16); ++j) {
+      const float4 t = __ldg(b4 + j);
+      p.b[4 * j] = t.x; p.b[4 * j + 1] = t.y; p.b[4 * j + 2] = t.z; p.b[4 * j + 3] = t.w;
+    }
+  }
+  // r = accumulator columns col0 + off .. + 31
+  template <class P> __device__ __forceinline__ void operator()(int col0, int off, const uint32_t (&r)[32], const P& p) const {
+    if (!p.valid) return;
+    uint32_t o[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      o[j] = pack_bf16x2(fmaxf(__uint_as_float(r[2 * j]) + p.b[off + 2 * j], 0.f),
+                         fmaxf(__uint_as_float(r[2 * j + 1]) + p.b[off + 2 * j + 1], 0.f));
+    uint4* dst = reinterpret_cast<uint4*>(out + (size_t)p.row * 64 + col0 + off);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
   }
 };
 template <class Map, int OUT_H, int OUT_W> struct ShiftReluMaskEpi {
-  template <int BN> struct Pre { typedef MaskPre<BN> type; };
+  template <int COLS> struct Pre { typedef MaskPre<COLS> type; };
   Map map; bf16* out; const bf16* act;
-  template <class P> __device__ __forceinline__ void prefetch(int pos, P& p) const {
+  template <class P> __device__ __forceinline__ void prefetch(int pos, int col0, P& p) const {
     int b, y, x;
     p.valid = map(pos, b, y, x);
-    p.idx = ((size_t)(b * OUT_H + y) * OUT_W + x) * 64;
+    p.idx = ((size_t)(b * OUT_H + y) * OUT_W + x) * 64 + col0;
     if (!p.valid) return;
     const uint4* a4 = reinterpret_cast<const uint4*>(act + p.idx);
 #pragma unroll
     for (int j = 0; j < (int)(sizeof(p.m) / sizeof(uint4)); ++j) p.m[j] = __ldg(a4 + j);
   }
-  template <class P> __device__ __forceinline__ void operator()(int, int n0, const uint32_t (&r)[32], const P& p) const {
-    if (p.valid) relu_mask_store_pre(out, p.idx + n0, r, &p.m[n0 / 8]);
+  template <class P> __device__ __forceinline__ void operator()(int, int off, const uint32_t (&r)[32], const P& p) const {
+    if (p.valid) relu_mask_store_pre(out, p.idx + off, r, &p.m[off / 8]);
   }
 };
-// stride-2 data gradient: column slice n0 is parity class n0 / 32 of raster pixel (yy, xx)
+// stride-2 data gradient: accumulator columns 32 c .. 32 c + 31 are parity class c of raster pixel (yy, xx)
 template <class Map> struct ShiftReluMaskEpiS2 {
-  template <int BN> struct Pre { typedef MaskPre<BN> type; };
+  template <int COLS> struct Pre { typedef MaskPre<COLS> type; };
   Map map; bf16* out; const bf16* act;
   __device__ __forceinline__ size_t class_idx(size_t base, int cls) const {      // base = pixel (2 yy, 2 xx)
     return base + (size_t)((cls >> 1) * 20 + (cls & 1)) * 32;
   }
-  template <class P> __device__ __forceinline__ void prefetch(int pos, P& p) const {
+  template <class P> __device__ __forceinline__ void prefetch(int pos, int col0, P& p) const {
     int b, yy, xx;
     p.valid = map(pos, b, yy, xx);
     p.idx = ((size_t)(b * 20 + 2 * yy) * 20 + 2 * xx) * 32;
     if (!p.valid) return;
 #pragma unroll
-    for (int cls = 0; cls < 4; ++cls) {
-      const uint4* a4 = reinterpret_cast<const uint4*>(act + class_idx(p.idx, cls));
+    for (int c = 0; c < (int)(sizeof(p.m) / (4 * sizeof(uint4))); ++c) {
+      const uint4* a4 = reinterpret_cast<const uint4*>(act + class_idx(p.idx, (col0 >> 5) + c));
 #pragma unroll
-      for (int j = 0; j < 4; ++j) p.m[4 * cls + j] = __ldg(a4 + j);
+      for (int j = 0; j < 4; ++j) p.m[4 * c + j] = __ldg(a4 + j);
     }
   }
-  template <class P> __device__ __forceinline__ void operator()(int, int n0, const uint32_t (&r)[32], const P& p) const {
-    if (p.valid) relu_mask_store_pre(out, class_idx(p.idx, n0 >> 5), r, &p.m[n0 / 8]);
+  template <class P> __device__ __forceinline__ void operator()(int col0, int off, const uint32_t (&r)[32], const P& p) const {
+    if (p.valid) relu_mask_store_pre(out, class_idx(p.idx, (col0 + off) >> 5), r, &p.m[off / 8]);
   }
 };
 
@@ -1122,11 +1153,11 @@ static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_t
   kern<<<dim3(gx, gy), PK_THREADS, smem, lc.st>>>(a, w, n_total, e, tiles_m, err);
 }
 
-template <class Cfg, class Epi, int BN, int STAGES>
+template <class Cfg, class Epi, int BN, int STAGES, int NACC>
 static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int positions, uint32_t* err) {
   constexpr int smem = Cfg::NT * BN * 128 + STAGES * Cfg::PLANES * Cfg::STAGE_ROWS * 128 + 1024;
   static_assert(smem <= 227 * 1024, "shared memory budget");
-  auto kern = tc_shift_kernel<Cfg, Epi, BN, STAGES>;
+  auto kern = tc_shift_kernel<Cfg, Epi, BN, STAGES, NACC>;
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -1134,7 +1165,7 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
   }
   const int tiles = (positions + TC_BM - 1) / TC_BM;
   KernelScope scope(lc, kid);
-  kern<<<tiles < sm_count() ? tiles : sm_count(), PK_THREADS, smem, lc.st>>>(cfg, w, e, tiles, err);
+  kern<<<tiles < sm_count() ? tiles : sm_count(), SH_THREADS, smem, lc.st>>>(cfg, w, e, tiles, err);
 }
 
 template <class G, class Epi>
@@ -1206,13 +1237,13 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
                                 n, err);
     {
       typedef RasterMap<100, 10, 9, 9> Map;
-      tc_shift<C2FwdCfg, ShiftBiasReluEpi<Map, 9, 9>, 64, 4>(
+      tc_shift<C2FwdCfg, ShiftBiasReluEpi<Map, 9, 9>, 64, 4, 1>(
           lc, KID_CONV2_FWD, C2FwdCfg{(const bf16*)act[0], n}, w + d[1].w_off,
           ShiftBiasReluEpi<Map, 9, 9>{Map{n}, (bf16*)act[1], theta + d[1].b_off}, n * 100, err);
     }
     {
       typedef RasterMap<81, 9, 7, 7> Map;
-      tc_shift<C3FwdCfg, ShiftBiasReluEpi<Map, 7, 7>, 64, 6>(
+      tc_shift<C3FwdCfg, ShiftBiasReluEpi<Map, 7, 7>, 64, 6, 1>(
           lc, KID_CONV3_FWD, C3FwdCfg{(const bf16*)act[1], n * 81}, w + d[2].w_off,
           ShiftBiasReluEpi<Map, 7, 7>{Map{n}, (bf16*)act[2], theta + d[2].b_off}, n * 81, err);
     }
@@ -1848,7 +1879,7 @@ void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* con
   typedef NatConv3 C3;
   const int M = n * C3::H * C3::W;
   typedef RasterMap<121, 11, 9, 9> Map;
-  tc_shift<C3DgradCfg, ShiftReluMaskEpi<Map, 9, 9>, 64, 6>(
+  tc_shift<C3DgradCfg, ShiftReluMaskEpi<Map, 9, 9>, 64, 6, 1>(
       lc, KID_CONV3_DGRAD, C3DgradCfg{(const bf16*)gact[2], n}, images + 4 * 32 * 256,
       ShiftReluMaskEpi<Map, 9, 9>{Map{n}, (bf16*)gact[1], (const bf16*)act[1]}, n * 121, err);
   (void)M;
@@ -1857,7 +1888,7 @@ void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* con
   typedef NatConv2 C2;
   const int M = n * (C2::H / 2) * (C2::W / 2);
   typedef RasterMap<121, 11, 10, 10> Map;
-  tc_shift<C2DgradCfg, ShiftReluMaskEpiS2<Map>, 128, 6>(
+  tc_shift<C2DgradCfg, ShiftReluMaskEpiS2<Map>, 128, 6, 1>(
       lc, KID_CONV2_DGRAD, C2DgradCfg{(const bf16*)gact[1], n}, images,
       ShiftReluMaskEpiS2<Map>{Map{n}, (bf16*)gact[0], (const bf16*)act[0]}, n * 121, err);
   (void)M;
