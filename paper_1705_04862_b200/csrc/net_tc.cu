@@ -539,7 +539,7 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
 // Cfg supplies: PLANES (row blocks staged per tile), NT (taps), STAGE_ROWS (multiple of 8, >= 128 + largest
 // shift), src(plane, g, valid) -> address of the 128 bytes of raster row g (valid = false: zeros),
 // tap_plane(t), tap_shift(t).  The weights are [BN][NT * 64] K-major, block t belonging to tap t.
-constexpr int SH_LAG = 2, SH_THREADS = 416;     // warps 0-7 epilogue, 8-11 producers, 12 MMA
+constexpr int SH_THREADS = 544;     // warps 0-7 epilogue, 8-15 producers, 16 MMA
 
 // Consecutive MMAs go to NACC different accumulators in turn (any partition of the tap x k products sums to the
 // same result), so that an MMA does not have to wait for the one before it; the epilogue adds the NACC pieces.
@@ -548,22 +548,25 @@ __global__ void __launch_bounds__(SH_THREADS, 1)
 tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_t* error_word) {
   static_assert(BN == 64 || BN == 128, "tile width");
   static_assert(2 * NACC * BN <= 512 && (NACC == 1 || NACC == 2 || NACC == 4), "tensor memory budget");
-  static_assert(STAGES >= SH_LAG + 2 && STAGES <= 8 && Cfg::STAGE_ROWS % 8 == 0, "pipeline shape");
+  static_assert(STAGES >= 2 && STAGES <= 8 && Cfg::STAGE_ROWS % 8 == 0, "pipeline shape");
   constexpr int NT = Cfg::NT, SR = Cfg::STAGE_ROWS, PLANES = Cfg::PLANES;
   constexpr uint32_t PLANE_BYTES = SR * 128, STAGE_BYTES = PLANES * PLANE_BYTES, B_BLOCK = BN * 128, B_BYTES = NT * B_BLOCK;
   extern __shared__ uint8_t dyn_smem[];
   __shared__ PkShared sh;
+  __shared__ int cell_table[Cfg::RASTER > 0 ? Cfg::RASTER : 1];   // per-state raster cell -> source offset (or -1)
   const uint32_t b_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
   const uint32_t a_base0 = b_base + B_BYTES;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 256); mbar_init(&sh.empty[s], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 8); }
     sh.abort = 0u;
     fence_barrier_init();
   }
-  if (warp == 12) tmem_alloc(&sh.tmem_base, 2 * NACC * BN);
+  if (warp == 16) tmem_alloc(&sh.tmem_base, 2 * NACC * BN);
+  if constexpr (Cfg::RASTER > 0)
+    for (int i = threadIdx.x; i < Cfg::RASTER; i += SH_THREADS) cell_table[i] = Cfg::cell(i);
   for (int i = threadIdx.x; i < NT * BN * 8; i += SH_THREADS) {
     const int c = i & 7, row = (i >> 3) % BN, t = i / (8 * BN);
     cp_async16(b_base + t * B_BLOCK + sw128_offset(row, c), w + ((size_t)row * NT + t) * TC_BK + c * 8, 16u);
@@ -576,8 +579,8 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
 
-  if (warp >= 8 && warp < 12) {
-    // ---------------- producers: eight lanes per 128-byte row, 16 rows per pass ----------------
+  if (warp >= 8 && warp < 16) {
+    // ---------------- producers: eight lanes per 128-byte row, 32 rows per pass ----------------
     const int c = lane & 7, sub = (warp - 8) * 4 + (lane >> 3);
     int it = 0;
     bool alive = true;
@@ -586,25 +589,19 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
       const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
       if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
       const uint32_t stage = a_base0 + s * STAGE_BYTES;
-      for (int idx = sub; idx < PLANES * SR; idx += 16) {
-        const int plane = idx / SR, ri = idx % SR;
+      for (int idx = sub; idx < PLANES * SR; idx += 32) {
+        const int plane = PLANES == 1 ? 0 : idx / SR, ri = PLANES == 1 ? idx : idx % SR;
         bool valid;
-        const bf16* src = cfg.src(plane, t * TC_BM + ri, valid);
+        const bf16* src;
+        if constexpr (Cfg::RASTER > 0) src = cfg.src_cell(t * TC_BM + ri, cell_table, valid);
+        else src = cfg.src(plane, t * TC_BM + ri, valid);
         cp_async16(stage + plane * PLANE_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), src + c * 8, valid ? 16u : 0u);
       }
-      cp_async_commit();
-      if (it >= SH_LAG) {
-        cp_async_wait<SH_LAG>();
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.full[(it - SH_LAG) % STAGES]);
-      }
+      // no waiting here: the hardware arrives on the stage's barrier for this thread when its copies have landed
+      cp_async_mbar_arrive(&sh.full[s]);
     }
+    cp_async_commit();
     cp_async_wait<0>();
-    fence_proxy_async_smem();
-    __syncwarp();
-    if (alive && lane == 0)
-      for (int j = it > SH_LAG ? it - SH_LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % STAGES]);
   } else if (warp < 8) {
     // ---------------- epilogue: warps e and e + 4 share TMEM lane quarter e & 3 and split the columns ----------------
     constexpr int COLS = BN / 2;
@@ -634,7 +631,7 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
     }
-  } else if (warp == 12 && lane == 0) {
+  } else if (warp == 16 && lane == 0) {
     // ---------------- MMA issuer ----------------
     constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
     int it = 0;
@@ -645,6 +642,7 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
       if (!ok) break;
       ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
       if (!ok) break;
+      fence_proxy_async_smem();        // the copies observed through the barrier -> visible to the MMA's operand reads
       tcgen05_fence_after();
       // descriptor low words: (address >> 4); every operand slice is a compile-time offset from the stage
       const uint32_t a_lo = ((a_base0 + s * STAGE_BYTES) >> 4) & 0x3FFFu, b_lo = (b_base >> 4) & 0x3FFFu;
@@ -668,7 +666,7 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
   }
   tcgen05_fence_before();
   __syncthreads();
-  if (warp == 12) {
+  if (warp == 16) {
     __syncwarp();
     tcgen05_fence_after();
     tmem_dealloc(tmem, 2 * NACC * BN);
@@ -677,7 +675,7 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
 
 // conv3 forward: rows = the 9 x 9 x 64 input pixels in memory order; tap (r, s) is 9 r + s rows down
 struct C3FwdCfg {
-  static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152;
+  static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152, RASTER = 0;      // RASTER = 0: no cell table
   const bf16* x; int rows;                                   // rows = states * 81
   __device__ __forceinline__ const bf16* src(int, int g, bool& valid) const {
     valid = g < rows;
@@ -690,7 +688,7 @@ struct C3FwdCfg {
 // order seen as [state][y][10 pairs]; even and odd image rows go to separate planes, so that tap row r
 // lives in plane r & 1, 10 (r >> 1) + (pair offset) rows down, and tile rows run over a 10 x 10 raster
 struct C2FwdCfg {
-  static constexpr int PLANES = 2, NT = 8, STAGE_ROWS = 144;
+  static constexpr int PLANES = 2, NT = 8, STAGE_ROWS = 144, RASTER = 0;
   const bf16* x; int states;
   __device__ __forceinline__ const bf16* src(int plane, int g, bool& valid) const {
     // plane row g = (b, oh, X) is pair row 2 g - X + 10 plane of the input in memory order
@@ -703,12 +701,17 @@ struct C2FwdCfg {
 // conv3 data gradient: the 7 x 7 x 64 output gradient on a zero-padded 11 x 11 raster; input pixel (y, x) is
 // raster position 11 y + x and tap (r, s) reads (2 - r) * 11 + (2 - s) rows down
 struct C3DgradCfg {
-  static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152;
+  static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152, RASTER = 121;
   const bf16* g3; int states;
-  __device__ __forceinline__ const bf16* src(int, int g, bool& valid) const {
-    const int b = g / 121, rem = g % 121, Y = rem / 11, X = rem % 11;
-    valid = b < states && Y >= 2 && Y <= 8 && X >= 2 && X <= 8;
-    return valid ? g3 + ((size_t)b * 49 + (Y - 2) * 7 + (X - 2)) * 64 : g3;
+  // element offset of raster cell `rem` inside a state's 7 x 7 x 64 gradient, or -1 for a padding cell
+  __device__ static __forceinline__ int cell(int rem) {
+    const int Y = rem / 11, X = rem % 11;
+    return (Y >= 2 && Y <= 8 && X >= 2 && X <= 8) ? ((Y - 2) * 7 + (X - 2)) * 64 : -1;
+  }
+  __device__ __forceinline__ const bf16* src_cell(int g, const int* table, bool& valid) const {
+    const int b = g / RASTER, off = table[g - b * RASTER];
+    valid = b < states && off >= 0;
+    return valid ? g3 + (size_t)b * 49 * 64 + off : g3;
   }
   __host__ __device__ static constexpr int tap_plane(int) { return 0; }
   __host__ __device__ static constexpr int tap_shift(int t) { return (2 - t / 3) * 11 + (2 - t % 3); }
@@ -716,12 +719,16 @@ struct C3DgradCfg {
 // conv2 data gradient (all four parity classes along N): the 9 x 9 x 64 gradient on a zero-padded 11 x 11
 // raster; class pixel (yy, xx) is position 11 yy + xx and tap (i, j) reads (1 - i) * 11 + (1 - j) rows down
 struct C2DgradCfg {
-  static constexpr int PLANES = 1, NT = 4, STAGE_ROWS = 144;
+  static constexpr int PLANES = 1, NT = 4, STAGE_ROWS = 144, RASTER = 121;
   const bf16* g2; int states;
-  __device__ __forceinline__ const bf16* src(int, int g, bool& valid) const {
-    const int b = g / 121, rem = g % 121, Y = rem / 11, X = rem % 11;
-    valid = b < states && Y >= 1 && Y <= 9 && X >= 1 && X <= 9;
-    return valid ? g2 + ((size_t)b * 81 + (Y - 1) * 9 + (X - 1)) * 64 : g2;
+  __device__ static __forceinline__ int cell(int rem) {
+    const int Y = rem / 11, X = rem % 11;
+    return (Y >= 1 && Y <= 9 && X >= 1 && X <= 9) ? ((Y - 1) * 9 + (X - 1)) * 64 : -1;
+  }
+  __device__ __forceinline__ const bf16* src_cell(int g, const int* table, bool& valid) const {
+    const int b = g / RASTER, off = table[g - b * RASTER];
+    valid = b < states && off >= 0;
+    return valid ? g2 + (size_t)b * 81 * 64 + off : g2;
   }
   __host__ __device__ static constexpr int tap_plane(int) { return 0; }
   __host__ __device__ static constexpr int tap_shift(int t) { return (1 - (t >> 1)) * 11 + (1 - (t & 1)); }

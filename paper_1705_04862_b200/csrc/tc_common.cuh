@@ -143,6 +143,12 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// the calling thread's arrival on `bar` is triggered by the hardware once all of its earlier cp.async copies have
+// landed; it counts as one of the arrivals the barrier was initialised to expect (.noinc)
+__device__ __forceinline__ void cp_async_mbar_arrive(uint64_t* bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
 // ---- shared-memory images ----------------------------------------------------------------------
 // 128-byte swizzle: within each 1024-byte group of eight 128-byte rows, the 16-byte chunk c of
 // row r lives at chunk position c ^ (r & 7).  The same image serves a K-major operand (rows =
