@@ -242,6 +242,11 @@ __device__ __forceinline__ void relu_mask_store(bf16* out, const bf16* act, size
     dst[j] = make_uint4(o[0], o[1], o[2], o[3]);
   }
 }
+// value words (two bf16 each) survive where the activation word's halves are non-zero
+__device__ __forceinline__ uint32_t mask_pair(uint32_t v, uint32_t a) {
+  return v & ((a & 0x7FFFu ? 0xFFFFu : 0u) | (a & 0x7FFF0000u ? 0xFFFF0000u : 0u));
+}
+
 // the same with the 32 activations of the slice already in registers (four 16-byte words)
 __device__ __forceinline__ void relu_mask_store_pre(bf16* out, size_t idx, const uint32_t (&r)[32], const uint4* a4) {
   uint4* dst = reinterpret_cast<uint4*>(out + idx);
@@ -604,19 +609,36 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
     cp_async_wait<0>();
   } else if (warp < 8) {
     // ---------------- epilogue: warps e and e + 4 share TMEM lane quarter e & 3 and split the columns ----------------
-    constexpr int COLS = BN / 2;
-    const int quarter = warp & 3, col0 = (warp >> 2) * COLS, rowi = quarter * 32 + lane;
+    constexpr int COLS = BN / 2, CH = COLS / 8, RPP = 32 / CH, ROWB = COLS * 2;   // 16-byte chunks per row part
+    const int quarter = warp & 3, col0 = (warp >> 2) * COLS;
+    const uint32_t stg = a_base0 + STAGES * STAGE_BYTES + warp * (32 * ROWB);    // this warp's staging tile
+    const int rr0 = lane / CH, ch = lane % CH;
     int local = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
-      const int ab = local & 1, pos = t * TC_BM + rowi;
-      typename Epi::template Pre<COLS>::type pre;
-      epi.prefetch(pos, col0, pre);
+      const int ab = local & 1, pos0 = t * TC_BM + quarter * 32;
+      // where this lane's chunks go (and, for masked epilogues, the activations there), before the tile is ready
+      uint32_t idx[CH];                                          // element offsets (every tensor here is < 2^32 elements)
+      uint4 m[CH];
+      uint32_t valid = 0;
+      {
+        int b, y, x;
+        epi.map.split(pos0 + rr0, b, y, x);
+#pragma unroll
+        for (int p = 0; p < CH; ++p) {
+          idx[p] = epi.index(b, y, x, col0 + ch * 8);
+          if (epi.map.is_output(b, y, x)) {
+            valid |= 1u << p;
+            if (Epi::MASK) m[p] = __ldg(reinterpret_cast<const uint4*>(epi.act + idx[p]));
+          }
+          epi.map.advance(b, y, x, RPP);
+        }
+      }
       const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
 #pragma unroll
       for (int cc = 0; cc < COLS / 32; ++cc) {
-        uint32_t r[32];
+        uint32_t r[32], o[16];
         tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + ab * NACC * BN + col0 + cc * 32, r);
 #pragma unroll
         for (int a = 1; a < NACC; ++a) {
@@ -625,11 +647,27 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
 #pragma unroll
           for (int q = 0; q < 32; ++q) r[q] = __float_as_uint(__uint_as_float(r[q]) + __uint_as_float(r2[q]));
         }
-        epi(col0, cc * 32, r, pre);
+        epi.values(col0 + cc * 32, r, o);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * ROWB + ((uint32_t)((cc * 4 + q) ^ (lane & (CH - 1))) << 4)),
+                       "r"(o[4 * q]), "r"(o[4 * q + 1]), "r"(o[4 * q + 2]), "r"(o[4 * q + 3]) : "memory");
       }
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
+      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);            // the accumulator is free again
+#pragma unroll
+      for (int p = 0; p < CH; ++p) {
+        const int rr = p * RPP + rr0;
+        uint4 v;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                     : "r"(stg + rr * ROWB + ((uint32_t)(ch ^ (rr & (CH - 1))) << 4)) : "memory");
+        if ((valid >> p) & 1u) {
+          if (Epi::MASK) { v.x = mask_pair(v.x, m[p].x); v.y = mask_pair(v.y, m[p].y); v.z = mask_pair(v.z, m[p].z); v.w = mask_pair(v.w, m[p].w); }
+          *reinterpret_cast<uint4*>(epi.out + idx[p]) = v;
+        }
+      }
+      __syncwarp();                                              // staging tile free for the next tile
     }
   } else if (warp == 16 && lane == 0) {
     // ---------------- MMA issuer ----------------
@@ -737,84 +775,63 @@ struct C2DgradCfg {
 // epilogues of the shifted kernels: raster position -> output row, or nothing for a margin position
 template <int RASTER, int WIDTH, int OUT_H, int OUT_W> struct RasterMap {
   int states;
-  __device__ __forceinline__ bool operator()(int pos, int& b, int& y, int& x) const {
+  __device__ __forceinline__ void split(int pos, int& b, int& y, int& x) const {
     b = pos / RASTER;
-    const int rem = pos % RASTER;
-    y = rem / WIDTH; x = rem % WIDTH;
-    return b < states && y < OUT_H && x < OUT_W;
+    const int rem = pos - b * RASTER;
+    y = rem / WIDTH; x = rem - y * WIDTH;
   }
+  // n raster cells further (n < WIDTH)
+  __device__ __forceinline__ void advance(int& b, int& y, int& x, int n) const {
+    x += n;
+    if (x >= WIDTH) { x -= WIDTH; if (++y >= RASTER / WIDTH) { y = 0; ++b; } }
+  }
+  __device__ __forceinline__ bool is_output(int b, int y, int x) const { return b < states && y < OUT_H && x < OUT_W; }
 };
-// An epilogue thread finishes COLS consecutive columns (starting at col0) of its tile row.  It may fetch what
-// it needs from global memory (bias, the ReLU mask of the layer below) into `Pre` before the accumulator is
-// ready, so that the latency hides behind the tile's MMAs.
-template <int COLS> struct BiasPre { float b[COLS]; int row; bool valid; };
+// Epilogues of the shifted kernels work in two phases per tile.  First the thread that owns a TMEM lane turns
+// its row's accumulators into bf16 (`values`) and parks them in a swizzled shared-memory staging tile.  Then
+// the warp re-reads the tile with eight (or four) lanes per row, so that every global access of a warp
+// instruction covers whole contiguous rows: `locate` gives the output element of (raster position, column),
+// and epilogues with MASK also fetch the activation there and zero the value where the activation is zero
+// (the gradient through the ReLU of the layer below).  Row-per-thread global accesses, 32 cache lines per
+// instruction, were what bounded these kernels before.
 template <class Map, int OUT_H, int OUT_W> struct ShiftBiasReluEpi {
-  template <int COLS> struct Pre { typedef BiasPre<COLS> type; };
-  Map map; bf16* out; const float* bias;
-  template <class P> __device__ __forceinline__ void prefetch(int pos, int col0, P& p) const {
-    int b, y, x;
-    p.valid = map(pos, b, y, x);
-    p.row = (b * OUT_H + y) * OUT_W + x;
-    const float4* b4 = reinterpret_cast<const float4*>(bias + col0);
+  static constexpr bool MASK = false;
+  Map map; bf16* out; const float* bias; const bf16* act;       // act unused
+  __device__ __forceinline__ void values(int col, const uint32_t (&r)[32], uint32_t (&o)[16]) const {
+    const float4* b4 = reinterpret_cast<const float4*>(bias + col);
 #pragma unroll
-    for (int j = 0; j < (int)(sizeof(p.b) / 16); ++j) {
+    for (int j = 0; j < 8; ++j) {
       const float4 t = __ldg(b4 + j);
-      p.b[4 * j] = t.x; p.b[4 * j + 1] = t.y; p.b[4 * j + 2] = t.z; p.b[4 * j + 3] = t.w;
+      o[2 * j] = pack_bf16x2(fmaxf(__uint_as_float(r[4 * j]) + t.x, 0.f), fmaxf(__uint_as_float(r[4 * j + 1]) + t.y, 0.f));
+      o[2 * j + 1] = pack_bf16x2(fmaxf(__uint_as_float(r[4 * j + 2]) + t.z, 0.f), fmaxf(__uint_as_float(r[4 * j + 3]) + t.w, 0.f));
     }
   }
-  // r = accumulator columns col0 + off .. + 31
-  template <class P> __device__ __forceinline__ void operator()(int col0, int off, const uint32_t (&r)[32], const P& p) const {
-    if (!p.valid) return;
-    uint32_t o[16];
-#pragma unroll
-    for (int j = 0; j < 16; ++j)
-      o[j] = pack_bf16x2(fmaxf(__uint_as_float(r[2 * j]) + p.b[off + 2 * j], 0.f),
-                         fmaxf(__uint_as_float(r[2 * j + 1]) + p.b[off + 2 * j + 1], 0.f));
-    uint4* dst = reinterpret_cast<uint4*>(out + (size_t)p.row * 64 + col0 + off);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+  __device__ __forceinline__ uint32_t index(int b, int y, int x, int col) const {
+    return (uint32_t)(((b * OUT_H + y) * OUT_W + x) * 64 + col);
   }
 };
-template <class Map, int OUT_H, int OUT_W> struct ShiftReluMaskEpi {
-  template <int COLS> struct Pre { typedef MaskPre<COLS> type; };
-  Map map; bf16* out; const bf16* act;
-  template <class P> __device__ __forceinline__ void prefetch(int pos, int col0, P& p) const {
-    int b, y, x;
-    p.valid = map(pos, b, y, x);
-    p.idx = ((size_t)(b * OUT_H + y) * OUT_W + x) * 64 + col0;
-    if (!p.valid) return;
-    const uint4* a4 = reinterpret_cast<const uint4*>(act + p.idx);
+__device__ __forceinline__ void plain_bf16_values(const uint32_t (&r)[32], uint32_t (&o)[16]) {
 #pragma unroll
-    for (int j = 0; j < (int)(sizeof(p.m) / sizeof(uint4)); ++j) p.m[j] = __ldg(a4 + j);
-  }
-  template <class P> __device__ __forceinline__ void operator()(int, int off, const uint32_t (&r)[32], const P& p) const {
-    if (p.valid) relu_mask_store_pre(out, p.idx + off, r, &p.m[off / 8]);
+  for (int j = 0; j < 16; ++j) o[j] = pack_bf16x2(__uint_as_float(r[2 * j]), __uint_as_float(r[2 * j + 1]));
+}
+template <class Map, int OUT_H, int OUT_W> struct ShiftReluMaskEpi {
+  static constexpr bool MASK = true;
+  Map map; bf16* out; const bf16* act;
+  __device__ __forceinline__ void values(int, const uint32_t (&r)[32], uint32_t (&o)[16]) const { plain_bf16_values(r, o); }
+  __device__ __forceinline__ uint32_t index(int b, int y, int x, int col) const {
+    return (uint32_t)(((b * OUT_H + y) * OUT_W + x) * 64 + col);
   }
 };
 // stride-2 data gradient: accumulator columns 32 c .. 32 c + 31 are parity class c of raster pixel (yy, xx)
 template <class Map> struct ShiftReluMaskEpiS2 {
-  template <int COLS> struct Pre { typedef MaskPre<COLS> type; };
+  static constexpr bool MASK = true;
   Map map; bf16* out; const bf16* act;
-  __device__ __forceinline__ size_t class_idx(size_t base, int cls) const {      // base = pixel (2 yy, 2 xx)
-    return base + (size_t)((cls >> 1) * 20 + (cls & 1)) * 32;
-  }
-  template <class P> __device__ __forceinline__ void prefetch(int pos, int col0, P& p) const {
-    int b, yy, xx;
-    p.valid = map(pos, b, yy, xx);
-    p.idx = ((size_t)(b * 20 + 2 * yy) * 20 + 2 * xx) * 32;
-    if (!p.valid) return;
-#pragma unroll
-    for (int c = 0; c < (int)(sizeof(p.m) / (4 * sizeof(uint4))); ++c) {
-      const uint4* a4 = reinterpret_cast<const uint4*>(act + class_idx(p.idx, (col0 >> 5) + c));
-#pragma unroll
-      for (int j = 0; j < 4; ++j) p.m[4 * c + j] = __ldg(a4 + j);
-    }
-  }
-  template <class P> __device__ __forceinline__ void operator()(int col0, int off, const uint32_t (&r)[32], const P& p) const {
-    if (p.valid) relu_mask_store_pre(out, class_idx(p.idx, (col0 + off) >> 5), r, &p.m[off / 8]);
+  __device__ __forceinline__ void values(int, const uint32_t (&r)[32], uint32_t (&o)[16]) const { plain_bf16_values(r, o); }
+  __device__ __forceinline__ uint32_t index(int b, int yy, int xx, int col) const {
+    const int cls = col >> 5;
+    return (uint32_t)(((b * 20 + 2 * yy + (cls >> 1)) * 20 + 2 * xx + (cls & 1)) * 32 + (col & 31));
   }
 };
-
 // ---- plain split-k GEMM with both operands streamed (the fully connected layer, forward) ----------------
 // C[m][n] = sum_k A[m][k] W[n][k] for A[M][K], W[N][K] row-major bf16.  Same persistent skeleton; a work item
 // is (row tile, 128-column tile, k split), the stage holds the A and the W tile of one K block, and the
@@ -1162,7 +1179,7 @@ static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_t
 
 template <class Cfg, class Epi, int BN, int STAGES, int NACC>
 static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int positions, uint32_t* err) {
-  constexpr int smem = Cfg::NT * BN * 128 + STAGES * Cfg::PLANES * Cfg::STAGE_ROWS * 128 + 1024;
+  constexpr int smem = Cfg::NT * BN * 128 + STAGES * Cfg::PLANES * Cfg::STAGE_ROWS * 128 + 8 * 32 * BN + 1024;
   static_assert(smem <= 227 * 1024, "shared memory budget");
   auto kern = tc_shift_kernel<Cfg, Epi, BN, STAGES, NACC>;
   static bool configured = false;
@@ -1244,15 +1261,15 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
                                 n, err);
     {
       typedef RasterMap<100, 10, 9, 9> Map;
-      tc_shift<C2FwdCfg, ShiftBiasReluEpi<Map, 9, 9>, 64, 4, 1>(
+      tc_shift<C2FwdCfg, ShiftBiasReluEpi<Map, 9, 9>, 64, 3, 1>(
           lc, KID_CONV2_FWD, C2FwdCfg{(const bf16*)act[0], n}, w + d[1].w_off,
-          ShiftBiasReluEpi<Map, 9, 9>{Map{n}, (bf16*)act[1], theta + d[1].b_off}, n * 100, err);
+          ShiftBiasReluEpi<Map, 9, 9>{Map{n}, (bf16*)act[1], theta + d[1].b_off, nullptr}, n * 100, err);
     }
     {
       typedef RasterMap<81, 9, 7, 7> Map;
       tc_shift<C3FwdCfg, ShiftBiasReluEpi<Map, 7, 7>, 64, 6, 1>(
           lc, KID_CONV3_FWD, C3FwdCfg{(const bf16*)act[1], n * 81}, w + d[2].w_off,
-          ShiftBiasReluEpi<Map, 7, 7>{Map{n}, (bf16*)act[2], theta + d[2].b_off}, n * 81, err);
+          ShiftBiasReluEpi<Map, 7, 7>{Map{n}, (bf16*)act[2], theta + d[2].b_off, nullptr}, n * 81, err);
     }
     (void)M2; (void)M3;
     tc_fc_forward(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, (bf16*)act[3], n, 512, 3136, fc_scratch, err);
