@@ -206,6 +206,10 @@ def run_ours(args, cfg):
               clip_norm=COMMON["clip_norm"], entropy_beta=COMMON["entropy_beta"], value_coef=COMMON["value_coef"],
               term_denom=cfg["term_denom"])
     prec = pb.BF16 if cfg["precision"] == "bf16" else pb.FP32
+    # a stream of our own: the library records its launch sequences into CUDA graphs, which the legacy default
+    # stream does not allow; every event below is recorded on this stream too
+    side = torch.cuda.Stream()
+    torch.cuda.set_stream(side)
     g = pb.Paac(cfg["arch"], cfg["n_e"], cfg["t_max"], cfg["n_actions"], COMMON["seed"] + rank, precision=prec,
                 device="cuda:%d" % local, **hp)
     n_e, T = cfg["n_e"], cfg["t_max"]

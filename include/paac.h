@@ -194,8 +194,11 @@ int paac_debug_write(paac_ctx* ctx, int which, const void* src /* host */, size_
 /* Run-time options.  PAAC_OPT_CUDA_CORES_ONLY != 0 keeps the bf16 network off the tensor cores
  * (same rounding points, CUDA-core contractions): a second implementation to compare against.
  * PAAC_OPT_TC_WGRAD_LAYERS: bit mask (bit l = layer l, conv1 = 0) of the layers whose weight gradient
- * runs on the tensor cores; the others use the CUDA-core contraction.  Default: all. */
-enum { PAAC_OPT_CUDA_CORES_ONLY = 1, PAAC_OPT_TC_WGRAD_LAYERS = 2 };
+ * runs on the tensor cores; the others use the CUDA-core contraction.  Default: all.
+ * PAAC_OPT_CUDA_GRAPHS: != 0 (default) lets paac_rollout / paac_update record their kernel sequence into CUDA
+ * graphs after two plain iterations and replay them; 0 keeps every call on plain launches.  (Graphs are also
+ * bypassed while actions are forced or per-kernel profiling is on.) */
+enum { PAAC_OPT_CUDA_CORES_ONLY = 1, PAAC_OPT_TC_WGRAD_LAYERS = 2, PAAC_OPT_CUDA_GRAPHS = 3 };
 int paac_set_option(paac_ctx* ctx, int option, int value);
 
 /* Number of kernels the library has launched on this context since init. */

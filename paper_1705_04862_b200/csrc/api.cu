@@ -25,6 +25,14 @@ struct paac_ctx {
   bool forced_on;
   int tc_wgrad_mask;       // bit l: layer l's weight gradient runs on the tensor cores
   GradSegments grad_segs;  // partial-sum regions of the update in flight
+  uint64_t* step_dev;      // device copy of env_step; kernels read the step index from here
+  // Recorded launch sequences.  The kernels of a rollout (and of an update) take the same arguments every
+  // second iteration (the two frame buffers alternate), so after two plain iterations each parity is captured
+  // once into a CUDA graph and replayed from then on.  Anything that changes the sequence drops the graphs.
+  bool graphs_on;          // option: allow recording
+  int plain_calls[2][2];   // [rollout / update][parity]: calls made with plain launches
+  cudaGraphExec_t graph[2][2];
+  uint64_t graph_launches[2][2];
   bool simt_only;          // keep the bf16 network on the CUDA cores (cross-check of the tensor-core path)
 
   // device buffers (all inside the workspace)
@@ -104,6 +112,7 @@ size_t carve(paac_ctx* c, char* base) {
   c->rewards = k.take<int8_t>(B);
   c->terminals = k.take<uint8_t>(B);
   c->stats = k.take<DeviceStats>(1);
+  c->step_dev = k.take<uint64_t>(1);
   return (k.off + 255) & ~(size_t)255;
 }
 
@@ -128,7 +137,7 @@ void refresh_weight_copies(paac_ctx* c, bool cast) {
 }
 
 // network + heads on the n_e states of `frames`, activations into slot `slot`
-void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, uint64_t step) {
+void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample) {
   void* act[MAX_LAYERS];
   for (int l = 0; l <= c->nd.n_conv; ++l)
     act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
@@ -139,9 +148,54 @@ void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, uin
     simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
   const size_t row = (size_t)slot * c->n_e;
   launch_heads(c->lc, c->prec, c->nd, c->theta, c->theta16, act[c->nd.n_conv], c->n_e,
-               c->logits + row * c->A, c->values + row, c->seed, step,
+               c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot,
                sample && c->forced_on ? c->forced + row : nullptr, sample ? c->actions + row : nullptr,
                sample ? c->sampled + row : nullptr, sample ? c->uniforms + row : nullptr);
+}
+
+void drop_graphs(paac_ctx* c) {
+  for (int k = 0; k < 2; ++k)
+    for (int par = 0; par < 2; ++par) {
+      if (c->graph[k][par]) { cudaGraphExecDestroy(c->graph[k][par]); c->graph[k][par] = nullptr; }
+      c->plain_calls[k][par] = 0;
+    }
+}
+
+// Runs `enqueue` (which only launches kernels on c->st) either directly, or -- once this kind/parity has run
+// directly before -- records it into a graph and replays the graph.
+template <class F> void run_recorded(paac_ctx* c, int kind, int parity, F enqueue) {
+  const bool allowed = c->graphs_on && !c->lc.profiling && !c->forced_on;
+  if (allowed && c->graph[kind][parity]) {
+    if (cudaGraphLaunch(c->graph[kind][parity], c->st) == cudaSuccess) { c->lc.count += c->graph_launches[kind][parity]; return; }
+    cudaGetLastError();
+    drop_graphs(c);
+  }
+  if (allowed && c->plain_calls[kind][parity] >= 1) {
+    cudaGraph_t g = nullptr;
+    if (cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+      const uint64_t before = c->lc.count;
+      enqueue();
+      const uint64_t launched = c->lc.count - before;
+      cudaGraphExec_t exec = nullptr;
+      if (cudaStreamEndCapture(c->st, &g) == cudaSuccess && g != nullptr &&
+          cudaGraphInstantiate(&exec, g, 0) == cudaSuccess) {
+        cudaGraphDestroy(g);
+        c->graph[kind][parity] = exec;
+        c->graph_launches[kind][parity] = launched;
+        if (cudaGraphLaunch(exec, c->st) == cudaSuccess) return;
+      }
+      if (g) cudaGraphDestroy(g);
+      cudaGetLastError();
+      c->lc.count = before;
+      c->graphs_on = false;        // recording does not work here (e.g. the caller is capturing): plain launches only
+      drop_graphs(c);
+    } else {
+      cudaGetLastError();
+      c->graphs_on = false;
+    }
+  }
+  enqueue();
+  ++c->plain_calls[kind][parity];
 }
 
 }  // namespace
@@ -171,6 +225,7 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   if (!c) return PAAC_ERR_CUDA;
   fill_shape(c, arch, n_e, t_max, n_actions, hp);
   c->tc_wgrad_mask = 0xF;
+  c->graphs_on = true;
   c->seed = seed; c->device = dev; c->st = (cudaStream_t)hp->stream; c->lc.st = c->st;
   const size_t need = carve(c, nullptr);
   if (hp->workspace) {
@@ -187,7 +242,7 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   launch_init_params(c->lc, c->nd, seed, c->theta);
   refresh_weight_copies(c, true);
   c->cur = 1;   // the first rollout flips to buffer 0; its start states are written there now
-  launch_env_step(c->lc, seed, n_e, 0u, nullptr, hp->term_denom, c->frames[0], nullptr, nullptr, nullptr);
+  launch_env_step(c->lc, seed, n_e, c->step_dev, 0u, nullptr, hp->term_denom, c->frames[0], nullptr, nullptr, nullptr);
   if (cudaStreamSynchronize(c->st) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
     if (c->owns_workspace) cudaFree(c->ws);
     delete c;
@@ -204,14 +259,17 @@ int paac_rollout(paac_ctx* c, paac_rollout_view* view) {
   uint8_t* fr = c->frames[c->cur];
   uint8_t* nxt = c->frames[c->cur ^ 1];
   const size_t fstep = (size_t)c->n_e * FRAME_BYTES;
-  for (int t = 0; t < c->t_max; ++t) {
-    forward_slot(c, fr + t * fstep, t, true, c->env_step + t);
-    uint8_t* dst = t + 1 < c->t_max ? fr + (t + 1) * fstep : nxt;
-    const size_t row = (size_t)t * c->n_e;
-    launch_env_step(c->lc, c->seed, c->n_e, (uint32_t)(c->env_step + t), c->actions + row,
-                    c->hp.term_denom, dst, c->rewards + row, c->terminals + row, c->counters);
-  }
-  forward_slot(c, nxt, c->t_max, false, 0);
+  run_recorded(c, 0, c->cur, [&]() {
+    for (int t = 0; t < c->t_max; ++t) {
+      forward_slot(c, fr + t * fstep, t, true);
+      uint8_t* dst = t + 1 < c->t_max ? fr + (t + 1) * fstep : nxt;
+      const size_t row = (size_t)t * c->n_e;
+      launch_env_step(c->lc, c->seed, c->n_e, c->step_dev, (uint32_t)t, c->actions + row, c->hp.term_denom, dst,
+                      c->rewards + row, c->terminals + row, c->counters);
+    }
+    forward_slot(c, nxt, c->t_max, false);
+    launch_advance_step(c->lc, c->step_dev, (uint32_t)c->t_max);
+  });
   c->env_step += c->t_max;
   c->rollout_fresh = true;
   if (view) {
@@ -225,35 +283,37 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
   if (!c) return PAAC_ERR_ARG;
   if (!c->rollout_fresh) return PAAC_ERR_STATE;
   const paac_hparams& hp = c->hp;
-  launch_returns(c->lc, c->n_e, c->t_max, hp.gamma, c->rewards, c->terminals, c->values, c->R, c->adv);
-  launch_head_grad(c->lc, c->B, c->A, hp.entropy_beta, hp.value_coef, c->logits, c->values, c->actions,
-                   c->R, c->adv, c->dz, c->dV, c->loss_terms, c->stats);
-  const int L = c->nd.n_conv;
-  heads_backward(c->lc, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
-                 c->grad, c->scratch);
-  uint32_t* err = &c->stats->error_word;
-  for (int l = L; l >= 0; --l) {
-    // tensor-core kernels where they exist, the CUDA-core contraction otherwise
-    bool dgrad_done = false;
-    if (use_tc(c)) {
-      if (l == 3) { tc_backward_dgrad_fc(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
-      if (l == 2) { tc_backward_dgrad_conv3(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
-      if (l == 1) { tc_backward_dgrad_conv2(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
+  run_recorded(c, 1, c->cur, [&]() {
+    launch_returns(c->lc, c->n_e, c->t_max, hp.gamma, c->rewards, c->terminals, c->values, c->R, c->adv);
+    launch_head_grad(c->lc, c->B, c->A, hp.entropy_beta, hp.value_coef, c->logits, c->values, c->actions,
+                     c->R, c->adv, c->dz, c->dV, c->loss_terms, c->stats);
+    const int L = c->nd.n_conv;
+    heads_backward(c->lc, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
+                   c->grad, c->scratch);
+    uint32_t* err = &c->stats->error_word;
+    for (int l = L; l >= 0; --l) {
+      // tensor-core kernels where they exist, the CUDA-core contraction otherwise
+      bool dgrad_done = false;
+      if (use_tc(c)) {
+        if (l == 3) { tc_backward_dgrad_fc(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
+        if (l == 2) { tc_backward_dgrad_conv3(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
+        if (l == 1) { tc_backward_dgrad_conv2(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
+      }
+      bool wgrad_done = false;
+      if (use_tc(c) && (c->tc_wgrad_mask >> l) & 1) {
+        tc_backward_wgrad(c->lc, c->nd, c->frames[c->cur], c->B, c->act, c->gact, c->grad, c->scratch, l, &c->grad_segs, err);
+        wgrad_done = true;
+      }
+      if (!wgrad_done || (l > 0 && !dgrad_done))
+        simt_backward_layer(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
+                            c->gact, c->grad, c->scratch, l, !wgrad_done, l > 0 && !dgrad_done);
     }
-    bool wgrad_done = false;
-    if (use_tc(c) && (c->tc_wgrad_mask >> l) & 1) {
-      tc_backward_wgrad(c->lc, c->nd, c->frames[c->cur], c->B, c->act, c->gact, c->grad, c->scratch, l, &c->grad_segs, err);
-      wgrad_done = true;
-    }
-    if (!wgrad_done || (l > 0 && !dgrad_done))
-      simt_backward_layer(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
-                          c->gact, c->grad, c->scratch, l, !wgrad_done, l > 0 && !dgrad_done);
-  }
-  if (use_tc(c)) tc_backward_finish(c->lc, &c->grad_segs);
-  launch_clip_rmsprop(c->lc, c->nd.P, c->theta, c->rms, c->grad,
-                      c->prec == PAAC_BF16 ? c->theta16 : nullptr, hp.lr, hp.rms_decay, hp.rms_eps, hp.clip_norm,
-                      c->norm_partials, c->stats);
-  if (c->prec == PAAC_BF16) refresh_weight_copies(c, false);
+    if (use_tc(c)) tc_backward_finish(c->lc, &c->grad_segs);
+    launch_clip_rmsprop(c->lc, c->nd.P, c->theta, c->rms, c->grad,
+                        c->prec == PAAC_BF16 ? c->theta16 : nullptr, hp.lr, hp.rms_decay, hp.rms_eps, hp.clip_norm,
+                        c->norm_partials, c->stats);
+    if (c->prec == PAAC_BF16) refresh_weight_copies(c, false);
+  });
   c->N += (uint64_t)c->B;
   c->rollout_fresh = false;
   if (cuda_status(c) != PAAC_OK) return PAAC_ERR_CUDA;
@@ -311,6 +371,7 @@ int paac_force_actions(paac_ctx* c, const int32_t* actions) {
 int paac_destroy(paac_ctx* c) {
   if (!c) return PAAC_ERR_ARG;
   cudaStreamSynchronize(c->st);
+  drop_graphs(c);
   c->lc.release();
   if (c->owns_workspace) cudaFree(c->ws);
   cudaGetLastError();
@@ -336,8 +397,9 @@ uint64_t paac_launch_count(const paac_ctx* c) { return c ? c->lc.count : 0; }
 
 int paac_set_option(paac_ctx* c, int option, int value) {
   if (!c) return PAAC_ERR_ARG;
-  if (option == PAAC_OPT_CUDA_CORES_ONLY) { c->simt_only = value != 0; return PAAC_OK; }
-  if (option == PAAC_OPT_TC_WGRAD_LAYERS) { c->tc_wgrad_mask = value & 0xF; return PAAC_OK; }
+  if (option == PAAC_OPT_CUDA_CORES_ONLY) { c->simt_only = value != 0; drop_graphs(c); return PAAC_OK; }
+  if (option == PAAC_OPT_TC_WGRAD_LAYERS) { c->tc_wgrad_mask = value & 0xF; drop_graphs(c); return PAAC_OK; }
+  if (option == PAAC_OPT_CUDA_GRAPHS) { c->graphs_on = value != 0; drop_graphs(c); return PAAC_OK; }
   return PAAC_ERR_ARG;
 }
 
@@ -374,12 +436,15 @@ int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, f
     cudaGetLastError(); return PAAC_ERR_CUDA;
   }
   const bool sample = t < c->t_max;
-  forward_slot(c, dst, t, sample, c->env_step + t);
+  forward_slot(c, dst, t, sample);
   const size_t row = (size_t)t * c->n_e;
   if (sample) cudaMemcpyAsync(actions, c->actions + row, c->n_e * sizeof(int32_t), cudaMemcpyDeviceToHost, c->st);
   if (values) cudaMemcpyAsync(values, c->values + row, c->n_e * sizeof(float), cudaMemcpyDeviceToHost, c->st);
   if (cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
-  if (t == c->t_max) { c->host_t = 0; c->env_step += c->t_max; c->rollout_fresh = true; }
+  if (t == c->t_max) {
+    launch_advance_step(c->lc, c->step_dev, (uint32_t)c->t_max);
+    c->host_t = 0; c->env_step += c->t_max; c->rollout_fresh = true;
+  }
   else c->host_t = t + 1;
   return cuda_status(c);
 }

@@ -56,7 +56,8 @@ constexpr int ENV_THREADS = 256;
 constexpr int FRAME_WORDS = FRAME_H * FRAME_W;   // 7056, a multiple of 4
 
 __global__ void __launch_bounds__(ENV_THREADS)
-env_step_kernel(uint64_t seed, int n_e, uint32_t step, const int32_t* __restrict__ actions, uint32_t term_denom,
+env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, uint32_t t,
+                const int32_t* __restrict__ actions, uint32_t term_denom,
                 uint8_t* __restrict__ next_frames, int8_t* __restrict__ rewards, uint8_t* __restrict__ terminals,
                 int32_t* __restrict__ counters) {
   __shared__ uint32_t s_base;
@@ -64,6 +65,7 @@ env_step_kernel(uint64_t seed, int n_e, uint32_t step, const int32_t* __restrict
   if (threadIdx.x == 0) {
     uint32_t tag = 0u, frame_step = 0u;
     if (actions != nullptr) {
+      const uint32_t step = (uint32_t)(*step_base) + t;       // global step index of this transition
       const int32_t a = actions[e];
       const uint32_t base = env_hash_base(seed, e, step, (uint32_t)a + 1u);
       const uint32_t hr = hash_mix(base ^ HASH_TAG_REWARD) & 15u;
@@ -94,12 +96,20 @@ env_step_kernel(uint64_t seed, int n_e, uint32_t step, const int32_t* __restrict
   }
 }
 
-void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, uint32_t step,
+void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step_base, uint32_t t,
                      const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
                      uint8_t* terminals, int32_t* counters) {
   KernelScope scope(lc, KID_ENV_STEP);
-  env_step_kernel<<<n_e, ENV_THREADS, 0, lc.st>>>(seed, n_e, step, actions, term_denom, next_frames, rewards,
+  env_step_kernel<<<n_e, ENV_THREADS, 0, lc.st>>>(seed, n_e, step_base, t, actions, term_denom, next_frames, rewards,
                                                   terminals, counters);
+}
+
+// the environments' global step index lives on the device, so that a recorded sequence of launches can be
+// replayed for the next iteration without new arguments
+__global__ void advance_step_kernel(uint64_t* step_base, uint32_t by) { *step_base += by; }
+void launch_advance_step(LaunchCtx& lc, uint64_t* step_base, uint32_t by) {
+  KernelScope scope(lc, KID_ENV_STEP);
+  advance_step_kernel<<<1, 1, 0, lc.st>>>(step_base, by);
 }
 
 }  // namespace paac

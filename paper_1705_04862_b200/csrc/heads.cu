@@ -40,7 +40,7 @@ template <class T, class TW, int EPL>
 __global__ void __launch_bounds__(128)
 heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* __restrict__ bpi,
              const TW* __restrict__ wv, const float* __restrict__ bv, int n, int A,
-             float* __restrict__ logits, float* __restrict__ values, uint64_t seed, uint64_t step,
+             float* __restrict__ logits, float* __restrict__ values, uint64_t seed, const uint64_t* __restrict__ step_base, uint32_t t,
              const int32_t* __restrict__ forced, int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
              float* __restrict__ uniforms) {
   constexpr int F = 32 * EPL;
@@ -71,6 +71,7 @@ heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* _
   const float ex = lane < A ? expf(z - m) : 0.f;
   const float lse = m + logf(warp_sum(ex));
   const float p = lane < A ? expf(z - lse) : 0.f;
+  const uint64_t step = *step_base + t;
   const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
   float c = 0.f;
   int a = A - 1;
@@ -95,7 +96,7 @@ template <class T, class TW>
 __global__ void __launch_bounds__(128)
 heads_slow_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* __restrict__ bpi,
              const TW* __restrict__ wv, const float* __restrict__ bv, int n, int F, int A,
-             float* __restrict__ logits, float* __restrict__ values, uint64_t seed, uint64_t step,
+             float* __restrict__ logits, float* __restrict__ values, uint64_t seed, const uint64_t* __restrict__ step_base, uint32_t t,
              const int32_t* __restrict__ forced, int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
              float* __restrict__ uniforms) {
   const int lane = threadIdx.x & 31;
@@ -120,6 +121,7 @@ heads_slow_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const flo
   const float ex = lane < A ? expf(z - m) : 0.f;
   const float lse = m + logf(warp_sum(ex));
   const float p = lane < A ? expf(z - lse) : 0.f;
+  const uint64_t step = *step_base + t;
   const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
   float c = 0.f;
   int a = A - 1;
@@ -138,7 +140,8 @@ heads_slow_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const flo
 
 void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
                   const bf16* theta16, const void* h, int n, float* logits, float* values, uint64_t seed,
-                  uint64_t step, const int32_t* forced, int32_t* actions, int32_t* sampled, float* uniforms) {
+                  const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
+                  float* uniforms) {
   const int blocks = (n + 3) / 4;
   KernelScope scope(lc, KID_HEADS_FWD);
   cudaStream_t st = lc.st;
@@ -146,17 +149,17 @@ void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta
   const bool aligned = nd.pi_w % 8 == 0;      // 16-byte loads of the policy rows
   if (prec == PAAC_BF16 && nd.F == 512 && aligned)
     heads_kernel<bf16, bf16, 16><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
-                                                         nd.A, logits, values, seed, step, forced, actions, sampled, uniforms);
+                                                         nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms);
   else if (prec == PAAC_BF16 && nd.F == 256 && aligned)
     heads_kernel<bf16, bf16, 8><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
-                                                        nd.A, logits, values, seed, step, forced, actions, sampled, uniforms);
+                                                        nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms);
   else if (prec == PAAC_BF16)
     heads_slow_kernel<bf16, bf16><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv,
-                                                          n, nd.F, nd.A, logits, values, seed, step, forced, actions,
+                                                          n, nd.F, nd.A, logits, values, seed, step_base, t, forced, actions,
                                                           sampled, uniforms);
   else
     heads_slow_kernel<float, float><<<blocks, 128, 0, st>>>((const float*)h, theta + nd.pi_w, bpi, theta + nd.v_w, bv,
-                                                            n, nd.F, nd.A, logits, values, seed, step, forced, actions,
+                                                            n, nd.F, nd.A, logits, values, seed, step_base, t, forced, actions,
                                                             sampled, uniforms);
 }
 

@@ -9,9 +9,11 @@ namespace paac {
 void launch_init_params(LaunchCtx& lc, const NetDims& nd, uint64_t seed, float* theta);
 void launch_cast_bf16(LaunchCtx& lc, const float* src, bf16* dst, size_t n);
 // actions == nullptr: start states (step index 0) for every environment
-void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, uint32_t step,
+void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step_base /* device */, uint32_t t,
                      const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
                      uint8_t* terminals, int32_t* counters /* [3][n_e] */);
+
+void launch_advance_step(LaunchCtx& lc, uint64_t* step_base, uint32_t by);
 
 // ---- network on the CUDA cores (net_simt.cu) --------------------------------------------
 // act[l]: stored activation of layer l for the n states, storage float (PAAC_FP32) or bf16
@@ -56,7 +58,7 @@ void simt_backward_layer(LaunchCtx& lc, int arch, int prec, const NetDims& nd, c
 // logits/values of n states from the fc activation; if actions != nullptr also samples
 void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
                   const bf16* theta16, const void* h, int n, float* logits, float* values, uint64_t seed,
-                  uint64_t step, const int32_t* forced, int32_t* actions, int32_t* sampled /* action before forcing */,
+                  const uint64_t* step_base /* device */, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled /* action before forcing */,
                   float* uniforms);
 void launch_returns(LaunchCtx& lc, int n_e, int t_max, float gamma, const int8_t* rewards,
                     const uint8_t* terminals, const float* values, float* R, float* adv);

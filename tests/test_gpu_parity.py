@@ -46,14 +46,24 @@ def test_config2_nips_fp32_params_after_10_updates(orc):
     g.close()
 
 
-def test_config2_free_running_actions_agree(orc):
-    """Without forcing: both sides sample for themselves; with float parameters the draws agree."""
+@pytest.mark.parametrize("own_stream", [False, True])
+def test_config2_free_running_actions_agree(orc, own_stream):
+    """Without forcing: both sides sample for themselves; with float parameters the draws agree.  On a stream
+    of its own the library replays recorded CUDA graphs from the third iteration on (the legacy default stream
+    cannot be captured, so there every iteration is plain launches): both must walk with the oracle."""
+    import torch
     cfg = CONFIGS[1]
-    o, g = make_pair(orc, cfg)
-    for it in range(3):
-        ro, r1 = check_rollout(orc, o, g, TOL["fp32"], lockstep=False)
-        check_update(orc, o, g, TOL["fp32"], check_acts=False)
-    g.close()
+    stream = torch.cuda.Stream() if own_stream else torch.cuda.current_stream()
+    with torch.cuda.stream(stream):
+        o, g = make_pair(orc, cfg)
+        launches = []
+        for it in range(7):
+            before = g.launch_count()
+            ro, r1 = check_rollout(orc, o, g, TOL["fp32"], lockstep=False)
+            check_update(orc, o, g, TOL["fp32"], check_acts=False)
+            launches.append(g.launch_count() - before)
+        assert len(set(launches)) == 1            # replayed sequences count the same kernels as plain ones
+        g.close()
 
 
 def _bf16_iterations(orc, cfg, iters):
@@ -179,7 +189,9 @@ def test_ragged_sizes_and_action_counts(orc):
 def test_resync_after_many_updates(orc):
     """Free-run the library for 60 updates (config 2), copy its parameters and RMSProp state into
     the oracle and compare one more iteration from there."""
+    import torch
     cfg = CONFIGS[1]
+    torch.cuda.set_stream(torch.cuda.Stream())      # own stream: the 60 free-running updates replay CUDA graphs
     o, g = make_pair(orc, cfg)
     for it in range(60):
         g.rollout()
@@ -194,19 +206,25 @@ def test_resync_after_many_updates(orc):
     check_rollout(orc, o, g, TOL["fp32"])
     check_update(orc, o, g, TOL["fp32"], check_acts=False)
     g.close()
+    torch.cuda.set_stream(torch.cuda.default_stream())
 
 
 def test_determinism_bitwise(orc):
+    """Same seed, same bits -- with plain launches and with replayed graphs (own stream), tensor-core path."""
+    import torch
     cfg = CONFIGS[2]
     outs = []
-    for rep in range(2):
-        _, g = make_pair(orc, cfg)
-        for it in range(3):
-            g.rollout()
-            g.update()
-        outs.append((g.params(), g.debug_read(pb.DBG_GRAD).copy()))
-        g.close()
-    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    for rep in range(3):
+        stream = torch.cuda.Stream() if rep == 2 else torch.cuda.current_stream()
+        with torch.cuda.stream(stream):
+            _, g = make_pair(orc, cfg)
+            for it in range(5):
+                g.rollout()
+                g.update()
+            outs.append((g.params(), g.debug_read(pb.DBG_GRAD).copy()))
+            g.close()
+    for k in (1, 2):
+        assert np.array_equal(outs[0][0], outs[k][0]) and np.array_equal(outs[0][1], outs[k][1])
 
 
 def test_error_paths(orc):
