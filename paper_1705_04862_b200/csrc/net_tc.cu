@@ -1607,6 +1607,218 @@ static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, int rows, int n_a
   add_segment(segs, bias_part, gb, splits, 1, CO, 1.f);
 }
 
+// ---- weight gradients of the middle convolutions without im2col ----------------------------------------------
+// The same shifted views as in the forward kernels, seen from the reduction side:
+//   dW[tap][ci][co] = sum over raster positions m of X[m + shift(tap)][ci] * G[m][co],
+// where X is the layer input in raster order and G the output gradient laid on the SAME raster (zero at the
+// positions that are not outputs).  A stage holds 128 + max-shift rows of X (per plane) and 128 rows of G, each
+// fetched once; both operands are MN-major (a shared-memory row = one raster position, 64 values of ci or co),
+// and the A operand of tap t is the X image entered shift(t) rows down.  Two taps share one M = 128 instruction:
+// the descriptor's leading-dimension offset, the distance between the first and the second block of 64 rows of
+// M, is simply the distance between the two taps' entry rows, so the second half of the accumulator belongs to
+// the next tap.  (An odd tap count leaves the upper half of the last accumulator unused.)
+// The bias gradient, the column sums of G, is added up by one extra warp from the staged rows.
+// A CTA owns a contiguous range of 128-row raster tiles (split-k); partial sums go to scratch as
+// part[split][tap * 64 + ci][co] and the finishing kernel adds the splits in a fixed order.
+constexpr int SWG_THREADS = 320;      // warps 0-7 producers (and the final epilogue), 8 MMA issuer, 9 bias sums
+constexpr int SWG_MAX_SPLITS = 148;
+
+template <int RASTER_, int WIDTH, int OUT_H, int OUT_W> struct GradCells {
+  static constexpr int RASTER = RASTER_, STATE = OUT_H * OUT_W * 64;
+  // element offset of raster cell `rem` inside a state's OUT_H x OUT_W x 64 gradient, or -1 for a margin cell
+  __device__ static __forceinline__ int cell(int rem) {
+    const int y = rem / WIDTH, x = rem % WIDTH;
+    return (y < OUT_H && x < OUT_W) ? (y * OUT_W + x) * 64 : -1;
+  }
+};
+
+struct SwgShared {
+  uint64_t full[8], empty[8], acc;
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+__device__ __forceinline__ void mma_bf16_lo_rt(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+template <class Cfg, class Cells, int STAGES>
+__global__ void __launch_bounds__(SWG_THREADS, 1)
+tc_shift_wgrad_kernel(Cfg cfg, const bf16* __restrict__ g, int states, float* __restrict__ partial,
+                      float* __restrict__ bias_partial, int tiles, int tiles_per_cta, uint32_t* error_word) {
+  constexpr int NT = Cfg::NT, NP = (NT + 1) / 2, SR = Cfg::STAGE_ROWS, PLANES = Cfg::PLANES, J = NT * 64;
+  constexpr uint32_t PLANE_BYTES = SR * 128, X_BYTES = PLANES * PLANE_BYTES, G_BYTES = TC_BM * 128,
+                     STAGE_BYTES = X_BYTES + G_BYTES;
+  constexpr uint32_t TMEM_COLS = NP * 64 <= 256 ? 256 : 512;
+  static_assert(STAGES >= 2 && STAGES <= 8 && SR % 8 == 0 && NP * 64 <= 512, "pipeline shape");
+  extern __shared__ uint8_t dyn_smem[];
+  __shared__ SwgShared sh;
+  __shared__ int cell_table[Cells::RASTER];
+  const uint32_t stage0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int split = blockIdx.x, t0 = split * tiles_per_cta, t1 = min(tiles, t0 + tiles_per_cta);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 256); mbar_init(&sh.empty[s], 2); }
+    mbar_init(&sh.acc, 1);
+    sh.abort = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 8) tmem_alloc(&sh.tmem_base, TMEM_COLS);
+  for (int i = threadIdx.x; i < Cells::RASTER; i += SWG_THREADS) cell_table[i] = Cells::cell(i);
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+
+  if (warp < 8) {
+    // ---------------- producers: eight lanes per 128-byte row, 32 rows per pass ----------------
+    const int c = lane & 7, sub = warp * 4 + (lane >> 3);
+    for (int t = t0; t < t1; ++t) {
+      const int it = t - t0, s = it % STAGES;
+      const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const uint32_t stage = stage0 + s * STAGE_BYTES;
+      for (int idx = sub; idx < PLANES * SR; idx += 32) {
+        const int plane = PLANES == 1 ? 0 : idx / SR, ri = PLANES == 1 ? idx : idx % SR;
+        bool valid;
+        const bf16* src = cfg.src(plane, t * TC_BM + ri, valid);
+        cp_async16(stage + plane * PLANE_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), src + c * 8, valid ? 16u : 0u);
+      }
+#pragma unroll
+      for (int ri = sub; ri < TC_BM; ri += 32) {
+        const int pos = t * TC_BM + ri, b = pos / Cells::RASTER, off = cell_table[pos - b * Cells::RASTER];
+        const bool valid = b < states && off >= 0;
+        const bf16* src = valid ? g + (size_t)b * Cells::STATE + off : g;
+        cp_async16(stage + X_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), src + c * 8, valid ? 16u : 0u);
+      }
+      // the hardware arrives on the stage's barrier for this thread once its copies have landed
+      cp_async_mbar_arrive(&sh.full[s]);
+    }
+    cp_async_commit();
+    cp_async_wait<0>();
+    // ---------------- epilogue: float partial tile to scratch ----------------
+    // warps e and e + 4 share TMEM lane quarter e & 3 and take 32 of the 64 columns each
+    if (t1 > t0 && mbar_wait(&sh.acc, 0, &sh.abort, error_word, ERR_WAIT_ACC)) {
+      tcgen05_fence_after();
+      const int quarter = warp & 3, col0 = (warp >> 2) * 32;
+#pragma unroll 1
+      for (int p = 0; p < NP; ++p) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + p * 64 + col0, r);
+        const int j = p * 128 + quarter * 32 + lane;
+        if (j < J) {
+          float4* dst = reinterpret_cast<float4*>(partial + ((size_t)split * J + j) * 64 + col0);
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
+                                 __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+        }
+      }
+    }
+  } else if (warp == 8) {
+    if (lane == 0) {
+      // ---------------- MMA issuer ----------------
+      constexpr uint32_t idesc = make_idesc_bf16(TC_BM, 64, 1, 1);
+      const uint32_t hi = desc_hi_kmajor_sw128();                 // stride between 8-row groups 1024 B, 128B swizzle
+      bool ok = true;
+      for (int t = t0; t < t1 && ok; ++t) {
+        const int it = t - t0, s = it % STAGES;
+        ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+        if (!ok) break;
+        fence_proxy_async_smem();        // the copies observed through the barrier -> visible to the MMA's operand reads
+        tcgen05_fence_after();
+        const uint32_t stage = stage0 + s * STAGE_BYTES;
+        const uint32_t b_lo0 = ((stage + X_BYTES) >> 4) & 0x3FFFu;
+#pragma unroll
+        for (int k = 0; k < TC_BM / 16; ++k) {
+#pragma unroll
+          for (int p = 0; p < NP; ++p) {
+            const int ta = 2 * p, tb = 2 * p + 1 < NT ? 2 * p + 1 : -1;
+            const uint32_t a_off = Cfg::tap_plane(ta) * PLANE_BYTES + Cfg::tap_shift(ta) * 128u;
+            // second half of M: the next tap's entry row (or simply the next row, result unused)
+            const uint32_t lbo = tb >= 0 ? (Cfg::tap_plane(tb) * PLANE_BYTES + Cfg::tap_shift(tb) * 128u) - a_off : 128u;
+            const uint32_t a_lo = (((stage + a_off + k * 2048u) >> 4) & 0x3FFFu) | ((lbo >> 4) << 16);
+            mma_bf16_lo_rt(tmem + p * 64, a_lo, b_lo0 + k * (2048u >> 4), hi, idesc, (it | k) != 0 ? 1u : 0u);
+          }
+        }
+        mma_commit(&sh.empty[s]);
+      }
+      if (ok && t1 > t0) mma_commit(&sh.acc);
+    }
+  } else {
+    // ---------------- bias gradient: lane l adds up columns 2 l and 2 l + 1 of the staged G rows ----------------
+    float acc[4][2] = {};
+    bool ok = true;
+    for (int t = t0; t < t1 && ok; ++t) {
+      const int it = t - t0, s = it % STAGES;
+      ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      const uint32_t gbase = stage0 + s * STAGE_BYTES + X_BYTES + (uint32_t)(lane & 3) * 4u;
+#pragma unroll 4
+      for (int r8 = 0; r8 < TC_BM; r8 += 8) {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+          uint32_t v;
+          asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(gbase + (r8 + r) * 128u + ((uint32_t)((lane >> 2) ^ r) << 4)) : "memory");
+          acc[r & 3][0] += __uint_as_float(v << 16);
+          acc[r & 3][1] += __uint_as_float(v & 0xFFFF0000u);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.empty[s]);
+    }
+    if (ok && t1 > t0) {
+      bias_partial[(size_t)split * 64 + 2 * lane] = (acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]);
+      bias_partial[(size_t)split * 64 + 2 * lane + 1] = (acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]);
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    __syncwarp();
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
+}
+
+static int swg_splits(int positions) {
+  const int tiles = (positions + TC_BM - 1) / TC_BM;
+  int ctas = sm_count() < SWG_MAX_SPLITS ? sm_count() : SWG_MAX_SPLITS;
+  if (ctas > tiles) ctas = tiles;
+  const int per = (tiles + ctas - 1) / ctas;
+  return (tiles + per - 1) / per;
+}
+
+template <class Cfg, class Cells, int STAGES>
+static void tc_shift_wgrad(LaunchCtx& lc, int kid, Cfg cfg, const bf16* g, int states, int positions, float* gw, float* gb,
+                           float* scratch, GradSegments* segs, uint32_t* err) {
+  constexpr int smem = STAGES * (Cfg::PLANES * Cfg::STAGE_ROWS + TC_BM) * 128 + 1024;
+  static_assert(smem <= 227 * 1024, "shared memory budget");
+  auto kern = tc_shift_wgrad_kernel<Cfg, Cells, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  constexpr int J = Cfg::NT * 64;
+  const int tiles = (positions + TC_BM - 1) / TC_BM;
+  const int splits = swg_splits(positions), per = (tiles + splits - 1) / splits;
+  float* bias_part = scratch + (size_t)splits * J * 64;
+  KernelScope scope(lc, kid);
+  kern<<<splits, SWG_THREADS, smem, lc.st>>>(cfg, g, states, scratch, bias_part, tiles, per, err);
+  add_segment(segs, scratch, gw, splits, J, 64, 1.f);
+  add_segment(segs, bias_part, gb, splits, 1, 64, 1.f);
+}
+
 // ---- first layer, weight gradient: one state at a time ----------------------------------------------------
 // dW1^T[j][co] = sum over (state, oh, ow) of window[j] * G[co].  A CTA walks over its share of the states;
 // each state's raw uint8 frame (28,224 bytes) and its 400 x 32 gradient rows are brought into shared memory
@@ -1802,8 +2014,8 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
 static size_t tc_layer_scratch_floats(int n, int layer) {
   switch (layer) {
     case 0: return wg_scratch_floats(n * 400, 256, 32, 1);
-    case 1: return wg_scratch_floats(n * 81, 512, 64, 2);
-    case 2: return wg_scratch_floats(n * 49, 576, 64, 3);
+    case 1: return (size_t)SWG_MAX_SPLITS * (512 * 64 + 64);
+    case 2: return (size_t)SWG_MAX_SPLITS * (576 * 64 + 64);
     default: return wg_scratch_floats(n, 3136, 512, 25 * 4);
   }
 }
@@ -1837,15 +2049,11 @@ void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, 
     typedef NatConv1 C1;
     tc_conv1_wgrad<C1>(lc, frames, g, n, gw, gb, sc, &segs, err);
   } else if (layer == 1) {
-    typedef NatConv2 C2;
-    const int rows = n * C2::OH * C2::OW;
-    tc_wgrad<ConvSrc<C2>, GradSrc<64>, 2, 64, 5, 64>(lc, KID_CONV2_WGRAD, ConvSrc<C2>{(const bf16*)act[0], rows},
-                                                     GradSrc<64>{g, 64, rows}, rows, 8, 1.f, gw, gb, sc, &segs, err);
+    tc_shift_wgrad<C2FwdCfg, GradCells<100, 10, 9, 9>, 4>(lc, KID_CONV2_WGRAD, C2FwdCfg{(const bf16*)act[0], n}, g, n, n * 100,
+                                                          gw, gb, sc, &segs, err);
   } else if (layer == 2) {
-    typedef NatConv3 C3;
-    const int rows = n * C3::OH * C3::OW;
-    tc_wgrad<ConvSrc<C3>, GradSrc<64>, 2, 64, 5, 64>(lc, KID_CONV3_WGRAD, ConvSrc<C3>{(const bf16*)act[1], rows},
-                                                     GradSrc<64>{g, 64, rows}, rows, 9, 1.f, gw, gb, sc, &segs, err);
+    tc_shift_wgrad<C3FwdCfg, GradCells<81, 9, 7, 7>, 5>(lc, KID_CONV3_WGRAD, C3FwdCfg{(const bf16*)act[1], n * 81}, g, n, n * 81,
+                                                        gw, gb, sc, &segs, err);
   } else {
     tc_wgrad<PlainSrc, GradSrc<64>, 1, 128, 6, 512>(lc, KID_FC_WGRAD, PlainSrc{(const bf16*)act[2], 3136, n},
                                                     GradSrc<64>{g, 512, n}, n, 49, 1.f, gw, gb, sc, &segs, err);
