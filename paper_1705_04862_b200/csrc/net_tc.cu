@@ -995,37 +995,62 @@ __device__ __forceinline__ void u8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_
 // Space-to-depth view: with stride 4 and an 8 x 8 kernel, the window of output (oh, ow) is the 2 x 2 group of
 // 4 x 4-pixel blocks (oh + i, ow + j), i, j in {0, 1}.  A block is 4 x 4 x 4 channels = 64 values = one 128-byte
 // bf16 operand row, so the layer is a 2 x 2, stride-1 convolution over the 21 x 21 raster of blocks and runs
-// as four shifted views (0, 1, 21, 22 rows) of one staged row block, like the other convolutions.  Every input
-// byte is expanded to bf16 once per tile instead of once per window that contains it.
-constexpr int C1_THREADS = 416;      // warps 0-3 epilogue, 4-11 producers, 12 MMA
-constexpr int C1_RAW_BYTES = 12288;  // >= 36 frame rows of 336 bytes
-constexpr int C1_STAGE_ROWS = 152, C1_USED_ROWS = 150, C1_RASTER = 21;
+// as shifted views of one staged row block, like the other convolutions.  Every input byte is expanded to bf16
+// once per tile instead of once per window that contains it.
+//
+// With only 32 output channels an MMA would be 32 columns wide, and a narrow MMA costs almost as much as a wide
+// one (the 128 x 16 A slice is fetched either way).  So an accumulator row stands for TWO neighbouring raster
+// positions 2 i and 2 i + 1 (columns 0-31 and 32-63): blocks at even positions are staged in plane E, blocks at
+// odd positions in plane O, and with taps W00, W01, W10, W11 (block shifts 0, 1, 21, 22) the tile is the sum of
+// six views, each multiplied by a 64-row weight matrix (left half | right half):
+//   E+0: (W00 | 0)   O+0: (W01 | W00)   E+1: (0 | W01)   O+10: (W10 | 0)   E+11: (W11 | W10)   O+11: (0 | W11)
+// The six matrices are windows of two block sequences [0, W01, W00, 0] and [0, W11, W10, 0] kept in shared memory.
+//
+// Roles: warps 0-7 epilogue (warp e: TMEM lane quarter e & 3, position parity e >> 2), warps 8-15 expand the raw
+// bytes of a tile to bf16, warp 16 issues the MMAs, warp 17 fetches the frame rows a tile needs with one or two
+// bulk copies (a tile's positions lie in at most two states, contiguous rows in each) into a ring of raw slots.
+constexpr int C1_THREADS = 576;
+constexpr int C1_RASTER = 21, C1_TILE_POS = 256, C1_USED_POS = 278;     // positions 2 i + 23, i <= 127
+constexpr int C1_PLANE_ROWS = 144;                                      // >= 128 + 11, multiple of 8
+constexpr int C1_RAW_BYTES = 20480;                                     // >= 15 block rows of 4 x 336 bytes
+constexpr int C1_RAW_SLOTS = 3;
+
+struct C1Shared {
+  uint64_t full[4], empty[4], acc_full[2], acc_empty[2], raw_full[C1_RAW_SLOTS], raw_empty[C1_RAW_SLOTS];
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
 
 template <class G, class Epi, int STAGES>
 __global__ void __launch_bounds__(C1_THREADS, 1)
 tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, Epi epi, int n_states, int tiles,
                 uint32_t* error_word) {
   static_assert(G::K == 8 && G::S == 4 && G::C == 4 && G::CO == 32 && G::H == 84 && G::W == 84, "geometry");
-  constexpr int BN = 32, NT = 4, NPROD = 256, POS = C1_RASTER * C1_RASTER, ROW_BYTES = G::W * G::C;
-  constexpr uint32_t A_BYTES = C1_STAGE_ROWS * 128, B_BLOCK = BN * 128, B_BYTES = NT * B_BLOCK, RAW_BYTES = C1_RAW_BYTES;
+  static_assert(STAGES >= 2 && STAGES <= 4, "pipeline depth");
+  constexpr int BN = 64, NPROD = 256, POS = C1_RASTER * C1_RASTER, ROW_BYTES = G::W * G::C;
+  constexpr uint32_t PLANE_BYTES = C1_PLANE_ROWS * 128, A_BYTES = 2 * PLANE_BYTES, W_BLOCK = 32 * 128, B_BYTES = 8 * W_BLOCK;
   extern __shared__ uint8_t dyn_smem[];
-  __shared__ PkShared sh;
+  __shared__ C1Shared sh;
   const uint32_t b_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
   const uint32_t a_base0 = b_base + B_BYTES;
-  const uint32_t raw_base = a_base0 + STAGES * A_BYTES;       // ring of three slots of up to 36 frame rows
+  const uint32_t raw_base = a_base0 + STAGES * A_BYTES;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_pos = n_states * POS;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], NPROD / 32); mbar_init(&sh.empty[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 8); }
+    for (int i = 0; i < C1_RAW_SLOTS; ++i) { mbar_init(&sh.raw_full[i], 1); mbar_init(&sh.raw_empty[i], NPROD / 32); }
     sh.abort = 0u;
     fence_barrier_init();
   }
-  if (warp == 12) tmem_alloc(&sh.tmem_base, 2 * BN);
-  for (int i = threadIdx.x; i < NT * BN * 8; i += C1_THREADS) {     // weights regrouped per block tap: [32][4 * 64]
-    const int c = i & 7, row = (i >> 3) % BN, t = i / (8 * BN);
-    cp_async16(b_base + t * B_BLOCK + sw128_offset(row, c), w + ((size_t)row * NT + t) * TC_BK + c * 8, 16u);
+  if (warp == 16) tmem_alloc(&sh.tmem_base, 2 * BN);
+  // weight blocks: sequence q (0: taps of block row 0, 1: block row 1) = [zeros, tap 2q+1, tap 2q, zeros]
+  for (int i = threadIdx.x; i < 8 * 32 * 8; i += C1_THREADS) {
+    const int c = i & 7, row = (i >> 3) & 31, blk = i >> 8, q = blk >> 2, k = blk & 3;
+    const int tap = 2 * q + (k == 1 ? 1 : 0);
+    cp_async16(b_base + blk * W_BLOCK + sw128_offset(row, c), w + ((size_t)row * 4 + tap) * TC_BK + c * 8,
+               (k == 1 || k == 2) ? 16u : 0u);
   }
   cp_async_commit();
   cp_async_wait<0>();
@@ -1035,114 +1060,136 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
 
-  if (warp >= 4 && warp < 12) {
-    // ---------------- producers ----------------
-    const int p = threadIdx.x - 128;
-    // block rows of a tile: raster positions q0 .. q0 + 149 (clamped to the last one), at most nine block rows in
-    // at most two states, i.e. at most 36 whole frame rows, contiguous per state
-    auto tile_ranges = [&](int t, int& b0, int& r0, int& n0, int& n1) {
-      const int qf = t * TC_BM, ql = min(qf + C1_USED_ROWS - 1, total_pos - 1);
-      b0 = qf / POS;
-      const int b1 = ql / POS, yf = (qf % POS) / C1_RASTER, yl = (ql % POS) / C1_RASTER;
-      r0 = 4 * yf;
-      if (b1 == b0) { n0 = 4 * (yl - yf + 1); n1 = 0; }
-      else { n0 = G::H - r0; n1 = 4 * (yl + 1); }
-    };
-    auto stage_rows = [&](int t, int slot) {
-      if (t < tiles) {
-        int b0, r0, n0, n1;
-        tile_ranges(t, b0, r0, n0, n1);
-        const uint8_t* src0 = frames + ((size_t)b0 * G::H + r0) * ROW_BYTES;
-        const uint8_t* src1 = frames + (size_t)(b0 + 1) * G::H * ROW_BYTES;
-        const int c0 = n0 * (ROW_BYTES / 16), c1 = n1 * (ROW_BYTES / 16);
-        const uint32_t dst = raw_base + slot * RAW_BYTES;
-        for (int i = p; i < c0 + c1; i += NPROD)
-          cp_async16(dst + i * 16, i < c0 ? src0 + (size_t)i * 16 : src1 + (size_t)(i - c0) * 16, 16u);
-      }
-      cp_async_commit();        // always one group per call, so the wait counts stay uniform
-    };
+  // frame rows of tile t: raster positions qf .. ql, at most fifteen block rows in at most two states
+  auto tile_ranges = [&](int t, int& b0, int& r0, int& n0, int& n1) {
+    const int qf = t * C1_TILE_POS, ql = min(qf + C1_USED_POS - 1, total_pos - 1);
+    b0 = qf / POS;
+    const int b1 = ql / POS, yf = (qf % POS) / C1_RASTER, yl = (ql % POS) / C1_RASTER;
+    r0 = 4 * yf;
+    if (b1 == b0) { n0 = 4 * (yl - yf + 1); n1 = 0; }
+    else { n0 = G::H - r0; n1 = 4 * (yl + 1); }
+  };
+
+  if (warp >= 8 && warp < 16) {
+    // ---------------- producers: raw bytes -> bf16 operand rows ----------------
+    const int p = threadIdx.x - 256;
     int local = 0;
-    bool alive = true;
-    stage_rows(blockIdx.x, 0);
-    stage_rows(blockIdx.x + gridDim.x, 1);
-    for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x, ++local) {
-      cp_async_wait<1>();                                              // this tile's rows (my share) have landed
-      asm volatile("bar.sync 1, %0;" ::"n"(NPROD) : "memory");        // everyone's share has; the slot of tile-1 is free
-      stage_rows(t + 2 * gridDim.x, (local + 2) % 3);
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
+      const int s = local % STAGES, slot = local % C1_RAW_SLOTS;
       int b0, r0, n0, n1;
       tile_ranges(t, b0, r0, n0, n1);
-      const int s = local % STAGES;
-      const bool ok = mbar_wait(&sh.empty[s], ((local / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
-      if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
-      const uint32_t stage = a_base0 + s * A_BYTES, raw = raw_base + (local % 3) * RAW_BYTES;
-      // work item = (block row ri of the stage, pixel row py of the block): 16 raw bytes -> two operand chunks
-      for (int item = p; item < C1_USED_ROWS * 4; item += NPROD) {
-        const int ri = item >> 2, py = item & 3;
-        const int q = min(t * TC_BM + ri, total_pos - 1);
-        const int b = q / POS, rem = q % POS, Y = rem / C1_RASTER, X = rem % C1_RASTER;
+      bool ok = mbar_wait(&sh.raw_full[slot], (local / C1_RAW_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      ok = ok && mbar_wait(&sh.empty[s], ((local / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const uint32_t stage = a_base0 + s * A_BYTES, raw = raw_base + slot * C1_RAW_BYTES;
+      // work item = (position u of the tile, pixel row py of its block): 16 raw bytes -> two operand chunks;
+      // thread p takes items p, p + 256, ...: the same py, positions 64 apart (3 block rows + 1 block)
+      const int py = p & 3;
+      int u = p >> 2, b, Y, X;
+      {
+        const int q = t * C1_TILE_POS + u;
+        b = q / POS;
+        const int rem = q - b * POS;
+        Y = rem / C1_RASTER; X = rem - Y * C1_RASTER;
+      }
+      uint4 rw[5];
+#pragma unroll
+      for (int k = 0; k < 5; ++k) {
+        if (b >= n_states) { b = n_states - 1; Y = C1_RASTER - 1; X = C1_RASTER - 1; }     // past the end: repeat the last block
         const int slot_row = (b == b0 ? 4 * Y - r0 : n0 + 4 * Y) + py;
-        uint32_t r0w, r1w, r2w, r3w, o[8];
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0w), "=r"(r1w), "=r"(r2w), "=r"(r3w)
-                     : "r"(raw + (uint32_t)(slot_row * ROW_BYTES + X * 16)) : "memory");
-        u8x4_to_bf16x4(r0w, o[0], o[1]); u8x4_to_bf16x4(r1w, o[2], o[3]);
-        u8x4_to_bf16x4(r2w, o[4], o[5]); u8x4_to_bf16x4(r3w, o[6], o[7]);
-        const uint32_t dst = stage + (uint32_t)ri * 128u;
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py) ^ (ri & 7)) << 4)),
-                     "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py + 1) ^ (ri & 7)) << 4)),
-                     "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+        if (u + 64 * k < C1_USED_POS)
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(rw[k].x), "=r"(rw[k].y), "=r"(rw[k].z), "=r"(rw[k].w)
+                       : "r"(raw + (uint32_t)(slot_row * ROW_BYTES + X * 16)) : "memory");
+        X += 1; Y += 3;
+        if (X >= C1_RASTER) { X -= C1_RASTER; ++Y; }
+        if (Y >= C1_RASTER) { Y -= C1_RASTER; ++b; }
+      }
+#pragma unroll
+      for (int k = 0; k < 5; ++k) {
+        const int uu = u + 64 * k;
+        if (uu < C1_USED_POS) {
+          uint32_t o[8];
+          u8x4_to_bf16x4(rw[k].x, o[0], o[1]); u8x4_to_bf16x4(rw[k].y, o[2], o[3]);
+          u8x4_to_bf16x4(rw[k].z, o[4], o[5]); u8x4_to_bf16x4(rw[k].w, o[6], o[7]);
+          const uint32_t ri = (uint32_t)(uu >> 1), dst = stage + (uu & 1) * PLANE_BYTES + ri * 128u;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py) ^ (ri & 7)) << 4)),
+                       "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py + 1) ^ (ri & 7)) << 4)),
+                       "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+        }
       }
       fence_proxy_async_smem();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.full[s]);
+      if (lane == 0) { mbar_arrive(&sh.full[s]); mbar_arrive(&sh.raw_empty[slot]); }
     }
-    cp_async_wait<0>();
-  } else if (warp < 4) {
+  } else if (warp < 8) {
     // ---------------- epilogue ----------------
+    const int quarter = warp & 3, h = warp >> 2;
     int local = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
-      const int ab = local & 1, pos = t * TC_BM + threadIdx.x;
+      const int ab = local & 1, pos = t * C1_TILE_POS + 2 * (quarter * 32 + lane) + h;
+      const int b = pos / POS, rem = pos % POS, Y = rem / C1_RASTER, X = rem % C1_RASTER;
       const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
       uint32_t r[32];
-      tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN, r);
-      const int b = pos / POS, rem = pos % POS, Y = rem / C1_RASTER, X = rem % C1_RASTER;
-      if (b < n_states && Y < G::OH && X < G::OW) epi((b * G::OH + Y) * G::OW + X, 0, 0, r);
+      tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + ab * BN + h * 32, r);
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
+      if (b < n_states && Y < G::OH && X < G::OW) epi((b * G::OH + Y) * G::OW + X, 0, 0, r);
     }
-  } else if (warp == 12 && lane == 0) {
-    // ---------------- MMA issuer ----------------
-    constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
-    const uint32_t hi = desc_hi_kmajor_sw128(), b_lo = (b_base >> 4) & 0x3FFFu;
-    int local = 0;
-    bool ok = true;
-    for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++local) {
-      const int ab = local & 1, s = local % STAGES;
-      ok = mbar_wait(&sh.acc_empty[ab], ((local >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
-      if (!ok) break;
-      ok = mbar_wait(&sh.full[s], (local / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
-      if (!ok) break;
-      tcgen05_fence_after();
-      const uint32_t a_lo = ((a_base0 + s * A_BYTES) >> 4) & 0x3FFFu, d = tmem + ab * BN;
+  } else if (warp == 16) {
+    if (lane == 0) {
+      // ---------------- MMA issuer ----------------
+      constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
+      const uint32_t hi = desc_hi_kmajor_sw128(), b_lo = (b_base >> 4) & 0x3FFFu;
+      int local = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++local) {
+        const int ab = local & 1, s = local % STAGES;
+        ok = mbar_wait(&sh.acc_empty[ab], ((local >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
+        if (!ok) break;
+        ok = mbar_wait(&sh.full[s], (local / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const uint32_t a_lo = ((a_base0 + s * A_BYTES) >> 4) & 0x3FFFu, d = tmem + ab * BN;
 #pragma unroll
-      for (int tap = 0; tap < NT; ++tap) {
-        const uint32_t a_off = (((tap >> 1) * C1_RASTER + (tap & 1)) * 128u) >> 4, b_off = (tap * B_BLOCK) >> 4;
+        for (int v = 0; v < 6; ++v) {
+          // view v: plane (E = 0, O = 1), rows down, first weight block of its 64-row window
+          constexpr int plane[6] = {0, 1, 0, 1, 0, 1}, shift[6] = {0, 0, 1, 10, 11, 11}, wblk[6] = {2, 1, 0, 6, 5, 4};
+          const uint32_t a_off = (plane[v] * PLANE_BYTES + shift[v] * 128u) >> 4, b_off = (wblk[v] * W_BLOCK) >> 4;
 #pragma unroll
-        for (int k = 0; k < TC_BK / 16; ++k) {
-          if (tap == 0 && k == 0) mma_bf16_lo<false>(d, a_lo + a_off, b_lo + b_off, hi, idesc);
-          else mma_bf16_lo<true>(d, a_lo + a_off + k * 2, b_lo + b_off + k * 2, hi, idesc);
+          for (int k = 0; k < TC_BK / 16; ++k) {
+            if (v == 0 && k == 0) mma_bf16_lo<false>(d, a_lo + a_off, b_lo + b_off, hi, idesc);
+            else mma_bf16_lo<true>(d, a_lo + a_off + k * 2, b_lo + b_off + k * 2, hi, idesc);
+          }
         }
+        mma_commit(&sh.empty[s]);
+        mma_commit(&sh.acc_full[ab]);
       }
-      mma_commit(&sh.empty[s]);
-      mma_commit(&sh.acc_full[ab]);
+    }
+  } else if (lane == 0) {
+    // ---------------- raw loader ----------------
+    int local = 0;
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
+      const int slot = local % C1_RAW_SLOTS;
+      if (!mbar_wait(&sh.raw_empty[slot], ((local / C1_RAW_SLOTS) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY)) break;
+      int b0, r0, n0, n1;
+      tile_ranges(t, b0, r0, n0, n1);
+      const uint32_t dst = raw_base + slot * C1_RAW_BYTES;
+      mbar_arrive_expect_tx(&sh.raw_full[slot], (uint32_t)((n0 + n1) * ROW_BYTES));
+      bulk_copy_g2s(dst, frames + ((size_t)b0 * G::H + r0) * ROW_BYTES, (uint32_t)(n0 * ROW_BYTES), &sh.raw_full[slot]);
+      if (n1 > 0)
+        bulk_copy_g2s(dst + n0 * ROW_BYTES, frames + (size_t)(b0 + 1) * G::H * ROW_BYTES, (uint32_t)(n1 * ROW_BYTES),
+                      &sh.raw_full[slot]);
     }
   }
+  // Every issued bulk copy has been waited for by the producers (or the CTA is aborting after a bounded wait gave
+  // up, in which case the copies in flight still land in this CTA's shared memory before it retires).
   tcgen05_fence_before();
   __syncthreads();
-  if (warp == 12) {
+  if (warp == 16) {
     __syncwarp();
     tcgen05_fence_after();
     tmem_dealloc(tmem, 2 * BN);
@@ -1194,15 +1241,16 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
 
 template <class G, class Epi>
 static void tc_conv1(LaunchCtx& lc, const uint8_t* frames, const bf16* w_blocks, Epi e, int n_states, uint32_t* err) {
-  constexpr int STAGES = 6;
-  constexpr int smem = 4 * 32 * 128 + STAGES * C1_STAGE_ROWS * 128 + 3 * C1_RAW_BYTES + 1024;
+  constexpr int STAGES = 3;
+  constexpr int smem = 8 * 32 * 128 + STAGES * 2 * C1_PLANE_ROWS * 128 + C1_RAW_SLOTS * C1_RAW_BYTES + 1024;
+  static_assert(smem <= 227 * 1024, "shared memory budget");
   auto kern = tc_conv1_kernel<G, Epi, STAGES>;
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     configured = true;
   }
-  const int tiles = (n_states * C1_RASTER * C1_RASTER + TC_BM - 1) / TC_BM;
+  const int tiles = (n_states * C1_RASTER * C1_RASTER + C1_TILE_POS - 1) / C1_TILE_POS;
   const int gx = tiles < sm_count() ? tiles : sm_count();
   KernelScope scope(lc, KID_CONV1_FWD);
   kern<<<gx, C1_THREADS, smem, lc.st>>>(frames, w_blocks, e, n_states, tiles, err);
@@ -1527,37 +1575,70 @@ __global__ void tc_bias_final_kernel(const float* __restrict__ part, int blocks,
 
 // One launch finishes every tensor-core weight gradient of an update: for each segment (a layer's weights, or
 // its bias with J = 1) dst[co * J + j] = scale * sum over splits of part[split][j][co], the splits added in a
-// fixed order.  Segments with many splits give eight threads to every output (each adds every 8th split,
-// the eight sums are then added in order); segments with few splits give one thread to every output.
+// fixed order.  The partial sums have co innermost and the gradient has j innermost, so every group of outputs
+// goes through a shared-memory tile: reads are whole 128-byte rows of co, writes whole runs of j.
+//   many splits: a group is 8 j x 32 co; warp w adds the splits w, w + 8, ... for all eight j (eight loads in
+//                flight per thread), the eight warps' sums are then added in warp order;
+//   few splits:  a group is 32 j x 32 co; warp w adds all splits, in order, for rows w, w + 8, w + 16, w + 24.
 __global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments segs) {
-  __shared__ float sh[8][33];
-  const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
+  __shared__ float sh[8 * 8 * 33];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int grp = blockIdx.x; grp < segs.total_groups; grp += gridDim.x) {
     int si = 0;
     while (si + 1 < segs.n && grp >= segs.seg[si + 1].first_group) ++si;
     const GradSegment& sg = segs.seg[si];
-    const int total = sg.J * sg.CO, local = grp - sg.first_group;
+    const int local = grp - sg.first_group, co_tiles = (sg.CO + 31) / 32;
+    const int co0 = (local % co_tiles) * 32, J = sg.J, CO = sg.CO;
+    const size_t total = (size_t)J * CO;
+    const bool co_ok = co0 + lane < CO;
     if (sg.wide) {
-      const int i = local * 32 + lane;
-      float s = 0.f;
-      if (i < total)
-        for (int p = part; p < sg.splits; p += 8) s += sg.part[(size_t)p * total + i];
-      sh[part][lane] = s;
+      const int j0 = (local / co_tiles) * 8;
+      float acc[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+      const float* src = sg.part + (size_t)j0 * CO + co0 + lane;
+      for (int p = warp; p < sg.splits; p += 8) {
+        float v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = (co_ok && j0 + q < J) ? __ldg(src + (size_t)p * total + (size_t)q * CO) : 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) acc[q] += v[q];
+      }
+#pragma unroll
+      for (int q = 0; q < 8; ++q) sh[(warp * 8 + q) * 33 + lane] = acc[q];
       __syncthreads();
-      if (part == 0 && i < total) {
+      {
+        const int c = threadIdx.x >> 3, q = threadIdx.x & 7;       // eight consecutive threads write 32 contiguous bytes
         float t = 0.f;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) t += sh[q][lane];
-        sg.dst[(size_t)(i % sg.CO) * sg.J + i / sg.CO] = t * sg.scale;
+        for (int w = 0; w < 8; ++w) t += sh[(w * 8 + q) * 33 + c];
+        if (co0 + c < CO && j0 + q < J) sg.dst[(size_t)(co0 + c) * J + j0 + q] = t * sg.scale;
       }
       __syncthreads();
     } else {
-      const int i = local * 256 + threadIdx.x;
-      if (i < total) {
-        float s = 0.f;
-        for (int p = 0; p < sg.splits; ++p) s += sg.part[(size_t)p * total + i];
-        sg.dst[(size_t)(i % sg.CO) * sg.J + i / sg.CO] = s * sg.scale;
+      const int j0 = (local / co_tiles) * 32;
+      float t[4] = {0.f, 0.f, 0.f, 0.f};
+      const float* src = sg.part + (size_t)(j0 + warp) * CO + co0 + lane;
+      bool ok[4];
+#pragma unroll
+      for (int rr = 0; rr < 4; ++rr) ok[rr] = co_ok && j0 + warp + 8 * rr < J;
+#pragma unroll 4
+      for (int p = 0; p < sg.splits; ++p) {
+        float v[4];
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr) v[rr] = ok[rr] ? __ldg(src + (size_t)p * total + (size_t)(8 * rr) * CO) : 0.f;
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr) t[rr] += v[rr];
       }
+#pragma unroll
+      for (int rr = 0; rr < 4; ++rr) sh[(warp + 8 * rr) * 33 + lane] = t[rr];
+      __syncthreads();
+#pragma unroll
+      for (int rr = 0; rr < 4; ++rr) {
+        const int c = warp + 8 * rr;
+        if (co0 + c < CO && j0 + lane < J) sg.dst[(size_t)(co0 + c) * J + j0 + lane] = sh[lane * 33 + c] * sg.scale;
+      }
+      __syncthreads();
     }
   }
 }
@@ -1567,7 +1648,7 @@ static void add_segment(GradSegments* segs, const float* part, float* dst, int s
   g.part = part; g.dst = dst; g.splits = splits; g.J = J; g.CO = CO; g.scale = scale;
   g.wide = splits > 8;
   g.first_group = segs->total_groups;
-  g.groups = (J * CO + (g.wide ? 32 : 256) - 1) / (g.wide ? 32 : 256);
+  g.groups = ((J + (g.wide ? 8 : 32) - 1) / (g.wide ? 8 : 32)) * ((CO + 31) / 32);
   segs->total_groups += g.groups;
 }
 

@@ -149,6 +149,17 @@ __device__ __forceinline__ void cp_async_mbar_arrive(uint64_t* bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// ---- bulk copies global -> shared, completion counted in bytes on an mbarrier -----------------------------------
+// the calling thread's arrival, which also tells the barrier how many bytes of bulk copies to expect in this phase
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// contiguous copy by the copy engine; both addresses 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
 // ---- shared-memory images ----------------------------------------------------------------------
 // 128-byte swizzle: within each 1024-byte group of eight 128-byte rows, the 16-byte chunk c of
 // row r lives at chunk position c ^ (r & 7).  The same image serves a K-major operand (rows =
