@@ -197,8 +197,12 @@ int paac_debug_write(paac_ctx* ctx, int which, const void* src /* host */, size_
  * runs on the tensor cores; the others use the CUDA-core contraction.  Default: all.
  * PAAC_OPT_CUDA_GRAPHS: != 0 (default) lets paac_rollout / paac_update record their kernel sequence into CUDA
  * graphs after two plain iterations and replay them; 0 keeps every call on plain launches.  (Graphs are also
- * bypassed while actions are forced or per-kernel profiling is on.) */
-enum { PAAC_OPT_CUDA_CORES_ONLY = 1, PAAC_OPT_TC_WGRAD_LAYERS = 2, PAAC_OPT_CUDA_GRAPHS = 3 };
+ * bypassed while actions are forced or per-kernel profiling is on.)
+ * PAAC_OPT_DEPENDENT_LAUNCH: != 0 (default) launches every kernel with programmatic stream serialization, so
+ * that a kernel's CTAs are scheduled while the kernel before it drains (each kernel waits on the device for its
+ * predecessor before it touches that kernel's data); 0 launches with plain stream order.  The setting is
+ * process-wide.  Results are bit-identical either way. */
+enum { PAAC_OPT_CUDA_CORES_ONLY = 1, PAAC_OPT_TC_WGRAD_LAYERS = 2, PAAC_OPT_CUDA_GRAPHS = 3, PAAC_OPT_DEPENDENT_LAUNCH = 4 };
 int paac_set_option(paac_ctx* ctx, int option, int value);
 
 /* Number of kernels the library has launched on this context since init. */

@@ -174,6 +174,7 @@ template <class F> void run_recorded(paac_ctx* c, int kind, int parity, F enqueu
     cudaGraph_t g = nullptr;
     if (cudaStreamBeginCapture(c->st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
       const uint64_t before = c->lc.count;
+      c->lc.serialize_next = true;
       enqueue();
       const uint64_t launched = c->lc.count - before;
       cudaGraphExec_t exec = nullptr;
@@ -194,6 +195,7 @@ template <class F> void run_recorded(paac_ctx* c, int kind, int parity, F enqueu
       c->graphs_on = false;
     }
   }
+  c->lc.serialize_next = true;
   enqueue();
   ++c->plain_calls[kind][parity];
 }
@@ -348,6 +350,7 @@ int paac_params(paac_ctx* c, float* dst, size_t n) {
 }
 
 int paac_set_params(paac_ctx* c, const float* src, size_t n) {
+  if (c) c->lc.serialize_next = true;
   if (!c || !src || n != c->nd.P) return PAAC_ERR_ARG;
   if (cudaMemcpyAsync(c->theta, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
     cudaGetLastError(); return PAAC_ERR_CUDA;
@@ -400,6 +403,7 @@ int paac_set_option(paac_ctx* c, int option, int value) {
   if (option == PAAC_OPT_CUDA_CORES_ONLY) { c->simt_only = value != 0; drop_graphs(c); return PAAC_OK; }
   if (option == PAAC_OPT_TC_WGRAD_LAYERS) { c->tc_wgrad_mask = value & 0xF; drop_graphs(c); return PAAC_OK; }
   if (option == PAAC_OPT_CUDA_GRAPHS) { c->graphs_on = value != 0; drop_graphs(c); return PAAC_OK; }
+  if (option == PAAC_OPT_DEPENDENT_LAUNCH) { pdl_enabled() = value != 0; drop_graphs(c); return PAAC_OK; }
   return PAAC_ERR_ARG;
 }
 
@@ -427,6 +431,7 @@ int paac_profile_read(paac_ctx* c, int max_entries, const char** names, double* 
 
 // ---- external-environment mode ------------------------------------------------------------------
 int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, float* values) {
+  if (c) c->lc.serialize_next = true;
   if (!c || !frames || t < 0 || t > c->t_max || (t < c->t_max && !actions)) return PAAC_ERR_ARG;
   if (t != c->host_t) return PAAC_ERR_STATE;
   const size_t fstep = (size_t)c->n_e * FRAME_BYTES;
@@ -450,6 +455,7 @@ int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, f
 }
 
 int paac_observe_host(paac_ctx* c, int t, const int8_t* rewards, const uint8_t* terminals) {
+  if (c) c->lc.serialize_next = true;
   if (!c || !rewards || !terminals || t < 0 || t >= c->t_max) return PAAC_ERR_ARG;
   if (t + 1 != c->host_t) return PAAC_ERR_STATE;
   const size_t row = (size_t)t * c->n_e;
@@ -512,6 +518,7 @@ int paac_debug_read(paac_ctx* c, int which, void* dst, size_t bytes) {
 }
 
 int paac_debug_write(paac_ctx* c, int which, const void* src, size_t bytes) {
+  if (c) c->lc.serialize_next = true;
   if (!c || !src) return PAAC_ERR_ARG;
   size_t b = 0;
   void* p = debug_ptr(c, which, &b);

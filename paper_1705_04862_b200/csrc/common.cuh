@@ -142,6 +142,7 @@ struct LaunchCtx {
   cudaStream_t st = nullptr;
   uint64_t count = 0;                 // kernels launched so far
   bool profiling = false;             // record a CUDA event pair around every launch
+  bool serialize_next = true;         // the next launch takes plain stream order (no overlap with its predecessor)
   static constexpr int MAX_PENDING = 512;
   cudaEvent_t ev[MAX_PENDING][2];
   int ev_kid[MAX_PENDING];
@@ -180,6 +181,48 @@ struct KernelScope {
   }
   ~KernelScope() { if (slot >= 0) cudaEventRecord(lc.ev[slot][1], lc.st); }
 };
+
+// ---- programmatic dependent launch ----------------------------------------------------------------------------
+// The tensor-core kernels are launched with programmatic stream serialization: their CTAs may be scheduled while
+// the kernel before them in the stream is still draining, which hides the launch latency and lets a CTA set itself
+// up on an SM as soon as the previous kernel's CTA there has left.  The contract every kernel keeps:
+//   pdl_wait() comes before the first access to anything the PREVIOUS kernel in the stream writes or reads-then-
+//   overwrites; it returns once that kernel has completed and its writes are visible.  Only work on data that no
+//   neighbouring kernel touches (barrier set-up, tensor-memory allocation, weight tiles written several kernels
+//   earlier) may precede it;
+//   pdl_launch_dependents() comes after pdl_wait(), so at most two kernels ever overlap and everything older than
+//   the previous kernel is complete when a kernel starts.
+// Launched without the attribute (pdl_enabled() == false) both calls do nothing and stream order is the usual one.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_entry() { pdl_wait(); pdl_launch_dependents(); }
+
+inline bool& pdl_enabled() { static bool on = true; return on; }
+
+// The first launch after serialize_next was set (every API call sets it before it enqueues anything) gets plain
+// stream order, so that no kernel's set-up ever overlaps the last kernel of an earlier call (parameter updates
+// and weight re-layouts close an update).
+template <bool OVERLAP, class... KArgs, class... Args>
+inline cudaError_t launch_kernel_impl(LaunchCtx& lc, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = lc.st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = (OVERLAP && pdl_enabled() && !lc.serialize_next) ? 1 : 0;
+  lc.serialize_next = false;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+// plain stream order: for kernels that need their predecessor's data from the first instruction on
+template <class... KArgs, class... Args>
+inline cudaError_t launch_kernel(LaunchCtx& lc, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
+  return launch_kernel_impl<false>(lc, kern, grid, block, smem, args...);
+}
+// may start while its predecessor drains: for kernels whose set-up before pdl_wait() is worth overlapping
+template <class... KArgs, class... Args>
+inline cudaError_t launch_kernel_overlapped(LaunchCtx& lc, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
+  return launch_kernel_impl<true>(lc, kern, grid, block, smem, args...);
+}
 
 // device-side statistics block written by the update kernels
 struct DeviceStats {

@@ -7,6 +7,7 @@ namespace paac {
 // Philox uniform of counter (i, layer, 0, RNG_STREAM_INIT).  2u-1 is exact in float, so the
 // single rounding of the product is the same on any IEEE machine.
 __global__ void xavier_kernel(float* w, uint32_t count, float bound, uint32_t layer, uint64_t seed) {
+  pdl_entry();
   for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < count; i += gridDim.x * blockDim.x) {
     const float u = philox_uniform(i, layer, 0u, RNG_STREAM_INIT, seed);
     w[i] = __fmul_rn(__fsub_rn(__fmul_rn(2.0f, u), 1.0f), bound);
@@ -19,7 +20,7 @@ static void xavier(LaunchCtx& lc, float* w, size_t count, double fan_in, double 
   int blocks = (int)((count + 255) / 256);
   if (blocks > 1184) blocks = 1184;
   KernelScope scope(lc, KID_INIT);
-  xavier_kernel<<<blocks, 256, 0, lc.st>>>(w, (uint32_t)count, bound, layer, seed);
+  launch_kernel(lc, xavier_kernel, blocks, 256, 0, w, (uint32_t)count, bound, layer, seed);
 }
 
 void launch_init_params(LaunchCtx& lc, const NetDims& nd, uint64_t seed, float* theta) {
@@ -38,6 +39,7 @@ void launch_init_params(LaunchCtx& lc, const NetDims& nd, uint64_t seed, float* 
 }
 
 __global__ void cast_bf16_kernel(const float* src, bf16* dst, size_t n) {
+  pdl_entry();
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
     dst[i] = __float2bfloat16_rn(src[i]);
 }
@@ -45,7 +47,7 @@ void launch_cast_bf16(LaunchCtx& lc, const float* src, bf16* dst, size_t n) {
   int blocks = (int)((n + 255) / 256);
   if (blocks > 1184) blocks = 1184;
   KernelScope scope(lc, KID_CAST);
-  cast_bf16_kernel<<<blocks, 256, 0, lc.st>>>(src, dst, n);
+  launch_kernel(lc, cast_bf16_kernel, blocks, 256, 0, src, dst, n);
 }
 
 // One block per environment.  The block's first thread decides reward and terminal flag of
@@ -60,6 +62,7 @@ env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, 
                 const int32_t* __restrict__ actions, uint32_t term_denom,
                 uint8_t* __restrict__ next_frames, int8_t* __restrict__ rewards, uint8_t* __restrict__ terminals,
                 int32_t* __restrict__ counters) {
+  pdl_entry();
   __shared__ uint32_t s_base;
   const uint32_t e = blockIdx.x;
   if (threadIdx.x == 0) {
@@ -100,16 +103,17 @@ void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step
                      const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
                      uint8_t* terminals, int32_t* counters) {
   KernelScope scope(lc, KID_ENV_STEP);
-  env_step_kernel<<<n_e, ENV_THREADS, 0, lc.st>>>(seed, n_e, step_base, t, actions, term_denom, next_frames, rewards,
+  launch_kernel(lc, env_step_kernel, n_e, ENV_THREADS, 0, seed, n_e, step_base, t, actions, term_denom, next_frames, rewards,
                                                   terminals, counters);
 }
 
 // the environments' global step index lives on the device, so that a recorded sequence of launches can be
 // replayed for the next iteration without new arguments
-__global__ void advance_step_kernel(uint64_t* step_base, uint32_t by) { *step_base += by; }
+__global__ void advance_step_kernel(uint64_t* step_base, uint32_t by) {
+  pdl_entry(); *step_base += by; }
 void launch_advance_step(LaunchCtx& lc, uint64_t* step_base, uint32_t by) {
   KernelScope scope(lc, KID_ENV_STEP);
-  advance_step_kernel<<<1, 1, 0, lc.st>>>(step_base, by);
+  launch_kernel(lc, advance_step_kernel, 1, 1, 0, step_base, by);
 }
 
 }  // namespace paac

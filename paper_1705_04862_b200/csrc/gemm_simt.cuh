@@ -14,6 +14,7 @@ constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16, SG_THREADS = 256;
 template <class LA, class LB, class EP>
 __global__ void __launch_bounds__(SG_THREADS)
 gemm_simt_kernel(int M, int N, int K, int k_per_split, LA la, LB lb, EP ep) {
+  pdl_entry();
   __shared__ float As[SG_BK][SG_BM + 4];
   __shared__ float Bs[SG_BK][SG_BN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
@@ -74,7 +75,7 @@ inline void gemm_simt(LaunchCtx& lc, int kid, int M, int N, int K, int splits, L
   int kps = (K + splits - 1) / splits;
   kps = (kps + SG_BK - 1) / SG_BK * SG_BK;
   dim3 grid((M + SG_BM - 1) / SG_BM, (N + SG_BN - 1) / SG_BN, (K + kps - 1) / kps);
-  gemm_simt_kernel<<<grid, SG_THREADS, 0, lc.st>>>(M, N, K, kps, la, lb, ep);
+  launch_kernel(lc, gemm_simt_kernel<LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
 }
 // number of k-splits gemm_simt will really launch for a requested count
 inline int gemm_simt_splits(int K, int splits) {
@@ -181,6 +182,7 @@ struct PartialEp {
 // gradient) for rows row0 .. row0+rows-1 into the canonical gradient vector
 static __global__ void wgrad_reduce_kernel(const float* part, int splits, int part_rows, int row0, int rows, int cols,
                                            float scale, float* gw, float* gb) {
+  pdl_entry();
   const size_t total = (size_t)rows * (cols + 1), stride = (size_t)part_rows * (cols + 1);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const float* src = part + (size_t)row0 * (cols + 1) + i;

@@ -43,6 +43,7 @@ heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* _
              float* __restrict__ logits, float* __restrict__ values, uint64_t seed, const uint64_t* __restrict__ step_base, uint32_t t,
              const int32_t* __restrict__ forced, int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
              float* __restrict__ uniforms) {
+  pdl_entry();
   constexpr int F = 32 * EPL;
   const int lane = threadIdx.x & 31;
   const int e = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -99,6 +100,7 @@ heads_slow_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const flo
              float* __restrict__ logits, float* __restrict__ values, uint64_t seed, const uint64_t* __restrict__ step_base, uint32_t t,
              const int32_t* __restrict__ forced, int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
              float* __restrict__ uniforms) {
+  pdl_entry();
   const int lane = threadIdx.x & 31;
   const int e = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (e >= n) return;
@@ -148,17 +150,17 @@ void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta
   const float* bpi = theta + nd.pi_b; const float* bv = theta + nd.v_b;
   const bool aligned = nd.pi_w % 8 == 0;      // 16-byte loads of the policy rows
   if (prec == PAAC_BF16 && nd.F == 512 && aligned)
-    heads_kernel<bf16, bf16, 16><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
+    launch_kernel(lc, heads_kernel<bf16, bf16, 16>, blocks, 128, 0, (const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
                                                          nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms);
   else if (prec == PAAC_BF16 && nd.F == 256 && aligned)
-    heads_kernel<bf16, bf16, 8><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
+    launch_kernel(lc, heads_kernel<bf16, bf16, 8>, blocks, 128, 0, (const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
                                                         nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms);
   else if (prec == PAAC_BF16)
-    heads_slow_kernel<bf16, bf16><<<blocks, 128, 0, st>>>((const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv,
+    launch_kernel(lc, heads_slow_kernel<bf16, bf16>, blocks, 128, 0, (const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv,
                                                           n, nd.F, nd.A, logits, values, seed, step_base, t, forced, actions,
                                                           sampled, uniforms);
   else
-    heads_slow_kernel<float, float><<<blocks, 128, 0, st>>>((const float*)h, theta + nd.pi_w, bpi, theta + nd.v_w, bv,
+    launch_kernel(lc, heads_slow_kernel<float, float>, blocks, 128, 0, (const float*)h, theta + nd.pi_w, bpi, theta + nd.v_w, bv,
                                                             n, nd.F, nd.A, logits, values, seed, step_base, t, forced, actions,
                                                             sampled, uniforms);
 }
@@ -168,6 +170,7 @@ void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta
 __global__ void returns_kernel(int n_e, int t_max, float gamma, const int8_t* __restrict__ rewards,
                                const uint8_t* __restrict__ terminals, const float* __restrict__ values,
                                float* __restrict__ R, float* __restrict__ adv) {
+  pdl_entry();
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= n_e) return;
   float next = values[(size_t)t_max * n_e + e];
@@ -183,7 +186,7 @@ __global__ void returns_kernel(int n_e, int t_max, float gamma, const int8_t* __
 void launch_returns(LaunchCtx& lc, int n_e, int t_max, float gamma, const int8_t* rewards,
                     const uint8_t* terminals, const float* values, float* R, float* adv) {
   KernelScope scope(lc, KID_RETURNS);
-  returns_kernel<<<(n_e + 127) / 128, 128, 0, lc.st>>>(n_e, t_max, gamma, rewards, terminals, values, R, adv);
+  launch_kernel(lc, returns_kernel, (n_e + 127) / 128, 128, 0, n_e, t_max, gamma, rewards, terminals, values, R, adv);
 }
 
 // One warp per experience: d/dz and d/dV of
@@ -194,6 +197,7 @@ head_grad_kernel(int B, int A, float beta, float value_coef, const float* __rest
                  const float* __restrict__ values, const int32_t* __restrict__ actions, const float* __restrict__ R,
                  const float* __restrict__ adv, float* __restrict__ dz, float* __restrict__ dV,
                  float* __restrict__ loss_terms) {
+  pdl_entry();
   const int lane = threadIdx.x & 31;
   const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (i >= B) return;
@@ -222,6 +226,7 @@ head_grad_kernel(int B, int A, float beta, float value_coef, const float* __rest
 
 // single block: fixed-order (hence reproducible) means of the three loss terms
 __global__ void __launch_bounds__(256) loss_stats_kernel(int B, const float* __restrict__ loss_terms, DeviceStats* stats) {
+  pdl_entry();
   __shared__ float sh[3][256];
   float acc[3] = {0.f, 0.f, 0.f};
   for (int i = threadIdx.x; i < B; i += 256)
@@ -245,11 +250,11 @@ void launch_head_grad(LaunchCtx& lc, int B, int A, float beta, float value_coef,
                       const float* adv, float* dz, float* dV, float* loss_terms, DeviceStats* stats) {
   {
     KernelScope scope(lc, KID_HEAD_GRAD);
-    head_grad_kernel<<<(B + 3) / 4, 128, 0, lc.st>>>(B, A, beta, value_coef, logits, values, actions, R, adv, dz, dV,
+    launch_kernel(lc, head_grad_kernel, (B + 3) / 4, 128, 0, B, A, beta, value_coef, logits, values, actions, R, adv, dz, dV,
                                                      loss_terms);
   }
   KernelScope scope(lc, KID_HEAD_GRAD);
-  loss_stats_kernel<<<1, 256, 0, lc.st>>>(B, loss_terms, stats);
+  launch_kernel(lc, loss_stats_kernel, 1, 256, 0, B, loss_terms, stats);
 }
 
 }  // namespace paac

@@ -22,7 +22,7 @@ static void reduce_wgrad(LaunchCtx& lc, const float* part, int splits, int part_
   int blocks = (int)((total + 255) / 256);
   if (blocks > 2368) blocks = 2368;
   KernelScope scope(lc, KID_WGRAD_REDUCE);
-  wgrad_reduce_kernel<<<blocks, 256, 0, lc.st>>>(part, splits, part_rows, row0, rows, cols, scale, gw, gb);
+  launch_kernel(lc, wgrad_reduce_kernel, blocks, 256, 0, part, splits, part_rows, row0, rows, cols, scale, gw, gb);
 }
 
 template <class G, class TIn, class T, class TW>

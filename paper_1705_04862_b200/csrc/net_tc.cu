@@ -303,6 +303,7 @@ template <class G> struct ReluMaskEpiS2 {
 template <class ASrc, class BSrc, class Epi, int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS)
 tc_gemm_kernel(ASrc a_src, BSrc b_src, Epi epi, int num_kb, uint32_t* error_word) {
+  pdl_entry();
   static_assert(BN == 32 || BN == 64 || BN == 128, "tile width");
   constexpr uint32_t A_BYTES = TC_BM * 128, B_BYTES = BN * 128, STAGE_BYTES = A_BYTES + B_BYTES;
   extern __shared__ uint8_t dyn_smem[];
@@ -437,6 +438,7 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
+  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
   if (warp >= 4 && warp < 8) {
     // ---------------- producers ----------------
@@ -583,6 +585,7 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
+  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
   if (warp >= 8 && warp < 16) {
     // ---------------- producers: eight lanes per 128-byte row, 32 rows per pass ----------------
@@ -860,6 +863,7 @@ tc_splitk_kernel(const bf16* __restrict__ a, const bf16* __restrict__ w, float* 
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
+  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
   if (warp >= 4 && warp < 8) {
     // ---------------- producers: lane l copies chunk l & 7 of rows 32 pw + 4 p + (l >> 3) of both tiles ----------------
@@ -958,6 +962,7 @@ tc_splitk_kernel(const bf16* __restrict__ a, const bf16* __restrict__ w, float* 
 // out[m][n..n+7] = bf16(relu(sum_s part[s][m][n] + bias[n]))
 __global__ void __launch_bounds__(256) fc_finish_kernel(const float* __restrict__ part, int splits, int M, int N,
                                                         const float* __restrict__ bias, bf16* __restrict__ out) {
+  pdl_entry();
   const size_t total = (size_t)M * N / 8;
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
     const size_t e = i * 8;
@@ -1059,6 +1064,7 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
+  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
   // frame rows of tile t: raster positions qf .. ql, at most fifteen block rows in at most two states
   auto tile_ranges = [&](int t, int& b0, int& r0, int& n0, int& n1) {
@@ -1221,7 +1227,7 @@ static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_t
   if (gx < 1) gx = 1;
   if (gx > NCLS * tiles_m) gx = NCLS * tiles_m;
   KernelScope scope(lc, kid);
-  kern<<<dim3(gx, gy), PK_THREADS, smem, lc.st>>>(a, w, n_total, e, tiles_m, err);
+  launch_kernel_overlapped(lc, kern, dim3(gx, gy), PK_THREADS, smem, a, w, n_total, e, tiles_m, err);
 }
 
 template <class Cfg, class Epi, int BN, int STAGES, int NACC>
@@ -1236,7 +1242,7 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
   }
   const int tiles = (positions + TC_BM - 1) / TC_BM;
   KernelScope scope(lc, kid);
-  kern<<<tiles < sm_count() ? tiles : sm_count(), SH_THREADS, smem, lc.st>>>(cfg, w, e, tiles, err);
+  launch_kernel_overlapped(lc, kern, tiles < sm_count() ? tiles : sm_count(), SH_THREADS, smem, cfg, w, e, tiles, err);
 }
 
 template <class G, class Epi>
@@ -1253,7 +1259,7 @@ static void tc_conv1(LaunchCtx& lc, const uint8_t* frames, const bf16* w_blocks,
   const int tiles = (n_states * C1_RASTER * C1_RASTER + C1_TILE_POS - 1) / C1_TILE_POS;
   const int gx = tiles < sm_count() ? tiles : sm_count();
   KernelScope scope(lc, KID_CONV1_FWD);
-  kern<<<gx, C1_THREADS, smem, lc.st>>>(frames, w_blocks, e, n_states, tiles, err);
+  launch_kernel_overlapped(lc, kern, gx, C1_THREADS, smem, frames, w_blocks, e, n_states, tiles, err);
 }
 
 template <class ASrc, class BSrc, class Epi, int BN, int STAGES>
@@ -1267,7 +1273,7 @@ static void tc_gemm(LaunchCtx& lc, int kid, ASrc a, BSrc b, Epi e, int M, int N,
   }
   KernelScope scope(lc, kid);
   dim3 grid((M + TC_BM - 1) / TC_BM, N / BN, Z);
-  kern<<<grid, TC_THREADS, smem, lc.st>>>(a, b, e, num_kb, error_word);
+  launch_kernel_overlapped(lc, kern, grid, TC_THREADS, smem, a, b, e, num_kb, error_word);
 }
 
 constexpr int FC_SPLITS = 7;
@@ -1286,12 +1292,12 @@ static void tc_fc_forward(LaunchCtx& lc, const bf16* a, const bf16* w, const flo
   const int total = tiles_m * tiles_n * splits;
   {
     KernelScope scope(lc, KID_FC_FWD);
-    tc_splitk_kernel<<<total < sm_count() ? total : sm_count(), PK_THREADS, smem, lc.st>>>(a, w, part, M, N, K, tiles_m,
+    launch_kernel_overlapped(lc, tc_splitk_kernel, total < sm_count() ? total : sm_count(), PK_THREADS, smem, a, w, part, M, N, K, tiles_m,
                                                                                          tiles_n, splits, kb_per, err);
   }
   KernelScope scope(lc, KID_FC_FWD);
   const int blocks = (M * N / 8 + 255) / 256;
-  fc_finish_kernel<<<blocks < 1184 ? blocks : 1184, 256, 0, lc.st>>>(part, splits, M, N, bias, out);
+  launch_kernel(lc, fc_finish_kernel, blocks < 1184 ? blocks : 1184, 256, 0, part, splits, M, N, bias, out);
 }
 
 // ---- forward ---------------------------------------------------------------------------------------------
@@ -1395,6 +1401,7 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, float* __re
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
+  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
   if (warp < 4) {
     // ---------------- producers: thread = (row of the block, half) ----------------
@@ -1547,6 +1554,7 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, float* __re
 // its 8 thread rows each add every 8th split, then the 8 sums are added in a fixed order.
 __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* __restrict__ partial, int splits, int J, int CO,
                                                               float scale, float* __restrict__ gw) {
+  pdl_entry();
   __shared__ float sh[8][33];
   const int total = J * CO, lane = threadIdx.x & 31, part = threadIdx.x >> 5;
   const int i = blockIdx.x * 32 + lane;
@@ -1566,6 +1574,7 @@ __global__ void __launch_bounds__(256) tc_wgrad_reduce_kernel(const float* __res
 
 // bias gradient: the per-split column sums written by the weight-gradient kernel, added in split order
 __global__ void tc_bias_final_kernel(const float* __restrict__ part, int blocks, int CO, float* __restrict__ gb) {
+  pdl_entry();
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (c >= CO) return;
   float s = 0.f;
@@ -1581,6 +1590,7 @@ __global__ void tc_bias_final_kernel(const float* __restrict__ part, int blocks,
 //                flight per thread), the eight warps' sums are then added in warp order;
 //   few splits:  a group is 32 j x 32 co; warp w adds all splits, in order, for rows w, w + 8, w + 16, w + 24.
 __global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments segs) {
+  pdl_entry();
   __shared__ float sh[8 * 8 * 33];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int grp = blockIdx.x; grp < segs.total_groups; grp += gridDim.x) {
@@ -1683,7 +1693,7 @@ static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, int rows, int n_a
   const int splits = (num_blocks + bps - 1) / bps;
   float* bias_part = scratch + (size_t)splits * J * CO;
   KernelScope scope(lc, kid);
-  kern<<<dim3(splits, gy, gz), TC_THREADS, smem, lc.st>>>(xs, gs, scratch, bias_part, n_atoms, J, CO, num_blocks, bps, err);
+  launch_kernel_overlapped(lc, kern, dim3(splits, gy, gz), TC_THREADS, smem, xs, gs, scratch, bias_part, n_atoms, J, CO, num_blocks, bps, err);
   add_segment(segs, scratch, gw, splits, J, CO, scale);
   add_segment(segs, bias_part, gb, splits, 1, CO, 1.f);
 }
@@ -1759,6 +1769,7 @@ tc_shift_wgrad_kernel(Cfg cfg, const bf16* __restrict__ g, int states, float* __
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
+  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
   if (warp < 8) {
     // ---------------- producers: eight lanes per 128-byte row, 32 rows per pass ----------------
@@ -1895,7 +1906,7 @@ static void tc_shift_wgrad(LaunchCtx& lc, int kid, Cfg cfg, const bf16* g, int s
   const int splits = swg_splits(positions), per = (tiles + splits - 1) / splits;
   float* bias_part = scratch + (size_t)splits * J * 64;
   KernelScope scope(lc, kid);
-  kern<<<splits, SWG_THREADS, smem, lc.st>>>(cfg, g, states, scratch, bias_part, tiles, per, err);
+  launch_kernel_overlapped(lc, kern, splits, SWG_THREADS, smem, cfg, g, states, scratch, bias_part, tiles, per, err);
   add_segment(segs, scratch, gw, splits, J, 64, 1.f);
   add_segment(segs, bias_part, gb, splits, 1, 64, 1.f);
 }
@@ -1942,6 +1953,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
+  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
   float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 
   if (warp < 10) {
@@ -2086,7 +2098,7 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
   const int splits = n_states < sm_count() ? n_states : sm_count();
   float* bias_part = scratch + (size_t)splits * 256 * 32;
   KernelScope scope(lc, KID_CONV1_WGRAD);
-  kern<<<splits, W1_THREADS, smem, lc.st>>>(frames, g, scratch, bias_part, n_states, err);
+  launch_kernel_overlapped(lc, kern, splits, W1_THREADS, smem, frames, g, scratch, bias_part, n_states, err);
   add_segment(segs, scratch, gw, splits, 256, 32, 1.0f / 255.0f);
   add_segment(segs, bias_part, gb, splits, 1, 32, 1.f);
 }
@@ -2114,7 +2126,7 @@ void tc_backward_finish(LaunchCtx& lc, GradSegments* segs) {
   if (segs->n > 0) {
     KernelScope scope(lc, KID_WGRAD_REDUCE);
     const int blocks = segs->total_groups < 8 * sm_count() ? segs->total_groups : 8 * sm_count();
-    tc_finalize_grads_kernel<<<blocks, 256, 0, lc.st>>>(*segs);
+    launch_kernel(lc, tc_finalize_grads_kernel, blocks, 256, 0, *segs);
   }
   segs->n = 0; segs->total_groups = 0;
 }
@@ -2149,6 +2161,7 @@ __global__ void relayout_weights_kernel(const bf16* __restrict__ w1, const bf16*
                                         const bf16* __restrict__ w3, const bf16* __restrict__ wfc,
                                         bf16* __restrict__ w2_d, bf16* __restrict__ w3_d, bf16* __restrict__ wfc_t,
                                         bf16* __restrict__ w1_b) {
+  pdl_entry();
   typedef NatConv2 C2; typedef NatConv3 C3;
   constexpr int N2 = 4 * C2::C * 4 * C2::CO, N3 = C3::C * 9 * C3::CO, NF = 3136 * 512, N1 = 32 * 256;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N2 + N3 + NF + N1; i += gridDim.x * blockDim.x) {
@@ -2176,7 +2189,7 @@ size_t tc_weight_image_elems() { return TC_IMG_END; }
 void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, bf16* images) {
   const LayerDims* d = nd.layer;
   KernelScope scope(lc, KID_CAST);
-  relayout_weights_kernel<<<592, 256, 0, lc.st>>>(theta16 + d[0].w_off, theta16 + d[1].w_off, theta16 + d[2].w_off,
+  launch_kernel(lc, relayout_weights_kernel, 592, 256, 0, theta16 + d[0].w_off, theta16 + d[1].w_off, theta16 + d[2].w_off,
                                                   theta16 + d[3].w_off, images + TC_IMG_W2, images + TC_IMG_W3,
                                                   images + TC_IMG_WFC, images + TC_IMG_W1);
 }

@@ -8,6 +8,7 @@ constexpr int OPT_THREADS = 256;
 // pass 1: block b sums g^2 over its fixed slice of the parameter vector
 __global__ void __launch_bounds__(OPT_THREADS)
 sumsq_kernel(const float* __restrict__ g, size_t P, float* __restrict__ partials) {
+  pdl_entry();
   __shared__ float sh[OPT_THREADS];
   const size_t per = ((P + gridDim.x - 1) / gridDim.x + 3) / 4 * 4;
   const size_t lo = (size_t)blockIdx.x * per, hi = lo + per < P ? lo + per : P;
@@ -39,6 +40,7 @@ __global__ void __launch_bounds__(OPT_THREADS)
 clip_rmsprop_kernel(size_t P, float* __restrict__ theta, float* __restrict__ rms, const float* __restrict__ g,
                     bf16* __restrict__ theta16, float lr, float rho, float eps, float clip,
                     const float* __restrict__ partials, int n_partials, DeviceStats* stats) {
+  pdl_entry();
   __shared__ float sh[OPT_THREADS];
   __shared__ float s_scale;
   float acc = 0.f;
@@ -103,10 +105,10 @@ void launch_clip_rmsprop(LaunchCtx& lc, size_t P, float* theta, float* rms, cons
                          DeviceStats* stats) {
   {
     KernelScope scope(lc, KID_SUMSQ);
-    sumsq_kernel<<<NORM_BLOCKS, OPT_THREADS, 0, lc.st>>>(grad, P, norm_partials);
+    launch_kernel(lc, sumsq_kernel, NORM_BLOCKS, OPT_THREADS, 0, grad, P, norm_partials);
   }
   KernelScope scope(lc, KID_CLIP_RMSPROP);
-  clip_rmsprop_kernel<<<NORM_BLOCKS, OPT_THREADS, 0, lc.st>>>(P, theta, rms, grad, theta16, lr, rho, eps, clip,
+  launch_kernel(lc, clip_rmsprop_kernel, NORM_BLOCKS, OPT_THREADS, 0, P, theta, rms, grad, theta16, lr, rho, eps, clip,
                                                               norm_partials, NORM_BLOCKS, stats);
 }
 
