@@ -560,7 +560,6 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
   constexpr uint32_t PLANE_BYTES = SR * 128, STAGE_BYTES = PLANES * PLANE_BYTES, B_BLOCK = BN * 128, B_BYTES = NT * B_BLOCK;
   extern __shared__ uint8_t dyn_smem[];
   __shared__ PkShared sh;
-  __shared__ int cell_table[Cfg::RASTER > 0 ? Cfg::RASTER : 1];   // per-state raster cell -> source offset (or -1)
   const uint32_t b_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
   const uint32_t a_base0 = b_base + B_BYTES;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -572,8 +571,6 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
     fence_barrier_init();
   }
   if (warp == 16) tmem_alloc(&sh.tmem_base, 2 * NACC * BN);
-  if constexpr (Cfg::RASTER > 0)
-    for (int i = threadIdx.x; i < Cfg::RASTER; i += SH_THREADS) cell_table[i] = Cfg::cell(i);
   for (int i = threadIdx.x; i < NT * BN * 8; i += SH_THREADS) {
     const int c = i & 7, row = (i >> 3) % BN, t = i / (8 * BN);
     cp_async16(b_base + t * B_BLOCK + sw128_offset(row, c), w + ((size_t)row * NT + t) * TC_BK + c * 8, 16u);
@@ -597,13 +594,33 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
       const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
       if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
       const uint32_t stage = a_base0 + s * STAGE_BYTES;
-      for (int idx = sub; idx < PLANES * SR; idx += 32) {
-        const int plane = PLANES == 1 ? 0 : idx / SR, ri = PLANES == 1 ? idx : idx % SR;
-        bool valid;
-        const bf16* src;
-        if constexpr (Cfg::RASTER > 0) src = cfg.src_cell(t * TC_BM + ri, cell_table, valid);
-        else src = cfg.src(plane, t * TC_BM + ri, valid);
-        cp_async16(stage + plane * PLANE_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), src + c * 8, valid ? 16u : 0u);
+      // Source addresses by arithmetic only, all of them before the first copy.  A warp that has asynchronous copies
+      // in flight must not read shared memory (a table of raster cells, say): the load is made to wait until every
+      // one of those copies has landed, which chains the tiles to the memory latency.
+      constexpr int NIT = (PLANES * SR + 31) / 32;
+      uint32_t srcs[NIT], vmask = 0;                    // element offsets from the tensor's base (< 2^32 elements)
+#pragma unroll
+      for (int k = 0; k < NIT; ++k) {
+        const int idx = sub + 32 * k;
+        srcs[k] = 0u;
+        if (idx < PLANES * SR) {
+          const int plane = PLANES == 1 ? 0 : idx / SR, ri = PLANES == 1 ? idx : idx % SR;
+          bool valid;
+          const bf16* ptr;
+          if constexpr (Cfg::RASTER > 0) ptr = cfg.src_cell(t * TC_BM + ri, valid);
+          else ptr = cfg.src(plane, t * TC_BM + ri, valid);
+          srcs[k] = (uint32_t)(ptr - cfg.base());
+          vmask |= valid ? 1u << k : 0u;
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < NIT; ++k) {
+        const int idx = sub + 32 * k;
+        if (idx < PLANES * SR) {
+          const int plane = PLANES == 1 ? 0 : idx / SR, ri = PLANES == 1 ? idx : idx % SR;
+          cp_async16(stage + plane * PLANE_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), cfg.base() + srcs[k] + c * 8,
+                     (vmask >> k) & 1u ? 16u : 0u);
+        }
       }
       // no waiting here: the hardware arrives on the stage's barrier for this thread when its copies have landed
       cp_async_mbar_arrive(&sh.full[s]);
@@ -716,8 +733,9 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
 
 // conv3 forward: rows = the 9 x 9 x 64 input pixels in memory order; tap (r, s) is 9 r + s rows down
 struct C3FwdCfg {
-  static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152, RASTER = 0;      // RASTER = 0: no cell table
+  static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152, RASTER = 0;      // RASTER = 0: rows are plain memory order
   const bf16* x; int rows;                                   // rows = states * 81
+  __device__ __forceinline__ const bf16* base() const { return x; }
   __device__ __forceinline__ const bf16* src(int, int g, bool& valid) const {
     valid = g < rows;
     return valid ? x + (size_t)g * 64 : x;
@@ -731,6 +749,7 @@ struct C3FwdCfg {
 struct C2FwdCfg {
   static constexpr int PLANES = 2, NT = 8, STAGE_ROWS = 144, RASTER = 0;
   const bf16* x; int states;
+  __device__ __forceinline__ const bf16* base() const { return x; }
   __device__ __forceinline__ const bf16* src(int plane, int g, bool& valid) const {
     // plane row g = (b, oh, X) is pair row 2 g - X + 10 plane of the input in memory order
     valid = g < states * 100;
@@ -744,13 +763,14 @@ struct C2FwdCfg {
 struct C3DgradCfg {
   static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152, RASTER = 121;
   const bf16* g3; int states;
+  __device__ __forceinline__ const bf16* base() const { return g3; }
   // element offset of raster cell `rem` inside a state's 7 x 7 x 64 gradient, or -1 for a padding cell
   __device__ static __forceinline__ int cell(int rem) {
     const int Y = rem / 11, X = rem % 11;
     return (Y >= 2 && Y <= 8 && X >= 2 && X <= 8) ? ((Y - 2) * 7 + (X - 2)) * 64 : -1;
   }
-  __device__ __forceinline__ const bf16* src_cell(int g, const int* table, bool& valid) const {
-    const int b = g / RASTER, off = table[g - b * RASTER];
+  __device__ __forceinline__ const bf16* src_cell(int g, bool& valid) const {
+    const int b = g / RASTER, off = cell(g - b * RASTER);
     valid = b < states && off >= 0;
     return valid ? g3 + (size_t)b * 49 * 64 + off : g3;
   }
@@ -762,12 +782,13 @@ struct C3DgradCfg {
 struct C2DgradCfg {
   static constexpr int PLANES = 1, NT = 4, STAGE_ROWS = 144, RASTER = 121;
   const bf16* g2; int states;
+  __device__ __forceinline__ const bf16* base() const { return g2; }
   __device__ static __forceinline__ int cell(int rem) {
     const int Y = rem / 11, X = rem % 11;
     return (Y >= 1 && Y <= 9 && X >= 1 && X <= 9) ? ((Y - 1) * 9 + (X - 1)) * 64 : -1;
   }
-  __device__ __forceinline__ const bf16* src_cell(int g, const int* table, bool& valid) const {
-    const int b = g / RASTER, off = table[g - b * RASTER];
+  __device__ __forceinline__ const bf16* src_cell(int g, bool& valid) const {
+    const int b = g / RASTER, off = cell(g - b * RASTER);
     valid = b < states && off >= 0;
     return valid ? g2 + (size_t)b * 81 * 64 + off : g2;
   }
@@ -1752,7 +1773,6 @@ tc_shift_wgrad_kernel(Cfg cfg, const bf16* __restrict__ g, int states, float* __
   static_assert(STAGES >= 2 && STAGES <= 8 && SR % 8 == 0 && NP * 64 <= 512, "pipeline shape");
   extern __shared__ uint8_t dyn_smem[];
   __shared__ SwgShared sh;
-  __shared__ int cell_table[Cells::RASTER];
   const uint32_t stage0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int split = blockIdx.x, t0 = split * tiles_per_cta, t1 = min(tiles, t0 + tiles_per_cta);
@@ -1764,7 +1784,6 @@ tc_shift_wgrad_kernel(Cfg cfg, const bf16* __restrict__ g, int states, float* __
     fence_barrier_init();
   }
   if (warp == 8) tmem_alloc(&sh.tmem_base, TMEM_COLS);
-  for (int i = threadIdx.x; i < Cells::RASTER; i += SWG_THREADS) cell_table[i] = Cells::cell(i);
   tcgen05_fence_before();
   __syncthreads();
   tcgen05_fence_after();
@@ -1785,12 +1804,18 @@ tc_shift_wgrad_kernel(Cfg cfg, const bf16* __restrict__ g, int states, float* __
         const bf16* src = cfg.src(plane, t * TC_BM + ri, valid);
         cp_async16(stage + plane * PLANE_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), src + c * 8, valid ? 16u : 0u);
       }
+      // gradient rows (offsets by arithmetic: no shared-memory reads in a warp with copies in flight)
+      int goff[4];
 #pragma unroll
-      for (int ri = sub; ri < TC_BM; ri += 32) {
-        const int pos = t * TC_BM + ri, b = pos / Cells::RASTER, off = cell_table[pos - b * Cells::RASTER];
-        const bool valid = b < states && off >= 0;
-        const bf16* src = valid ? g + (size_t)b * Cells::STATE + off : g;
-        cp_async16(stage + X_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), src + c * 8, valid ? 16u : 0u);
+      for (int k = 0; k < 4; ++k) {
+        const int pos = t * TC_BM + sub + 32 * k, b = pos / Cells::RASTER, cell = Cells::cell(pos - b * Cells::RASTER);
+        goff[k] = (b < states && cell >= 0) ? b * Cells::STATE + cell : -1;                // < 2^31 elements
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int ri = sub + 32 * k;
+        cp_async16(stage + X_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), g + (goff[k] >= 0 ? goff[k] : 0) + c * 8,
+                   goff[k] >= 0 ? 16u : 0u);
       }
       // the hardware arrives on the stage's barrier for this thread once its copies have landed
       cp_async_mbar_arrive(&sh.full[s]);
@@ -1911,183 +1936,285 @@ static void tc_shift_wgrad(LaunchCtx& lc, int kid, Cfg cfg, const bf16* g, int s
   add_segment(segs, bias_part, gb, splits, 1, 64, 1.f);
 }
 
-// ---- first layer, weight gradient: one state at a time ----------------------------------------------------
-// dW1^T[j][co] = sum over (state, oh, ow) of window[j] * G[co].  A CTA walks over its share of the states;
-// each state's raw uint8 frame (28,224 bytes) and its 400 x 32 gradient rows are brought into shared memory
-// once by cp.async (one state ahead), so no byte is fetched twice, and the 400 rows are consumed as five
-// blocks of 80: thread (row, q) expands kernel rows 2q, 2q+1 of its window (64 bytes) to bf16 into atom
-// column q of the MN-major image, and thread t copies 16 bytes of G, adding them to its bias sums on the way.
-constexpr int W1_PRODUCERS = 320, W1_THREADS = 352, W1_ROWS = 80, W1_STAGES = 2;
+// ---- first layer, weight gradient: space-to-depth, all four block taps in one MMA ----------------------------
+// In the block view of the first layer (see the forward kernel) the weight gradient is
+//   dW[tap][e][co] = sum over raster positions m of X[m + shift(tap)][e] * G[m][co],   shift = 0, 1, 21, 22,
+// X[q] = the 64 values of 4 x 4-pixel block q, G = the output gradient on the 21-wide raster (zero in the margin).
+// Both operands are MN-major images whose rows are raster positions.  One M = 128, N = 64 instruction covers all
+// four taps: the two halves of M are the X image entered at rows m + 1 and m + 22 (leading-dimension offset of
+// 21 rows), and the two halves of N are G[m] and G[m + 1] (each gradient row is staged twice, 64 bytes each):
+//   D[a * 64 + e][h * 32 + co] = sum_m X[m + (a ? 22 : 1)][e] * G[m + h][co]  =  tap shift (a ? 22 : 1) - h.
+// The right half sees every gradient row one position early, so tile t stands for positions 128 t - 1 .. 128 t + 126
+// and the tiles of all CTAs together cover -1 .. total: every (tap, position) pair is counted exactly once.
+// Raw frame rows arrive by bulk copy and are expanded to bf16 once per tile, as in the forward kernel.
+// Roles: warps 0-7 expand X (warps 0-3 also write the result at the end), warp 8 issues the MMAs, warp 9 fetches
+// frame rows, warp 10 adds up the bias gradient from the staged gradient rows, warps 11-18 copy the gradient rows.
+// The kernel is bound by how many bytes an SM keeps in flight from DRAM, so the gradient rows and the frame rows
+// have rings of their own that run several tiles ahead of the expansion.
+constexpr int W1_THREADS = 608, W1_STAGES = 3, W1_G_SLOTS = 6, W1_G_AHEAD = 5, W1_X_ROWS = 152, W1_USED = 149,
+              W1_RAW_BYTES = 12288, W1_RAW_SLOTS = 5;
+
+struct W1Shared {
+  uint64_t full[W1_STAGES], empty[W1_STAGES], g_full[W1_G_SLOTS], g_empty[W1_G_SLOTS], raw_full[W1_RAW_SLOTS],
+           raw_empty[W1_RAW_SLOTS], acc;
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
 
 template <class G>
 __global__ void __launch_bounds__(W1_THREADS, 1)
 tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ g, float* __restrict__ partial,
-                      float* __restrict__ bias_partial, int n_states, uint32_t* error_word) {
-  static_assert(G::OH * G::OW == 5 * W1_ROWS && G::CO == 32 && G::K == 8 && G::C == 4 && G::S == 4, "geometry");
-  constexpr uint32_t ATOM_COL = W1_ROWS * 128, A_BYTES = 4 * ATOM_COL, STAGE_BYTES = A_BYTES + ATOM_COL;
-  constexpr uint32_t FRAME_PAD = 28672, GRAW_BYTES = G::OH * G::OW * 64;           // 28,224 rounded up; 25,600
-  constexpr int ROW_BYTES = G::W * G::C;                                          // 336
+                      float* __restrict__ bias_partial, int n_states, int tiles, int tiles_per_cta, uint32_t* error_word) {
+  static_assert(G::OH == 20 && G::OW == 20 && G::CO == 32 && G::K == 8 && G::C == 4 && G::S == 4, "geometry");
+  constexpr int POS = C1_RASTER * C1_RASTER, ROW_BYTES = G::W * G::C, NPROD = 256;
+  constexpr uint32_t X_BYTES = W1_X_ROWS * 128, G_BYTES = TC_BM * 128;
   extern __shared__ uint8_t dyn_smem[];
-  __shared__ TcShared sh;
-  const uint32_t tiles = (smem_u32(dyn_smem) + 1023u) & ~1023u;
-  const uint32_t frame_base = tiles + W1_STAGES * STAGE_BYTES;                     // [2][FRAME_PAD]
-  const uint32_t graw_base = frame_base + 2 * FRAME_PAD;                           // [2][GRAW_BYTES]
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, tid = threadIdx.x;
-  const int per = (n_states + gridDim.x - 1) / gridDim.x;
-  const int s0 = blockIdx.x * per, s1 = min(n_states, s0 + per);
+  __shared__ W1Shared sh;
+  const uint32_t stage0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+  const uint32_t g_base = stage0 + W1_STAGES * X_BYTES;
+  const uint32_t raw_base = g_base + W1_G_SLOTS * G_BYTES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int total_pos = n_states * POS;
+  const int split = blockIdx.x, t0 = split * tiles_per_cta, t1 = min(tiles, t0 + tiles_per_cta);
 
-  if (tid == 0) {
-    for (int s = 0; s < W1_STAGES; ++s) { mbar_init(&sh.full[s], W1_PRODUCERS / 32); mbar_init(&sh.empty[s], 1); }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < W1_STAGES; ++s) { mbar_init(&sh.full[s], NPROD / 32); mbar_init(&sh.empty[s], 1); }
+    for (int i = 0; i < W1_G_SLOTS; ++i) { mbar_init(&sh.g_full[i], 8); mbar_init(&sh.g_empty[i], 2); }
+    for (int i = 0; i < W1_RAW_SLOTS; ++i) { mbar_init(&sh.raw_full[i], 1); mbar_init(&sh.raw_empty[i], NPROD / 32); }
     mbar_init(&sh.acc, 1);
     sh.abort = 0u;
     fence_barrier_init();
   }
-  if (warp == 10) tmem_alloc(&sh.tmem_base, 128);
-  // the G image has 128-byte rows of which only 64 bytes carry data: clear both stages once
-  for (uint32_t i = tid; i < W1_STAGES * ATOM_COL / 16; i += W1_THREADS) {
-    const uint32_t st = i / (ATOM_COL / 16), o = i % (ATOM_COL / 16);
-    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(tiles + st * STAGE_BYTES + A_BYTES + o * 16), "r"(0u) : "memory");
-  }
-  fence_proxy_async_smem();
+  if (warp == 8) tmem_alloc(&sh.tmem_base, 64);
   tcgen05_fence_before();
   __syncthreads();
   tcgen05_fence_after();
   const uint32_t tmem = sh.tmem_base;
-  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
-  float bias[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+  pdl_entry();          // everything above touches only this CTA's own resources
 
-  if (warp < 10) {
+  // frame rows of tile t: blocks at positions qf .. ql, at most nine block rows in at most two states
+  auto tile_ranges = [&](int t, int& b0, int& r0, int& n0, int& n1) {
+    const int qf = min(t * TC_BM, total_pos - 1), ql = min(t * TC_BM + W1_USED - 1, total_pos - 1);
+    b0 = qf / POS;
+    const int b1 = ql / POS, yf = (qf % POS) / C1_RASTER, yl = (ql % POS) / C1_RASTER;
+    r0 = 4 * yf;
+    if (b1 == b0) { n0 = 4 * (yl - yf + 1); n1 = 0; }
+    else { n0 = G::H - r0; n1 = 4 * (yl + 1); }
+  };
+
+  if (warp < 8) {
     // ---------------- producers ----------------
-    auto prefetch = [&](int st, int buf) {
-      const uint8_t* fsrc = frames + (size_t)st * G::IN_SIZE;
-      for (int i = tid; i < G::IN_SIZE / 16; i += W1_PRODUCERS) cp_async16(frame_base + buf * FRAME_PAD + i * 16, fsrc + i * 16, 16u);
-      const bf16* gsrc = g + (size_t)st * G::OH * G::OW * G::CO;
-      for (int i = tid; i < (int)GRAW_BYTES / 16; i += W1_PRODUCERS) cp_async16(graw_base + buf * GRAW_BYTES + i * 16, gsrc + i * 8, 16u);
-      cp_async_commit();
-    };
-    const int row = tid % W1_ROWS, q = tid / W1_ROWS;       // X work item: row of the block, kernel-row pair
-    const int grow = tid >> 2, gc = tid & 3;                 // G work item: row of the block, 16-byte chunk
-    const uint32_t x_off = (uint32_t)q * ATOM_COL + (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u;
-    const uint32_t g_off = A_BYTES + (uint32_t)(grow >> 3) * 1024u + (uint32_t)(grow & 7) * 128u +
-                           ((uint32_t)(gc ^ (grow & 7)) << 4);
-    int it = 0;
-    bool alive = true;
-    if (s0 < s1) prefetch(s0, 0);
-    for (int st = s0; st < s1 && alive; ++st) {
-      const int buf = (st - s0) & 1;
-      cp_async_wait<0>();
-      asm volatile("bar.sync 1, %0;" ::"n"(W1_PRODUCERS) : "memory");   // this state's bytes are in; the other buffer is free
-      if (st + 1 < s1) prefetch(st + 1, buf ^ 1);
-      const uint32_t fb = frame_base + buf * FRAME_PAD, gb = graw_base + buf * GRAW_BYTES;
-      for (int blk = 0; blk < 5; ++blk, ++it) {
-        const int s = it % W1_STAGES;
-        const bool ok = mbar_wait(&sh.empty[s], ((it / W1_STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
-        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
-        const uint32_t stage = tiles + s * STAGE_BYTES;
-        const int ml = blk * W1_ROWS + row, oh = ml / G::OW, ow = ml % G::OW;
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          const uint32_t src = fb + (uint32_t)((oh * G::S + 2 * q + j) * ROW_BYTES + ow * G::S * G::C);
-#pragma unroll
-          for (int h = 0; h < 2; ++h) {
-            uint32_t r0, r1, r2, r3, o[8];
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(src + h * 16) : "memory");
-            u8x4_to_bf16x4(r0, o[0], o[1]); u8x4_to_bf16x4(r1, o[2], o[3]);
-            u8x4_to_bf16x4(r2, o[4], o[5]); u8x4_to_bf16x4(r3, o[6], o[7]);
-            const int c0 = 4 * j + 2 * h;                     // 16 pixels-channels -> two operand chunks
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + x_off + ((uint32_t)(c0 ^ (row & 7)) << 4)),
-                         "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
-            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + x_off + ((uint32_t)((c0 + 1) ^ (row & 7)) << 4)),
-                         "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
-          }
-        }
-        {
-          uint32_t r0, r1, r2, r3;
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                       : "r"(gb + (uint32_t)((blk * W1_ROWS + grow) * 64 + gc * 16)) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + g_off), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
-          const uint32_t w[4] = {r0, r1, r2, r3};
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            bias[2 * i] += __uint_as_float(w[i] << 16);
-            bias[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
-          }
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.full[s]);
+    const int p = threadIdx.x;
+    for (int t = t0; t < t1; ++t) {
+      const int it = t - t0, s = it % W1_STAGES, slot = it % W1_RAW_SLOTS;
+      int b0, r0, n0, n1;
+      tile_ranges(t, b0, r0, n0, n1);
+      bool ok = mbar_wait(&sh.empty[s], ((it / W1_STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const uint32_t stage = stage0 + s * X_BYTES;
+      ok = mbar_wait(&sh.raw_full[slot], (it / W1_RAW_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const uint32_t raw = raw_base + slot * W1_RAW_BYTES;
+      // X rows: work item = (position u of the tile, pixel row py of its block): 16 raw bytes -> two operand chunks;
+      // thread p takes items p, p + 256, p + 512: the same py, positions 64 apart (3 block rows + 1 block)
+      const int py = p & 3, u = p >> 2;
+      int b, Y, X;
+      {
+        const int q = t * TC_BM + u;
+        b = q / POS;
+        const int rem = q - b * POS;
+        Y = rem / C1_RASTER; X = rem - Y * C1_RASTER;
       }
-    }
-    cp_async_wait<0>();
-  } else if (lane == 0) {
-    // ---------------- MMA issuer ----------------
-    constexpr uint32_t idesc = make_idesc_bf16(TC_BM, 64, 1, 1);
-    const int n_it = (s1 > s0 ? s1 - s0 : 0) * 5;
-    bool ok = true;
-    for (int it = 0; it < n_it && ok; ++it) {
-      const int s = it % W1_STAGES;
-      ok = mbar_wait(&sh.full[s], (it / W1_STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
-      if (!ok) break;
-      tcgen05_fence_after();
-      const uint32_t a_base = tiles + s * STAGE_BYTES, b_base = a_base + A_BYTES;
+      uint4 rw[3];
 #pragma unroll
-      for (int jt = 0; jt < 2; ++jt) {
-#pragma unroll
-        for (int t = 0; t < W1_ROWS / 16; ++t)
-          mma_bf16(tmem + jt * 64, make_smem_desc(a_base + jt * 2 * ATOM_COL + t * 2048, ATOM_COL, 1024, SWIZZLE_128B),
-                   make_smem_desc(b_base + t * 2048, ATOM_COL, 1024, SWIZZLE_128B), idesc, (it | t) != 0 ? 1u : 0u);
+      for (int k = 0; k < 3; ++k) {
+        if (b >= n_states) { b = n_states - 1; Y = C1_RASTER - 1; X = C1_RASTER - 1; }     // past the end: repeat the last block
+        const int slot_row = (b == b0 ? 4 * Y - r0 : n0 + 4 * Y) + py;
+        if (u + 64 * k < W1_USED)
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(rw[k].x), "=r"(rw[k].y), "=r"(rw[k].z), "=r"(rw[k].w)
+                       : "r"(raw + (uint32_t)(slot_row * ROW_BYTES + X * 16)) : "memory");
+        X += 1; Y += 3;
+        if (X >= C1_RASTER) { X -= C1_RASTER; ++Y; }
+        if (Y >= C1_RASTER) { Y -= C1_RASTER; ++b; }
       }
-      mma_commit(&sh.empty[s]);
-    }
-    if (ok && n_it > 0) mma_commit(&sh.acc);
-  }
-  __syncthreads();
-  // bias: channel (gc, i) summed over the 80 threads that carried it, in thread order
-  {
-    float* red = reinterpret_cast<float*>(dyn_smem + (frame_base - smem_u32(dyn_smem)));
-    if (warp < 10) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) red[tid * 8 + i] = bias[i];
+      for (int k = 0; k < 3; ++k) {
+        const uint32_t ri = (uint32_t)(u + 64 * k);
+        if (ri < (uint32_t)W1_USED) {
+          uint32_t o[8];
+          u8x4_to_bf16x4(rw[k].x, o[0], o[1]); u8x4_to_bf16x4(rw[k].y, o[2], o[3]);
+          u8x4_to_bf16x4(rw[k].z, o[4], o[5]); u8x4_to_bf16x4(rw[k].w, o[6], o[7]);
+          const uint32_t dst = stage + ri * 128u;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py) ^ (ri & 7)) << 4)),
+                       "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py + 1) ^ (ri & 7)) << 4)),
+                       "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+        }
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&sh.full[s]); mbar_arrive(&sh.raw_empty[slot]); }
     }
-    __syncthreads();
-    if (tid < 32) {
-      const int gcc = tid >> 3, i = tid & 7;
-      float sum = 0.f;
-      for (int r = 0; r < W1_ROWS; ++r) sum += red[(r * 4 + gcc) * 8 + i];
-      bias_partial[(size_t)blockIdx.x * 32 + tid] = s1 > s0 ? sum : 0.f;
-    }
-  }
-  if (warp < 4) {
-    if (s1 > s0 && mbar_wait(&sh.acc, 0, &sh.abort, error_word, ERR_WAIT_ACC)) {
+    // ---------------- epilogue: float partial tile to scratch, rows regrouped to the canonical weight order ----------------
+    if (warp < 4 && t1 > t0 && mbar_wait(&sh.acc, 0, &sh.abort, error_word, ERR_WAIT_ACC)) {
       tcgen05_fence_after();
+      const int row = threadIdx.x, a = row >> 6, e = row & 63, py = e >> 4, px = (e >> 2) & 3, ci = e & 3;
 #pragma unroll 1
-      for (int jt = 0; jt < 2; ++jt) {
+      for (int h = 0; h < 2; ++h) {
         uint32_t r[32];
-        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + jt * 64, r);
-        float4* dst = reinterpret_cast<float4*>(partial + ((size_t)blockIdx.x * 256 + jt * 128 + tid) * 32);
+        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + h * 32, r);
+        const int i = a, jj = 1 - h;                                    // block tap (i, jj): shift 21 i + jj
+        const int jcan = ((4 * i + py) * 8 + 4 * jj + px) * 4 + ci;    // (r, s, ci) of the 8 x 8 x 4 filter
+        float4* dst = reinterpret_cast<float4*>(partial + ((size_t)split * 256 + jcan) * 32);
 #pragma unroll
         for (int v = 0; v < 8; ++v)
           dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
                                __uint_as_float(r[4 * v + 3]));
       }
-    } else if (s1 <= s0) {
-      for (int jt = 0; jt < 2; ++jt)
-        for (int v = 0; v < 32; ++v) partial[((size_t)blockIdx.x * 256 + jt * 128 + tid) * 32 + v] = 0.f;
+    }
+  } else if (warp == 8) {
+    if (lane == 0) {
+      // ---------------- MMA issuer ----------------
+      constexpr uint32_t idesc = make_idesc_bf16(TC_BM, 64, 1, 1);
+      const uint32_t hi = desc_hi_kmajor_sw128();
+      constexpr uint32_t LBO = 21u * 128u;                 // second half of M: the X image 21 rows further down
+      bool ok = true;
+      for (int t = t0; t < t1 && ok; ++t) {
+        const int it = t - t0, s = it % W1_STAGES, gs = it % W1_G_SLOTS;
+        ok = mbar_wait(&sh.g_full[gs], (it / W1_G_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+        if (!ok) break;
+        ok = mbar_wait(&sh.full[s], (it / W1_STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+        if (!ok) break;
+        fence_proxy_async_smem();        // the copies observed through the barrier -> visible to the MMA's operand reads
+        tcgen05_fence_after();
+        const uint32_t a_lo0 = (((stage0 + s * X_BYTES) >> 4) & 0x3FFFu) | ((LBO >> 4) << 16);
+        const uint32_t b_lo0 = ((g_base + gs * G_BYTES) >> 4) & 0x3FFFu;
+#pragma unroll
+        for (int k = 0; k < TC_BM / 16; ++k)
+          mma_bf16_lo_rt(tmem, a_lo0 + k * (2048u >> 4), b_lo0 + k * (2048u >> 4), hi, idesc, (it | k) != 0 ? 1u : 0u);
+        mma_commit(&sh.empty[s]);
+        mma_commit(&sh.g_empty[gs]);
+      }
+      if (ok && t1 > t0) mma_commit(&sh.acc);
+    }
+  } else if (warp == 9) {
+    if (lane == 0) {
+      // ---------------- raw loader ----------------
+      for (int t = t0; t < t1; ++t) {
+        const int it = t - t0, slot = it % W1_RAW_SLOTS;
+        if (!mbar_wait(&sh.raw_empty[slot], ((it / W1_RAW_SLOTS) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY)) break;
+        int b0, r0, n0, n1;
+        tile_ranges(t, b0, r0, n0, n1);
+        const uint32_t dst = raw_base + slot * W1_RAW_BYTES;
+        mbar_arrive_expect_tx(&sh.raw_full[slot], (uint32_t)((n0 + n1) * ROW_BYTES));
+        bulk_copy_g2s(dst, frames + ((size_t)b0 * G::H + r0) * ROW_BYTES, (uint32_t)(n0 * ROW_BYTES), &sh.raw_full[slot]);
+        if (n1 > 0)
+          bulk_copy_g2s(dst + n0 * ROW_BYTES, frames + (size_t)(b0 + 1) * G::H * ROW_BYTES, (uint32_t)(n1 * ROW_BYTES),
+                        &sh.raw_full[slot]);
+      }
+    }
+  } else if (warp >= 11) {
+    // ---------------- gradient rows: image row r = [G[m] | G[m + 1]], m = 128 t - 1 + r ----------------
+    // thread p copies chunk p & 7 of rows (p >> 3) + 32 k, W1_G_AHEAD tiles ahead of the tile it publishes
+    const int p = threadIdx.x - 352, c8 = p & 7, half = c8 >> 2, chunk = c8 & 3;
+    int b1, Y, X;
+    {
+      const int mm = t0 * TC_BM - 1 + (p >> 3) + half + POS;       // one state further, so that position -1 is not negative
+      b1 = mm / POS;
+      const int rem = mm - b1 * POS;
+      Y = rem / C1_RASTER; X = rem - Y * C1_RASTER;
+    }
+    bool alive = true;
+    for (int t = t0; t < t1 + W1_G_AHEAD && alive; ++t) {
+      // publish first, fetch second: the slot a fetch waits for must not be the one whose consumers are waiting
+      // for this very publication
+      if (t - W1_G_AHEAD >= t0) {
+        cp_async_wait<W1_G_AHEAD - 1>();           // the rows of tile t - W1_G_AHEAD (my share) have landed
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.g_full[(t - W1_G_AHEAD - t0) % W1_G_SLOTS]);
+      }
+      if (t < t1) {
+        const int it = t - t0, gs = it % W1_G_SLOTS;
+        const bool ok = mbar_wait(&sh.g_empty[gs], ((it / W1_G_SLOTS) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+        const uint32_t dst = g_base + gs * G_BYTES;
+        // Source offsets: the raster cell (state + 1, Y, X) of this thread's first row is carried from tile to tile
+        // and stepped by 32 positions from row to row; these few warps have no one to hide a division's latency.
+        int off[4];
+        {
+          int bb = b1, yy = Y, xx = X;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const bool valid = bb >= 1 && bb <= n_states && yy < G::OH && xx < G::OW;
+            off[k] = valid ? ((bb - 1) * (G::OH * G::OW) + yy * G::OW + xx) * G::CO + chunk * 8 : -1;     // < 2^31 elements
+            xx += 32 - C1_RASTER; ++yy;                       // 32 positions on
+            if (xx >= C1_RASTER) { xx -= C1_RASTER; ++yy; }
+            if (yy >= C1_RASTER) { yy -= C1_RASTER; ++bb; }
+          }
+          X += TC_BM - 6 * C1_RASTER; Y += 6;                 // the next tile is 128 = 6 * 21 + 2 positions on
+          if (X >= C1_RASTER) { X -= C1_RASTER; ++Y; }
+          if (Y >= C1_RASTER) { Y -= C1_RASTER; ++b1; }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int r = (p >> 3) + 32 * k;
+          cp_async16(dst + r * 128u + ((uint32_t)(c8 ^ (r & 7)) << 4), g + (off[k] >= 0 ? off[k] : 0), off[k] >= 0 ? 16u : 0u);
+        }
+      }
+      cp_async_commit();                           // one group per iteration, also when there is nothing left to fetch
+    }
+    cp_async_wait<0>();
+  } else {
+    // ---------------- bias gradient: the left halves of the staged gradient rows hold every position once ----------------
+    // lane l adds channels 8 (l & 3) .. 8 (l & 3) + 7 (one 16-byte chunk) over the rows (l >> 2) + 8 i
+    float acc[8] = {};
+    bool ok = true;
+    const int q = lane & 3, rr = lane >> 2;
+    for (int t = t0; t < t1 && ok; ++t) {
+      const int it = t - t0, gs = it % W1_G_SLOTS;
+      ok = mbar_wait(&sh.g_full[gs], (it / W1_G_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      const uint32_t gaddr = g_base + gs * G_BYTES + (uint32_t)rr * 128u + ((uint32_t)(q ^ rr) << 4);
+#pragma unroll 4
+      for (int i = 0; i < TC_BM / 8; ++i) {
+        uint32_t v[4];
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
+                     : "r"(gaddr + (uint32_t)i * 1024u) : "memory");
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          acc[2 * j] += __uint_as_float(v[j] << 16);
+          acc[2 * j + 1] += __uint_as_float(v[j] & 0xFFFF0000u);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh.g_empty[gs]);
+    }
+    // the eight row groups, added in a fixed order
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], 4);
+      acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], 8);
+      acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], 16);
+    }
+    if (ok && t1 > t0 && lane < 4) {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) bias_partial[(size_t)split * 32 + 8 * q + j] = acc[j];
     }
   }
   tcgen05_fence_before();
   __syncthreads();
-  if (warp == 10) {
+  if (warp == 8) {
     __syncwarp();
     tcgen05_fence_after();
-    tmem_dealloc(tmem, 128);
+    tmem_dealloc(tmem, 64);
   }
 }
 
 template <class G>
 static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, int n_states, float* gw, float* gb,
                            float* scratch, GradSegments* segs, uint32_t* err) {
-  constexpr int smem = W1_STAGES * 5 * W1_ROWS * 128 + 2 * 28672 + 2 * 25600 + 1024;
+  constexpr int smem = (W1_STAGES * W1_X_ROWS + W1_G_SLOTS * TC_BM) * 128 + W1_RAW_SLOTS * W1_RAW_BYTES + 1024;
   static_assert(smem <= 227 * 1024, "shared memory budget");
   auto kern = tc_conv1_wgrad_kernel<G>;
   static bool configured = false;
@@ -2095,10 +2222,13 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     configured = true;
   }
-  const int splits = n_states < sm_count() ? n_states : sm_count();
+  const int tiles = (n_states * C1_RASTER * C1_RASTER + 1 + TC_BM - 1) / TC_BM;      // positions -1 .. total - 1
+  int ctas = sm_count() < SWG_MAX_SPLITS ? sm_count() : SWG_MAX_SPLITS;
+  if (ctas > tiles) ctas = tiles;
+  const int per = (tiles + ctas - 1) / ctas, splits = (tiles + per - 1) / per;
   float* bias_part = scratch + (size_t)splits * 256 * 32;
   KernelScope scope(lc, KID_CONV1_WGRAD);
-  launch_kernel_overlapped(lc, kern, splits, W1_THREADS, smem, frames, g, scratch, bias_part, n_states, err);
+  launch_kernel_overlapped(lc, kern, splits, W1_THREADS, smem, frames, g, scratch, bias_part, n_states, tiles, per, err);
   add_segment(segs, scratch, gw, splits, 256, 32, 1.0f / 255.0f);
   add_segment(segs, bias_part, gb, splits, 1, 32, 1.f);
 }
