@@ -1948,10 +1948,11 @@ static void tc_shift_wgrad(LaunchCtx& lc, int kid, Cfg cfg, const bf16* g, int s
 // and the tiles of all CTAs together cover -1 .. total: every (tap, position) pair is counted exactly once.
 // Raw frame rows arrive by bulk copy and are expanded to bf16 once per tile, as in the forward kernel.
 // Roles: warps 0-7 expand X (warps 0-3 also write the result at the end), warp 8 issues the MMAs, warp 9 fetches
-// frame rows, warp 10 adds up the bias gradient from the staged gradient rows, warps 11-18 copy the gradient rows.
+// frame rows, warps 10 and 19 add up the bias gradient from the staged gradient rows (half of the rows each), warps
+// 11-18 copy the gradient rows.
 // The kernel is bound by how many bytes an SM keeps in flight from DRAM, so the gradient rows and the frame rows
 // have rings of their own that run several tiles ahead of the expansion.
-constexpr int W1_THREADS = 608, W1_STAGES = 3, W1_G_SLOTS = 6, W1_G_AHEAD = 5, W1_X_ROWS = 152, W1_USED = 149,
+constexpr int W1_THREADS = 640, W1_STAGES = 3, W1_G_SLOTS = 6, W1_G_AHEAD = 5, W1_X_ROWS = 152, W1_USED = 149,
               W1_RAW_BYTES = 12288, W1_RAW_SLOTS = 5;
 
 struct W1Shared {
@@ -1979,7 +1980,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < W1_STAGES; ++s) { mbar_init(&sh.full[s], NPROD / 32); mbar_init(&sh.empty[s], 1); }
-    for (int i = 0; i < W1_G_SLOTS; ++i) { mbar_init(&sh.g_full[i], 8); mbar_init(&sh.g_empty[i], 2); }
+    for (int i = 0; i < W1_G_SLOTS; ++i) { mbar_init(&sh.g_full[i], 8); mbar_init(&sh.g_empty[i], 3); }
     for (int i = 0; i < W1_RAW_SLOTS; ++i) { mbar_init(&sh.raw_full[i], 1); mbar_init(&sh.raw_empty[i], NPROD / 32); }
     mbar_init(&sh.acc, 1);
     sh.abort = 0u;
@@ -2113,7 +2114,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
                         &sh.raw_full[slot]);
       }
     }
-  } else if (warp >= 11) {
+  } else if (warp >= 11 && warp < 19) {
     // ---------------- gradient rows: image row r = [G[m] | G[m + 1]], m = 128 t - 1 + r ----------------
     // thread p copies chunk p & 7 of rows (p >> 3) + 32 k, W1_G_AHEAD tiles ahead of the tile it publishes
     const int p = threadIdx.x - 352, c8 = p & 7, half = c8 >> 2, chunk = c8 & 3;
@@ -2167,24 +2168,26 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
     cp_async_wait<0>();
   } else {
     // ---------------- bias gradient: the left halves of the staged gradient rows hold every position once ----------------
-    // lane l adds channels 8 (l & 3) .. 8 (l & 3) + 7 (one 16-byte chunk) over the rows (l >> 2) + 8 i
+    // lane l adds channels 8 (l & 3) .. 8 (l & 3) + 7 (one 16-byte chunk) over the rows (l >> 2) + 8 i, i of this warp's parity
     float acc[8] = {};
     bool ok = true;
-    const int q = lane & 3, rr = lane >> 2;
+    const int q = lane & 3, rr = lane >> 2, which = warp == 10 ? 0 : 1;
     for (int t = t0; t < t1 && ok; ++t) {
       const int it = t - t0, gs = it % W1_G_SLOTS;
       ok = mbar_wait(&sh.g_full[gs], (it / W1_G_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-      const uint32_t gaddr = g_base + gs * G_BYTES + (uint32_t)rr * 128u + ((uint32_t)(q ^ rr) << 4);
-#pragma unroll 4
-      for (int i = 0; i < TC_BM / 8; ++i) {
-        uint32_t v[4];
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
-                     : "r"(gaddr + (uint32_t)i * 1024u) : "memory");
+      const uint32_t gaddr = g_base + gs * G_BYTES + (uint32_t)(rr + 8 * which) * 128u + ((uint32_t)(q ^ rr) << 4);
+      uint32_t v[TC_BM / 16][4];
+#pragma unroll
+      for (int i = 0; i < TC_BM / 16; ++i)
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[i][0]), "=r"(v[i][1]), "=r"(v[i][2]), "=r"(v[i][3])
+                     : "r"(gaddr + (uint32_t)i * 2048u) : "memory");
+#pragma unroll
+      for (int i = 0; i < TC_BM / 16; ++i) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          acc[2 * j] += __uint_as_float(v[j] << 16);
-          acc[2 * j + 1] += __uint_as_float(v[j] & 0xFFFF0000u);
+          acc[2 * j] += __uint_as_float(v[i][j] << 16);
+          acc[2 * j + 1] += __uint_as_float(v[i][j] & 0xFFFF0000u);
         }
       }
       __syncwarp();
@@ -2199,7 +2202,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
     }
     if (ok && t1 > t0 && lane < 4) {
 #pragma unroll
-      for (int j = 0; j < 8; ++j) bias_partial[(size_t)split * 32 + 8 * q + j] = acc[j];
+      for (int j = 0; j < 8; ++j) bias_partial[((size_t)split * 2 + which) * 32 + 8 * q + j] = acc[j];
     }
   }
   tcgen05_fence_before();
@@ -2230,7 +2233,7 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
   KernelScope scope(lc, KID_CONV1_WGRAD);
   launch_kernel_overlapped(lc, kern, splits, W1_THREADS, smem, frames, g, scratch, bias_part, n_states, tiles, per, err);
   add_segment(segs, scratch, gw, splits, 256, 32, 1.0f / 255.0f);
-  add_segment(segs, bias_part, gb, splits, 1, 32, 1.f);
+  add_segment(segs, bias_part, gb, 2 * splits, 1, 32, 1.f);      // two bias warps per CTA, a row each
 }
 
 // every layer keeps its own partial-sum region until the finishing kernel has run
