@@ -141,16 +141,28 @@ void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample) {
   void* act[MAX_LAYERS];
   for (int l = 0; l <= c->nd.n_conv; ++l)
     act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
+  const size_t row = (size_t)slot * c->n_e;
+  const int32_t* forced = sample && c->forced_on ? c->forced + row : nullptr;
+  int32_t* actions = sample ? c->actions + row : nullptr;
+  int32_t* sampled = sample ? c->sampled + row : nullptr;
+  float* uniforms = sample ? c->uniforms + row : nullptr;
+  if (use_tc(c) && heads_fused_supported(c->nd)) {
+    int splits = 0;
+    tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, c->w_images, frames, c->n_e, act, c->scratch,
+               &c->stats->error_word, &splits);
+    launch_heads_fused(c->lc, c->nd, c->theta, c->theta16, c->scratch, splits, (bf16*)act[c->nd.n_conv], c->n_e,
+                       c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot, forced, actions,
+                       sampled, uniforms);
+    return;
+  }
   if (use_tc(c))
     tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, c->w_images, frames, c->n_e, act, c->scratch,
                &c->stats->error_word);
   else
     simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
-  const size_t row = (size_t)slot * c->n_e;
   launch_heads(c->lc, c->prec, c->nd, c->theta, c->theta16, act[c->nd.n_conv], c->n_e,
-               c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot,
-               sample && c->forced_on ? c->forced + row : nullptr, sample ? c->actions + row : nullptr,
-               sample ? c->sampled + row : nullptr, sample ? c->uniforms + row : nullptr);
+               c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot, forced, actions, sampled,
+               uniforms);
 }
 
 void drop_graphs(paac_ctx* c) {

@@ -89,6 +89,146 @@ heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* _
   }
 }
 
+// The same, fused with the end of the fully connected layer of the tensor-core path: the warp first finishes
+// its state's 512 hidden units from the split-k partial sums, h = bf16(relu(sum_s part[s][e][:] + bias)), the
+// splits added in order, stores them for the backward pass and goes on with the rounded values.  The A dot
+// products are reduced together: every lane keeps one partial sum per action, and a butterfly that halves the
+// number of live values at each step leaves lane k with logit k after 31 shuffles instead of 5 per action; the
+// additions pair up exactly as in warp_sum, so the logits are bit-identical to the unfused kernel's.
+// The head weights (A + 1 rows of 512) are brought into shared memory once per block, before the wait on the
+// previous kernel: they are older than that kernel.  Row k is stored as two halves, [lane][first 8 of the lane's
+// 16 elements] then [lane][last 8], so that a warp's 16-byte reads are contiguous.
+constexpr int HF_WARPS = 8;
+__global__ void __launch_bounds__(HF_WARPS * 32)
+heads_fused_kernel(const float* __restrict__ part, int splits, const float* __restrict__ fc_bias, bf16* __restrict__ h_out,
+                   const bf16* __restrict__ wpi, const float* __restrict__ bpi, const bf16* __restrict__ wv,
+                   const float* __restrict__ bv, int n, int A, float* __restrict__ logits, float* __restrict__ values,
+                   uint64_t seed, const uint64_t* __restrict__ step_base, uint32_t t, const int32_t* __restrict__ forced,
+                   int32_t* __restrict__ actions, int32_t* __restrict__ sampled, float* __restrict__ uniforms) {
+  constexpr int EPL = 16, F = 32 * EPL;
+  __shared__ uint4 wsh[33 * 64];                     // row k: 64 chunks of 8 bf16; row A = value head
+  const int lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < (A + 1) * 64; i += HF_WARPS * 32) {
+    const int k = i >> 6, c = i & 63, l = c >> 1, half = c & 1;          // chunk c of the row = lane l, half
+    uint4 v;
+    if (k < A) v = __ldg(reinterpret_cast<const uint4*>(wpi + (size_t)k * F) + c);
+    else {                                            // the value row is not 16-byte aligned
+      uint32_t w4[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        w4[j] = (uint32_t)__bfloat16_as_ushort(wv[c * 8 + 2 * j]) | ((uint32_t)__bfloat16_as_ushort(wv[c * 8 + 2 * j + 1]) << 16);
+      v = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+    }
+    wsh[k * 64 + half * 32 + l] = v;
+  }
+  __syncthreads();
+  pdl_entry();          // the head weights above were written several kernels ago
+  const int e = blockIdx.x * HF_WARPS + (threadIdx.x >> 5);
+  if (e >= n) return;
+  float x[EPL];
+  {
+    float v[EPL];
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) v[i] = 0.f;
+    const float* p0 = part + (size_t)e * F + lane * EPL;
+#pragma unroll 7
+    for (int s = 0; s < splits; ++s) {
+      const float4* q = reinterpret_cast<const float4*>(p0 + (size_t)s * n * F);
+#pragma unroll
+      for (int i = 0; i < EPL / 4; ++i) {
+        const float4 a = __ldg(q + i);
+        v[4 * i] += a.x; v[4 * i + 1] += a.y; v[4 * i + 2] += a.z; v[4 * i + 3] += a.w;
+      }
+    }
+    uint32_t o[EPL / 2];
+#pragma unroll
+    for (int i = 0; i < EPL / 2; ++i) {
+      const bf16 lo = __float2bfloat16_rn(fmaxf(v[2 * i] + __ldg(fc_bias + lane * EPL + 2 * i), 0.f));
+      const bf16 hi = __float2bfloat16_rn(fmaxf(v[2 * i + 1] + __ldg(fc_bias + lane * EPL + 2 * i + 1), 0.f));
+      x[2 * i] = __bfloat162float(lo); x[2 * i + 1] = __bfloat162float(hi);
+      o[i] = (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
+    }
+    uint4* dst = reinterpret_cast<uint4*>(h_out + (size_t)e * F + lane * EPL);
+    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+  }
+  float pr[32];
+#pragma unroll
+  for (int k = 0; k < 32; ++k) {
+    pr[k] = 0.f;
+    if (k < A) {
+      const uint4 lo = wsh[k * 64 + lane], hi = wsh[k * 64 + 32 + lane];
+      const uint32_t w8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+      float acc = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        acc = fmaf(__uint_as_float(w8[i] << 16), x[2 * i], acc);
+        acc = fmaf(__uint_as_float(w8[i] & 0xFFFF0000u), x[2 * i + 1], acc);
+      }
+      pr[k] = acc;
+    }
+  }
+  // reduce-scatter: at the step with offset o a lane keeps the half of its values whose index has bit o equal to
+  // its own lane bit and adds the partner's copy of them
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const bool up = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < o; ++i) {
+      const float send = up ? pr[i] : pr[i + o];
+      const float keep = up ? pr[i + o] : pr[i];
+      pr[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+    }
+  }
+  const float z = lane < A ? pr[0] + bpi[lane < A ? lane : 0] : -INFINITY;
+  float v = 0.f;
+  {
+    const uint4 lo = wsh[A * 64 + lane], hi = wsh[A * 64 + 32 + lane];
+    const uint32_t w8[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      v = fmaf(__uint_as_float(w8[i] << 16), x[2 * i], v);
+      v = fmaf(__uint_as_float(w8[i] & 0xFFFF0000u), x[2 * i + 1], v);
+    }
+  }
+  v = warp_sum(v) + bv[0];
+  if (lane < A) logits[(size_t)e * A + lane] = z;
+  if (lane == 0) values[e] = v;
+  if (actions == nullptr) return;
+
+  const float m = warp_max(z);
+  const float ex = lane < A ? expf(z - m) : 0.f;
+  const float lse = m + logf(warp_sum(ex));
+  const float p = lane < A ? expf(z - lse) : 0.f;
+  const uint64_t step = *step_base + t;
+  const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
+  float c = 0.f;
+  int a = A - 1;
+  bool found = false;
+  for (int k = 0; k < A; ++k) {
+    c += __shfl_sync(0xffffffffu, p, k);
+    if (!found && u < c) { a = k; found = true; }
+  }
+  if (lane == 0) {
+    sampled[e] = a;
+    if (forced != nullptr && forced[e] >= 0) a = forced[e];
+    actions[e] = a;
+    uniforms[e] = u;
+  }
+}
+
+bool heads_fused_supported(const NetDims& nd) { return nd.F == 512 && nd.pi_w % 8 == 0 && nd.A <= 32; }
+
+void launch_heads_fused(LaunchCtx& lc, const NetDims& nd, const float* theta, const bf16* theta16, const float* part,
+                        int splits, bf16* h_out, int n, float* logits, float* values, uint64_t seed,
+                        const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
+                        float* uniforms) {
+  KernelScope scope(lc, KID_HEADS_FWD);
+  launch_kernel(lc, heads_fused_kernel, (n + HF_WARPS - 1) / HF_WARPS, HF_WARPS * 32, 0, part, splits, theta + nd.layer[nd.n_conv].b_off, h_out,
+                theta16 + nd.pi_w, theta + nd.pi_b, theta16 + nd.v_w, theta + nd.v_b, n, nd.A, logits, values, seed,
+                step_base, t, forced, actions, sampled, uniforms);
+}
+
 // Element-wise variant of the heads kernel for layouts without 16-byte alignment and for float storage.
 // One warp per state.  Lane k ends up holding logit k (A <= 32).  If `actions` is given,
 // the warp also draws a_t: u from Philox counter (env, step_lo, step_hi, ACTION stream), then the

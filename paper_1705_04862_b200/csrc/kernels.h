@@ -30,8 +30,11 @@ size_t simt_scratch_floats(int arch, const NetDims& nd, int n);
 bool tc_supported(int arch, int prec);
 // fc_scratch: tc_fc_scratch_floats(n) floats for the split-k partial sums of the fully connected layer
 size_t tc_fc_scratch_floats(int n);
+// with fc_splits != nullptr the fully connected layer is left as *fc_splits split-k partial sums in fc_scratch
+// (part[split][n][512]) for launch_heads_fused to finish
 void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* theta16, const bf16* images,
-                const uint8_t* frames, int n, void* const act[], float* fc_scratch, uint32_t* error_word);
+                const uint8_t* frames, int n, void* const act[], float* fc_scratch, uint32_t* error_word,
+                int* fc_splits = nullptr);
 // transposed / regrouped bf16 weight images the backward contractions read (refreshed after every
 // parameter change), and the data-gradient kernels that use them
 size_t tc_weight_image_elems();
@@ -60,6 +63,13 @@ void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta
                   const bf16* theta16, const void* h, int n, float* logits, float* values, uint64_t seed,
                   const uint64_t* step_base /* device */, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled /* action before forcing */,
                   float* uniforms);
+// the same for the tensor-core path, which leaves the fully connected layer as split-k partial sums
+// part[split][n][F]: finishes h (sum, bias, ReLU, bf16) into h_out on the way
+bool heads_fused_supported(const NetDims& nd);
+void launch_heads_fused(LaunchCtx& lc, const NetDims& nd, const float* theta, const bf16* theta16, const float* part,
+                        int splits, bf16* h_out, int n, float* logits, float* values, uint64_t seed,
+                        const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
+                        float* uniforms);
 void launch_returns(LaunchCtx& lc, int n_e, int t_max, float gamma, const int8_t* rewards,
                     const uint8_t* terminals, const float* values, float* R, float* adv);
 void launch_head_grad(LaunchCtx& lc, int B, int A, float beta, float value_coef,

@@ -1301,7 +1301,7 @@ constexpr int FC_SPLITS = 7;
 size_t tc_fc_scratch_floats(int n) { return (size_t)FC_SPLITS * n * 512; }
 
 static void tc_fc_forward(LaunchCtx& lc, const bf16* a, const bf16* w, const float* bias, bf16* out, int M, int N, int K,
-                          float* part, uint32_t* err) {
+                          float* part, uint32_t* err, int* splits_out) {
   constexpr int smem = SK_STAGES * (TC_BM * 128 + SK_BN * 128) + 1024;
   static bool configured = false;
   if (!configured) {
@@ -1316,6 +1316,7 @@ static void tc_fc_forward(LaunchCtx& lc, const bf16* a, const bf16* w, const flo
     launch_kernel_overlapped(lc, tc_splitk_kernel, total < sm_count() ? total : sm_count(), PK_THREADS, smem, a, w, part, M, N, K, tiles_m,
                                                                                          tiles_n, splits, kb_per, err);
   }
+  if (splits_out) { *splits_out = splits; return; }      // the caller's next kernel adds the partial sums up
   KernelScope scope(lc, KID_FC_FWD);
   const int blocks = (M * N / 8 + 255) / 256;
   launch_kernel(lc, fc_finish_kernel, blocks < 1184 ? blocks : 1184, 256, 0, part, splits, M, N, bias, out);
@@ -1325,7 +1326,7 @@ static void tc_fc_forward(LaunchCtx& lc, const bf16* a, const bf16* w, const flo
 bool tc_supported(int arch, int prec) { return arch == PAAC_ARCH_NATURE && prec == PAAC_BF16; }
 
 void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* w, const bf16* images,
-                const uint8_t* frames, int n, void* const act[], float* fc_scratch, uint32_t* err) {
+                const uint8_t* frames, int n, void* const act[], float* fc_scratch, uint32_t* err, int* fc_splits) {
   const LayerDims* d = nd.layer;
   const float s255 = 1.0f / 255.0f;
   if (arch != PAAC_ARCH_NATURE) return;   // the caller routes the smaller network to the CUDA-core path
@@ -1347,7 +1348,8 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
           ShiftBiasReluEpi<Map, 7, 7>{Map{n}, (bf16*)act[2], theta + d[2].b_off, nullptr}, n * 81, err);
     }
     (void)M2; (void)M3;
-    tc_fc_forward(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, (bf16*)act[3], n, 512, 3136, fc_scratch, err);
+    tc_fc_forward(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, (bf16*)act[3], n, 512, 3136, fc_scratch, err,
+                  fc_splits);
   }
 }
 
