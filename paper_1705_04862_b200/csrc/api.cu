@@ -302,8 +302,12 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
     launch_head_grad(c->lc, c->B, c->A, hp.entropy_beta, hp.value_coef, c->logits, c->values, c->actions,
                      c->R, c->adv, c->dz, c->dV, c->loss_terms, c->stats);
     const int L = c->nd.n_conv;
-    heads_backward(c->lc, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
-                   c->grad, c->scratch);
+    if (use_tc(c) && tc_heads_backward_supported(c->nd))
+      tc_heads_backward(c->lc, c->nd, c->theta16, (const bf16*)c->act[L], c->B, c->dz, c->dV, (bf16*)c->gact[L], c->grad,
+                        c->scratch, &c->grad_segs);
+    else
+      heads_backward(c->lc, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
+                     c->grad, c->scratch);
     uint32_t* err = &c->stats->error_word;
     for (int l = L; l >= 0; --l) {
       // tensor-core kernels where they exist, the CUDA-core contraction otherwise

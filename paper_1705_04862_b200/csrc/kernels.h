@@ -46,11 +46,16 @@ void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* con
 // scratch of tc_scratch_floats(B) floats; the regions are noted in a GradSegments list, and
 // tc_backward_finish() adds them up into the gradient vector with one launch and empties the list
 struct GradSegment { const float* part; float* dst; int splits, J, CO; float scale; int first_group, groups, wide; };
-struct GradSegments { GradSegment seg[8]; int n; int total_groups; };
+struct GradSegments { GradSegment seg[12]; int n; int total_groups; };
 size_t tc_scratch_floats(int n);
 void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, int n, void* const act[],
                        void* const gact[], float* grad, float* scratch, int layer, GradSegments* segs, uint32_t* err);
 void tc_backward_finish(LaunchCtx& lc, GradSegments* segs);
+// both heads in one kernel: gradient at the fc pre-activation into g_fc, the heads' parameter gradients as one more
+// set of partial sums for tc_backward_finish()
+bool tc_heads_backward_supported(const NetDims& nd);
+void tc_heads_backward(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, const bf16* h, int n, const float* dz,
+                       const float* dV, bf16* g_fc, float* grad, float* scratch, GradSegments* segs);
 // single layers of the CUDA-core backward pass (the tensor-core update mixes them in where it has no
 // kernel of its own yet)
 void simt_backward_layer(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta, const bf16* theta16,

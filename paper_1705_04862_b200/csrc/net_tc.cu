@@ -2253,7 +2253,8 @@ static size_t tc_layer_scratch_offset(int n, int layer) {
   return off;
 }
 
-size_t tc_scratch_floats(int n) { return tc_layer_scratch_offset(n, 4); }
+static size_t tc_heads_scratch_floats();
+size_t tc_scratch_floats(int n) { return tc_layer_scratch_offset(n, 4) + tc_heads_scratch_floats(); }
 
 // Enqueues the weight-gradient kernel of `layer` (0 = conv1 .. 3 = fc) and notes in *segs where its partial
 // sums are; tc_backward_finish() then turns all noted partial sums into the gradient vector in one launch.
@@ -2286,6 +2287,109 @@ void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, 
     tc_wgrad<PlainSrc, GradSrc<64>, 1, 128, 6, 512>(lc, KID_FC_WGRAD, PlainSrc{(const bf16*)act[2], 3136, n},
                                                     GradSrc<64>{g, 512, n}, n, 49, 1.f, gw, gb, sc, &segs, err);
   }
+}
+
+// ---- backward through the two heads, one kernel ---------------------------------------------------------------
+// With dz[b][k] the loss gradient at the logits and dV[b] at the value (row k = A of a combined matrix):
+//   g_fc[b][i] = (h[b][i] > 0) * sum_k dz[b][k] W[k][i],      dW[k][i] = sum_b dz[b][k] h[b][i],     db[k] = sum_b dz[b][k].
+// A thread owns two of the 512 hidden units: their weight columns live in registers, every row costs it one 4-byte
+// load of h and NK multiply-adds each way, and the row's dz values are broadcast from shared memory.  A CTA walks a
+// contiguous range of rows and leaves its dW / db sums as one more split for the finishing kernel.
+constexpr int HB_THREADS = 256, HB_ROWS = 32;
+
+template <int NK>
+__global__ void __launch_bounds__(HB_THREADS, 2)
+heads_backward_kernel(const bf16* __restrict__ h, const float* __restrict__ dz, const float* __restrict__ dV,
+                      const bf16* __restrict__ wpi, const bf16* __restrict__ wv, int n, int A, int rows_per,
+                      bf16* __restrict__ g_fc, float* __restrict__ part_w, float* __restrict__ part_b,
+                      float* __restrict__ part_vw, float* __restrict__ part_vb) {
+  constexpr int F = 512;
+  static_assert(NK % 4 == 0, "rows of dz are read as float4");
+  __shared__ __align__(16) float dzs[HB_ROWS][NK];
+  const int tid = threadIdx.x, col = 2 * tid;
+  float w[NK][2], acc[NK][2], accb = 0.f;            // accb: thread k < NK adds up column k of dz
+#pragma unroll
+  for (int k = 0; k < NK; ++k) {
+    acc[k][0] = acc[k][1] = 0.f;
+    w[k][0] = w[k][1] = 0.f;
+    if (k < A) { w[k][0] = to_f(wpi[(size_t)k * F + col]); w[k][1] = to_f(wpi[(size_t)k * F + col + 1]); }
+    else if (k == A) { w[k][0] = to_f(wv[col]); w[k][1] = to_f(wv[col + 1]); }
+  }
+  pdl_entry();          // the head weights above were written several kernels ago
+  const int r0 = blockIdx.x * rows_per, r1 = min(n, r0 + rows_per);
+  for (int rb = r0; rb < r1; rb += HB_ROWS) {
+    __syncthreads();
+    for (int i = tid; i < HB_ROWS * NK; i += HB_THREADS) {
+      const int r = rb + i / NK, k = i % NK;
+      dzs[i / NK][k] = r < r1 ? (k < A ? dz[(size_t)r * A + k] : (k == A ? dV[r] : 0.f)) : 0.f;
+    }
+    __syncthreads();
+    if (tid < NK)
+      for (int r = 0; r < HB_ROWS; ++r) accb += dzs[r][tid];        // rows past the end hold zeros
+#pragma unroll 1
+    for (int q = 0; q < HB_ROWS && rb + q < r1; q += 8) {
+      uint32_t hv[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        hv[j] = rb + q + j < r1 ? __ldg(reinterpret_cast<const uint32_t*>(h + (size_t)(rb + q + j) * F + col)) : 0u;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (rb + q + j >= r1) break;
+        const float h0 = __uint_as_float(hv[j] << 16), h1 = __uint_as_float(hv[j] & 0xFFFF0000u);
+        float g0 = 0.f, g1 = 0.f;
+#pragma unroll
+        for (int k4 = 0; k4 < NK; k4 += 4) {
+          const float4 d4 = *reinterpret_cast<const float4*>(&dzs[q + j][k4]);
+          const float d[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            g0 = fmaf(d[i], w[k4 + i][0], g0); g1 = fmaf(d[i], w[k4 + i][1], g1);
+            acc[k4 + i][0] = fmaf(d[i], h0, acc[k4 + i][0]); acc[k4 + i][1] = fmaf(d[i], h1, acc[k4 + i][1]);
+          }
+        }
+        if (rb + q + j < r1)
+          *reinterpret_cast<uint32_t*>(g_fc + (size_t)(rb + q + j) * F + col) =
+              pack_bf16x2(h0 > 0.f ? g0 : 0.f, h1 > 0.f ? g1 : 0.f);
+      }
+    }
+  }
+  // partial sums of this CTA in the layout of the parameters themselves: policy rows [action][hidden unit], the
+  // value row, the two biases
+  const size_t cta = blockIdx.x;
+#pragma unroll
+  for (int k = 0; k < NK; ++k) {
+    if (k < A) *reinterpret_cast<float2*>(part_w + (cta * A + k) * F + col) = make_float2(acc[k][0], acc[k][1]);
+    else if (k == A) *reinterpret_cast<float2*>(part_vw + cta * F + col) = make_float2(acc[k][0], acc[k][1]);
+  }
+  if (tid < A) part_b[cta * A + tid] = accb;
+  else if (tid == A) part_vb[cta] = accb;
+}
+
+constexpr int HB_MAX_SPLITS = 148;
+static size_t tc_heads_scratch_floats() { return (size_t)HB_MAX_SPLITS * (512 * 20 + 20); }
+
+bool tc_heads_backward_supported(const NetDims& nd) { return nd.F == 512 && nd.A + 1 <= 20; }
+
+void tc_heads_backward(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, const bf16* h, int n, const float* dz,
+                       const float* dV, bf16* g_fc, float* grad, float* scratch, GradSegments* segs) {
+  const int A = nd.A;
+  int ctas = sm_count() < HB_MAX_SPLITS ? sm_count() : HB_MAX_SPLITS;
+  if (ctas > n) ctas = n;
+  const int rows_per = (n + ctas - 1) / ctas, splits = (n + rows_per - 1) / rows_per;
+  float* sc = scratch + tc_layer_scratch_offset(n, 4);
+  float* part_w = sc; float* part_b = part_w + (size_t)splits * 512 * A;
+  float* part_vw = part_b + (size_t)splits * A; float* part_vb = part_vw + (size_t)splits * 512;
+  KernelScope scope(lc, KID_HEADS_BWD);
+  if (A + 1 <= 8)
+    launch_kernel(lc, heads_backward_kernel<8>, splits, HB_THREADS, 0, h, dz, dV, theta16 + nd.pi_w, theta16 + nd.v_w, n, A,
+                  rows_per, g_fc, part_w, part_b, part_vw, part_vb);
+  else
+    launch_kernel(lc, heads_backward_kernel<20>, splits, HB_THREADS, 0, h, dz, dV, theta16 + nd.pi_w, theta16 + nd.v_w, n, A,
+                  rows_per, g_fc, part_w, part_b, part_vw, part_vb);
+  add_segment(segs, part_w, grad + nd.pi_w, splits, 1, 512 * A, 1.f);      // already in parameter order: a plain sum
+  add_segment(segs, part_b, grad + nd.pi_b, splits, 1, A, 1.f);
+  add_segment(segs, part_vw, grad + nd.v_w, splits, 1, 512, 1.f);
+  add_segment(segs, part_vb, grad + nd.v_b, splits, 1, 1, 1.f);
 }
 
 // ---- weight images for the backward contractions ------------------------------------------------------
