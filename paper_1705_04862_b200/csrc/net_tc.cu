@@ -244,7 +244,9 @@ __device__ __forceinline__ void relu_mask_store(bf16* out, const bf16* act, size
 }
 // value words (two bf16 each) survive where the activation word's halves are non-zero
 __device__ __forceinline__ uint32_t mask_pair(uint32_t v, uint32_t a) {
-  return v & ((a & 0x7FFFu ? 0xFFFFu : 0u) | (a & 0x7FFF0000u ? 0xFFFF0000u : 0u));
+  // stored activations are ReLU outputs, never negative: non-zero is the same as greater than zero
+  const __nv_bfloat162 a2 = *reinterpret_cast<const __nv_bfloat162*>(&a);
+  return v & __hgt2_mask(a2, __floats2bfloat162_rn(0.f, 0.f));
 }
 
 // the same with the 32 activations of the slice already in registers (four 16-byte words)
@@ -632,25 +634,40 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
     constexpr int COLS = BN / 2, CH = COLS / 8, RPP = 32 / CH, ROWB = COLS * 2;   // 16-byte chunks per row part
     const int quarter = warp & 3, col0 = (warp >> 2) * COLS;
     const uint32_t stg = a_base0 + STAGES * STAGE_BYTES + warp * (32 * ROWB);    // this warp's staging tile
+    // masked epilogues: the activations under a tile come from DRAM, so they are fetched two tiles ahead by
+    // asynchronous copies into a two-slot ring of this warp (every lane reads back only what it copied itself)
+    const uint32_t mring = a_base0 + STAGES * STAGE_BYTES + 8 * (32 * ROWB) + warp * (2 * 32 * ROWB);
     const int rr0 = lane / CH, ch = lane % CH;
+    auto fetch_mask = [&](int t, int slot) {
+      if (t < tiles) {
+        int b, y, x;
+        epi.map.split(t * TC_BM + quarter * 32 + rr0, b, y, x);
+        uint32_t at = epi.index(b, y, x, col0 + ch * 8);
+#pragma unroll
+        for (int p = 0; p < CH; ++p) {
+          const bool v = epi.map.is_output(b, y, x);
+          cp_async16(mring + slot * (32 * ROWB) + (p * RPP + rr0) * ROWB + ch * 16, epi.act + (v ? at : 0u), v ? 16u : 0u);
+          epi.map.template advance<Epi>(b, y, x, at, RPP);
+        }
+      }
+      cp_async_commit();            // one group per call, so the wait counts stay uniform
+    };
+    if constexpr (Epi::MASK) { fetch_mask(blockIdx.x, 0); fetch_mask(blockIdx.x + gridDim.x, 1); }
     int local = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
       const int ab = local & 1, pos0 = t * TC_BM + quarter * 32;
-      // where this lane's chunks go (and, for masked epilogues, the activations there), before the tile is ready
+      // where this lane's chunks go, before the tile is ready
       uint32_t idx[CH];                                          // element offsets (every tensor here is < 2^32 elements)
-      uint4 m[CH];
       uint32_t valid = 0;
       {
         int b, y, x;
         epi.map.split(pos0 + rr0, b, y, x);
+        uint32_t at = epi.index(b, y, x, col0 + ch * 8);
 #pragma unroll
         for (int p = 0; p < CH; ++p) {
-          idx[p] = epi.index(b, y, x, col0 + ch * 8);
-          if (epi.map.is_output(b, y, x)) {
-            valid |= 1u << p;
-            if (Epi::MASK) m[p] = __ldg(reinterpret_cast<const uint4*>(epi.act + idx[p]));
-          }
-          epi.map.advance(b, y, x, RPP);
+          idx[p] = at;
+          if (epi.map.is_output(b, y, x)) valid |= 1u << p;
+          epi.map.template advance<Epi>(b, y, x, at, RPP);
         }
       }
       const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
@@ -676,6 +693,7 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);            // the accumulator is free again
+      if constexpr (Epi::MASK) cp_async_wait<1>();               // this tile's activations have landed
 #pragma unroll
       for (int p = 0; p < CH; ++p) {
         const int rr = p * RPP + rr0;
@@ -683,12 +701,19 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                      : "r"(stg + rr * ROWB + ((uint32_t)(ch ^ (rr & (CH - 1))) << 4)) : "memory");
         if ((valid >> p) & 1u) {
-          if (Epi::MASK) { v.x = mask_pair(v.x, m[p].x); v.y = mask_pair(v.y, m[p].y); v.z = mask_pair(v.z, m[p].z); v.w = mask_pair(v.w, m[p].w); }
+          if constexpr (Epi::MASK) {
+            uint4 m;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(m.x), "=r"(m.y), "=r"(m.z), "=r"(m.w)
+                         : "r"(mring + (local & 1) * (32 * ROWB) + rr * ROWB + ch * 16) : "memory");
+            v.x = mask_pair(v.x, m.x); v.y = mask_pair(v.y, m.y); v.z = mask_pair(v.z, m.z); v.w = mask_pair(v.w, m.w);
+          }
           *reinterpret_cast<uint4*>(epi.out + idx[p]) = v;
         }
       }
       __syncwarp();                                              // staging tile free for the next tile
+      if constexpr (Epi::MASK) fetch_mask(t + 2 * gridDim.x, local & 1);
     }
+    if constexpr (Epi::MASK) cp_async_wait<0>();
   } else if (warp == 16 && lane == 0) {
     // ---------------- MMA issuer ----------------
     constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
@@ -810,6 +835,14 @@ template <int RASTER, int WIDTH, int OUT_H, int OUT_W> struct RasterMap {
     if (x >= WIDTH) { x -= WIDTH; if (++y >= RASTER / WIDTH) { y = 0; ++b; } }
   }
   __device__ __forceinline__ bool is_output(int b, int y, int x) const { return b < states && y < OUT_H && x < OUT_W; }
+  // the same step for an epilogue whose output offset is affine in (b, y, x): idx = b * E::SB + y * E::SY + x * E::SX + ...
+  template <class E> __device__ __forceinline__ void advance(int& b, int& y, int& x, uint32_t& idx, int n) const {
+    x += n; idx += (uint32_t)(n * E::SX);
+    if (x >= WIDTH) {
+      x -= WIDTH; idx += (uint32_t)(E::SY - WIDTH * E::SX);
+      if (++y >= RASTER / WIDTH) { y = 0; ++b; idx += (uint32_t)(E::SB - (RASTER / WIDTH) * E::SY); }
+    }
+  }
 };
 // Epilogues of the shifted kernels work in two phases per tile.  First the thread that owns a TMEM lane turns
 // its row's accumulators into bf16 (`values`) and parks them in a swizzled shared-memory staging tile.  Then
@@ -820,6 +853,7 @@ template <int RASTER, int WIDTH, int OUT_H, int OUT_W> struct RasterMap {
 // instruction, were what bounded these kernels before.
 template <class Map, int OUT_H, int OUT_W> struct ShiftBiasReluEpi {
   static constexpr bool MASK = false;
+  static constexpr int SX = 64, SY = OUT_W * 64, SB = OUT_H * OUT_W * 64;
   Map map; bf16* out; const float* bias; const bf16* act;       // act unused
   __device__ __forceinline__ void values(int col, const uint32_t (&r)[32], uint32_t (&o)[16]) const {
     const float4* b4 = reinterpret_cast<const float4*>(bias + col);
@@ -840,6 +874,7 @@ __device__ __forceinline__ void plain_bf16_values(const uint32_t (&r)[32], uint3
 }
 template <class Map, int OUT_H, int OUT_W> struct ShiftReluMaskEpi {
   static constexpr bool MASK = true;
+  static constexpr int SX = 64, SY = OUT_W * 64, SB = OUT_H * OUT_W * 64;
   Map map; bf16* out; const bf16* act;
   __device__ __forceinline__ void values(int, const uint32_t (&r)[32], uint32_t (&o)[16]) const { plain_bf16_values(r, o); }
   __device__ __forceinline__ uint32_t index(int b, int y, int x, int col) const {
@@ -849,6 +884,7 @@ template <class Map, int OUT_H, int OUT_W> struct ShiftReluMaskEpi {
 // stride-2 data gradient: accumulator columns 32 c .. 32 c + 31 are parity class c of raster pixel (yy, xx)
 template <class Map> struct ShiftReluMaskEpiS2 {
   static constexpr bool MASK = true;
+  static constexpr int SX = 2 * 32, SY = 2 * 20 * 32, SB = 20 * 20 * 32;
   Map map; bf16* out; const bf16* act;
   __device__ __forceinline__ void values(int, const uint32_t (&r)[32], uint32_t (&o)[16]) const { plain_bf16_values(r, o); }
   __device__ __forceinline__ uint32_t index(int b, int yy, int xx, int col) const {
@@ -1253,7 +1289,8 @@ static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_t
 
 template <class Cfg, class Epi, int BN, int STAGES, int NACC>
 static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int positions, uint32_t* err) {
-  constexpr int smem = Cfg::NT * BN * 128 + STAGES * Cfg::PLANES * Cfg::STAGE_ROWS * 128 + 8 * 32 * BN + 1024;
+  constexpr int smem = Cfg::NT * BN * 128 + STAGES * Cfg::PLANES * Cfg::STAGE_ROWS * 128 + 8 * 32 * BN +
+                       (Epi::MASK ? 2 * 8 * 32 * BN : 0) + 1024;        // weights, stages, staging tiles, activation rings
   static_assert(smem <= 227 * 1024, "shared memory budget");
   auto kern = tc_shift_kernel<Cfg, Epi, BN, STAGES, NACC>;
   static bool configured = false;
@@ -2444,7 +2481,7 @@ void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* con
   typedef NatConv3 C3;
   const int M = n * C3::H * C3::W;
   typedef RasterMap<121, 11, 9, 9> Map;
-  tc_shift<C3DgradCfg, ShiftReluMaskEpi<Map, 9, 9>, 64, 6, 1>(
+  tc_shift<C3DgradCfg, ShiftReluMaskEpi<Map, 9, 9>, 64, 4, 1>(
       lc, KID_CONV3_DGRAD, C3DgradCfg{(const bf16*)gact[2], n}, images + 4 * 32 * 256,
       ShiftReluMaskEpi<Map, 9, 9>{Map{n}, (bf16*)gact[1], (const bf16*)act[1]}, n * 121, err);
   (void)M;
@@ -2453,7 +2490,7 @@ void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* con
   typedef NatConv2 C2;
   const int M = n * (C2::H / 2) * (C2::W / 2);
   typedef RasterMap<121, 11, 10, 10> Map;
-  tc_shift<C2DgradCfg, ShiftReluMaskEpiS2<Map>, 128, 6, 1>(
+  tc_shift<C2DgradCfg, ShiftReluMaskEpiS2<Map>, 128, 3, 1>(
       lc, KID_CONV2_DGRAD, C2DgradCfg{(const bf16*)gact[1], n}, images,
       ShiftReluMaskEpiS2<Map>{Map{n}, (bf16*)gact[0], (const bf16*)act[0]}, n * 121, err);
   (void)M;
