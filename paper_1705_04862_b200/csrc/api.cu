@@ -326,10 +326,13 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
         simt_backward_layer(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
                             c->gact, c->grad, c->scratch, l, !wgrad_done, l > 0 && !dgrad_done);
     }
-    if (use_tc(c)) tc_backward_finish(c->lc, &c->grad_segs);
+    // when every gradient goes through the finishing kernel, it also delivers the squared norm
+    const bool all_finished = use_tc(c) && c->tc_wgrad_mask == 0xF && tc_heads_backward_supported(c->nd);
+    int ready = 0;
+    if (use_tc(c)) ready = tc_backward_finish(c->lc, &c->grad_segs, all_finished ? c->norm_partials : nullptr);
     launch_clip_rmsprop(c->lc, c->nd.P, c->theta, c->rms, c->grad,
                         c->prec == PAAC_BF16 ? c->theta16 : nullptr, hp.lr, hp.rms_decay, hp.rms_eps, hp.clip_norm,
-                        c->norm_partials, c->stats);
+                        c->norm_partials, c->stats, all_finished ? ready : 0);
     if (c->prec == PAAC_BF16) refresh_weight_copies(c, false);
   });
   c->N += (uint64_t)c->B;

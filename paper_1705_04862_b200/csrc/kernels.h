@@ -50,7 +50,9 @@ struct GradSegments { GradSegment seg[12]; int n; int total_groups; };
 size_t tc_scratch_floats(int n);
 void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, int n, void* const act[],
                        void* const gact[], float* grad, float* scratch, int layer, GradSegments* segs, uint32_t* err);
-void tc_backward_finish(LaunchCtx& lc, GradSegments* segs);
+// sumsq_partials != nullptr: every block also leaves the sum of squares of the gradient values it wrote in
+// sumsq_partials[block]; returns the number of blocks launched
+int tc_backward_finish(LaunchCtx& lc, GradSegments* segs, float* sumsq_partials);
 // both heads in one kernel: gradient at the fc pre-activation into g_fc, the heads' parameter gradients as one more
 // set of partial sums for tc_backward_finish()
 bool tc_heads_backward_supported(const NetDims& nd);
@@ -86,9 +88,10 @@ void heads_backward(LaunchCtx& lc, int prec, const NetDims& nd, const float* the
                     float* grad, float* scratch);
 
 // ---- optimiser (optim.cu) -------------------------------------------------------------------
-constexpr int NORM_BLOCKS = 592;
+constexpr int NORM_BLOCKS = 1184;
 void launch_clip_rmsprop(LaunchCtx& lc, size_t P, float* theta, float* rms, const float* grad,
                          bf16* theta16 /* nullable */, float lr, float rho, float eps, float clip,
-                         float* norm_partials /* [NORM_BLOCKS] */, DeviceStats* stats);
+                         float* norm_partials /* [NORM_BLOCKS] */, DeviceStats* stats,
+                         int ready_partials = 0 /* > 0: norm_partials[0..ready_partials) already hold the squared norm */);
 
 }  // namespace paac

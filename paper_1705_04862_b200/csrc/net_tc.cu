@@ -1649,10 +1649,11 @@ __global__ void tc_bias_final_kernel(const float* __restrict__ part, int blocks,
 //   many splits: a group is 8 j x 32 co; warp w adds the splits w, w + 8, ... for all eight j (eight loads in
 //                flight per thread), the eight warps' sums are then added in warp order;
 //   few splits:  a group is 32 j x 32 co; warp w adds all splits, in order, for rows w, w + 8, w + 16, w + 24.
-__global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments segs) {
+__global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments segs, float* __restrict__ sumsq_partials) {
   pdl_entry();
   __shared__ float sh[8 * 8 * 33];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float ss = 0.f;                       // sum of squares of the gradient values this thread writes
   for (int grp = blockIdx.x; grp < segs.total_groups; grp += gridDim.x) {
     int si = 0;
     while (si + 1 < segs.n && grp >= segs.seg[si + 1].first_group) ++si;
@@ -1682,7 +1683,7 @@ __global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments seg
         float t = 0.f;
 #pragma unroll
         for (int w = 0; w < 8; ++w) t += sh[(w * 8 + q) * 33 + c];
-        if (co0 + c < CO && j0 + q < J) sg.dst[(size_t)(co0 + c) * J + j0 + q] = t * sg.scale;
+        if (co0 + c < CO && j0 + q < J) { const float v = t * sg.scale; sg.dst[(size_t)(co0 + c) * J + j0 + q] = v; ss = fmaf(v, v, ss); }
       }
       __syncthreads();
     } else {
@@ -1706,9 +1707,22 @@ __global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments seg
 #pragma unroll
       for (int rr = 0; rr < 4; ++rr) {
         const int c = warp + 8 * rr;
-        if (co0 + c < CO && j0 + lane < J) sg.dst[(size_t)(co0 + c) * J + j0 + lane] = sh[lane * 33 + c] * sg.scale;
+        if (co0 + c < CO && j0 + lane < J) { const float v = sh[lane * 33 + c] * sg.scale; sg.dst[(size_t)(co0 + c) * J + j0 + lane] = v; ss = fmaf(v, v, ss); }
       }
       __syncthreads();
+    }
+  }
+  // this block's share of the squared gradient norm (the optimiser adds the blocks' shares in block order)
+  if (sumsq_partials != nullptr) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+    if (lane == 0) sh[warp] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) t += sh[w];
+      sumsq_partials[blockIdx.x] = t;
     }
   }
 }
@@ -2295,13 +2309,15 @@ size_t tc_scratch_floats(int n) { return tc_layer_scratch_offset(n, 4) + tc_head
 
 // Enqueues the weight-gradient kernel of `layer` (0 = conv1 .. 3 = fc) and notes in *segs where its partial
 // sums are; tc_backward_finish() then turns all noted partial sums into the gradient vector in one launch.
-void tc_backward_finish(LaunchCtx& lc, GradSegments* segs) {
+int tc_backward_finish(LaunchCtx& lc, GradSegments* segs, float* sumsq_partials) {
+  int blocks = 0;
   if (segs->n > 0) {
     KernelScope scope(lc, KID_WGRAD_REDUCE);
-    const int blocks = segs->total_groups < 8 * sm_count() ? segs->total_groups : 8 * sm_count();
-    launch_kernel(lc, tc_finalize_grads_kernel, blocks, 256, 0, *segs);
+    blocks = segs->total_groups < NORM_BLOCKS ? segs->total_groups : NORM_BLOCKS;
+    launch_kernel(lc, tc_finalize_grads_kernel, blocks, 256, 0, *segs, sumsq_partials);
   }
   segs->n = 0; segs->total_groups = 0;
+  return blocks;
 }
 
 void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, int n, void* const act[],

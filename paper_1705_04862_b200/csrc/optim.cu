@@ -41,18 +41,27 @@ clip_rmsprop_kernel(size_t P, float* __restrict__ theta, float* __restrict__ rms
                     bf16* __restrict__ theta16, float lr, float rho, float eps, float clip,
                     const float* __restrict__ partials, int n_partials, DeviceStats* stats) {
   pdl_entry();
-  __shared__ float sh[OPT_THREADS];
+  __shared__ float sh[OPT_THREADS / 32];
   __shared__ float s_scale;
+  // this thread's first elements do not depend on the norm: fetch them before the norm is known
+  const size_t n4 = P / 4;
+  float4* t4 = reinterpret_cast<float4*>(theta);
+  float4* m4 = reinterpret_cast<float4*>(rms);
+  const float4* g4 = reinterpret_cast<const float4*>(g);
+  const size_t i0 = blockIdx.x * (size_t)OPT_THREADS + threadIdx.x;
+  float4 gv0 = make_float4(0.f, 0.f, 0.f, 0.f), mv0 = gv0, tv0 = gv0;
+  if (i0 < n4) { gv0 = g4[i0]; mv0 = m4[i0]; tv0 = t4[i0]; }
   float acc = 0.f;
   for (int i = threadIdx.x; i < n_partials; i += OPT_THREADS) acc += partials[i];
-  sh[threadIdx.x] = acc;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = acc;
   __syncthreads();
-  for (int s = OPT_THREADS / 2; s > 0; s >>= 1) {
-    if (threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s];
-    __syncthreads();
-  }
   if (threadIdx.x == 0) {
-    const float norm = sqrtf(sh[0]);
+    float total = 0.f;
+#pragma unroll
+    for (int w = 0; w < OPT_THREADS / 32; ++w) total += sh[w];
+    const float norm = sqrtf(total);
     float scale = 1.f;
     const bool ok = isfinite(norm);
     if (ok && clip > 0.f && norm > clip) scale = clip / norm;
@@ -67,12 +76,10 @@ clip_rmsprop_kernel(size_t P, float* __restrict__ theta, float* __restrict__ rms
   const float scale = s_scale;
   if (scale < 0.f) return;
   const float one_m_rho = 1.f - rho;
-  const size_t n4 = P / 4;
-  float4* t4 = reinterpret_cast<float4*>(theta);
-  float4* m4 = reinterpret_cast<float4*>(rms);
-  const float4* g4 = reinterpret_cast<const float4*>(g);
-  for (size_t i = blockIdx.x * (size_t)OPT_THREADS + threadIdx.x; i < n4; i += (size_t)gridDim.x * OPT_THREADS) {
-    float4 gv = g4[i], mv = m4[i], tv = t4[i];
+  for (size_t i = i0; i < n4; i += (size_t)gridDim.x * OPT_THREADS) {
+    float4 gv, mv, tv;
+    if (i == i0) { gv = gv0; mv = mv0; tv = tv0; }
+    else { gv = g4[i]; mv = m4[i]; tv = t4[i]; }
     float* gp = &gv.x; float* mp = &mv.x; float* tp = &tv.x;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -102,14 +109,16 @@ clip_rmsprop_kernel(size_t P, float* __restrict__ theta, float* __restrict__ rms
 
 void launch_clip_rmsprop(LaunchCtx& lc, size_t P, float* theta, float* rms, const float* grad,
                          bf16* theta16, float lr, float rho, float eps, float clip, float* norm_partials,
-                         DeviceStats* stats) {
-  {
+                         DeviceStats* stats, int ready_partials) {
+  int n_partials = ready_partials;
+  if (ready_partials <= 0) {
     KernelScope scope(lc, KID_SUMSQ);
     launch_kernel(lc, sumsq_kernel, NORM_BLOCKS, OPT_THREADS, 0, grad, P, norm_partials);
+    n_partials = NORM_BLOCKS;
   }
   KernelScope scope(lc, KID_CLIP_RMSPROP);
   launch_kernel(lc, clip_rmsprop_kernel, NORM_BLOCKS, OPT_THREADS, 0, P, theta, rms, grad, theta16, lr, rho, eps, clip,
-                                                              norm_partials, NORM_BLOCKS, stats);
+                                                              norm_partials, n_partials, stats);
 }
 
 }  // namespace paac
