@@ -217,6 +217,48 @@ heads_fused_kernel(const float* __restrict__ part, int splits, const float* __re
   }
 }
 
+// The tail of the heads for the cluster path of the fully connected layer, which has already taken the head dot
+// products over each half of the hidden units: hp[half][e][k], k < A the policy rows, k = A the value row, rows
+// HS_LD floats apart.  One warp per state, lane k holds logit k; softmax and sampling as in heads_kernel.
+constexpr int HS_LD = 32, HS_WARPS = 4;
+__global__ void __launch_bounds__(HS_WARPS * 32)
+heads_sample_kernel(const float* __restrict__ hp, const float* __restrict__ bpi, const float* __restrict__ bv, int n, int A,
+                    float* __restrict__ logits, float* __restrict__ values, uint64_t seed,
+                    const uint64_t* __restrict__ step_base, uint32_t t, const int32_t* __restrict__ forced,
+                    int32_t* __restrict__ actions, int32_t* __restrict__ sampled, float* __restrict__ uniforms) {
+  const int lane = threadIdx.x & 31;
+  const int e = blockIdx.x * HS_WARPS + (threadIdx.x >> 5);
+  const float b = lane < A ? __ldg(bpi + lane) : (lane == A ? __ldg(bv) : 0.f);     // biases are older than the previous kernel
+  pdl_entry();
+  if (e >= n) return;
+  float s = -INFINITY;
+  if (lane <= A) s = (hp[(size_t)e * HS_LD + lane] + hp[((size_t)n + e) * HS_LD + lane]) + b;
+  const float z = lane < A ? s : -INFINITY;
+  if (lane < A) logits[(size_t)e * A + lane] = z;
+  if (lane == A) values[e] = s;
+  if (actions == nullptr) return;
+
+  const float m = warp_max(z);
+  const float ex = lane < A ? expf(z - m) : 0.f;
+  const float lse = m + logf(warp_sum(ex));
+  const float p = lane < A ? expf(z - lse) : 0.f;
+  const uint64_t step = *step_base + t;
+  const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
+  float c = 0.f;
+  int a = A - 1;
+  bool found = false;
+  for (int k = 0; k < A; ++k) {
+    c += __shfl_sync(0xffffffffu, p, k);
+    if (!found && u < c) { a = k; found = true; }
+  }
+  if (lane == 0) {
+    sampled[e] = a;
+    if (forced != nullptr && forced[e] >= 0) a = forced[e];
+    actions[e] = a;
+    uniforms[e] = u;
+  }
+}
+
 bool heads_fused_supported(const NetDims& nd) { return nd.F == 512 && nd.pi_w % 8 == 0 && nd.A <= 32; }
 
 void launch_heads_fused(LaunchCtx& lc, const NetDims& nd, const float* theta, const bf16* theta16, const float* part,
@@ -224,6 +266,11 @@ void launch_heads_fused(LaunchCtx& lc, const NetDims& nd, const float* theta, co
                         const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
                         float* uniforms) {
   KernelScope scope(lc, KID_HEADS_FWD);
+  if (splits == 0) {          // `part` holds the head dot products of the two halves of the hidden units
+    launch_kernel_overlapped(lc, heads_sample_kernel, (n + HS_WARPS - 1) / HS_WARPS, HS_WARPS * 32, 0, part, theta + nd.pi_b,
+                             theta + nd.v_b, n, nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms);
+    return;
+  }
   launch_kernel(lc, heads_fused_kernel, (n + HF_WARPS - 1) / HF_WARPS, HF_WARPS * 32, 0, part, splits, theta + nd.layer[nd.n_conv].b_off, h_out,
                 theta16 + nd.pi_w, theta + nd.pi_b, theta16 + nd.v_w, theta + nd.v_b, n, nd.A, logits, values, seed,
                 step_base, t, forced, actions, sampled, uniforms);

@@ -30,8 +30,10 @@ size_t simt_scratch_floats(int arch, const NetDims& nd, int n);
 bool tc_supported(int arch, int prec);
 // fc_scratch: tc_fc_scratch_floats(n) floats for the split-k partial sums of the fully connected layer
 size_t tc_fc_scratch_floats(int n);
-// with fc_splits != nullptr the fully connected layer is left as *fc_splits split-k partial sums in fc_scratch
-// (part[split][n][512]) for launch_heads_fused to finish
+// with fc_splits != nullptr the end of the fully connected layer is shared with launch_heads_fused: either the layer
+// is left as *fc_splits > 0 split-k partial sums in fc_scratch (part[split][n][512]) for that kernel to finish, or
+// (*fc_splits == 0) the layer is complete and fc_scratch holds the head dot products of the two halves of the
+// hidden units, hp[2][n][32], which that call only has to add up
 void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* theta16, const bf16* images,
                 const uint8_t* frames, int n, void* const act[], float* fc_scratch, uint32_t* error_word,
                 int* fc_splits = nullptr);

@@ -1040,6 +1040,311 @@ __global__ void __launch_bounds__(256) fc_finish_kernel(const float* __restrict_
   }
 }
 
+// ---- fully connected layer, forward, as one cluster per output tile --------------------------------------------
+// h[m][n] = bf16(relu(sum_k A[m][k] W[n][k] + bias[n])) and the head dot products that follow it, in one launch.
+// An output tile is 128 rows x 256 columns; the CTAs of a cluster (its size = the number of K slices, chosen on
+// the host so that all clusters are resident at once) each multiply a slice of K into a tensor-memory accumulator,
+// park it as floats in their own shared memory (on top of the operand stages, which are no longer needed), write
+// it from there with whole-row accesses to their slice of part[split][m][n] and meet at a cluster barrier.  The
+// slices are read back microseconds later, from L2.  (Reading the parked tiles of the other CTAs directly through
+// distributed shared memory was measured two to three times slower than this round trip, in every access order
+// tried.)  CTA r of the cluster then owns an equal share of the tile's rows: it adds the slices in split order (so
+// the sum does not depend on timing), applies bias, ReLU and the bf16 rounding, stores h for the backward pass
+// and, from the rounded values, its share of the A + 1 head dot products (256 of the 512 hidden units) as
+// hp[column tile][m][k]; heads_sample_kernel adds the two shares.
+// Warps 0-3 move the accumulator, warps 4-7 stream the operands (cp.async), lane 0 of warp 8 issues the MMAs.
+constexpr int FCC_BN = 256, FCC_STAGES = 4, FCC_MAX_SPLITS = 8, FCC_LAG = 3, FCC_THREADS = 288, FCC_HP_LD = 32;
+constexpr uint32_t FCC_STAGE_BYTES = TC_BM * 128 + FCC_BN * 128, FCC_ACC_BYTES = TC_BM * FCC_BN * 4;
+constexpr uint32_t FCC_HEADW_BYTES = 33 * FCC_BN * 2;
+static_assert(FCC_ACC_BYTES <= FCC_STAGES * FCC_STAGE_BYTES, "the parked accumulator reuses the operand stages");
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// all threads of all CTAs of the cluster; release / acquire order the writes before it against the reads after it
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+struct FccShared {
+  uint64_t full[FCC_STAGES], empty[FCC_STAGES], acc_full;
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+__global__ void __launch_bounds__(FCC_THREADS, 1)
+tc_fc_cluster_kernel(const bf16* __restrict__ a, const bf16* __restrict__ w, const float* __restrict__ bias,
+                     const bf16* __restrict__ wpi, const bf16* __restrict__ wv, int A, bf16* __restrict__ h_out,
+                     float* part, float* __restrict__ hp, int M, int N, int K, int tiles_n, int splits,
+                     uint32_t* error_word) {
+  extern __shared__ uint8_t dyn_smem[];
+  __shared__ FccShared sh;
+  const uint32_t base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
+  const uint32_t headw = base + FCC_STAGES * FCC_STAGE_BYTES;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank(), tile = blockIdx.x / splits;
+  const int nt = tile % tiles_n, mt = tile / tiles_n;
+  const int kb_total = K / TC_BK, kb_base = kb_total / splits, kb_rem = kb_total % splits;
+  const int kb0 = rank * kb_base + min(rank, kb_rem), kb1 = kb0 + kb_base + (rank < kb_rem ? 1 : 0);
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < FCC_STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    mbar_init(&sh.acc_full, 1);
+    sh.abort = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 8) tmem_alloc(&sh.tmem_base, FCC_BN);
+  // head weights of this column tile: row k = policy row k (k < A, 16-byte aligned) or the value row (k = A, which
+  // follows the policy biases in the parameter vector and is only 2-byte aligned), 256 bf16 each
+  for (int i = threadIdx.x; i < A * (FCC_BN / 8); i += FCC_THREADS) {
+    const int k = i / (FCC_BN / 8), c = i % (FCC_BN / 8);
+    const uint4 v = __ldg(reinterpret_cast<const uint4*>(wpi + (size_t)k * N + nt * FCC_BN) + c);
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(headw + (uint32_t)(k * FCC_BN + 8 * c) * 2u),
+                 "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+  }
+  for (int c = threadIdx.x; c < FCC_BN / 2; c += FCC_THREADS) {
+    const bf16* src = wv + nt * FCC_BN + 2 * c;
+    const uint32_t v = (uint32_t)__bfloat16_as_ushort(src[0]) | ((uint32_t)__bfloat16_as_ushort(src[1]) << 16);
+    asm volatile("st.shared.b32 [%0], %1;" ::"r"(headw + (uint32_t)(A * FCC_BN + 2 * c) * 2u), "r"(v) : "memory");
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
+
+  if (warp >= 4 && warp < 8) {
+    // ---------------- producers: lane l copies chunk l & 7 of rows 32 pw + 4 p + (l >> 3) ----------------
+    const int pw = warp - 4, c = lane & 7, r4 = lane >> 3;
+    int it = 0;
+    bool alive = true;
+    for (int kb = kb0; kb < kb1; ++kb, ++it) {
+      const int s = it % FCC_STAGES;
+      const bool ok = mbar_wait(&sh.empty[s], ((it / FCC_STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+      if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+      const uint32_t stage = base + s * FCC_STAGE_BYTES + (uint32_t)(32 * pw) * 128u;
+#pragma unroll
+      for (int p = 0; p < 8; ++p) {
+        const uint32_t row = 4 * p + r4, off = row * 128u + ((uint32_t)(c ^ (row & 7)) << 4);
+        const int m = min(mt * TC_BM + 32 * pw + (int)row, M - 1), n = nt * FCC_BN + 32 * pw + (int)row;
+        cp_async16(stage + off, a + (size_t)m * K + kb * TC_BK + c * 8, 16u);
+        cp_async16(stage + TC_BM * 128 + off, w + (size_t)n * K + kb * TC_BK + c * 8, 16u);
+        cp_async16(stage + TC_BM * 128 + 128 * 128 + off, w + (size_t)(n + 128) * K + kb * TC_BK + c * 8, 16u);
+      }
+      cp_async_commit();
+      if (it >= FCC_LAG) {
+        cp_async_wait<FCC_LAG>();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.full[(it - FCC_LAG) % FCC_STAGES]);
+      }
+    }
+    cp_async_wait<0>();
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (alive && lane == 0)
+      for (int j = it > FCC_LAG ? it - FCC_LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % FCC_STAGES]);
+  } else if (warp == 8) {
+    if (lane == 0) {
+      // ---------------- MMA issuer ----------------
+      constexpr uint32_t idesc = make_idesc_bf16(TC_BM, FCC_BN, 0, 0);
+      int it = 0;
+      bool ok = true;
+      for (int kb = kb0; kb < kb1 && ok; ++kb, ++it) {
+        const int s = it % FCC_STAGES;
+        ok = mbar_wait(&sh.full[s], (it / FCC_STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+        if (!ok) break;
+        tcgen05_fence_after();
+        const uint32_t a_addr = base + s * FCC_STAGE_BYTES, b_addr = a_addr + TC_BM * 128;
+#pragma unroll
+        for (int k = 0; k < TC_BK / 16; ++k)
+          mma_bf16(tmem, make_smem_desc(a_addr + k * 32, 0, 1024, SWIZZLE_128B),
+                   make_smem_desc(b_addr + k * 32, 0, 1024, SWIZZLE_128B), idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+        mma_commit(&sh.empty[s]);
+      }
+      if (ok) mma_commit(&sh.acc_full);
+    }
+  } else {
+    // ---------------- accumulator -> this CTA's shared memory (float, 16-byte chunks swizzled by row) ----------------
+    const bool ok = mbar_wait(&sh.acc_full, 0, &sh.abort, error_word, ERR_WAIT_ACC);
+    if (__all_sync(0xffffffffu, ok)) {
+      tcgen05_fence_after();
+      const uint32_t row = (uint32_t)threadIdx.x, dst = base + row * (FCC_BN * 4u);
+#pragma unroll 1
+      for (int cc = 0; cc < FCC_BN / 32; ++cc) {
+        uint32_t r[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + cc * 32, r);
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((cc * 8 + q) ^ (row & 7u)) << 4)),
+                       "r"(r[4 * q]), "r"(r[4 * q + 1]), "r"(r[4 * q + 2]), "r"(r[4 * q + 3]) : "memory");
+      }
+      tcgen05_fence_before();
+    }
+  }
+  // The parked tile goes to this split's slice of part[split][m][n] with whole-row accesses (a warp writes 512
+  // contiguous bytes); the slices stay in L2 for the few microseconds until they are read back.
+  __syncthreads();
+  if (threadIdx.x < 256) {
+#pragma unroll 4
+    for (int i = 0; i < TC_BM * FCC_BN / 4 / 256; ++i) {
+      const uint32_t q = (uint32_t)threadIdx.x + 256u * i, row = q >> 6, c = q & 63u;
+      const int m = mt * TC_BM + (int)row;
+      uint32_t r0, r1, r2, r3;
+      asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                   : "r"(base + row * (FCC_BN * 4u) + ((c ^ (row & 7u)) << 4)) : "memory");
+      if (m < M)
+        __stcg(reinterpret_cast<float4*>(part + ((size_t)rank * M + m) * N + nt * FCC_BN) + c,
+               make_float4(__uint_as_float(r0), __uint_as_float(r1), __uint_as_float(r2), __uint_as_float(r3)));
+    }
+    __threadfence();
+  }
+  // Every CTA of the cluster reaches the barrier whatever happened above (a wait that gave up only raises the
+  // error word; the numbers of that launch are then meaningless and the host reports the time-out).
+  __syncwarp();
+  cluster_sync_all();
+  // ---------------- this CTA's share of the tile's rows: sum over the cluster, bias, ReLU, heads ----------------
+  // rows [128 rank / splits, 128 (rank + 1) / splits), sixteen at a time; thread (rl, cg) owns the 16-byte chunks
+  // cg, cg + 16, cg + 32, cg + 48 of row rl, i.e. columns 4 (cg + 16 j) .. + 3: the sixteen threads of a row read
+  // 256 contiguous bytes at a time
+  const int row_lo = TC_BM * rank / splits, row_hi = TC_BM * (rank + 1) / splits;
+  for (int row0 = row_lo + 2 * warp; warp < 8 && row0 < row_hi; row0 += 16) {
+    const int cg = lane & 15;
+    const uint32_t row = (uint32_t)(row0 + (lane >> 4));
+    const bool live = (int)row < row_hi;
+    const int m = live ? mt * TC_BM + (int)row : M;
+    float v[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = 0.f;
+    if (m < M) {
+      const float4* src = reinterpret_cast<const float4*>(part + (size_t)m * N + nt * FCC_BN) + cg;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        float4 t[4][4];
+#pragma unroll
+        for (int s = 0; s < 4; ++s)
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            t[s][j] = 4 * half + s < splits ? __ldcg(src + (size_t)(4 * half + s) * M * (N / 4) + 16 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s = 0; s < 4; ++s)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            v[4 * j] += t[s][j].x; v[4 * j + 1] += t[s][j].y; v[4 * j + 2] += t[s][j].z; v[4 * j + 3] += t[s][j].w;
+          }
+      }
+    }
+    float x[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int n = nt * FCC_BN + 4 * (cg + 16 * j);
+      const float4 b = __ldg(reinterpret_cast<const float4*>(bias + n));
+      const bf16 h0 = __float2bfloat16_rn(fmaxf(v[4 * j] + b.x, 0.f)), h1 = __float2bfloat16_rn(fmaxf(v[4 * j + 1] + b.y, 0.f));
+      const bf16 h2 = __float2bfloat16_rn(fmaxf(v[4 * j + 2] + b.z, 0.f)), h3 = __float2bfloat16_rn(fmaxf(v[4 * j + 3] + b.w, 0.f));
+      x[4 * j] = __bfloat162float(h0); x[4 * j + 1] = __bfloat162float(h1);
+      x[4 * j + 2] = __bfloat162float(h2); x[4 * j + 3] = __bfloat162float(h3);
+      if (m < M)
+        *reinterpret_cast<uint2*>(h_out + (size_t)m * N + n) =
+            make_uint2((uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16),
+                       (uint32_t)__bfloat16_as_ushort(h2) | ((uint32_t)__bfloat16_as_ushort(h3) << 16));
+    }
+    // head dot products over this thread's 16 hidden units: independent sums first, then a butterfly over the 16
+    // threads of the row that halves the number of live values at each step and leaves thread cg with heads
+    // 2 cg and 2 cg + 1 (the additions pair up in a fixed pattern)
+    float pr[FCC_HP_LD];
+#pragma unroll
+    for (int k = 0; k < FCC_HP_LD; ++k) {
+      pr[k] = 0.f;
+      if (k <= A) {
+        float acc0 = 0.f, acc1 = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint32_t w0, w1;
+          asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(w0), "=r"(w1)
+                       : "r"(headw + (uint32_t)(k * FCC_BN + 4 * (cg + 16 * j)) * 2u) : "memory");
+          acc0 = fmaf(__uint_as_float(w0 << 16), x[4 * j], acc0);
+          acc1 = fmaf(__uint_as_float(w0 & 0xFFFF0000u), x[4 * j + 1], acc1);
+          acc0 = fmaf(__uint_as_float(w1 << 16), x[4 * j + 2], acc0);
+          acc1 = fmaf(__uint_as_float(w1 & 0xFFFF0000u), x[4 * j + 3], acc1);
+        }
+        pr[k] = acc0 + acc1;
+      }
+    }
+#pragma unroll
+    for (int o = 8, len = FCC_HP_LD / 2; o > 0; o >>= 1, len >>= 1) {
+      const bool up = (cg & o) != 0;
+#pragma unroll
+      for (int i = 0; i < len; ++i) {
+        const float send = up ? pr[i] : pr[i + len];
+        const float keep = up ? pr[i + len] : pr[i];
+        pr[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+      }
+    }
+    if (m < M) *reinterpret_cast<float2*>(hp + ((size_t)nt * M + m) * FCC_HP_LD + 2 * cg) = make_float2(pr[0], pr[1]);
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 8) {
+    __syncwarp();
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, FCC_BN);
+  }
+}
+
+static bool tc_fc_cluster_supported(int N, int K, int A) {
+  return N % FCC_BN == 0 && K % TC_BK == 0 && K / TC_BK >= FCC_MAX_SPLITS && A + 1 <= FCC_HP_LD;
+}
+
+constexpr int FCC_SMEM = FCC_STAGES * FCC_STAGE_BYTES + FCC_HEADW_BYTES + 1024;
+static_assert(FCC_SMEM <= 227 * 1024, "shared memory budget");
+
+// The largest cluster size (= number of K slices) with which all `tiles` clusters are resident at once, so that
+// the launch is one wave; how many clusters of a size fit depends on how the SMs are grouped on the part.
+static int tc_fc_cluster_splits(int tiles) {
+  static int max_active[FCC_MAX_SPLITS + 1] = {};          // 0 = not asked yet, -1 = the query failed
+  for (int sp = FCC_MAX_SPLITS; sp >= 4; --sp) {
+    if (max_active[sp] == 0) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(sp * 16); cfg.blockDim = dim3(FCC_THREADS); cfg.dynamicSmemBytes = FCC_SMEM;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = sp; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr; cfg.numAttrs = 1;
+      int n = 0;
+      max_active[sp] = cudaOccupancyMaxActiveClusters(&n, tc_fc_cluster_kernel, &cfg) == cudaSuccess && n > 0 ? n : -1;
+    }
+    if (max_active[sp] >= tiles) return sp;
+  }
+  return 4;
+}
+
+static void tc_fc_forward_cluster(LaunchCtx& lc, const bf16* a, const bf16* w, const float* bias, const bf16* wpi,
+                                  const bf16* wv, int A, bf16* h_out, float* part, float* hp, int M, int N, int K,
+                                  uint32_t* err) {
+  constexpr int smem = FCC_SMEM;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(tc_fc_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  const int tiles_m = (M + TC_BM - 1) / TC_BM, tiles_n = N / FCC_BN;
+  const int splits = tc_fc_cluster_splits(tiles_m * tiles_n);
+  KernelScope scope(lc, KID_FC_FWD);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(tiles_m * tiles_n * splits); cfg.blockDim = dim3(FCC_THREADS); cfg.dynamicSmemBytes = smem;
+  cfg.stream = lc.st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = splits; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = (pdl_enabled() && !lc.serialize_next) ? 2 : 1;
+  lc.serialize_next = false;
+  cudaLaunchKernelEx(&cfg, tc_fc_cluster_kernel, a, w, bias, wpi, wv, A, h_out, part, hp, M, N, K, tiles_n, splits, err);
+}
+
 // ---- first layer, forward: uint8 frames -> bf16 operand on the fly --------------------------------------
 // Same persistent skeleton, with eight producer warps: the frame rows a tile needs are copied once into
 // shared memory with cp.async (two tiles ahead); thread (row, half) then expands window rows
@@ -1335,7 +1640,7 @@ static void tc_gemm(LaunchCtx& lc, int kid, ASrc a, BSrc b, Epi e, int M, int N,
 }
 
 constexpr int FC_SPLITS = 7;
-size_t tc_fc_scratch_floats(int n) { return (size_t)FC_SPLITS * n * 512; }
+size_t tc_fc_scratch_floats(int n) { return (size_t)FCC_MAX_SPLITS * n * 512 + (size_t)2 * n * FCC_HP_LD; }
 
 static void tc_fc_forward(LaunchCtx& lc, const bf16* a, const bf16* w, const float* bias, bf16* out, int M, int N, int K,
                           float* part, uint32_t* err, int* splits_out) {
@@ -1385,8 +1690,15 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
           ShiftBiasReluEpi<Map, 7, 7>{Map{n}, (bf16*)act[2], theta + d[2].b_off, nullptr}, n * 81, err);
     }
     (void)M2; (void)M3;
-    tc_fc_forward(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, (bf16*)act[3], n, 512, 3136, fc_scratch, err,
-                  fc_splits);
+    if (fc_splits != nullptr && tc_fc_cluster_supported(512, 3136, nd.A)) {
+      // cluster path: h is complete and fc_scratch holds the head dot products as hp[2][n][32] (*fc_splits = 0)
+      tc_fc_forward_cluster(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, w + nd.pi_w, w + nd.v_w, nd.A,
+                            (bf16*)act[3], fc_scratch + (size_t)2 * n * FCC_HP_LD, fc_scratch, n, 512, 3136, err);
+      *fc_splits = 0;
+    } else {
+      tc_fc_forward(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, (bf16*)act[3], n, 512, 3136, fc_scratch, err,
+                    fc_splits);
+    }
   }
 }
 
