@@ -279,7 +279,8 @@ struct ReluMaskEpiTc {
     if (!p.valid) return;
     const uint4* a4 = reinterpret_cast<const uint4*>(act + p.idx);
 #pragma unroll
-    for (int j = 0; j < (int)(sizeof(p.m) / sizeof(uint4)); ++j) p.m[j] = __ldg(a4 + j);
+    for (int j = 0; j < (int)(sizeof(p.m) / sizeof(uint4)); ++j)
+      if (n0 + 8 * j < ld) p.m[j] = __ldg(a4 + j);          // a ragged last tile stops at the end of the row
   }
   template <class P> __device__ __forceinline__ void store(int col, const uint32_t (&r)[32], const P& p) const {
     if (p.valid) relu_mask_store_pre(out, p.idx + col, r, &p.m[col / 8]);
@@ -410,7 +411,8 @@ template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES>
 __global__ void __launch_bounds__(PK_THREADS, 1)
 tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi epi, int tiles_m, uint32_t* error_word) {
   static_assert(BN == 32 || BN == 64 || BN == 128, "tile width");
-  static_assert(STAGES >= PK_LAG + 2 && STAGES <= 8, "pipeline depth");
+  static_assert(STAGES >= 4 && STAGES <= 8, "pipeline depth");
+  constexpr int LAG = STAGES - 2 < PK_LAG ? STAGES - 2 : PK_LAG;      // copies in flight behind the one being issued
   constexpr uint32_t A_BYTES = TC_BM * 128, B_BLOCK = BN * 128, B_BYTES = NCLS * KB * B_BLOCK;
   extern __shared__ uint8_t dyn_smem[];
   __shared__ PkShared sh;
@@ -430,7 +432,8 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
   // resident weights: chunk index -> (class, k block, row, 16-byte chunk)
   for (int i = threadIdx.x; i < NCLS * KB * BN * 8; i += PK_THREADS) {
     const int c = i & 7, row = (i >> 3) % BN, kb = (i / (8 * BN)) % KB, cls = i / (8 * BN * KB);
-    const bf16* src = w + ((size_t)(cls * n_total + n0 + row) * KB + kb) * TC_BK + c * 8;
+    // rows past the last output column (a ragged last tile) repeat the last one; the epilogue drops their results
+    const bf16* src = w + ((size_t)(cls * n_total + min(n0 + row, n_total - 1)) * KB + kb) * TC_BK + c * 8;
     cp_async16(b_base + (cls * KB + kb) * B_BLOCK + sw128_offset(row, c), src, 16u);
   }
   cp_async_commit();
@@ -467,11 +470,11 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
           cp_async16(stage + row * 128u + ((uint32_t)(c ^ (row & 7)) << 4), src + c * 8, valid ? 16u : 0u);
         }
         cp_async_commit();
-        if (it >= PK_LAG) {
-          cp_async_wait<PK_LAG>();
+        if (it >= LAG) {
+          cp_async_wait<LAG>();
           fence_proxy_async_smem();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.full[(it - PK_LAG) % STAGES]);
+          if (lane == 0) mbar_arrive(&sh.full[(it - LAG) % STAGES]);
         }
       }
     }
@@ -480,27 +483,57 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
     fence_proxy_async_smem();
     __syncwarp();
     if (alive && lane == 0)
-      for (int j = it > PK_LAG ? it - PK_LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % STAGES]);
+      for (int j = it > LAG ? it - LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % STAGES]);
   } else if (warp < 4) {
-    // ---------------- epilogue ----------------
+    // ---------------- epilogue: accumulator -> bf16 through the ReLU mask of the layer below ----------------
+    // Two phases, so that global memory only sees whole rows: lane = accumulator row packs its BN values into a
+    // staging tile of the warp's own (16-byte chunks swizzled by row); then CH lanes cover one row, the warp
+    // reads RPP rows per pass, applies the mask (fetched with the same row-wise pattern before the accumulator
+    // was ready) and writes RPP x BN x 2 contiguous bytes per row.
+    constexpr int CH = BN / 8, RPP = 32 / CH, ROWB = BN * 2;
+    const uint32_t stg = a_base0 + STAGES * A_BYTES + warp * (32 * ROWB);
+    const int ch = lane % CH, rr0 = lane / CH;
+    const bool col_ok = n0 + ch * 8 < n_total;
     int local = 0;
     for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++local) {
-      const int ab = local & 1, z = t / tiles_m, m = (t % tiles_m) * TC_BM + threadIdx.x;
-      MaskPre<BN> pre;
-      epi.prefetch(m, n0, pre);
-      (void)z;
+      const int ab = local & 1, m0 = (t % tiles_m) * TC_BM + warp * 32;
+      uint4 mk[CH];
+#pragma unroll
+      for (int p = 0; p < CH; ++p) {
+        const int m = m0 + p * RPP + rr0;
+        mk[p] = make_uint4(0u, 0u, 0u, 0u);
+        if (m < epi.M && col_ok) mk[p] = __ldg(reinterpret_cast<const uint4*>(epi.act + (size_t)m * epi.ld + n0 + ch * 8));
+      }
       const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
 #pragma unroll
-      for (int c = 0; c < BN / 32; ++c) {
+      for (int cc = 0; cc < BN / 32; ++cc) {
         uint32_t r[32];
-        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN + c * 32, r);
-        epi.store(c * 32, r, pre);
+        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + ab * BN + cc * 32, r);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * ROWB + ((uint32_t)((cc * 4 + q) ^ (lane & (CH - 1))) << 4)),
+                       "r"(pack_bf16x2(__uint_as_float(r[8 * q]), __uint_as_float(r[8 * q + 1]))),
+                       "r"(pack_bf16x2(__uint_as_float(r[8 * q + 2]), __uint_as_float(r[8 * q + 3]))),
+                       "r"(pack_bf16x2(__uint_as_float(r[8 * q + 4]), __uint_as_float(r[8 * q + 5]))),
+                       "r"(pack_bf16x2(__uint_as_float(r[8 * q + 6]), __uint_as_float(r[8 * q + 7]))) : "memory");
       }
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
+      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);            // the accumulator is free again
+#pragma unroll
+      for (int p = 0; p < CH; ++p) {
+        const int rr = p * RPP + rr0, m = m0 + rr;
+        uint4 v;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                     : "r"(stg + rr * ROWB + ((uint32_t)(ch ^ (rr & (CH - 1))) << 4)) : "memory");
+        if (m < epi.M && col_ok) {
+          v.x = mask_pair(v.x, mk[p].x); v.y = mask_pair(v.y, mk[p].y); v.z = mask_pair(v.z, mk[p].z); v.w = mask_pair(v.w, mk[p].w);
+          *reinterpret_cast<uint4*>(epi.out + (size_t)m * epi.ld + n0 + ch * 8) = v;
+        }
+      }
+      __syncwarp();                                              // staging tile free for the next tile
     }
   } else if (lane == 0) {
     // ---------------- MMA issuer ----------------
@@ -1576,7 +1609,7 @@ static int sm_count() {
 
 template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES>
 static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_total, Epi e, int M, uint32_t* err) {
-  constexpr int smem = NCLS * KB * BN * 128 + STAGES * TC_BM * 128 + 1024;
+  constexpr int smem = NCLS * KB * BN * 128 + STAGES * TC_BM * 128 + 4 * 32 * BN * 2 + 1024;      // weights, stages, staging tiles
   static_assert(smem <= 227 * 1024, "shared memory budget");
   auto kern = tc_persistent_kernel<ASrc, Epi, BN, KB, NCLS, STAGES>;
   static bool configured = false;
@@ -1584,7 +1617,7 @@ static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_t
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     configured = true;
   }
-  const int tiles_m = (M + TC_BM - 1) / TC_BM, gy = n_total / BN;
+  const int tiles_m = (M + TC_BM - 1) / TC_BM, gy = (n_total + BN - 1) / BN;
   int gx = sm_count() / gy;
   if (gx < 1) gx = 1;
   if (gx > NCLS * tiles_m) gx = NCLS * tiles_m;
@@ -2801,7 +2834,7 @@ void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, 
 // ---- backward: data gradients ---------------------------------------------------------------------------
 void tc_backward_dgrad_fc(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   const bf16* wfc_t = images + 4 * 32 * 256 + 64 * 576;
-  tc_persistent<PlainSrc, ReluMaskEpiTc, 64, 8, 1, 8>(
+  tc_persistent<PlainSrc, ReluMaskEpiTc, 128, 8, 1, 4>(
       lc, KID_FC_DGRAD, PlainSrc{(const bf16*)gact[3], 512, n}, wfc_t, 3136,
       ReluMaskEpiTc{(bf16*)gact[2], (const bf16*)act[2], 3136, n}, n, err);
 }
