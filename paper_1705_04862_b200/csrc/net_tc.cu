@@ -2082,7 +2082,7 @@ static void add_segment(GradSegments* segs, const float* part, float* dst, int s
 }
 
 static int wg_splits(int num_blocks, int tiles_yz) {
-  int s = (296 + tiles_yz - 1) / tiles_yz;           // about two CTAs per SM in total
+  int s = sm_count() / tiles_yz;                     // one wave: the kernel's shared memory allows one CTA per SM
   if (s > num_blocks) s = num_blocks;
   if (s < 1) s = 1;
   return s;
@@ -2637,7 +2637,7 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
 // every layer keeps its own partial-sum region until the finishing kernel has run
 static size_t tc_layer_scratch_floats(int n, int layer) {
   switch (layer) {
-    case 0: return wg_scratch_floats(n * 400, 256, 32, 1);
+    case 0: return (size_t)SWG_MAX_SPLITS * (256 * 32 + 2 * 32);      // per CTA: the weight tile and two bias rows
     case 1: return (size_t)SWG_MAX_SPLITS * (512 * 64 + 64);
     case 2: return (size_t)SWG_MAX_SPLITS * (576 * 64 + 64);
     default: return wg_scratch_floats(n, 3136, 512, 25 * 4);
