@@ -14,6 +14,8 @@
 //              stage to its "empty" barrier, then commits the accumulator barrier.
 // Every wait is bounded; a wait that gives up raises a CTA-wide abort flag and an error bit
 // the host reads, and all threads still meet at the final barrier so TMEM is released.
+#include <cuda.h>          // CUtensorMap and its enums only; the encoder is looked up at run time, nothing links to libcuda
+
 #include "kernels.h"
 #include "tc_common.cuh"
 
@@ -25,6 +27,47 @@ constexpr int TC_BM = 128, TC_BK = 64, TC_THREADS = 160;
 constexpr size_t TC_IMG_W2 = 0, TC_IMG_W3 = 4 * 32 * 256, TC_IMG_WFC = TC_IMG_W3 + 64 * 576,
                  TC_IMG_W1 = TC_IMG_WFC + (size_t)3136 * 512, TC_IMG_END = TC_IMG_W1 + 32 * 256;
 
+
+// ---- tensor maps for the plain row-major bf16 matrices (fully connected layer) ---------------------------------
+// map of matrix x[rows][cols] (row pitch `ld` elements) for boxes of box_rows x 64 elements with the 128-byte swizzle.
+// Maps are cached by their defining values: the matrices live at fixed places of the workspace, so after the first
+// iteration every call is a look-up.  Returns nullptr if the driver's encoder is unavailable or refuses.
+struct TmapKey { const void* p; uint64_t rows, cols, ld; uint32_t box_rows; };
+static const CUtensorMap* tc_tensor_map(const bf16* x, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn encode = nullptr;
+  static bool looked_up = false;
+  constexpr int MAX_MAPS = 64;
+  static TmapKey keys[MAX_MAPS];
+  static CUtensorMap maps[MAX_MAPS];
+  static int n_maps = 0;
+  for (int i = 0; i < n_maps; ++i)
+    if (keys[i].p == x && keys[i].rows == rows && keys[i].cols == cols && keys[i].ld == ld && keys[i].box_rows == box_rows)
+      return &maps[i];
+  if (!looked_up) {
+    looked_up = true;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      encode = (EncodeFn)fn;
+  }
+  if (encode == nullptr) return nullptr;
+  static int next = 0;                                   // a full cache is overwritten in turn: launches copy the map
+  const int slot = n_maps < MAX_MAPS ? n_maps : next++ % MAX_MAPS;
+  const cuuint64_t gdim[2] = {cols, rows}, gstride[1] = {ld * sizeof(bf16)};
+  const cuuint32_t box[2] = {64u, box_rows}, estride[2] = {1u, 1u};
+  keys[slot].p = nullptr;
+  if (encode(&maps[slot], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<bf16*>(x), gdim, gstride, box, estride,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return nullptr;
+  keys[slot] = TmapKey{x, rows, cols, ld, box_rows};
+  if (n_maps < MAX_MAPS) ++n_maps;
+  return &maps[slot];
+}
 
 struct TcShared {
   uint64_t full[8], empty[8], acc;
@@ -1085,8 +1128,9 @@ __global__ void __launch_bounds__(256) fc_finish_kernel(const float* __restrict_
 // the sum does not depend on timing), applies bias, ReLU and the bf16 rounding, stores h for the backward pass
 // and, from the rounded values, its share of the A + 1 head dot products (256 of the 512 hidden units) as
 // hp[column tile][m][k]; heads_sample_kernel adds the two shares.
-// Warps 0-3 move the accumulator, warps 4-7 stream the operands (cp.async), lane 0 of warp 8 issues the MMAs.
-constexpr int FCC_BN = 256, FCC_STAGES = 4, FCC_MAX_SPLITS = 8, FCC_LAG = 3, FCC_THREADS = 288, FCC_HP_LD = 32;
+// Warps 0-3 move the accumulator, one thread of warp 4 streams the operands (tiled bulk copies), lane 0 of warp 8
+// issues the MMAs; warps 0-7 share the finishing phase.
+constexpr int FCC_BN = 256, FCC_STAGES = 4, FCC_MAX_SPLITS = 8, FCC_THREADS = 288, FCC_HP_LD = 32;
 constexpr uint32_t FCC_STAGE_BYTES = TC_BM * 128 + FCC_BN * 128, FCC_ACC_BYTES = TC_BM * FCC_BN * 4;
 constexpr uint32_t FCC_HEADW_BYTES = 33 * FCC_BN * 2;
 static_assert(FCC_ACC_BYTES <= FCC_STAGES * FCC_STAGE_BYTES, "the parked accumulator reuses the operand stages");
@@ -1108,7 +1152,8 @@ struct FccShared {
 };
 
 __global__ void __launch_bounds__(FCC_THREADS, 1)
-tc_fc_cluster_kernel(const bf16* __restrict__ a, const bf16* __restrict__ w, const float* __restrict__ bias,
+tc_fc_cluster_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+                     const float* __restrict__ bias,
                      const bf16* __restrict__ wpi, const bf16* __restrict__ wv, int A, bf16* __restrict__ h_out,
                      float* part, float* __restrict__ hp, int M, int N, int K, int tiles_n, int splits,
                      uint32_t* error_word) {
@@ -1123,8 +1168,10 @@ tc_fc_cluster_kernel(const bf16* __restrict__ a, const bf16* __restrict__ w, con
   const int kb0 = rank * kb_base + min(rank, kb_rem), kb1 = kb0 + kb_base + (rank < kb_rem ? 1 : 0);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < FCC_STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < FCC_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
     mbar_init(&sh.acc_full, 1);
+    tma_prefetch_desc(&tm_a);
+    tma_prefetch_desc(&tm_w);
     sh.abort = 0u;
     fence_barrier_init();
   }
@@ -1149,36 +1196,19 @@ tc_fc_cluster_kernel(const bf16* __restrict__ a, const bf16* __restrict__ w, con
   pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
   if (warp >= 4 && warp < 8) {
-    // ---------------- producers: lane l copies chunk l & 7 of rows 32 pw + 4 p + (l >> 3) ----------------
-    const int pw = warp - 4, c = lane & 7, r4 = lane >> 3;
-    int it = 0;
-    bool alive = true;
-    for (int kb = kb0; kb < kb1; ++kb, ++it) {
-      const int s = it % FCC_STAGES;
-      const bool ok = mbar_wait(&sh.empty[s], ((it / FCC_STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
-      if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
-      const uint32_t stage = base + s * FCC_STAGE_BYTES + (uint32_t)(32 * pw) * 128u;
-#pragma unroll
-      for (int p = 0; p < 8; ++p) {
-        const uint32_t row = 4 * p + r4, off = row * 128u + ((uint32_t)(c ^ (row & 7)) << 4);
-        const int m = min(mt * TC_BM + 32 * pw + (int)row, M - 1), n = nt * FCC_BN + 32 * pw + (int)row;
-        cp_async16(stage + off, a + (size_t)m * K + kb * TC_BK + c * 8, 16u);
-        cp_async16(stage + TC_BM * 128 + off, w + (size_t)n * K + kb * TC_BK + c * 8, 16u);
-        cp_async16(stage + TC_BM * 128 + 128 * 128 + off, w + (size_t)(n + 128) * K + kb * TC_BK + c * 8, 16u);
-      }
-      cp_async_commit();
-      if (it >= FCC_LAG) {
-        cp_async_wait<FCC_LAG>();
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.full[(it - FCC_LAG) % FCC_STAGES]);
+    // ---------------- producer: one thread asks the copy engine for the two boxes of each K block ----------------
+    // (rows of A past M read as zeros)
+    if (warp == 4 && lane == 0) {
+      int it = 0;
+      for (int kb = kb0; kb < kb1; ++kb, ++it) {
+        const int s = it % FCC_STAGES;
+        if (!mbar_wait(&sh.empty[s], ((it / FCC_STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY)) break;
+        const uint32_t stage = base + s * FCC_STAGE_BYTES;
+        mbar_arrive_expect_tx(&sh.full[s], FCC_STAGE_BYTES);
+        tma_load_2d(stage, &tm_a, kb * TC_BK, mt * TC_BM, &sh.full[s]);
+        tma_load_2d(stage + TC_BM * 128, &tm_w, kb * TC_BK, nt * FCC_BN, &sh.full[s]);
       }
     }
-    cp_async_wait<0>();
-    fence_proxy_async_smem();
-    __syncwarp();
-    if (alive && lane == 0)
-      for (int j = it > FCC_LAG ? it - FCC_LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % FCC_STAGES]);
   } else if (warp == 8) {
     if (lane == 0) {
       // ---------------- MMA issuer ----------------
@@ -1353,10 +1383,14 @@ static int tc_fc_cluster_splits(int tiles) {
   return 4;
 }
 
-static void tc_fc_forward_cluster(LaunchCtx& lc, const bf16* a, const bf16* w, const float* bias, const bf16* wpi,
+// false (nothing launched) if the tensor maps cannot be made; the caller then takes the split-k kernel
+static bool tc_fc_forward_cluster(LaunchCtx& lc, const bf16* a, const bf16* w, const float* bias, const bf16* wpi,
                                   const bf16* wv, int A, bf16* h_out, float* part, float* hp, int M, int N, int K,
                                   uint32_t* err) {
   constexpr int smem = FCC_SMEM;
+  const CUtensorMap* tm_a = tc_tensor_map(a, (uint64_t)M, (uint64_t)K, (uint64_t)K, TC_BM);
+  const CUtensorMap* tm_w = tc_tensor_map(w, (uint64_t)N, (uint64_t)K, (uint64_t)K, FCC_BN);
+  if (tm_a == nullptr || tm_w == nullptr) return false;
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(tc_fc_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -1375,7 +1409,8 @@ static void tc_fc_forward_cluster(LaunchCtx& lc, const bf16* a, const bf16* w, c
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = (pdl_enabled() && !lc.serialize_next) ? 2 : 1;
   lc.serialize_next = false;
-  cudaLaunchKernelEx(&cfg, tc_fc_cluster_kernel, a, w, bias, wpi, wv, A, h_out, part, hp, M, N, K, tiles_n, splits, err);
+  cudaLaunchKernelEx(&cfg, tc_fc_cluster_kernel, *tm_a, *tm_w, bias, wpi, wv, A, h_out, part, hp, M, N, K, tiles_n, splits, err);
+  return true;
 }
 
 // ---- first layer, forward: uint8 frames -> bf16 operand on the fly --------------------------------------
@@ -1723,10 +1758,10 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
           ShiftBiasReluEpi<Map, 7, 7>{Map{n}, (bf16*)act[2], theta + d[2].b_off, nullptr}, n * 81, err);
     }
     (void)M2; (void)M3;
-    if (fc_splits != nullptr && tc_fc_cluster_supported(512, 3136, nd.A)) {
+    if (fc_splits != nullptr && tc_fc_cluster_supported(512, 3136, nd.A) &&
+        tc_fc_forward_cluster(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, w + nd.pi_w, w + nd.v_w, nd.A,
+                              (bf16*)act[3], fc_scratch + (size_t)2 * n * FCC_HP_LD, fc_scratch, n, 512, 3136, err)) {
       // cluster path: h is complete and fc_scratch holds the head dot products as hp[2][n][32] (*fc_splits = 0)
-      tc_fc_forward_cluster(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, w + nd.pi_w, w + nd.v_w, nd.A,
-                            (bf16*)act[3], fc_scratch + (size_t)2 * n * FCC_HP_LD, fc_scratch, n, 512, 3136, err);
       *fc_splits = 0;
     } else {
       tc_fc_forward(lc, (const bf16*)act[2], w + d[3].w_off, theta + d[3].b_off, (bf16*)act[3], n, 512, 3136, fc_scratch, err,

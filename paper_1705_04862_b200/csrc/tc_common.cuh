@@ -160,6 +160,20 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void* src
                ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
+// ---- tiled bulk copies (TMA) global -> shared through a tensor map -----------------------------------------------
+// One thread copies a box of a 2-D row-major matrix: coordinates (x = element column, y = row) of the box's first
+// element; x times the element size must be a multiple of 16 bytes.  Rows and columns outside the matrix read as
+// zeros.  With the map's 128-byte swizzle and a box 64 bf16 wide, the box lands as 128-byte rows whose 16-byte
+// chunks sit at position chunk ^ (row & 7): the image sw128_offset() describes (destination 1024-byte aligned).
+// Completion is counted in bytes on `bar`.  No multicast: every CTA fetches its own tiles.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void* tmap, int x, int y, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst_smem), "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");
+}
+
 // ---- shared-memory images ----------------------------------------------------------------------
 // 128-byte swizzle: within each 1024-byte group of eight 128-byte rows, the 16-byte chunk c of
 // row r lives at chunk position c ^ (r & 7).  The same image serves a K-major operand (rows =
