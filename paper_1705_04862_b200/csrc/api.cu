@@ -124,8 +124,8 @@ void fill_shape(paac_ctx* c, int arch, int n_e, int t_max, int A, const paac_hpa
 }
 
 int cuda_status(paac_ctx* c) {
-  (void)c;
-  return cudaGetLastError() == cudaSuccess ? PAAC_OK : PAAC_ERR_CUDA;
+  const bool launches_ok = cudaGetLastError() == cudaSuccess;
+  return launches_ok && !c->lc.host_failure ? PAAC_OK : PAAC_ERR_CUDA;
 }
 
 bool use_tc(const paac_ctx* c) { return tc_supported(c->arch, c->prec) && !c->simt_only; }

@@ -143,6 +143,7 @@ struct LaunchCtx {
   uint64_t count = 0;                 // kernels launched so far
   bool profiling = false;             // record a CUDA event pair around every launch
   bool serialize_next = true;         // the next launch takes plain stream order (no overlap with its predecessor)
+  bool host_failure = false;          // a launch could not be prepared on the host (sticky; reported as PAAC_ERR_CUDA)
   static constexpr int MAX_PENDING = 512;
   cudaEvent_t ev[MAX_PENDING][2];
   int ev_kid[MAX_PENDING];

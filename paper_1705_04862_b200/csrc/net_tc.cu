@@ -452,10 +452,10 @@ struct PkShared {
 
 template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES>
 __global__ void __launch_bounds__(PK_THREADS, 1)
-tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi epi, int tiles_m, uint32_t* error_word) {
+tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_a, const bf16* __restrict__ w, int n_total, Epi epi, int tiles_m,
+                     uint32_t* error_word) {
   static_assert(BN == 32 || BN == 64 || BN == 128, "tile width");
   static_assert(STAGES >= 4 && STAGES <= 8, "pipeline depth");
-  constexpr int LAG = STAGES - 2 < PK_LAG ? STAGES - 2 : PK_LAG;      // copies in flight behind the one being issued
   constexpr uint32_t A_BYTES = TC_BM * 128, B_BLOCK = BN * 128, B_BYTES = NCLS * KB * B_BLOCK;
   extern __shared__ uint8_t dyn_smem[];
   __shared__ PkShared sh;
@@ -466,7 +466,8 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
   const int total_tiles = NCLS * tiles_m;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    tma_prefetch_desc(&tm_a);
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 4); }
     sh.abort = 0u;
     fence_barrier_init();
@@ -489,44 +490,22 @@ tc_persistent_kernel(ASrc a_src, const bf16* __restrict__ w, int n_total, Epi ep
   pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
   if (warp >= 4 && warp < 8) {
-    // ---------------- producers ----------------
-    // Eight lanes cover the 128 bytes of one row, so every warp-wide copy instruction moves four whole
-    // rows; lane l handles chunk l & 7 of rows 32 pw + 4 p + (l >> 3), p = 0..7.
-    const int pw = warp - 4, c = lane & 7, r4 = lane >> 3;
-    int it = 0;
-    bool alive = true;
-    for (int t = blockIdx.x; t < total_tiles && alive; t += gridDim.x) {
-      const int m0 = (t % tiles_m) * TC_BM + 32 * pw + r4;
-      RowRef ref[8];
-#pragma unroll
-      for (int p = 0; p < 8; ++p) ref[p] = a_src.row(m0 + 4 * p);
-      for (int kb = 0; kb < KB; ++kb, ++it) {
-        const int s = it % STAGES;
-        const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
-        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
-        const uint32_t stage = a_base0 + s * A_BYTES + (uint32_t)(32 * pw) * 128u;
-#pragma unroll
-        for (int p = 0; p < 8; ++p) {
-          bool valid;
-          const bf16* src = a_src.at(ref[p], kb, valid);
-          const uint32_t row = 4 * p + r4;                       // row inside the warp's 32-row slice
-          cp_async16(stage + row * 128u + ((uint32_t)(c ^ (row & 7)) << 4), src + c * 8, valid ? 16u : 0u);
-        }
-        cp_async_commit();
-        if (it >= LAG) {
-          cp_async_wait<LAG>();
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.full[(it - LAG) % STAGES]);
+    // ---------------- producer: one thread asks the copy engine for the 128 x 64 box of each K block ----------------
+    // (rows past the end of the matrix read as zeros)
+    if (warp == 4 && lane == 0) {
+      int it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const int m0 = (t % tiles_m) * TC_BM;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % STAGES;
+          ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&sh.full[s], A_BYTES);
+          tma_load_2d(a_base0 + s * A_BYTES, &tm_a, kb * TC_BK, m0, &sh.full[s]);
         }
       }
     }
-    // publish the last blocks
-    cp_async_wait<0>();
-    fence_proxy_async_smem();
-    __syncwarp();
-    if (alive && lane == 0)
-      for (int j = it > LAG ? it - LAG : 0; j < it; ++j) mbar_arrive(&sh.full[j % STAGES]);
   } else if (warp < 4) {
     // ---------------- epilogue: accumulator -> bf16 through the ReLU mask of the layer below ----------------
     // Two phases, so that global memory only sees whole rows: lane = accumulator row packs its BN values into a
@@ -1644,6 +1623,8 @@ static int sm_count() {
 
 template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES>
 static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_total, Epi e, int M, uint32_t* err) {
+  const CUtensorMap* tm_a = tc_tensor_map(a.x, (uint64_t)a.M, (uint64_t)KB * TC_BK, (uint64_t)a.ld, TC_BM);
+  if (tm_a == nullptr) { lc.host_failure = true; return; }      // no tensor-map encoder: the API call reports PAAC_ERR_CUDA
   constexpr int smem = NCLS * KB * BN * 128 + STAGES * TC_BM * 128 + 4 * 32 * BN * 2 + 1024;      // weights, stages, staging tiles
   static_assert(smem <= 227 * 1024, "shared memory budget");
   auto kern = tc_persistent_kernel<ASrc, Epi, BN, KB, NCLS, STAGES>;
@@ -1657,7 +1638,7 @@ static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_t
   if (gx < 1) gx = 1;
   if (gx > NCLS * tiles_m) gx = NCLS * tiles_m;
   KernelScope scope(lc, kid);
-  launch_kernel_overlapped(lc, kern, dim3(gx, gy), PK_THREADS, smem, a, w, n_total, e, tiles_m, err);
+  launch_kernel_overlapped(lc, kern, dim3(gx, gy), PK_THREADS, smem, *tm_a, w, n_total, e, tiles_m, err);
 }
 
 template <class Cfg, class Epi, int BN, int STAGES, int NACC>
