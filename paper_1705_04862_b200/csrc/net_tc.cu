@@ -1783,8 +1783,11 @@ template <int VALID> struct GradSrc {
 
 template <class XSrc, class GSrc, int VALID_N, int JT, int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS)
-tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, float* __restrict__ bias_partial, int n_atoms,
-                int J, int CO, int num_blocks, int blocks_per_split, uint32_t* error_word) {
+tc_wgrad_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_g, XSrc x_src, GSrc g_src,
+                float* __restrict__ partial, float* __restrict__ bias_partial, int n_atoms, int J, int CO, int num_blocks,
+                int blocks_per_split, uint32_t* error_word) {
+  // plain row-major matrices: one thread fetches a stage as 64 x 64 boxes (rows and columns outside read as zeros)
+  constexpr bool TMA = XSrc::ASYNC && VALID_N == 64;
   static_assert(BN == 64 || BN == 128, "tile width");
   static_assert(JT == 1 || JT == 2, "row tiles per CTA");
   constexpr uint32_t ATOM_COL = WG_ROWS * 128;                      // 8 KB: one atom column of a stage
@@ -1803,8 +1806,9 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, float* __re
   const uint32_t ones_base = tiles + STAGES * STAGE_BYTES;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 4); mbar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], TMA ? 1 : 4); mbar_init(&sh.empty[s], 1); }
     mbar_init(&sh.acc, 1);
+    if (TMA) { tma_prefetch_desc(&tm_x); tma_prefetch_desc(&tm_g); }
     sh.abort = 0u;
     fence_barrier_init();
   }
@@ -1834,35 +1838,15 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, float* __re
       if (!__all_sync(0xffffffffu, ok)) break;
       const uint32_t a_base = tiles + s * STAGE_BYTES, b_base = a_base + A_BYTES;
       const int m = kb * WG_ROWS + row;
-      if constexpr (XSrc::ASYNC && VALID_N == 64) {
-        // Eight lanes cover the 128 bytes of one row: lane l copies chunk l & 7 of rows 16 w + 4 p + (l >> 3),
-        // p = 0..3, for every atom column; the stage is published WG_LAG blocks later.
-        const int c = lane & 7, r4 = lane >> 3;
+      if constexpr (TMA) {
+        if (threadIdx.x == 0) {
+          mbar_arrive_expect_tx(&sh.full[s], STAGE_BYTES);
 #pragma unroll
-        for (int p = 0; p < 4; ++p) {
-          const int rw = 16 * warp + 4 * p + r4, mm = kb * WG_ROWS + rw;
-          const uint32_t off = (uint32_t)(rw >> 3) * 1024u + (uint32_t)(rw & 7) * 128u + ((uint32_t)(c ^ (rw & 7)) << 4);
-          const RowRef ref = x_src.row(mm);
+          for (int col = 0; col < 2 * JT; ++col)
+            tma_load_2d(a_base + col * ATOM_COL, &tm_x, (atom0 + col) * 64, kb * WG_ROWS, &sh.full[s]);
 #pragma unroll
-          for (int col = 0; col < 2 * JT; ++col) {
-            bool valid = false;
-            const bf16* src = x_src.x;
-            if (atom0 + col < n_atoms) src = x_src.at(ref, atom0 + col, valid);
-            cp_async16(a_base + col * ATOM_COL + off, src + c * 8, valid ? 16u : 0u);
-          }
-#pragma unroll
-          for (int gc = 0; gc < B_COLS; ++gc) {
-            bool valid;
-            const bf16* src = g_src.ptr(mm, n0 + gc * 64, valid);
-            cp_async16(b_base + gc * ATOM_COL + off, src + c * 8, valid ? 16u : 0u);
-          }
-        }
-        cp_async_commit();
-        if (it >= WG_LAG) {
-          cp_async_wait<WG_LAG>();
-          fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sh.full[(it - WG_LAG) % STAGES]);
+          for (int gc = 0; gc < B_COLS; ++gc)
+            tma_load_2d(b_base + gc * ATOM_COL, &tm_g, n0 + gc * 64, kb * WG_ROWS, &sh.full[s]);
         }
       } else {
         uint4 v[8];
@@ -1891,14 +1875,6 @@ tc_wgrad_kernel(XSrc x_src, GSrc g_src, float* __restrict__ partial, float* __re
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.full[s]);
       }
-    }
-    if constexpr (XSrc::ASYNC && VALID_N == 64) {
-      const int n_it = kb1 > kb0 ? kb1 - kb0 : 0;
-      cp_async_wait<0>();
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0 && !sh.abort)
-        for (int j = n_it > WG_LAG ? n_it - WG_LAG : 0; j < n_it; ++j) mbar_arrive(&sh.full[j % STAGES]);
     }
     // ---------------- epilogue: float partial tile to scratch ----------------
     if (kb1 > kb0 && mbar_wait(&sh.acc, 0, &sh.abort, error_word, ERR_WAIT_ACC)) {
@@ -2127,8 +2103,12 @@ static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, int rows, int n_a
   const int bps = (num_blocks + wg_splits(num_blocks, gy * gz) - 1) / wg_splits(num_blocks, gy * gz);
   const int splits = (num_blocks + bps - 1) / bps;
   float* bias_part = scratch + (size_t)splits * J * CO;
+  const CUtensorMap* tm_x = tc_tensor_map(xs.x, (uint64_t)xs.M, (uint64_t)J, (uint64_t)xs.ld, WG_ROWS);
+  const CUtensorMap* tm_g = tc_tensor_map(gs.g, (uint64_t)gs.M, (uint64_t)CO, (uint64_t)gs.ld, WG_ROWS);
+  if (tm_x == nullptr || tm_g == nullptr) { lc.host_failure = true; return; }      // no tensor-map encoder
   KernelScope scope(lc, kid);
-  launch_kernel_overlapped(lc, kern, dim3(splits, gy, gz), TC_THREADS, smem, xs, gs, scratch, bias_part, n_atoms, J, CO, num_blocks, bps, err);
+  launch_kernel_overlapped(lc, kern, dim3(splits, gy, gz), TC_THREADS, smem, *tm_x, *tm_g, xs, gs, scratch, bias_part, n_atoms, J, CO,
+                           num_blocks, bps, err);
   add_segment(segs, scratch, gw, splits, J, CO, scale);
   add_segment(segs, bias_part, gb, splits, 1, CO, 1.f);
 }
