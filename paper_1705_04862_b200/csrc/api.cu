@@ -298,9 +298,9 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
   if (!c->rollout_fresh) return PAAC_ERR_STATE;
   const paac_hparams& hp = c->hp;
   run_recorded(c, 1, c->cur, [&]() {
-    launch_returns(c->lc, c->n_e, c->t_max, hp.gamma, c->rewards, c->terminals, c->values, c->R, c->adv);
-    launch_head_grad(c->lc, c->B, c->A, hp.entropy_beta, hp.value_coef, c->logits, c->values, c->actions,
-                     c->R, c->adv, c->dz, c->dV, c->loss_terms, c->stats);
+    launch_returns_head_grad(c->lc, c->n_e, c->t_max, c->A, hp.gamma, hp.entropy_beta, hp.value_coef, c->rewards,
+                             c->terminals, c->logits, c->values, c->actions, c->R, c->adv, c->dz, c->dV, c->loss_terms,
+                             c->stats);
     const int L = c->nd.n_conv;
     if (use_tc(c) && tc_heads_backward_supported(c->nd))
       tc_heads_backward(c->lc, c->nd, c->theta16, (const bf16*)c->act[L], c->B, c->dz, c->dV, (bf16*)c->gact[L], c->grad,

@@ -230,7 +230,7 @@ struct DeviceStats {
   float policy_loss, value_loss, entropy, grad_norm, clip_scale;
   int32_t status;
   uint32_t error_word;   // bit set by a kernel whose bounded wait or bounds check gave up
-  uint32_t pad;
+  uint32_t arrivals;     // blocks of the head-gradient kernel that have finished (back to zero when it ends)
 };
 
 }  // namespace paac

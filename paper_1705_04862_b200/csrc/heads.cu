@@ -352,96 +352,112 @@ void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta
                                                             sampled, uniforms);
 }
 
-// One thread per environment walks its t_max transitions backwards:
-// R_t = r_t + gamma * (1 - terminal_t) * R_{t+1}, starting from the bootstrap value.
-__global__ void returns_kernel(int n_e, int t_max, float gamma, const int8_t* __restrict__ rewards,
-                               const uint8_t* __restrict__ terminals, const float* __restrict__ values,
-                               float* __restrict__ R, float* __restrict__ adv) {
-  pdl_entry();
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= n_e) return;
-  float next = values[(size_t)t_max * n_e + e];
-  for (int t = t_max - 1; t >= 0; --t) {
-    const size_t i = (size_t)t * n_e + e;
-    const float keep = terminals[i] ? 0.f : 1.f;
-    next = __fadd_rn((float)rewards[i], __fmul_rn(__fmul_rn(gamma, keep), next));
-    R[i] = next;
-    adv[i] = __fsub_rn(next, values[i]);
-  }
-}
-
-void launch_returns(LaunchCtx& lc, int n_e, int t_max, float gamma, const int8_t* rewards,
-                    const uint8_t* terminals, const float* values, float* R, float* adv) {
-  KernelScope scope(lc, KID_RETURNS);
-  launch_kernel(lc, returns_kernel, (n_e + 127) / 128, 128, 0, n_e, t_max, gamma, rewards, terminals, values, R, adv);
-}
-
-// One warp per experience: d/dz and d/dV of
+// One warp per experience i = (t, e).  Lane 0 first walks the environment's transitions backwards from the bootstrap
+// value down to step t, R_u = r_u + gamma * (1 - terminal_u) * R_{u+1} (one multiply by gamma * keep, one add, the
+// same operations in the same order for every t, so all warps of an environment see the same bits), which gives
+// R_t and adv_t = R_t - V_t.  Then d/dz and d/dV of
 //   (1/B) [ -adv log pi(a) - beta H + c_v (R - V)^2 ]
-// with adv and R constants; also the three per-sample loss terms for the statistics.
+// with adv and R constants, and the three per-sample loss terms.  The block that finishes last adds the loss terms
+// up in a fixed order (a reproducible mean) and resets the arrival counter for the next launch.
 __global__ void __launch_bounds__(128)
-head_grad_kernel(int B, int A, float beta, float value_coef, const float* __restrict__ logits,
-                 const float* __restrict__ values, const int32_t* __restrict__ actions, const float* __restrict__ R,
-                 const float* __restrict__ adv, float* __restrict__ dz, float* __restrict__ dV,
-                 float* __restrict__ loss_terms) {
+returns_head_grad_kernel(int n_e, int t_max, int A, float gamma, float beta, float value_coef,
+                         const int8_t* __restrict__ rewards, const uint8_t* __restrict__ terminals,
+                         const float* __restrict__ logits, const float* __restrict__ values,
+                         const int32_t* __restrict__ actions, float* __restrict__ R, float* __restrict__ adv,
+                         float* __restrict__ dz, float* __restrict__ dV, float* loss_terms, DeviceStats* stats) {
   pdl_entry();
+  const int B = n_e * t_max;
   const int lane = threadIdx.x & 31;
   const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (i >= B) return;
-  const float z = lane < A ? logits[(size_t)i * A + lane] : -INFINITY;
-  const float m = warp_max(z);
-  const float ex = lane < A ? expf(z - m) : 0.f;
-  const float lse = m + logf(warp_sum(ex));
-  const float lp = z - lse;
-  const float p = lane < A ? expf(lp) : 0.f;
-  const float H = -warp_sum(lane < A ? p * lp : 0.f);
-  const int a = actions[i];
-  const float ad = adv[i], invB = 1.0f / (float)B;
-  if (lane < A) {
-    const float g = -ad * ((lane == a ? 1.f : 0.f) - p) + beta * p * (lp + H);
-    dz[(size_t)i * A + lane] = g * invB;
+  __shared__ bool last;
+  __shared__ float sh[3][128], wsum[3][4];
+  if (i < B) {
+    float ret, ad;
+    {
+      const int t = i / n_e, e = i - t * n_e;
+      float next = values[(size_t)t_max * n_e + e];
+      if (t_max <= 32) {
+        // lane u fetches transition u, so that the loads are in flight together; the scan itself is serial
+        float rw = 0.f, keep = 0.f;
+        if (lane >= t && lane < t_max) {
+          const size_t j = (size_t)lane * n_e + e;
+          rw = (float)rewards[j];
+          keep = terminals[j] ? 0.f : 1.f;
+        }
+        for (int u = t_max - 1; u >= t; --u)
+          next = __fadd_rn(__shfl_sync(0xffffffffu, rw, u), __fmul_rn(__fmul_rn(gamma, __shfl_sync(0xffffffffu, keep, u)), next));
+      } else {
+        for (int u = t_max - 1; u >= t; --u) {
+          const size_t j = (size_t)u * n_e + e;
+          const float keep = terminals[j] ? 0.f : 1.f;
+          next = __fadd_rn((float)rewards[j], __fmul_rn(__fmul_rn(gamma, keep), next));
+        }
+      }
+      ret = next;
+      ad = __fsub_rn(next, values[i]);
+      if (lane == 0) { R[i] = ret; adv[i] = ad; }
+    }
+    const float z = lane < A ? logits[(size_t)i * A + lane] : -INFINITY;
+    const float m = warp_max(z);
+    const float ex = lane < A ? expf(z - m) : 0.f;
+    const float lse = m + logf(warp_sum(ex));
+    const float lp = z - lse;
+    const float p = lane < A ? expf(lp) : 0.f;
+    const float H = -warp_sum(lane < A ? p * lp : 0.f);
+    const int a = actions[i];
+    const float invB = 1.0f / (float)B;
+    if (lane < A) {
+      const float g = -ad * ((lane == a ? 1.f : 0.f) - p) + beta * p * (lp + H);
+      dz[(size_t)i * A + lane] = g * invB;
+    }
+    const float lp_a = __shfl_sync(0xffffffffu, lp, a);
+    if (lane == 0) {
+      const float d = values[i] - ret;
+      dV[i] = 2.f * value_coef * d * invB;
+      wsum[0][threadIdx.x >> 5] = -ad * lp_a;
+      wsum[1][threadIdx.x >> 5] = value_coef * d * d;
+      wsum[2][threadIdx.x >> 5] = H;
+    }
+  } else if (lane == 0) {
+    for (int j = 0; j < 3; ++j) wsum[j][threadIdx.x >> 5] = 0.f;
   }
-  const float lp_a = __shfl_sync(0xffffffffu, lp, a);
-  if (lane == 0) {
-    const float d = values[i] - R[i];
-    dV[i] = 2.f * value_coef * d * invB;
-    loss_terms[i] = -ad * lp_a;
-    loss_terms[(size_t)B + i] = value_coef * d * d;
-    loss_terms[2 * (size_t)B + i] = H;
-  }
-}
-
-// single block: fixed-order (hence reproducible) means of the three loss terms
-__global__ void __launch_bounds__(256) loss_stats_kernel(int B, const float* __restrict__ loss_terms, DeviceStats* stats) {
-  pdl_entry();
-  __shared__ float sh[3][256];
+  // the block's three sums go to loss_terms[j][block]; the last block to arrive adds all blocks' sums in a fixed order
+  __syncthreads();
+  if (threadIdx.x < 3)
+    loss_terms[(size_t)threadIdx.x * gridDim.x + blockIdx.x] =
+        ((wsum[threadIdx.x][0] + wsum[threadIdx.x][1]) + wsum[threadIdx.x][2]) + wsum[threadIdx.x][3];
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) last = atomicAdd(&stats->arrivals, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!last) return;
+  __threadfence();
   float acc[3] = {0.f, 0.f, 0.f};
-  for (int i = threadIdx.x; i < B; i += 256)
-    for (int j = 0; j < 3; ++j) acc[j] += loss_terms[(size_t)j * B + i];
+  for (int k = threadIdx.x; k < (int)gridDim.x; k += 128)
+    for (int j = 0; j < 3; ++j) acc[j] += __ldcg(loss_terms + (size_t)j * gridDim.x + k);
   for (int j = 0; j < 3; ++j) sh[j][threadIdx.x] = acc[j];
   __syncthreads();
-  for (int s = 128; s > 0; s >>= 1) {
-    if (threadIdx.x < s)
-      for (int j = 0; j < 3; ++j) sh[j][threadIdx.x] += sh[j][threadIdx.x + s];
+  for (int s2 = 64; s2 > 0; s2 >>= 1) {
+    if (threadIdx.x < s2)
+      for (int j = 0; j < 3; ++j) sh[j][threadIdx.x] += sh[j][threadIdx.x + s2];
     __syncthreads();
   }
   if (threadIdx.x == 0) {
     stats->policy_loss = sh[0][0] / B;
     stats->value_loss = sh[1][0] / B;
     stats->entropy = sh[2][0] / B;
+    stats->arrivals = 0u;
   }
 }
 
-void launch_head_grad(LaunchCtx& lc, int B, int A, float beta, float value_coef,
-                      const float* logits, const float* values, const int32_t* actions, const float* R,
-                      const float* adv, float* dz, float* dV, float* loss_terms, DeviceStats* stats) {
-  {
-    KernelScope scope(lc, KID_HEAD_GRAD);
-    launch_kernel(lc, head_grad_kernel, (B + 3) / 4, 128, 0, B, A, beta, value_coef, logits, values, actions, R, adv, dz, dV,
-                                                     loss_terms);
-  }
+void launch_returns_head_grad(LaunchCtx& lc, int n_e, int t_max, int A, float gamma, float beta, float value_coef,
+                              const int8_t* rewards, const uint8_t* terminals, const float* logits, const float* values,
+                              const int32_t* actions, float* R, float* adv, float* dz, float* dV, float* loss_terms,
+                              DeviceStats* stats) {
+  const int B = n_e * t_max;
   KernelScope scope(lc, KID_HEAD_GRAD);
-  launch_kernel(lc, loss_stats_kernel, 1, 256, 0, B, loss_terms, stats);
+  launch_kernel(lc, returns_head_grad_kernel, (B + 3) / 4, 128, 0, n_e, t_max, A, gamma, beta, value_coef, rewards, terminals,
+                logits, values, actions, R, adv, dz, dV, loss_terms, stats);
 }
 
 }  // namespace paac

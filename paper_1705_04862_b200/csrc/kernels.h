@@ -79,11 +79,11 @@ void launch_heads_fused(LaunchCtx& lc, const NetDims& nd, const float* theta, co
                         int splits, bf16* h_out, int n, float* logits, float* values, uint64_t seed,
                         const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
                         float* uniforms);
-void launch_returns(LaunchCtx& lc, int n_e, int t_max, float gamma, const int8_t* rewards,
-                    const uint8_t* terminals, const float* values, float* R, float* adv);
-void launch_head_grad(LaunchCtx& lc, int B, int A, float beta, float value_coef,
-                      const float* logits, const float* values, const int32_t* actions, const float* R,
-                      const float* adv, float* dz, float* dV, float* loss_terms /* [3][B] */, DeviceStats* stats);
+// n-step returns and advantages, the loss gradient at the heads and the loss statistics, in one launch
+void launch_returns_head_grad(LaunchCtx& lc, int n_e, int t_max, int A, float gamma, float beta, float value_coef,
+                              const int8_t* rewards, const uint8_t* terminals, const float* logits, const float* values,
+                              const int32_t* actions, float* R, float* adv, float* dz, float* dV,
+                              float* loss_terms /* [3][B] */, DeviceStats* stats);
 // gradient of the two heads' parameters and of the fc pre-activation
 void heads_backward(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
                     const bf16* theta16, const void* h, int n, const float* dz, const float* dV, void* gact_fc,
