@@ -445,7 +445,7 @@ tc_gemm_kernel(ASrc a_src, BSrc b_src, Epi epi, int num_kb, uint32_t* error_word
 //   warp 8     lane 0 issues the MMAs and commits stages / accumulators
 constexpr int PK_THREADS = 288, PK_LAG = 5;
 struct PkShared {
-  uint64_t full[8], empty[8], acc_full[2], acc_empty[2];
+  uint64_t full[8], empty[8], acc_full[2], acc_empty[2], mask_full[2], mask_empty[2];
   uint32_t tmem_base;
   volatile uint32_t abort;
 };
@@ -624,6 +624,7 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 256); mbar_init(&sh.empty[s], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 8); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.mask_full[i], 256); mbar_init(&sh.mask_empty[i], 8); }
     sh.abort = 0u;
     fence_barrier_init();
   }
@@ -681,6 +682,27 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
       }
       // no waiting here: the hardware arrives on the stage's barrier for this thread when its copies have landed
       cp_async_mbar_arrive(&sh.full[s]);
+      if constexpr (Epi::MASK) {
+        // The activations under the tile (the ReLU mask of its epilogue) travel the same way, into a two-slot ring
+        // laid out per epilogue warp: producer warp w fetches what epilogue warp w will read.  The epilogue warps
+        // cannot fetch them themselves: a warp with asynchronous copies in flight waits for all of them at its next
+        // shared-memory load, which would chain every staging-tile read to the DRAM latency.
+        constexpr int COLS = BN / 2, CH = COLS / 8, RPP = 32 / CH, ROWB = COLS * 2;
+        const int ms = it & 1, ew = warp - 8, quarter = ew & 3, col0 = (ew >> 2) * COLS, rr0 = lane / CH, ch = lane % CH;
+        const bool okm = mbar_wait(&sh.mask_empty[ms], ((it >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+        if (!__all_sync(0xffffffffu, okm)) { alive = false; break; }
+        const uint32_t dst = a_base0 + STAGES * STAGE_BYTES + 8 * (32 * ROWB) + ew * (2 * 32 * ROWB) + ms * (32 * ROWB);
+        int b, y, x;
+        epi.map.split(t * TC_BM + quarter * 32 + rr0, b, y, x);
+        uint32_t at = epi.index(b, y, x, col0 + ch * 8);
+#pragma unroll
+        for (int p = 0; p < CH; ++p) {
+          const bool v = epi.map.is_output(b, y, x);
+          cp_async16(dst + (p * RPP + rr0) * ROWB + ch * 16, epi.act + (v ? at : 0u), v ? 16u : 0u);
+          epi.map.template advance<Epi>(b, y, x, at, RPP);
+        }
+        cp_async_mbar_arrive(&sh.mask_full[ms]);
+      }
     }
     cp_async_commit();
     cp_async_wait<0>();
@@ -689,25 +711,10 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
     constexpr int COLS = BN / 2, CH = COLS / 8, RPP = 32 / CH, ROWB = COLS * 2;   // 16-byte chunks per row part
     const int quarter = warp & 3, col0 = (warp >> 2) * COLS;
     const uint32_t stg = a_base0 + STAGES * STAGE_BYTES + warp * (32 * ROWB);    // this warp's staging tile
-    // masked epilogues: the activations under a tile come from DRAM, so they are fetched two tiles ahead by
-    // asynchronous copies into a two-slot ring of this warp (every lane reads back only what it copied itself)
+    // masked epilogues: the activations under a tile arrive in a two-slot ring of this warp, filled by producer
+    // warp (this warp + 8) and handed over through the mask_full / mask_empty barriers
     const uint32_t mring = a_base0 + STAGES * STAGE_BYTES + 8 * (32 * ROWB) + warp * (2 * 32 * ROWB);
     const int rr0 = lane / CH, ch = lane % CH;
-    auto fetch_mask = [&](int t, int slot) {
-      if (t < tiles) {
-        int b, y, x;
-        epi.map.split(t * TC_BM + quarter * 32 + rr0, b, y, x);
-        uint32_t at = epi.index(b, y, x, col0 + ch * 8);
-#pragma unroll
-        for (int p = 0; p < CH; ++p) {
-          const bool v = epi.map.is_output(b, y, x);
-          cp_async16(mring + slot * (32 * ROWB) + (p * RPP + rr0) * ROWB + ch * 16, epi.act + (v ? at : 0u), v ? 16u : 0u);
-          epi.map.template advance<Epi>(b, y, x, at, RPP);
-        }
-      }
-      cp_async_commit();            // one group per call, so the wait counts stay uniform
-    };
-    if constexpr (Epi::MASK) { fetch_mask(blockIdx.x, 0); fetch_mask(blockIdx.x + gridDim.x, 1); }
     int local = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
       const int ab = local & 1, pos0 = t * TC_BM + quarter * 32;
@@ -748,7 +755,10 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);            // the accumulator is free again
-      if constexpr (Epi::MASK) cp_async_wait<1>();               // this tile's activations have landed
+      if constexpr (Epi::MASK) {                                 // this tile's activations have landed
+        const bool okm = mbar_wait(&sh.mask_full[local & 1], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+        if (!__all_sync(0xffffffffu, okm)) break;
+      }
 #pragma unroll
       for (int p = 0; p < CH; ++p) {
         const int rr = p * RPP + rr0;
@@ -765,10 +775,9 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
           *reinterpret_cast<uint4*>(epi.out + idx[p]) = v;
         }
       }
-      __syncwarp();                                              // staging tile free for the next tile
-      if constexpr (Epi::MASK) fetch_mask(t + 2 * gridDim.x, local & 1);
+      __syncwarp();                                              // staging tile and ring slot free again
+      if constexpr (Epi::MASK) { if (lane == 0) mbar_arrive(&sh.mask_empty[local & 1]); }
     }
-    if constexpr (Epi::MASK) cp_async_wait<0>();
   } else if (warp == 16 && lane == 0) {
     // ---------------- MMA issuer ----------------
     constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
