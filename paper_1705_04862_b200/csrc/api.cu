@@ -136,8 +136,10 @@ void refresh_weight_copies(paac_ctx* c, bool cast) {
   if (tc_supported(c->arch, c->prec)) tc_relayout_weights(c->lc, c->nd, c->theta16, c->w_images);
 }
 
-// network + heads on the n_e states of `frames`, activations into slot `slot`
-void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample) {
+// network + heads on the n_e states of `frames`, activations into slot `slot`.  With `tail` the caller is about
+// to step the synthetic environments and can take the actions there: if the forward pass left the heads as partial
+// sums (see HeadsTail), no sampling kernel is launched, *tail describes what is left, and the result is true.
+bool forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, HeadsTail* tail = nullptr) {
   void* act[MAX_LAYERS];
   for (int l = 0; l <= c->nd.n_conv; ++l)
     act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
@@ -150,10 +152,15 @@ void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample) {
     int splits = 0;
     tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, c->w_images, frames, c->n_e, act, c->scratch,
                &c->stats->error_word, &splits);
+    if (tail != nullptr && splits == 0 && sample) {
+      *tail = HeadsTail{c->scratch, c->theta + c->nd.pi_b, c->theta + c->nd.v_b, c->A, c->logits + row * c->A,
+                        c->values + row, forced, actions, sampled, uniforms};
+      return true;
+    }
     launch_heads_fused(c->lc, c->nd, c->theta, c->theta16, c->scratch, splits, (bf16*)act[c->nd.n_conv], c->n_e,
                        c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot, forced, actions,
                        sampled, uniforms);
-    return;
+    return false;
   }
   if (use_tc(c))
     tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, c->w_images, frames, c->n_e, act, c->scratch,
@@ -163,6 +170,7 @@ void forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample) {
   launch_heads(c->lc, c->prec, c->nd, c->theta, c->theta16, act[c->nd.n_conv], c->n_e,
                c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot, forced, actions, sampled,
                uniforms);
+  return false;
 }
 
 void drop_graphs(paac_ctx* c) {
@@ -275,11 +283,16 @@ int paac_rollout(paac_ctx* c, paac_rollout_view* view) {
   const size_t fstep = (size_t)c->n_e * FRAME_BYTES;
   run_recorded(c, 0, c->cur, [&]() {
     for (int t = 0; t < c->t_max; ++t) {
-      forward_slot(c, fr + t * fstep, t, true);
+      HeadsTail tail;
+      const bool deferred = forward_slot(c, fr + t * fstep, t, true, &tail);
       uint8_t* dst = t + 1 < c->t_max ? fr + (t + 1) * fstep : nxt;
       const size_t row = (size_t)t * c->n_e;
-      launch_env_step(c->lc, c->seed, c->n_e, c->step_dev, (uint32_t)t, c->actions + row, c->hp.term_denom, dst,
-                      c->rewards + row, c->terminals + row, c->counters);
+      if (deferred)
+        launch_env_step_sampling(c->lc, c->seed, c->n_e, c->step_dev, (uint32_t)t, c->hp.term_denom, dst, c->rewards + row,
+                                 c->terminals + row, c->counters, tail);
+      else
+        launch_env_step(c->lc, c->seed, c->n_e, c->step_dev, (uint32_t)t, c->actions + row, c->hp.term_denom, dst,
+                        c->rewards + row, c->terminals + row, c->counters);
     }
     forward_slot(c, nxt, c->t_max, false);
     launch_advance_step(c->lc, c->step_dev, (uint32_t)c->t_max);

@@ -57,19 +57,60 @@ void launch_cast_bf16(LaunchCtx& lc, const float* src, bf16* dst, size_t n) {
 constexpr int ENV_THREADS = 256;
 constexpr int FRAME_WORDS = FRAME_H * FRAME_W;   // 7056, a multiple of 4
 
+// With SAMPLE the block's first warp also takes the action first: it finishes the heads of its environment from the
+// two partial dot products hp[half][e][k] the fully connected kernel left (k < A policy rows, k = A value row;
+// rows 32 floats apart), softmax, inverse-CDF draw from the Philox uniform of (env, step) exactly as the stand-alone
+// sampling kernel does, and writes logits, value, uniform and action; the transition then uses that action.
+template <bool SAMPLE>
 __global__ void __launch_bounds__(ENV_THREADS)
 env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, uint32_t t,
-                const int32_t* __restrict__ actions, uint32_t term_denom,
+                const int32_t* actions, uint32_t term_denom,
                 uint8_t* __restrict__ next_frames, int8_t* __restrict__ rewards, uint8_t* __restrict__ terminals,
-                int32_t* __restrict__ counters) {
-  pdl_entry();
+                int32_t* __restrict__ counters, HeadsTail ht) {
   __shared__ uint32_t s_base;
   const uint32_t e = blockIdx.x;
+  int32_t a_sampled = 0;
+  if (SAMPLE && threadIdx.x < 32) {
+    const int lane = threadIdx.x, A = ht.A;
+    const float bias = lane < A ? __ldg(ht.bpi + lane) : (lane == A ? __ldg(ht.bv) : 0.f);   // older than the previous kernel
+    pdl_entry();
+    float sum = -INFINITY;
+    if (lane <= A) sum = (ht.hp[(size_t)e * 32 + lane] + ht.hp[((size_t)n_e + e) * 32 + lane]) + bias;
+    const float z = lane < A ? sum : -INFINITY;
+    if (lane < A) ht.logits[(size_t)e * A + lane] = z;
+    if (lane == A) ht.values[e] = sum;
+    float m = z;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float se = lane < A ? expf(z - m) : 0.f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+    const float lse = m + logf(se);
+    const float p = lane < A ? expf(z - lse) : 0.f;
+    const uint64_t step64 = *step_base + t;
+    const float u = philox_uniform(e, (uint32_t)step64, (uint32_t)(step64 >> 32), RNG_STREAM_ACTION, seed);
+    float c = 0.f;
+    int a = A - 1;
+    bool found = false;
+    for (int k = 0; k < A; ++k) {
+      c += __shfl_sync(0xffffffffu, p, k);
+      if (!found && u < c) { a = k; found = true; }
+    }
+    if (lane == 0) {
+      ht.sampled[e] = a;
+      if (ht.forced != nullptr && ht.forced[e] >= 0) a = ht.forced[e];
+      ht.actions[e] = a;
+      ht.uniforms[e] = u;
+    }
+    a_sampled = a;
+  } else {
+    pdl_entry();
+  }
   if (threadIdx.x == 0) {
     uint32_t tag = 0u, frame_step = 0u;
-    if (actions != nullptr) {
+    if (SAMPLE || actions != nullptr) {
       const uint32_t step = (uint32_t)(*step_base) + t;       // global step index of this transition
-      const int32_t a = actions[e];
+      const int32_t a = SAMPLE ? a_sampled : actions[e];
       const uint32_t base = env_hash_base(seed, e, step, (uint32_t)a + 1u);
       const uint32_t hr = hash_mix(base ^ HASH_TAG_REWARD) & 15u;
       const int r = hr == 0u ? 1 : (hr == 1u ? -1 : 0);
@@ -103,8 +144,16 @@ void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step
                      const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
                      uint8_t* terminals, int32_t* counters) {
   KernelScope scope(lc, KID_ENV_STEP);
-  launch_kernel(lc, env_step_kernel, n_e, ENV_THREADS, 0, seed, n_e, step_base, t, actions, term_denom, next_frames, rewards,
-                                                  terminals, counters);
+  launch_kernel(lc, env_step_kernel<false>, n_e, ENV_THREADS, 0, seed, n_e, step_base, t, actions, term_denom, next_frames, rewards,
+                                                  terminals, counters, HeadsTail{});
+}
+
+void launch_env_step_sampling(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step_base, uint32_t t, uint32_t term_denom,
+                              uint8_t* next_frames, int8_t* rewards, uint8_t* terminals, int32_t* counters,
+                              const HeadsTail& ht) {
+  KernelScope scope(lc, KID_ENV_STEP);
+  launch_kernel(lc, env_step_kernel<true>, n_e, ENV_THREADS, 0, seed, n_e, step_base, t, (const int32_t*)nullptr, term_denom,
+                next_frames, rewards, terminals, counters, ht);
 }
 
 // the environments' global step index lives on the device, so that a recorded sequence of launches can be

@@ -13,6 +13,17 @@ void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step
                      const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
                      uint8_t* terminals, int32_t* counters /* [3][n_e] */);
 
+// What is left of the heads after the cluster kernel of the fully connected layer: the two halves' dot products
+// hp[2][n_e][32], the head biases, and where logits, values, uniforms and actions go (see launch_heads_fused).
+struct HeadsTail {
+  const float* hp; const float* bpi; const float* bv; int A;
+  float* logits; float* values; const int32_t* forced; int32_t* actions; int32_t* sampled; float* uniforms;
+};
+// the same step with the action taken inside the kernel, from the heads' partial sums
+void launch_env_step_sampling(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step_base, uint32_t t, uint32_t term_denom,
+                              uint8_t* next_frames, int8_t* rewards, uint8_t* terminals, int32_t* counters,
+                              const HeadsTail& ht);
+
 void launch_advance_step(LaunchCtx& lc, uint64_t* step_base, uint32_t by);
 
 // ---- network on the CUDA cores (net_simt.cu) --------------------------------------------
