@@ -2014,12 +2014,22 @@ __global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments seg
 #pragma unroll
       for (int q = 0; q < 8; ++q) acc[q] = 0.f;
       const float* src = sg.part + (size_t)j0 * CO + co0 + lane;
-      for (int p = warp; p < sg.splits; p += 8) {
-        float v[8];
+      // four of this warp's splits at a time: 32 loads in flight per thread (a group is 150 KB for one block to
+      // pull in; with eight loads in flight its latency, not the bandwidth, set the pace); the additions keep
+      // their order
+      for (int p = warp; p < sg.splits; p += 32) {
+        float v[4][8];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) v[q] = (co_ok && j0 + q < J) ? __ldg(src + (size_t)p * total + (size_t)q * CO) : 0.f;
+        for (int u = 0; u < 4; ++u)
 #pragma unroll
-        for (int q = 0; q < 8; ++q) acc[q] += v[q];
+          for (int q = 0; q < 8; ++q)
+            v[u][q] = (co_ok && j0 + q < J && p + 8 * u < sg.splits) ? __ldg(src + (size_t)(p + 8 * u) * total + (size_t)q * CO) : 0.f;
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (p + 8 * u < sg.splits) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc[q] += v[u][q];
+          }
       }
 #pragma unroll
       for (int q = 0; q < 8; ++q) sh[(warp * 8 + q) * 33 + lane] = acc[q];
@@ -2350,12 +2360,14 @@ static void tc_shift_wgrad(LaunchCtx& lc, int kid, Cfg cfg, const bf16* g, int s
 // The right half sees every gradient row one position early, so tile t stands for positions 128 t - 1 .. 128 t + 126
 // and the tiles of all CTAs together cover -1 .. total: every (tap, position) pair is counted exactly once.
 // Raw frame rows arrive by bulk copy and are expanded to bf16 once per tile, as in the forward kernel.
-// Roles: warps 0-7 expand X (warps 0-3 also write the result at the end), warp 8 issues the MMAs, warp 9 fetches
-// frame rows, warps 10 and 19 add up the bias gradient from the staged gradient rows (half of the rows each), warps
-// 11-18 copy the gradient rows.
+// Roles, with E = W1_EXPAND_WARPS: warps 0 .. E-1 expand X (warps 0-3 also write the result at the end), warp E issues
+// the MMAs, warp E+1 fetches frame rows, warps E+2 and E+11 add up the bias gradient from the staged gradient rows
+// (half of the rows each), warps E+3 .. E+10 copy the gradient rows.  Role timers show the expansion busy three
+// quarters of the kernel (1200 cycles per tile against 400 for the tile's eight MMAs); sixteen expansion warps
+// were measured 8 % slower than eight: the role is bound by issue slots and shared-memory traffic, not by latency.
 // The kernel is bound by how many bytes an SM keeps in flight from DRAM, so the gradient rows and the frame rows
 // have rings of their own that run several tiles ahead of the expansion.
-constexpr int W1_THREADS = 640, W1_STAGES = 3, W1_G_SLOTS = 6, W1_G_AHEAD = 5, W1_X_ROWS = 152, W1_USED = 149,
+constexpr int W1_EXPAND_WARPS = 8, W1_THREADS = (W1_EXPAND_WARPS + 12) * 32, W1_STAGES = 3, W1_G_SLOTS = 6, W1_G_AHEAD = 5, W1_X_ROWS = 152, W1_USED = 149,
               W1_RAW_BYTES = 12288, W1_RAW_SLOTS = 5;
 
 struct W1Shared {
@@ -2370,7 +2382,8 @@ __global__ void __launch_bounds__(W1_THREADS, 1)
 tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ g, float* __restrict__ partial,
                       float* __restrict__ bias_partial, int n_states, int tiles, int tiles_per_cta, uint32_t* error_word) {
   static_assert(G::OH == 20 && G::OW == 20 && G::CO == 32 && G::K == 8 && G::C == 4 && G::S == 4, "geometry");
-  constexpr int POS = C1_RASTER * C1_RASTER, ROW_BYTES = G::W * G::C, NPROD = 256;
+  constexpr int POS = C1_RASTER * C1_RASTER, ROW_BYTES = G::W * G::C, E = W1_EXPAND_WARPS, NPROD = E * 32;
+  constexpr int STEP = NPROD / 4, ITEMS = (W1_USED + STEP - 1) / STEP;          // positions between a thread's items
   constexpr uint32_t X_BYTES = W1_X_ROWS * 128, G_BYTES = TC_BM * 128;
   extern __shared__ uint8_t dyn_smem[];
   __shared__ W1Shared sh;
@@ -2389,7 +2402,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
     sh.abort = 0u;
     fence_barrier_init();
   }
-  if (warp == 8) tmem_alloc(&sh.tmem_base, 64);
+  if (warp == E) tmem_alloc(&sh.tmem_base, 64);
   tcgen05_fence_before();
   __syncthreads();
   tcgen05_fence_after();
@@ -2406,7 +2419,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
     else { n0 = G::H - r0; n1 = 4 * (yl + 1); }
   };
 
-  if (warp < 8) {
+  if (warp < E) {
     // ---------------- producers ----------------
     const int p = threadIdx.x;
     for (int t = t0; t < t1; ++t) {
@@ -2420,7 +2433,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
       if (!__all_sync(0xffffffffu, ok)) break;
       const uint32_t raw = raw_base + slot * W1_RAW_BYTES;
       // X rows: work item = (position u of the tile, pixel row py of its block): 16 raw bytes -> two operand chunks;
-      // thread p takes items p, p + 256, p + 512: the same py, positions 64 apart (3 block rows + 1 block)
+      // thread p takes items p, p + NPROD, ...: the same py, positions STEP apart
       const int py = p & 3, u = p >> 2;
       int b, Y, X;
       {
@@ -2429,21 +2442,21 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
         const int rem = q - b * POS;
         Y = rem / C1_RASTER; X = rem - Y * C1_RASTER;
       }
-      uint4 rw[3];
+      uint4 rw[ITEMS];
 #pragma unroll
-      for (int k = 0; k < 3; ++k) {
+      for (int k = 0; k < ITEMS; ++k) {
         if (b >= n_states) { b = n_states - 1; Y = C1_RASTER - 1; X = C1_RASTER - 1; }     // past the end: repeat the last block
         const int slot_row = (b == b0 ? 4 * Y - r0 : n0 + 4 * Y) + py;
-        if (u + 64 * k < W1_USED)
+        if (u + STEP * k < W1_USED)
           asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(rw[k].x), "=r"(rw[k].y), "=r"(rw[k].z), "=r"(rw[k].w)
                        : "r"(raw + (uint32_t)(slot_row * ROW_BYTES + X * 16)) : "memory");
-        X += 1; Y += 3;
+        X += STEP % C1_RASTER; Y += STEP / C1_RASTER;
         if (X >= C1_RASTER) { X -= C1_RASTER; ++Y; }
         if (Y >= C1_RASTER) { Y -= C1_RASTER; ++b; }
       }
 #pragma unroll
-      for (int k = 0; k < 3; ++k) {
-        const uint32_t ri = (uint32_t)(u + 64 * k);
+      for (int k = 0; k < ITEMS; ++k) {
+        const uint32_t ri = (uint32_t)(u + STEP * k);
         if (ri < (uint32_t)W1_USED) {
           uint32_t o[8];
           u8x4_to_bf16x4(rw[k].x, o[0], o[1]); u8x4_to_bf16x4(rw[k].y, o[2], o[3]);
@@ -2476,7 +2489,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
                                __uint_as_float(r[4 * v + 3]));
       }
     }
-  } else if (warp == 8) {
+  } else if (warp == E) {
     if (lane == 0) {
       // ---------------- MMA issuer ----------------
       constexpr uint32_t idesc = make_idesc_bf16(TC_BM, 64, 1, 1);
@@ -2501,7 +2514,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
       }
       if (ok && t1 > t0) mma_commit(&sh.acc);
     }
-  } else if (warp == 9) {
+  } else if (warp == E + 1) {
     if (lane == 0) {
       // ---------------- raw loader ----------------
       for (int t = t0; t < t1; ++t) {
@@ -2517,10 +2530,10 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
                         &sh.raw_full[slot]);
       }
     }
-  } else if (warp >= 11 && warp < 19) {
+  } else if (warp >= E + 3 && warp < E + 11) {
     // ---------------- gradient rows: image row r = [G[m] | G[m + 1]], m = 128 t - 1 + r ----------------
     // thread p copies chunk p & 7 of rows (p >> 3) + 32 k, W1_G_AHEAD tiles ahead of the tile it publishes
-    const int p = threadIdx.x - 352, c8 = p & 7, half = c8 >> 2, chunk = c8 & 3;
+    const int p = threadIdx.x - (E + 3) * 32, c8 = p & 7, half = c8 >> 2, chunk = c8 & 3;
     int b1, Y, X;
     {
       const int mm = t0 * TC_BM - 1 + (p >> 3) + half + POS;       // one state further, so that position -1 is not negative
@@ -2574,7 +2587,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
     // lane l adds channels 8 (l & 3) .. 8 (l & 3) + 7 (one 16-byte chunk) over the rows (l >> 2) + 8 i, i of this warp's parity
     float acc[8] = {};
     bool ok = true;
-    const int q = lane & 3, rr = lane >> 2, which = warp == 10 ? 0 : 1;
+    const int q = lane & 3, rr = lane >> 2, which = warp == E + 2 ? 0 : 1;
     for (int t = t0; t < t1 && ok; ++t) {
       const int it = t - t0, gs = it % W1_G_SLOTS;
       ok = mbar_wait(&sh.g_full[gs], (it / W1_G_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
@@ -2610,7 +2623,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
   }
   tcgen05_fence_before();
   __syncthreads();
-  if (warp == 8) {
+  if (warp == E) {
     __syncwarp();
     tcgen05_fence_after();
     tmem_dealloc(tmem, 64);
