@@ -173,10 +173,13 @@ def test_tensor_core_path_matches_cuda_core_path(orc):
 
 
 def test_ragged_sizes_and_action_counts(orc):
-    """n_e that is no multiple of any tile, every action-set size of the configs."""
+    """n_e that is no multiple of any tile (below one tile, and one full 128-row tile plus a ragged tail on the
+    tensor-core path), every action-set size of the configs, the largest action set the cluster kernel of the fully
+    connected layer takes (31) and the one beyond it (32, which goes through the split-k kernel)."""
     for arch, prec, n_e, t_max, A in (("nips", "fp32", 5, 3, 18), ("nips", "bf16", 3, 2, 4),
                                       ("nature", "fp32", 7, 2, 6), ("nature", "bf16", 13, 1, 2),
-                                      ("nips", "fp32", 1, 1, 32)):
+                                      ("nips", "fp32", 1, 1, 32), ("nature", "bf16", 133, 2, 31),
+                                      ("nature", "bf16", 130, 1, 32)):
         cfg = dict(arch=arch, precision=prec, n_e=n_e, t_max=t_max, n_actions=A, lr=0.01, term_denom=3)
         o, g = make_pair(orc, cfg, seed=77)
         for it in range(2):
