@@ -2812,16 +2812,40 @@ void tc_heads_backward(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, co
 // From the canonical bf16 copy: wfc_t[i][o] = Wfc[o][i];  w3_d[ci][r][s][co] = W3[co][r][s][ci];
 // w2_d[z][ci][i][j][co] = W2[co][py + 2i][px + 2j][ci] with z = 2 py + px;
 // w1_b[co][2i + j][py][px][ci] = W1[co][4i + py][4j + px][ci] (the first layer's weights per 4 x 4 block tap).
-__global__ void relayout_weights_kernel(const bf16* __restrict__ w1, const bf16* __restrict__ w2,
+constexpr int RL_FC_TILES = (3136 / 64) * (512 / 64), RL_SMALL_BLOCKS = 76;
+__global__ void __launch_bounds__(256) relayout_weights_kernel(const bf16* __restrict__ w1, const bf16* __restrict__ w2,
                                         const bf16* __restrict__ w3, const bf16* __restrict__ wfc,
                                         bf16* __restrict__ w2_d, bf16* __restrict__ w3_d, bf16* __restrict__ wfc_t,
                                         bf16* __restrict__ w1_b) {
   pdl_entry();
   typedef NatConv2 C2; typedef NatConv3 C3;
   constexpr int N2 = 4 * C2::C * 4 * C2::CO, N3 = C3::C * 9 * C3::CO, NF = 3136 * 512, N1 = 32 * 256;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N2 + N3 + NF + N1; i += gridDim.x * blockDim.x) {
-    if (i >= N2 + N3 + NF) {
-      const int j = i - N2 - N3 - NF, ci = j & 3, px = (j >> 2) & 3, py = (j >> 4) & 3, tap = (j >> 6) & 3, co = j >> 8;
+  // Blocks 0 .. RL_FC_TILES - 1 transpose the fully connected matrix, the bulk of the work, one 64 x 64 tile each
+  // through shared memory, so that both sides are whole 128-byte rows; the other blocks gather the small images.
+  if (blockIdx.x < RL_FC_TILES) {
+    __shared__ uint16_t tile[64][66];                              // row pitch of 33 words: column reads spread over the banks
+    const int o0 = (blockIdx.x % 8) * 64, in0 = (blockIdx.x / 8) * 64;
+    const int r = threadIdx.x >> 2, c = threadIdx.x & 3;
+    {
+      const uint4* src = reinterpret_cast<const uint4*>(wfc + (size_t)(o0 + r) * 3136 + in0 + 16 * c);
+      const uint4 lo = __ldg(src), hi = __ldg(src + 1);
+      const uint32_t v[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+      for (int e = 0; e < 8; ++e) *reinterpret_cast<uint32_t*>(&tile[r][16 * c + 2 * e]) = v[e];
+    }
+    __syncthreads();
+    uint32_t v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+      v[e] = (uint32_t)tile[16 * c + 2 * e][r] | ((uint32_t)tile[16 * c + 2 * e + 1][r] << 16);
+    uint4* dst = reinterpret_cast<uint4*>(wfc_t + (size_t)(in0 + r) * 512 + o0 + 16 * c);
+    dst[0] = make_uint4(v[0], v[1], v[2], v[3]);
+    dst[1] = make_uint4(v[4], v[5], v[6], v[7]);
+    return;
+  }
+  for (int i = (blockIdx.x - RL_FC_TILES) * blockDim.x + threadIdx.x; i < N2 + N3 + N1; i += (gridDim.x - RL_FC_TILES) * blockDim.x) {
+    if (i >= N2 + N3) {
+      const int j = i - N2 - N3, ci = j & 3, px = (j >> 2) & 3, py = (j >> 4) & 3, tap = (j >> 6) & 3, co = j >> 8;
       const int r = 4 * (tap >> 1) + py, sx = 4 * (tap & 1) + px;
       w1_b[j] = w1[((co * 8 + r) * 8 + sx) * 4 + ci];
       continue;
@@ -2830,12 +2854,9 @@ __global__ void relayout_weights_kernel(const bf16* __restrict__ w1, const bf16*
       const int co = i % 64, t = (i / 64) % 4, ci = (i / 256) % 32, z = i / (256 * 32);
       const int r = (z >> 1) + 2 * (t >> 1), s = (z & 1) + 2 * (t & 1);
       w2_d[i] = w2[((co * 4 + r) * 4 + s) * 32 + ci];
-    } else if (i < N2 + N3) {
+    } else {
       const int j = i - N2, co = j % 64, tap = (j / 64) % 9, ci = j / 576;
       w3_d[j] = w3[(co * 9 + tap) * 64 + ci];
-    } else {
-      const int j = i - N2 - N3, o = j % 512, in = j / 512;
-      wfc_t[j] = wfc[(size_t)o * 3136 + in];
     }
   }
 }
@@ -2844,7 +2865,7 @@ size_t tc_weight_image_elems() { return TC_IMG_END; }
 void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, bf16* images) {
   const LayerDims* d = nd.layer;
   KernelScope scope(lc, KID_CAST);
-  launch_kernel(lc, relayout_weights_kernel, 592, 256, 0, theta16 + d[0].w_off, theta16 + d[1].w_off, theta16 + d[2].w_off,
+  launch_kernel(lc, relayout_weights_kernel, RL_FC_TILES + RL_SMALL_BLOCKS, 256, 0, theta16 + d[0].w_off, theta16 + d[1].w_off, theta16 + d[2].w_off,
                                                   theta16 + d[3].w_off, images + TC_IMG_W2, images + TC_IMG_W3,
                                                   images + TC_IMG_WFC, images + TC_IMG_W1);
 }
