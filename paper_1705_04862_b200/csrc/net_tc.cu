@@ -1992,9 +1992,10 @@ __global__ void tc_bias_final_kernel(const float* __restrict__ part, int blocks,
 // its bias with J = 1) dst[co * J + j] = scale * sum over splits of part[split][j][co], the splits added in a
 // fixed order.  The partial sums have co innermost and the gradient has j innermost, so every group of outputs
 // goes through a shared-memory tile: reads are whole 128-byte rows of co, writes whole runs of j.
-//   many splits: a group is 8 j x 32 co; warp w adds the splits w, w + 8, ... for all eight j (eight loads in
-//                flight per thread), the eight warps' sums are then added in warp order;
+//   many splits: a group is FG_J j x 32 co; warp w adds the splits w, w + 8, ... for these j, the eight warps' sums
+//                are then added in warp order;
 //   few splits:  a group is 32 j x 32 co; warp w adds all splits, in order, for rows w, w + 8, w + 16, w + 24.
+constexpr int FG_J = 2;          // rows of j per group of a many-split segment
 __global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments segs, float* __restrict__ sumsq_partials) {
   pdl_entry();
   __shared__ float sh[8 * 8 * 33];
@@ -2009,36 +2010,37 @@ __global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments seg
     const size_t total = (size_t)J * CO;
     const bool co_ok = co0 + lane < CO;
     if (sg.wide) {
-      const int j0 = (local / co_tiles) * 8;
-      float acc[8];
+      // a group is FG_J j x 32 co: small, so that the many-split layers spread over all blocks of the grid; warp w
+      // adds the splits w, w + 8, ... with 32 loads in flight per thread (its latency, not the bandwidth, sets the
+      // pace of a group); the additions keep their order
+      constexpr int SPI = 32 / FG_J;                      // splits per iteration and warp
+      const int j0 = (local / co_tiles) * FG_J;
+      float acc[FG_J];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+      for (int q = 0; q < FG_J; ++q) acc[q] = 0.f;
       const float* src = sg.part + (size_t)j0 * CO + co0 + lane;
-      // four of this warp's splits at a time: 32 loads in flight per thread (a group is 150 KB for one block to
-      // pull in; with eight loads in flight its latency, not the bandwidth, set the pace); the additions keep
-      // their order
-      for (int p = warp; p < sg.splits; p += 32) {
-        float v[4][8];
+      for (int p = warp; p < sg.splits; p += 8 * SPI) {
+        float v[SPI][FG_J];
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < SPI; ++u)
 #pragma unroll
-          for (int q = 0; q < 8; ++q)
+          for (int q = 0; q < FG_J; ++q)
             v[u][q] = (co_ok && j0 + q < J && p + 8 * u < sg.splits) ? __ldg(src + (size_t)(p + 8 * u) * total + (size_t)q * CO) : 0.f;
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < SPI; ++u)
           if (p + 8 * u < sg.splits) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) acc[q] += v[u][q];
+            for (int q = 0; q < FG_J; ++q) acc[q] += v[u][q];
           }
       }
 #pragma unroll
-      for (int q = 0; q < 8; ++q) sh[(warp * 8 + q) * 33 + lane] = acc[q];
+      for (int q = 0; q < FG_J; ++q) sh[(warp * FG_J + q) * 33 + lane] = acc[q];
       __syncthreads();
-      {
-        const int c = threadIdx.x >> 3, q = threadIdx.x & 7;       // eight consecutive threads write 32 contiguous bytes
+      if (threadIdx.x < 32 * FG_J) {
+        const int c = threadIdx.x / FG_J, q = threadIdx.x % FG_J;   // consecutive threads write consecutive j
         float t = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) t += sh[(w * 8 + q) * 33 + c];
+        for (int w = 0; w < 8; ++w) t += sh[(w * FG_J + q) * 33 + c];
         if (co0 + c < CO && j0 + q < J) { const float v = t * sg.scale; sg.dst[(size_t)(co0 + c) * J + j0 + q] = v; ss = fmaf(v, v, ss); }
       }
       __syncthreads();
@@ -2088,7 +2090,7 @@ static void add_segment(GradSegments* segs, const float* part, float* dst, int s
   g.part = part; g.dst = dst; g.splits = splits; g.J = J; g.CO = CO; g.scale = scale;
   g.wide = splits > 8;
   g.first_group = segs->total_groups;
-  g.groups = ((J + (g.wide ? 8 : 32) - 1) / (g.wide ? 8 : 32)) * ((CO + 31) / 32);
+  g.groups = ((J + (g.wide ? FG_J : 32) - 1) / (g.wide ? FG_J : 32)) * ((CO + 31) / 32);
   segs->total_groups += g.groups;
 }
 
