@@ -1810,7 +1810,7 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
   const int kb0 = split * blocks_per_split, kb1 = min(num_blocks, kb0 + blocks_per_split);
   // The bias gradient sum_m G[m][co] rides along as one more row tile whose operand is constant: row j = 0
   // is all ones, the other rows zero.  Only the CTAs of the first row-tile group compute it.
-  constexpr uint32_t TMEM_COLS = (JT + 1) * BN <= 128 ? 128 : 256;
+  constexpr uint32_t TMEM_COLS = (JT + 1) * BN <= 128 ? 128 : ((JT + 1) * BN <= 256 ? 256 : 512);
   const bool do_bias = blockIdx.y == 0;
   const uint32_t ones_base = tiles + STAGES * STAGE_BYTES;
 
@@ -2660,7 +2660,7 @@ static size_t tc_layer_scratch_floats(int n, int layer) {
     case 0: return (size_t)SWG_MAX_SPLITS * (256 * 32 + 2 * 32);      // per CTA: the weight tile and two bias rows
     case 1: return (size_t)SWG_MAX_SPLITS * (512 * 64 + 64);
     case 2: return (size_t)SWG_MAX_SPLITS * (576 * 64 + 64);
-    default: return wg_scratch_floats(n, 3136, 512, 25 * 4);
+    default: return wg_scratch_floats(n, 3136, 512, 13 * 4);      // 256 x 128 tiles of the 3136 x 512 matrix
   }
 }
 static size_t tc_layer_scratch_offset(int n, int layer) {
@@ -2702,7 +2702,7 @@ void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, 
     tc_shift_wgrad<C3FwdCfg, GradCells<81, 9, 7, 7>, 5>(lc, KID_CONV3_WGRAD, C3FwdCfg{(const bf16*)act[1], n * 81}, g, n, n * 81,
                                                         gw, gb, sc, &segs, err);
   } else {
-    tc_wgrad<PlainSrc, GradSrc<64>, 1, 128, 6, 512>(lc, KID_FC_WGRAD, PlainSrc{(const bf16*)act[2], 3136, n},
+    tc_wgrad<PlainSrc, GradSrc<64>, 2, 128, 4, 512>(lc, KID_FC_WGRAD, PlainSrc{(const bf16*)act[2], 3136, n},
                                                     GradSrc<64>{g, 512, n}, n, 49, 1.f, gw, gb, sc, &segs, err);
   }
 }
