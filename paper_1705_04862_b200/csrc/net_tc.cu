@@ -1406,6 +1406,15 @@ static bool tc_fc_forward_cluster(LaunchCtx& lc, const bf16* a, const bf16* w, c
 // shared memory with cp.async (two tiles ahead); thread (row, half) then expands window rows
 // 4*half .. 4*half+3 of its output pixel to bf16 into the two K blocks it owns.  Integers 0..255 are exact in bf16: the bytes are
 // spliced into floats 2^23 + n, 2^23 is subtracted, and the upper halves of two results are packed.
+// The forward kernel of the first layer multiplies in fp16 instead: a byte n placed in the low half of a 16-bit word
+// IS the fp16 subnormal n * 2^-24, so the expansion is two byte permutations per four pixels and nothing else (the
+// logic pipe that runs them was the kernel's bound with the ten instructions of the bf16 route).  Its weights are the
+// bf16 weights times 2^8 as fp16 (exact down to 2^-25); the epilogue's scale carries the 2^16 / 255.
+__device__ __forceinline__ void u8x4_to_f16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
+  lo = __byte_perm(w, 0u, 0x4140);
+  hi = __byte_perm(w, 0u, 0x4342);
+}
+constexpr float C1_F16_WEIGHT_SCALE = 256.f, C1_F16_OUTPUT_SCALE = 16777216.f / C1_F16_WEIGHT_SCALE / 255.f;     // 2^24 / 2^8 / 255
 __device__ __forceinline__ void u8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
   const float f0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7440)) - 8388608.f;
   const float f1 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7441)) - 8388608.f;
@@ -1533,8 +1542,8 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
         const int uu = u + 64 * k;
         if (uu < C1_USED_POS) {
           uint32_t o[8];
-          u8x4_to_bf16x4(rw[k].x, o[0], o[1]); u8x4_to_bf16x4(rw[k].y, o[2], o[3]);
-          u8x4_to_bf16x4(rw[k].z, o[4], o[5]); u8x4_to_bf16x4(rw[k].w, o[6], o[7]);
+          u8x4_to_f16x4(rw[k].x, o[0], o[1]); u8x4_to_f16x4(rw[k].y, o[2], o[3]);
+          u8x4_to_f16x4(rw[k].z, o[4], o[5]); u8x4_to_f16x4(rw[k].w, o[6], o[7]);
           const uint32_t ri = (uint32_t)(uu >> 1), dst = stage + (uu & 1) * PLANE_BYTES + ri * 128u;
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py) ^ (ri & 7)) << 4)),
                        "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
@@ -1566,7 +1575,7 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
   } else if (warp == 16) {
     if (lane == 0) {
       // ---------------- MMA issuer ----------------
-      constexpr uint32_t idesc = make_idesc_bf16(TC_BM, BN, 0, 0);
+      constexpr uint32_t idesc = make_idesc_f16(TC_BM, BN);        // fp16 operands (see u8x4_to_f16x4)
       const uint32_t hi = desc_hi_kmajor_sw128(), b_lo = (b_base >> 4) & 0x3FFFu;
       int local = 0;
       bool ok = true;
@@ -1728,12 +1737,11 @@ bool tc_supported(int arch, int prec) { return arch == PAAC_ARCH_NATURE && prec 
 void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const bf16* w, const bf16* images,
                 const uint8_t* frames, int n, void* const act[], float* fc_scratch, uint32_t* err, int* fc_splits) {
   const LayerDims* d = nd.layer;
-  const float s255 = 1.0f / 255.0f;
   if (arch != PAAC_ARCH_NATURE) return;   // the caller routes the smaller network to the CUDA-core path
   {
     typedef NatConv1 C1; typedef NatConv2 C2; typedef NatConv3 C3;
     const int M1 = n * C1::OH * C1::OW, M2 = n * C2::OH * C2::OW, M3 = n * C3::OH * C3::OW;
-    tc_conv1<C1, BiasReluEpiTc>(lc, frames, images + TC_IMG_W1, BiasReluEpiTc{(bf16*)act[0], theta + d[0].b_off, 32, s255, M1},
+    tc_conv1<C1, BiasReluEpiTc>(lc, frames, images + TC_IMG_W1, BiasReluEpiTc{(bf16*)act[0], theta + d[0].b_off, 32, C1_F16_OUTPUT_SCALE, M1},
                                 n, err);
     {
       typedef RasterMap<100, 10, 9, 9> Map;
@@ -2849,7 +2857,8 @@ __global__ void __launch_bounds__(256) relayout_weights_kernel(const bf16* __res
     if (i >= N2 + N3) {
       const int j = i - N2 - N3, ci = j & 3, px = (j >> 2) & 3, py = (j >> 4) & 3, tap = (j >> 6) & 3, co = j >> 8;
       const int r = 4 * (tap >> 1) + py, sx = 4 * (tap & 1) + px;
-      w1_b[j] = w1[((co * 8 + r) * 8 + sx) * 4 + ci];
+      // the forward kernel's copy of the first layer is fp16, scaled by 2^8 (see u8x4_to_f16x4)
+      reinterpret_cast<__half*>(w1_b)[j] = __float2half_rn(__bfloat162float(w1[((co * 8 + r) * 8 + sx) * 4 + ci]) * C1_F16_WEIGHT_SCALE);
       continue;
     }
     if (i < N2) {
