@@ -1511,12 +1511,10 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
       const int s = local % STAGES, slot = local % C1_RAW_SLOTS;
       int b0, r0, n0, n1;
       tile_ranges(t, b0, r0, n0, n1);
-      bool ok = mbar_wait(&sh.raw_full[slot], (local / C1_RAW_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
-      ok = ok && mbar_wait(&sh.empty[s], ((local / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
-      if (!__all_sync(0xffffffffu, ok)) break;
       const uint32_t stage = a_base0 + s * A_BYTES, raw = raw_base + slot * C1_RAW_BYTES;
       // work item = (position u of the tile, pixel row py of its block): 16 raw bytes -> two operand chunks;
-      // thread p takes items p, p + 256, ...: the same py, positions 64 apart (3 block rows + 1 block)
+      // thread p takes items p, p + 256, ...: the same py, positions 64 apart (3 block rows + 1 block).
+      // Where the items sit in the raw slot is worked out before the waits, whose idle time hides the arithmetic.
       const int py = p & 3;
       int u = p >> 2, b, Y, X;
       {
@@ -1525,18 +1523,25 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
         const int rem = q - b * POS;
         Y = rem / C1_RASTER; X = rem - Y * C1_RASTER;
       }
-      uint4 rw[5];
+      uint32_t src[5];
 #pragma unroll
       for (int k = 0; k < 5; ++k) {
         if (b >= n_states) { b = n_states - 1; Y = C1_RASTER - 1; X = C1_RASTER - 1; }     // past the end: repeat the last block
         const int slot_row = (b == b0 ? 4 * Y - r0 : n0 + 4 * Y) + py;
-        if (u + 64 * k < C1_USED_POS)
-          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(rw[k].x), "=r"(rw[k].y), "=r"(rw[k].z), "=r"(rw[k].w)
-                       : "r"(raw + (uint32_t)(slot_row * ROW_BYTES + X * 16)) : "memory");
+        src[k] = raw + (uint32_t)(slot_row * ROW_BYTES + X * 16);
         X += 1; Y += 3;
         if (X >= C1_RASTER) { X -= C1_RASTER; ++Y; }
         if (Y >= C1_RASTER) { Y -= C1_RASTER; ++b; }
       }
+      bool ok = mbar_wait(&sh.raw_full[slot], (local / C1_RAW_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      ok = ok && mbar_wait(&sh.empty[s], ((local / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      uint4 rw[5];
+#pragma unroll
+      for (int k = 0; k < 5; ++k)
+        if (u + 64 * k < C1_USED_POS)
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(rw[k].x), "=r"(rw[k].y), "=r"(rw[k].z), "=r"(rw[k].w)
+                       : "r"(src[k]) : "memory");
 #pragma unroll
       for (int k = 0; k < 5; ++k) {
         const int uu = u + 64 * k;
