@@ -1581,6 +1581,7 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
     if (lane == 0) {
       // ---------------- MMA issuer ----------------
       constexpr uint32_t idesc = make_idesc_f16(TC_BM, BN);        // fp16 operands (see u8x4_to_f16x4)
+      constexpr uint32_t idesc32 = make_idesc_f16(TC_BM, 32);
       const uint32_t hi = desc_hi_kmajor_sw128(), b_lo = (b_base >> 4) & 0x3FFFu;
       int local = 0;
       bool ok = true;
@@ -1593,14 +1594,22 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
         tcgen05_fence_after();
         const uint32_t a_lo = ((a_base0 + s * A_BYTES) >> 4) & 0x3FFFu, d = tmem + ab * BN;
 #pragma unroll
-        for (int v = 0; v < 6; ++v) {
-          // view v: plane (E = 0, O = 1), rows down, first weight block of its 64-row window
-          constexpr int plane[6] = {0, 1, 0, 1, 0, 1}, shift[6] = {0, 0, 1, 10, 11, 11}, wblk[6] = {2, 1, 0, 6, 5, 4};
+        for (int i = 0; i < 6; ++i) {
+          // view v: plane (E = 0, O = 1), rows down, and what it is multiplied with.  The two views that feed both
+          // positions of a row take a 64-row window of a block sequence (first block given); the four that feed one
+          // position take the 32 rows of their tap alone and go to that position's half of the accumulator: a 32-column
+          // MMA fetches a kilobyte less than a 64-column one whose other half is zeros.  A 64-column view comes
+          // first, so that it can initialise the whole accumulator.
+          constexpr int order[6] = {1, 0, 2, 3, 4, 5};
+          constexpr int plane[6] = {0, 1, 0, 1, 0, 1}, shift[6] = {0, 0, 1, 10, 11, 11};
+          constexpr int wblk[6] = {2, 1, 1, 6, 5, 5}, dcol[6] = {0, 0, 32, 0, 0, 32};
+          constexpr bool wide[6] = {false, true, false, false, true, false};
+          const int v = order[i];
           const uint32_t a_off = (plane[v] * PLANE_BYTES + shift[v] * 128u) >> 4, b_off = (wblk[v] * W_BLOCK) >> 4;
 #pragma unroll
           for (int k = 0; k < TC_BK / 16; ++k) {
-            if (v == 0 && k == 0) mma_bf16_lo<false>(d, a_lo + a_off, b_lo + b_off, hi, idesc);
-            else mma_bf16_lo<true>(d, a_lo + a_off + k * 2, b_lo + b_off + k * 2, hi, idesc);
+            if (i == 0 && k == 0) mma_bf16_lo<false>(d, a_lo + a_off, b_lo + b_off, hi, idesc);
+            else mma_bf16_lo<true>(d + dcol[v], a_lo + a_off + k * 2, b_lo + b_off + k * 2, hi, wide[v] ? idesc : idesc32);
           }
         }
         mma_commit(&sh.empty[s]);
