@@ -1562,11 +1562,39 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
     }
   } else if (warp < 8) {
     // ---------------- epilogue ----------------
+    // Two phases, so that a store instruction covers eight positions (64 bytes each) instead of thirty-two sixteen-
+    // byte pieces of thirty-two different lines: lane = accumulator row turns its 32 channels into bf16 and parks them
+    // in the warp's staging tile (32 rows of 64 bytes, chunks swizzled by row pair); then four lanes cover a row.
+    // The load / store pipe, which the expansion shares, was what every role of this kernel was waiting for.
     const int quarter = warp & 3, h = warp >> 2;
+    const uint32_t stg = raw_base + C1_RAW_SLOTS * C1_RAW_BYTES + warp * 2048;
+    const int ch = lane & 3, rr0 = lane >> 2;
+    const float4 bq0 = __ldg(reinterpret_cast<const float4*>(epi.bias) + 0), bq1 = __ldg(reinterpret_cast<const float4*>(epi.bias) + 1);
+    const float4 bq2 = __ldg(reinterpret_cast<const float4*>(epi.bias) + 2), bq3 = __ldg(reinterpret_cast<const float4*>(epi.bias) + 3);
+    const float4 bq4 = __ldg(reinterpret_cast<const float4*>(epi.bias) + 4), bq5 = __ldg(reinterpret_cast<const float4*>(epi.bias) + 5);
+    const float4 bq6 = __ldg(reinterpret_cast<const float4*>(epi.bias) + 6), bq7 = __ldg(reinterpret_cast<const float4*>(epi.bias) + 7);
+    const float bias_r[32] = {bq0.x, bq0.y, bq0.z, bq0.w, bq1.x, bq1.y, bq1.z, bq1.w, bq2.x, bq2.y, bq2.z, bq2.w, bq3.x, bq3.y, bq3.z, bq3.w,
+                              bq4.x, bq4.y, bq4.z, bq4.w, bq5.x, bq5.y, bq5.z, bq5.w, bq6.x, bq6.y, bq6.z, bq6.w, bq7.x, bq7.y, bq7.z, bq7.w};
     int local = 0;
     for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
-      const int ab = local & 1, pos = t * C1_TILE_POS + 2 * (quarter * 32 + lane) + h;
-      const int b = pos / POS, rem = pos % POS, Y = rem / C1_RASTER, X = rem % C1_RASTER;
+      const int ab = local & 1;
+      // where the four rows this lane writes in the second phase go (rows rr0, rr0 + 8, ...: positions 16 apart)
+      uint32_t out_at[4];
+      uint32_t valid = 0;
+      {
+        const int pos = t * C1_TILE_POS + 2 * (quarter * 32 + rr0) + h;
+        int b = pos / POS;
+        const int rem = pos - b * POS;
+        int Y = rem / C1_RASTER, X = rem - Y * C1_RASTER;
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+          if (b < n_states && Y < G::OH && X < G::OW) valid |= 1u << p;
+          out_at[p] = (uint32_t)(((b * G::OH + Y) * G::OW + X) * 32 + ch * 8);
+          X += 16;
+          if (X >= C1_RASTER) { X -= C1_RASTER; ++Y; }
+          if (Y >= C1_RASTER) { Y -= C1_RASTER; ++b; }
+        }
+      }
       const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
@@ -1575,7 +1603,28 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
       tcgen05_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
-      if (b < n_states && Y < G::OH && X < G::OW) epi((b * G::OH + Y) * G::OW + X, 0, 0, r);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float a0 = fmaxf(fmaf(__uint_as_float(r[8 * q + 2 * j]), epi.scale, bias_r[8 * q + 2 * j]), 0.f);
+          const float a1 = fmaxf(fmaf(__uint_as_float(r[8 * q + 2 * j + 1]), epi.scale, bias_r[8 * q + 2 * j + 1]), 0.f);
+          o[j] = pack_bf16x2(a0, a1);
+        }
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 64 + ((uint32_t)(q ^ ((lane >> 1) & 3)) << 4)),
+                     "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+      }
+      __syncwarp();
+#pragma unroll
+      for (int p = 0; p < 4; ++p) {
+        const int rr = p * 8 + rr0;
+        uint4 v;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                     : "r"(stg + rr * 64 + ((uint32_t)(ch ^ ((rr >> 1) & 3)) << 4)) : "memory");
+        if ((valid >> p) & 1u) *reinterpret_cast<uint4*>(epi.out + out_at[p]) = v;
+      }
+      __syncwarp();                                              // staging tile free for the next tile
     }
   } else if (warp == 16) {
     if (lane == 0) {
@@ -1692,7 +1741,7 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
 template <class G, class Epi>
 static void tc_conv1(LaunchCtx& lc, const uint8_t* frames, const bf16* w_blocks, Epi e, int n_states, uint32_t* err) {
   constexpr int STAGES = 3;
-  constexpr int smem = 8 * 32 * 128 + STAGES * 2 * C1_PLANE_ROWS * 128 + C1_RAW_SLOTS * C1_RAW_BYTES + 1024;
+  constexpr int smem = 8 * 32 * 128 + STAGES * 2 * C1_PLANE_ROWS * 128 + C1_RAW_SLOTS * C1_RAW_BYTES + 8 * 2048 + 1024;   // + staging tiles
   static_assert(smem <= 227 * 1024, "shared memory budget");
   auto kern = tc_conv1_kernel<G, Epi, STAGES>;
   static bool configured = false;
