@@ -174,6 +174,28 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float a, float b) {
   __nv_bfloat162 t = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&t);
 }
+// A warp's 32 rows x 32 floats (thread = row, registers = columns) go to the global rows dst0 + row * ld through a
+// 4 KB staging tile of the warp's own, so that every store instruction writes four whole 128-byte rows instead of
+// sixteen bytes of thirty-two different rows.  Bit `row` of row_mask says whether that row exists.
+__device__ __forceinline__ void warp_store_rows_f32(uint32_t stg, int lane, const uint32_t (&r)[32], float* dst0, size_t ld,
+                                                    uint32_t row_mask) {
+#pragma unroll
+  for (int q = 0; q < 8; ++q)
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + lane * 128 + ((uint32_t)(q ^ (lane & 7)) << 4)),
+                 "r"(r[4 * q]), "r"(r[4 * q + 1]), "r"(r[4 * q + 2]), "r"(r[4 * q + 3]) : "memory");
+  __syncwarp();
+  const int ch = lane & 7, rr0 = lane >> 3;
+#pragma unroll
+  for (int p = 0; p < 8; ++p) {
+    const int rr = p * 4 + rr0;
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(stg + rr * 128 + ((uint32_t)(ch ^ (rr & 7)) << 4)) : "memory");
+    if ((row_mask >> rr) & 1u) *reinterpret_cast<uint4*>(dst0 + (size_t)rr * ld + ch * 4) = v;
+  }
+  __syncwarp();
+}
+
 // out[m][n] = bf16(relu(acc * scale + bias[n]))
 struct BiasReluEpiTc {
   bf16* out; const float* bias; int ld; float scale; int M;
@@ -1966,12 +1988,11 @@ tc_wgrad_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant_
         for (int c = 0; c < BN / 32; ++c) {
           uint32_t r[32];
           tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + jt * BN + c * 32, r);
-          if (j < J && n0 + c * 32 < CO) {
-            float4* dst = reinterpret_cast<float4*>(partial + ((size_t)split * J + j) * CO + n0 + c * 32);
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-              dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
-                                   __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+          if (n0 + c * 32 < CO) {
+            const int j0 = j - lane;                              // this warp's rows j0 .. j0 + 31
+            const uint32_t rows = j0 + 32 <= J ? 0xFFFFFFFFu : (j0 < J ? (1u << (J - j0)) - 1u : 0u);
+            // the operand stages are idle by now (every MMA has completed): their memory serves as staging tiles
+            warp_store_rows_f32(tiles + warp * 4096, lane, r, partial + ((size_t)split * J + j0) * CO + n0 + c * 32, CO, rows);
           }
         }
       }
@@ -2317,14 +2338,13 @@ tc_shift_wgrad_kernel(Cfg cfg, const bf16* __restrict__ g, int states, float* __
       for (int p = 0; p < NP; ++p) {
         uint32_t r[32];
         tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + p * 64 + col0, r);
-        const int j = p * 128 + quarter * 32 + lane;
-        if (j < J) {
-          float4* dst = reinterpret_cast<float4*>(partial + ((size_t)split * J + j) * 64 + col0);
-#pragma unroll
-          for (int q = 0; q < 8; ++q)
-            dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
-                                 __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
-        }
+        const int j0 = p * 128 + quarter * 32;                   // this warp's rows j0 .. j0 + 31
+        const uint32_t rows = j0 + 32 <= J ? 0xFFFFFFFFu : (j0 < J ? (1u << (J - j0)) - 1u : 0u);
+        // Every MMA has completed, so the X parts of the operand stages are idle and serve as staging tiles (the G
+        // parts are not touched: the bias warp may still be reading the last ones).
+        static_assert(X_BYTES >= ((8 + STAGES - 1) / STAGES) * 4096, "room for the staging tiles");
+        warp_store_rows_f32(stage0 + (warp % STAGES) * STAGE_BYTES + (warp / STAGES) * 4096, lane, r,
+                            partial + ((size_t)split * J + j0) * 64 + col0, 64, rows);
       }
     }
   } else if (warp == 8) {
