@@ -139,7 +139,8 @@ void refresh_weight_copies(paac_ctx* c, bool cast) {
 // network + heads on the n_e states of `frames`, activations into slot `slot`.  With `tail` the caller is about
 // to step the synthetic environments and can take the actions there: if the forward pass left the heads as partial
 // sums (see HeadsTail), no sampling kernel is launched, *tail describes what is left, and the result is true.
-bool forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, HeadsTail* tail = nullptr) {
+bool forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, HeadsTail* tail = nullptr,
+                  bool* advanced = nullptr) {
   void* act[MAX_LAYERS];
   for (int l = 0; l <= c->nd.n_conv; ++l)
     act[l] = (char*)c->act[l] + (size_t)slot * c->n_e * c->nd.layer[l].out_size * c->elt;
@@ -159,7 +160,8 @@ bool forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, Hea
     }
     launch_heads_fused(c->lc, c->nd, c->theta, c->theta16, c->scratch, splits, (bf16*)act[c->nd.n_conv], c->n_e,
                        c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot, forced, actions,
-                       sampled, uniforms);
+                       sampled, uniforms, (advanced && splits == 0 && !sample) ? c->step_dev : nullptr, (uint32_t)c->t_max);
+    if (advanced) *advanced = splits == 0 && !sample;      // the sampling kernel has moved the step index on
     return false;
   }
   if (use_tc(c))
@@ -294,8 +296,9 @@ int paac_rollout(paac_ctx* c, paac_rollout_view* view) {
         launch_env_step(c->lc, c->seed, c->n_e, c->step_dev, (uint32_t)t, c->actions + row, c->hp.term_denom, dst,
                         c->rewards + row, c->terminals + row, c->counters);
     }
-    forward_slot(c, nxt, c->t_max, false);
-    launch_advance_step(c->lc, c->step_dev, (uint32_t)c->t_max);
+    bool advanced = false;
+    forward_slot(c, nxt, c->t_max, false, nullptr, &advanced);
+    if (!advanced) launch_advance_step(c->lc, c->step_dev, (uint32_t)c->t_max);
   });
   c->env_step += c->t_max;
   c->rollout_fresh = true;

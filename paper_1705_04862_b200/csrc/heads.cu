@@ -225,11 +225,14 @@ __global__ void __launch_bounds__(HS_WARPS * 32)
 heads_sample_kernel(const float* __restrict__ hp, const float* __restrict__ bpi, const float* __restrict__ bv, int n, int A,
                     float* __restrict__ logits, float* __restrict__ values, uint64_t seed,
                     const uint64_t* __restrict__ step_base, uint32_t t, const int32_t* __restrict__ forced,
-                    int32_t* __restrict__ actions, int32_t* __restrict__ sampled, float* __restrict__ uniforms) {
+                    int32_t* __restrict__ actions, int32_t* __restrict__ sampled, float* __restrict__ uniforms,
+                    uint64_t* advance_step, uint32_t advance_by) {
   const int lane = threadIdx.x & 31;
   const int e = blockIdx.x * HS_WARPS + (threadIdx.x >> 5);
   const float b = lane < A ? __ldg(bpi + lane) : (lane == A ? __ldg(bv) : 0.f);     // biases are older than the previous kernel
   pdl_entry();
+  // the last kernel of a rollout also moves the environments' step index on (nothing in this launch reads it then)
+  if (advance_step != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *advance_step += advance_by;
   if (e >= n) return;
   float s = -INFINITY;
   if (lane <= A) s = (hp[(size_t)e * HS_LD + lane] + hp[((size_t)n + e) * HS_LD + lane]) + b;
@@ -264,11 +267,12 @@ bool heads_fused_supported(const NetDims& nd) { return nd.F == 512 && nd.pi_w % 
 void launch_heads_fused(LaunchCtx& lc, const NetDims& nd, const float* theta, const bf16* theta16, const float* part,
                         int splits, bf16* h_out, int n, float* logits, float* values, uint64_t seed,
                         const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
-                        float* uniforms) {
+                        float* uniforms, uint64_t* advance_step, uint32_t advance_by) {
   KernelScope scope(lc, KID_HEADS_FWD);
   if (splits == 0) {          // `part` holds the head dot products of the two halves of the hidden units
     launch_kernel_overlapped(lc, heads_sample_kernel, (n + HS_WARPS - 1) / HS_WARPS, HS_WARPS * 32, 0, part, theta + nd.pi_b,
-                             theta + nd.v_b, n, nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms);
+                             theta + nd.v_b, n, nd.A, logits, values, seed, advance_step ? nullptr : step_base, t, forced,
+                             actions, sampled, uniforms, advance_step, advance_by);
     return;
   }
   launch_kernel(lc, heads_fused_kernel, (n + HF_WARPS - 1) / HF_WARPS, HF_WARPS * 32, 0, part, splits, theta + nd.layer[nd.n_conv].b_off, h_out,

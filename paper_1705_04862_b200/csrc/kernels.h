@@ -89,7 +89,9 @@ bool heads_fused_supported(const NetDims& nd);
 void launch_heads_fused(LaunchCtx& lc, const NetDims& nd, const float* theta, const bf16* theta16, const float* part,
                         int splits, bf16* h_out, int n, float* logits, float* values, uint64_t seed,
                         const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
-                        float* uniforms);
+                        float* uniforms, uint64_t* advance_step = nullptr, uint32_t advance_by = 0);
+// advance_step (only honoured with splits == 0, only valid without sampling): the kernel also adds advance_by to the
+// environments' step index, which saves the rollout its last launch
 // n-step returns and advantages, the loss gradient at the heads and the loss statistics, in one launch
 void launch_returns_head_grad(LaunchCtx& lc, int n_e, int t_max, int A, float gamma, float beta, float value_coef,
                               const int8_t* rewards, const uint8_t* terminals, const float* logits, const float* values,
