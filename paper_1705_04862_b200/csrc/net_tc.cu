@@ -2890,10 +2890,10 @@ void tc_heads_backward(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, co
   float* part_vw = part_b + (size_t)splits * A; float* part_vb = part_vw + (size_t)splits * 512;
   KernelScope scope(lc, KID_HEADS_BWD);
   if (A + 1 <= 8)
-    launch_kernel(lc, heads_backward_kernel<8>, splits, HB_THREADS, 0, h, dz, dV, theta16 + nd.pi_w, theta16 + nd.v_w, n, A,
+    launch_kernel_overlapped(lc, heads_backward_kernel<8>, splits, HB_THREADS, 0, h, dz, dV, theta16 + nd.pi_w, theta16 + nd.v_w, n, A,
                   rows_per, g_fc, part_w, part_b, part_vw, part_vb);
   else
-    launch_kernel(lc, heads_backward_kernel<20>, splits, HB_THREADS, 0, h, dz, dV, theta16 + nd.pi_w, theta16 + nd.v_w, n, A,
+    launch_kernel_overlapped(lc, heads_backward_kernel<20>, splits, HB_THREADS, 0, h, dz, dV, theta16 + nd.pi_w, theta16 + nd.v_w, n, A,
                   rows_per, g_fc, part_w, part_b, part_vw, part_vb);
   add_segment(segs, part_w, grad + nd.pi_w, splits, 1, 512 * A, 1.f);      // already in parameter order: a plain sum
   add_segment(segs, part_b, grad + nd.pi_b, splits, 1, A, 1.f);
