@@ -631,7 +631,8 @@ constexpr int SH_THREADS = 544;     // warps 0-7 epilogue, 8-15 producers, 16 MM
 // same result), so that an MMA does not have to wait for the one before it; the epilogue adds the NACC pieces.
 template <class Cfg, class Epi, int BN, int STAGES, int NACC>
 __global__ void __launch_bounds__(SH_THREADS, 1)
-tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_t* error_word) {
+tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles,
+                uint32_t* error_word) {
   static_assert(BN == 64 || BN == 128, "tile width");
   static_assert(2 * NACC * BN <= 512 && (NACC == 1 || NACC == 2 || NACC == 4), "tensor memory budget");
   static_assert(STAGES >= 2 && STAGES <= 8 && Cfg::STAGE_ROWS % 8 == 0, "pipeline shape");
@@ -644,7 +645,7 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 256); mbar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], Cfg::BULK ? 1 : 256); mbar_init(&sh.empty[s], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 8); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.mask_full[i], 256); mbar_init(&sh.mask_empty[i], 8); }
     sh.abort = 0u;
@@ -664,7 +665,21 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
   const uint32_t tmem = sh.tmem_base;
   pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
-  if (warp >= 8 && warp < 16) {
+  if (Cfg::BULK && warp >= 8 && warp < 16) {
+    // ---------------- producer: the rows of a stage are contiguous in memory, one tiled bulk copy brings them
+    // (128-byte swizzle; rows past the end of the tensor read as zeros) ----------------
+    static_assert(!Cfg::BULK || (!Epi::MASK && PLANES == 1), "bulk-copied stages: plain forward layers only");
+    if (warp == 8 && lane == 0) {
+      tma_prefetch_desc(&tm_a);
+      int it = 0;
+      for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
+        const int s = it % STAGES;
+        if (!mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY)) break;
+        mbar_arrive_expect_tx(&sh.full[s], STAGE_BYTES);
+        tma_load_2d(a_base0 + s * STAGE_BYTES, &tm_a, 0, t * TC_BM, &sh.full[s]);
+      }
+    }
+  } else if (warp >= 8 && warp < 16) {
     // ---------------- producers: eight lanes per 128-byte row, 32 rows per pass ----------------
     const int c = lane & 7, sub = (warp - 8) * 4 + (lane >> 3);
     int it = 0;
@@ -845,7 +860,10 @@ tc_shift_kernel(Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles, uint32_
 // conv3 forward: rows = the 9 x 9 x 64 input pixels in memory order; tap (r, s) is 9 r + s rows down
 struct C3FwdCfg {
   static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152, RASTER = 0;      // RASTER = 0: rows are plain memory order
+  static constexpr bool BULK = true;      // a stage is one contiguous run of 128-byte rows: one tiled bulk copy fetches it
   const bf16* x; int rows;                                   // rows = states * 81
+  const bf16* base_host() const { return x; }
+  int row_count() const { return rows; }
   __device__ __forceinline__ const bf16* base() const { return x; }
   __device__ __forceinline__ const bf16* src(int, int g, bool& valid) const {
     valid = g < rows;
@@ -859,6 +877,7 @@ struct C3FwdCfg {
 // lives in plane r & 1, 10 (r >> 1) + (pair offset) rows down, and tile rows run over a 10 x 10 raster
 struct C2FwdCfg {
   static constexpr int PLANES = 2, NT = 8, STAGE_ROWS = 144, RASTER = 0;
+  static constexpr bool BULK = false;
   const bf16* x; int states;
   __device__ __forceinline__ const bf16* base() const { return x; }
   __device__ __forceinline__ const bf16* src(int plane, int g, bool& valid) const {
@@ -873,6 +892,7 @@ struct C2FwdCfg {
 // raster position 11 y + x and tap (r, s) reads (2 - r) * 11 + (2 - s) rows down
 struct C3DgradCfg {
   static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152, RASTER = 121;
+  static constexpr bool BULK = false;
   const bf16* g3; int states;
   __device__ __forceinline__ const bf16* base() const { return g3; }
   // element offset of raster cell `rem` inside a state's 7 x 7 x 64 gradient, or -1 for a padding cell
@@ -892,6 +912,7 @@ struct C3DgradCfg {
 // raster; class pixel (yy, xx) is position 11 yy + xx and tap (i, j) reads (1 - i) * 11 + (1 - j) rows down
 struct C2DgradCfg {
   static constexpr int PLANES = 1, NT = 4, STAGE_ROWS = 144, RASTER = 121;
+  static constexpr bool BULK = false;
   const bf16* g2; int states;
   __device__ __forceinline__ const bf16* base() const { return g2; }
   __device__ static __forceinline__ int cell(int rem) {
@@ -1756,8 +1777,15 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
     configured = true;
   }
   const int tiles = (positions + TC_BM - 1) / TC_BM;
+  // bulk-copied stages: the layer input as a matrix of 128-byte rows, fetched in boxes of one stage
+  static CUtensorMap no_map;
+  const CUtensorMap* tm_a = &no_map;
+  if constexpr (Cfg::BULK) {
+    tm_a = tc_tensor_map(cfg.base_host(), (uint64_t)cfg.row_count(), 64, 64, Cfg::STAGE_ROWS);
+    if (tm_a == nullptr) { lc.host_failure = true; return; }      // no tensor-map encoder
+  }
   KernelScope scope(lc, kid);
-  launch_kernel_overlapped(lc, kern, tiles < sm_count() ? tiles : sm_count(), SH_THREADS, smem, cfg, w, e, tiles, err);
+  launch_kernel_overlapped(lc, kern, tiles < sm_count() ? tiles : sm_count(), SH_THREADS, smem, *tm_a, cfg, w, e, tiles, err);
 }
 
 template <class G, class Epi>
