@@ -69,6 +69,33 @@ static const CUtensorMap* tc_tensor_map(const bf16* x, uint64_t rows, uint64_t c
   return &maps[slot];
 }
 
+// map of a 3-D bf16 tensor x[d2][d1][64] (strides in bytes) for boxes of box2 x box1 rows of 128 bytes, 128-byte swizzle;
+// made afresh at every call (a handful of host instructions), nullptr if the encoder is unavailable
+static const CUtensorMap* tc_tensor_map3(CUtensorMap* out, const bf16* x, uint64_t d1, uint64_t d2, uint64_t stride1,
+                                         uint64_t stride2, uint32_t box1, uint32_t box2) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn encode = nullptr;
+  static bool looked_up = false;
+  if (!looked_up) {
+    looked_up = true;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      encode = (EncodeFn)fn;
+  }
+  if (encode == nullptr) return nullptr;
+  const cuuint64_t gdim[3] = {64, d1, d2}, gstride[2] = {stride1, stride2};
+  const cuuint32_t box[3] = {64u, box1, box2}, estride[3] = {1u, 1u, 1u};
+  if (encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(x), gdim, gstride, box, estride,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return nullptr;
+  return out;
+}
+
 struct TcShared {
   uint64_t full[8], empty[8], acc;
   uint32_t tmem_base;
@@ -631,7 +658,7 @@ constexpr int SH_THREADS = 544;     // warps 0-7 epilogue, 8-15 producers, 16 MM
 // same result), so that an MMA does not have to wait for the one before it; the epilogue adds the NACC pieces.
 template <class Cfg, class Epi, int BN, int STAGES, int NACC>
 __global__ void __launch_bounds__(SH_THREADS, 1)
-tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles,
+tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, Cfg cfg, const bf16* __restrict__ w, Epi epi, int tiles,
                 uint32_t* error_word) {
   static_assert(BN == 64 || BN == 128, "tile width");
   static_assert(2 * NACC * BN <= 512 && (NACC == 1 || NACC == 2 || NACC == 4), "tensor memory budget");
@@ -645,7 +672,7 @@ tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, Cfg cfg, const bf16* _
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], Cfg::BULK ? 1 : 256); mbar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], Cfg::BULK != 0 ? 1 : 256); mbar_init(&sh.empty[s], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 8); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.mask_full[i], 256); mbar_init(&sh.mask_empty[i], 8); }
     sh.abort = 0u;
@@ -665,18 +692,24 @@ tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, Cfg cfg, const bf16* _
   const uint32_t tmem = sh.tmem_base;
   pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
-  if (Cfg::BULK && warp >= 8 && warp < 16) {
-    // ---------------- producer: the rows of a stage are contiguous in memory, one tiled bulk copy brings them
+  if (Cfg::BULK != 0 && warp >= 8 && warp < 16) {
+    // ---------------- producer: a stage is one box of the layer input per plane, fetched by tiled bulk copies
     // (128-byte swizzle; rows past the end of the tensor read as zeros) ----------------
-    static_assert(!Cfg::BULK || (!Epi::MASK && PLANES == 1), "bulk-copied stages: plain forward layers only");
+    static_assert(Cfg::BULK == 0 || !Epi::MASK, "bulk-copied stages: plain forward layers only");
     if (warp == 8 && lane == 0) {
       tma_prefetch_desc(&tm_a);
+      if (Cfg::BULK == 2) tma_prefetch_desc(&tm_b);
       int it = 0;
       for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
         const int s = it % STAGES;
         if (!mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY)) break;
         mbar_arrive_expect_tx(&sh.full[s], STAGE_BYTES);
-        tma_load_2d(a_base0 + s * STAGE_BYTES, &tm_a, 0, t * TC_BM, &sh.full[s]);
+        if (Cfg::BULK == 1) {
+          tma_load_2d(a_base0 + s * STAGE_BYTES, &tm_a, 0, t * TC_BM, &sh.full[s]);
+        } else {
+          tma_load_3d(a_base0 + s * STAGE_BYTES, &tm_a, 0, 0, (t * TC_BM) / 10, &sh.full[s]);
+          tma_load_3d(a_base0 + s * STAGE_BYTES + PLANE_BYTES, &tm_b, 0, 0, (t * TC_BM) / 10, &sh.full[s]);
+        }
       }
     }
   } else if (warp >= 8 && warp < 16) {
@@ -829,7 +862,9 @@ tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, Cfg cfg, const bf16* _
       fence_proxy_async_smem();        // the copies observed through the barrier -> visible to the MMA's operand reads
       tcgen05_fence_after();
       // descriptor low words: (address >> 4); every operand slice is a compile-time offset from the stage
-      const uint32_t a_lo = ((a_base0 + s * STAGE_BYTES) >> 4) & 0x3FFFu, b_lo = (b_base >> 4) & 0x3FFFu;
+      // (with boxes that start at the tile's first oh, the tile's own rows begin a few rows into the stage)
+      const uint32_t row0 = Cfg::BULK == 2 ? (uint32_t)((t * TC_BM) % 10) : 0u;
+      const uint32_t a_lo = (((a_base0 + s * STAGE_BYTES) >> 4) & 0x3FFFu) + row0 * 8u, b_lo = (b_base >> 4) & 0x3FFFu;
       const uint32_t hi = desc_hi_kmajor_sw128(), d = tmem + ab * NACC * BN;
 #pragma unroll
       for (int tap = 0; tap < NT; ++tap) {
@@ -860,7 +895,7 @@ tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, Cfg cfg, const bf16* _
 // conv3 forward: rows = the 9 x 9 x 64 input pixels in memory order; tap (r, s) is 9 r + s rows down
 struct C3FwdCfg {
   static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152, RASTER = 0;      // RASTER = 0: rows are plain memory order
-  static constexpr bool BULK = true;      // a stage is one contiguous run of 128-byte rows: one tiled bulk copy fetches it
+  static constexpr int BULK = 1;          // a stage is one contiguous run of 128-byte rows: one tiled bulk copy fetches it
   const bf16* x; int rows;                                   // rows = states * 81
   const bf16* base_host() const { return x; }
   int row_count() const { return rows; }
@@ -876,9 +911,13 @@ struct C3FwdCfg {
 // order seen as [state][y][10 pairs]; even and odd image rows go to separate planes, so that tap row r
 // lives in plane r & 1, 10 (r >> 1) + (pair offset) rows down, and tile rows run over a 10 x 10 raster
 struct C2FwdCfg {
-  static constexpr int PLANES = 2, NT = 8, STAGE_ROWS = 144, RASTER = 0;
-  static constexpr bool BULK = false;
+  // A plane is the 3-D tensor [state * 10 + oh][10 pairs][64] (20 pair rows from one oh to the next), so a stage is one
+  // box of 16 x 10 rows per plane that starts at the tile's first oh; the tile's own rows begin (first position % 10)
+  // rows into it, which the MMA descriptors add.
+  static constexpr int PLANES = 2, NT = 8, STAGE_ROWS = 160, RASTER = 0;
+  static constexpr int BULK = 2;
   const bf16* x; int states;
+  const bf16* base_host() const { return x; }
   __device__ __forceinline__ const bf16* base() const { return x; }
   __device__ __forceinline__ const bf16* src(int plane, int g, bool& valid) const {
     // plane row g = (b, oh, X) is pair row 2 g - X + 10 plane of the input in memory order
@@ -892,7 +931,7 @@ struct C2FwdCfg {
 // raster position 11 y + x and tap (r, s) reads (2 - r) * 11 + (2 - s) rows down
 struct C3DgradCfg {
   static constexpr int PLANES = 1, NT = 9, STAGE_ROWS = 152, RASTER = 121;
-  static constexpr bool BULK = false;
+  static constexpr int BULK = 0;
   const bf16* g3; int states;
   __device__ __forceinline__ const bf16* base() const { return g3; }
   // element offset of raster cell `rem` inside a state's 7 x 7 x 64 gradient, or -1 for a padding cell
@@ -912,7 +951,7 @@ struct C3DgradCfg {
 // raster; class pixel (yy, xx) is position 11 yy + xx and tap (i, j) reads (1 - i) * 11 + (1 - j) rows down
 struct C2DgradCfg {
   static constexpr int PLANES = 1, NT = 4, STAGE_ROWS = 144, RASTER = 121;
-  static constexpr bool BULK = false;
+  static constexpr int BULK = 0;
   const bf16* g2; int states;
   __device__ __forceinline__ const bf16* base() const { return g2; }
   __device__ static __forceinline__ int cell(int rem) {
@@ -1779,13 +1818,19 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
   const int tiles = (positions + TC_BM - 1) / TC_BM;
   // bulk-copied stages: the layer input as a matrix of 128-byte rows, fetched in boxes of one stage
   static CUtensorMap no_map;
+  CUtensorMap plane_map[2];
   const CUtensorMap* tm_a = &no_map;
-  if constexpr (Cfg::BULK) {
+  const CUtensorMap* tm_b = &no_map;
+  if constexpr (Cfg::BULK == 1) {
     tm_a = tc_tensor_map(cfg.base_host(), (uint64_t)cfg.row_count(), 64, 64, Cfg::STAGE_ROWS);
-    if (tm_a == nullptr) { lc.host_failure = true; return; }      // no tensor-map encoder
+  } else if constexpr (Cfg::BULK == 2) {
+    // plane p: [states * 10][10 pairs][64], 2560 bytes from one oh to the next, starting 10 p pair rows in
+    tm_a = tc_tensor_map3(&plane_map[0], cfg.base_host(), 10, (uint64_t)cfg.states * 10, 128, 2560, 10, Cfg::STAGE_ROWS / 10);
+    tm_b = tc_tensor_map3(&plane_map[1], cfg.base_host() + 10 * 64, 10, (uint64_t)cfg.states * 10, 128, 2560, 10, Cfg::STAGE_ROWS / 10);
   }
+  if (tm_a == nullptr || tm_b == nullptr) { lc.host_failure = true; return; }      // no tensor-map encoder
   KernelScope scope(lc, kid);
-  launch_kernel_overlapped(lc, kern, tiles < sm_count() ? tiles : sm_count(), SH_THREADS, smem, *tm_a, cfg, w, e, tiles, err);
+  launch_kernel_overlapped(lc, kern, tiles < sm_count() ? tiles : sm_count(), SH_THREADS, smem, *tm_a, *tm_b, cfg, w, e, tiles, err);
 }
 
 template <class G, class Epi>
