@@ -70,9 +70,22 @@ static const CUtensorMap* tc_tensor_map(const bf16* x, uint64_t rows, uint64_t c
 }
 
 // map of a 3-D bf16 tensor x[d2][d1][64] (strides in bytes) for boxes of box2 x box1 rows of 128 bytes, 128-byte swizzle;
-// made afresh at every call (a handful of host instructions), nullptr if the encoder is unavailable
-static const CUtensorMap* tc_tensor_map3(CUtensorMap* out, const bf16* x, uint64_t d1, uint64_t d2, uint64_t stride1,
-                                         uint64_t stride2, uint32_t box1, uint32_t box2) {
+// cached by its defining values like the 2-D maps (a full cache is overwritten in turn: launches copy the map);
+// nullptr if the encoder is unavailable
+static const CUtensorMap* tc_tensor_map3(const bf16* x, uint64_t d1, uint64_t d2, uint64_t stride1, uint64_t stride2,
+                                         uint32_t box1, uint32_t box2) {
+  struct Key { const void* p; uint64_t d1, d2, s1, s2; uint32_t b1, b2; };
+  constexpr int MAX_MAPS = 32;
+  static Key keys[MAX_MAPS];
+  static CUtensorMap maps[MAX_MAPS];
+  static int n_maps = 0, next = 0;
+  for (int i = 0; i < n_maps; ++i)
+    if (keys[i].p == x && keys[i].d1 == d1 && keys[i].d2 == d2 && keys[i].s1 == stride1 && keys[i].s2 == stride2 &&
+        keys[i].b1 == box1 && keys[i].b2 == box2)
+      return &maps[i];
+  const int slot = n_maps < MAX_MAPS ? n_maps : next++ % MAX_MAPS;
+  CUtensorMap* out = &maps[slot];
+  keys[slot].p = nullptr;
   typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -93,6 +106,8 @@ static const CUtensorMap* tc_tensor_map3(CUtensorMap* out, const bf16* x, uint64
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return nullptr;
+  keys[slot] = Key{x, d1, d2, stride1, stride2, box1, box2};
+  if (n_maps < MAX_MAPS) ++n_maps;
   return out;
 }
 
@@ -1818,15 +1833,14 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
   const int tiles = (positions + TC_BM - 1) / TC_BM;
   // bulk-copied stages: the layer input as a matrix of 128-byte rows, fetched in boxes of one stage
   static CUtensorMap no_map;
-  CUtensorMap plane_map[2];
   const CUtensorMap* tm_a = &no_map;
   const CUtensorMap* tm_b = &no_map;
   if constexpr (Cfg::BULK == 1) {
     tm_a = tc_tensor_map(cfg.base_host(), (uint64_t)cfg.row_count(), 64, 64, Cfg::STAGE_ROWS);
   } else if constexpr (Cfg::BULK == 2) {
     // plane p: [states * 10][10 pairs][64], 2560 bytes from one oh to the next, starting 10 p pair rows in
-    tm_a = tc_tensor_map3(&plane_map[0], cfg.base_host(), 10, (uint64_t)cfg.states * 10, 128, 2560, 10, Cfg::STAGE_ROWS / 10);
-    tm_b = tc_tensor_map3(&plane_map[1], cfg.base_host() + 10 * 64, 10, (uint64_t)cfg.states * 10, 128, 2560, 10, Cfg::STAGE_ROWS / 10);
+    tm_a = tc_tensor_map3(cfg.base_host(), 10, (uint64_t)cfg.states * 10, 128, 2560, 10, Cfg::STAGE_ROWS / 10);
+    tm_b = tc_tensor_map3(cfg.base_host() + 10 * 64, 10, (uint64_t)cfg.states * 10, 128, 2560, 10, Cfg::STAGE_ROWS / 10);
   }
   if (tm_a == nullptr || tm_b == nullptr) { lc.host_failure = true; return; }      // no tensor-map encoder
   KernelScope scope(lc, kid);
