@@ -88,6 +88,9 @@ def check_rollout(orc, o, g, tol, lockstep=True):
 
 
 FLIP_L2 = 5e-2
+# how often check_update met ReLU flips (library updating from its own rollout): calls without injection, calls
+# that took the flip branch, and the largest number of flipped units seen in one call
+FLIP_STATS = {"calls": 0, "with_flips": 0, "max_flips": 0, "units_checked": 0}
 
 
 def check_update(orc, o, g, tol, check_acts=True, inject=False):
@@ -103,9 +106,12 @@ def check_update(orc, o, g, tol, check_acts=True, inject=False):
     a flip moves gradient elements below it by a whole term of their sums.  If no unit flipped,
     every tensor must meet the tolerance; if some did (they must be rare and sit at numerically
     zero activation), the activation gradients are compared where the masks agree and the
-    parameter gradients in the L2 sense against FLIP_L2, and the caller should re-synchronise.
+    parameter gradients in the L2 sense against FLIP_L2; the parameters must still meet
+    TOL_PARAMS_10 after the step, and the step and the RMSProp state agree in the L2 sense.
+    FLIP_STATS records how often this branch is taken.
     Returns (oracle update, library stats, report); report["flips"] counts flipped units."""
     L = o.net.n_conv
+    theta_before = o.theta.copy()
     up = o.update()
     if inject:
         for l in range(L + 1):
@@ -155,6 +161,32 @@ def check_update(orc, o, g, tol, check_acts=True, inject=False):
     assert abs(st["clip_scale"] - up["clip_scale"]) <= stat_tol
     rep.update(loose)
     rep["flips"] = flips
-    rep["theta"] = rel(g.params(), o.theta)
-    rep["rms"] = rel(g.debug_read(pb.DBG_RMS), o.m)
+    theta_g, rms_g = g.params(), g.debug_read(pb.DBG_RMS)
+    rep["theta"] = rel(theta_g, o.theta)
+    rep["rms"] = rel(rms_g, o.m)
+    if not inject:
+        FLIP_STATS["calls"] += 1
+        FLIP_STATS["units_checked"] += int(sum(a.size for a in acts_o))
+        if flips:
+            FLIP_STATS["with_flips"] += 1
+            FLIP_STATS["max_flips"] = max(FLIP_STATS["max_flips"], flips)
+    if flips:
+        # the flip branch still pins the optimiser: parameters within TOL_PARAMS_10, step and state in the L2 sense
+        assert rep["theta"] <= TOL_PARAMS_10, rep
+        ds = (theta_g.astype(np.float64) - theta_before) - (o.theta.astype(np.float64) - theta_before)
+        rep["step_l2"] = float(np.linalg.norm(ds) / (np.linalg.norm(o.theta.astype(np.float64) - theta_before) + 1e-30))
+        rep["rms_l2"] = float(np.linalg.norm(rms_g.astype(np.float64) - o.m) / (np.linalg.norm(o.m) + 1e-30))
+        assert rep["step_l2"] <= FLIP_L2 and rep["rms_l2"] <= 2 * FLIP_L2, rep
     return up, st, rep
+
+
+def adopt_library_state(o, g, updates):
+    """Continue the oracle from where a free-running library stands after `updates` updates: parameters, RMSProp
+    state, timestep counter, current states and episode counters are read from the library (integers and stored
+    floats, copied bit for bit); nothing the comparison that follows checks is taken from it."""
+    o.theta = g.params()
+    o.m = g.debug_read(pb.DBG_RMS).copy()
+    o.N = updates * o.n_e * o.t_max
+    o.state = g.debug_read(pb.DBG_NEXT_FRAMES).reshape(o.n_e, 84, 84, 4).copy()
+    for j, c in enumerate(g.debug_read(pb.DBG_COUNTERS).reshape(3, -1)):
+        o.counters[j][:] = c
