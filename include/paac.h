@@ -12,7 +12,10 @@
  *   - All functions return an int status (PAAC_OK = 0) unless stated; nothing is
  *     printed, nothing aborts.  paac_strerror() names a status.
  *   - "host" / "device" on a pointer says where the memory lives.
- *   - A context is not thread-safe.  Calls must follow init -> (rollout -> update)*.
+ *   - A context is not thread-safe, and the library keeps per-process caches (tensor maps, kernel
+ *     attributes) that are neither locked nor keyed by device: one calling thread and one device per
+ *     process (paac_init on a second device returns PAAC_ERR_STATE).  Calls must follow
+ *     init -> (rollout -> update)*.
  *   - Work is enqueued on the stream given at init; calls that return data to the
  *     host synchronise that stream, the others do not.
  *   - Indices: t in [0, t_max) is the step inside the current rollout, e in [0, n_e)
@@ -52,7 +55,9 @@ enum {
   PAAC_ERR_NONFINITE = 4,  /* gradient norm was inf/nan: the update was skipped */
   PAAC_ERR_TIMEOUT = 5,    /* a bounded device-side wait gave up */
   PAAC_ERR_STATE = 6,      /* call out of order (update without a fresh rollout, ...) */
-  PAAC_ERR_LIMIT = 7       /* size beyond the fixed capacity of an entry point that cannot allocate */
+  PAAC_ERR_LIMIT = 7,      /* size beyond the fixed capacity of an entry point that cannot allocate */
+  PAAC_ERR_RANGE = 8       /* a parameter lies outside the range a kernel's operand format can hold (see
+                              paac_set_params) */
 };
 
 /* Hyper-parameters.  paac_default_hparams() fills in the values of Section 5.1:
@@ -110,7 +115,7 @@ typedef struct {
   float entropy;       /* (1/B) sum H(pi(. | s_i)) */
   float grad_norm;     /* global L2 norm before clipping */
   float clip_scale;    /* factor applied to the gradient (1 when not clipped) */
-  int32_t status;      /* PAAC_OK or PAAC_ERR_NONFINITE */
+  int32_t status;      /* PAAC_OK, PAAC_ERR_NONFINITE, PAAC_ERR_TIMEOUT or PAAC_ERR_RANGE */
   uint64_t timesteps;  /* N after this update */
 } paac_update_stats;
 
@@ -119,7 +124,9 @@ typedef struct {
  * gradient of  -adv log pi - beta H + value_coef (R - V)^2  (Eqs. 9-10) through the
  * whole network, global-norm clipping, RMSProp, N += n_e * t_max.
  * stats == NULL: asynchronous.  stats != NULL: synchronises and fills it; returns
- * PAAC_ERR_NONFINITE if the update was skipped. */
+ * PAAC_ERR_NONFINITE if the update was skipped because the gradient norm was not finite, and
+ * PAAC_ERR_TIMEOUT / PAAC_ERR_RANGE if a kernel of this or an earlier call left a device error: the
+ * optimiser kernel itself checks the error word and then changes neither parameters nor RMSProp state. */
 int paac_update(paac_ctx* ctx, paac_update_stats* stats /* host, out, nullable */);
 
 size_t paac_param_count(const paac_ctx* ctx);
@@ -150,7 +157,14 @@ int paac_observe_host(paac_ctx* ctx, int t, const int8_t* rewards /* host */, co
 
 /* ---- test and resume hooks ---- */
 
-/* Overwrite the master parameters (and their bf16 copies) from the host. Synchronises. */
+/* Overwrite the master parameters (and their bf16 copies) from the host. Synchronises.
+ * Domain of the first layer in PAAC_BF16 on the Nature network: its forward kernel multiplies fp16 images (the
+ * bf16 weight times 2^8 against pixel values as fp16 subnormals), exact for 2^-25 <= |w| <= 255 after the bf16
+ * rounding; smaller magnitudes lose low bits (absolute error below 2^-26), larger ones cannot be held.  A vector
+ * with a first-layer weight whose bf16 value exceeds 255 in magnitude (or is not finite) is refused with
+ * PAAC_ERR_RANGE and nothing is changed.  Should training itself drive such a weight out of range, the update
+ * that finds it reports PAAC_ERR_RANGE and the following updates are skipped until the word is cleared
+ * (PAAC_DBG_ERROR_WORD). */
 int paac_set_params(paac_ctx* ctx, const float* src /* host */, size_t n);
 
 /* Actions to take instead of sampling in the following rollouts: host int32
@@ -177,6 +191,11 @@ enum {
   PAAC_DBG_GRAD,           /* f32 [P] gradient of the last update, before clipping */
   PAAC_DBG_RMS,            /* f32 [P] RMSProp state */
   PAAC_DBG_SAMPLED,        /* i32 [t_max][n_e]: the action inverse-CDF sampling gave, before any forcing */
+  PAAC_DBG_ERROR_WORD,     /* u32 [1]: sticky device error bits (1, 2, 4: a bounded wait gave up; 8: first-layer
+                              weight out of range).  While it is non-zero paac_update leaves parameters and
+                              optimiser state untouched and reports the error; a caller that has dealt with the
+                              cause (say, restored parameters with paac_set_params) clears it by writing 0.
+                              Reading it returns the word together with the status it stands for. */
   PAAC_DBG_ACT0 = 32,      /* T [B][...] stored activation of layer l = which - PAAC_DBG_ACT0
                               (conv layers, then fc) */
   PAAC_DBG_GACT0 = 48      /* T [B][...] gradient w.r.t. the pre-activation of layer l */
@@ -204,6 +223,13 @@ int paac_debug_write(paac_ctx* ctx, int which, const void* src /* host */, size_
  * process-wide.  Results are bit-identical either way. */
 enum { PAAC_OPT_CUDA_CORES_ONLY = 1, PAAC_OPT_TC_WGRAD_LAYERS = 2, PAAC_OPT_CUDA_GRAPHS = 3, PAAC_OPT_DEPENDENT_LAUNCH = 4 };
 int paac_set_option(paac_ctx* ctx, int option, int value);
+
+/* Failure-path check that cannot hang: launches one small kernel whose only thread block waits, at most
+ * max_polls polls (1 .. 1,000,000, a fraction of a second), on a barrier that nothing ever signals.  The wait
+ * runs out, the kernel records that in the context's error word exactly as the network kernels do, releases
+ * what it holds and returns; the call synchronises and returns PAAC_ERR_TIMEOUT.  The error word stays set
+ * (see PAAC_DBG_ERROR_WORD). */
+int paac_debug_wait_probe(paac_ctx* ctx, uint32_t max_polls);
 
 /* Number of kernels the library has launched on this context since init. */
 uint64_t paac_launch_count(const paac_ctx* ctx);

@@ -15,14 +15,15 @@ LIB_PATH = os.path.join(_HERE, "libpaac_b200.so")
 
 ARCH_NIPS, ARCH_NATURE = 0, 1
 FP32, BF16 = 0, 1
-OK, ERR_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_STATE, ERR_LIMIT = range(8)
+OK, ERR_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_STATE, ERR_LIMIT, ERR_RANGE = range(9)
 (DBG_FRAMES, DBG_NEXT_FRAMES, DBG_ACTIONS, DBG_REWARDS, DBG_TERMINALS, DBG_VALUES, DBG_LOGITS, DBG_UNIFORMS,
- DBG_COUNTERS, DBG_RETURNS, DBG_ADVANTAGES, DBG_DLOGITS, DBG_DVALUES, DBG_GRAD, DBG_RMS, DBG_SAMPLED) = range(16)
+ DBG_COUNTERS, DBG_RETURNS, DBG_ADVANTAGES, DBG_DLOGITS, DBG_DVALUES, DBG_GRAD, DBG_RMS, DBG_SAMPLED,
+ DBG_ERROR_WORD) = range(17)
 DBG_ACT0, DBG_GACT0 = 32, 48
 OPT_CUDA_CORES_ONLY, OPT_TC_WGRAD_LAYERS, OPT_CUDA_GRAPHS, OPT_DEPENDENT_LAUNCH = 1, 2, 3, 4
 
 _DBG_DTYPE = {DBG_FRAMES: np.uint8, DBG_NEXT_FRAMES: np.uint8, DBG_ACTIONS: np.int32, DBG_REWARDS: np.int8,
-              DBG_TERMINALS: np.uint8, DBG_COUNTERS: np.int32, DBG_SAMPLED: np.int32}
+              DBG_TERMINALS: np.uint8, DBG_COUNTERS: np.int32, DBG_SAMPLED: np.int32, DBG_ERROR_WORD: np.uint32}
 
 
 class HParams(C.Structure):
@@ -46,7 +47,7 @@ class UpdateStats(C.Structure):
 EXPORTS = ["paac_default_hparams", "paac_workspace_bytes", "paac_init", "paac_rollout", "paac_update",
            "paac_param_count", "paac_params", "paac_destroy", "paac_strerror", "paac_act_host",
            "paac_observe_host", "paac_set_params", "paac_force_actions", "paac_debug_bytes", "paac_debug_read",
-           "paac_debug_write", "paac_launch_count", "paac_profile", "paac_profile_read", "paac_set_option", "paac_clip_rmsprop_noalloc",
+           "paac_debug_write", "paac_debug_wait_probe", "paac_launch_count", "paac_profile", "paac_profile_read", "paac_set_option", "paac_clip_rmsprop_noalloc",
            "paac_noalloc_max_params"]
 
 _lib = None
@@ -82,6 +83,7 @@ def lib():
         L.paac_debug_bytes.restype = sz
         L.paac_debug_read.argtypes = [vp, i, vp, sz]
         L.paac_debug_write.argtypes = [vp, i, vp, sz]
+        L.paac_debug_wait_probe.argtypes = [vp, C.c_uint32]
         L.paac_launch_count.argtypes = [vp]
         L.paac_launch_count.restype = u64
         L.paac_profile.argtypes = [vp, i]
@@ -175,7 +177,7 @@ class Paac:
             _check(lib().paac_update(self._h, None))
             return None
         s = UpdateStats()
-        _check(lib().paac_update(self._h, C.byref(s)), allow=(ERR_NONFINITE,))
+        _check(lib().paac_update(self._h, C.byref(s)), allow=(ERR_NONFINITE, ERR_TIMEOUT, ERR_RANGE))
         return {n: getattr(s, n) for n, _ in UpdateStats._fields_}
 
     def params(self):
@@ -230,6 +232,19 @@ class Paac:
             assert not np.any(bits & 0xFFFF), "not bf16 values"
             arr = (bits >> 16).astype(np.uint16)
         self.debug_write(DBG_ACT0 + layer, arr)
+
+    def error_word(self):
+        """The sticky device error bits (0 when every kernel so far ran to the end)."""
+        w = np.zeros(1, np.uint32)
+        lib().paac_debug_read(self._h, DBG_ERROR_WORD, w.ctypes.data, 4)      # the status only repeats the word
+        return int(w[0])
+
+    def clear_error_word(self):
+        self.debug_write(DBG_ERROR_WORD, np.zeros(1, np.uint32))
+
+    def wait_probe(self, max_polls):
+        """Status of a wait that is made to run out (ERR_TIMEOUT when the device-side bound works)."""
+        return int(lib().paac_debug_wait_probe(self._h, max_polls))
 
     def launch_count(self):
         return int(lib().paac_launch_count(self._h))

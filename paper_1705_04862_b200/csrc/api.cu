@@ -45,6 +45,7 @@ struct paac_ctx {
   void* act[MAX_LAYERS];   // [(t_max+1)*n_e][out_size], slot t_max is bootstrap scratch
   void* gact[MAX_LAYERS];  // [B][out_size]
   float *logits, *values, *uniforms, *R, *adv, *dz, *dV, *loss_terms, *scratch, *norm_partials;
+  size_t simt_scratch_off; // floats: where the CUDA-core kernels' split-k scratch starts inside `scratch`
   int32_t *actions, *sampled, *forced, *counters;
   int8_t* rewards;
   uint8_t* terminals;
@@ -99,9 +100,15 @@ size_t carve(paac_ctx* c, char* base) {
   c->dV = k.take<float>(B);
   c->loss_terms = k.take<float>(3 * B);
   {
+    // the tensor-core weight gradients keep their partial sums until the finishing kernel has run, so a layer that
+    // is taken on the CUDA cores in the same update works in a region of its own behind them
     size_t sc = simt_scratch_floats(c->arch, nd, (int)B);
-    if (tc_supported(c->arch, c->prec) && tc_scratch_floats((int)B) > sc) sc = tc_scratch_floats((int)B);
-    if (tc_supported(c->arch, c->prec) && tc_fc_scratch_floats((int)n_e) > sc) sc = tc_fc_scratch_floats((int)n_e);
+    c->simt_scratch_off = 0;
+    if (tc_supported(c->arch, c->prec)) {
+      c->simt_scratch_off = (tc_scratch_floats((int)B) + 63) / 64 * 64;
+      sc += c->simt_scratch_off;
+      if (tc_fc_scratch_floats((int)n_e) > sc) sc = tc_fc_scratch_floats((int)n_e);
+    }
     c->scratch = k.take<float>(sc);
   }
   c->norm_partials = k.take<float>(NORM_BLOCKS);
@@ -133,7 +140,7 @@ bool use_tc(const paac_ctx* c) { return tc_supported(c->arch, c->prec) && !c->si
 // bf16 copies of the master parameters, in the canonical layout and regrouped for the backward kernels
 void refresh_weight_copies(paac_ctx* c, bool cast) {
   if (cast) launch_cast_bf16(c->lc, c->theta, c->theta16, c->nd.P);
-  if (tc_supported(c->arch, c->prec)) tc_relayout_weights(c->lc, c->nd, c->theta16, c->w_images);
+  if (tc_supported(c->arch, c->prec)) tc_relayout_weights(c->lc, c->nd, c->theta16, c->w_images, &c->stats->error_word);
 }
 
 // network + heads on the n_e states of `frames`, activations into slot `slot`.  With `tail` the caller is about
@@ -245,6 +252,10 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   if (!out || !valid_shape(arch, n_e, t_max, n_actions, hp)) return PAAC_ERR_ARG;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  // the per-process caches (tensor maps, kernel attributes, SM count) belong to the first device used
+  static int process_device = -1;
+  if (process_device < 0) process_device = dev;
+  if (dev != process_device) return PAAC_ERR_STATE;
   paac_ctx* c = new (std::nothrow) paac_ctx{};
   if (!c) return PAAC_ERR_CUDA;
   fill_shape(c, arch, n_e, t_max, n_actions, hp);
@@ -323,7 +334,7 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
                         c->scratch, &c->grad_segs);
     else
       heads_backward(c->lc, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
-                     c->grad, c->scratch);
+                     c->grad, c->scratch + c->simt_scratch_off);
     uint32_t* err = &c->stats->error_word;
     for (int l = L; l >= 0; --l) {
       // tensor-core kernels where they exist, the CUDA-core contraction otherwise
@@ -340,7 +351,7 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
       }
       if (!wgrad_done || (l > 0 && !dgrad_done))
         simt_backward_layer(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, c->frames[c->cur], c->B, c->act,
-                            c->gact, c->grad, c->scratch, l, !wgrad_done, l > 0 && !dgrad_done);
+                            c->gact, c->grad, c->scratch + c->simt_scratch_off, l, !wgrad_done, l > 0 && !dgrad_done);
     }
     // when every gradient goes through the finishing kernel, it also delivers the squared norm
     const bool all_finished = use_tc(c) && c->tc_wgrad_mask == 0xF && tc_heads_backward_supported(c->nd);
@@ -361,7 +372,7 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
     stats->policy_loss = ds.policy_loss; stats->value_loss = ds.value_loss; stats->entropy = ds.entropy;
     stats->grad_norm = ds.grad_norm; stats->clip_scale = ds.clip_scale; stats->status = ds.status;
     stats->timesteps = c->N;
-    if (ds.error_word) return PAAC_ERR_TIMEOUT;
+    if (ds.error_word) return status_of_error_word(ds.error_word);
     if (ds.status != PAAC_OK) return ds.status;
   }
   return PAAC_OK;
@@ -374,7 +385,7 @@ static int device_error(paac_ctx* c) {
   uint32_t w = 0;
   if (cudaMemcpyAsync(&w, &c->stats->error_word, sizeof(w), cudaMemcpyDeviceToHost, c->st) != cudaSuccess ||
       cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
-  return w ? PAAC_ERR_TIMEOUT : PAAC_OK;
+  return status_of_error_word(w);
 }
 
 int paac_params(paac_ctx* c, float* dst, size_t n) {
@@ -387,6 +398,19 @@ int paac_params(paac_ctx* c, float* dst, size_t n) {
 int paac_set_params(paac_ctx* c, const float* src, size_t n) {
   if (c) c->lc.serialize_next = true;
   if (!c || !src || n != c->nd.P) return PAAC_ERR_ARG;
+  if (tc_supported(c->arch, c->prec)) {
+    // the forward kernel of the first layer holds its weights as fp16(bf16(w) * 2^8): |bf16(w)| <= 255
+    const LayerDims& d = c->nd.layer[0];
+    const size_t count = (size_t)d.CO * d.K * d.K * d.C;
+    for (size_t i = 0; i < count; ++i) {
+      uint32_t u;
+      memcpy(&u, &src[d.w_off + i], 4);
+      u &= 0x7FFFFFFFu;
+      if (u >= 0x7F800000u) return PAAC_ERR_RANGE;                  // inf / nan
+      u += 0x7FFFu + ((u >> 16) & 1u);                              // round to nearest even at bit 16
+      if ((u >> 16) > 0x437Fu) return PAAC_ERR_RANGE;               // bf16 bits of 255.0
+    }
+  }
   if (cudaMemcpyAsync(c->theta, src, n * sizeof(float), cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
     cudaGetLastError(); return PAAC_ERR_CUDA;
   }
@@ -427,8 +451,17 @@ const char* paac_strerror(int s) {
     case PAAC_ERR_TIMEOUT: return "a bounded device-side wait gave up";
     case PAAC_ERR_STATE: return "call out of order";
     case PAAC_ERR_LIMIT: return "size beyond the fixed capacity of a non-allocating entry point";
+    case PAAC_ERR_RANGE: return "a parameter lies outside the range a kernel's operand format can hold";
     default: return "unknown status";
   }
+}
+
+int paac_debug_wait_probe(paac_ctx* c, uint32_t max_polls) {
+  if (c) c->lc.serialize_next = true;
+  if (!c || max_polls < 1u || max_polls > 1000000u) return PAAC_ERR_ARG;
+  launch_wait_probe(c->lc, max_polls, &c->stats->error_word);
+  if (cuda_status(c) != PAAC_OK) return PAAC_ERR_CUDA;
+  return device_error(c);
 }
 
 uint64_t paac_launch_count(const paac_ctx* c) { return c ? c->lc.count : 0; }
@@ -521,6 +554,7 @@ static void* debug_ptr(const paac_ctx* c, int which, size_t* bytes) {
     case PAAC_DBG_GRAD: *bytes = P * 4; return c->grad;
     case PAAC_DBG_RMS: *bytes = P * 4; return c->rms;
     case PAAC_DBG_SAMPLED: *bytes = B * 4; return c->sampled;
+    case PAAC_DBG_ERROR_WORD: *bytes = 4; return &c->stats->error_word;
     default: break;
   }
   if (which >= PAAC_DBG_ACT0 && which <= PAAC_DBG_ACT0 + c->nd.n_conv) {

@@ -225,6 +225,13 @@ inline cudaError_t launch_kernel_overlapped(LaunchCtx& lc, void (*kern)(KArgs...
   return launch_kernel_impl<true>(lc, kern, grid, block, smem, args...);
 }
 
+// bits of DeviceStats::error_word: 1, 2, 4 = a bounded wait gave up (which kind: see tc_common.cuh);
+// 8 = a first-layer weight does not fit the fp16 image the forward kernel multiplies with
+constexpr uint32_t DEV_ERR_WAIT_MASK = 7u, DEV_ERR_RANGE = 8u;
+inline int status_of_error_word(uint32_t w) {
+  return (w & DEV_ERR_WAIT_MASK) ? PAAC_ERR_TIMEOUT : ((w & DEV_ERR_RANGE) ? PAAC_ERR_RANGE : PAAC_OK);
+}
+
 // device-side statistics block written by the update kernels
 struct DeviceStats {
   float policy_loss, value_loss, entropy, grad_norm, clip_scale;

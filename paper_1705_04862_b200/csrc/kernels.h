@@ -51,7 +51,10 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
 // transposed / regrouped bf16 weight images the backward contractions read (refreshed after every
 // parameter change), and the data-gradient kernels that use them
 size_t tc_weight_image_elems();
-void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, bf16* images);
+// (a first-layer weight whose fp16 image would overflow raises DEV_ERR_RANGE in *error_word)
+void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, bf16* images, uint32_t* error_word);
+// one block waits at most max_polls polls on a barrier nobody signals, then records the time-out in *error_word
+void launch_wait_probe(LaunchCtx& lc, uint32_t max_polls, uint32_t* error_word);
 void tc_backward_dgrad_fc(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err);
 void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err);
 void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err);

@@ -2264,13 +2264,15 @@ __global__ void __launch_bounds__(256) tc_finalize_grads_kernel(GradSegments seg
   }
 }
 
-static void add_segment(GradSegments* segs, const float* part, float* dst, int splits, int J, int CO, float scale) {
+static bool add_segment(GradSegments* segs, const float* part, float* dst, int splits, int J, int CO, float scale) {
+  if (segs->n >= (int)(sizeof(segs->seg) / sizeof(segs->seg[0]))) return false;      // the caller reports a host failure
   GradSegment& g = segs->seg[segs->n++];
   g.part = part; g.dst = dst; g.splits = splits; g.J = J; g.CO = CO; g.scale = scale;
   g.wide = splits > 8;
   g.first_group = segs->total_groups;
   g.groups = ((J + (g.wide ? FG_J : 32) - 1) / (g.wide ? FG_J : 32)) * ((CO + 31) / 32);
   segs->total_groups += g.groups;
+  return true;
 }
 
 static int wg_splits(int num_blocks, int tiles_yz) {
@@ -2309,8 +2311,8 @@ static void tc_wgrad(LaunchCtx& lc, int kid, XSrc xs, GSrc gs, int rows, int n_a
   KernelScope scope(lc, kid);
   launch_kernel_overlapped(lc, kern, dim3(splits, gy, gz), TC_THREADS, smem, *tm_x, *tm_g, xs, gs, scratch, bias_part, n_atoms, J, CO,
                            num_blocks, bps, err);
-  add_segment(segs, scratch, gw, splits, J, CO, scale);
-  add_segment(segs, bias_part, gb, splits, 1, CO, 1.f);
+  if (!add_segment(segs, scratch, gw, splits, J, CO, scale) || !add_segment(segs, bias_part, gb, splits, 1, CO, 1.f))
+    lc.host_failure = true;
 }
 
 // ---- weight gradients of the middle convolutions without im2col ----------------------------------------------
@@ -2525,8 +2527,8 @@ static void tc_shift_wgrad(LaunchCtx& lc, int kid, Cfg cfg, const bf16* g, int s
   float* bias_part = scratch + (size_t)splits * J * 64;
   KernelScope scope(lc, kid);
   launch_kernel_overlapped(lc, kern, splits, SWG_THREADS, smem, cfg, g, states, scratch, bias_part, tiles, per, err);
-  add_segment(segs, scratch, gw, splits, J, 64, 1.f);
-  add_segment(segs, bias_part, gb, splits, 1, 64, 1.f);
+  if (!add_segment(segs, scratch, gw, splits, J, 64, 1.f) || !add_segment(segs, bias_part, gb, splits, 1, 64, 1.f))
+    lc.host_failure = true;
 }
 
 // ---- first layer, weight gradient: space-to-depth, all four block taps in one MMA ----------------------------
@@ -2828,8 +2830,9 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
   float* bias_part = scratch + (size_t)splits * 256 * 32;
   KernelScope scope(lc, KID_CONV1_WGRAD);
   launch_kernel_overlapped(lc, kern, splits, W1_THREADS, smem, frames, g, scratch, bias_part, n_states, tiles, per, err);
-  add_segment(segs, scratch, gw, splits, 256, 32, 1.0f / 255.0f);
-  add_segment(segs, bias_part, gb, 2 * splits, 1, 32, 1.f);      // two bias warps per CTA, a row each
+  if (!add_segment(segs, scratch, gw, splits, 256, 32, 1.0f / 255.0f) ||
+      !add_segment(segs, bias_part, gb, 2 * splits, 1, 32, 1.f))      // two bias warps per CTA, a row each
+    lc.host_failure = true;
 }
 
 // every layer keeps its own partial-sum region until the finishing kernel has run
@@ -2982,10 +2985,10 @@ void tc_heads_backward(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, co
   else
     launch_kernel_overlapped(lc, heads_backward_kernel<20>, splits, HB_THREADS, 0, h, dz, dV, theta16 + nd.pi_w, theta16 + nd.v_w, n, A,
                   rows_per, g_fc, part_w, part_b, part_vw, part_vb);
-  add_segment(segs, part_w, grad + nd.pi_w, splits, 1, 512 * A, 1.f);      // already in parameter order: a plain sum
-  add_segment(segs, part_b, grad + nd.pi_b, splits, 1, A, 1.f);
-  add_segment(segs, part_vw, grad + nd.v_w, splits, 1, 512, 1.f);
-  add_segment(segs, part_vb, grad + nd.v_b, splits, 1, 1, 1.f);
+  // already in parameter order: plain sums
+  if (!add_segment(segs, part_w, grad + nd.pi_w, splits, 1, 512 * A, 1.f) || !add_segment(segs, part_b, grad + nd.pi_b, splits, 1, A, 1.f) ||
+      !add_segment(segs, part_vw, grad + nd.v_w, splits, 1, 512, 1.f) || !add_segment(segs, part_vb, grad + nd.v_b, splits, 1, 1, 1.f))
+    lc.host_failure = true;
 }
 
 // ---- weight images for the backward contractions ------------------------------------------------------
@@ -2996,7 +2999,7 @@ constexpr int RL_FC_TILES = (3136 / 64) * (512 / 64), RL_SMALL_BLOCKS = 76;
 __global__ void __launch_bounds__(256) relayout_weights_kernel(const bf16* __restrict__ w1, const bf16* __restrict__ w2,
                                         const bf16* __restrict__ w3, const bf16* __restrict__ wfc,
                                         bf16* __restrict__ w2_d, bf16* __restrict__ w3_d, bf16* __restrict__ wfc_t,
-                                        bf16* __restrict__ w1_b) {
+                                        bf16* __restrict__ w1_b, uint32_t* __restrict__ error_word) {
   pdl_entry();
   typedef NatConv2 C2; typedef NatConv3 C3;
   constexpr int N2 = 4 * C2::C * 4 * C2::CO, N3 = C3::C * 9 * C3::CO, NF = 3136 * 512, N1 = 32 * 256;
@@ -3028,7 +3031,9 @@ __global__ void __launch_bounds__(256) relayout_weights_kernel(const bf16* __res
       const int j = i - N2 - N3, ci = j & 3, px = (j >> 2) & 3, py = (j >> 4) & 3, tap = (j >> 6) & 3, co = j >> 8;
       const int r = 4 * (tap >> 1) + py, sx = 4 * (tap & 1) + px;
       // the forward kernel's copy of the first layer is fp16, scaled by 2^8 (see u8x4_to_f16x4)
-      reinterpret_cast<__half*>(w1_b)[j] = __float2half_rn(__bfloat162float(w1[((co * 8 + r) * 8 + sx) * 4 + ci]) * C1_F16_WEIGHT_SCALE);
+      const float scaled = __bfloat162float(w1[((co * 8 + r) * 8 + sx) * 4 + ci]) * C1_F16_WEIGHT_SCALE;
+      if (!(fabsf(scaled) <= 65504.f)) atomicOr(error_word, DEV_ERR_RANGE);      // beyond fp16 (or not a number)
+      reinterpret_cast<__half*>(w1_b)[j] = __float2half_rn(scaled);
       continue;
     }
     if (i < N2) {
@@ -3043,12 +3048,27 @@ __global__ void __launch_bounds__(256) relayout_weights_kernel(const bf16* __res
 }
 size_t tc_weight_image_elems() { return TC_IMG_END; }
 
-void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, bf16* images) {
+void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, bf16* images, uint32_t* error_word) {
   const LayerDims* d = nd.layer;
   KernelScope scope(lc, KID_CAST);
   launch_kernel(lc, relayout_weights_kernel, RL_FC_TILES + RL_SMALL_BLOCKS, 256, 0, theta16 + d[0].w_off, theta16 + d[1].w_off, theta16 + d[2].w_off,
                                                   theta16 + d[3].w_off, images + TC_IMG_W2, images + TC_IMG_W3,
-                                                  images + TC_IMG_WFC, images + TC_IMG_W1);
+                                                  images + TC_IMG_WFC, images + TC_IMG_W1, error_word);
+}
+
+// ---- failure-path probe: a bounded wait that is made to run out ------------------------------------------------
+// One warp initialises a barrier that expects one arrival, nobody arrives, and every lane waits for its first
+// phase with the given poll limit: the wait gives up, the error bit is recorded, the block returns.
+__global__ void __launch_bounds__(32) wait_probe_kernel(uint32_t max_polls, uint32_t* error_word) {
+  __shared__ uint64_t bar;
+  __shared__ volatile uint32_t abort_flag;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); abort_flag = 0u; fence_barrier_init(); }
+  __syncwarp();
+  mbar_wait_limit(&bar, 0, &abort_flag, error_word, ERR_WAIT_FULL, max_polls);
+}
+void launch_wait_probe(LaunchCtx& lc, uint32_t max_polls, uint32_t* error_word) {
+  KernelScope scope(lc, KID_INIT);
+  launch_kernel(lc, wait_probe_kernel, 1, 32, 0, max_polls, error_word);
 }
 
 // ---- backward: data gradients ---------------------------------------------------------------------------

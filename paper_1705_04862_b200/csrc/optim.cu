@@ -35,7 +35,9 @@ sumsq_kernel(const float* __restrict__ g, size_t P, float* __restrict__ partials
 // pass 2: every block re-adds the partials in the same order (so all agree bit for bit),
 // forms scale = min(1, clip / norm) and applies
 //   m <- rho m + (1 - rho) (scale g)^2,  theta <- theta - lr (scale g) / sqrt(m + eps)
-// and refreshes the bf16 copy.  A non-finite norm leaves theta and m untouched.
+// and refreshes the bf16 copy.  A non-finite norm leaves theta and m untouched, and so does a device error
+// left by any earlier kernel (a bounded wait that gave up means some tile or partial sum of this update is
+// garbage): the status then names the error.
 __global__ void __launch_bounds__(OPT_THREADS)
 clip_rmsprop_kernel(size_t P, float* __restrict__ theta, float* __restrict__ rms, const float* __restrict__ g,
                     bf16* __restrict__ theta16, float lr, float rho, float eps, float clip,
@@ -63,13 +65,16 @@ clip_rmsprop_kernel(size_t P, float* __restrict__ theta, float* __restrict__ rms
     for (int w = 0; w < OPT_THREADS / 32; ++w) total += sh[w];
     const float norm = sqrtf(total);
     float scale = 1.f;
-    const bool ok = isfinite(norm);
+    const uint32_t dev_err = *reinterpret_cast<const volatile uint32_t*>(&stats->error_word);
+    const bool ok = isfinite(norm) && dev_err == 0u;
     if (ok && clip > 0.f && norm > clip) scale = clip / norm;
     s_scale = ok ? scale : -1.f;
     if (blockIdx.x == 0) {
       stats->grad_norm = norm;
       stats->clip_scale = ok ? scale : 0.f;
-      stats->status = ok ? PAAC_OK : PAAC_ERR_NONFINITE;
+      stats->status = ok ? PAAC_OK
+                         : ((dev_err & DEV_ERR_WAIT_MASK) ? PAAC_ERR_TIMEOUT
+                                                           : ((dev_err & DEV_ERR_RANGE) ? PAAC_ERR_RANGE : PAAC_ERR_NONFINITE));
     }
   }
   __syncthreads();

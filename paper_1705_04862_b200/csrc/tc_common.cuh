@@ -7,6 +7,8 @@ namespace paac {
 namespace tc {
 
 constexpr uint32_t ERR_WAIT_FULL = 1u, ERR_WAIT_EMPTY = 2u, ERR_WAIT_ACC = 4u;
+// the three bits above: a bounded wait gave up (PAAC_ERR_TIMEOUT)
+constexpr uint32_t ERR_WAIT_ANY = 7u;
 // A healthy wait ends within microseconds.  try_wait itself suspends the thread for a
 // hardware time slice, so this cap is of the order of a second before the kernel gives up.
 constexpr uint32_t WAIT_POLLS = 4000000u;
@@ -30,18 +32,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Waits for the phase with the given parity.  Gives up after WAIT_POLLS polls or as soon as
+// Waits for the phase with the given parity.  Gives up after `limit` polls or as soon as
 // another thread of the CTA has given up (*abort != 0): records `code` in *error_word, raises
 // *abort and returns false; the caller then leaves its loop and goes to the common tear-down.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort,
-                                          uint32_t* error_word, uint32_t code) {
-  for (uint32_t i = 0; i < WAIT_POLLS; ++i) {
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, volatile uint32_t* abort,
+                                                uint32_t* error_word, uint32_t code, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023u) == 1023u && *abort) return false;
   }
   *abort = 1u;
   atomicOr(error_word, code);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort,
+                                          uint32_t* error_word, uint32_t code) {
+  return mbar_wait_limit(bar, parity, abort, error_word, code, WAIT_POLLS);
 }
 
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }

@@ -295,3 +295,74 @@ def test_external_environment_mode_matches_device_environment(orc):
     assert np.array_equal(g2.params(), g.params())
     g.close()
     g2.close()
+
+
+def test_bounded_wait_gives_up_and_the_update_is_skipped(orc):
+    """A wait on a barrier nobody signals runs out after its poll limit: the kernel returns, the error word is set,
+    the call reports ERR_TIMEOUT, and the context stays usable.  While the word is set an update changes neither
+    parameters nor RMSProp state and says why; after it is cleared the learner carries on."""
+    g = pb.Paac("nature", 8, 2, 6, seed=3, precision=pb.BF16, lr=0.01, term_denom=50)
+    g.rollout()
+    assert g.update()["status"] == 0 and g.error_word() == 0
+    theta0, rms0 = g.params(), g.debug_read(pb.DBG_RMS).copy()
+    assert g.wait_probe(0) == pb.ERR_ARG
+    assert g.wait_probe(20000) == pb.ERR_TIMEOUT
+    assert g.error_word() == 1
+    g.rollout()
+    st = g.update()
+    assert st["status"] == pb.ERR_TIMEOUT and st["clip_scale"] == 0.0
+    g.clear_error_word()
+    assert np.array_equal(g.params(), theta0) and np.array_equal(g.debug_read(pb.DBG_RMS), rms0)
+    with pytest.raises(pb.PaacError):       # out of order: the skipped update consumed the rollout
+        g.update()
+    g.rollout()
+    assert g.update()["status"] == 0
+    assert not np.array_equal(g.params(), theta0)
+    g.close()
+
+
+def test_first_layer_weight_domain(orc):
+    """The fp16 image of the first layer holds |bf16(w)| <= 255: the largest such weight gives the oracle's logits,
+    anything beyond is refused and nothing changes; tiny weights (below 2^-25) only lose bits far below the tolerance."""
+    cfg = dict(arch="nature", precision="bf16", n_e=6, t_max=1, n_actions=4, lr=0.01, term_denom=50)
+    o, g = make_pair(orc, cfg, seed=11)
+    th = o.theta.copy()
+    th[:64] = 0.0
+    th[3] = 255.0            # largest magnitude the image holds
+    th[7] = -255.0
+    th[10] = 1e-9            # far below 2^-25
+    th[11] = 2.0 ** -25
+    o.theta = th
+    g.set_params(th)
+    check_rollout(orc, o, g, TOL["bf16"])
+    bad = th.copy()
+    bad[5] = 256.0
+    import ctypes as C
+    assert pb.lib().paac_set_params(g._h, bad.ctypes.data, bad.size) == pb.ERR_RANGE
+    bad[5] = np.inf
+    assert pb.lib().paac_set_params(g._h, bad.ctypes.data, bad.size) == pb.ERR_RANGE
+    assert np.array_equal(g.params(), th) and g.error_word() == 0
+    # the other layers have no such limit
+    ok = th.copy()
+    ok[9000] = 300.0
+    g.set_params(ok)
+    g.close()
+
+
+def test_partial_tensor_core_weight_gradient_mask(orc):
+    """Layers whose weight gradient is taken off the tensor cores (option TC_WGRAD_LAYERS) give the same gradient
+    within the bf16 tolerance as the all-tensor-core update."""
+    grads = []
+    for mask in (0xF, 0b0101):
+        g = pb.Paac("nature", 21, 2, 6, seed=9, precision=pb.BF16, lr=0.01, term_denom=50)
+        g.set_option(pb.OPT_TC_WGRAD_LAYERS, mask)
+        if grads:
+            g.force_actions(grads[0][1])
+        g.rollout()
+        acts = g.debug_read(pb.DBG_ACTIONS).copy()
+        st = g.update()
+        assert st["status"] == 0
+        grads.append((g.debug_read(pb.DBG_GRAD).copy(), acts, st["grad_norm"]))
+        g.close()
+    assert rel(grads[0][0], grads[1][0]) <= TOL["bf16"]
+    assert abs(grads[0][2] - grads[1][2]) <= TOL["bf16"] * grads[0][2]
