@@ -921,6 +921,10 @@ struct C3FwdCfg {
   }
   __host__ __device__ static constexpr int tap_plane(int) { return 0; }
   __host__ __device__ static constexpr int tap_shift(int t) { return (t / 3) * 9 + t % 3; }
+  // tap pairs one raster position apart (see tc_shift_t_kernel): per kernel row (s = 0, s = 1) and s = 2 alone
+  static constexpr int NSTEP = 6;
+  __host__ __device__ static constexpr int step_lo(int j) { return 3 * (j / 2) + 2 * (j & 1); }
+  __host__ __device__ static constexpr int step_hi(int j) { return (j & 1) ? -1 : 3 * (j / 2) + 1; }
 };
 // conv2 forward: rows = pairs of horizontally adjacent 32-channel pixels (128 bytes), i.e. the input in memory
 // order seen as [state][y][10 pairs]; even and odd image rows go to separate planes, so that tap row r
@@ -941,6 +945,10 @@ struct C2FwdCfg {
   }
   __host__ __device__ static constexpr int tap_plane(int t) { return (t >> 1) & 1; }
   __host__ __device__ static constexpr int tap_shift(int t) { return 10 * (t >> 2) + (t & 1); }
+  // tap pairs one raster position apart: the two pixel pairs of a kernel row
+  static constexpr int NSTEP = 4;
+  __host__ __device__ static constexpr int step_lo(int j) { return 2 * j; }
+  __host__ __device__ static constexpr int step_hi(int j) { return 2 * j + 1; }
 };
 // conv3 data gradient: the 7 x 7 x 64 output gradient on a zero-padded 11 x 11 raster; input pixel (y, x) is
 // raster position 11 y + x and tap (r, s) reads (2 - r) * 11 + (2 - s) rows down
@@ -961,6 +969,10 @@ struct C3DgradCfg {
   }
   __host__ __device__ static constexpr int tap_plane(int) { return 0; }
   __host__ __device__ static constexpr int tap_shift(int t) { return (2 - t / 3) * 11 + (2 - t % 3); }
+  // tap pairs one raster position apart, by rising shift: kernel row r = 2 - j / 2; (s = 2, s = 1) and s = 0 alone
+  static constexpr int NSTEP = 6;
+  __host__ __device__ static constexpr int step_lo(int j) { return 3 * (2 - j / 2) + ((j & 1) ? 0 : 2); }
+  __host__ __device__ static constexpr int step_hi(int j) { return (j & 1) ? -1 : 3 * (2 - j / 2) + 1; }
 };
 // conv2 data gradient (all four parity classes along N): the 9 x 9 x 64 gradient on a zero-padded 11 x 11
 // raster; class pixel (yy, xx) is position 11 yy + xx and tap (i, j) reads (1 - i) * 11 + (1 - j) rows down
@@ -1053,6 +1065,336 @@ template <class Map> struct ShiftReluMaskEpiS2 {
     return (uint32_t)(((b * 20 + 2 * yy + (cls >> 1)) * 20 + 2 * xx + (cls & 1)) * 32 + (col & 31));
   }
 };
+// ---- the same convolutions with the operand roles exchanged: weights as the A operand, held in tensor memory ----
+// An M = 128 instruction costs max(~50, N / 2) cycles, so a 64-channel layer that puts its channels along N runs the
+// tensor pipe at under two thirds of its rate and fetches 6 KB of operands from shared memory per instruction.  Here the
+// raster positions run along N = 128 and the weights are the A operand: the 128 rows of A are the 64 output channels of
+// TWO filter taps that lie one raster position apart (row 2 c = tap `lo`, channel c; row 2 c + 1 = tap `hi`, channel c),
+// written once per CTA into tensor memory (tcgen05.st: row -> lane, two bf16 per 32-bit column), from where the
+// instruction reads them without touching shared memory.  The B operand of a step is the staged input entered
+// shift(lo) rows down.  All steps accumulate into one 128 x 128 accumulator; with L = even lanes and H = odd lanes
+//   out[c][p] = L[c][p] + H[c][p + 1]
+// (the `hi` tap saw every position one row early).  The epilogue thread that owns TMEM lane l holds 32 consecutive
+// positions of its row; lanes 2 c and 2 c + 1 exchange what the other needs with one shuffle per two outputs, the even
+// lane finishing the even positions and the odd lane the odd ones.  Column 127 of a tile only feeds column 126, so a
+// tile yields 127 positions and tiles advance by 127.  The finished bf16 values are parked position-major in a staging
+// tile (128 bytes per position) and leave with whole-row stores, as in tc_shift_kernel.
+// Cfg adds: NSTEP, step_lo(j), step_hi(j) (tap indices, -1 = none; shift(hi) = shift(lo) + 1, same plane).
+// Roles: warps 0-7 epilogue (warp e: TMEM lane quarter e & 3, columns 64 (e >> 2) ..), warps 8-15 producers,
+// warp 16 issues the MMAs.  Warps 0-3 also write the weights into tensor memory before the first tile.
+constexpr int ST_TILE = 127;
+constexpr int ST_THREADS = 576;      // warps 0-7 (0-15 with bulk-copied stages) epilogue, 8-15 producers otherwise, 16 MMA, 17 bulk producer
+
+__device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// 32 columns of this warp's 32 lanes and, if `more`, the column that follows them
+__device__ __forceinline__ void tmem_ld_32x32_next(uint32_t taddr, uint32_t r[32], uint32_t& next, bool more) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  next = 0u;
+  if (more) asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(next) : "r"(taddr + 32u) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]: A's 128 rows in the lanes of a_tmem, 16 bf16 of K in eight 32-bit columns
+template <bool ACC>
+__device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "n"(ACC ? 1 : 0)
+      : "memory");
+}
+__device__ __forceinline__ void group_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+template <class Cfg, class Epi, int STAGES>
+__global__ void __launch_bounds__(ST_THREADS, 1)
+tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, Cfg cfg, const bf16* __restrict__ w,
+                  Epi epi, int tiles, uint32_t* error_word) {
+  static_assert(STAGES >= 2 && STAGES <= 8 && Cfg::STAGE_ROWS % 8 == 0, "pipeline shape");
+  constexpr int NT = Cfg::NT, NS = Cfg::NSTEP, SR = Cfg::STAGE_ROWS, PLANES = Cfg::PLANES;
+  constexpr uint32_t PLANE_BYTES = SR * 128, STAGE_BYTES = PLANES * PLANE_BYTES, STG_BYTES = 128 * 128;
+  constexpr uint32_t ACC_COLS = 128, A_COL0 = 2 * ACC_COLS, TMEM_COLS = 512;
+  // bulk-copied stages need one producer thread (warp 17), so warps 8-15 join the epilogue there
+  constexpr int EW = Cfg::BULK != 0 ? 16 : 8, ROWS_PER_WARP = 128 / EW;
+  static_assert(A_COL0 + NS * 32 <= TMEM_COLS, "tensor memory budget: two accumulators and the weights");
+  extern __shared__ uint8_t dyn_smem[];
+  __shared__ PkShared sh;
+  const uint32_t a_base0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;          // operand stages
+  const uint32_t stg0 = a_base0 + STAGES * STAGE_BYTES;                    // two staging tiles (tile parity)
+  const uint32_t mring0 = stg0 + 2 * STG_BYTES;                            // masked epilogues: two slots of activations
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], Cfg::BULK != 0 ? 1 : 256); mbar_init(&sh.empty[s], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], EW); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sh.mask_full[i], 256); mbar_init(&sh.mask_empty[i], 8); }
+    sh.abort = 0u;
+    fence_barrier_init();
+  }
+  if (warp == 16) tmem_alloc(&sh.tmem_base, TMEM_COLS);
+  // The weights pass through shared memory (the operand stages are not in use yet) so that all threads fetch them in
+  // one round of copies: A row a of step j (128 bytes) lands at (j * 128 + a) * 128, 16-byte chunks swizzled by row.
+  for (int i = threadIdx.x; i < NS * 128 * 8; i += ST_THREADS) {
+    const int q = i & 7, arow = (i >> 3) & 127, j = i >> 10;
+    const int tap = (arow & 1) ? Cfg::step_hi(j) : Cfg::step_lo(j);
+    cp_async16(a_base0 + (uint32_t)(j * 128 + arow) * 128u + ((uint32_t)(q ^ (arow & 7)) << 4),
+               w + ((size_t)(arow >> 1) * NT + (tap >= 0 ? tap : 0)) * TC_BK + q * 8, tap >= 0 ? 16u : 0u);
+  }
+  cp_async_commit();
+  cp_async_wait<0>();
+  tcgen05_fence_before();
+  __syncthreads();
+  tcgen05_fence_after();
+  const uint32_t tmem = sh.tmem_base;
+  if (warp < 4) {
+    // shared memory -> tensor memory: lane l of quarter `warp` is A row 32 warp + l = (tap lo / hi, channel)
+    const uint32_t arow = 32u * warp + lane;
+#pragma unroll 2
+    for (int j = 0; j < NS; ++j) {
+      uint32_t r[32];
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r[4 * q]), "=r"(r[4 * q + 1]), "=r"(r[4 * q + 2]), "=r"(r[4 * q + 3])
+                     : "r"(a_base0 + ((uint32_t)j * 128u + arow) * 128u + (((uint32_t)q ^ (arow & 7u)) << 4)) : "memory");
+      tmem_st_32x32(tmem + ((uint32_t)(32 * warp) << 16) + A_COL0 + j * 32, r);
+    }
+    tmem_st_wait();
+  }
+  tcgen05_fence_before();
+  __syncthreads();          // the stage area is free for the first tiles from here on
+  tcgen05_fence_after();
+  pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
+
+  if (Cfg::BULK != 0 && warp == 17) {
+    // ---------------- producer: a stage is one box of the layer input per plane (tiled bulk copies) ----------------
+    static_assert(Cfg::BULK == 0 || !Epi::MASK, "bulk-copied stages: plain forward layers only");
+    if (lane == 0) {
+      tma_prefetch_desc(&tm_a);
+      if (Cfg::BULK == 2) tma_prefetch_desc(&tm_b);
+      int it = 0;
+      for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++it) {
+        const int s = it % STAGES;
+        if (!mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY)) break;
+        mbar_arrive_expect_tx(&sh.full[s], STAGE_BYTES);
+        if (Cfg::BULK == 1) {
+          tma_load_2d(a_base0 + s * STAGE_BYTES, &tm_a, 0, t * ST_TILE, &sh.full[s]);
+        } else {
+          tma_load_3d(a_base0 + s * STAGE_BYTES, &tm_a, 0, 0, (t * ST_TILE) / 10, &sh.full[s]);
+          tma_load_3d(a_base0 + s * STAGE_BYTES + PLANE_BYTES, &tm_b, 0, 0, (t * ST_TILE) / 10, &sh.full[s]);
+        }
+      }
+    }
+  } else if (Cfg::BULK == 0 && warp >= 8 && warp < 16) {
+    // ---------------- producers: eight lanes per 128-byte row, 32 rows per pass ----------------
+    const int c = lane & 7, sub = (warp - 8) * 4 + (lane >> 3);
+    int it = 0;
+    bool alive = true;
+    for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x, ++it) {
+      const int s = it % STAGES;
+      const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+      if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+      const uint32_t stage = a_base0 + s * STAGE_BYTES;
+      // source addresses by arithmetic only, all of them before the first copy (a warp with asynchronous copies in
+      // flight waits for all of them at its next shared-memory load)
+      constexpr int NIT = (PLANES * SR + 31) / 32;
+      uint32_t srcs[NIT], vmask = 0;                    // element offsets from the tensor's base (< 2^32 elements)
+#pragma unroll
+      for (int k = 0; k < NIT; ++k) {
+        const int idx = sub + 32 * k;
+        srcs[k] = 0u;
+        if (idx < PLANES * SR) {
+          const int plane = PLANES == 1 ? 0 : idx / SR, ri = PLANES == 1 ? idx : idx % SR;
+          bool valid;
+          const bf16* ptr;
+          if constexpr (Cfg::RASTER > 0) ptr = cfg.src_cell(t * ST_TILE + ri, valid);
+          else ptr = cfg.src(plane, t * ST_TILE + ri, valid);
+          srcs[k] = (uint32_t)(ptr - cfg.base());
+          vmask |= valid ? 1u << k : 0u;
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < NIT; ++k) {
+        const int idx = sub + 32 * k;
+        if (idx < PLANES * SR) {
+          const int plane = PLANES == 1 ? 0 : idx / SR, ri = PLANES == 1 ? idx : idx % SR;
+          cp_async16(stage + plane * PLANE_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), cfg.base() + srcs[k] + c * 8,
+                     (vmask >> k) & 1u ? 16u : 0u);
+        }
+      }
+      cp_async_mbar_arrive(&sh.full[s]);
+      if constexpr (Epi::MASK) {
+        // the activations under the tile (the ReLU mask of its epilogue): ring slot row r = position 127 t + r,
+        // laid out exactly as the staging tile the epilogue reads them against
+        const int ms = it & 1;
+        const bool okm = mbar_wait(&sh.mask_empty[ms], ((it >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+        if (!__all_sync(0xffffffffu, okm)) { alive = false; break; }
+        const uint32_t dst = mring0 + ms * STG_BYTES;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int r = sub + 32 * k;
+          int b, y, x;
+          epi.map.split(t * ST_TILE + r, b, y, x);
+          const bool v = r < ST_TILE && epi.map.is_output(b, y, x);
+          cp_async16(dst + r * 128u + ((uint32_t)(c ^ ((r & 3) << 1)) << 4), epi.act + (v ? epi.index(b, y, x, c * 8) : 0u), v ? 16u : 0u);
+        }
+        cp_async_mbar_arrive(&sh.mask_full[ms]);
+      }
+    }
+    cp_async_commit();
+    cp_async_wait<0>();
+  } else if (warp < EW) {
+    // ---------------- epilogue: warp e reads TMEM lane quarter e & 3, columns (128 / (EW / 4)) * (e >> 2) .. ----------------
+    const int quarter = warp & 3, grp = warp >> 2;
+    constexpr int GCOLS = 128 / (EW / 4);                              // columns (= staging rows) of a group of four warps
+    const int ch = 16 * quarter + (lane >> 1), par = lane & 1;          // this lane's channel and tap half
+    float bias = 0.f;
+    if constexpr (!Epi::MASK) bias = __ldg(epi.bias + ch);
+    const int rr0 = lane >> 3, c16 = lane & 7;                          // second phase: row within a pass, 16-byte chunk
+    bool dead = false;
+    int local = 0;
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++local) {
+      const int ab = local & 1;
+      const uint32_t stg = stg0 + (local & 1) * STG_BYTES;
+      // where the rows this lane writes in the second phase go: rows GCOLS grp + ROWS_PER_WARP quarter + 4 p + rr0
+      uint32_t idx[ROWS_PER_WARP / 4];
+      uint32_t valid = 0;
+      {
+        const int r_first = GCOLS * grp + ROWS_PER_WARP * quarter + rr0;
+        int b, y, x;
+        epi.map.split(t * ST_TILE + r_first, b, y, x);
+        uint32_t at = epi.index(b, y, x, c16 * 8);
+#pragma unroll
+        for (int p = 0; p < ROWS_PER_WARP / 4; ++p) {
+          idx[p] = at;
+          if (r_first + 4 * p < ST_TILE && epi.map.is_output(b, y, x)) valid |= 1u << p;
+          epi.map.template advance<Epi>(b, y, x, at, 4);
+        }
+      }
+      if (!dead) {
+        const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
+        if (!__all_sync(0xffffffffu, ok)) dead = true;
+      }
+      if (!dead) {
+        tcgen05_fence_after();
+#pragma unroll
+        for (int cc = 0; cc < GCOLS / 32; ++cc) {
+          const int c0 = GCOLS * grp + 32 * cc;
+          uint32_t r[32], nxt;
+          tmem_ld_32x32_next(tmem + ((uint32_t)(quarter * 32) << 16) + ab * ACC_COLS + c0, r, nxt, c0 + 32 < 128);
+          if (cc == GCOLS / 32 - 1) {
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);            // the accumulator is free again
+          }
+          // even lane: out[2 i] = L[2 i] + H[2 i + 1];  odd lane: out[2 i + 1] = L[2 i + 1] + H[2 i + 2].
+          // Staging row = position (128 bytes, channel-major); its 16-byte chunks are swizzled by 2 (pos & 3), so that
+          // the two rows a store instruction touches use different banks; rows 2 i + par and 2 i + 4 + par share a swizzle,
+          // which leaves two base addresses and compile-time offsets.
+          const uint32_t row = (uint32_t)(c0 + par);
+          const uint32_t sb0 = stg + row * 128u + ((((uint32_t)ch >> 3) ^ ((row & 3u) << 1)) << 4) + ((uint32_t)ch & 7u) * 2u;
+          const uint32_t sb1 = stg + row * 128u + ((((uint32_t)ch >> 3) ^ (((row + 2u) & 3u) << 1)) << 4) + ((uint32_t)ch & 7u) * 2u;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float got = __shfl_xor_sync(0xffffffffu, __uint_as_float(r[2 * i + 1]), 1);
+            const float mine = __uint_as_float(par ? (i < 15 ? r[2 * i + 2] : nxt) : r[2 * i]);
+            const float v = (got + mine) + bias;
+            uint16_t hv;
+            if constexpr (!Epi::MASK) asm("cvt.rn.relu.bf16.f32 %0, %1;" : "=h"(hv) : "f"(v));
+            else asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(hv) : "f"(v));
+            asm volatile("st.shared.b16 [%0], %1;" ::"r"(((i & 1) ? sb1 : sb0) + (uint32_t)(i * 256)), "h"(hv) : "memory");
+          }
+        }
+      }
+      group_barrier(1 + grp, 128);                                  // the GCOLS rows of this group are complete
+      if constexpr (Epi::MASK) {
+        if (!dead) {
+          const bool okm = mbar_wait(&sh.mask_full[local & 1], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+          if (!__all_sync(0xffffffffu, okm)) dead = true;
+        }
+      }
+      if (!dead) {
+#pragma unroll
+        for (int p = 0; p < ROWS_PER_WARP / 4; ++p) {
+          const uint32_t rr = (uint32_t)(GCOLS * grp + ROWS_PER_WARP * quarter + 4 * p + rr0);
+          const uint32_t off = rr * 128u + (((uint32_t)c16 ^ ((rr & 3u) << 1)) << 4);
+          uint4 v;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg + off) : "memory");
+          if constexpr (Epi::MASK) {
+            uint4 m;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(m.x), "=r"(m.y), "=r"(m.z), "=r"(m.w)
+                         : "r"(mring0 + (local & 1) * STG_BYTES + off) : "memory");
+            v.x = mask_pair(v.x, m.x); v.y = mask_pair(v.y, m.y); v.z = mask_pair(v.z, m.z); v.w = mask_pair(v.w, m.w);
+          }
+          if ((valid >> p) & 1u) *reinterpret_cast<uint4*>(epi.out + idx[p]) = v;
+        }
+      }
+      if constexpr (Epi::MASK) {
+        __syncwarp();
+        if (!dead && lane == 0) mbar_arrive(&sh.mask_empty[local & 1]);
+      }
+    }
+  } else if (warp == 16 && lane == 0) {
+    // ---------------- MMA issuer ----------------
+    constexpr uint32_t idesc = make_idesc_bf16(TC_BM, 128, 0, 0);
+    const uint32_t hi = desc_hi_kmajor_sw128(), a_t = tmem + A_COL0;
+    int it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
+      const int ab = it & 1, s = it % STAGES;
+      ok = mbar_wait(&sh.acc_empty[ab], ((it >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      if (!ok) break;
+      ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      if (!ok) break;
+      fence_proxy_async_smem();        // the copies observed through the barrier -> visible to the MMA's operand reads
+      tcgen05_fence_after();
+      const uint32_t row0 = Cfg::BULK == 2 ? (uint32_t)((t * ST_TILE) % 10) : 0u;
+      const uint32_t b_lo = (((a_base0 + s * STAGE_BYTES) >> 4) & 0x3FFFu) + row0 * 8u;
+      const uint32_t d = tmem + ab * ACC_COLS;
+#pragma unroll
+      for (int j = 0; j < NS; ++j) {
+        constexpr uint32_t K_STEP = 32 >> 4;
+        const uint32_t b_off = (Cfg::tap_plane(Cfg::step_lo(j)) * PLANE_BYTES + Cfg::tap_shift(Cfg::step_lo(j)) * 128u) >> 4;
+#pragma unroll
+        for (int k = 0; k < TC_BK / 16; ++k) {
+          if (j == 0 && k == 0) mma_bf16_ts<false>(d, a_t, b_lo + b_off, hi, idesc);
+          else mma_bf16_ts<true>(d, a_t + (j * 4 + k) * 8, b_lo + b_off + k * K_STEP, hi, idesc);
+        }
+      }
+      mma_commit(&sh.empty[s]);
+      mma_commit(&sh.acc_full[ab]);
+    }
+  }
+  tcgen05_fence_before();
+  __syncthreads();
+  if (warp == 16) {
+    __syncwarp();
+    tcgen05_fence_after();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
+}
+
 // ---- plain split-k GEMM with both operands streamed (the fully connected layer, forward) ----------------
 // C[m][n] = sum_k A[m][k] W[n][k] for A[M][K], W[N][K] row-major bf16.  Same persistent skeleton; a work item
 // is (row tile, 128-column tile, k split), the stage holds the A and the W tile of one K block, and the
@@ -1847,6 +2189,32 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
   launch_kernel_overlapped(lc, kern, tiles < sm_count() ? tiles : sm_count(), SH_THREADS, smem, *tm_a, *tm_b, cfg, w, e, tiles, err);
 }
 
+template <class Cfg, class Epi, int STAGES>
+static void tc_shift_t(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int positions, uint32_t* err) {
+  constexpr int smem = STAGES * Cfg::PLANES * Cfg::STAGE_ROWS * 128 + 2 * 128 * 128 + (Epi::MASK ? 2 * 128 * 128 : 0) + 1024;
+  static_assert(smem <= 227 * 1024, "shared memory budget");
+  static_assert(smem - 1024 >= Cfg::NSTEP * 128 * 128, "the weights pass through the stage area on their way to tensor memory");
+  auto kern = tc_shift_t_kernel<Cfg, Epi, STAGES>;
+  static bool configured = false;
+  if (!configured) {
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    configured = true;
+  }
+  const int tiles = (positions + ST_TILE - 1) / ST_TILE;
+  static CUtensorMap no_map;
+  const CUtensorMap* tm_a = &no_map;
+  const CUtensorMap* tm_b = &no_map;
+  if constexpr (Cfg::BULK == 1) {
+    tm_a = tc_tensor_map(cfg.base_host(), (uint64_t)cfg.row_count(), 64, 64, Cfg::STAGE_ROWS);
+  } else if constexpr (Cfg::BULK == 2) {
+    tm_a = tc_tensor_map3(cfg.base_host(), 10, (uint64_t)cfg.states * 10, 128, 2560, 10, Cfg::STAGE_ROWS / 10);
+    tm_b = tc_tensor_map3(cfg.base_host() + 10 * 64, 10, (uint64_t)cfg.states * 10, 128, 2560, 10, Cfg::STAGE_ROWS / 10);
+  }
+  if (tm_a == nullptr || tm_b == nullptr) { lc.host_failure = true; return; }      // no tensor-map encoder
+  KernelScope scope(lc, kid);
+  launch_kernel_overlapped(lc, kern, tiles < sm_count() ? tiles : sm_count(), ST_THREADS, smem, *tm_a, *tm_b, cfg, w, e, tiles, err);
+}
+
 template <class G, class Epi>
 static void tc_conv1(LaunchCtx& lc, const uint8_t* frames, const bf16* w_blocks, Epi e, int n_states, uint32_t* err) {
   constexpr int STAGES = 3;
@@ -1917,13 +2285,13 @@ void tc_forward(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, 
                                 n, err);
     {
       typedef RasterMap<100, 10, 9, 9> Map;
-      tc_shift<C2FwdCfg, ShiftBiasReluEpi<Map, 9, 9>, 64, 3, 1>(
+      tc_shift_t<C2FwdCfg, ShiftBiasReluEpi<Map, 9, 9>, 4>(
           lc, KID_CONV2_FWD, C2FwdCfg{(const bf16*)act[0], n}, w + d[1].w_off,
           ShiftBiasReluEpi<Map, 9, 9>{Map{n}, (bf16*)act[1], theta + d[1].b_off, nullptr}, n * 100, err);
     }
     {
       typedef RasterMap<81, 9, 7, 7> Map;
-      tc_shift<C3FwdCfg, ShiftBiasReluEpi<Map, 7, 7>, 64, 6, 1>(
+      tc_shift_t<C3FwdCfg, ShiftBiasReluEpi<Map, 7, 7>, 6>(
           lc, KID_CONV3_FWD, C3FwdCfg{(const bf16*)act[1], n * 81}, w + d[2].w_off,
           ShiftBiasReluEpi<Map, 7, 7>{Map{n}, (bf16*)act[2], theta + d[2].b_off, nullptr}, n * 81, err);
     }
