@@ -1147,9 +1147,17 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], Cfg::BULK != 0 ? 1 : 256); mbar_init(&sh.empty[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], EW); }
+    // Two barriers per stage slot instead of four per tile: every wait, even one that is already satisfied, costs
+    // the single issuing thread a couple of hundred cycles during which the tensor pipe runs dry.
+    //   full[s]  ("ready"): the stage's copies have landed AND the accumulator of the tile that will use the slot
+    //            has been read out by the epilogue of the tile two before it (the first two tiles find that
+    //            arrival made here);
+    //   empty[s] ("done"):  the tile's instructions have completed: the producer may refill the slot and the
+    //            epilogue may read the accumulator.
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], (Cfg::BULK != 0 ? 1 : 256) + EW); mbar_init(&sh.empty[s], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.mask_full[i], 256); mbar_init(&sh.mask_empty[i], 8); }
+    for (int s = 0; s < 2; ++s)
+      for (int e = 0; e < EW; ++e) mbar_arrive(&sh.full[s]);
     sh.abort = 0u;
     fence_barrier_init();
   }
@@ -1293,7 +1301,7 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         }
       }
       if (!dead) {
-        const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
+        const bool ok = mbar_wait(&sh.empty[local % STAGES], (local / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
         if (!__all_sync(0xffffffffu, ok)) dead = true;
       }
       if (!dead) {
@@ -1306,7 +1314,7 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
           if (cc == GCOLS / 32 - 1) {
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);            // the accumulator is free again
+            if (lane == 0) mbar_arrive(&sh.full[(local + 2) % STAGES]);      // the accumulator is free for the tile after next
           }
           // even lane: out[2 i] = L[2 i] + H[2 i + 1];  odd lane: out[2 i + 1] = L[2 i + 1] + H[2 i + 2].
           // Staging row = position (128 bytes, channel-major); its 16-byte chunks are swizzled by 2 (pos & 3), so that
@@ -1363,8 +1371,6 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     bool ok = true;
     for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
       const int ab = it & 1, s = it % STAGES;
-      ok = mbar_wait(&sh.acc_empty[ab], ((it >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
-      if (!ok) break;
       ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
       if (!ok) break;
       fence_proxy_async_smem();        // the copies observed through the barrier -> visible to the MMA's operand reads
@@ -1383,7 +1389,6 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         }
       }
       mma_commit(&sh.empty[s]);
-      mma_commit(&sh.acc_full[ab]);
     }
   }
   tcgen05_fence_before();
@@ -3450,6 +3455,9 @@ void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* con
   typedef NatConv3 C3;
   const int M = n * C3::H * C3::W;
   typedef RasterMap<121, 11, 9, 9> Map;
+  // (the role-exchanged kernel also takes this layer -- tc_shift_t<C3DgradCfg, ShiftReluMaskEpi<Map, 9, 9>, 4> -- but with
+  // its stages fetched by eight cp.async warps only eight warps are left for the transposing epilogue, which then sets
+  // the pace: measured 71 us against 64 us for the kernel below)
   tc_shift<C3DgradCfg, ShiftReluMaskEpi<Map, 9, 9>, 64, 4, 1>(
       lc, KID_CONV3_DGRAD, C3DgradCfg{(const bf16*)gact[2], n}, images + 4 * 32 * 256,
       ShiftReluMaskEpi<Map, 9, 9>{Map{n}, (bf16*)gact[1], (const bf16*)act[1]}, n * 121, err);
