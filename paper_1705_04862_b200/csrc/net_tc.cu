@@ -687,9 +687,16 @@ tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], Cfg::BULK != 0 ? 1 : 256); mbar_init(&sh.empty[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 8); }
+    // Two barriers per stage slot (a wait costs the single issuing thread a couple of hundred cycles even when it is
+    // already satisfied, and the tensor pipe runs dry meanwhile):
+    //   full[s]  the stage's copies have landed AND the accumulator of the tile that will use the slot has been read
+    //            out by the epilogue of the tile two before it (the first two tiles find that arrival made here);
+    //   empty[s] the tile's instructions have completed: the producers may refill the slot, the epilogue may read.
+    static_assert(STAGES >= 2, "the accumulator release of tile i arrives on the slot of tile i + 2");
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], (Cfg::BULK != 0 ? 1 : 256) + 8); mbar_init(&sh.empty[s], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&sh.mask_full[i], 256); mbar_init(&sh.mask_empty[i], 8); }
+    for (int s = 0; s < 2; ++s)
+      for (int e = 0; e < 8; ++e) mbar_arrive(&sh.full[s]);
     sh.abort = 0u;
     fence_barrier_init();
   }
@@ -817,7 +824,7 @@ tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
           epi.map.template advance<Epi>(b, y, x, at, RPP);
         }
       }
-      const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      const bool ok = mbar_wait(&sh.empty[local % STAGES], (local / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
 #pragma unroll
@@ -839,7 +846,7 @@ tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
       }
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);            // the accumulator is free again
+      if (lane == 0) mbar_arrive(&sh.full[(local + 2) % STAGES]);      // the accumulator is free for the tile after next
       if constexpr (Epi::MASK) {                                 // this tile's activations have landed
         const bool okm = mbar_wait(&sh.mask_full[local & 1], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
         if (!__all_sync(0xffffffffu, okm)) break;
@@ -870,8 +877,6 @@ tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
     bool ok = true;
     for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++it) {
       const int ab = it & 1, s = it % STAGES;
-      ok = mbar_wait(&sh.acc_empty[ab], ((it >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
-      if (!ok) break;
       ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
       if (!ok) break;
       fence_proxy_async_smem();        // the copies observed through the barrier -> visible to the MMA's operand reads
@@ -895,7 +900,6 @@ tc_shift_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant_
         }
       }
       mma_commit(&sh.empty[s]);
-      mma_commit(&sh.acc_full[ab]);
     }
   }
   tcgen05_fence_before();
@@ -1914,8 +1918,13 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
   const int total_pos = n_states * POS;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], NPROD / 32); mbar_init(&sh.empty[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.acc_full[i], 1); mbar_init(&sh.acc_empty[i], 8); }
+    // full[s]: the stage has been expanded AND the accumulator of the tile that will use the slot has been read out by
+    // the epilogue of the tile two before it (the first two tiles find that arrival made here); empty[s]: the tile's
+    // instructions have completed (producers may refill the slot, the epilogue may read).  One wait and one commit per
+    // tile: a wait costs the issuing thread a couple of hundred cycles even when it is already satisfied.
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], NPROD / 32 + 8); mbar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < 2; ++s)
+      for (int e = 0; e < 8; ++e) mbar_arrive(&sh.full[s]);
     for (int i = 0; i < C1_RAW_SLOTS; ++i) { mbar_init(&sh.raw_full[i], 1); mbar_init(&sh.raw_empty[i], NPROD / 32); }
     sh.abort = 0u;
     fence_barrier_init();
@@ -2039,14 +2048,14 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
           if (Y >= C1_RASTER) { Y -= C1_RASTER; ++b; }
         }
       }
-      const bool ok = mbar_wait(&sh.acc_full[ab], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
+      const bool ok = mbar_wait(&sh.empty[local % STAGES], (local / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!__all_sync(0xffffffffu, ok)) break;
       tcgen05_fence_after();
       uint32_t r[32];
       tmem_ld_32x32(tmem + ((uint32_t)(quarter * 32) << 16) + ab * BN + h * 32, r);
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.acc_empty[ab]);
+      if (lane == 0) mbar_arrive(&sh.full[(local + 2) % STAGES]);      // the accumulator is free for the tile after next
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         uint32_t o[4];
@@ -2080,8 +2089,6 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
       bool ok = true;
       for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, ++local) {
         const int ab = local & 1, s = local % STAGES;
-        ok = mbar_wait(&sh.acc_empty[ab], ((local >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
-        if (!ok) break;
         ok = mbar_wait(&sh.full[s], (local / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
         if (!ok) break;
         tcgen05_fence_after();
@@ -2106,7 +2113,6 @@ tc_conv1_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict__ w, 
           }
         }
         mma_commit(&sh.empty[s]);
-        mma_commit(&sh.acc_full[ab]);
       }
     }
   } else if (lane == 0) {
