@@ -73,6 +73,9 @@ def lib():
         L.orc_cdf_margin.restype = C.c_float
         L.orc_loss_double.restype = C.c_double
         L.orc_clip_rmsprop.restype = C.c_int
+        L.orc_q_greedy.restype = C.c_int32
+        L.orc_q_select.restype = C.c_int32
+        L.orc_q_margin.restype = C.c_float
         _lib = L
     return _lib
 
@@ -224,6 +227,34 @@ def head_grad(beta, value_coef, logits, values, actions, R, adv):
     return dz, dV, dict(policy_loss=stats[0], value_loss=stats[1], entropy=stats[2])
 
 
+def q_greedy(q):
+    q = np.ascontiguousarray(q, np.float32)
+    return int(lib().orc_q_greedy(_p(q), q.shape[0]))
+
+
+def q_select(q, u, eps):
+    """Epsilon-greedy action from Q-values [A] and one uniform (Section 3: the policy may be implicit)."""
+    q = np.ascontiguousarray(q, np.float32)
+    return int(lib().orc_q_select(_p(q), q.shape[0], C.c_float(u), C.c_float(eps)))
+
+
+def q_margin(q):
+    q = np.ascontiguousarray(q, np.float32)
+    return float(lib().orc_q_margin(_p(q), q.shape[0]))
+
+
+def q_head_grad(value_coef, q, actions, R):
+    """Gradient of the n-step Q loss (Eqs. 3-4) at the Q-values [B, A] -> (dq, stats)."""
+    q = np.ascontiguousarray(q, np.float32)
+    B, A = q.shape
+    actions = np.ascontiguousarray(actions, np.int32).reshape(B)
+    R = np.ascontiguousarray(R, np.float32).reshape(B)
+    dq = np.zeros((B, A), np.float32)
+    stats = (C.c_double * 2)()
+    lib().orc_q_head_grad(B, A, C.c_float(value_coef), _p(q), _p(actions), _p(R), _p(dq), stats)
+    return dq, dict(value_loss=stats[0], mean_max_q=stats[1])
+
+
 def loss_double(net, theta64, frames, beta, value_coef, actions, R, adv):
     theta64 = np.ascontiguousarray(theta64, np.float64)
     frames = np.ascontiguousarray(frames, np.uint8)
@@ -257,11 +288,16 @@ def clip_rmsprop(theta, m, grad, lr, rho, eps, clip):
 
 
 DEFAULT_HP = dict(gamma=0.99, lr=0.0224, rms_decay=0.99, rms_eps=0.1, clip_norm=40.0,
-                  entropy_beta=0.01, value_coef=1.0, term_denom=200)
+                  entropy_beta=0.01, value_coef=1.0, term_denom=200, algorithm="a2c", epsilon=0.1)
 
 
 class OraclePAAC:
-    """State of one PAAC learner on the CPU; rollout() and update() are Algorithm 1's two halves."""
+    """State of one PAAC learner on the CPU; rollout() and update() are Algorithm 1's two halves.
+
+    hp["algorithm"] = "a2c" is Algorithm 1 as printed; "nstep_q" keeps the framework (Section 3) and swaps
+    what the heads mean (Section 2.2): the A outputs are Q-values, acting is epsilon-greedy, the stored
+    value of a step is Q(s_t, a_t), the bootstrap is max_a Q(s_{t_max+1}, a), the loss is Eq. 3 on n-step
+    targets.  The value head is carried along unused (its gradient is zero)."""
 
     def __init__(self, arch, n_e, t_max, n_actions, seed, bf16=False, hp=None, net=None):
         self.net = net if net is not None else arch_net(arch, n_actions)
@@ -288,20 +324,25 @@ class OraclePAAC:
         for t in range(T):
             acts, logits, values = forward(self.net, self.theta, ro["frames"][t], self.bf16)
             p, _, _ = softmax(logits)
+            qmode = self.hp["algorithm"] == "nstep_q"
+            ro.setdefault("sampled", np.zeros((T, n_e), np.int32))
             for e in range(n_e):
                 u = action_uniform(self.seed, e, step0 + t)
                 ro["uniforms"][t, e] = u
-                a = sample(p[e], u)
+                a = q_select(logits[e], u, self.hp["epsilon"]) if qmode else sample(p[e], u)
+                ro["sampled"][t, e] = a
                 if forced_actions is not None and forced_actions[t, e] >= 0:
                     a = int(forced_actions[t, e])
                 ro["actions"][t, e] = a
+                if qmode:
+                    values[e] = logits[e, a]          # what the step is worth to the learner: Q(s_t, a_t)
             ro["logits"][t], ro["values"][t], ro["probs"][t] = logits, values, p
             ro["acts"].append(acts)
             f, r, term = env_step(self.seed, step0 + t, ro["actions"][t], self.hp["term_denom"], self.counters,
                                   self.h, self.w)
             ro["frames"][t + 1], ro["rewards"][t], ro["terminals"][t] = f, r, term
-        _, _, vb = forward(self.net, self.theta, ro["frames"][T], self.bf16)
-        ro["values"][T] = vb
+        _, zb, vb = forward(self.net, self.theta, ro["frames"][T], self.bf16)
+        ro["values"][T] = zb.max(axis=1) if self.hp["algorithm"] == "nstep_q" else vb
         self.state = ro["frames"][T].copy()
         self.ro = ro
         return ro
@@ -312,8 +353,13 @@ class OraclePAAC:
         R, adv = returns(hp["gamma"], ro["rewards"], ro["terminals"], ro["values"])
         frames = ro["frames"][:T].reshape(B, self.h, self.w, 4)
         acts, logits, values = forward(self.net, self.theta, frames, self.bf16)
-        dz, dV, stats = head_grad(hp["entropy_beta"], hp["value_coef"], logits, values, ro["actions"].reshape(B),
-                                  R.reshape(B), adv.reshape(B))
+        if hp["algorithm"] == "nstep_q":
+            dz, qs = q_head_grad(hp["value_coef"], logits, ro["actions"].reshape(B), R.reshape(B))
+            dV = np.zeros(B, np.float32)
+            stats = dict(policy_loss=0.0, value_loss=qs["value_loss"], entropy=0.0)
+        else:
+            dz, dV, stats = head_grad(hp["entropy_beta"], hp["value_coef"], logits, values, ro["actions"].reshape(B),
+                                      R.reshape(B), adv.reshape(B))
         grad, gacts = backward(self.net, self.theta, frames, acts, dz, dV, self.bf16)
         st, norm, scale = clip_rmsprop(self.theta, self.m, grad, hp["lr"], hp["rms_decay"], hp["rms_eps"],
                                        hp["clip_norm"])

@@ -22,6 +22,8 @@
  *   softmax / sampling   sum-to-one, entropy bounds, shift invariance, brute force
  *   returns              closed form sum gamma^k r + gamma^n V, worked cases
  *   clip / RMSProp       closed forms
+ *   n-step Q variant     brute-force arg max and exploration branch, exploration frequency,
+ *                        PyTorch autograd and central differences of the loss, hand case
  * The whole iteration has no printed value in the paper to compare with:
  * beyond the pieces above it is "parity unpinned".
  */
@@ -380,6 +382,60 @@ void orc_head_grad(int B, int A, float beta, float value_coef, const float* logi
     val += d * d; ent += H;
   }
   stats[0] = pol / B; stats[1] = (double)value_coef * val / B; stats[2] = ent / B;
+}
+
+/* ------------------------------------------------------------------ */
+/* Value-based variant on the same framework (Section 3: the policy may */
+/* be implicit; Section 2.2, Eqs. 2-4): the A outputs of the first head */
+/* are Q(s, a; theta).  Acting is epsilon-greedy on Q; the target of    */
+/* experience t is the n-step return bootstrapped from                  */
+/* max_a' Q(s_{tmax+1}, a'; theta) (Eq. 3's target with the rewards of  */
+/* the rollout in between, cut at terminals: orc_returns with that      */
+/* bootstrap), and the loss is the batch mean of c (R_t - Q(s_t,a_t))^2 */
+/* with R constant.  Eq. 4 prints the factor -1/2 where the derivative  */
+/* of Eq. 3's square gives -2: the scale is the hyper-parameter c       */
+/* (value_coef), as for the critic.                                     */
+/* ------------------------------------------------------------------ */
+/* arg max_a q[a], the smallest index among equals */
+int32_t orc_q_greedy(const float* q, int A) {
+  int best = 0;
+  for (int k = 1; k < A; ++k) if (q[k] > q[best]) best = k;
+  return best;
+}
+/* One uniform u in [0,1) decides both whether to explore and where: u < eps picks action
+ * floor((u / eps) * A) (u / eps is uniform on [0,1) given u < eps), anything else is greedy.
+ * The two float operations are single IEEE roundings, so any machine takes the same decision. */
+int32_t orc_q_select(const float* q, int A, float u, float eps) {
+  if (u < eps) {
+    volatile float scaled = u / eps;
+    volatile float pos = scaled * (float)A;
+    int k = (int)pos;
+    return k < A - 1 ? k : A - 1;
+  }
+  return orc_q_greedy(q, A);
+}
+/* gap between the largest and the second largest Q-value: a greedy mismatch between two
+ * implementations is tolerated only when this is within their rounding */
+float orc_q_margin(const float* q, int A) {
+  int b = orc_q_greedy(q, A);
+  float second = -INFINITY;
+  for (int k = 0; k < A; ++k) if (k != b && q[k] > second) second = q[k];
+  return q[b] - second;
+}
+/* L = (c / B) sum_i (R_i - Q_i[a_i])^2;  dL/dQ_i[k] = (2 c / B) (Q_i[a_i] - R_i) for k = a_i, else 0.
+ * stats = {loss, mean of max_a Q} */
+void orc_q_head_grad(int B, int A, float value_coef, const float* q, const int32_t* actions, const float* R,
+                     float* dq /* [B][A] */, double stats[2]) {
+  double loss = 0.0, qmax = 0.0;
+  for (int i = 0; i < B; ++i) {
+    const float* qi = q + (size_t)i * A;
+    for (int k = 0; k < A; ++k) dq[(size_t)i * A + k] = 0.f;
+    double d = (double)qi[actions[i]] - (double)R[i];
+    dq[(size_t)i * A + actions[i]] = (float)(2.0 * (double)value_coef * d / B);
+    loss += d * d;
+    qmax += (double)qi[orc_q_greedy(qi, A)];
+  }
+  stats[0] = (double)value_coef * loss / B; stats[1] = qmax / B;
 }
 
 /* scalar loss in double with exact (unrounded) weights; used by the
