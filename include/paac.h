@@ -47,6 +47,18 @@ enum { PAAC_ARCH_NIPS = 0, PAAC_ARCH_NATURE = 1 };
  *            float accumulation, float master parameters and optimiser. */
 enum { PAAC_FP32 = 0, PAAC_BF16 = 1 };
 
+/* What the learner is (Section 3: the framework does not care how the policy is represented).
+ * PAAC_ALGO_A2C:     the parallel advantage actor-critic of Algorithm 1 (Section 4, Eqs. 9-10).
+ * PAAC_ALGO_NSTEP_Q: value-based (Section 2.2, Eqs. 2-4): the A outputs of the first head are Q(s, a; theta);
+ *                    acting is epsilon-greedy (one Philox uniform u per environment and step: u < epsilon
+ *                    explores into action floor((u / epsilon) A), anything else takes the first arg max);
+ *                    the value stored for a step is Q(s_t, a_t), the bootstrap value is max_a Q(s_{t_max}, a),
+ *                    targets are the same n-step returns, and the loss is the batch mean of
+ *                    value_coef (R_t - Q(s_t, a_t))^2 with R constant (Eq. 4 prints the factor -1/2 where the
+ *                    derivative of Eq. 3's square has -2: value_coef carries the scale).  The value head is
+ *                    carried along unused and receives a zero gradient; entropy_beta is ignored. */
+enum { PAAC_ALGO_A2C = 0, PAAC_ALGO_NSTEP_Q = 1 };
+
 enum {
   PAAC_OK = 0,
   PAAC_ERR_ARG = 1,        /* null pointer, size or enum out of range */
@@ -77,6 +89,8 @@ typedef struct {
                            NULL: the library allocates and owns it */
   size_t workspace_bytes;
   void* stream;         /* cudaStream_t the work is enqueued on; NULL: the default stream */
+  int algorithm;        /* PAAC_ALGO_A2C (default) or PAAC_ALGO_NSTEP_Q */
+  float epsilon;        /* PAAC_ALGO_NSTEP_Q: exploration probability in [0, 1] (default 0.1) */
 } paac_hparams;
 
 void paac_default_hparams(paac_hparams* hp /* host, out */);
@@ -110,9 +124,9 @@ typedef struct {
 int paac_rollout(paac_ctx* ctx, paac_rollout_view* view /* host, out, nullable */);
 
 typedef struct {
-  float policy_loss;   /* -(1/B) sum adv_i log pi(a_i | s_i) */
-  float value_loss;    /* (value_coef/B) sum (R_i - V_i)^2 */
-  float entropy;       /* (1/B) sum H(pi(. | s_i)) */
+  float policy_loss;   /* -(1/B) sum adv_i log pi(a_i | s_i)                    (0 for PAAC_ALGO_NSTEP_Q) */
+  float value_loss;    /* (value_coef/B) sum (R_i - V_i)^2, or (R_i - Q(s_i, a_i))^2 for PAAC_ALGO_NSTEP_Q */
+  float entropy;       /* (1/B) sum H(pi(. | s_i))                              (0 for PAAC_ALGO_NSTEP_Q) */
   float grad_norm;     /* global L2 norm before clipping */
   float clip_scale;    /* factor applied to the gradient (1 when not clipped) */
   int32_t status;      /* PAAC_OK, PAAC_ERR_NONFINITE, PAAC_ERR_TIMEOUT or PAAC_ERR_RANGE */

@@ -72,6 +72,8 @@ bool valid_shape(int arch, int n_e, int t_max, int A, const paac_hparams* hp) {
   if (n_e < 1 || n_e > 65536 || t_max < 1 || t_max > 64 || A < 2 || A > 32) return false;
   if ((long long)n_e * (t_max + 1) > 131072) return false;   // keeps every row index below 2^31
   if (hp->term_denom == 0) return false;
+  if (hp->algorithm != PAAC_ALGO_A2C && hp->algorithm != PAAC_ALGO_NSTEP_Q) return false;
+  if (!(hp->epsilon >= 0.f && hp->epsilon <= 1.f)) return false;
   return true;
 }
 
@@ -136,6 +138,7 @@ int cuda_status(paac_ctx* c) {
 }
 
 bool use_tc(const paac_ctx* c) { return tc_supported(c->arch, c->prec) && !c->simt_only; }
+HeadMode head_mode(const paac_ctx* c) { return HeadMode{c->hp.algorithm, c->hp.epsilon}; }
 
 // bf16 copies of the master parameters, in the canonical layout and regrouped for the backward kernels
 void refresh_weight_copies(paac_ctx* c, bool cast) {
@@ -162,12 +165,12 @@ bool forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, Hea
                &c->stats->error_word, &splits);
     if (tail != nullptr && splits == 0 && sample) {
       *tail = HeadsTail{c->scratch, c->theta + c->nd.pi_b, c->theta + c->nd.v_b, c->A, c->logits + row * c->A,
-                        c->values + row, forced, actions, sampled, uniforms};
+                        c->values + row, forced, actions, sampled, uniforms, head_mode(c)};
       return true;
     }
     launch_heads_fused(c->lc, c->nd, c->theta, c->theta16, c->scratch, splits, (bf16*)act[c->nd.n_conv], c->n_e,
                        c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot, forced, actions,
-                       sampled, uniforms, (advanced && splits == 0 && !sample) ? c->step_dev : nullptr, (uint32_t)c->t_max);
+                       sampled, uniforms, head_mode(c), (advanced && splits == 0 && !sample) ? c->step_dev : nullptr, (uint32_t)c->t_max);
     if (advanced) *advanced = splits == 0 && !sample;      // the sampling kernel has moved the step index on
     return false;
   }
@@ -178,7 +181,7 @@ bool forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, Hea
     simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
   launch_heads(c->lc, c->prec, c->nd, c->theta, c->theta16, act[c->nd.n_conv], c->n_e,
                c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot, forced, actions, sampled,
-               uniforms);
+               uniforms, head_mode(c));
   return false;
 }
 
@@ -239,6 +242,7 @@ void paac_default_hparams(paac_hparams* hp) {
   hp->gamma = 0.99f; hp->lr = 0.0224f; hp->rms_decay = 0.99f; hp->rms_eps = 0.1f;
   hp->clip_norm = 40.f; hp->entropy_beta = 0.01f; hp->value_coef = 1.f;
   hp->term_denom = 200; hp->precision = PAAC_FP32;
+  hp->algorithm = PAAC_ALGO_A2C; hp->epsilon = 0.1f;
 }
 
 size_t paac_workspace_bytes(int arch, int n_e, int t_max, int n_actions, const paac_hparams* hp) {
@@ -325,7 +329,7 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
   if (!c->rollout_fresh) return PAAC_ERR_STATE;
   const paac_hparams& hp = c->hp;
   run_recorded(c, 1, c->cur, [&]() {
-    launch_returns_head_grad(c->lc, c->n_e, c->t_max, c->A, hp.gamma, hp.entropy_beta, hp.value_coef, c->rewards,
+    launch_returns_head_grad(c->lc, head_mode(c), c->n_e, c->t_max, c->A, hp.gamma, hp.entropy_beta, hp.value_coef, c->rewards,
                              c->terminals, c->logits, c->values, c->actions, c->R, c->adv, c->dz, c->dV, c->loss_terms,
                              c->stats);
     const int L = c->nd.n_conv;

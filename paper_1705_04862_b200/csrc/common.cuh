@@ -46,6 +46,66 @@ __host__ __device__ __forceinline__ float philox_uniform(uint32_t c0, uint32_t c
   return (float)(o[0] >> 8) * (1.0f / 16777216.0f);
 }
 
+// ---- what the heads mean -----------------------------------------------------------
+// PAAC_ALGO_A2C: softmax policy over the A outputs of the first head plus a state value (Algorithm 1).
+// PAAC_ALGO_NSTEP_Q: the A outputs are Q(s, a) (Section 2.2 on the framework of Section 3): acting is
+// epsilon-greedy, the value stored for a step is Q(s_t, a_t), the bootstrap value is max_a Q.
+struct HeadMode { int algo; float eps; };
+
+#ifdef __CUDACC__
+// Everything that follows the heads' dot products, done by one full warp for state e.  Lane k < A holds head output
+// z_k (the other lanes -inf); v is the value head's output, the same in all lanes.  Writes the A outputs and the
+// stored value; with `sample` it also draws the action from the Philox uniform of (e, step) -- inverse CDF of the
+// softmax in index order on a float running sum, or epsilon-greedy on the Q-values with the one uniform deciding
+// both whether to explore (u < eps) and where (floor((u / eps) A)) --, honours a forced action, and returns the
+// action taken (-1 without sampling).
+__device__ __forceinline__ int warp_finish_heads(const HeadMode hm, float z, float v, int lane, int A, size_t e,
+                                                 float* __restrict__ logits, float* __restrict__ values, bool sample,
+                                                 uint64_t seed, uint64_t step, const int32_t* __restrict__ forced,
+                                                 int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
+                                                 float* __restrict__ uniforms) {
+  if (lane < A) logits[e * A + lane] = z;
+  float m = z;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (hm.algo == PAAC_ALGO_NSTEP_Q) {
+    const uint32_t at_max = __ballot_sync(0xffffffffu, lane < A && z == m);
+    const int greedy = at_max ? __ffs(at_max) - 1 : 0;                  // smallest index among equal maxima
+    if (!sample) { if (lane == 0) values[e] = m; return -1; }
+    const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
+    int a = greedy;
+    if (u < hm.eps) {
+      const int k = (int)__fmul_rn(__fdiv_rn(u, hm.eps), (float)A);     // two single roundings: the same on any machine
+      a = k < A - 1 ? k : A - 1;
+    }
+    const int drawn = a;
+    if (forced != nullptr && forced[e] >= 0) a = forced[e];
+    const float qa = __shfl_sync(0xffffffffu, z, a);
+    if (lane == 0) { sampled[e] = drawn; actions[e] = a; uniforms[e] = u; values[e] = qa; }
+    return a;
+  }
+  if (lane == 0) values[e] = v;
+  if (!sample) return -1;
+  float ex = lane < A ? expf(z - m) : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ex += __shfl_xor_sync(0xffffffffu, ex, o);
+  const float lse = m + logf(ex);
+  const float p = lane < A ? expf(z - lse) : 0.f;
+  const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
+  float c = 0.f;
+  int a = A - 1;
+  bool found = false;
+  for (int k = 0; k < A; ++k) {
+    c += __shfl_sync(0xffffffffu, p, k);
+    if (!found && u < c) { a = k; found = true; }
+  }
+  const int drawn = a;
+  if (forced != nullptr && forced[e] >= 0) a = forced[e];
+  if (lane == 0) { sampled[e] = drawn; actions[e] = a; uniforms[e] = u; }
+  return a;
+}
+#endif
+
 // ---- environment hash -----------------------------------------------------------
 constexpr uint32_t HASH_K0 = 0x9E3779B9u, HASH_K1 = 0xBB67AE85u, HASH_K2 = 0x6A09E667u;
 constexpr uint32_t HASH_TAG_REWARD = 0x52455744u, HASH_TAG_TERMINAL = 0x5445524Du;

@@ -77,32 +77,8 @@ env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, 
     float sum = -INFINITY;
     if (lane <= A) sum = (ht.hp[(size_t)e * 32 + lane] + ht.hp[((size_t)n_e + e) * 32 + lane]) + bias;
     const float z = lane < A ? sum : -INFINITY;
-    if (lane < A) ht.logits[(size_t)e * A + lane] = z;
-    if (lane == A) ht.values[e] = sum;
-    float m = z;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float se = lane < A ? expf(z - m) : 0.f;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
-    const float lse = m + logf(se);
-    const float p = lane < A ? expf(z - lse) : 0.f;
-    const uint64_t step64 = *step_base + t;
-    const float u = philox_uniform(e, (uint32_t)step64, (uint32_t)(step64 >> 32), RNG_STREAM_ACTION, seed);
-    float c = 0.f;
-    int a = A - 1;
-    bool found = false;
-    for (int k = 0; k < A; ++k) {
-      c += __shfl_sync(0xffffffffu, p, k);
-      if (!found && u < c) { a = k; found = true; }
-    }
-    if (lane == 0) {
-      ht.sampled[e] = a;
-      if (ht.forced != nullptr && ht.forced[e] >= 0) a = ht.forced[e];
-      ht.actions[e] = a;
-      ht.uniforms[e] = u;
-    }
-    a_sampled = a;
+    a_sampled = warp_finish_heads(ht.mode, z, __shfl_sync(0xffffffffu, sum, A), lane, A, (size_t)e, ht.logits, ht.values, true,
+                                  seed, *step_base + t, ht.forced, ht.actions, ht.sampled, ht.uniforms);
   } else {
     pdl_entry();
   }

@@ -42,7 +42,7 @@ heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* _
              const TW* __restrict__ wv, const float* __restrict__ bv, int n, int A,
              float* __restrict__ logits, float* __restrict__ values, uint64_t seed, const uint64_t* __restrict__ step_base, uint32_t t,
              const int32_t* __restrict__ forced, int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
-             float* __restrict__ uniforms) {
+             float* __restrict__ uniforms, HeadMode mode) {
   pdl_entry();
   constexpr int F = 32 * EPL;
   const int lane = threadIdx.x & 31;
@@ -64,29 +64,8 @@ heads_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const float* _
 #pragma unroll
   for (int i = 0; i < EPL; ++i) v = fmaf(to_f(wv[lane * EPL + i]), x[i], v);
   v = warp_sum(v) + bv[0];
-  if (lane < A) logits[(size_t)e * A + lane] = z;
-  if (lane == 0) values[e] = v;
-  if (actions == nullptr) return;
-
-  const float m = warp_max(z);
-  const float ex = lane < A ? expf(z - m) : 0.f;
-  const float lse = m + logf(warp_sum(ex));
-  const float p = lane < A ? expf(z - lse) : 0.f;
-  const uint64_t step = *step_base + t;
-  const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
-  float c = 0.f;
-  int a = A - 1;
-  bool found = false;
-  for (int k = 0; k < A; ++k) {
-    c += __shfl_sync(0xffffffffu, p, k);
-    if (!found && u < c) { a = k; found = true; }
-  }
-  if (lane == 0) {
-    sampled[e] = a;
-    if (forced != nullptr && forced[e] >= 0) a = forced[e];
-    actions[e] = a;
-    uniforms[e] = u;
-  }
+  warp_finish_heads(mode, z, v, lane, A, (size_t)e, logits, values, actions != nullptr, seed,
+                    actions != nullptr ? *step_base + t : 0ull, forced, actions, sampled, uniforms);
 }
 
 // The same, fused with the end of the fully connected layer of the tensor-core path: the warp first finishes
@@ -104,7 +83,7 @@ heads_fused_kernel(const float* __restrict__ part, int splits, const float* __re
                    const bf16* __restrict__ wpi, const float* __restrict__ bpi, const bf16* __restrict__ wv,
                    const float* __restrict__ bv, int n, int A, float* __restrict__ logits, float* __restrict__ values,
                    uint64_t seed, const uint64_t* __restrict__ step_base, uint32_t t, const int32_t* __restrict__ forced,
-                   int32_t* __restrict__ actions, int32_t* __restrict__ sampled, float* __restrict__ uniforms) {
+                   int32_t* __restrict__ actions, int32_t* __restrict__ sampled, float* __restrict__ uniforms, HeadMode mode) {
   constexpr int EPL = 16, F = 32 * EPL;
   __shared__ uint4 wsh[33 * 64];                     // row k: 64 chunks of 8 bf16; row A = value head
   const int lane = threadIdx.x & 31;
@@ -192,29 +171,8 @@ heads_fused_kernel(const float* __restrict__ part, int splits, const float* __re
     }
   }
   v = warp_sum(v) + bv[0];
-  if (lane < A) logits[(size_t)e * A + lane] = z;
-  if (lane == 0) values[e] = v;
-  if (actions == nullptr) return;
-
-  const float m = warp_max(z);
-  const float ex = lane < A ? expf(z - m) : 0.f;
-  const float lse = m + logf(warp_sum(ex));
-  const float p = lane < A ? expf(z - lse) : 0.f;
-  const uint64_t step = *step_base + t;
-  const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
-  float c = 0.f;
-  int a = A - 1;
-  bool found = false;
-  for (int k = 0; k < A; ++k) {
-    c += __shfl_sync(0xffffffffu, p, k);
-    if (!found && u < c) { a = k; found = true; }
-  }
-  if (lane == 0) {
-    sampled[e] = a;
-    if (forced != nullptr && forced[e] >= 0) a = forced[e];
-    actions[e] = a;
-    uniforms[e] = u;
-  }
+  warp_finish_heads(mode, z, v, lane, A, (size_t)e, logits, values, actions != nullptr, seed,
+                    actions != nullptr ? *step_base + t : 0ull, forced, actions, sampled, uniforms);
 }
 
 // The tail of the heads for the cluster path of the fully connected layer, which has already taken the head dot
@@ -226,7 +184,7 @@ heads_sample_kernel(const float* __restrict__ hp, const float* __restrict__ bpi,
                     float* __restrict__ logits, float* __restrict__ values, uint64_t seed,
                     const uint64_t* __restrict__ step_base, uint32_t t, const int32_t* __restrict__ forced,
                     int32_t* __restrict__ actions, int32_t* __restrict__ sampled, float* __restrict__ uniforms,
-                    uint64_t* advance_step, uint32_t advance_by) {
+                    uint64_t* advance_step, uint32_t advance_by, HeadMode mode) {
   const int lane = threadIdx.x & 31;
   const int e = blockIdx.x * HS_WARPS + (threadIdx.x >> 5);
   const float b = lane < A ? __ldg(bpi + lane) : (lane == A ? __ldg(bv) : 0.f);     // biases are older than the previous kernel
@@ -237,29 +195,8 @@ heads_sample_kernel(const float* __restrict__ hp, const float* __restrict__ bpi,
   float s = -INFINITY;
   if (lane <= A) s = (hp[(size_t)e * HS_LD + lane] + hp[((size_t)n + e) * HS_LD + lane]) + b;
   const float z = lane < A ? s : -INFINITY;
-  if (lane < A) logits[(size_t)e * A + lane] = z;
-  if (lane == A) values[e] = s;
-  if (actions == nullptr) return;
-
-  const float m = warp_max(z);
-  const float ex = lane < A ? expf(z - m) : 0.f;
-  const float lse = m + logf(warp_sum(ex));
-  const float p = lane < A ? expf(z - lse) : 0.f;
-  const uint64_t step = *step_base + t;
-  const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
-  float c = 0.f;
-  int a = A - 1;
-  bool found = false;
-  for (int k = 0; k < A; ++k) {
-    c += __shfl_sync(0xffffffffu, p, k);
-    if (!found && u < c) { a = k; found = true; }
-  }
-  if (lane == 0) {
-    sampled[e] = a;
-    if (forced != nullptr && forced[e] >= 0) a = forced[e];
-    actions[e] = a;
-    uniforms[e] = u;
-  }
+  warp_finish_heads(mode, z, __shfl_sync(0xffffffffu, s, A), lane, A, (size_t)e, logits, values, actions != nullptr, seed,
+                    actions != nullptr ? *step_base + t : 0ull, forced, actions, sampled, uniforms);
 }
 
 bool heads_fused_supported(const NetDims& nd) { return nd.F == 512 && nd.pi_w % 8 == 0 && nd.A <= 32; }
@@ -267,17 +204,17 @@ bool heads_fused_supported(const NetDims& nd) { return nd.F == 512 && nd.pi_w % 
 void launch_heads_fused(LaunchCtx& lc, const NetDims& nd, const float* theta, const bf16* theta16, const float* part,
                         int splits, bf16* h_out, int n, float* logits, float* values, uint64_t seed,
                         const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
-                        float* uniforms, uint64_t* advance_step, uint32_t advance_by) {
+                        float* uniforms, HeadMode mode, uint64_t* advance_step, uint32_t advance_by) {
   KernelScope scope(lc, KID_HEADS_FWD);
   if (splits == 0) {          // `part` holds the head dot products of the two halves of the hidden units
     launch_kernel_overlapped(lc, heads_sample_kernel, (n + HS_WARPS - 1) / HS_WARPS, HS_WARPS * 32, 0, part, theta + nd.pi_b,
                              theta + nd.v_b, n, nd.A, logits, values, seed, advance_step ? nullptr : step_base, t, forced,
-                             actions, sampled, uniforms, advance_step, advance_by);
+                             actions, sampled, uniforms, advance_step, advance_by, mode);
     return;
   }
   launch_kernel(lc, heads_fused_kernel, (n + HF_WARPS - 1) / HF_WARPS, HF_WARPS * 32, 0, part, splits, theta + nd.layer[nd.n_conv].b_off, h_out,
                 theta16 + nd.pi_w, theta + nd.pi_b, theta16 + nd.v_w, theta + nd.v_b, n, nd.A, logits, values, seed,
-                step_base, t, forced, actions, sampled, uniforms);
+                step_base, t, forced, actions, sampled, uniforms, mode);
 }
 
 // Element-wise variant of the heads kernel for layouts without 16-byte alignment and for float storage.
@@ -290,7 +227,7 @@ heads_slow_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const flo
              const TW* __restrict__ wv, const float* __restrict__ bv, int n, int F, int A,
              float* __restrict__ logits, float* __restrict__ values, uint64_t seed, const uint64_t* __restrict__ step_base, uint32_t t,
              const int32_t* __restrict__ forced, int32_t* __restrict__ actions, int32_t* __restrict__ sampled,
-             float* __restrict__ uniforms) {
+             float* __restrict__ uniforms, HeadMode mode) {
   pdl_entry();
   const int lane = threadIdx.x & 31;
   const int e = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -306,35 +243,14 @@ heads_slow_kernel(const T* __restrict__ h, const TW* __restrict__ wpi, const flo
   float v = 0.f;
   for (int i = lane; i < F; i += 32) v = fmaf(to_f(wv[i]), to_f(x[i]), v);
   v = warp_sum(v) + bv[0];
-  if (lane < A) logits[(size_t)e * A + lane] = z;
-  if (lane == 0) values[e] = v;
-  if (actions == nullptr) return;
-
-  const float m = warp_max(z);
-  const float ex = lane < A ? expf(z - m) : 0.f;
-  const float lse = m + logf(warp_sum(ex));
-  const float p = lane < A ? expf(z - lse) : 0.f;
-  const uint64_t step = *step_base + t;
-  const float u = philox_uniform((uint32_t)e, (uint32_t)step, (uint32_t)(step >> 32), RNG_STREAM_ACTION, seed);
-  float c = 0.f;
-  int a = A - 1;
-  bool found = false;
-  for (int k = 0; k < A; ++k) {
-    c += __shfl_sync(0xffffffffu, p, k);
-    if (!found && u < c) { a = k; found = true; }
-  }
-  if (lane == 0) {
-    sampled[e] = a;
-    if (forced != nullptr && forced[e] >= 0) a = forced[e];
-    actions[e] = a;
-    uniforms[e] = u;
-  }
+  warp_finish_heads(mode, z, v, lane, A, (size_t)e, logits, values, actions != nullptr, seed,
+                    actions != nullptr ? *step_base + t : 0ull, forced, actions, sampled, uniforms);
 }
 
 void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
                   const bf16* theta16, const void* h, int n, float* logits, float* values, uint64_t seed,
                   const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
-                  float* uniforms) {
+                  float* uniforms, HeadMode mode) {
   const int blocks = (n + 3) / 4;
   KernelScope scope(lc, KID_HEADS_FWD);
   cudaStream_t st = lc.st;
@@ -342,18 +258,18 @@ void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta
   const bool aligned = nd.pi_w % 8 == 0;      // 16-byte loads of the policy rows
   if (prec == PAAC_BF16 && nd.F == 512 && aligned)
     launch_kernel(lc, heads_kernel<bf16, bf16, 16>, blocks, 128, 0, (const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
-                                                         nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms);
+                                                         nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms, mode);
   else if (prec == PAAC_BF16 && nd.F == 256 && aligned)
     launch_kernel(lc, heads_kernel<bf16, bf16, 8>, blocks, 128, 0, (const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv, n,
-                                                        nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms);
+                                                        nd.A, logits, values, seed, step_base, t, forced, actions, sampled, uniforms, mode);
   else if (prec == PAAC_BF16)
     launch_kernel(lc, heads_slow_kernel<bf16, bf16>, blocks, 128, 0, (const bf16*)h, theta16 + nd.pi_w, bpi, theta16 + nd.v_w, bv,
                                                           n, nd.F, nd.A, logits, values, seed, step_base, t, forced, actions,
-                                                          sampled, uniforms);
+                                                          sampled, uniforms, mode);
   else
     launch_kernel(lc, heads_slow_kernel<float, float>, blocks, 128, 0, (const float*)h, theta + nd.pi_w, bpi, theta + nd.v_w, bv,
                                                             n, nd.F, nd.A, logits, values, seed, step_base, t, forced, actions,
-                                                            sampled, uniforms);
+                                                            sampled, uniforms, mode);
 }
 
 // One warp per experience i = (t, e).  Lane 0 first walks the environment's transitions backwards from the bootstrap
@@ -364,7 +280,7 @@ void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta
 // with adv and R constants, and the three per-sample loss terms.  The block that finishes last adds the loss terms
 // up in a fixed order (a reproducible mean) and resets the arrival counter for the next launch.
 __global__ void __launch_bounds__(128)
-returns_head_grad_kernel(int n_e, int t_max, int A, float gamma, float beta, float value_coef,
+returns_head_grad_kernel(int algo, int n_e, int t_max, int A, float gamma, float beta, float value_coef,
                          const int8_t* __restrict__ rewards, const uint8_t* __restrict__ terminals,
                          const float* __restrict__ logits, const float* __restrict__ values,
                          const int32_t* __restrict__ actions, float* __restrict__ R, float* __restrict__ adv,
@@ -410,17 +326,29 @@ returns_head_grad_kernel(int n_e, int t_max, int A, float gamma, float beta, flo
     const float H = -warp_sum(lane < A ? p * lp : 0.f);
     const int a = actions[i];
     const float invB = 1.0f / (float)B;
-    if (lane < A) {
-      const float g = -ad * ((lane == a ? 1.f : 0.f) - p) + beta * p * (lp + H);
-      dz[(size_t)i * A + lane] = g * invB;
-    }
-    const float lp_a = __shfl_sync(0xffffffffu, lp, a);
-    if (lane == 0) {
-      const float d = values[i] - ret;
-      dV[i] = 2.f * value_coef * d * invB;
-      wsum[0][threadIdx.x >> 5] = -ad * lp_a;
-      wsum[1][threadIdx.x >> 5] = value_coef * d * d;
-      wsum[2][threadIdx.x >> 5] = H;
+    if (algo == PAAC_ALGO_NSTEP_Q) {
+      // value-based variant: L = value_coef (R - Q(s, a))^2, R constant; only the taken action's output has a gradient
+      const float d = __shfl_sync(0xffffffffu, z, a) - ret;
+      if (lane < A) dz[(size_t)i * A + lane] = lane == a ? 2.f * value_coef * d * invB : 0.f;
+      if (lane == 0) {
+        dV[i] = 0.f;
+        wsum[0][threadIdx.x >> 5] = 0.f;
+        wsum[1][threadIdx.x >> 5] = value_coef * d * d;
+        wsum[2][threadIdx.x >> 5] = 0.f;
+      }
+    } else {
+      if (lane < A) {
+        const float g = -ad * ((lane == a ? 1.f : 0.f) - p) + beta * p * (lp + H);
+        dz[(size_t)i * A + lane] = g * invB;
+      }
+      const float lp_a = __shfl_sync(0xffffffffu, lp, a);
+      if (lane == 0) {
+        const float d = values[i] - ret;
+        dV[i] = 2.f * value_coef * d * invB;
+        wsum[0][threadIdx.x >> 5] = -ad * lp_a;
+        wsum[1][threadIdx.x >> 5] = value_coef * d * d;
+        wsum[2][threadIdx.x >> 5] = H;
+      }
     }
   } else if (lane == 0) {
     for (int j = 0; j < 3; ++j) wsum[j][threadIdx.x >> 5] = 0.f;
@@ -454,13 +382,13 @@ returns_head_grad_kernel(int n_e, int t_max, int A, float gamma, float beta, flo
   }
 }
 
-void launch_returns_head_grad(LaunchCtx& lc, int n_e, int t_max, int A, float gamma, float beta, float value_coef,
+void launch_returns_head_grad(LaunchCtx& lc, HeadMode mode, int n_e, int t_max, int A, float gamma, float beta, float value_coef,
                               const int8_t* rewards, const uint8_t* terminals, const float* logits, const float* values,
                               const int32_t* actions, float* R, float* adv, float* dz, float* dV, float* loss_terms,
                               DeviceStats* stats) {
   const int B = n_e * t_max;
   KernelScope scope(lc, KID_HEAD_GRAD);
-  launch_kernel(lc, returns_head_grad_kernel, (B + 3) / 4, 128, 0, n_e, t_max, A, gamma, beta, value_coef, rewards, terminals,
+  launch_kernel(lc, returns_head_grad_kernel, (B + 3) / 4, 128, 0, mode.algo, n_e, t_max, A, gamma, beta, value_coef, rewards, terminals,
                 logits, values, actions, R, adv, dz, dV, loss_terms, stats);
 }
 

@@ -18,6 +18,7 @@ void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step
 struct HeadsTail {
   const float* hp; const float* bpi; const float* bv; int A;
   float* logits; float* values; const int32_t* forced; int32_t* actions; int32_t* sampled; float* uniforms;
+  HeadMode mode;
 };
 // the same step with the action taken inside the kernel, from the heads' partial sums
 void launch_env_step_sampling(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step_base, uint32_t t, uint32_t term_denom,
@@ -85,18 +86,19 @@ void simt_backward_layer(LaunchCtx& lc, int arch, int prec, const NetDims& nd, c
 void launch_heads(LaunchCtx& lc, int prec, const NetDims& nd, const float* theta,
                   const bf16* theta16, const void* h, int n, float* logits, float* values, uint64_t seed,
                   const uint64_t* step_base /* device */, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled /* action before forcing */,
-                  float* uniforms);
+                  float* uniforms, HeadMode mode);
 // the same for the tensor-core path, which leaves the fully connected layer as split-k partial sums
 // part[split][n][F]: finishes h (sum, bias, ReLU, bf16) into h_out on the way
 bool heads_fused_supported(const NetDims& nd);
 void launch_heads_fused(LaunchCtx& lc, const NetDims& nd, const float* theta, const bf16* theta16, const float* part,
                         int splits, bf16* h_out, int n, float* logits, float* values, uint64_t seed,
                         const uint64_t* step_base, uint32_t t, const int32_t* forced, int32_t* actions, int32_t* sampled,
-                        float* uniforms, uint64_t* advance_step = nullptr, uint32_t advance_by = 0);
+                        float* uniforms, HeadMode mode, uint64_t* advance_step = nullptr, uint32_t advance_by = 0);
 // advance_step (only honoured with splits == 0, only valid without sampling): the kernel also adds advance_by to the
 // environments' step index, which saves the rollout its last launch
 // n-step returns and advantages, the loss gradient at the heads and the loss statistics, in one launch
-void launch_returns_head_grad(LaunchCtx& lc, int n_e, int t_max, int A, float gamma, float beta, float value_coef,
+// mode.algo == PAAC_ALGO_NSTEP_Q: the loss is value_coef * (R - Q(s, a))^2 instead (dV = 0, no policy or entropy term)
+void launch_returns_head_grad(LaunchCtx& lc, HeadMode mode, int n_e, int t_max, int A, float gamma, float beta, float value_coef,
                               const int8_t* rewards, const uint8_t* terminals, const float* logits, const float* values,
                               const int32_t* actions, float* R, float* adv, float* dz, float* dV,
                               float* loss_terms /* [3][B] */, DeviceStats* stats);

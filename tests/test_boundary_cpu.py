@@ -22,7 +22,8 @@ def test_library_builds_and_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_header():
-    assert C.sizeof(pb.HParams) == 64 and pb.HParams.workspace.offset == 40 and pb.HParams.stream.offset == 56
+    assert C.sizeof(pb.HParams) == 72 and pb.HParams.workspace.offset == 40 and pb.HParams.stream.offset == 56
+    assert pb.HParams.algorithm.offset == 64 and pb.HParams.epsilon.offset == 68
     assert C.sizeof(pb.UpdateStats) == 32 and pb.UpdateStats.timesteps.offset == 24
     assert C.sizeof(pb.RolloutView) == 64
 
@@ -33,6 +34,7 @@ def test_defaults_are_the_papers_hyperparameters():
     want = (0.99, 0.0224, 0.99, 0.1, 40.0, 0.01, 1.0)
     assert all(abs(a - b) < 1e-7 for a, b in zip(got, want))
     assert hp.term_denom == 200 and hp.precision == pb.FP32
+    assert hp.algorithm == pb.ALGO_A2C and abs(hp.epsilon - 0.1) < 1e-7
 
 
 def test_workspace_sizing_and_argument_checks():
@@ -56,8 +58,8 @@ def test_null_handles_and_strerror():
     assert L.paac_update(None, None) == pb.ERR_ARG
     assert L.paac_destroy(None) == pb.ERR_ARG
     assert L.paac_param_count(None) == 0 and L.paac_debug_bytes(None, 0) == 0
-    names = {L.paac_strerror(i) for i in range(8)}
-    assert len(names) == 8 and L.paac_strerror(99) == b"unknown status"
+    names = {L.paac_strerror(i) for i in range(9)}
+    assert len(names) == 9 and L.paac_strerror(99) == b"unknown status"
 
 
 def test_init_fails_loudly_without_a_gpu():

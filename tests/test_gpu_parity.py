@@ -366,3 +366,41 @@ def test_partial_tensor_core_weight_gradient_mask(orc):
         g.close()
     assert rel(grads[0][0], grads[1][0]) <= TOL["bf16"]
     assert abs(grads[0][2] - grads[1][2]) <= TOL["bf16"] * grads[0][2]
+
+
+@pytest.mark.parametrize("base,iters", [(0, 3), (2, 4)])
+def test_value_based_variant_matches_the_oracle(orc, base, iters):
+    """n-step Q-learning on the same framework (Section 2.2, Eqs. 2-4; Section 3), configurations 1 (float, CUDA
+    cores) and 3 (bf16, tensor cores): epsilon-greedy actions from the shared uniforms, Q(s_t, a_t) as the stored
+    value, max_a Q as the bootstrap, the Q-loss gradient, and the update, all against the oracle's variant."""
+    cfg = dict(CONFIGS[base], algorithm="nstep_q", epsilon=0.25)
+    prec = cfg["precision"]
+    o, g = make_pair(orc, cfg)
+    explored = 0
+    for it in range(iters):
+        if prec == "bf16":
+            resync(o, g)
+        ro, r1 = check_rollout(orc, o, g, TOL[prec])
+        explored += int((ro["uniforms"] < 0.25).sum())
+        # the stored values are the taken actions' Q-values, the last row the greedy value of the final states
+        T, n_e = cfg["t_max"], cfg["n_e"]
+        vals = g.debug_read(pb.DBG_VALUES).reshape(T + 1, n_e)
+        lg = g.debug_read(pb.DBG_LOGITS).reshape(T, n_e, -1)
+        acts = g.debug_read(pb.DBG_ACTIONS).reshape(T, n_e)
+        assert np.array_equal(vals[:T], np.take_along_axis(lg, acts[..., None], 2)[..., 0])
+        up, st, r2 = check_update(orc, o, g, TOL[prec], inject=(prec == "bf16" and it % 2 == 1))
+        assert st["policy_loss"] == 0.0 and st["entropy"] == 0.0
+        dz = g.debug_read(pb.DBG_DLOGITS).reshape(T * n_e, -1)
+        assert np.count_nonzero(dz) <= T * n_e and np.all(g.debug_read(pb.DBG_DVALUES) == 0)
+        if r2["flips"] == 0:
+            assert r2["theta"] <= TOL_PARAMS_10
+    assert explored > 0
+    g.close()
+
+
+def test_value_based_variant_bad_hyperparameters():
+    import ctypes as C
+    h = C.c_void_p()
+    for bad in (dict(algorithm=2), dict(algorithm=pb.ALGO_NSTEP_Q, epsilon=1.5), dict(algorithm=pb.ALGO_NSTEP_Q, epsilon=-0.1)):
+        hp = pb.default_hparams(**bad)
+        assert pb.lib().paac_init(C.byref(h), 0, 4, 5, 4, C.byref(hp), 1) == pb.ERR_ARG
