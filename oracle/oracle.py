@@ -161,6 +161,22 @@ def env_step(seed, step, actions, term_denom, counters, h=84, w=84):
     return f, r, t
 
 
+def preprocess(raw_prev, raw_last, state_in=None):
+    """Section 5.1 pre-processing: raw uint8 [n, 210, 160, 3] x 2 (+ previous state [n, 84, 84, 4]) -> state."""
+    raw_prev = np.ascontiguousarray(raw_prev, np.uint8)
+    raw_last = np.ascontiguousarray(raw_last, np.uint8)
+    n = raw_prev.shape[0]
+    assert raw_prev.shape == (n, 210, 160, 3) and raw_last.shape == raw_prev.shape
+    out = np.zeros((n, 84, 84, 4), np.uint8)
+    sin = None
+    if state_in is not None:
+        state_in = np.ascontiguousarray(state_in, np.uint8)
+        assert state_in.shape == out.shape
+        sin = _p(state_in)
+    lib().orc_preprocess(_p(raw_prev), _p(raw_last), sin, _p(out), n)
+    return out
+
+
 def _ptr_array(arrs):
     return (C.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
 

@@ -22,6 +22,8 @@
  *   softmax / sampling   sum-to-one, entropy bounds, shift invariance, brute force
  *   returns              closed form sum gamma^k r + gamma^n V, worked cases
  *   clip / RMSProp       closed forms
+ *   pre-processing       block means of an integer-upsampled image (independent definition),
+ *                        pure-colour and constant images, hand-computed rows, channel shift
  *   n-step Q variant     brute-force arg max and exploration branch, exploration frequency,
  *                        PyTorch autograd and central differences of the loss, hand case
  * The whole iteration has no printed value in the paper to compare with:
@@ -301,6 +303,64 @@ void orc_forward(const orc_net* net, const float* theta, int bf16, const uint8_t
       values[b] = (float)(acc + (double)bv[0]);
     }
   }
+}
+
+/* ------------------------------------------------------------------ */
+/* Frame pre-processing (Section 5.1): of the raw frames an action      */
+/* repeated four times produces, the per-pixel maximum of the two       */
+/* latest is kept, turned into one channel of pixel intensity, scaled   */
+/* from 210 x 160 down to 84 x 84, and becomes the newest of the four   */
+/* frames that make a state.  Readings where the paper is silent:       */
+/*  - the maximum is taken per colour channel, before the intensity;    */
+/*  - intensity = (77 R + 150 G + 29 B + 128) >> 8 (the 0.299 / 0.587 / */
+/*    0.114 luminance weights in 8-bit fixed point, rounded);           */
+/*  - scaling is the area average: output pixel (y, x) is the mean of   */
+/*    the source over [2.5 y, 2.5 (y+1)) x [160 x / 84, 160 (x+1) / 84),*/
+/*    every source pixel weighted by the area it shares with that box,  */
+/*    rounded half up; in integers, with lengths in units of 1/84 of a  */
+/*    source pixel, weights are overlap lengths and the total 210 * 160;*/
+/*  - a state's channels are its four latest frames, oldest first; with */
+/*    no previous state (after a reset) the new frame fills all four.   */
+/* raw_*: [n][210][160][3] uint8; state_*: [n][84][84][4] uint8.        */
+/* ------------------------------------------------------------------ */
+static int overlap(int a0, int a1, int b0, int b1) {
+  int lo = a0 > b0 ? a0 : b0, hi = a1 < b1 ? a1 : b1;
+  return hi > lo ? hi - lo : 0;
+}
+void orc_preprocess(const uint8_t* raw_prev, const uint8_t* raw_last, const uint8_t* state_in /* nullable */,
+                    uint8_t* state_out, int n) {
+  enum { SH = 210, SW = 160, OH = 84, OW = 84 };
+  uint8_t* grey = (uint8_t*)malloc((size_t)SH * SW);
+  for (int e = 0; e < n; ++e) {
+    const uint8_t* a = raw_prev + (size_t)e * SH * SW * 3;
+    const uint8_t* b = raw_last + (size_t)e * SH * SW * 3;
+    for (int p = 0; p < SH * SW; ++p) {
+      int c[3];
+      for (int k = 0; k < 3; ++k) c[k] = a[3 * p + k] > b[3 * p + k] ? a[3 * p + k] : b[3 * p + k];
+      grey[p] = (uint8_t)((77 * c[0] + 150 * c[1] + 29 * c[2] + 128) >> 8);
+    }
+    for (int y = 0; y < OH; ++y)
+      for (int x = 0; x < OW; ++x) {
+        long long acc = 0;
+        for (int r = 0; r < SH; ++r) {
+          int wy = overlap(SH * y, SH * (y + 1), OH * r, OH * (r + 1));
+          if (!wy) continue;
+          for (int cidx = 0; cidx < SW; ++cidx) {
+            int wx = overlap(SW * x, SW * (x + 1), OW * cidx, OW * (cidx + 1));
+            if (wx) acc += (long long)wy * wx * grey[r * SW + cidx];
+          }
+        }
+        uint8_t v = (uint8_t)((acc + (long long)SH * SW / 2) / ((long long)SH * SW));
+        size_t o = (((size_t)e * OH + y) * OW + x) * 4;
+        if (state_in) {
+          uint8_t c1 = state_in[o + 1], c2 = state_in[o + 2], c3 = state_in[o + 3];
+          state_out[o] = c1; state_out[o + 1] = c2; state_out[o + 2] = c3; state_out[o + 3] = v;
+        } else {
+          state_out[o] = state_out[o + 1] = state_out[o + 2] = state_out[o + 3] = v;
+        }
+      }
+  }
+  free(grey);
 }
 
 /* ------------------------------------------------------------------ */
