@@ -169,6 +169,22 @@ int paac_act_host(paac_ctx* ctx, int t, const uint8_t* frames /* host */, int32_
  * paac_update() may be called. */
 int paac_observe_host(paac_ctx* ctx, int t, const int8_t* rewards /* host */, const uint8_t* terminals /* host */);
 
+/* Frame pre-processing of Section 5.1 for real emulators feeding the external-environment mode: of the raw
+ * frames one (four times repeated) action produces, the two latest are combined by a per-pixel maximum, turned
+ * into pixel intensity, scaled from 210 x 160 to 84 x 84 and appended to the state as its newest channel.
+ * Readings where the paper is silent: the maximum is per colour channel; intensity = (77 R + 150 G + 29 B + 128) >> 8;
+ * the scaling is the exact area average (every source pixel weighted by the area it shares with the output
+ * pixel's box of 2.5 x 40/21 source pixels), rounded half up; channels of a state are its four latest frames,
+ * oldest first.
+ *   raw_prev, raw_last  device uint8 [n][210][160][3] (row, column, RGB), 16-byte aligned
+ *   state_in            device uint8 [n][84][84][4], nullable: the states before this step; NULL (after a reset):
+ *                       the new frame fills all four channels
+ *   state_out           device uint8 [n][84][84][4]; may be the same buffer as state_in
+ *   n in [1, 65535]; stream: cudaStream_t.  Asynchronous; allocates nothing.  Integer arithmetic: results are
+ *   the same bits on any machine. */
+int paac_preprocess(const uint8_t* raw_prev /* device */, const uint8_t* raw_last /* device */,
+                    const uint8_t* state_in /* device, nullable */, uint8_t* state_out /* device */, int n, void* stream);
+
 /* ---- test and resume hooks ---- */
 
 /* Overwrite the master parameters (and their bf16 copies) from the host. Synchronises.

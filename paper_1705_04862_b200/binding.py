@@ -49,7 +49,7 @@ class UpdateStats(C.Structure):
 EXPORTS = ["paac_default_hparams", "paac_workspace_bytes", "paac_init", "paac_rollout", "paac_update",
            "paac_param_count", "paac_params", "paac_destroy", "paac_strerror", "paac_act_host",
            "paac_observe_host", "paac_set_params", "paac_force_actions", "paac_debug_bytes", "paac_debug_read",
-           "paac_debug_write", "paac_debug_wait_probe", "paac_launch_count", "paac_profile", "paac_profile_read", "paac_set_option", "paac_clip_rmsprop_noalloc",
+           "paac_debug_write", "paac_debug_wait_probe", "paac_preprocess", "paac_launch_count", "paac_profile", "paac_profile_read", "paac_set_option", "paac_clip_rmsprop_noalloc",
            "paac_noalloc_max_params"]
 
 _lib = None
@@ -86,6 +86,7 @@ def lib():
         L.paac_debug_read.argtypes = [vp, i, vp, sz]
         L.paac_debug_write.argtypes = [vp, i, vp, sz]
         L.paac_debug_wait_probe.argtypes = [vp, C.c_uint32]
+        L.paac_preprocess.argtypes = [vp, vp, vp, vp, i, vp]
         L.paac_launch_count.argtypes = [vp]
         L.paac_launch_count.restype = u64
         L.paac_profile.argtypes = [vp, i]
@@ -140,6 +141,14 @@ def clip_rmsprop_noalloc(theta, rms, grad, n, lr, rms_decay, rms_eps, clip_norm,
         return None if x is None else (x if isinstance(x, int) else x.data_ptr())
     return int(lib().paac_clip_rmsprop_noalloc(addr(theta), addr(rms), addr(grad), addr(theta_bf16), n, lr, rms_decay,
                                                rms_eps, clip_norm, addr(norm_and_scale), addr(stream)))
+
+
+def preprocess(raw_prev, raw_last, state_in, state_out, n, stream=None):
+    """Section 5.1 pre-processing on device buffers (torch CUDA uint8 tensors or raw addresses): see paac_preprocess
+    in include/paac.h.  Returns the library status."""
+    def addr(x):
+        return None if x is None else (x if isinstance(x, int) else x.data_ptr())
+    return int(lib().paac_preprocess(addr(raw_prev), addr(raw_last), addr(state_in), addr(state_out), n, addr(stream)))
 
 
 class Paac:
