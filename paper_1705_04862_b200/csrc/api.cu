@@ -104,7 +104,7 @@ size_t carve(paac_ctx* c, char* base) {
   {
     // the tensor-core weight gradients keep their partial sums until the finishing kernel has run, so a layer that
     // is taken on the CUDA cores in the same update works in a region of its own behind them
-    size_t sc = simt_scratch_floats(c->arch, nd, (int)B);
+    size_t sc = simt_scratch_floats(c->arch, nd, (int)B, (int)n_e);
     c->simt_scratch_off = 0;
     if (tc_supported(c->arch, c->prec)) {
       c->simt_scratch_off = (tc_scratch_floats((int)B) + 63) / 64 * 64;
@@ -178,7 +178,7 @@ bool forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, Hea
     tc_forward(c->lc, c->arch, c->nd, c->theta, c->theta16, c->w_images, frames, c->n_e, act, c->scratch,
                &c->stats->error_word);
   else
-    simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act);
+    simt_forward(c->lc, c->arch, c->prec, c->nd, c->theta, c->theta16, frames, c->n_e, act, c->scratch + c->simt_scratch_off);
   launch_heads(c->lc, c->prec, c->nd, c->theta, c->theta16, act[c->nd.n_conv], c->n_e,
                c->logits + row * c->A, c->values + row, c->seed, c->step_dev, (uint32_t)slot, forced, actions, sampled,
                uniforms, head_mode(c));

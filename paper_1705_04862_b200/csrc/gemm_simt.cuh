@@ -143,6 +143,29 @@ template <class G, class T> struct ConvDgradOp {
     return to_f(g[((size_t)(b * G::OH + oh) * G::OW + ow) * G::CO + co]);
   }
 };
+// Stride-2, 4 x 4 kernel: the input pixels of parity class (py, px) = (y & 1, x & 1) are touched only by the four taps
+// (py + 2 i, px + 2 j), so each class is a dense contraction of its own with a quarter of the reduction length and
+// no structural zeros.  Row m = (state, y >> 1, x >> 1), k = (i, j, co).
+template <class G, class T> struct ConvDgradClassOp {
+  static constexpr bool K_CONTIG = true;
+  const T* g; int py, px;
+  __device__ __forceinline__ float operator()(int m, int k) const {
+    constexpr int HH = G::H / 2, WW = G::W / 2;
+    const int b = m / (HH * WW), rem = m % (HH * WW), yy = rem / WW, xx = rem % WW;
+    const int i = k / (2 * G::CO), j = (k / G::CO) & 1, co = k % G::CO;
+    const int oh = yy - i, ow = xx - j;                       // ((2 yy + py) - (py + 2 i)) / 2
+    if (oh < 0 || ow < 0 || oh >= G::OH || ow >= G::OW) return 0.f;
+    return to_f(g[((size_t)(b * G::OH + oh) * G::OW + ow) * G::CO + co]);
+  }
+};
+template <class G, class T> struct ConvWeightClassOp {        // row ci, k = (i, j, co) -> tap (py + 2 i, px + 2 j)
+  static constexpr bool K_CONTIG = true;
+  const T* w; int py, px;
+  __device__ __forceinline__ float operator()(int ci, int k) const {
+    const int i = k / (2 * G::CO), j = (k / G::CO) & 1, co = k % G::CO;
+    return to_f(w[((size_t)(co * G::K + py + 2 * i) * G::K + px + 2 * j) * G::C + ci]);
+  }
+};
 // weights seen from the data gradient: row ci, k = (r, s, co)
 template <class G, class T> struct ConvWeightTOp {
   static constexpr bool K_CONTIG = true;
@@ -167,6 +190,16 @@ template <class T> struct ReluMaskEp {
   T* out; const T* act; int ld;
   __device__ __forceinline__ void operator()(int m, int n, float acc, int) const {
     const size_t i = (size_t)m * ld + n;
+    out[i] = to_f(act[i]) > 0.f ? from_f<T>(acc) : from_f<T>(0.f);
+  }
+};
+// the same for one parity class of a stride-2 layer: row m = (state, y >> 1, x >> 1) -> pixel (2 yy + py, 2 xx + px)
+template <class G, class T> struct ReluMaskClassEp {
+  T* out; const T* act; int py, px;
+  __device__ __forceinline__ void operator()(int m, int n, float acc, int) const {
+    constexpr int HH = G::H / 2, WW = G::W / 2;
+    const int b = m / (HH * WW), rem = m % (HH * WW), yy = rem / WW, xx = rem % WW;
+    const size_t i = ((size_t)(b * G::H + 2 * yy + py) * G::W + 2 * xx + px) * G::C + n;
     out[i] = to_f(act[i]) > 0.f ? from_f<T>(acc) : from_f<T>(0.f);
   }
 };

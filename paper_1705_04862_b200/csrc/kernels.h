@@ -29,14 +29,15 @@ void launch_advance_step(LaunchCtx& lc, uint64_t* step_base, uint32_t by);
 
 // ---- network on the CUDA cores (net_simt.cu) --------------------------------------------
 // act[l]: stored activation of layer l for the n states, storage float (PAAC_FP32) or bf16
+// scratch: simt_scratch_floats() floats for the split-k partial sums of the fully connected layer (nullptr: no split)
 void simt_forward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
-                  const bf16* theta16, const uint8_t* frames, int n, void* const act[]);
+                  const bf16* theta16, const uint8_t* frames, int n, void* const act[], float* scratch);
 // from gact[fc] (gradient at the fc pre-activation) down to conv1; fills grad for conv and fc layers
 void simt_backward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
                    const bf16* theta16, const uint8_t* frames, int n, void* const act[], void* const gact[],
                    float* grad, float* scratch);
-// scratch floats simt_backward / heads_backward need for split-k partials
-size_t simt_scratch_floats(int arch, const NetDims& nd, int n);
+// scratch floats simt_backward / heads_backward (n states) and simt_forward (n_fwd states) need for split-k partials
+size_t simt_scratch_floats(int arch, const NetDims& nd, int n, int n_fwd);
 
 // ---- network on the tensor cores (net_tc.cu): Nature CNN, bf16 ------------------------------
 bool tc_supported(int arch, int prec);

@@ -31,13 +31,46 @@ static void conv_fwd(LaunchCtx& lc, int kid, const TIn* x, const TW* w, const fl
   gemm_simt(lc, kid, n * G::OH * G::OW, G::CO, G::KK, 1, ConvWindowOp<G, TIn>{x}, RowMajorOp<TW>{w, G::KK},
             BiasReluEp<T>{out, bias, G::CO, scale});
 }
+// out[m][n] = relu(sum over splits (in order) of part[split][m][n] + bias[n])
+template <class T>
+static __global__ void fc_finish_simt_kernel(const float* __restrict__ part, int splits, int M, int N,
+                                             const float* __restrict__ bias, T* __restrict__ out) {
+  pdl_entry();
+  const size_t total = (size_t)M * N;
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+    // the partial sums are added in double: the pre-activation then differs from an exactly rounded one only by the
+    // error inside each short partial sum, and fewer units near zero end up on the other side of the ReLU
+    double s = 0.0;
+    for (int p = 0; p < splits; ++p) s += (double)part[(size_t)p * total + i];
+    out[i] = from_f<T>(fmaxf((float)(s + (double)bias[i % N]), 0.f));
+  }
+}
+// With few states the fully connected layer is a handful of 64 x 64 tiles over a reduction of thousands: the
+// reduction is then split over many blocks (partial sums in scratch, added in a fixed order by a finishing kernel)
+// so that the weight matrix is streamed by the whole device instead of by four blocks.
 template <class T, class TW>
 static void fc_fwd(LaunchCtx& lc, int kid, const T* x, const TW* w, const float* bias, T* out, int n,
-                   int IN, int F) {
-  gemm_simt(lc, kid, n, F, IN, 1, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, BiasReluEp<T>{out, bias, F, 1.f});
+                   int IN, int F, float* scratch) {
+  const int splits = scratch != nullptr ? pick_splits(n, F, IN) : 1;
+  if (splits <= 1) {
+    gemm_simt(lc, kid, n, F, IN, 1, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, BiasReluEp<T>{out, bias, F, 1.f});
+    return;
+  }
+  gemm_simt(lc, kid, n, F, IN, splits, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, PartialEp{scratch, n, F});
+  KernelScope scope(lc, kid);
+  int blocks = (n * F + 255) / 256;
+  if (blocks > 1184) blocks = 1184;
+  launch_kernel(lc, fc_finish_simt_kernel<T>, blocks, 256, 0, scratch, splits, n, F, bias, out);
 }
 template <class G, class T, class TW>
 static void conv_dgrad(LaunchCtx& lc, int kid, const T* g, const TW* w, const T* act_in, T* gin, int n) {
+  if constexpr (G::S == 2 && G::K == 4 && G::H % 2 == 0 && G::W % 2 == 0) {
+    // four parity classes, each a dense contraction over its own four taps (a quarter of the multiply-adds)
+    for (int z = 0; z < 4; ++z)
+      gemm_simt(lc, kid, n * (G::H / 2) * (G::W / 2), G::C, 4 * G::CO, 1, ConvDgradClassOp<G, T>{g, z >> 1, z & 1},
+                ConvWeightClassOp<G, TW>{w, z >> 1, z & 1}, ReluMaskClassEp<G, T>{gin, act_in, z >> 1, z & 1});
+    return;
+  }
   gemm_simt(lc, kid, n * G::H * G::W, G::C, G::K * G::K * G::CO, 1, ConvDgradOp<G, T>{g}, ConvWeightTOp<G, TW>{w},
             ReluMaskEp<T>{gin, act_in, G::C});
 }
@@ -65,18 +98,18 @@ static void fc_wgrad(LaunchCtx& lc, int kid, const T* g, const T* x, int n, int 
 
 template <class T, class TW>
 static void forward_t(LaunchCtx& lc, int arch, const NetDims& nd, const float* theta, const TW* w,
-                      const uint8_t* frames, int n, void* const act[]) {
+                      const uint8_t* frames, int n, void* const act[], float* scratch) {
   const LayerDims* d = nd.layer;
   const float s255 = 1.0f / 255.0f;
   if (arch == PAAC_ARCH_NIPS) {
     conv_fwd<NipsConv1, uint8_t, T, TW>(lc, KID_CONV1_FWD, frames, w + d[0].w_off, theta + d[0].b_off, (T*)act[0], n, s255);
     conv_fwd<NipsConv2, T, T, TW>(lc, KID_CONV2_FWD, (const T*)act[0], w + d[1].w_off, theta + d[1].b_off, (T*)act[1], n, 1.f);
-    fc_fwd<T, TW>(lc, KID_FC_FWD, (const T*)act[1], w + d[2].w_off, theta + d[2].b_off, (T*)act[2], n, 2592, 256);
+    fc_fwd<T, TW>(lc, KID_FC_FWD, (const T*)act[1], w + d[2].w_off, theta + d[2].b_off, (T*)act[2], n, 2592, 256, scratch);
   } else {
     conv_fwd<NatConv1, uint8_t, T, TW>(lc, KID_CONV1_FWD, frames, w + d[0].w_off, theta + d[0].b_off, (T*)act[0], n, s255);
     conv_fwd<NatConv2, T, T, TW>(lc, KID_CONV2_FWD, (const T*)act[0], w + d[1].w_off, theta + d[1].b_off, (T*)act[1], n, 1.f);
     conv_fwd<NatConv3, T, T, TW>(lc, KID_CONV3_FWD, (const T*)act[1], w + d[2].w_off, theta + d[2].b_off, (T*)act[2], n, 1.f);
-    fc_fwd<T, TW>(lc, KID_FC_FWD, (const T*)act[2], w + d[3].w_off, theta + d[3].b_off, (T*)act[3], n, 3136, 512);
+    fc_fwd<T, TW>(lc, KID_FC_FWD, (const T*)act[2], w + d[3].w_off, theta + d[3].b_off, (T*)act[3], n, 3136, 512, scratch);
   }
 }
 
@@ -128,9 +161,9 @@ void simt_backward_layer(LaunchCtx& lc, int arch, int prec, const NetDims& nd, c
 }
 
 void simt_forward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
-                  const bf16* theta16, const uint8_t* frames, int n, void* const act[]) {
-  if (prec == PAAC_BF16) forward_t<bf16, bf16>(lc, arch, nd, theta, theta16, frames, n, act);
-  else forward_t<float, float>(lc, arch, nd, theta, theta, frames, n, act);
+                  const bf16* theta16, const uint8_t* frames, int n, void* const act[], float* scratch) {
+  if (prec == PAAC_BF16) forward_t<bf16, bf16>(lc, arch, nd, theta, theta16, frames, n, act, scratch);
+  else forward_t<float, float>(lc, arch, nd, theta, theta, frames, n, act, scratch);
 }
 
 void simt_backward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const float* theta,
@@ -140,7 +173,7 @@ void simt_backward(LaunchCtx& lc, int arch, int prec, const NetDims& nd, const f
     simt_backward_layer(lc, arch, prec, nd, theta, theta16, frames, n, act, gact, grad, scratch, l, true, l > 0);
 }
 
-size_t simt_scratch_floats(int arch, const NetDims& nd, int n) {
+size_t simt_scratch_floats(int arch, const NetDims& nd, int n, int n_fwd) {
   size_t best = 0;
   for (int l = 0; l <= nd.n_conv; ++l) {
     const LayerDims& d = nd.layer[l];
@@ -152,7 +185,11 @@ size_t simt_scratch_floats(int arch, const NetDims& nd, int n) {
   }
   const size_t heads = (size_t)pick_splits(nd.A + 1, nd.F + 1, n) * (nd.A + 1) * (nd.F + 1);
   (void)arch;
-  return best > heads ? best : heads;
+  if (heads > best) best = heads;
+  // split-k partial sums of the fully connected layer's forward pass, which only ever sees n_fwd states at a time
+  const LayerDims& f = nd.layer[nd.n_conv];
+  const size_t fwd = (size_t)pick_splits(n_fwd, nd.F, f.H * f.W * f.C) * n_fwd * nd.F;
+  return best > fwd ? best : fwd;
 }
 
 // ---- heads backward (tiny contractions over the A+1 head units) ------------------------------
