@@ -973,10 +973,6 @@ struct C3DgradCfg {
   }
   __host__ __device__ static constexpr int tap_plane(int) { return 0; }
   __host__ __device__ static constexpr int tap_shift(int t) { return (2 - t / 3) * 11 + (2 - t % 3); }
-  // tap pairs one raster position apart, by rising shift: kernel row r = 2 - j / 2; (s = 2, s = 1) and s = 0 alone
-  static constexpr int NSTEP = 6;
-  __host__ __device__ static constexpr int step_lo(int j) { return 3 * (2 - j / 2) + ((j & 1) ? 0 : 2); }
-  __host__ __device__ static constexpr int step_hi(int j) { return (j & 1) ? -1 : 3 * (2 - j / 2) + 1; }
 };
 // conv2 data gradient (all four parity classes along N): the 9 x 9 x 64 gradient on a zero-padded 11 x 11
 // raster; class pixel (yy, xx) is position 11 yy + xx and tap (i, j) reads (1 - i) * 11 + (1 - j) rows down
@@ -1084,10 +1080,15 @@ template <class Map> struct ShiftReluMaskEpiS2 {
 // tile yields 127 positions and tiles advance by 127.  The finished bf16 values are parked position-major in a staging
 // tile (128 bytes per position) and leave with whole-row stores, as in tc_shift_kernel.
 // Cfg adds: NSTEP, step_lo(j), step_hi(j) (tap indices, -1 = none; shift(hi) = shift(lo) + 1, same plane).
-// Roles: warps 0-7 epilogue (warp e: TMEM lane quarter e & 3, columns 64 (e >> 2) ..), warps 8-15 producers,
-// warp 16 issues the MMAs.  Warps 0-3 also write the weights into tensor memory before the first tile.
+// Roles: warps 0-15 epilogue (warp e: TMEM lane quarter e & 3, columns 32 (e >> 2) ..), warp 16 issues the MMAs, one
+// thread of warp 17 asks the copy engine for the stages.  Warps 0-3 also write the weights into tensor memory before
+// the first tile.  Forward layers only: with a masked epilogue and gathered stages (the data gradients) this
+// arrangement measured slower than tc_shift_kernel -- eight warps are too few for the transposing epilogue and
+// twenty-four warps in all too many for the SM's issue slots (71 and 77 us against 64 us for the conv3 data gradient),
+// and a zero-padded raster fetched as one tiled box per raster row made the producer the bottleneck (a tiled copy
+// costs its issuing warp about 80 cycles whatever its size).
 constexpr int ST_TILE = 127;
-constexpr int ST_THREADS = 576;      // warps 0-7 (0-15 with bulk-copied stages) epilogue, 8-15 producers otherwise, 16 MMA, 17 bulk producer
+constexpr int ST_THREADS = 576;      // warps 0-15 epilogue, 16 MMA, 17 bulk-copy producer
 
 __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
@@ -1137,17 +1138,16 @@ __global__ void __launch_bounds__(ST_THREADS, 1)
 tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b, Cfg cfg, const bf16* __restrict__ w,
                   Epi epi, int tiles, uint32_t* error_word) {
   static_assert(STAGES >= 2 && STAGES <= 8 && Cfg::STAGE_ROWS % 8 == 0, "pipeline shape");
+  static_assert(Cfg::BULK != 0 && !Epi::MASK, "forward layers with bulk-copied stages");
   constexpr int NT = Cfg::NT, NS = Cfg::NSTEP, SR = Cfg::STAGE_ROWS, PLANES = Cfg::PLANES;
   constexpr uint32_t PLANE_BYTES = SR * 128, STAGE_BYTES = PLANES * PLANE_BYTES, STG_BYTES = 128 * 128;
   constexpr uint32_t ACC_COLS = 128, A_COL0 = 2 * ACC_COLS, TMEM_COLS = 512;
-  // bulk-copied stages need one producer thread (warp 17), so warps 8-15 join the epilogue there
-  constexpr int EW = Cfg::BULK != 0 ? 16 : 8, ROWS_PER_WARP = 128 / EW;
+  constexpr int EW = 16, ROWS_PER_WARP = 128 / EW;                         // epilogue warps
   static_assert(A_COL0 + NS * 32 <= TMEM_COLS, "tensor memory budget: two accumulators and the weights");
   extern __shared__ uint8_t dyn_smem[];
   __shared__ PkShared sh;
   const uint32_t a_base0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;          // operand stages
   const uint32_t stg0 = a_base0 + STAGES * STAGE_BYTES;                    // two staging tiles (tile parity)
-  const uint32_t mring0 = stg0 + 2 * STG_BYTES;                            // masked epilogues: two slots of activations
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
@@ -1158,8 +1158,7 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
     //            arrival made here);
     //   empty[s] ("done"):  the tile's instructions have completed: the producer may refill the slot and the
     //            epilogue may read the accumulator.
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], (Cfg::BULK != 0 ? 1 : 256) + EW); mbar_init(&sh.empty[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sh.mask_full[i], 256); mbar_init(&sh.mask_empty[i], 8); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sh.full[s], 1 + EW); mbar_init(&sh.empty[s], 1); }
     for (int s = 0; s < 2; ++s)
       for (int e = 0; e < EW; ++e) mbar_arrive(&sh.full[s]);
     sh.abort = 0u;
@@ -1199,9 +1198,8 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
   tcgen05_fence_after();
   pdl_entry();          // everything above touches only this CTA's own resources and weights that are several kernels old
 
-  if (Cfg::BULK != 0 && warp == 17) {
+  if (warp == 17) {
     // ---------------- producer: a stage is one box of the layer input per plane (tiled bulk copies) ----------------
-    static_assert(Cfg::BULK == 0 || !Epi::MASK, "bulk-copied stages: plain forward layers only");
     if (lane == 0) {
       tma_prefetch_desc(&tm_a);
       if (Cfg::BULK == 2) tma_prefetch_desc(&tm_b);
@@ -1218,71 +1216,12 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
         }
       }
     }
-  } else if (Cfg::BULK == 0 && warp >= 8 && warp < 16) {
-    // ---------------- producers: eight lanes per 128-byte row, 32 rows per pass ----------------
-    const int c = lane & 7, sub = (warp - 8) * 4 + (lane >> 3);
-    int it = 0;
-    bool alive = true;
-    for (int t = blockIdx.x; t < tiles && alive; t += gridDim.x, ++it) {
-      const int s = it % STAGES;
-      const bool ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
-      if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
-      const uint32_t stage = a_base0 + s * STAGE_BYTES;
-      // source addresses by arithmetic only, all of them before the first copy (a warp with asynchronous copies in
-      // flight waits for all of them at its next shared-memory load)
-      constexpr int NIT = (PLANES * SR + 31) / 32;
-      uint32_t srcs[NIT], vmask = 0;                    // element offsets from the tensor's base (< 2^32 elements)
-#pragma unroll
-      for (int k = 0; k < NIT; ++k) {
-        const int idx = sub + 32 * k;
-        srcs[k] = 0u;
-        if (idx < PLANES * SR) {
-          const int plane = PLANES == 1 ? 0 : idx / SR, ri = PLANES == 1 ? idx : idx % SR;
-          bool valid;
-          const bf16* ptr;
-          if constexpr (Cfg::RASTER > 0) ptr = cfg.src_cell(t * ST_TILE + ri, valid);
-          else ptr = cfg.src(plane, t * ST_TILE + ri, valid);
-          srcs[k] = (uint32_t)(ptr - cfg.base());
-          vmask |= valid ? 1u << k : 0u;
-        }
-      }
-#pragma unroll
-      for (int k = 0; k < NIT; ++k) {
-        const int idx = sub + 32 * k;
-        if (idx < PLANES * SR) {
-          const int plane = PLANES == 1 ? 0 : idx / SR, ri = PLANES == 1 ? idx : idx % SR;
-          cp_async16(stage + plane * PLANE_BYTES + ri * 128u + ((uint32_t)(c ^ (ri & 7)) << 4), cfg.base() + srcs[k] + c * 8,
-                     (vmask >> k) & 1u ? 16u : 0u);
-        }
-      }
-      cp_async_mbar_arrive(&sh.full[s]);
-      if constexpr (Epi::MASK) {
-        // the activations under the tile (the ReLU mask of its epilogue): ring slot row r = position 127 t + r,
-        // laid out exactly as the staging tile the epilogue reads them against
-        const int ms = it & 1;
-        const bool okm = mbar_wait(&sh.mask_empty[ms], ((it >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
-        if (!__all_sync(0xffffffffu, okm)) { alive = false; break; }
-        const uint32_t dst = mring0 + ms * STG_BYTES;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int r = sub + 32 * k;
-          int b, y, x;
-          epi.map.split(t * ST_TILE + r, b, y, x);
-          const bool v = r < ST_TILE && epi.map.is_output(b, y, x);
-          cp_async16(dst + r * 128u + ((uint32_t)(c ^ ((r & 3) << 1)) << 4), epi.act + (v ? epi.index(b, y, x, c * 8) : 0u), v ? 16u : 0u);
-        }
-        cp_async_mbar_arrive(&sh.mask_full[ms]);
-      }
-    }
-    cp_async_commit();
-    cp_async_wait<0>();
   } else if (warp < EW) {
     // ---------------- epilogue: warp e reads TMEM lane quarter e & 3, columns (128 / (EW / 4)) * (e >> 2) .. ----------------
     const int quarter = warp & 3, grp = warp >> 2;
     constexpr int GCOLS = 128 / (EW / 4);                              // columns (= staging rows) of a group of four warps
     const int ch = 16 * quarter + (lane >> 1), par = lane & 1;          // this lane's channel and tap half
-    float bias = 0.f;
-    if constexpr (!Epi::MASK) bias = __ldg(epi.bias + ch);
+    const float bias = __ldg(epi.bias + ch);
     const int rr0 = lane >> 3, c16 = lane & 7;                          // second phase: row within a pass, 16-byte chunk
     bool dead = false;
     int local = 0;
@@ -1333,19 +1272,12 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
             const float mine = __uint_as_float(par ? (i < 15 ? r[2 * i + 2] : nxt) : r[2 * i]);
             const float v = (got + mine) + bias;
             uint16_t hv;
-            if constexpr (!Epi::MASK) asm("cvt.rn.relu.bf16.f32 %0, %1;" : "=h"(hv) : "f"(v));
-            else asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(hv) : "f"(v));
+            asm("cvt.rn.relu.bf16.f32 %0, %1;" : "=h"(hv) : "f"(v));                  // bias, ReLU and the bf16 rounding
             asm volatile("st.shared.b16 [%0], %1;" ::"r"(((i & 1) ? sb1 : sb0) + (uint32_t)(i * 256)), "h"(hv) : "memory");
           }
         }
       }
       group_barrier(1 + grp, 128);                                  // the GCOLS rows of this group are complete
-      if constexpr (Epi::MASK) {
-        if (!dead) {
-          const bool okm = mbar_wait(&sh.mask_full[local & 1], (local >> 1) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
-          if (!__all_sync(0xffffffffu, okm)) dead = true;
-        }
-      }
       if (!dead) {
 #pragma unroll
         for (int p = 0; p < ROWS_PER_WARP / 4; ++p) {
@@ -1353,18 +1285,8 @@ tc_shift_t_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constan
           const uint32_t off = rr * 128u + (((uint32_t)c16 ^ ((rr & 3u) << 1)) << 4);
           uint4 v;
           asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg + off) : "memory");
-          if constexpr (Epi::MASK) {
-            uint4 m;
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(m.x), "=r"(m.y), "=r"(m.z), "=r"(m.w)
-                         : "r"(mring0 + (local & 1) * STG_BYTES + off) : "memory");
-            v.x = mask_pair(v.x, m.x); v.y = mask_pair(v.y, m.y); v.z = mask_pair(v.z, m.z); v.w = mask_pair(v.w, m.w);
-          }
           if ((valid >> p) & 1u) *reinterpret_cast<uint4*>(epi.out + idx[p]) = v;
         }
-      }
-      if constexpr (Epi::MASK) {
-        __syncwarp();
-        if (!dead && lane == 0) mbar_arrive(&sh.mask_empty[local & 1]);
       }
     }
   } else if (warp == 16 && lane == 0) {
@@ -2202,7 +2124,7 @@ static void tc_shift(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int 
 
 template <class Cfg, class Epi, int STAGES>
 static void tc_shift_t(LaunchCtx& lc, int kid, Cfg cfg, const bf16* w, Epi e, int positions, uint32_t* err) {
-  constexpr int smem = STAGES * Cfg::PLANES * Cfg::STAGE_ROWS * 128 + 2 * 128 * 128 + (Epi::MASK ? 2 * 128 * 128 : 0) + 1024;
+  constexpr int smem = STAGES * Cfg::PLANES * Cfg::STAGE_ROWS * 128 + 2 * 128 * 128 + 1024;
   static_assert(smem <= 227 * 1024, "shared memory budget");
   static_assert(smem - 1024 >= Cfg::NSTEP * 128 * 128, "the weights pass through the stage area on their way to tensor memory");
   auto kern = tc_shift_t_kernel<Cfg, Epi, STAGES>;
@@ -3461,9 +3383,6 @@ void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* con
   typedef NatConv3 C3;
   const int M = n * C3::H * C3::W;
   typedef RasterMap<121, 11, 9, 9> Map;
-  // (the role-exchanged kernel also takes this layer -- tc_shift_t<C3DgradCfg, ShiftReluMaskEpi<Map, 9, 9>, 4> -- but with
-  // its stages fetched by eight cp.async warps only eight warps are left for the transposing epilogue, which then sets
-  // the pace: measured 71 us against 64 us for the kernel below)
   tc_shift<C3DgradCfg, ShiftReluMaskEpi<Map, 9, 9>, 64, 4, 1>(
       lc, KID_CONV3_DGRAD, C3DgradCfg{(const bf16*)gact[2], n}, images + 4 * 32 * 256,
       ShiftReluMaskEpi<Map, 9, 9>{Map{n}, (bf16*)gact[1], (const bf16*)act[1]}, n * 121, err);
