@@ -45,6 +45,7 @@ struct paac_ctx {
   void* act[MAX_LAYERS];   // [(t_max+1)*n_e][out_size], slot t_max is bootstrap scratch
   void* gact[MAX_LAYERS];  // [B][out_size]
   float *logits, *values, *uniforms, *R, *adv, *dz, *dV, *loss_terms, *scratch, *norm_partials;
+  float gact0_scale;       // power of two gact[0] was stored with by the last update (1 unless the tensor cores took both kernels)
   size_t simt_scratch_off; // floats: where the CUDA-core kernels' split-k scratch starts inside `scratch`
   int32_t *actions, *sampled, *forced, *counters;
   int8_t* rewards;
@@ -264,6 +265,7 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   if (!c) return PAAC_ERR_CUDA;
   fill_shape(c, arch, n_e, t_max, n_actions, hp);
   c->tc_wgrad_mask = 0xF;
+  c->gact0_scale = 1.f;
   c->graphs_on = true;
   c->seed = seed; c->device = dev; c->st = (cudaStream_t)hp->stream; c->lc.st = c->st;
   const size_t need = carve(c, nullptr);
@@ -340,13 +342,19 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
       heads_backward(c->lc, c->prec, c->nd, c->theta, c->theta16, c->act[L], c->B, c->dz, c->dV, c->gact[L],
                      c->grad, c->scratch + c->simt_scratch_off);
     uint32_t* err = &c->stats->error_word;
+    c->gact0_scale = 1.f;
     for (int l = L; l >= 0; --l) {
       // tensor-core kernels where they exist, the CUDA-core contraction otherwise
       bool dgrad_done = false;
       if (use_tc(c)) {
         if (l == 3) { tc_backward_dgrad_fc(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
         if (l == 2) { tc_backward_dgrad_conv3(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
-        if (l == 1) { tc_backward_dgrad_conv2(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
+        if (l == 1) {
+          // the first layer's tensor-core weight gradient takes its gradient operand times a power of two
+          c->gact0_scale = (c->tc_wgrad_mask & 1) ? tc_conv1_grad_scale() : 1.f;
+          tc_backward_dgrad_conv2(c->lc, c->w_images, c->B, c->act, c->gact, err, c->gact0_scale);
+          dgrad_done = true;
+        }
       }
       bool wgrad_done = false;
       if (use_tc(c) && (c->tc_wgrad_mask >> l) & 1) {
@@ -587,6 +595,19 @@ int paac_debug_read(paac_ctx* c, int which, void* dst, size_t bytes) {
   if (!p || b != bytes) return PAAC_ERR_ARG;
   if (cudaMemcpyAsync(dst, p, b, cudaMemcpyDeviceToHost, c->st) != cudaSuccess ||
       cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  if (which == PAAC_DBG_GACT0 && c->prec == PAAC_BF16 && c->gact0_scale != 1.f) {
+    // stored times a power of two for the first layer's weight-gradient kernel: hand out the gradient itself
+    uint16_t* h = (uint16_t*)dst;
+    const float inv = 1.f / c->gact0_scale;
+    for (size_t i = 0; i < b / 2; ++i) {
+      uint32_t u = (uint32_t)h[i] << 16;
+      float f;
+      memcpy(&f, &u, 4);
+      f *= inv;                                  // exact: a shift of the exponent (denormal results lose low bits)
+      memcpy(&u, &f, 4);
+      h[i] = (uint16_t)(u >> 16);
+    }
+  }
   return device_error(c);
 }
 

@@ -59,7 +59,11 @@ void tc_relayout_weights(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, 
 void launch_wait_probe(LaunchCtx& lc, uint32_t max_polls, uint32_t* error_word);
 void tc_backward_dgrad_fc(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err);
 void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err);
-void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err);
+// out_scale: power of two the gradient handed to the first layer is stored with (tc_conv1_grad_scale() when that
+// layer's weight gradient runs on the tensor cores, which expects it so; 1 otherwise)
+void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err,
+                             float out_scale);
+float tc_conv1_grad_scale();
 // weight + bias gradient of one layer (0 = conv1 .. 3 = fc) as split-k partial sums in its own region of a
 // scratch of tc_scratch_floats(B) floats; the regions are noted in a GradSegments list, and
 // tc_backward_finish() adds them up into the gradient vector with one launch and empties the list

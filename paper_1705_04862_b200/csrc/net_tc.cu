@@ -1055,11 +1055,16 @@ template <class Map, int OUT_H, int OUT_W> struct ShiftReluMaskEpi {
   }
 };
 // stride-2 data gradient: accumulator columns 32 c .. 32 c + 31 are parity class c of raster pixel (yy, xx)
+// `scale` is a power of two the stored gradient is multiplied by before its bf16 rounding (an exact shift of the
+// exponent): the first layer's weight-gradient kernel wants its gradient operand that way (see C1_GRAD_SCALE)
 template <class Map> struct ShiftReluMaskEpiS2 {
   static constexpr bool MASK = true;
   static constexpr int SX = 2 * 32, SY = 2 * 20 * 32, SB = 20 * 20 * 32;
-  Map map; bf16* out; const bf16* act;
-  __device__ __forceinline__ void values(int, const uint32_t (&r)[32], uint32_t (&o)[16]) const { plain_bf16_values(r, o); }
+  Map map; bf16* out; const bf16* act; float scale;
+  __device__ __forceinline__ void values(int, const uint32_t (&r)[32], uint32_t (&o)[16]) const {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) o[j] = pack_bf16x2(__uint_as_float(r[2 * j]) * scale, __uint_as_float(r[2 * j + 1]) * scale);
+  }
   __device__ __forceinline__ uint32_t index(int b, int yy, int xx, int col) const {
     const int cls = col >> 5;
     return (uint32_t)(((b * 20 + 2 * yy + (cls >> 1)) * 20 + 2 * xx + (cls & 1)) * 32 + (col & 31));
@@ -1785,6 +1790,15 @@ __device__ __forceinline__ void u8x4_to_f16x4(uint32_t w, uint32_t& lo, uint32_t
   hi = __byte_perm(w, 0u, 0x4342);
 }
 constexpr float C1_F16_WEIGHT_SCALE = 256.f, C1_F16_OUTPUT_SCALE = 16777216.f / C1_F16_WEIGHT_SCALE / 255.f;     // 2^24 / 2^8 / 255
+// The weight-gradient kernel of the first layer plays the same trick in bf16, where it needs no second number format:
+// a byte n in the low half of a 16-bit word is the bf16 value n * 2^-133 whether n < 128 (a subnormal) or not (exponent
+// field 1, which has the same scale), and the tensor cores multiply these exactly (checked against exact products).
+// Such operands times gradients of size 1e-6 would sink below what a float accumulator holds, so the data-gradient
+// kernel of the layer above stores the gradient it hands down multiplied by 2^64 -- a shift of the exponent, exact
+// before the bf16 rounding as after it -- and the finished sums are multiplied by 2^(133 - 64) / 255.
+constexpr float C1_GRAD_SCALE = 18446744073709551616.f;                       // 2^64
+constexpr float C1_WGRAD_OUTPUT_SCALE = 590295810358705651712.f / 255.f;      // 2^69 / 255
+constexpr float C1_BIAS_OUTPUT_SCALE = 1.f / C1_GRAD_SCALE;
 __device__ __forceinline__ void u8x4_to_bf16x4(uint32_t w, uint32_t& lo, uint32_t& hi) {
   const float f0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7440)) - 8388608.f;
   const float f1 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7441)) - 8388608.f;
@@ -2850,11 +2864,11 @@ static void tc_shift_wgrad(LaunchCtx& lc, int kid, Cfg cfg, const bf16* g, int s
 // were measured 8 % slower than eight: the role is bound by issue slots and shared-memory traffic, not by latency.
 // The kernel is bound by how many bytes an SM keeps in flight from DRAM, so the gradient rows and the frame rows
 // have rings of their own that run several tiles ahead of the expansion.
-constexpr int W1_EXPAND_WARPS = 8, W1_THREADS = (W1_EXPAND_WARPS + 12) * 32, W1_STAGES = 3, W1_G_SLOTS = 6, W1_G_AHEAD = 5, W1_X_ROWS = 152, W1_USED = 149,
+constexpr int W1_EXPAND_WARPS = 8, W1_THREADS = (W1_EXPAND_WARPS + 12) * 32, W1_STAGES = 4, W1_G_SLOTS = W1_STAGES, W1_G_AHEAD = 3, W1_X_ROWS = 152, W1_USED = 149,
               W1_RAW_BYTES = 12288, W1_RAW_SLOTS = 5;
 
 struct W1Shared {
-  uint64_t full[W1_STAGES], empty[W1_STAGES], g_full[W1_G_SLOTS], g_empty[W1_G_SLOTS], raw_full[W1_RAW_SLOTS],
+  uint64_t full[W1_STAGES], empty[W1_STAGES], raw_full[W1_RAW_SLOTS],
            raw_empty[W1_RAW_SLOTS], acc;
   uint32_t tmem_base;
   volatile uint32_t abort;
@@ -2878,8 +2892,12 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
   const int split = blockIdx.x, t0 = split * tiles_per_cta, t1 = min(tiles, t0 + tiles_per_cta);
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < W1_STAGES; ++s) { mbar_init(&sh.full[s], NPROD / 32); mbar_init(&sh.empty[s], 1); }
-    for (int i = 0; i < W1_G_SLOTS; ++i) { mbar_init(&sh.g_full[i], 8); mbar_init(&sh.g_empty[i], 3); }
+    // One barrier pair per slot serves the expanded X rows and the gradient rows alike (both rings have W1_STAGES
+    // slots): full[s] gathers the eight expansion warps and the eight copy warps, empty[s] the commit of the tile's
+    // instructions and the two bias warps.  The issuing thread then waits once and commits once per tile; with eight
+    // short instructions per tile every further wait or commit (a couple of hundred cycles each, even when
+    // satisfied) was what set the kernel's pace.
+    for (int s = 0; s < W1_STAGES; ++s) { mbar_init(&sh.full[s], NPROD / 32 + 8); mbar_init(&sh.empty[s], 3); }
     for (int i = 0; i < W1_RAW_SLOTS; ++i) { mbar_init(&sh.raw_full[i], 1); mbar_init(&sh.raw_empty[i], NPROD / 32); }
     mbar_init(&sh.acc, 1);
     sh.abort = 0u;
@@ -2942,8 +2960,8 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
         const uint32_t ri = (uint32_t)(u + STEP * k);
         if (ri < (uint32_t)W1_USED) {
           uint32_t o[8];
-          u8x4_to_bf16x4(rw[k].x, o[0], o[1]); u8x4_to_bf16x4(rw[k].y, o[2], o[3]);
-          u8x4_to_bf16x4(rw[k].z, o[4], o[5]); u8x4_to_bf16x4(rw[k].w, o[6], o[7]);
+          u8x4_to_f16x4(rw[k].x, o[0], o[1]); u8x4_to_f16x4(rw[k].y, o[2], o[3]);          // bytes as bf16 values n * 2^-133
+          u8x4_to_f16x4(rw[k].z, o[4], o[5]); u8x4_to_f16x4(rw[k].w, o[6], o[7]);
           const uint32_t dst = stage + ri * 128u;
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + ((uint32_t)((2 * py) ^ (ri & 7)) << 4)),
                        "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
@@ -2981,8 +2999,6 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
       bool ok = true;
       for (int t = t0; t < t1 && ok; ++t) {
         const int it = t - t0, s = it % W1_STAGES, gs = it % W1_G_SLOTS;
-        ok = mbar_wait(&sh.g_full[gs], (it / W1_G_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
-        if (!ok) break;
         ok = mbar_wait(&sh.full[s], (it / W1_STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
         if (!ok) break;
         fence_proxy_async_smem();        // the copies observed through the barrier -> visible to the MMA's operand reads
@@ -2993,7 +3009,6 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
         for (int k = 0; k < TC_BM / 16; ++k)
           mma_bf16_lo_rt(tmem, a_lo0 + k * (2048u >> 4), b_lo0 + k * (2048u >> 4), hi, idesc, (it | k) != 0 ? 1u : 0u);
         mma_commit(&sh.empty[s]);
-        mma_commit(&sh.g_empty[gs]);
       }
       if (ok && t1 > t0) mma_commit(&sh.acc);
     }
@@ -3032,11 +3047,11 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
         cp_async_wait<W1_G_AHEAD - 1>();           // the rows of tile t - W1_G_AHEAD (my share) have landed
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.g_full[(t - W1_G_AHEAD - t0) % W1_G_SLOTS]);
+        if (lane == 0) mbar_arrive(&sh.full[(t - W1_G_AHEAD - t0) % W1_G_SLOTS]);
       }
       if (t < t1) {
         const int it = t - t0, gs = it % W1_G_SLOTS;
-        const bool ok = mbar_wait(&sh.g_empty[gs], ((it / W1_G_SLOTS) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
+        const bool ok = mbar_wait(&sh.empty[gs], ((it / W1_G_SLOTS) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
         if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
         const uint32_t dst = g_base + gs * G_BYTES;
         // Source offsets: the raster cell (state + 1, Y, X) of this thread's first row is carried from tile to tile
@@ -3073,7 +3088,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
     const int q = lane & 3, rr = lane >> 2, which = warp == E + 2 ? 0 : 1;
     for (int t = t0; t < t1 && ok; ++t) {
       const int it = t - t0, gs = it % W1_G_SLOTS;
-      ok = mbar_wait(&sh.g_full[gs], (it / W1_G_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
+      ok = mbar_wait(&sh.full[gs], (it / W1_G_SLOTS) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
       const uint32_t gaddr = g_base + gs * G_BYTES + (uint32_t)(rr + 8 * which) * 128u + ((uint32_t)(q ^ rr) << 4);
       uint32_t v[TC_BM / 16][4];
@@ -3090,7 +3105,7 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
         }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.g_empty[gs]);
+      if (lane == 0) mbar_arrive(&sh.empty[gs]);
     }
     // the eight row groups, added in a fixed order
 #pragma unroll
@@ -3131,8 +3146,9 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
   float* bias_part = scratch + (size_t)splits * 256 * 32;
   KernelScope scope(lc, KID_CONV1_WGRAD);
   launch_kernel_overlapped(lc, kern, splits, W1_THREADS, smem, frames, g, scratch, bias_part, n_states, tiles, per, err);
-  if (!add_segment(segs, scratch, gw, splits, 256, 32, 1.0f / 255.0f) ||
-      !add_segment(segs, bias_part, gb, 2 * splits, 1, 32, 1.f))      // two bias warps per CTA, a row each
+  // the gradient rows arrive multiplied by C1_GRAD_SCALE (see tc_backward_dgrad_conv2), the pixels as n * 2^-133
+  if (!add_segment(segs, scratch, gw, splits, 256, 32, C1_WGRAD_OUTPUT_SCALE) ||
+      !add_segment(segs, bias_part, gb, 2 * splits, 1, 32, C1_BIAS_OUTPUT_SCALE))      // two bias warps per CTA, a row each
     lc.host_failure = true;
 }
 
@@ -3388,13 +3404,16 @@ void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* con
       ShiftReluMaskEpi<Map, 9, 9>{Map{n}, (bf16*)gact[1], (const bf16*)act[1]}, n * 121, err);
   (void)M;
 }
-void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
+float tc_conv1_grad_scale() { return C1_GRAD_SCALE; }
+
+void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err,
+                             float out_scale) {
   typedef NatConv2 C2;
   const int M = n * (C2::H / 2) * (C2::W / 2);
   typedef RasterMap<121, 11, 10, 10> Map;
   tc_shift<C2DgradCfg, ShiftReluMaskEpiS2<Map>, 128, 3, 1>(
       lc, KID_CONV2_DGRAD, C2DgradCfg{(const bf16*)gact[1], n}, images,
-      ShiftReluMaskEpiS2<Map>{Map{n}, (bf16*)gact[0], (const bf16*)act[0]}, n * 121, err);
+      ShiftReluMaskEpiS2<Map>{Map{n}, (bf16*)gact[0], (const bf16*)act[0], out_scale}, n * 121, err);
   (void)M;
 }
 
