@@ -514,13 +514,15 @@ struct PkShared {
   volatile uint32_t abort;
 };
 
-template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES>
+template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES, int KPS>
 __global__ void __launch_bounds__(PK_THREADS, 1)
 tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_a, const bf16* __restrict__ w, int n_total, Epi epi, int tiles_m,
                      uint32_t* error_word) {
   static_assert(BN == 32 || BN == 64 || BN == 128, "tile width");
-  static_assert(STAGES >= 4 && STAGES <= 8, "pipeline depth");
-  constexpr uint32_t A_BYTES = TC_BM * 128, B_BLOCK = BN * 128, B_BYTES = NCLS * KB * B_BLOCK;
+  // KPS K blocks share a stage, i.e. one wait and one commit of the issuing thread: with four instructions per K block
+  // a wait per block (a couple of hundred cycles even when satisfied) left the tensor pipe idle half of the time
+  static_assert(STAGES >= 2 && STAGES <= 8 && KB % KPS == 0, "pipeline shape");
+  constexpr uint32_t A_BLOCK = TC_BM * 128, A_BYTES = KPS * A_BLOCK, B_BLOCK = BN * 128, B_BYTES = NCLS * KB * B_BLOCK;
   extern __shared__ uint8_t dyn_smem[];
   __shared__ PkShared sh;
   const uint32_t b_base = (smem_u32(dyn_smem) + 1023u) & ~1023u;
@@ -561,12 +563,13 @@ tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_a, const bf16* __res
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         const int m0 = (t % tiles_m) * TC_BM;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
+        for (int kb = 0; kb < KB; kb += KPS, ++it) {
           const int s = it % STAGES;
           ok = mbar_wait(&sh.empty[s], ((it / STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
           if (!ok) break;
           mbar_arrive_expect_tx(&sh.full[s], A_BYTES);
-          tma_load_2d(a_base0 + s * A_BYTES, &tm_a, kb * TC_BK, m0, &sh.full[s]);
+#pragma unroll
+          for (int j = 0; j < KPS; ++j) tma_load_2d(a_base0 + s * A_BYTES + j * A_BLOCK, &tm_a, (kb + j) * TC_BK, m0, &sh.full[s]);
         }
       }
     }
@@ -631,16 +634,19 @@ tc_persistent_kernel(const __grid_constant__ CUtensorMap tm_a, const bf16* __res
       ok = mbar_wait(&sh.acc_empty[ab], ((local >> 1) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_ACC);
       if (!ok) break;
       tcgen05_fence_after();
-      for (int kb = 0; kb < KB; ++kb, ++it) {
+      for (int kb = 0; kb < KB; kb += KPS, ++it) {
         const int s = it % STAGES;
         ok = mbar_wait(&sh.full[s], (it / STAGES) & 1, &sh.abort, error_word, ERR_WAIT_FULL);
         if (!ok) break;
         tcgen05_fence_after();
-        const uint32_t a_addr = a_base0 + s * A_BYTES, b_addr = b_base + (z * KB + kb) * B_BLOCK;
 #pragma unroll
-        for (int k = 0; k < TC_BK / 16; ++k)
-          mma_bf16(tmem + ab * BN, make_smem_desc(a_addr + k * 32, 0, 1024, SWIZZLE_128B),
-                   make_smem_desc(b_addr + k * 32, 0, 1024, SWIZZLE_128B), idesc, (kb | k) != 0 ? 1u : 0u);
+        for (int j = 0; j < KPS; ++j) {
+          const uint32_t a_addr = a_base0 + s * A_BYTES + j * A_BLOCK, b_addr = b_base + (z * KB + kb + j) * B_BLOCK;
+#pragma unroll
+          for (int k = 0; k < TC_BK / 16; ++k)
+            mma_bf16(tmem + ab * BN, make_smem_desc(a_addr + k * 32, 0, 1024, SWIZZLE_128B),
+                     make_smem_desc(b_addr + k * 32, 0, 1024, SWIZZLE_128B), idesc, (kb | j | k) != 0 ? 1u : 0u);
+        }
         mma_commit(&sh.empty[s]);
       }
       if (ok) mma_commit(&sh.acc_full[ab]);
@@ -2088,13 +2094,13 @@ static int sm_count() {
   return n;
 }
 
-template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES>
+template <class ASrc, class Epi, int BN, int KB, int NCLS, int STAGES, int KPS>
 static void tc_persistent(LaunchCtx& lc, int kid, ASrc a, const bf16* w, int n_total, Epi e, int M, uint32_t* err) {
   const CUtensorMap* tm_a = tc_tensor_map(a.x, (uint64_t)a.M, (uint64_t)KB * TC_BK, (uint64_t)a.ld, TC_BM);
   if (tm_a == nullptr) { lc.host_failure = true; return; }      // no tensor-map encoder: the API call reports PAAC_ERR_CUDA
-  constexpr int smem = NCLS * KB * BN * 128 + STAGES * TC_BM * 128 + 4 * 32 * BN * 2 + 1024;      // weights, stages, staging tiles
+  constexpr int smem = NCLS * KB * BN * 128 + STAGES * KPS * TC_BM * 128 + 4 * 32 * BN * 2 + 1024;      // weights, stages, staging tiles
   static_assert(smem <= 227 * 1024, "shared memory budget");
-  auto kern = tc_persistent_kernel<ASrc, Epi, BN, KB, NCLS, STAGES>;
+  auto kern = tc_persistent_kernel<ASrc, Epi, BN, KB, NCLS, STAGES, KPS>;
   static bool configured = false;
   if (!configured) {
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -3391,7 +3397,7 @@ void launch_wait_probe(LaunchCtx& lc, uint32_t max_polls, uint32_t* error_word) 
 // ---- backward: data gradients ---------------------------------------------------------------------------
 void tc_backward_dgrad_fc(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err) {
   const bf16* wfc_t = images + 4 * 32 * 256 + 64 * 576;
-  tc_persistent<PlainSrc, ReluMaskEpiTc, 128, 8, 1, 4>(
+  tc_persistent<PlainSrc, ReluMaskEpiTc, 128, 8, 1, 2, 2>(
       lc, KID_FC_DGRAD, PlainSrc{(const bf16*)gact[3], 512, n}, wfc_t, 3136,
       ReluMaskEpiTc{(bf16*)gact[2], (const bf16*)act[2], 3136, n}, n, err);
 }
