@@ -289,7 +289,7 @@ def run_ours(args, cfg):
     # ---- the pre-processing kernel of Section 5.1 on n_e pairs of synthetic raw frames (bytes = two raw frames and the
     # previous state read, the new state written); the inputs (over 200 MB at n_e = 1024) exceed L2
     prep = None
-    if rank == 0:
+    if rank == 0 and not args.no_e2e:
         raw = torch.randint(0, 256, (2, n_e, 210, 160, 3), dtype=torch.uint8, device="cuda")
         st_in = torch.randint(0, 256, (n_e, 84, 84, 4), dtype=torch.uint8, device="cuda")
         st_out = torch.empty_like(st_in)
@@ -307,7 +307,7 @@ def run_ours(args, cfg):
     # ---- end to end through the external-environment entry points (host frames in, actions out)
     frames_dev = torch.empty(0)
     e2e = None
-    if rank == 0 or world > 1:
+    if (rank == 0 or world > 1) and not args.no_e2e:
         g.rollout()
         import numpy as np
         fr = g.debug_read(pb.DBG_FRAMES).reshape(T, n_e, FRAME_BYTES)
@@ -422,6 +422,8 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="index into the five workloads (4 = n_e 1024, Nature CNN, bf16)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true",
+                    help="skip the end-to-end leg and the pre-processing kernel (short runs under a profiler)")
     ap.add_argument("--sustain-s", type=float, default=2.0,
                     help="seconds of back-to-back iterations in the sustained block (0 = skip it)")
     args = ap.parse_args()

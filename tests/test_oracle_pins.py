@@ -190,6 +190,22 @@ def test_xavier_init(orc):
     assert th[4112 + 5] == (np.float32(2) * u - np.float32(1)) * b2
     assert orc.param_count(orc.arch_net("nature", 18)) == 1693875
     assert not np.array_equal(th, orc.init_params(net, 2))
+    # the two heads: fan_in = hidden units, fan_out = actions (policy) and 1 (value); layer ids follow the fc layer's.
+    # With 18 x 512 and 512 samples the largest magnitude comes within a few per cent of the bound from below, the
+    # sample variance is that of a uniform, and one element of each goes through the Python Philox.
+    nat = orc.arch_net("nature", 18)
+    tn = orc.init_params(nat, 3)
+    o_pi = tn.size - (512 + 1) - (18 * 512 + 18)
+    wpi, bpi = tn[o_pi:o_pi + 18 * 512], tn[o_pi + 18 * 512:o_pi + 18 * 512 + 18]
+    wv, bv = tn[-513:-1], tn[-1]
+    b_pi, b_v = math.sqrt(6.0 / (512 + 18)), math.sqrt(6.0 / (512 + 1))
+    assert np.all(bpi == 0) and bv == 0
+    assert 0.995 * b_pi < np.abs(wpi).max() <= np.float32(b_pi) and 0.97 * b_v < np.abs(wv).max() <= np.float32(b_v)
+    assert abs(wpi.var() / (b_pi * b_pi / 3) - 1) < 0.05 and abs(wv.var() / (b_v * b_v / 3) - 1) < 0.2
+    for layer, off, bound, i in ((4, o_pi, b_pi, 7), (5, tn.size - 513, b_v, 100)):
+        out = py_philox([i, layer, 0, 1], [3, 0])
+        u = np.float32((out[0] >> 8) / 2.0 ** 24)
+        assert tn[off + i] == (np.float32(2) * u - np.float32(1)) * np.float32(bound)
 
 
 # ----------------------------------------------------------------------------- network vs PyTorch float64

@@ -19,7 +19,7 @@ def rel(x, y):
     return float(np.abs(x - y).max() / (np.abs(y).max() + 1e-12))
 
 
-def test_noalloc_optimiser_matches_update_twice_in_a_row():
+def test_noalloc_optimiser_matches_update_twice_in_a_row(orc):
     import torch
     hp = dict(lr=0.0224, rms_decay=0.99, rms_eps=0.1, clip_norm=0.5)      # low threshold: clipping is active
     g = pb.Paac("nips", 8, 3, 6, seed=21, precision=pb.BF16, **hp)
@@ -29,11 +29,14 @@ def test_noalloc_optimiser_matches_update_twice_in_a_row():
     shadow = torch.zeros(g.P, dtype=torch.int16, device=dev)
     out = torch.zeros(2, dtype=torch.float32, device=dev)
     clipped = 0
+    theta_o, rms_o = g.params().copy(), g.debug_read(pb.DBG_RMS).copy()       # the oracle's copies walk along
     for call in range(2):
         g.rollout()
         st = g.update()
         assert st["status"] == 0
         grad = torch.from_numpy(g.debug_read(pb.DBG_GRAD).copy()).to(dev)
+        st_o, norm_o, scale_o = orc.clip_rmsprop(theta_o, rms_o, grad.cpu().numpy(), hp["lr"], hp["rms_decay"],
+                                                 hp["rms_eps"], hp["clip_norm"])
         rc = pb.clip_rmsprop_noalloc(theta, rms, grad, g.P, hp["lr"], hp["rms_decay"], hp["rms_eps"], hp["clip_norm"],
                                      theta_bf16=shadow, norm_and_scale=out,
                                      stream=torch.cuda.current_stream().cuda_stream)
@@ -42,6 +45,9 @@ def test_noalloc_optimiser_matches_update_twice_in_a_row():
         norm, scale = out.cpu().numpy()
         assert abs(norm - st["grad_norm"]) <= 1e-5 * st["grad_norm"] and abs(scale - st["clip_scale"]) <= 1e-5
         clipped += scale < 1.0
+        # against the oracle's optimiser step on the same gradient (not only against paac_update)
+        assert st_o == 0 and abs(norm - norm_o) <= 1e-5 * norm_o and abs(scale - scale_o) <= 1e-5
+        assert rel(theta.cpu().numpy(), theta_o) <= 1e-4 and rel(rms.cpu().numpy(), rms_o) <= 1e-4
         # same tolerance as the float parity tests
         assert rel(theta.cpu().numpy(), g.params()) <= 1e-4
         assert rel(rms.cpu().numpy(), g.debug_read(pb.DBG_RMS)) <= 1e-4
