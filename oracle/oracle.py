@@ -177,6 +177,34 @@ def preprocess(raw_prev, raw_last, state_in=None):
     return out
 
 
+def pattern_goal(seed, env, step, n_actions):
+    lib().orc_pattern_goal.restype = C.c_uint32
+    return int(lib().orc_pattern_goal(C.c_uint64(seed), C.c_uint32(env), C.c_uint32(step), n_actions))
+
+
+def pattern_frame(seed, env, step, tag, n_actions, h=84, w=84):
+    f = np.zeros((h, w, 4), np.uint8)
+    lib().orc_pattern_frame(C.c_uint64(seed), C.c_uint32(env), C.c_uint32(step), C.c_uint32(tag), n_actions, h, w, _p(f))
+    return f
+
+
+def pattern_reset(seed, n_e, n_actions, h=84, w=84):
+    f = np.zeros((n_e, h, w, 4), np.uint8)
+    lib().orc_pattern_reset(C.c_uint64(seed), n_e, n_actions, h, w, _p(f))
+    return f
+
+
+def pattern_step(seed, step, actions, term_denom, n_actions, counters, h=84, w=84):
+    n_e = actions.shape[0]
+    actions = np.ascontiguousarray(actions, np.int32)
+    f = np.zeros((n_e, h, w, 4), np.uint8)
+    r = np.zeros(n_e, np.int8)
+    t = np.zeros(n_e, np.uint8)
+    lib().orc_pattern_step(C.c_uint64(seed), n_e, C.c_uint32(step), _p(actions), C.c_uint32(term_denom), n_actions, h, w,
+                           _p(f), _p(r), _p(t), _p(counters[0]), _p(counters[1]), _p(counters[2]))
+    return f, r, t
+
+
 def _ptr_array(arrs):
     return (C.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
 
@@ -304,7 +332,8 @@ def clip_rmsprop(theta, m, grad, lr, rho, eps, clip):
 
 
 DEFAULT_HP = dict(gamma=0.99, lr=0.0224, rms_decay=0.99, rms_eps=0.1, clip_norm=40.0,
-                  entropy_beta=0.01, value_coef=1.0, term_denom=200, algorithm="a2c", epsilon=0.1)
+                  entropy_beta=0.01, value_coef=1.0, term_denom=200, algorithm="a2c", epsilon=0.1,
+                  environment="hashed")
 
 
 class OraclePAAC:
@@ -324,7 +353,8 @@ class OraclePAAC:
         self.m = np.zeros_like(self.theta)
         self.N = 0
         self.h, self.w = self.net.in_h, self.net.in_w
-        self.state = env_reset(seed, n_e, self.h, self.w)
+        self.pattern = self.hp["environment"] == "pattern"
+        self.state = pattern_reset(seed, n_e, n_actions, self.h, self.w) if self.pattern else env_reset(seed, n_e, self.h, self.w)
         self.counters = [np.zeros(n_e, np.int32) for _ in range(3)]
 
     def rollout(self, forced_actions=None):
@@ -354,8 +384,12 @@ class OraclePAAC:
                     values[e] = logits[e, a]          # what the step is worth to the learner: Q(s_t, a_t)
             ro["logits"][t], ro["values"][t], ro["probs"][t] = logits, values, p
             ro["acts"].append(acts)
-            f, r, term = env_step(self.seed, step0 + t, ro["actions"][t], self.hp["term_denom"], self.counters,
-                                  self.h, self.w)
+            if self.pattern:
+                f, r, term = pattern_step(self.seed, step0 + t, ro["actions"][t], self.hp["term_denom"], A, self.counters,
+                                          self.h, self.w)
+            else:
+                f, r, term = env_step(self.seed, step0 + t, ro["actions"][t], self.hp["term_denom"], self.counters,
+                                      self.h, self.w)
             ro["frames"][t + 1], ro["rewards"][t], ro["terminals"][t] = f, r, term
         _, zb, vb = forward(self.net, self.theta, ro["frames"][T], self.bf16)
         ro["values"][T] = zb.max(axis=1) if self.hp["algorithm"] == "nstep_q" else vb

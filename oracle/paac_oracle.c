@@ -236,6 +236,46 @@ void orc_env_step(uint64_t seed, int n_e, uint32_t step, const int32_t* actions,
 }
 
 /* ------------------------------------------------------------------ */
+/* A second synthetic environment, one a learner can solve (the hashed  */
+/* one above has nothing to learn): every state shows which action is   */
+/* rewarded.  goal(env, step) = mix(base(env, step, 0) ^ 'GOAL') mod A; */
+/* the frame is the hashed frame of the same (env, step, tag) with the  */
+/* band of rows [band * goal, band * (goal + 1)), band = h / A, set to  */
+/* 255 in all channels; taking action a pays +1 if a is the goal of the */
+/* current state and 0 otherwise; terminals as in the hashed            */
+/* environment.  Used for the learning-rate rule of Section 5.3.        */
+/* ------------------------------------------------------------------ */
+#define TAG_GOAL 0x474F414Cu
+uint32_t orc_pattern_goal(uint64_t seed, uint32_t env, uint32_t step, int n_actions) {
+  return mix(env_base(seed, env, step, 0u) ^ TAG_GOAL) % (uint32_t)n_actions;
+}
+void orc_pattern_frame(uint64_t seed, uint32_t env, uint32_t step, uint32_t tag, int n_actions,
+                       int h, int w, uint8_t* frame) {
+  orc_env_frame(seed, env, step, tag, h, w, frame);
+  int band = h / n_actions, g = (int)orc_pattern_goal(seed, env, step, n_actions);
+  for (int y = band * g; y < band * (g + 1); ++y)
+    memset(frame + (size_t)y * w * 4, 255, (size_t)w * 4);
+}
+void orc_pattern_reset(uint64_t seed, int n_e, int n_actions, int h, int w, uint8_t* frames) {
+  for (int e = 0; e < n_e; ++e)
+    orc_pattern_frame(seed, (uint32_t)e, 0u, 0u, n_actions, h, w, frames + (size_t)e * h * w * 4);
+}
+void orc_pattern_step(uint64_t seed, int n_e, uint32_t step, const int32_t* actions, uint32_t term_denom, int n_actions,
+                      int h, int w, uint8_t* next_frames, int8_t* rewards, uint8_t* terminals,
+                      int32_t* ep_len, int32_t* ep_return, int32_t* episodes) {
+#pragma omp parallel for schedule(static)
+  for (int e = 0; e < n_e; ++e) {
+    int8_t unused;
+    orc_env_outcome(seed, (uint32_t)e, step, actions[e], term_denom, &unused, &terminals[e]);
+    rewards[e] = (uint32_t)actions[e] == orc_pattern_goal(seed, (uint32_t)e, step, n_actions) ? 1 : 0;
+    uint32_t tag = terminals[e] ? 0u : (uint32_t)actions[e] + 1u;
+    orc_pattern_frame(seed, (uint32_t)e, step + 1u, tag, n_actions, h, w, next_frames + (size_t)e * h * w * 4);
+    ep_len[e] += 1; ep_return[e] += rewards[e];
+    if (terminals[e]) { episodes[e] += 1; ep_len[e] = 0; ep_return[e] = 0; }
+  }
+}
+
+/* ------------------------------------------------------------------ */
 /* Forward pass f(s; theta) -> (logits, V)  (Section 5.1: one CNN, a     */
 /* softmax policy head and a linear scalar value head)                  */
 /* act[l]: float [n][h][w][c] of conv layer l (post ReLU), act[n_conv]: */

@@ -539,3 +539,33 @@ def test_iteration_is_consistent_with_its_steps(orc):
     ro2 = o.rollout(forced_actions=np.full((4, 3), 1, np.int32))
     assert np.array_equal(ro2["frames"][0], ro["frames"][4]) and np.all(ro2["actions"] == 1)
     assert ro2["uniforms"][0, 2] == np.float32(orc.action_uniform(5, 2, 4))
+
+
+# ----------------------------------------------------------------------------- the learnable environment
+def test_pattern_environment(orc):
+    """The second synthetic environment: hashed frames with a bright band of rows that names the rewarded action."""
+    seed, A = 9, 6
+    band = 84 // A
+    goals = []
+    for e, step, tag in ((0, 0, 0), (3, 7, 2), (11, 123, 0)):
+        g = orc.pattern_goal(seed, e, step, A)
+        goals.append(g)
+        # second implementation of the goal: the Python hash chain of the environment pins
+        assert g == py_mix(py_base(seed, e, step, 0) ^ 0x474F414C) % A
+        f = orc.pattern_frame(seed, e, step, tag, A)
+        ref = py_frame(seed, e, step, tag)
+        ref[band * g:band * (g + 1)] = 255
+        assert np.array_equal(f, ref)
+    # goals are spread over the actions; a matching action pays 1, any other 0; terminals are the hashed ones
+    gs = np.array([orc.pattern_goal(seed, e, 5, A) for e in range(3000)])
+    assert np.all(np.abs(np.bincount(gs, minlength=A) - 500) < 5 * math.sqrt(500))
+    n_e = 64
+    counters = [np.zeros(n_e, np.int32) for _ in range(3)]
+    acts = np.arange(n_e, dtype=np.int32) % A
+    f, r, t = orc.pattern_step(seed, 5, acts, 50, A, counters)
+    for e in range(n_e):
+        assert r[e] == (1 if acts[e] == orc.pattern_goal(seed, e, 5, A) else 0)
+        assert t[e] == orc.env_outcome(seed, e, 5, int(acts[e]), 50)[1]
+        tag = 0 if t[e] else int(acts[e]) + 1
+        assert np.array_equal(f[e], orc.pattern_frame(seed, e, 6, tag, A))
+    assert np.array_equal(orc.pattern_reset(seed, 2, A)[1], orc.pattern_frame(seed, 1, 0, 0, A))
