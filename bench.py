@@ -414,6 +414,47 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_lr_sweep(args):
+    """Section 5.3's learning-rate rule, alpha = 0.0007 * n_e for n_e in 16 .. 256, on the learnable synthetic
+    environment (a bright band of rows names the rewarded action; chance level 1 / A): mean reward per step at the
+    start and at the end of a fixed budget of timesteps, and where training stopped being finite if it did.
+    The environment is a contextual bandit (the next state's goal does not depend on the action), so the sweep runs
+    with gamma = 0: the one-step return is then the exact advantage target, and the value head predicts a quantity
+    of order one as it does under the clipped, sparse rewards of the paper's games (with gamma = 0.99 a reward on
+    every step makes the value targets of order 1 / (1 - gamma) and the paper's step sizes collapse the policy).
+    All other hyper-parameters are Section 5.1's."""
+    import numpy as np
+    import torch
+    from paper_1705_04862_b200 import binding as pb
+    torch.cuda.set_stream(torch.cuda.Stream())
+    A, T, budget = 6, 5, args.sweep_timesteps
+    rows = []
+    for arch, prec in (("nips", pb.FP32), ("nature", pb.BF16)):
+        for n_e in (16, 32, 64, 128, 256):
+            lr = 0.0007 * n_e
+            g = pb.Paac(arch, n_e, T, A, COMMON["seed"], precision=prec, lr=lr, term_denom=200, environment=pb.ENV_PATTERN,
+                        gamma=0.0, rms_decay=COMMON["rms_decay"], rms_eps=COMMON["rms_eps"],
+                        clip_norm=COMMON["clip_norm"], entropy_beta=COMMON["entropy_beta"], value_coef=COMMON["value_coef"])
+            updates = max(40, budget // (n_e * T))
+            rew, ent, bad = [], [], None
+            for u in range(updates):
+                g.rollout()
+                rew.append(float(g.debug_read(pb.DBG_REWARDS).astype(np.float64).mean()))
+                st = g.update()
+                ent.append(st["entropy"])
+                if st["status"] != 0 and bad is None:
+                    bad = u
+            k = max(5, updates // 10)
+            above = [i for i in range(len(rew) - 4) if np.mean(rew[i:i + 5]) >= 0.8]
+            rows.append({"arch": arch, "precision": "bf16" if prec == pb.BF16 else "fp32", "n_e": n_e, "lr": lr,
+                         "updates": updates, "timesteps": updates * n_e * T, "reward_first": float(np.mean(rew[:k])),
+                         "reward_last": float(np.mean(rew[-k:])), "entropy_last": float(np.mean(ent[-k:])),
+                         "timesteps_to_0.8": (above[0] + 5) * n_e * T if above else None, "first_nonfinite_update": bad})
+            g.close()
+    print(json.dumps({"experiment": "lr_rule_sweep", "rule": "lr = 0.0007 * n_e", "environment": "pattern", "n_actions": A,
+                      "t_max": T, "gamma": 0.0, "chance_reward": 1.0 / A, "rows": rows}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -426,8 +467,14 @@ def main():
                     help="skip the end-to-end leg and the pre-processing kernel (short runs under a profiler)")
     ap.add_argument("--sustain-s", type=float, default=2.0,
                     help="seconds of back-to-back iterations in the sustained block (0 = skip it)")
+    ap.add_argument("--lr-sweep", action="store_true",
+                    help="instead of the throughput line: the alpha = 0.0007 n_e rule on the learnable environment")
+    ap.add_argument("--sweep-timesteps", type=int, default=200000)
     args = ap.parse_args()
     cfg = CONFIGS[args.config]
+    if args.lr_sweep:
+        run_lr_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

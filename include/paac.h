@@ -59,6 +59,15 @@ enum { PAAC_FP32 = 0, PAAC_BF16 = 1 };
  *                    carried along unused and receives a zero gradient; entropy_beta is ignored. */
 enum { PAAC_ALGO_A2C = 0, PAAC_ALGO_NSTEP_Q = 1 };
 
+/* The synthetic environment inside the library (it stands in for the emulators of the paper's experiments).
+ * PAAC_ENV_HASHED:  frames, rewards in {-1, 0, 1} and terminals are hashes of (seed, environment, step, action):
+ *                   the workload of the throughput measurements; there is nothing to learn in it.
+ * PAAC_ENV_PATTERN: the same hashed frames dimmed to their low six bits, with a band of 84 / n_actions rows set to 255 that names the rewarded
+ *                   action of the state (goal = hash(seed, environment, step) mod n_actions); the goal action pays
+ *                   +1, any other 0; terminals as above.  A learner can solve it, which the learning-rate rule
+ *                   of Section 5.3 (alpha = 0.0007 n_e) is tried on. */
+enum { PAAC_ENV_HASHED = 0, PAAC_ENV_PATTERN = 1 };
+
 enum {
   PAAC_OK = 0,
   PAAC_ERR_ARG = 1,        /* null pointer, size or enum out of range */
@@ -91,6 +100,7 @@ typedef struct {
   void* stream;         /* cudaStream_t the work is enqueued on; NULL: the default stream */
   int algorithm;        /* PAAC_ALGO_A2C (default) or PAAC_ALGO_NSTEP_Q */
   float epsilon;        /* PAAC_ALGO_NSTEP_Q: exploration probability in [0, 1] (default 0.1) */
+  int environment;      /* PAAC_ENV_HASHED (default) or PAAC_ENV_PATTERN */
 } paac_hparams;
 
 void paac_default_hparams(paac_hparams* hp /* host, out */);

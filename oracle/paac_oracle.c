@@ -239,9 +239,10 @@ void orc_env_step(uint64_t seed, int n_e, uint32_t step, const int32_t* actions,
 /* A second synthetic environment, one a learner can solve (the hashed  */
 /* one above has nothing to learn): every state shows which action is   */
 /* rewarded.  goal(env, step) = mix(base(env, step, 0) ^ 'GOAL') mod A; */
-/* the frame is the hashed frame of the same (env, step, tag) with the  */
-/* band of rows [band * goal, band * (goal + 1)), band = h / A, set to  */
-/* 255 in all channels; taking action a pays +1 if a is the goal of the */
+/* the frame is the hashed frame of the same (env, step, tag) with every */
+/* byte reduced to its low six bits (a dim texture, 0..63) and the band */
+/* of rows [band * goal, band * (goal + 1)), band = h / A, set to 255   */
+/* in all channels; taking action a pays +1 if a is the goal of the     */
 /* current state and 0 otherwise; terminals as in the hashed            */
 /* environment.  Used for the learning-rate rule of Section 5.3.        */
 /* ------------------------------------------------------------------ */
@@ -252,6 +253,7 @@ uint32_t orc_pattern_goal(uint64_t seed, uint32_t env, uint32_t step, int n_acti
 void orc_pattern_frame(uint64_t seed, uint32_t env, uint32_t step, uint32_t tag, int n_actions,
                        int h, int w, uint8_t* frame) {
   orc_env_frame(seed, env, step, tag, h, w, frame);
+  for (size_t i = 0; i < (size_t)h * w * 4; ++i) frame[i] &= 63;
   int band = h / n_actions, g = (int)orc_pattern_goal(seed, env, step, n_actions);
   for (int y = band * g; y < band * (g + 1); ++y)
     memset(frame + (size_t)y * w * 4, 255, (size_t)w * 4);

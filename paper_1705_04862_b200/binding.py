@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libpaac_b200.so")
 ARCH_NIPS, ARCH_NATURE = 0, 1
 FP32, BF16 = 0, 1
 ALGO_A2C, ALGO_NSTEP_Q = 0, 1
+ENV_HASHED, ENV_PATTERN = 0, 1
 OK, ERR_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_STATE, ERR_LIMIT, ERR_RANGE = range(9)
 (DBG_FRAMES, DBG_NEXT_FRAMES, DBG_ACTIONS, DBG_REWARDS, DBG_TERMINALS, DBG_VALUES, DBG_LOGITS, DBG_UNIFORMS,
  DBG_COUNTERS, DBG_RETURNS, DBG_ADVANTAGES, DBG_DLOGITS, DBG_DVALUES, DBG_GRAD, DBG_RMS, DBG_SAMPLED,
@@ -32,7 +33,7 @@ class HParams(C.Structure):
                 ("clip_norm", C.c_float), ("entropy_beta", C.c_float), ("value_coef", C.c_float),
                 ("term_denom", C.c_uint32), ("precision", C.c_int), ("workspace", C.c_void_p),
                 ("workspace_bytes", C.c_size_t), ("stream", C.c_void_p), ("algorithm", C.c_int),
-                ("epsilon", C.c_float)]
+                ("epsilon", C.c_float), ("environment", C.c_int)]
 
 
 class RolloutView(C.Structure):

@@ -75,6 +75,7 @@ bool valid_shape(int arch, int n_e, int t_max, int A, const paac_hparams* hp) {
   if (hp->term_denom == 0) return false;
   if (hp->algorithm != PAAC_ALGO_A2C && hp->algorithm != PAAC_ALGO_NSTEP_Q) return false;
   if (!(hp->epsilon >= 0.f && hp->epsilon <= 1.f)) return false;
+  if (hp->environment != PAAC_ENV_HASHED && hp->environment != PAAC_ENV_PATTERN) return false;
   return true;
 }
 
@@ -140,6 +141,7 @@ int cuda_status(paac_ctx* c) {
 
 bool use_tc(const paac_ctx* c) { return tc_supported(c->arch, c->prec) && !c->simt_only; }
 HeadMode head_mode(const paac_ctx* c) { return HeadMode{c->hp.algorithm, c->hp.epsilon}; }
+int pattern_actions(const paac_ctx* c) { return c->hp.environment == PAAC_ENV_PATTERN ? c->A : 0; }
 
 // bf16 copies of the master parameters, in the canonical layout and regrouped for the backward kernels
 void refresh_weight_copies(paac_ctx* c, bool cast) {
@@ -243,7 +245,7 @@ void paac_default_hparams(paac_hparams* hp) {
   hp->gamma = 0.99f; hp->lr = 0.0224f; hp->rms_decay = 0.99f; hp->rms_eps = 0.1f;
   hp->clip_norm = 40.f; hp->entropy_beta = 0.01f; hp->value_coef = 1.f;
   hp->term_denom = 200; hp->precision = PAAC_FP32;
-  hp->algorithm = PAAC_ALGO_A2C; hp->epsilon = 0.1f;
+  hp->algorithm = PAAC_ALGO_A2C; hp->epsilon = 0.1f; hp->environment = PAAC_ENV_HASHED;
 }
 
 size_t paac_workspace_bytes(int arch, int n_e, int t_max, int n_actions, const paac_hparams* hp) {
@@ -283,7 +285,8 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   launch_init_params(c->lc, c->nd, seed, c->theta);
   refresh_weight_copies(c, true);
   c->cur = 1;   // the first rollout flips to buffer 0; its start states are written there now
-  launch_env_step(c->lc, seed, n_e, c->step_dev, 0u, nullptr, hp->term_denom, c->frames[0], nullptr, nullptr, nullptr);
+  launch_env_step(c->lc, seed, n_e, c->step_dev, 0u, nullptr, hp->term_denom, c->frames[0], nullptr, nullptr, nullptr,
+                  pattern_actions(c));
   if (cudaStreamSynchronize(c->st) != cudaSuccess || cudaGetLastError() != cudaSuccess) {
     if (c->owns_workspace) cudaFree(c->ws);
     delete c;
@@ -308,10 +311,10 @@ int paac_rollout(paac_ctx* c, paac_rollout_view* view) {
       const size_t row = (size_t)t * c->n_e;
       if (deferred)
         launch_env_step_sampling(c->lc, c->seed, c->n_e, c->step_dev, (uint32_t)t, c->hp.term_denom, dst, c->rewards + row,
-                                 c->terminals + row, c->counters, tail);
+                                 c->terminals + row, c->counters, tail, pattern_actions(c));
       else
         launch_env_step(c->lc, c->seed, c->n_e, c->step_dev, (uint32_t)t, c->actions + row, c->hp.term_denom, dst,
-                        c->rewards + row, c->terminals + row, c->counters);
+                        c->rewards + row, c->terminals + row, c->counters, pattern_actions(c));
     }
     bool advanced = false;
     forward_slot(c, nxt, c->t_max, false, nullptr, &advanced);

@@ -108,7 +108,7 @@ __device__ __forceinline__ int warp_finish_heads(const HeadMode hm, float z, flo
 
 // ---- environment hash -----------------------------------------------------------
 constexpr uint32_t HASH_K0 = 0x9E3779B9u, HASH_K1 = 0xBB67AE85u, HASH_K2 = 0x6A09E667u;
-constexpr uint32_t HASH_TAG_REWARD = 0x52455744u, HASH_TAG_TERMINAL = 0x5445524Du;
+constexpr uint32_t HASH_TAG_REWARD = 0x52455744u, HASH_TAG_TERMINAL = 0x5445524Du, HASH_TAG_GOAL = 0x474F414Cu;
 
 __host__ __device__ __forceinline__ uint32_t hash_mix(uint32_t x) {
   x ^= x >> 16; x *= HASH_K0; x ^= x >> 15; x *= HASH_K1; x ^= x >> 16;

@@ -66,8 +66,12 @@ __global__ void __launch_bounds__(ENV_THREADS)
 env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, uint32_t t,
                 const int32_t* actions, uint32_t term_denom,
                 uint8_t* __restrict__ next_frames, int8_t* __restrict__ rewards, uint8_t* __restrict__ terminals,
-                int32_t* __restrict__ counters, HeadsTail ht) {
-  __shared__ uint32_t s_base;
+                int32_t* __restrict__ counters, HeadsTail ht, int pattern_actions) {
+  // pattern_actions > 0: the learnable environment.  The state at step k of environment e has the goal
+  // hash(e, k, 'GOAL') mod A; its frame is the hashed frame with every byte reduced to its low six bits (a dim
+  // texture) and rows [band goal, band (goal + 1)), band = 84 / A, set to 255; an action pays 1 if it is the current
+  // state's goal and 0 otherwise.
+  __shared__ uint32_t s_base, s_band_lo, s_band_hi;
   const uint32_t e = blockIdx.x;
   int32_t a_sampled = 0;
   if (SAMPLE && threadIdx.x < 32) {
@@ -89,7 +93,9 @@ env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, 
       const int32_t a = SAMPLE ? a_sampled : actions[e];
       const uint32_t base = env_hash_base(seed, e, step, (uint32_t)a + 1u);
       const uint32_t hr = hash_mix(base ^ HASH_TAG_REWARD) & 15u;
-      const int r = hr == 0u ? 1 : (hr == 1u ? -1 : 0);
+      int r = hr == 0u ? 1 : (hr == 1u ? -1 : 0);
+      if (pattern_actions > 0)
+        r = (uint32_t)a == hash_mix(env_hash_base(seed, e, step, 0u) ^ HASH_TAG_GOAL) % (uint32_t)pattern_actions ? 1 : 0;
       const uint32_t ht = hash_mix(base ^ HASH_TAG_TERMINAL);
       const bool term = (uint32_t)(((uint64_t)ht * term_denom) >> 32) == 0u;
       rewards[e] = (int8_t)r;
@@ -101,9 +107,17 @@ env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, 
       frame_step = step + 1u;
     }
     s_base = env_hash_base(seed, e, frame_step, tag);
+    s_band_lo = s_band_hi = 0u;
+    if (pattern_actions > 0) {
+      const uint32_t goal = hash_mix(env_hash_base(seed, e, frame_step, 0u) ^ HASH_TAG_GOAL) % (uint32_t)pattern_actions;
+      const uint32_t band = (uint32_t)(FRAME_H / pattern_actions);
+      s_band_lo = band * goal * FRAME_W;                  // in pixel words; a row is 84 words, so four words never straddle it
+      s_band_hi = s_band_lo + band * FRAME_W;
+    }
   }
   __syncthreads();
-  const uint32_t base = s_base;
+  const uint32_t base = s_base, band_lo = s_band_lo, band_hi = s_band_hi;
+  const uint32_t keep = pattern_actions > 0 ? 0x3F3F3F3Fu : 0xFFFFFFFFu;
   uint4* out = reinterpret_cast<uint4*>(next_frames + (size_t)e * FRAME_BYTES);
   for (int q = threadIdx.x; q < FRAME_WORDS / 4; q += ENV_THREADS) {
     const uint32_t p = (uint32_t)q * 4u + 1u;
@@ -112,24 +126,26 @@ env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, 
     v.y = hash_mix(base + HASH_K0 * (p + 1u));
     v.z = hash_mix(base + HASH_K0 * (p + 2u));
     v.w = hash_mix(base + HASH_K0 * (p + 3u));
+    v.x &= keep; v.y &= keep; v.z &= keep; v.w &= keep;
+    if ((uint32_t)q * 4u >= band_lo && (uint32_t)q * 4u < band_hi) v = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
     out[q] = v;
   }
 }
 
 void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step_base, uint32_t t,
                      const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
-                     uint8_t* terminals, int32_t* counters) {
+                     uint8_t* terminals, int32_t* counters, int pattern_actions) {
   KernelScope scope(lc, KID_ENV_STEP);
   launch_kernel(lc, env_step_kernel<false>, n_e, ENV_THREADS, 0, seed, n_e, step_base, t, actions, term_denom, next_frames, rewards,
-                                                  terminals, counters, HeadsTail{});
+                                                  terminals, counters, HeadsTail{}, pattern_actions);
 }
 
 void launch_env_step_sampling(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step_base, uint32_t t, uint32_t term_denom,
                               uint8_t* next_frames, int8_t* rewards, uint8_t* terminals, int32_t* counters,
-                              const HeadsTail& ht) {
+                              const HeadsTail& ht, int pattern_actions) {
   KernelScope scope(lc, KID_ENV_STEP);
   launch_kernel(lc, env_step_kernel<true>, n_e, ENV_THREADS, 0, seed, n_e, step_base, t, (const int32_t*)nullptr, term_denom,
-                next_frames, rewards, terminals, counters, ht);
+                next_frames, rewards, terminals, counters, ht, pattern_actions);
 }
 
 // the environments' global step index lives on the device, so that a recorded sequence of launches can be

@@ -11,7 +11,8 @@ void launch_cast_bf16(LaunchCtx& lc, const float* src, bf16* dst, size_t n);
 // actions == nullptr: start states (step index 0) for every environment
 void launch_env_step(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step_base /* device */, uint32_t t,
                      const int32_t* actions, uint32_t term_denom, uint8_t* next_frames, int8_t* rewards,
-                     uint8_t* terminals, int32_t* counters /* [3][n_e] */);
+                     uint8_t* terminals, int32_t* counters /* [3][n_e] */, int pattern_actions = 0 /* > 0: the learnable
+                     environment with that many actions */);
 
 // What is left of the heads after the cluster kernel of the fully connected layer: the two halves' dot products
 // hp[2][n_e][32], the head biases, and where logits, values, uniforms and actions go (see launch_heads_fused).
@@ -23,7 +24,7 @@ struct HeadsTail {
 // the same step with the action taken inside the kernel, from the heads' partial sums
 void launch_env_step_sampling(LaunchCtx& lc, uint64_t seed, int n_e, const uint64_t* step_base, uint32_t t, uint32_t term_denom,
                               uint8_t* next_frames, int8_t* rewards, uint8_t* terminals, int32_t* counters,
-                              const HeadsTail& ht);
+                              const HeadsTail& ht, int pattern_actions = 0);
 
 void launch_advance_step(LaunchCtx& lc, uint64_t* step_base, uint32_t by);
 

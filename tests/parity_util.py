@@ -25,6 +25,9 @@ def make_pair(orc, cfg, seed=None):
     if cfg.get("algorithm", "a2c") == "nstep_q":
         ohp.update(algorithm="nstep_q", epsilon=cfg.get("epsilon", 0.1))
         hp.update(algorithm=pb.ALGO_NSTEP_Q, epsilon=cfg.get("epsilon", 0.1))
+    if cfg.get("environment", "hashed") == "pattern":
+        ohp.update(environment="pattern")
+        hp.update(environment=pb.ENV_PATTERN)
     o = orc.OraclePAAC(cfg["arch"], cfg["n_e"], cfg["t_max"], cfg["n_actions"], seed, bf16=bf16, hp=ohp)
     g = pb.Paac(cfg["arch"], cfg["n_e"], cfg["t_max"], cfg["n_actions"], seed,
                 precision=pb.BF16 if bf16 else pb.FP32, **hp)

@@ -22,8 +22,8 @@ def test_library_builds_and_exports_every_declared_symbol():
 
 
 def test_struct_layouts_match_header():
-    assert C.sizeof(pb.HParams) == 72 and pb.HParams.workspace.offset == 40 and pb.HParams.stream.offset == 56
-    assert pb.HParams.algorithm.offset == 64 and pb.HParams.epsilon.offset == 68
+    assert C.sizeof(pb.HParams) == 80 and pb.HParams.workspace.offset == 40 and pb.HParams.stream.offset == 56
+    assert pb.HParams.algorithm.offset == 64 and pb.HParams.epsilon.offset == 68 and pb.HParams.environment.offset == 72
     assert C.sizeof(pb.UpdateStats) == 32 and pb.UpdateStats.timesteps.offset == 24
     assert C.sizeof(pb.RolloutView) == 64
 

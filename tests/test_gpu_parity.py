@@ -404,3 +404,38 @@ def test_value_based_variant_bad_hyperparameters():
     for bad in (dict(algorithm=2), dict(algorithm=pb.ALGO_NSTEP_Q, epsilon=1.5), dict(algorithm=pb.ALGO_NSTEP_Q, epsilon=-0.1)):
         hp = pb.default_hparams(**bad)
         assert pb.lib().paac_init(C.byref(h), 0, 4, 5, 4, C.byref(hp), 1) == pb.ERR_ARG
+
+
+def test_pattern_environment_matches_the_oracle_and_can_be_learned(orc):
+    """The learnable environment (a bright band of rows names the rewarded action): bit-exact frames and rewards in
+    lock step with the oracle on both network paths, and a learner on it collects clearly more reward after some
+    hundred updates than at the start (chance level is 1 / A)."""
+    import torch
+    for base in (0, 2):
+        cfg = dict(CONFIGS[base], environment="pattern", term_denom=50)
+        o, g = make_pair(orc, cfg)
+        for it in range(2):
+            if cfg["precision"] == "bf16":
+                resync(o, g)
+            ro, _ = check_rollout(orc, o, g, TOL[cfg["precision"]])
+            assert set(np.unique(ro["rewards"])) <= {0, 1}
+            check_update(orc, o, g, TOL[cfg["precision"]], inject=(cfg["precision"] == "bf16"))
+        g.close()
+    with torch.cuda.stream(torch.cuda.Stream()):
+        # a contextual bandit: gamma = 0 makes the one-step return the exact target (see bench.py --lr-sweep)
+        g = pb.Paac("nature", 16, 5, 6, seed=1, precision=pb.BF16, lr=0.0007 * 16, term_denom=200, gamma=0.0,
+                    environment=pb.ENV_PATTERN)
+        def mean_reward(iters):
+            tot = 0.0
+            for _ in range(iters):
+                g.rollout()
+                tot += float(g.debug_read(pb.DBG_REWARDS).astype(np.float64).mean())
+                assert g.update()["status"] == 0
+            return tot / iters
+        first = mean_reward(20)
+        for _ in range(400):
+            g.rollout()
+            g.update(sync=False)
+        last = mean_reward(20)
+        assert last > 0.8 and last > first + 0.2, (first, last)
+        g.close()

@@ -553,7 +553,7 @@ def test_pattern_environment(orc):
         # second implementation of the goal: the Python hash chain of the environment pins
         assert g == py_mix(py_base(seed, e, step, 0) ^ 0x474F414C) % A
         f = orc.pattern_frame(seed, e, step, tag, A)
-        ref = py_frame(seed, e, step, tag)
+        ref = py_frame(seed, e, step, tag) & 63               # dim texture
         ref[band * g:band * (g + 1)] = 255
         assert np.array_equal(f, ref)
     # goals are spread over the actions; a matching action pays 1, any other 0; terminals are the hashed ones
