@@ -53,6 +53,9 @@ clip_rmsprop_kernel(size_t P, float* __restrict__ theta, float* __restrict__ rms
   const size_t i0 = blockIdx.x * (size_t)OPT_THREADS + threadIdx.x;
   float4 gv0 = make_float4(0.f, 0.f, 0.f, 0.f), mv0 = gv0, tv0 = gv0;
   if (i0 < n4) { gv0 = g4[i0]; mv0 = m4[i0]; tv0 = t4[i0]; }
+  // the device error word, fetched now so that its latency hides behind the sum of the partials
+  uint32_t dev_err = 0u;
+  if (threadIdx.x == 0) dev_err = *reinterpret_cast<const volatile uint32_t*>(&stats->error_word);
   float acc = 0.f;
   for (int i = threadIdx.x; i < n_partials; i += OPT_THREADS) acc += partials[i];
 #pragma unroll
@@ -65,7 +68,6 @@ clip_rmsprop_kernel(size_t P, float* __restrict__ theta, float* __restrict__ rms
     for (int w = 0; w < OPT_THREADS / 32; ++w) total += sh[w];
     const float norm = sqrtf(total);
     float scale = 1.f;
-    const uint32_t dev_err = *reinterpret_cast<const volatile uint32_t*>(&stats->error_word);
     const bool ok = isfinite(norm) && dev_err == 0u;
     if (ok && clip > 0.f && norm > clip) scale = clip / norm;
     s_scale = ok ? scale : -1.f;
