@@ -109,6 +109,74 @@ def test_config5_bf16_resync_at_update_199(orc, capsys):
     _free_run_then_compare(orc, CONFIGS[4], 199, capsys)
 
 
+def test_largest_batch_sampled_against_the_oracle(orc):
+    """The largest rollout the library accepts (n_e * (t_max + 1) = 131,072 states: n_e = 65,536, t_max = 1, a 15 GB
+    workspace) on the tensor-core path: every tensor's element offsets are close to the 32-bit range there.  The
+    oracle cannot walk 65,536 environments, so it is asked for sampled ones -- the first 8 in lock step, and
+    environments from the middle and the very end of the batch one state at a time (frames re-hashed from their
+    integer definition, the network evaluated per state) -- and for the whole batch's returns and head gradients,
+    which are cheap."""
+    import torch
+    n_e, T, A = 65536, 1, 18
+    free, _ = torch.cuda.mem_get_info()
+    if free < 24 << 30:
+        pytest.skip("needs 24 GB of free device memory")
+    cfg = dict(CONFIGS[4], n_e=8, t_max=T)
+    o, _g = make_pair(orc, cfg)
+    _g.close()
+    g = pb.Paac("nature", n_e, T, A, 1, precision=pb.BF16, lr=cfg["lr"], term_denom=cfg["term_denom"])
+    assert np.array_equal(g.params(), o.theta)
+    ro = o.rollout()
+    forced = np.full((T, n_e), -1, np.int32)
+    forced[:, :8] = ro["actions"]
+    g.force_actions(forced)
+    g.rollout()
+    tol = TOL["bf16"]
+    logits = g.debug_read(pb.DBG_LOGITS).reshape(T, n_e, A)
+    values = g.debug_read(pb.DBG_VALUES).reshape(T + 1, n_e)
+    assert rel(logits[:, :8], ro["logits"]) <= tol and rel(values[:, :8], ro["values"]) <= tol
+    acts = g.debug_read(pb.DBG_ACTIONS).reshape(T, n_e)
+    terms = g.debug_read(pb.DBG_TERMINALS).reshape(T, n_e)
+    rewards = g.debug_read(pb.DBG_REWARDS).reshape(T, n_e)
+    unif = g.debug_read(pb.DBG_UNIFORMS).reshape(T, n_e)
+    sampled_envs = [8, 127, 128, 32767, 32768, 50001, 65407, 65408, 65534, 65535]
+    # start states and the states after the step are hashes of (seed, env, step, tag); the network is per state
+    frames0 = np.stack([orc.env_frame(1, e, 0, 0) for e in sampled_envs])
+    nxt = g.debug_read(pb.DBG_NEXT_FRAMES).reshape(n_e, 84, 84, 4)
+    fr = g.debug_read(pb.DBG_FRAMES).reshape(T, n_e, 84, 84, 4)
+    acts_l, z0, v0 = orc.forward(o.net, o.theta, frames0, True)
+    scale_z, scale_v = np.abs(ro["logits"]).max(), np.abs(ro["values"]).max()
+    for j, e in enumerate(sampled_envs):
+        assert np.array_equal(fr[0, e], frames0[j])
+        assert np.abs(logits[0, e] - z0[j]).max() <= tol * scale_z and abs(values[0, e] - v0[j]) <= tol * scale_v
+        assert unif[0, e] == np.float32(orc.action_uniform(1, e, 0))
+        r, t = orc.env_outcome(1, e, 0, int(acts[0, e]), cfg["term_denom"])
+        assert (int(rewards[0, e]), int(terms[0, e])) == (r, t)
+        tag = 0 if t else int(acts[0, e]) + 1
+        f1 = orc.env_frame(1, e, 1, tag)
+        assert np.array_equal(nxt[e], f1)
+        _, _, vb = orc.forward(o.net, o.theta, f1[None], True)
+        assert abs(values[1, e] - vb[0]) <= tol * scale_v
+    # the stored hidden units of the sampled states (the convolution maps of 65,536 states would be gigabytes on the host)
+    h = g.debug_read(pb.DBG_ACT0 + 3).reshape(n_e, 512)
+    for j, e in enumerate(sampled_envs):
+        assert np.abs(h[e] - acts_l[3][j]).max() <= tol * np.abs(acts_l[3]).max()
+    # the update at B = 65,536: returns, advantages and head gradients of the whole batch from the oracle, the
+    # reported norm against the gradient vector, finite parameters
+    st = g.update()
+    assert st["status"] == 0 and st["timesteps"] == n_e * T
+    R, adv = orc.returns(0.99, rewards, terms, values)
+    assert rel(g.debug_read(pb.DBG_RETURNS), R) <= 1e-6 and rel(g.debug_read(pb.DBG_ADVANTAGES), adv) <= 1e-5
+    dz_o, dV_o, stats_o = orc.head_grad(0.01, 1.0, logits.reshape(-1, A), values[:T].reshape(-1), acts.reshape(-1),
+                                        R.reshape(-1), adv.reshape(-1))
+    assert rel(g.debug_read(pb.DBG_DLOGITS), dz_o) <= 1e-4 and rel(g.debug_read(pb.DBG_DVALUES), dV_o) <= 1e-4
+    assert abs(st["entropy"] - stats_o["entropy"]) <= 1e-4 and abs(st["value_loss"] - stats_o["value_loss"]) <= 1e-4
+    grad = g.debug_read(pb.DBG_GRAD)
+    assert abs(np.linalg.norm(grad.astype(np.float64)) - st["grad_norm"]) <= 1e-4 * st["grad_norm"]
+    assert np.isfinite(g.params()).all()
+    g.close()
+
+
 def test_zz_flip_branch_statistics(capsys):
     """Reports how often the update check met ReLU units switched on on one side only (both valid) in this
     session, i.e. how often gradients were compared in the L2 sense instead of element by element."""
