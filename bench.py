@@ -212,6 +212,8 @@ def run_ours(args, cfg):
     torch.cuda.set_stream(side)
     g = pb.Paac(cfg["arch"], cfg["n_e"], cfg["t_max"], cfg["n_actions"], COMMON["seed"] + rank, precision=prec,
                 device="cuda:%d" % local, **hp)
+    if args.fp32_tensor_cores:
+        g.set_option(pb.OPT_FP32_TENSOR_CORES, 1)
     n_e, T = cfg["n_e"], cfg["t_max"]
     small = cfg["n_e"] < 256
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if small else None
@@ -399,7 +401,8 @@ def run_ours(args, cfg):
     out = {
         "metric": "env_steps_per_sec", "value": value, "unit": "env-steps/s", "n_gpus": world, "steps": K,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": cfg["precision"], "data": "synthetic", "config": workload_config(cfg),
+        "vs_baseline": None, "dtype": cfg["precision"], "data": "synthetic",
+        "config": dict(workload_config(cfg), **({"contractions": "3xTF32 tensor cores"} if args.fp32_tensor_cores else {})),
         "updates_per_sec": world * 1e3 / ms_per_step, "rollout_ms": roll_ms, "update_ms": upd_ms,
         "rollout_tflops": roll_flops / (roll_ms * 1e-3) / 1e12,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "sustained": sustained,
@@ -467,6 +470,8 @@ def main():
                     help="skip the end-to-end leg and the pre-processing kernel (short runs under a profiler)")
     ap.add_argument("--sustain-s", type=float, default=2.0,
                     help="seconds of back-to-back iterations in the sustained block (0 = skip it)")
+    ap.add_argument("--fp32-tensor-cores", action="store_true",
+                    help="float configurations: every contraction as three TF32 tensor-core passes (float-accurate)")
     ap.add_argument("--lr-sweep", action="store_true",
                     help="instead of the throughput line: the alpha = 0.0007 n_e rule on the learnable environment")
     ap.add_argument("--sweep-timesteps", type=int, default=200000)

@@ -260,8 +260,15 @@ int paac_debug_write(paac_ctx* ctx, int which, const void* src /* host */, size_
  * PAAC_OPT_DEPENDENT_LAUNCH: != 0 (default) launches every kernel with programmatic stream serialization, so
  * that a kernel's CTAs are scheduled while the kernel before it drains (each kernel waits on the device for its
  * predecessor before it touches that kernel's data); 0 launches with plain stream order.  The setting is
- * process-wide.  Results are bit-identical either way. */
-enum { PAAC_OPT_CUDA_CORES_ONLY = 1, PAAC_OPT_TC_WGRAD_LAYERS = 2, PAAC_OPT_CUDA_GRAPHS = 3, PAAC_OPT_DEPENDENT_LAUNCH = 4 };
+ * process-wide.  Results are bit-identical either way.
+ * PAAC_OPT_FP32_TENSOR_CORES: != 0 runs every contraction of the CUDA-core path (PAAC_FP32 on either network, and
+ * PAAC_BF16 with PAAC_OPT_CUDA_CORES_ONLY) on the tensor cores at float accuracy: each float operand is split into two
+ * TF32 pieces (22 significant bits together) and three tcgen05 passes (hi*hi + hi*lo + lo*hi) are accumulated in one
+ * float accumulator; what is dropped is below 2^-21 of a product, so results stay within the 1e-4 tolerance of the
+ * float path, free-running over ten updates included.  Default 0:
+ * with the 20 to 160 rows of the float configurations a 128-row tensor tile is mostly padding. */
+enum { PAAC_OPT_CUDA_CORES_ONLY = 1, PAAC_OPT_TC_WGRAD_LAYERS = 2, PAAC_OPT_CUDA_GRAPHS = 3, PAAC_OPT_DEPENDENT_LAUNCH = 4,
+       PAAC_OPT_FP32_TENSOR_CORES = 5 };
 int paac_set_option(paac_ctx* ctx, int option, int value);
 
 /* Failure-path check that cannot hang: launches one small kernel whose only thread block waits, at most

@@ -280,6 +280,7 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   }
   c->ws_bytes = need;
   carve(c, c->ws);
+  c->lc.error_word = &c->stats->error_word;
   cudaMemsetAsync(c->ws, 0, need, c->st);
   cudaMemsetAsync(c->forced, 0xFF, (size_t)c->B * sizeof(int32_t), c->st);
   launch_init_params(c->lc, c->nd, seed, c->theta);
@@ -487,6 +488,7 @@ int paac_set_option(paac_ctx* c, int option, int value) {
   if (option == PAAC_OPT_TC_WGRAD_LAYERS) { c->tc_wgrad_mask = value & 0xF; drop_graphs(c); return PAAC_OK; }
   if (option == PAAC_OPT_CUDA_GRAPHS) { c->graphs_on = value != 0; drop_graphs(c); return PAAC_OK; }
   if (option == PAAC_OPT_DEPENDENT_LAUNCH) { pdl_enabled() = value != 0; drop_graphs(c); return PAAC_OK; }
+  if (option == PAAC_OPT_FP32_TENSOR_CORES) { c->lc.fp32_tensor_cores = value != 0; drop_graphs(c); return PAAC_OK; }
   return PAAC_ERR_ARG;
 }
 

@@ -204,6 +204,8 @@ struct LaunchCtx {
   bool profiling = false;             // record a CUDA event pair around every launch
   bool serialize_next = true;         // the next launch takes plain stream order (no overlap with its predecessor)
   bool host_failure = false;          // a launch could not be prepared on the host (sticky; reported as PAAC_ERR_CUDA)
+  bool fp32_tensor_cores = false;     // the float path's contractions go through the three-pass tensor-core kernel
+  uint32_t* error_word = nullptr;     // device word the bounded waits of that kernel report to
   static constexpr int MAX_PENDING = 512;
   cudaEvent_t ev[MAX_PENDING][2];
   int ev_kid[MAX_PENDING];

@@ -1,7 +1,7 @@
 // The network's layers as contractions on the CUDA cores (float accumulate):
 // forward with fused bias + ReLU, data gradients with the ReLU mask of the layer
 // below fused, weight gradients as split-k partial sums reduced in a fixed order.
-#include "gemm_simt.cuh"
+#include "gemm_tc3.cuh"
 #include "kernels.h"
 
 namespace paac {
@@ -28,7 +28,7 @@ static void reduce_wgrad(LaunchCtx& lc, const float* part, int splits, int part_
 template <class G, class TIn, class T, class TW>
 static void conv_fwd(LaunchCtx& lc, int kid, const TIn* x, const TW* w, const float* bias, T* out, int n,
                      float scale) {
-  gemm_simt(lc, kid, n * G::OH * G::OW, G::CO, G::KK, 1, ConvWindowOp<G, TIn>{x}, RowMajorOp<TW>{w, G::KK},
+  gemm_f32(lc, kid, n * G::OH * G::OW, G::CO, G::KK, 1, ConvWindowOp<G, TIn>{x}, RowMajorOp<TW>{w, G::KK},
             BiasReluEp<T>{out, bias, G::CO, scale});
 }
 // out[m][n] = relu(sum over splits (in order) of part[split][m][n] + bias[n])
@@ -53,10 +53,10 @@ static void fc_fwd(LaunchCtx& lc, int kid, const T* x, const TW* w, const float*
                    int IN, int F, float* scratch) {
   const int splits = scratch != nullptr ? pick_splits(n, F, IN) : 1;
   if (splits <= 1) {
-    gemm_simt(lc, kid, n, F, IN, 1, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, BiasReluEp<T>{out, bias, F, 1.f});
+    gemm_f32(lc, kid, n, F, IN, 1, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, BiasReluEp<T>{out, bias, F, 1.f});
     return;
   }
-  gemm_simt(lc, kid, n, F, IN, splits, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, PartialEp{scratch, n, F});
+  gemm_f32(lc, kid, n, F, IN, splits, RowMajorOp<T>{x, IN}, RowMajorOp<TW>{w, IN}, PartialEp{scratch, n, F});
   KernelScope scope(lc, kid);
   int blocks = (n * F + 255) / 256;
   if (blocks > 1184) blocks = 1184;
@@ -67,11 +67,11 @@ static void conv_dgrad(LaunchCtx& lc, int kid, const T* g, const TW* w, const T*
   if constexpr (G::S == 2 && G::K == 4 && G::H % 2 == 0 && G::W % 2 == 0) {
     // four parity classes, each a dense contraction over its own four taps (a quarter of the multiply-adds)
     for (int z = 0; z < 4; ++z)
-      gemm_simt(lc, kid, n * (G::H / 2) * (G::W / 2), G::C, 4 * G::CO, 1, ConvDgradClassOp<G, T>{g, z >> 1, z & 1},
+      gemm_f32(lc, kid, n * (G::H / 2) * (G::W / 2), G::C, 4 * G::CO, 1, ConvDgradClassOp<G, T>{g, z >> 1, z & 1},
                 ConvWeightClassOp<G, TW>{w, z >> 1, z & 1}, ReluMaskClassEp<G, T>{gin, act_in, z >> 1, z & 1});
     return;
   }
-  gemm_simt(lc, kid, n * G::H * G::W, G::C, G::K * G::K * G::CO, 1, ConvDgradOp<G, T>{g}, ConvWeightTOp<G, TW>{w},
+  gemm_f32(lc, kid, n * G::H * G::W, G::C, G::K * G::K * G::CO, 1, ConvDgradOp<G, T>{g}, ConvWeightTOp<G, TW>{w},
             ReluMaskEp<T>{gin, act_in, G::C});
 }
 template <class G, class TIn, class T>
@@ -79,20 +79,20 @@ static void conv_wgrad(LaunchCtx& lc, int kid, const T* g, const TIn* x, int n, 
                        float* gb, float* scratch) {
   const int M = G::CO, N = G::KK + 1, K = n * G::OH * G::OW;
   const int splits = pick_splits(M, N, K);
-  gemm_simt(lc, kid, M, N, K, splits, ColMajorOp<T>{g, G::CO}, ConvWindowTOp<G, TIn>{x}, PartialEp{scratch, M, N});
+  gemm_f32(lc, kid, M, N, K, splits, ColMajorOp<T>{g, G::CO}, ConvWindowTOp<G, TIn>{x}, PartialEp{scratch, M, N});
   reduce_wgrad(lc, scratch, splits, M, 0, M, G::KK, scale, gw, gb);
 }
 template <class T, class TW>
 static void fc_dgrad(LaunchCtx& lc, int kid, const T* g, const TW* w, const T* act_in, T* gin, int n,
                      int IN, int F) {
-  gemm_simt(lc, kid, n, IN, F, 1, RowMajorOp<T>{g, F}, ColMajorOp<TW>{w, IN}, ReluMaskEp<T>{gin, act_in, IN});
+  gemm_f32(lc, kid, n, IN, F, 1, RowMajorOp<T>{g, F}, ColMajorOp<TW>{w, IN}, ReluMaskEp<T>{gin, act_in, IN});
 }
 template <class T>
 static void fc_wgrad(LaunchCtx& lc, int kid, const T* g, const T* x, int n, int IN, int F, float* gw,
                      float* gb, float* scratch) {
   const int M = F, N = IN + 1, K = n;
   const int splits = pick_splits(M, N, K);
-  gemm_simt(lc, kid, M, N, K, splits, ColMajorOp<T>{g, F}, ColMajorOnesOp<T>{x, IN, IN}, PartialEp{scratch, M, N});
+  gemm_f32(lc, kid, M, N, K, splits, ColMajorOp<T>{g, F}, ColMajorOnesOp<T>{x, IN, IN}, PartialEp{scratch, M, N});
   reduce_wgrad(lc, scratch, splits, M, 0, M, IN, 1.f, gw, gb);
 }
 
@@ -215,10 +215,10 @@ template <class T, class TW>
 static void heads_backward_t(LaunchCtx& lc, const NetDims& nd, const TW* w, const T* h, int n,
                              const float* dz, const float* dV, T* gact_fc, float* grad, float* scratch) {
   const int A = nd.A, F = nd.F;
-  gemm_simt(lc, KID_HEADS_BWD, n, F, A + 1, 1, HeadGradOp{dz, dV, A}, HeadWeightOp<TW>{w + nd.pi_w, w + nd.v_w, F, A},
+  gemm_f32(lc, KID_HEADS_BWD, n, F, A + 1, 1, HeadGradOp{dz, dV, A}, HeadWeightOp<TW>{w + nd.pi_w, w + nd.v_w, F, A},
             ReluMaskEp<T>{gact_fc, h, F});
   const int splits = pick_splits(A + 1, F + 1, n);
-  gemm_simt(lc, KID_HEADS_BWD, A + 1, F + 1, n, splits, HeadGradTOp{dz, dV, A}, ColMajorOnesOp<T>{h, F, F},
+  gemm_f32(lc, KID_HEADS_BWD, A + 1, F + 1, n, splits, HeadGradTOp{dz, dV, A}, ColMajorOnesOp<T>{h, F, F},
             PartialEp{scratch, A + 1, F + 1});
   reduce_wgrad(lc, scratch, splits, A + 1, 0, A, F, 1.f, grad + nd.pi_w, grad + nd.pi_b);
   reduce_wgrad(lc, scratch, splits, A + 1, A, 1, F, 1.f, grad + nd.v_w, grad + nd.v_b);

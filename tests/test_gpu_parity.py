@@ -46,6 +46,50 @@ def test_config2_nips_fp32_params_after_10_updates(orc):
     g.close()
 
 
+@pytest.mark.parametrize("index,updates", [(0, 3), (1, 10)])
+def test_float_configurations_on_the_tensor_cores(orc, index, updates):
+    """The float path with every contraction on the tensor cores (operands split into two TF32 pieces, three passes,
+    float accumulator): same float tolerances as the CUDA-core path, no re-synchronisation."""
+    cfg = CONFIGS[index]
+    o, g = make_pair(orc, cfg)
+    g.set_option(pb.OPT_FP32_TENSOR_CORES, 1)
+    mism = 0
+    for it in range(updates):
+        ro, r1 = check_rollout(orc, o, g, TOL["fp32"])
+        up, st, r2 = check_update(orc, o, g, TOL["fp32"], check_acts=(it < 2))
+        mism += r1["action_mismatches"]
+    assert rel(g.params(), o.theta) <= TOL_PARAMS_10
+    assert rel(g.debug_read(pb.DBG_RMS), o.m) <= TOL_PARAMS_10
+    assert mism <= 1
+    assert g.error_word() == 0
+    g.close()
+
+
+def test_float_tensor_core_option_on_the_nature_network(orc):
+    """The three-pass kernel with bf16 storage and the larger network (CUDA-core-only mode routed through it): ragged
+    batch, several tiles in every dimension; compared with the CUDA-core contractions on the same rollout."""
+    outs = []
+    for three_pass in (0, 1):
+        g = pb.Paac("nature", 37, 3, 18, seed=5, precision=pb.BF16, lr=0.0224, term_denom=50)
+        g.set_option(pb.OPT_CUDA_CORES_ONLY, 1)
+        g.set_option(pb.OPT_FP32_TENSOR_CORES, three_pass)
+        if outs:
+            g.force_actions(outs[0]["actions"])
+        g.rollout()
+        acts = g.debug_read(pb.DBG_ACTIONS).copy()
+        st = g.update()
+        assert g.error_word() == 0
+        outs.append(dict(actions=acts, sampled=g.debug_read(pb.DBG_SAMPLED).copy(),
+                         logits=g.debug_read(pb.DBG_LOGITS).copy(), grad=g.debug_read(pb.DBG_GRAD).copy(),
+                         norm=st["grad_norm"]))
+        g.close()
+    assert np.mean(outs[0]["sampled"] != outs[1]["sampled"]) <= 0.02
+    assert rel(outs[0]["logits"], outs[1]["logits"]) <= TOL["bf16"]
+    d = outs[0]["grad"].astype(np.float64) - outs[1]["grad"]
+    assert np.linalg.norm(d) / np.linalg.norm(outs[1]["grad"]) <= TOL["bf16"]
+    assert abs(outs[0]["norm"] - outs[1]["norm"]) <= TOL["bf16"] * outs[1]["norm"]
+
+
 @pytest.mark.parametrize("own_stream", [False, True])
 def test_config2_free_running_actions_agree(orc, own_stream):
     """Without forcing: both sides sample for themselves; with float parameters the draws agree.  On a stream

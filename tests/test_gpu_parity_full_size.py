@@ -65,7 +65,7 @@ def test_config5_full_size_iteration_against_the_oracle(orc, capsys):
 
 
 def _free_run_then_compare(orc, cfg, updates, capsys):
-    """§ protocol for the bf16 configurations: the library runs `updates` iterations by itself on a stream of its
+    """Late-update check for the bf16 configurations: the library runs `updates` iterations by itself on a stream of its
     own (CUDA graphs replay from the third), then the oracle adopts its state and both do one more iteration
     that is compared tensor by tensor, once from the library's own forward pass and once from identical ones."""
     import torch
