@@ -11,59 +11,81 @@ namespace paac {
 
 constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16, SG_THREADS = 256;
 
-template <class LA, class LB, class EP>
+// BM = rows of the output tile: 64, or 32 / 16 for contractions with at most that many rows (the weight gradients of
+// layers with 16 or 32 output channels, a batch of four states), where most of a 64-row tile's multiply-adds would be
+// padding.
+template <int BM, class LA, class LB, class EP>
 __global__ void __launch_bounds__(SG_THREADS)
 gemm_simt_kernel(int M, int N, int K, int k_per_split, LA la, LB lb, EP ep) {
   pdl_entry();
-  __shared__ float As[SG_BK][SG_BM + 4];
+  constexpr int RM = BM / 16;                    // rows per thread
+  __shared__ float As[SG_BK][BM + 4];
   __shared__ float Bs[SG_BK][SG_BN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int m0 = blockIdx.x * SG_BM, n0 = blockIdx.y * SG_BN, split = blockIdx.z;
+  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * SG_BN, split = blockIdx.z;
   const int k_begin = split * k_per_split;
   const int k_end = min(K, k_begin + k_per_split);
-  float acc[4][4];
+  float acc[RM][4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < RM; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
-  for (int k0 = k_begin; k0 < k_end; k0 += SG_BK) {
+  // operand values of one k block, fetched into registers one block ahead of the multiply-adds that use them, so that
+  // the loads' latency overlaps the arithmetic of the block before (the order of the additions does not change)
+  constexpr int NA = BM * SG_BK / SG_THREADS, NB = SG_BN * SG_BK / SG_THREADS;
+  float ra[NA], rb[NB];
+  auto fetch = [&](int k0) {
 #pragma unroll
-    for (int i = 0; i < SG_BM * SG_BK / SG_THREADS; ++i) {
+    for (int i = 0; i < NA; ++i) {
       const int idx = tid + i * SG_THREADS;
       int kk, mm;
-      if (LA::K_CONTIG) { kk = idx % SG_BK; mm = idx / SG_BK; } else { mm = idx % SG_BM; kk = idx / SG_BM; }
+      if (LA::K_CONTIG) { kk = idx % SG_BK; mm = idx / SG_BK; } else { mm = idx % BM; kk = idx / BM; }
       const int m = m0 + mm, k = k0 + kk;
-      As[kk][mm] = (m < M && k < k_end) ? la(m, k) : 0.f;
+      ra[i] = (m < M && k < k_end) ? la(m, k) : 0.f;
     }
 #pragma unroll
-    for (int i = 0; i < SG_BN * SG_BK / SG_THREADS; ++i) {
+    for (int i = 0; i < NB; ++i) {
       const int idx = tid + i * SG_THREADS;
       int kk, nn;
       if (LB::K_CONTIG) { kk = idx % SG_BK; nn = idx / SG_BK; } else { nn = idx % SG_BN; kk = idx / SG_BN; }
       const int n = n0 + nn, k = k0 + kk;
-      Bs[kk][nn] = (n < N && k < k_end) ? lb(n, k) : 0.f;
+      rb[i] = (n < N && k < k_end) ? lb(n, k) : 0.f;
+    }
+  };
+  if (k_begin < k_end) fetch(k_begin);
+  for (int k0 = k_begin; k0 < k_end; k0 += SG_BK) {
+#pragma unroll
+    for (int i = 0; i < NA; ++i) {
+      const int idx = tid + i * SG_THREADS;
+      if (LA::K_CONTIG) As[idx % SG_BK][idx / SG_BK] = ra[i]; else As[idx / BM][idx % BM] = ra[i];
+    }
+#pragma unroll
+    for (int i = 0; i < NB; ++i) {
+      const int idx = tid + i * SG_THREADS;
+      if (LB::K_CONTIG) Bs[idx % SG_BK][idx / SG_BK] = rb[i]; else Bs[idx / SG_BN][idx % SG_BN] = rb[i];
     }
     __syncthreads();
+    if (k0 + SG_BK < k_end) fetch(k0 + SG_BK);
 #pragma unroll
     for (int kk = 0; kk < SG_BK; ++kk) {
-      float a[4], b[4];
+      float a[RM], b[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+      for (int i = 0; i < RM; ++i) a[i] = As[kk][ty * RM + i];
 #pragma unroll
       for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < RM; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
     }
     __syncthreads();
   }
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int i = 0; i < RM; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int m = m0 + ty * 4 + i, n = n0 + tx * 4 + j;
+      const int m = m0 + ty * RM + i, n = n0 + tx * 4 + j;
       if (m < M && n < N) ep(m, n, acc[i][j], split);
     }
 }
@@ -74,8 +96,14 @@ inline void gemm_simt(LaunchCtx& lc, int kid, int M, int N, int K, int splits, L
   KernelScope scope(lc, kid);
   int kps = (K + splits - 1) / splits;
   kps = (kps + SG_BK - 1) / SG_BK * SG_BK;
+  if (M <= 32) {
+    dim3 grid(1, (N + SG_BN - 1) / SG_BN, (K + kps - 1) / kps);
+    if (M <= 16) launch_kernel(lc, gemm_simt_kernel<16, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
+    else launch_kernel(lc, gemm_simt_kernel<32, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
+    return;
+  }
   dim3 grid((M + SG_BM - 1) / SG_BM, (N + SG_BN - 1) / SG_BN, (K + kps - 1) / kps);
-  launch_kernel(lc, gemm_simt_kernel<LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
+  launch_kernel(lc, gemm_simt_kernel<SG_BM, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
 }
 // number of k-splits gemm_simt will really launch for a requested count
 inline int gemm_simt_splits(int K, int splits) {
