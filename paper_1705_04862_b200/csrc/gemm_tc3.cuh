@@ -9,11 +9,11 @@
 // Operands come from the same index functors and results go to the same epilogue functors as the CUDA-core
 // kernel, so every layer of the float path (forward, data and weight gradients, split-k included) can run through it.
 // One CTA per 128 x 64 output tile and k split; 544 threads:
-//   warps 0-15 producers: thread = (tile row, one of four groups); per block of 32 k it evaluates eight of its row's 32
-//              operand values, splits them, and writes them into the hi and the lo image (128-byte rows, 128-byte
-//              swizzle); threads of the first 64 rows do the same for the B rows; then the thread adds its sixteen
-//              columns of the finished product of the block before to a running sum in registers (round to nearest),
-//              and after the last block calls the epilogue functor;
+//   warps 0-15 producers: per block of 32 k a thread evaluates two 16-byte chunks (four k of one row) of A and one of B,
+//              splits them, and writes them into the hi and the lo image (128-byte rows, 128-byte swizzle); then the
+//              thread (= tile row, one of four column groups) adds its sixteen columns of the finished product of
+//              the block before to a running sum in registers (round to nearest), and after the last block calls
+//              the epilogue functor;
 //   warp 16    lane 0 issues twelve MMAs per block (three passes of four K = 8 steps, small terms first) into one of
 //              two accumulators, starting each block from zero, and commits.
 // Only the twelve steps of one block are summed inside the tensor core, whose accumulation does not round to nearest;
@@ -29,7 +29,7 @@ namespace paac {
 
 constexpr int T3_BM = 128, T3_BN = 64, T3_BK = 32, T3_STAGES = 2;
 constexpr int T3_PWARPS = 16, T3_THREADS = (T3_PWARPS + 1) * 32;      // producer warps + the issuing warp
-constexpr int T3_GROUPS = T3_PWARPS / 4, T3_CHUNKS = 8 / T3_GROUPS, T3_COLS = T3_BN / T3_GROUPS;
+constexpr int T3_GROUPS = T3_PWARPS / 4, T3_COLS = T3_BN / T3_GROUPS;
 constexpr uint32_t T3_A_BYTES = T3_BM * 128, T3_B_BYTES = T3_BN * 128, T3_STAGE_BYTES = 2 * T3_A_BYTES + 2 * T3_B_BYTES;
 constexpr int T3_SMEM = T3_STAGES * T3_STAGE_BYTES + 1024;
 
@@ -110,7 +110,7 @@ gemm_tc3_kernel(int M, int N, int K, int k_per_split, LA la, LB lb, EP ep, uint3
     // thread = (tile row, group): the group picks which 16-byte chunks of the row it fills and which accumulator
     // columns it sums; the row is also the thread's lane of tensor memory (warp % 4 selects the 32-lane quarter)
     const int row = threadIdx.x & 127, grp = threadIdx.x >> 7;
-    const int m = m0 + row, n = n0 + row;
+    const int m = m0 + row;
     float sum[T3_COLS];
 #pragma unroll
     for (int j = 0; j < T3_COLS; ++j) sum[j] = 0.f;
@@ -131,32 +131,62 @@ gemm_tc3_kernel(int M, int N, int K, int k_per_split, LA la, LB lb, EP ep, uint3
       if (lane == 0) mbar_arrive(&sh.acc_empty[a]);
       return true;
     };
+    // Operand values of one k block are fetched into registers one block ahead of their use, so that the loads'
+    // latency overlaps the wait for the stage, the read-out of the accumulator and the MMAs of the block before.
+    // Which 16-byte chunks (four k of one row) a thread fetches follows the operand's layout in memory, so that a
+    // warp's loads are contiguous: eight neighbouring lanes take the eight chunks of one row where k is contiguous,
+    // 32 lanes take 32 rows where the row index is.
+    constexpr int A_SLOTS = T3_BM * 8 / (T3_PWARPS * 32);          // chunks of A per thread (2); B has one
+    static_assert(T3_BN * 8 == T3_PWARPS * 32, "one chunk of B per producer thread");
+    int a_row[A_SLOTS], a_chunk[A_SLOTS];
+#pragma unroll
+    for (int i = 0; i < A_SLOTS; ++i) {
+      const int slot = (int)threadIdx.x + i * T3_PWARPS * 32;
+      if (LA::K_CONTIG) { a_row[i] = slot >> 3; a_chunk[i] = slot & 7; }
+      else { a_row[i] = slot & (T3_BM - 1); a_chunk[i] = slot / T3_BM; }
+    }
+    const int b_row = LB::K_CONTIG ? (int)threadIdx.x >> 3 : (int)threadIdx.x & (T3_BN - 1);
+    const int b_chunk = LB::K_CONTIG ? (int)threadIdx.x & 7 : (int)threadIdx.x / T3_BN;
+    float xa[A_SLOTS][4], xb[4];
+    auto fetch = [&](int kb) {
+      const int k0 = k_begin + kb * T3_BK;
+#pragma unroll
+      for (int i = 0; i < A_SLOTS; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int k = k0 + 4 * a_chunk[i] + j;
+          xa[i][j] = (m0 + a_row[i] < M && k < k_end) ? la(m0 + a_row[i], k) : 0.f;
+        }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int k = k0 + 4 * b_chunk + j;
+        xb[j] = (n0 + b_row < N && k < k_end) ? lb(n0 + b_row, k) : 0.f;
+      }
+    };
+    if (num_kb > 0) fetch(0);
     for (int kb = 0; kb < num_kb; ++kb) {
-      const int s = kb % T3_STAGES, k0 = k_begin + kb * T3_BK;
+      const int s = kb % T3_STAGES;
       const bool ok = mbar_wait(&sh.empty[s], ((kb / T3_STAGES) & 1) ^ 1, &sh.abort, error_word, ERR_WAIT_EMPTY);
       if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
       const uint32_t a_hi = tiles + s * T3_STAGE_BYTES, a_lo = a_hi + T3_A_BYTES, b_hi = a_lo + T3_A_BYTES, b_lo = b_hi + T3_B_BYTES;
+      uint4 hi, lo;
 #pragma unroll
-      for (int c = grp * T3_CHUNKS; c < (grp + 1) * T3_CHUNKS; ++c) {
-        float x[4];
-        uint4 hi, lo;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { const int k = k0 + 4 * c + j; x[j] = (m < M && k < k_end) ? la(m, k) : 0.f; }
-        split_tf32x4(x, hi, lo);
-        const uint32_t off = sw128_offset(row, c);
+      for (int i = 0; i < A_SLOTS; ++i) {
+        split_tf32x4(xa[i], hi, lo);
+        const uint32_t off = sw128_offset((uint32_t)a_row[i], (uint32_t)a_chunk[i]);
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_hi + off), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a_lo + off), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
-        if (row < T3_BN) {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) { const int k = k0 + 4 * c + j; x[j] = (n < N && k < k_end) ? lb(n, k) : 0.f; }
-          split_tf32x4(x, hi, lo);
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_hi + off), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
-          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_lo + off), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
-        }
+      }
+      {
+        split_tf32x4(xb, hi, lo);
+        const uint32_t off = sw128_offset((uint32_t)b_row, (uint32_t)b_chunk);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_hi + off), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(b_lo + off), "r"(lo.x), "r"(lo.y), "r"(lo.z), "r"(lo.w) : "memory");
       }
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh.full[s]);
+      if (kb + 1 < num_kb) fetch(kb + 1);
       if (kb >= 1 && !collect(kb - 1)) { alive = false; break; }
     }
     if (alive && num_kb > 0 && collect(num_kb - 1) && m < M) {
