@@ -321,16 +321,18 @@ def run_ours(args, cfg):
         host_v = torch.zeros(n_e, dtype=torch.float32).pin_memory()
         g.update()
 
-        def e2e_step():
+        def e2e_step(first=False):
+            # s_0 of an iteration is s_{t_max} of the one before (Algorithm 1) and already on the device: only the
+            # first iteration sends it; every later one sends t_max states
             for t in range(T):
-                g.act_host(t, host_frames[t], host_a, host_v)
+                g.act_host(t, host_frames[t] if (first or t > 0) else None, host_a, host_v)
                 g.observe_host(t, host_r[t], host_t[t])
             g.act_host(T, host_frames[T], None, host_v)
             return g.update(sync=True)
 
         Ke = max(3, min(K, 10))
-        for _ in range(2):
-            e2e_step()
+        e2e_step(first=True)
+        e2e_step()
         barrier()
         w0 = time.time()
         for _ in range(Ke):
@@ -339,7 +341,7 @@ def run_ours(args, cfg):
         e_sec = (time.time() - w0) / Ke
         e_sec = max_over_ranks(e_sec, dist, "cuda")
         e2e = {"value": whole_job_value(n_e * T, world, e_sec * 1e3), "unit": "env-steps/s", "ms_per_step": e_sec * 1e3,
-               "h2d_bytes_per_step": (T + 1) * n_e * FRAME_BYTES + 2 * T * n_e,
+               "h2d_bytes_per_step": T * n_e * FRAME_BYTES + 2 * T * n_e,
                "d2h_bytes_per_step": T * n_e * 4 + (T + 1) * n_e * 4 + 32,
                "api": "paac_act_host / paac_observe_host / paac_update, pinned host buffers, wall clock"}
     del frames_dev

@@ -170,7 +170,11 @@ const char* paac_strerror(int status);
 /* Step t of a rollout with host frames s_t [n_e][84][84][4] (pinned memory advised):
  * copies them in, evaluates the network, samples a_t, copies actions (and values, if
  * values != NULL) out.  t == t_max evaluates the bootstrap value only (actions may be
- * NULL).  Synchronises.  t must run 0, 1, ..., t_max in order. */
+ * NULL).  Synchronises.  t must run 0, 1, ..., t_max in order.
+ * frames may be NULL at t == 0 when the call before it on this context was paac_act_host(t_max) of the previous
+ * rollout (with paac_observe_host / paac_update in between or not): s_0 of a rollout is s_{t_max} of the one before
+ * (Algorithm 1), and those frames are already on the device, so nothing is copied; the network is evaluated again,
+ * with the current parameters.  Anywhere else a NULL frames pointer is PAAC_ERR_ARG. */
 int paac_act_host(paac_ctx* ctx, int t, const uint8_t* frames /* host */, int32_t* actions /* host, out */,
                   float* values /* host, out, nullable */);
 

@@ -199,7 +199,8 @@ class Paac:
 
     # -- external environments -----------------------------------------------------------------
     def act_host(self, t, frames, actions=None, values=None):
-        _check(lib().paac_act_host(self._h, t, _host_ptr(frames), _host_ptr(actions) if actions is not None else None,
+        _check(lib().paac_act_host(self._h, t, _host_ptr(frames) if frames is not None else None,
+                                   _host_ptr(actions) if actions is not None else None,
                                    _host_ptr(values) if values is not None else None))
 
     def observe_host(self, t, rewards, terminals):

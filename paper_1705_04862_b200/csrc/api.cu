@@ -22,6 +22,7 @@ struct paac_ctx {
   uint64_t env_step;       // global step index of the environments (same for all)
   bool rollout_fresh;      // a rollout has completed since the last update
   int host_t;              // external-environment mode: next expected step
+  bool host_next_valid;    // the bootstrap state of the last host-mode rollout sits where step 0 of the next one goes
   bool forced_on;
   int tc_wgrad_mask;       // bit l: layer l's weight gradient runs on the tensor cores
   GradSegments grad_segs;  // partial-sum regions of the update in flight
@@ -300,6 +301,7 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
 int paac_rollout(paac_ctx* c, paac_rollout_view* view) {
   if (!c) return PAAC_ERR_ARG;
   if (c->host_t != 0) return PAAC_ERR_STATE;
+  c->host_next_valid = false;
   c->cur ^= 1;
   uint8_t* fr = c->frames[c->cur];
   uint8_t* nxt = c->frames[c->cur ^ 1];
@@ -517,12 +519,14 @@ int paac_profile_read(paac_ctx* c, int max_entries, const char** names, double* 
 // ---- external-environment mode ------------------------------------------------------------------
 int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, float* values) {
   if (c) c->lc.serialize_next = true;
-  if (!c || !frames || t < 0 || t > c->t_max || (t < c->t_max && !actions)) return PAAC_ERR_ARG;
+  if (!c || t < 0 || t > c->t_max || (t < c->t_max && !actions)) return PAAC_ERR_ARG;
   if (t != c->host_t) return PAAC_ERR_STATE;
+  // s_0 of a rollout is s_{t_max} of the one before (Algorithm 1): those frames are on the device already
+  if (!frames && !(t == 0 && c->host_next_valid)) return PAAC_ERR_ARG;
   const size_t fstep = (size_t)c->n_e * FRAME_BYTES;
   if (t == 0) c->cur ^= 1;
   uint8_t* dst = t < c->t_max ? c->frames[c->cur] + t * fstep : c->frames[c->cur ^ 1];
-  if (cudaMemcpyAsync(dst, frames, fstep, cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
+  if (frames && cudaMemcpyAsync(dst, frames, fstep, cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
     cudaGetLastError(); return PAAC_ERR_CUDA;
   }
   const bool sample = t < c->t_max;
@@ -533,7 +537,7 @@ int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, f
   if (cudaStreamSynchronize(c->st) != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
   if (t == c->t_max) {
     launch_advance_step(c->lc, c->step_dev, (uint32_t)c->t_max);
-    c->host_t = 0; c->env_step += c->t_max; c->rollout_fresh = true;
+    c->host_t = 0; c->env_step += c->t_max; c->rollout_fresh = true; c->host_next_valid = true;
   }
   else c->host_t = t + 1;
   return cuda_status(c);

@@ -314,29 +314,39 @@ def test_error_paths(orc):
 
 def test_external_environment_mode_matches_device_environment(orc):
     """Frames, rewards and terminals fed from the host (the oracle's environment) give the same
-    actions, values and update as the on-device environment."""
+    actions, values and update as the on-device environment; in the second iteration step 0 is not
+    sent again (it is the bootstrap state of the first, already on the device)."""
     cfg = CONFIGS[0]
     o, g = make_pair(orc, cfg)
     _, g2 = make_pair(orc, cfg)
     n_e, T = cfg["n_e"], cfg["t_max"]
-    g.rollout()
-    g.update()
-    # replay the same iteration on g2 through the host entry points
-    frames = g.debug_read(pb.DBG_FRAMES).reshape(T, n_e, 84, 84, 4)
-    nxt = g.debug_read(pb.DBG_NEXT_FRAMES).reshape(n_e, 84, 84, 4)
-    rewards = g.debug_read(pb.DBG_REWARDS).reshape(T, n_e)
-    terms = g.debug_read(pb.DBG_TERMINALS).reshape(T, n_e)
-    acts_dev = g.debug_read(pb.DBG_ACTIONS).reshape(T, n_e)
-    for t in range(T):
-        a = np.zeros(n_e, np.int32)
-        v = np.zeros(n_e, np.float32)
-        g2.act_host(t, np.ascontiguousarray(frames[t]), a, v)
-        assert np.array_equal(a, acts_dev[t])
-        g2.observe_host(t, np.ascontiguousarray(rewards[t]), np.ascontiguousarray(terms[t]))
-    vb = np.zeros(n_e, np.float32)
-    g2.act_host(T, np.ascontiguousarray(nxt), None, vb)
-    g2.update()
-    assert np.array_equal(g2.params(), g.params())
+    a = np.zeros(n_e, np.int32)
+    with pytest.raises(pb.PaacError):
+        g2.act_host(0, None, a)                   # nothing on the device yet
+    for it in range(2):
+        g.rollout()
+        g.update()
+        # replay the same iteration on g2 through the host entry points
+        frames = g.debug_read(pb.DBG_FRAMES).reshape(T, n_e, 84, 84, 4)
+        nxt = g.debug_read(pb.DBG_NEXT_FRAMES).reshape(n_e, 84, 84, 4)
+        rewards = g.debug_read(pb.DBG_REWARDS).reshape(T, n_e)
+        terms = g.debug_read(pb.DBG_TERMINALS).reshape(T, n_e)
+        acts_dev = g.debug_read(pb.DBG_ACTIONS).reshape(T, n_e)
+        vals_dev = g.debug_read(pb.DBG_VALUES).reshape(T + 1, n_e)
+        for t in range(T):
+            v = np.zeros(n_e, np.float32)
+            g2.act_host(t, None if (it == 1 and t == 0) else np.ascontiguousarray(frames[t]), a, v)
+            assert np.array_equal(a, acts_dev[t]) and np.array_equal(v, vals_dev[t])
+            if t == 0:
+                with pytest.raises(pb.PaacError):
+                    g2.act_host(1, None, a)       # only step 0 can be taken from the device
+            g2.observe_host(t, np.ascontiguousarray(rewards[t]), np.ascontiguousarray(terms[t]))
+        vb = np.zeros(n_e, np.float32)
+        g2.act_host(T, np.ascontiguousarray(nxt), None, vb)
+        assert np.array_equal(vb, vals_dev[T])
+        g2.update()
+        assert np.array_equal(g2.params(), g.params())
+        assert np.array_equal(g2.debug_read(pb.DBG_FRAMES), g.debug_read(pb.DBG_FRAMES))
     g.close()
     g2.close()
 
