@@ -3217,7 +3217,7 @@ void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, 
 // A thread owns two of the 512 hidden units: their weight columns live in registers, every row costs it one 4-byte
 // load of h and NK multiply-adds each way, and the row's dz values are broadcast from shared memory.  A CTA walks a
 // contiguous range of rows and leaves its dW / db sums as one more split for the finishing kernel.
-constexpr int HB_THREADS = 256, HB_ROWS = 32;
+constexpr int HB_THREADS = 256, HB_ROWS = 40;      // rows staged at a time: a CTA's whole share at the largest benchmark size
 
 template <int NK>
 __global__ void __launch_bounds__(HB_THREADS, 2)
@@ -3240,6 +3240,12 @@ heads_backward_kernel(const bf16* __restrict__ h, const float* __restrict__ dz, 
   pdl_entry();          // the head weights above were written several kernels ago
   const int r0 = blockIdx.x * rows_per, r1 = min(n, r0 + rows_per);
   for (int rb = r0; rb < r1; rb += HB_ROWS) {
+    // eight rows of h at a time, the next eight fetched while these are used (the loads' latency was the kernel's
+    // bound); the first eight are asked for before the block's dz rows are staged
+    uint32_t hv[8], hn[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      hv[j] = rb + j < r1 ? __ldg(reinterpret_cast<const uint32_t*>(h + (size_t)(rb + j) * F + col)) : 0u;
     __syncthreads();
     for (int i = tid; i < HB_ROWS * NK; i += HB_THREADS) {
       const int r = rb + i / NK, k = i % NK;
@@ -3250,10 +3256,10 @@ heads_backward_kernel(const bf16* __restrict__ h, const float* __restrict__ dz, 
       for (int r = 0; r < HB_ROWS; ++r) accb += dzs[r][tid];        // rows past the end hold zeros
 #pragma unroll 1
     for (int q = 0; q < HB_ROWS && rb + q < r1; q += 8) {
-      uint32_t hv[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j)
-        hv[j] = rb + q + j < r1 ? __ldg(reinterpret_cast<const uint32_t*>(h + (size_t)(rb + q + j) * F + col)) : 0u;
+        hn[j] = (q + 8 + j < HB_ROWS && rb + q + 8 + j < r1)
+                    ? __ldg(reinterpret_cast<const uint32_t*>(h + (size_t)(rb + q + 8 + j) * F + col)) : 0u;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         if (rb + q + j >= r1) break;
@@ -3269,10 +3275,11 @@ heads_backward_kernel(const bf16* __restrict__ h, const float* __restrict__ dz, 
             acc[k4 + i][0] = fmaf(d[i], h0, acc[k4 + i][0]); acc[k4 + i][1] = fmaf(d[i], h1, acc[k4 + i][1]);
           }
         }
-        if (rb + q + j < r1)
-          *reinterpret_cast<uint32_t*>(g_fc + (size_t)(rb + q + j) * F + col) =
-              pack_bf16x2(h0 > 0.f ? g0 : 0.f, h1 > 0.f ? g1 : 0.f);
+        *reinterpret_cast<uint32_t*>(g_fc + (size_t)(rb + q + j) * F + col) =
+            pack_bf16x2(h0 > 0.f ? g0 : 0.f, h1 > 0.f ? g1 : 0.f);
       }
+#pragma unroll
+      for (int j = 0; j < 8; ++j) hv[j] = hn[j];
     }
   }
   // partial sums of this CTA in the layout of the parameters themselves: policy rows [action][hidden unit], the
