@@ -214,6 +214,8 @@ def run_ours(args, cfg):
                 device="cuda:%d" % local, **hp)
     if args.fp32_tensor_cores:
         g.set_option(pb.OPT_FP32_TENSOR_CORES, 1)
+    if args.update_chunks > 1:
+        g.set_option(pb.OPT_UPDATE_CHUNKS, args.update_chunks)
     n_e, T = cfg["n_e"], cfg["t_max"]
     small = cfg["n_e"] < 256
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if small else None
@@ -404,7 +406,8 @@ def run_ours(args, cfg):
         "metric": "env_steps_per_sec", "value": value, "unit": "env-steps/s", "n_gpus": world, "steps": K,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg["precision"], "data": "synthetic",
-        "config": dict(workload_config(cfg), **({"contractions": "3xTF32 tensor cores"} if args.fp32_tensor_cores else {})),
+        "config": dict(workload_config(cfg), **({"contractions": "3xTF32 tensor cores"} if args.fp32_tensor_cores else {}),
+                       **({"update_chunks": args.update_chunks} if args.update_chunks > 1 else {})),
         "updates_per_sec": world * 1e3 / ms_per_step, "rollout_ms": roll_ms, "update_ms": upd_ms,
         "rollout_tflops": roll_flops / (roll_ms * 1e-3) / 1e12,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "sustained": sustained,
@@ -474,6 +477,8 @@ def main():
                     help="seconds of back-to-back iterations in the sustained block (0 = skip it)")
     ap.add_argument("--fp32-tensor-cores", action="store_true",
                     help="float configurations: every contraction as three TF32 tensor-core passes (float-accurate)")
+    ap.add_argument("--update-chunks", type=int, default=1,
+                    help="bf16 configurations: conv2 data gradient / conv1 weight gradient over this many groups of states")
     ap.add_argument("--lr-sweep", action="store_true",
                     help="instead of the throughput line: the alpha = 0.0007 n_e rule on the learnable environment")
     ap.add_argument("--sweep-timesteps", type=int, default=200000)

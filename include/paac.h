@@ -270,9 +270,13 @@ int paac_debug_write(paac_ctx* ctx, int which, const void* src /* host */, size_
  * TF32 pieces (22 significant bits together) and three tcgen05 passes (hi*hi + hi*lo + lo*hi) are accumulated in one
  * float accumulator; what is dropped is below 2^-21 of a product, so results stay within the 1e-4 tolerance of the
  * float path, free-running over ten updates included.  Default 0:
- * with the 20 to 160 rows of the float configurations a 128-row tensor tile is mostly padding. */
+ * with the 20 to 160 rows of the float configurations a 128-row tensor tile is mostly padding.
+ * PAAC_OPT_UPDATE_CHUNKS: 1 (default) .. 4.  With more than one, the tensor-core update runs the second layer's data
+ * gradient and the first layer's weight gradient alternately over that many groups of states, so that a group's slice
+ * of the gradient between them is read back from L2 instead of HBM.  The weight gradient's partial sums are then
+ * added in a different grouping: results agree to float rounding, not bit for bit, with the default. */
 enum { PAAC_OPT_CUDA_CORES_ONLY = 1, PAAC_OPT_TC_WGRAD_LAYERS = 2, PAAC_OPT_CUDA_GRAPHS = 3, PAAC_OPT_DEPENDENT_LAUNCH = 4,
-       PAAC_OPT_FP32_TENSOR_CORES = 5 };
+       PAAC_OPT_FP32_TENSOR_CORES = 5, PAAC_OPT_UPDATE_CHUNKS = 6 };
 int paac_set_option(paac_ctx* ctx, int option, int value);
 
 /* Failure-path check that cannot hang: launches one small kernel whose only thread block waits, at most

@@ -22,7 +22,8 @@ OK, ERR_ARG, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT, ERR_STATE, ERR
  DBG_COUNTERS, DBG_RETURNS, DBG_ADVANTAGES, DBG_DLOGITS, DBG_DVALUES, DBG_GRAD, DBG_RMS, DBG_SAMPLED,
  DBG_ERROR_WORD) = range(17)
 DBG_ACT0, DBG_GACT0 = 32, 48
-OPT_CUDA_CORES_ONLY, OPT_TC_WGRAD_LAYERS, OPT_CUDA_GRAPHS, OPT_DEPENDENT_LAUNCH, OPT_FP32_TENSOR_CORES = 1, 2, 3, 4, 5
+(OPT_CUDA_CORES_ONLY, OPT_TC_WGRAD_LAYERS, OPT_CUDA_GRAPHS, OPT_DEPENDENT_LAUNCH, OPT_FP32_TENSOR_CORES,
+ OPT_UPDATE_CHUNKS) = 1, 2, 3, 4, 5, 6
 
 _DBG_DTYPE = {DBG_FRAMES: np.uint8, DBG_NEXT_FRAMES: np.uint8, DBG_ACTIONS: np.int32, DBG_REWARDS: np.int8,
               DBG_TERMINALS: np.uint8, DBG_COUNTERS: np.int32, DBG_SAMPLED: np.int32, DBG_ERROR_WORD: np.uint32}

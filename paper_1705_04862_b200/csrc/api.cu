@@ -22,6 +22,7 @@ struct paac_ctx {
   uint64_t env_step;       // global step index of the environments (same for all)
   bool rollout_fresh;      // a rollout has completed since the last update
   int host_t;              // external-environment mode: next expected step
+  int update_chunks;       // > 1: conv2 data gradient and conv1 weight gradient alternate over this many groups of states
   bool host_next_valid;    // the bootstrap state of the last host-mode rollout sits where step 0 of the next one goes
   bool forced_on;
   int tc_wgrad_mask;       // bit l: layer l's weight gradient runs on the tensor cores
@@ -268,6 +269,7 @@ int paac_init(paac_ctx** out, int arch, int n_e, int t_max, int n_actions, const
   if (!c) return PAAC_ERR_CUDA;
   fill_shape(c, arch, n_e, t_max, n_actions, hp);
   c->tc_wgrad_mask = 0xF;
+  c->update_chunks = 1;
   c->gact0_scale = 1.f;
   c->graphs_on = true;
   c->seed = seed; c->device = dev; c->st = (cudaStream_t)hp->stream; c->lc.st = c->st;
@@ -349,8 +351,17 @@ int paac_update(paac_ctx* c, paac_update_stats* stats) {
                      c->grad, c->scratch + c->simt_scratch_off);
     uint32_t* err = &c->stats->error_word;
     c->gact0_scale = 1.f;
+    const bool chunked = use_tc(c) && c->update_chunks > 1 && (c->tc_wgrad_mask & 3) == 3;
     for (int l = L; l >= 0; --l) {
       // tensor-core kernels where they exist, the CUDA-core contraction otherwise
+      if (chunked && l == 1) {
+        // the layer's own weight gradient first, then data gradient and first-layer weight gradient group by group
+        tc_backward_wgrad(c->lc, c->nd, c->frames[c->cur], c->B, c->act, c->gact, c->grad, c->scratch, 1, &c->grad_segs, err);
+        c->gact0_scale = tc_conv1_grad_scale();
+        tc_backward_conv2d_conv1w_chunked(c->lc, c->nd, c->w_images, c->frames[c->cur], c->B, c->act, c->gact, c->grad,
+                                          c->scratch, c->update_chunks, &c->grad_segs, err);
+        break;
+      }
       bool dgrad_done = false;
       if (use_tc(c)) {
         if (l == 3) { tc_backward_dgrad_fc(c->lc, c->w_images, c->B, c->act, c->gact, err); dgrad_done = true; }
@@ -490,6 +501,10 @@ int paac_set_option(paac_ctx* c, int option, int value) {
   if (option == PAAC_OPT_TC_WGRAD_LAYERS) { c->tc_wgrad_mask = value & 0xF; drop_graphs(c); return PAAC_OK; }
   if (option == PAAC_OPT_CUDA_GRAPHS) { c->graphs_on = value != 0; drop_graphs(c); return PAAC_OK; }
   if (option == PAAC_OPT_DEPENDENT_LAUNCH) { pdl_enabled() = value != 0; drop_graphs(c); return PAAC_OK; }
+  if (option == PAAC_OPT_UPDATE_CHUNKS) {
+    if (value < 1 || value > TC_MAX_UPDATE_CHUNKS) return PAAC_ERR_ARG;
+    c->update_chunks = value; drop_graphs(c); return PAAC_OK;
+  }
   if (option == PAAC_OPT_FP32_TENSOR_CORES) { c->lc.fp32_tensor_cores = value != 0; drop_graphs(c); return PAAC_OK; }
   return PAAC_ERR_ARG;
 }

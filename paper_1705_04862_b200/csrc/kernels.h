@@ -71,6 +71,12 @@ float tc_conv1_grad_scale();
 struct GradSegment { const float* part; float* dst; int splits, J, CO; float scale; int first_group, groups, wide; };
 struct GradSegments { GradSegment seg[12]; int n; int total_groups; };
 size_t tc_scratch_floats(int n);
+// the same data gradient followed by the first layer's weight gradient, alternating over `chunks` (at most
+// TC_MAX_UPDATE_CHUNKS) groups of states; notes the weight gradient's partial sums in *segs
+constexpr int TC_MAX_UPDATE_CHUNKS = 4;
+void tc_backward_conv2d_conv1w_chunked(LaunchCtx& lc, const NetDims& nd, const bf16* images, const uint8_t* frames, int n,
+                                       void* const act[], void* const gact[], float* grad, float* scratch, int chunks,
+                                       GradSegments* segs, uint32_t* err);
 void tc_backward_wgrad(LaunchCtx& lc, const NetDims& nd, const uint8_t* frames, int n, void* const act[],
                        void* const gact[], float* grad, float* scratch, int layer, GradSegments* segs, uint32_t* err);
 // sumsq_partials != nullptr: every block also leaves the sum of squares of the gradient values it wrote in

@@ -3134,9 +3134,19 @@ tc_conv1_wgrad_kernel(const uint8_t* __restrict__ frames, const bf16* __restrict
   }
 }
 
+// how many CTAs (= split-k partial sums) the first layer's weight gradient uses for n_states states
+static int tc_conv1_wgrad_splits(int n_states) {
+  const int tiles = (n_states * C1_RASTER * C1_RASTER + 1 + TC_BM - 1) / TC_BM;      // positions -1 .. total - 1
+  int ctas = sm_count() < SWG_MAX_SPLITS ? sm_count() : SWG_MAX_SPLITS;
+  if (ctas > tiles) ctas = tiles;
+  const int per = (tiles + ctas - 1) / ctas;
+  return (tiles + per - 1) / per;
+}
+// launches the kernel on n_states states; its CTAs leave their weight tiles in partial[cta][256][32] and their two
+// bias rows in bias_part[2 cta + i][32]; returns the number of CTAs
 template <class G>
-static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, int n_states, float* gw, float* gb,
-                           float* scratch, GradSegments* segs, uint32_t* err) {
+static int tc_conv1_wgrad_launch(LaunchCtx& lc, const uint8_t* frames, const bf16* g, int n_states, float* partial,
+                                 float* bias_part, uint32_t* err) {
   constexpr int smem = (W1_STAGES * W1_X_ROWS + W1_G_SLOTS * TC_BM) * 128 + W1_RAW_SLOTS * W1_RAW_BYTES + 1024;
   static_assert(smem <= 227 * 1024, "shared memory budget");
   auto kern = tc_conv1_wgrad_kernel<G>;
@@ -3145,13 +3155,17 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
     cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     configured = true;
   }
-  const int tiles = (n_states * C1_RASTER * C1_RASTER + 1 + TC_BM - 1) / TC_BM;      // positions -1 .. total - 1
-  int ctas = sm_count() < SWG_MAX_SPLITS ? sm_count() : SWG_MAX_SPLITS;
-  if (ctas > tiles) ctas = tiles;
-  const int per = (tiles + ctas - 1) / ctas, splits = (tiles + per - 1) / per;
-  float* bias_part = scratch + (size_t)splits * 256 * 32;
+  const int tiles = (n_states * C1_RASTER * C1_RASTER + 1 + TC_BM - 1) / TC_BM;
+  const int splits = tc_conv1_wgrad_splits(n_states), per = (tiles + splits - 1) / splits;
   KernelScope scope(lc, KID_CONV1_WGRAD);
-  launch_kernel_overlapped(lc, kern, splits, W1_THREADS, smem, frames, g, scratch, bias_part, n_states, tiles, per, err);
+  launch_kernel_overlapped(lc, kern, splits, W1_THREADS, smem, frames, g, partial, bias_part, n_states, tiles, per, err);
+  return splits;
+}
+template <class G>
+static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, int n_states, float* gw, float* gb,
+                           float* scratch, GradSegments* segs, uint32_t* err) {
+  float* bias_part = scratch + (size_t)tc_conv1_wgrad_splits(n_states) * 256 * 32;
+  const int splits = tc_conv1_wgrad_launch<G>(lc, frames, g, n_states, scratch, bias_part, err);
   // the gradient rows arrive multiplied by C1_GRAD_SCALE (see tc_backward_dgrad_conv2), the pixels as n * 2^-133
   if (!add_segment(segs, scratch, gw, splits, 256, 32, C1_WGRAD_OUTPUT_SCALE) ||
       !add_segment(segs, bias_part, gb, 2 * splits, 1, 32, C1_BIAS_OUTPUT_SCALE))      // two bias warps per CTA, a row each
@@ -3161,7 +3175,7 @@ static void tc_conv1_wgrad(LaunchCtx& lc, const uint8_t* frames, const bf16* g, 
 // every layer keeps its own partial-sum region until the finishing kernel has run
 static size_t tc_layer_scratch_floats(int n, int layer) {
   switch (layer) {
-    case 0: return (size_t)SWG_MAX_SPLITS * (256 * 32 + 2 * 32);      // per CTA: the weight tile and two bias rows
+    case 0: return (size_t)TC_MAX_UPDATE_CHUNKS * SWG_MAX_SPLITS * (256 * 32 + 2 * 32);      // per chunk and CTA: the weight tile and two bias rows
     case 1: return (size_t)SWG_MAX_SPLITS * (512 * 64 + 64);
     case 2: return (size_t)SWG_MAX_SPLITS * (576 * 64 + 64);
     default: return wg_scratch_floats(n, 3136, 512, 13 * 4);      // 256 x 128 tiles of the 3136 x 512 matrix
@@ -3295,7 +3309,7 @@ heads_backward_kernel(const bf16* __restrict__ h, const float* __restrict__ dz, 
 }
 
 constexpr int HB_MAX_SPLITS = 148;
-static size_t tc_heads_scratch_floats() { return (size_t)HB_MAX_SPLITS * (512 * 20 + 20); }
+static size_t tc_heads_scratch_floats() { return (size_t)HB_MAX_SPLITS * (512 * 20 + 20) + 4; }
 
 bool tc_heads_backward_supported(const NetDims& nd) { return nd.F == 512 && nd.A + 1 <= 20; }
 
@@ -3306,8 +3320,9 @@ void tc_heads_backward(LaunchCtx& lc, const NetDims& nd, const bf16* theta16, co
   if (ctas > n) ctas = n;
   const int rows_per = (n + ctas - 1) / ctas, splits = (n + rows_per - 1) / rows_per;
   float* sc = scratch + tc_layer_scratch_offset(n, 4);
+  // the value row's partial sums are stored as float2: their area starts on an even float (splits * A can be odd)
   float* part_w = sc; float* part_b = part_w + (size_t)splits * 512 * A;
-  float* part_vw = part_b + (size_t)splits * A; float* part_vb = part_vw + (size_t)splits * 512;
+  float* part_vw = part_b + (((size_t)splits * A + 3) & ~(size_t)3); float* part_vb = part_vw + (size_t)splits * 512;
   KernelScope scope(lc, KID_HEADS_BWD);
   if (A + 1 <= 8)
     launch_kernel_overlapped(lc, heads_backward_kernel<8>, splits, HB_THREADS, 0, h, dz, dV, theta16 + nd.pi_w, theta16 + nd.v_w, n, A,
@@ -3418,6 +3433,39 @@ void tc_backward_dgrad_conv3(LaunchCtx& lc, const bf16* images, int n, void* con
   (void)M;
 }
 float tc_conv1_grad_scale() { return C1_GRAD_SCALE; }
+
+// The conv2 data gradient and the conv1 weight gradient over `chunks` groups of states, alternating, so that a group's
+// slice of the gradient at the first layer's output (25.6 KB per state) is read back while it is still in L2.  All groups' partial
+// sums lie one behind the other (weight tiles, then bias rows), in group order, and are added up as one segment.
+void tc_backward_conv2d_conv1w_chunked(LaunchCtx& lc, const NetDims& nd, const bf16* images, const uint8_t* frames, int n,
+                                       void* const act[], void* const gact[], float* grad, float* scratch, int chunks,
+                                       GradSegments* segs, uint32_t* err) {
+  typedef NatConv1 C1;
+  typedef NatConv2 C2;
+  typedef RasterMap<121, 11, 10, 10> Map;
+  if (chunks > TC_MAX_UPDATE_CHUNKS) chunks = TC_MAX_UPDATE_CHUNKS;
+  if (chunks > n) chunks = n;
+  const int per = (n + chunks - 1) / chunks;
+  int total_splits = 0;
+  for (int s0 = 0; s0 < n; s0 += per) total_splits += tc_conv1_wgrad_splits(n - s0 < per ? n - s0 : per);
+  float* part = scratch + tc_layer_scratch_offset(n, 0);
+  float* bias_part = part + (size_t)total_splits * 256 * 32;
+  const size_t a0 = (size_t)C2::H * C2::W * C2::C, g1 = (size_t)C2::OH * C2::OW * C2::CO;      // elements per state
+  int done = 0;
+  for (int s0 = 0; s0 < n; s0 += per) {
+    const int nc = n - s0 < per ? n - s0 : per;
+    bf16* gact0 = (bf16*)gact[0] + (size_t)s0 * a0;
+    tc_shift<C2DgradCfg, ShiftReluMaskEpiS2<Map>, 128, 3, 1>(
+        lc, KID_CONV2_DGRAD, C2DgradCfg{(const bf16*)gact[1] + (size_t)s0 * g1, nc}, images,
+        ShiftReluMaskEpiS2<Map>{Map{nc}, gact0, (const bf16*)act[0] + (size_t)s0 * a0, C1_GRAD_SCALE}, nc * 121, err);
+    done += tc_conv1_wgrad_launch<C1>(lc, frames + (size_t)s0 * FRAME_BYTES, gact0, nc, part + (size_t)done * 256 * 32,
+                                      bias_part + (size_t)done * 2 * 32, err);
+  }
+  const LayerDims* d = nd.layer;
+  if (!add_segment(segs, part, grad + d[0].w_off, total_splits, 256, 32, C1_WGRAD_OUTPUT_SCALE) ||
+      !add_segment(segs, bias_part, grad + d[0].b_off, 2 * total_splits, 1, 32, C1_BIAS_OUTPUT_SCALE))
+    lc.host_failure = true;
+}
 
 void tc_backward_dgrad_conv2(LaunchCtx& lc, const bf16* images, int n, void* const act[], void* const gact[], uint32_t* err,
                              float out_scale) {

@@ -422,6 +422,41 @@ def test_partial_tensor_core_weight_gradient_mask(orc):
     assert abs(grads[0][2] - grads[1][2]) <= TOL["bf16"] * grads[0][2]
 
 
+def test_odd_action_counts_on_the_tensor_core_path(orc):
+    """Action counts and batch sizes whose product is odd: the heads' partial sums (policy rows, policy biases, value
+    row, value bias, one behind the other per split) then start at odd float offsets unless padded; the value row is
+    stored in pairs.  (n_e * t_max <= 148 rows gives one split per row.)"""
+    for n_e, t_max, A in ((37, 5, 5), (33, 3, 19), (41, 1, 7)):
+        cfg = dict(CONFIGS[2], n_e=n_e, t_max=t_max, n_actions=A)
+        o, g = make_pair(orc, cfg)
+        check_rollout(orc, o, g, TOL["bf16"])
+        check_update(orc, o, g, TOL["bf16"])
+        assert g.error_word() == 0
+        g.close()
+
+
+def test_update_in_groups_of_states_matches_the_default(orc):
+    """PAAC_OPT_UPDATE_CHUNKS: the second layer's data gradient and the first layer's weight gradient alternating over
+    2, 3 or 4 groups of states give the default's gradient up to the grouping of the partial sums; against the oracle
+    the usual bf16 tolerances hold."""
+    cfg = dict(CONFIGS[2], n_e=37, n_actions=5)
+    grads = []
+    for chunks in (1, 2, 3, 4):
+        o, g = make_pair(orc, cfg)
+        g.set_option(pb.OPT_UPDATE_CHUNKS, chunks)
+        check_rollout(orc, o, g, TOL["bf16"])
+        check_update(orc, o, g, TOL["bf16"])
+        assert g.error_word() == 0
+        grads.append(g.debug_read(pb.DBG_GRAD).copy())
+        if chunks == 1:
+            for bad in (0, 5):
+                with pytest.raises(pb.PaacError):
+                    g.set_option(pb.OPT_UPDATE_CHUNKS, bad)
+        g.close()
+    for gr in grads[1:]:
+        assert np.abs(gr - grads[0]).max() <= 1e-5 * np.abs(grads[0]).max()
+
+
 @pytest.mark.parametrize("base,iters", [(0, 3), (2, 4)])
 def test_value_based_variant_matches_the_oracle(orc, base, iters):
     """n-step Q-learning on the same framework (Section 2.2, Eqs. 2-4; Section 3), configurations 1 (float, CUDA
