@@ -422,6 +422,35 @@ def test_partial_tensor_core_weight_gradient_mask(orc):
     assert abs(grads[0][2] - grads[1][2]) <= TOL["bf16"] * grads[0][2]
 
 
+def test_shape_sweep_two_implementations_agree():
+    """Forty ragged shapes (environments 1 .. 1025, steps 1 .. 13, actions 2 .. 32, seeded choice) through the bf16
+    network: the tensor-core path and the CUDA-core path of the library finish without a device error and agree on
+    the gradient within the bf16 tolerance (L2).  No oracle here: the point is every shape-dependent offset, split
+    count and tail."""
+    import random
+    rnd = random.Random(3)
+    combos = [(n, t, a) for n in (1, 2, 3, 5, 16, 37, 64, 100, 129, 255) for t in (1, 2, 3, 5, 7)
+              for a in (2, 3, 4, 5, 7, 18, 19, 20, 31, 32)]
+    rnd.shuffle(combos)
+    combos = combos[:36] + [(1000, 13, 19), (1023, 5, 32), (1025, 1, 3), (511, 5, 18)]
+    for n_e, T, A in combos:
+        outs = []
+        for cores_only in (0, 1):
+            g = pb.Paac("nature", n_e, T, A, seed=5, precision=pb.BF16, lr=0.0224, term_denom=50)
+            g.set_option(pb.OPT_CUDA_CORES_ONLY, cores_only)
+            if outs:
+                g.force_actions(outs[0][0])
+            g.rollout()
+            acts = g.debug_read(pb.DBG_ACTIONS).copy()
+            g.update()
+            grad = g.debug_read(pb.DBG_GRAD).copy()
+            assert g.error_word() == 0 and np.isfinite(grad).all(), (n_e, T, A)
+            outs.append((acts, grad))
+            g.close()
+        d = np.linalg.norm(outs[0][1].astype(np.float64) - outs[1][1]) / max(np.linalg.norm(outs[1][1]), 1e-30)
+        assert d <= 5e-2, (n_e, T, A, d)
+
+
 def test_odd_action_counts_on_the_tensor_core_path(orc):
     """Action counts and batch sizes whose product is odd: the heads' partial sums (policy rows, policy biases, value
     row, value bias, one behind the other per split) then start at odd float offsets unless padded; the value row is
