@@ -114,12 +114,15 @@ __host__ __device__ __forceinline__ uint32_t hash_mix(uint32_t x) {
   x ^= x >> 16; x *= HASH_K0; x ^= x >> 15; x *= HASH_K1; x ^= x >> 16;
   return x;
 }
-__host__ __device__ __forceinline__ uint32_t env_hash_base(uint64_t seed, uint32_t env, uint32_t step, uint32_t tag) {
+// the part of the chain that does not depend on the tag (an action, or 0), and the step that takes the tag in
+__host__ __device__ __forceinline__ uint32_t env_hash_prefix(uint64_t seed, uint32_t env, uint32_t step) {
   uint32_t h = hash_mix((uint32_t)seed ^ HASH_K2);
   h = hash_mix(h ^ (uint32_t)(seed >> 32));
   h = hash_mix(h ^ env);
-  h = hash_mix(h ^ step);
-  return hash_mix(h ^ tag);
+  return hash_mix(h ^ step);
+}
+__host__ __device__ __forceinline__ uint32_t env_hash_base(uint64_t seed, uint32_t env, uint32_t step, uint32_t tag) {
+  return hash_mix(env_hash_prefix(seed, env, step) ^ tag);
 }
 
 // ---- network geometry (compile time) ----------------------------------------------

@@ -71,9 +71,16 @@ env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, 
   // hash(e, k, 'GOAL') mod A; its frame is the hashed frame with every byte reduced to its low six bits (a dim
   // texture) and rows [band goal, band (goal + 1)), band = 84 / A, set to 255; an action pays 1 if it is the current
   // state's goal and 0 otherwise.
+  // Two roles run side by side until the action is known: the first warp takes it (SAMPLE), and the first thread of
+  // the second warp prepares everything of the transition that does not depend on it -- the hash chains of this step
+  // and the next up to the point where the action enters, and the environment's counters, whose loads would otherwise
+  // be waited for after the draw.  One hash step, the reward / terminal bits and the frame's base remain.
   __shared__ uint32_t s_base, s_band_lo, s_band_hi;
+  __shared__ int32_t s_action;
   const uint32_t e = blockIdx.x;
-  int32_t a_sampled = 0;
+  const bool stepping = SAMPLE || actions != nullptr;          // else: the start frames (step 0, tag 0)
+  uint32_t pre_step = 0u, pre_next = 0u, step = 0u;
+  int32_t len = 0, ret = 0, episodes = 0;
   if (SAMPLE && threadIdx.x < 32) {
     const int lane = threadIdx.x, A = ht.A;
     const float bias = lane < A ? __ldg(ht.bpi + lane) : (lane == A ? __ldg(ht.bv) : 0.f);   // older than the previous kernel
@@ -81,41 +88,56 @@ env_step_kernel(uint64_t seed, int n_e, const uint64_t* __restrict__ step_base, 
     float sum = -INFINITY;
     if (lane <= A) sum = (ht.hp[(size_t)e * 32 + lane] + ht.hp[((size_t)n_e + e) * 32 + lane]) + bias;
     const float z = lane < A ? sum : -INFINITY;
-    a_sampled = warp_finish_heads(ht.mode, z, __shfl_sync(0xffffffffu, sum, A), lane, A, (size_t)e, ht.logits, ht.values, true,
-                                  seed, *step_base + t, ht.forced, ht.actions, ht.sampled, ht.uniforms);
+    const int32_t a = warp_finish_heads(ht.mode, z, __shfl_sync(0xffffffffu, sum, A), lane, A, (size_t)e, ht.logits, ht.values, true,
+                                        seed, *step_base + t, ht.forced, ht.actions, ht.sampled, ht.uniforms);
+    if (lane == 0) s_action = a;
   } else {
     pdl_entry();
-  }
-  if (threadIdx.x == 0) {
-    uint32_t tag = 0u, frame_step = 0u;
-    if (SAMPLE || actions != nullptr) {
-      const uint32_t step = (uint32_t)(*step_base) + t;       // global step index of this transition
-      const int32_t a = SAMPLE ? a_sampled : actions[e];
-      const uint32_t base = env_hash_base(seed, e, step, (uint32_t)a + 1u);
-      const uint32_t hr = hash_mix(base ^ HASH_TAG_REWARD) & 15u;
-      int r = hr == 0u ? 1 : (hr == 1u ? -1 : 0);
-      if (pattern_actions > 0)
-        r = (uint32_t)a == hash_mix(env_hash_base(seed, e, step, 0u) ^ HASH_TAG_GOAL) % (uint32_t)pattern_actions ? 1 : 0;
-      const uint32_t ht = hash_mix(base ^ HASH_TAG_TERMINAL);
-      const bool term = (uint32_t)(((uint64_t)ht * term_denom) >> 32) == 0u;
-      rewards[e] = (int8_t)r;
-      terminals[e] = term ? 1 : 0;
-      int32_t len = counters[e] + 1, ret = counters[n_e + e] + r;
-      if (term) { counters[2 * n_e + e] += 1; len = 0; ret = 0; }
-      counters[e] = len; counters[n_e + e] = ret;
-      tag = term ? 0u : (uint32_t)a + 1u;
-      frame_step = step + 1u;
+    if (threadIdx.x == 32) {
+      if (stepping) {
+        step = (uint32_t)(*step_base) + t;                      // global step index of this transition
+        pre_step = env_hash_prefix(seed, e, step);
+        pre_next = env_hash_prefix(seed, e, step + 1u);
+        len = counters[e]; ret = counters[n_e + e]; episodes = counters[2 * n_e + e];
+        if (!SAMPLE) s_action = actions[e];
+      } else {
+        pre_next = env_hash_prefix(seed, e, 0u);
+      }
     }
-    s_base = env_hash_base(seed, e, frame_step, tag);
+  }
+  __syncthreads();
+  bool term = false;
+  int r = 0;
+  if (threadIdx.x == 32) {
+    uint32_t tag = 0u;
+    if (stepping) {
+      const int32_t a = s_action;
+      const uint32_t base = hash_mix(pre_step ^ ((uint32_t)a + 1u));
+      const uint32_t hr = hash_mix(base ^ HASH_TAG_REWARD) & 15u;
+      r = hr == 0u ? 1 : (hr == 1u ? -1 : 0);
+      if (pattern_actions > 0)
+        r = (uint32_t)a == hash_mix(hash_mix(pre_step) ^ HASH_TAG_GOAL) % (uint32_t)pattern_actions ? 1 : 0;
+      const uint32_t hterm = hash_mix(base ^ HASH_TAG_TERMINAL);
+      term = (uint32_t)(((uint64_t)hterm * term_denom) >> 32) == 0u;
+      tag = term ? 0u : (uint32_t)a + 1u;
+    }
+    s_base = hash_mix(pre_next ^ tag);
     s_band_lo = s_band_hi = 0u;
     if (pattern_actions > 0) {
-      const uint32_t goal = hash_mix(env_hash_base(seed, e, frame_step, 0u) ^ HASH_TAG_GOAL) % (uint32_t)pattern_actions;
+      const uint32_t goal = hash_mix(hash_mix(pre_next) ^ HASH_TAG_GOAL) % (uint32_t)pattern_actions;
       const uint32_t band = (uint32_t)(FRAME_H / pattern_actions);
       s_band_lo = band * goal * FRAME_W;                  // in pixel words; a row is 84 words, so four words never straddle it
       s_band_hi = s_band_lo + band * FRAME_W;
     }
   }
   __syncthreads();
+  if (threadIdx.x == 32 && stepping) {
+    rewards[e] = (int8_t)r;
+    terminals[e] = term ? 1 : 0;
+    len += 1; ret += r;
+    if (term) { counters[2 * n_e + e] = episodes + 1; len = 0; ret = 0; }
+    counters[e] = len; counters[n_e + e] = ret;
+  }
   const uint32_t base = s_base, band_lo = s_band_lo, band_hi = s_band_hi;
   const uint32_t keep = pattern_actions > 0 ? 0x3F3F3F3Fu : 0xFFFFFFFFu;
   uint4* out = reinterpret_cast<uint4*>(next_frames + (size_t)e * FRAME_BYTES);
