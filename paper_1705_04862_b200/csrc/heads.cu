@@ -293,6 +293,10 @@ returns_head_grad_kernel(int algo, int n_e, int t_max, int A, float gamma, float
   __shared__ float sh[3][128], wsum[3][4];
   if (i < B) {
     float ret, ad;
+    // everything the row needs is asked for at once (the kernel is a chain of memory latencies otherwise)
+    const float z = lane < A ? logits[(size_t)i * A + lane] : -INFINITY;
+    const int a = actions[i];
+    const float v_i = values[i];
     {
       const int t = i / n_e, e = i - t * n_e;
       float next = values[(size_t)t_max * n_e + e];
@@ -314,17 +318,15 @@ returns_head_grad_kernel(int algo, int n_e, int t_max, int A, float gamma, float
         }
       }
       ret = next;
-      ad = __fsub_rn(next, values[i]);
+      ad = __fsub_rn(next, v_i);
       if (lane == 0) { R[i] = ret; adv[i] = ad; }
     }
-    const float z = lane < A ? logits[(size_t)i * A + lane] : -INFINITY;
     const float m = warp_max(z);
     const float ex = lane < A ? expf(z - m) : 0.f;
     const float lse = m + logf(warp_sum(ex));
     const float lp = z - lse;
     const float p = lane < A ? expf(lp) : 0.f;
     const float H = -warp_sum(lane < A ? p * lp : 0.f);
-    const int a = actions[i];
     const float invB = 1.0f / (float)B;
     if (algo == PAAC_ALGO_NSTEP_Q) {
       // value-based variant: L = value_coef (R - Q(s, a))^2, R constant; only the taken action's output has a gradient
@@ -343,7 +345,7 @@ returns_head_grad_kernel(int algo, int n_e, int t_max, int A, float gamma, float
       }
       const float lp_a = __shfl_sync(0xffffffffu, lp, a);
       if (lane == 0) {
-        const float d = values[i] - ret;
+        const float d = v_i - ret;
         dV[i] = 2.f * value_coef * d * invB;
         wsum[0][threadIdx.x >> 5] = -ad * lp_a;
         wsum[1][threadIdx.x >> 5] = value_coef * d * d;
