@@ -177,6 +177,22 @@ def preprocess(raw_prev, raw_last, state_in=None):
     return out
 
 
+def stack_push(state_in, newest, restart=None):
+    """Section 5.1 frame stack: state [n, 84, 84, 4] + newest frame [n, 84, 84] (+ restart flags [n]) -> state."""
+    state_in = np.ascontiguousarray(state_in, np.uint8)
+    newest = np.ascontiguousarray(newest, np.uint8)
+    n = state_in.shape[0]
+    assert state_in.shape == (n, 84, 84, 4) and newest.shape == (n, 84, 84)
+    out = np.zeros_like(state_in)
+    rs = None
+    if restart is not None:
+        restart = np.ascontiguousarray(restart, np.uint8)
+        assert restart.shape == (n,)
+        rs = _p(restart)
+    lib().orc_stack_push(_p(state_in), _p(newest), rs, _p(out), n)
+    return out
+
+
 def pattern_goal(seed, env, step, n_actions):
     lib().orc_pattern_goal.restype = C.c_uint32
     return int(lib().orc_pattern_goal(C.c_uint64(seed), C.c_uint32(env), C.c_uint32(step), n_actions))

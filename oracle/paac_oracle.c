@@ -24,6 +24,7 @@
  *   clip / RMSProp       closed forms
  *   pre-processing       block means of an integer-upsampled image (independent definition),
  *                        pure-colour and constant images, hand-computed rows, channel shift
+ *   frame stack          equals the pre-processing's own stacking, known planes in order, restart, brute force
  *   n-step Q variant     brute-force arg max and exploration branch, exploration frequency,
  *                        PyTorch autograd and central differences of the loss, hand case
  * The whole iteration has no printed value in the paper to compare with:
@@ -403,6 +404,27 @@ void orc_preprocess(const uint8_t* raw_prev, const uint8_t* raw_last, const uint
       }
   }
   free(grey);
+}
+
+/* The stacking half of the above by itself (Section 5.1: a state is the */
+/* stack of the four latest pre-processed frames): the newest frame      */
+/* [n][84][84] joins the previous state [n][84][84][4], oldest first;    */
+/* where restart[e] != 0 (nullable: no restarts) the environment has     */
+/* begun a new episode and the new frame fills all four channels.        */
+void orc_stack_push(const uint8_t* state_in, const uint8_t* newest, const uint8_t* restart /* nullable */,
+                    uint8_t* state_out, int n) {
+  enum { OH = 84, OW = 84 };
+  for (int e = 0; e < n; ++e)
+    for (int p = 0; p < OH * OW; ++p) {
+      size_t o = ((size_t)e * OH * OW + p) * 4;
+      uint8_t v = newest[(size_t)e * OH * OW + p];
+      if (restart && restart[e]) {
+        state_out[o] = state_out[o + 1] = state_out[o + 2] = state_out[o + 3] = v;
+      } else {
+        uint8_t c1 = state_in[o + 1], c2 = state_in[o + 2], c3 = state_in[o + 3];
+        state_out[o] = c1; state_out[o + 1] = c2; state_out[o + 2] = c3; state_out[o + 3] = v;
+      }
+    }
 }
 
 /* ------------------------------------------------------------------ */

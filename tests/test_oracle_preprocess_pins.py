@@ -68,3 +68,29 @@ def test_hand_computed_rows_and_columns(orc):
     full = 255 * 42 * 84                      # weight 42 x 84 (in 1/84 units) is half a row times a whole column
     assert out[0, 0] == (full * 19 // 21 + 16800) // 33600 and out[1, 0] == out[0, 0]
     assert out[0, 1] == (full * 2 // 21 + 16800) // 33600 and out[2:, :].sum() == 0 and out[:, 2:].sum() == 0
+
+
+def test_stack_push_is_the_stacking_half_of_the_preprocessing(orc):
+    """The frame stack by itself: it must give what the whole pre-processing gives when the newest frame is the
+    pre-processed one; four pushes of known planes leave them in order, oldest first; a restart fills the state."""
+    rng = np.random.RandomState(4)
+    a = rng.randint(0, 256, (3, 210, 160, 3), dtype=np.uint8)
+    b = rng.randint(0, 256, (3, 210, 160, 3), dtype=np.uint8)
+    prev = rng.randint(0, 256, (3, 84, 84, 4), dtype=np.uint8)
+    whole = orc.preprocess(a, b, prev)
+    assert np.array_equal(orc.stack_push(prev, whole[..., 3]), whole)
+    assert np.array_equal(orc.stack_push(prev, whole[..., 3], np.ones(3, np.uint8)), orc.preprocess(a, b, None))
+    # planes 1, 2, 3, 4 pushed one after the other into a state of zeros
+    st = np.zeros((2, 84, 84, 4), np.uint8)
+    for v in (1, 2, 3, 4):
+        st = orc.stack_push(st, np.full((2, 84, 84), v, np.uint8))
+    assert np.array_equal(st[0, 5, 7], [1, 2, 3, 4]) and np.all(st == np.array([1, 2, 3, 4], np.uint8))
+    # a restart in environment 1 only
+    st2 = orc.stack_push(st, np.full((2, 84, 84), 9, np.uint8), np.array([0, 1], np.uint8))
+    assert np.all(st2[0] == np.array([2, 3, 4, 9], np.uint8)) and np.all(st2[1] == 9)
+    # brute force on random data, pixel by pixel
+    planes = rng.randint(0, 256, (3, 84, 84), dtype=np.uint8)
+    out = orc.stack_push(prev, planes, np.array([0, 1, 0], np.uint8))
+    for e, y, x in ((0, 0, 0), (0, 83, 83), (1, 40, 2), (2, 17, 60)):
+        want = [planes[e, y, x]] * 4 if e == 1 else list(prev[e, y, x, 1:]) + [planes[e, y, x]]
+        assert list(out[e, y, x]) == want
