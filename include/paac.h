@@ -178,6 +178,16 @@ const char* paac_strerror(int status);
 int paac_act_host(paac_ctx* ctx, int t, const uint8_t* frames /* host */, int32_t* actions /* host, out */,
                   float* values /* host, out, nullable */);
 
+/* The same step with the state built on the device (Section 5.1: a state is the stack of the four latest
+ * pre-processed frames, so three quarters of s_t are already there as part of s_{t-1}): newest [n_e][84][84] uint8
+ * (host, pinned memory advised) is the frame that joins the stack; s_t = (the three newest channels of s_{t-1},
+ * newest), oldest first.  Where restart[e] != 0 (host, [n_e], nullable = no restarts) environment e has begun a new
+ * episode and the new frame fills all four channels.  t = 1 .. t_max (step 0 of a rollout has no new frame: it is the
+ * state of the call before, see paac_act_host); calls of the two kinds may be mixed within a rollout.  Copies a
+ * quarter of the bytes paac_act_host copies.  Errors as paac_act_host. */
+int paac_act_host_newest(paac_ctx* ctx, int t, const uint8_t* newest /* host */, const uint8_t* restart /* host, nullable */,
+                         int32_t* actions /* host, out */, float* values /* host, out, nullable */);
+
 /* Outcome of the actions of step t, observed on the host: rewards in {-1,0,1} and
  * terminal flags, [n_e] each.  After step t_max-1 and the bootstrap paac_act_host(t_max),
  * paac_update() may be called. */
@@ -198,6 +208,14 @@ int paac_observe_host(paac_ctx* ctx, int t, const int8_t* rewards /* host */, co
  *   the same bits on any machine. */
 int paac_preprocess(const uint8_t* raw_prev /* device */, const uint8_t* raw_last /* device */,
                     const uint8_t* state_in /* device, nullable */, uint8_t* state_out /* device */, int n, void* stream);
+
+/* The frame stack of Section 5.1 by itself, on device buffers: state_out = (the three newest channels of state_in,
+ * newest), or four copies of newest where restart[e] != 0 (nullable).  state_in / state_out [n][84][84][4] uint8
+ * (device, 16-byte aligned; the same buffer may be given for both), newest [n][84][84] uint8 (device, 4-byte
+ * aligned), restart [n] uint8 (device).  n = 1 .. 65,535.  Asynchronous on `stream` (a cudaStream_t, 0 = default).
+ * The paper states the stack, not a procedure. */
+int paac_stack_push(const uint8_t* state_in, const uint8_t* newest, const uint8_t* restart /* nullable */,
+                    uint8_t* state_out, int n, void* stream);
 
 /* ---- test and resume hooks ---- */
 

@@ -51,7 +51,7 @@ class UpdateStats(C.Structure):
 EXPORTS = ["paac_default_hparams", "paac_workspace_bytes", "paac_init", "paac_rollout", "paac_update",
            "paac_param_count", "paac_params", "paac_destroy", "paac_strerror", "paac_act_host",
            "paac_observe_host", "paac_set_params", "paac_force_actions", "paac_debug_bytes", "paac_debug_read",
-           "paac_debug_write", "paac_debug_wait_probe", "paac_preprocess", "paac_launch_count", "paac_profile", "paac_profile_read", "paac_set_option", "paac_clip_rmsprop_noalloc",
+           "paac_debug_write", "paac_debug_wait_probe", "paac_preprocess", "paac_stack_push", "paac_act_host_newest", "paac_launch_count", "paac_profile", "paac_profile_read", "paac_set_option", "paac_clip_rmsprop_noalloc",
            "paac_noalloc_max_params"]
 
 _lib = None
@@ -89,6 +89,8 @@ def lib():
         L.paac_debug_write.argtypes = [vp, i, vp, sz]
         L.paac_debug_wait_probe.argtypes = [vp, C.c_uint32]
         L.paac_preprocess.argtypes = [vp, vp, vp, vp, i, vp]
+        L.paac_stack_push.argtypes = [vp, vp, vp, vp, i, vp]
+        L.paac_act_host_newest.argtypes = [vp, i, vp, vp, vp, vp]
         L.paac_launch_count.argtypes = [vp]
         L.paac_launch_count.restype = u64
         L.paac_profile.argtypes = [vp, i]
@@ -153,6 +155,13 @@ def preprocess(raw_prev, raw_last, state_in, state_out, n, stream=None):
     return int(lib().paac_preprocess(addr(raw_prev), addr(raw_last), addr(state_in), addr(state_out), n, addr(stream)))
 
 
+def stack_push(state_in, newest, restart, state_out, n, stream=None):
+    """The four-frame stack on device buffers: see paac_stack_push in include/paac.h.  Returns the library status."""
+    def addr(x):
+        return None if x is None else (x if isinstance(x, int) else x.data_ptr())
+    return int(lib().paac_stack_push(addr(state_in), addr(newest), addr(restart), addr(state_out), n, addr(stream)))
+
+
 class Paac:
     """One learner.  The device workspace is a torch uint8 tensor on `device`; kernels run on
     torch's current stream at construction time."""
@@ -203,6 +212,11 @@ class Paac:
         _check(lib().paac_act_host(self._h, t, _host_ptr(frames) if frames is not None else None,
                                    _host_ptr(actions) if actions is not None else None,
                                    _host_ptr(values) if values is not None else None))
+
+    def act_host_newest(self, t, newest, restart=None, actions=None, values=None):
+        _check(lib().paac_act_host_newest(self._h, t, _host_ptr(newest), _host_ptr(restart) if restart is not None else None,
+                                          _host_ptr(actions) if actions is not None else None,
+                                          _host_ptr(values) if values is not None else None))
 
     def observe_host(self, t, rewards, terminals):
         _check(lib().paac_observe_host(self._h, t, _host_ptr(rewards), _host_ptr(terminals)))

@@ -21,6 +21,7 @@ struct paac_ctx {
   uint64_t N;              // timesteps consumed by updates
   uint64_t env_step;       // global step index of the environments (same for all)
   bool rollout_fresh;      // a rollout has completed since the last update
+  uint8_t* newest;         // staging for paac_act_host_newest: [n_e][84][84] planes, then [n_e] restart flags
   int host_t;              // external-environment mode: next expected step
   int update_chunks;       // > 1: conv2 data gradient and conv1 weight gradient alternate over this many groups of states
   bool host_next_valid;    // the bootstrap state of the last host-mode rollout sits where step 0 of the next one goes
@@ -93,6 +94,7 @@ size_t carve(paac_ctx* c, char* base) {
   c->w_images = k.take<bf16>(tc_supported(c->arch, c->prec) ? tc_weight_image_elems() : 0);
   c->frames[0] = k.take<uint8_t>(T * n_e * FRAME_BYTES);
   c->frames[1] = k.take<uint8_t>(T * n_e * FRAME_BYTES);
+  c->newest = k.take<uint8_t>(n_e * (FRAME_H * FRAME_W + 4));          // newest planes from the host, then restart flags
   for (int l = 0; l <= nd.n_conv; ++l) {
     c->act[l] = k.take<char>((T + 1) * n_e * nd.layer[l].out_size * c->elt);
     c->gact[l] = k.take<char>(B * nd.layer[l].out_size * c->elt);
@@ -532,18 +534,8 @@ int paac_profile_read(paac_ctx* c, int max_entries, const char** names, double* 
 }
 
 // ---- external-environment mode ------------------------------------------------------------------
-int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, float* values) {
-  if (c) c->lc.serialize_next = true;
-  if (!c || t < 0 || t > c->t_max || (t < c->t_max && !actions)) return PAAC_ERR_ARG;
-  if (t != c->host_t) return PAAC_ERR_STATE;
-  // s_0 of a rollout is s_{t_max} of the one before (Algorithm 1): those frames are on the device already
-  if (!frames && !(t == 0 && c->host_next_valid)) return PAAC_ERR_ARG;
-  const size_t fstep = (size_t)c->n_e * FRAME_BYTES;
-  if (t == 0) c->cur ^= 1;
-  uint8_t* dst = t < c->t_max ? c->frames[c->cur] + t * fstep : c->frames[c->cur ^ 1];
-  if (frames && cudaMemcpyAsync(dst, frames, fstep, cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
-    cudaGetLastError(); return PAAC_ERR_CUDA;
-  }
+// the network on the state at `dst`, results to the host, bookkeeping of the external-environment rollout
+static int act_host_finish(paac_ctx* c, int t, uint8_t* dst, int32_t* actions, float* values) {
   const bool sample = t < c->t_max;
   forward_slot(c, dst, t, sample);
   const size_t row = (size_t)t * c->n_e;
@@ -556,6 +548,37 @@ int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, f
   }
   else c->host_t = t + 1;
   return cuda_status(c);
+}
+
+int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, float* values) {
+  if (c) c->lc.serialize_next = true;
+  if (!c || t < 0 || t > c->t_max || (t < c->t_max && !actions)) return PAAC_ERR_ARG;
+  if (t != c->host_t) return PAAC_ERR_STATE;
+  // s_0 of a rollout is s_{t_max} of the one before (Algorithm 1): those frames are on the device already
+  if (!frames && !(t == 0 && c->host_next_valid)) return PAAC_ERR_ARG;
+  const size_t fstep = (size_t)c->n_e * FRAME_BYTES;
+  if (t == 0) c->cur ^= 1;
+  uint8_t* dst = t < c->t_max ? c->frames[c->cur] + t * fstep : c->frames[c->cur ^ 1];
+  if (frames && cudaMemcpyAsync(dst, frames, fstep, cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
+    cudaGetLastError(); return PAAC_ERR_CUDA;
+  }
+  return act_host_finish(c, t, dst, actions, values);
+}
+
+int paac_act_host_newest(paac_ctx* c, int t, const uint8_t* newest, const uint8_t* restart, int32_t* actions, float* values) {
+  if (c) c->lc.serialize_next = true;
+  if (!c || !newest || t < 1 || t > c->t_max || (t < c->t_max && !actions)) return PAAC_ERR_ARG;
+  if (t != c->host_t) return PAAC_ERR_STATE;
+  const size_t fstep = (size_t)c->n_e * FRAME_BYTES, plane = (size_t)c->n_e * FRAME_H * FRAME_W;
+  const uint8_t* prev = c->frames[c->cur] + (size_t)(t - 1) * fstep;
+  uint8_t* dst = t < c->t_max ? c->frames[c->cur] + t * fstep : c->frames[c->cur ^ 1];
+  uint8_t* flags = restart ? c->newest + plane : nullptr;
+  if (cudaMemcpyAsync(c->newest, newest, plane, cudaMemcpyHostToDevice, c->st) != cudaSuccess ||
+      (restart && cudaMemcpyAsync(flags, restart, c->n_e, cudaMemcpyHostToDevice, c->st) != cudaSuccess)) {
+    cudaGetLastError(); return PAAC_ERR_CUDA;
+  }
+  launch_stack_push(c->lc, prev, c->newest, flags, dst, c->n_e);
+  return act_host_finish(c, t, dst, actions, values);
 }
 
 int paac_observe_host(paac_ctx* c, int t, const int8_t* rewards, const uint8_t* terminals) {

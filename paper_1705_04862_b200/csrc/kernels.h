@@ -71,6 +71,9 @@ float tc_conv1_grad_scale();
 struct GradSegment { const float* part; float* dst; int splits, J, CO; float scale; int first_group, groups, wide; };
 struct GradSegments { GradSegment seg[12]; int n; int total_groups; };
 size_t tc_scratch_floats(int n);
+// frame stack: out = (three newest channels of prev, newest plane), or four copies of the plane where restart[e] != 0
+void launch_stack_push(LaunchCtx& lc, const uint8_t* prev, const uint8_t* newest, const uint8_t* restart /* nullable */,
+                       uint8_t* out, int n);
 // the same data gradient followed by the first layer's weight gradient, alternating over `chunks` (at most
 // TC_MAX_UPDATE_CHUNKS) groups of states; notes the weight gradient's partial sums in *segs
 constexpr int TC_MAX_UPDATE_CHUNKS = 4;

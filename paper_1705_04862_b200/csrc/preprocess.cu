@@ -1,6 +1,7 @@
 // Frame pre-processing (Section 5.1 of the paper): per-pixel maximum of the two latest raw frames, pixel intensity,
 // 210 x 160 -> 84 x 84, newest channel of the four-frame state.  Integer arithmetic throughout.
 #include "common.cuh"
+#include "kernels.h"
 
 namespace paac {
 
@@ -68,7 +69,50 @@ preprocess_kernel(const uint8_t* __restrict__ raw_prev, const uint8_t* __restric
   }
 }
 
+// The frame stack by itself: out = (the three newest channels of prev, newest), or four copies of newest where the
+// environment restarts.  A thread takes four pixels: one 16-byte load of the previous state, one 4-byte load of the
+// new plane, one 16-byte store.  prev == out is allowed (every word is read before it is written, by the same thread).
+constexpr int SP_THREADS = 256, SP_QUADS = FRAME_H * FRAME_W / 4;          // 1764 groups of four pixels per state
+__global__ void __launch_bounds__(SP_THREADS)
+stack_push_kernel(const uint8_t* prev, const uint8_t* __restrict__ newest, const uint8_t* __restrict__ restart,
+                  uint8_t* out) {
+  pdl_entry();
+  const uint32_t e = blockIdx.y;
+  const bool fresh = restart != nullptr && restart[e] != 0;
+  const uint4* src = reinterpret_cast<const uint4*>(prev + (size_t)e * FRAME_BYTES);
+  const uint32_t* nw = reinterpret_cast<const uint32_t*>(newest + (size_t)e * FRAME_H * FRAME_W);
+  uint4* dst = reinterpret_cast<uint4*>(out + (size_t)e * FRAME_BYTES);
+  for (int q = blockIdx.x * SP_THREADS + threadIdx.x; q < SP_QUADS; q += gridDim.x * SP_THREADS) {
+    const uint32_t v = nw[q];
+    uint4 w;
+    if (fresh) {
+      w = make_uint4((v & 0xFFu) * 0x01010101u, ((v >> 8) & 0xFFu) * 0x01010101u, ((v >> 16) & 0xFFu) * 0x01010101u,
+                     (v >> 24) * 0x01010101u);
+    } else {
+      const uint4 p = src[q];
+      w = make_uint4((p.x >> 8) | (v << 24), (p.y >> 8) | ((v >> 8) << 24), (p.z >> 8) | ((v >> 16) << 24),
+                     (p.w >> 8) | ((v >> 24) << 24));
+    }
+    dst[q] = w;
+  }
+}
+
+void launch_stack_push(LaunchCtx& lc, const uint8_t* prev, const uint8_t* newest, const uint8_t* restart, uint8_t* out, int n) {
+  KernelScope scope(lc, KID_ENV_STEP);
+  launch_kernel(lc, stack_push_kernel, dim3(2, n), SP_THREADS, 0, prev, newest, restart, out);
+}
+
 }  // namespace paac
+
+extern "C" int paac_stack_push(const uint8_t* state_in, const uint8_t* newest, const uint8_t* restart, uint8_t* state_out,
+                               int n, void* stream) {
+  using namespace paac;
+  if (!state_in || !newest || !state_out || n < 1 || n > 65535) return PAAC_ERR_ARG;
+  if (((uintptr_t)state_in | (uintptr_t)state_out) & 15u) return PAAC_ERR_ARG;
+  if ((uintptr_t)newest & 3u) return PAAC_ERR_ARG;
+  stack_push_kernel<<<dim3(2, n), SP_THREADS, 0, (cudaStream_t)stream>>>(state_in, newest, restart, state_out);
+  return cudaGetLastError() == cudaSuccess ? PAAC_OK : PAAC_ERR_CUDA;
+}
 
 extern "C" int paac_preprocess(const uint8_t* raw_prev, const uint8_t* raw_last, const uint8_t* state_in,
                                uint8_t* state_out, int n, void* stream) {

@@ -351,6 +351,47 @@ def test_external_environment_mode_matches_device_environment(orc):
     g2.close()
 
 
+def test_external_environment_mode_with_newest_frames(orc):
+    """paac_act_host_newest: the host sends only the frame that joins the four-frame stack (and restart flags); the
+    states built on the device are the oracle's stack of the same planes, and the iteration (actions, values,
+    update) is the one a context gets that is sent those whole states."""
+    cfg = CONFIGS[0]
+    n_e, T = cfg["n_e"], cfg["t_max"]
+    _, g = make_pair(orc, cfg)
+    _, g2 = make_pair(orc, cfg)
+    rng = np.random.RandomState(5)
+    state = rng.randint(0, 256, (n_e, 84, 84, 4), dtype=np.uint8)
+    a, a2 = np.zeros(n_e, np.int32), np.zeros(n_e, np.int32)
+    v, v2 = np.zeros(n_e, np.float32), np.zeros(n_e, np.float32)
+    with pytest.raises(pb.PaacError):
+        g.act_host_newest(0, state[..., 3].copy(), None, a, v)             # step 0 has no new frame
+    for it in range(2):
+        for t in range(T + 1):
+            if t == 0:
+                g.act_host(0, state if it == 0 else None, a, v)               # whole state once, then the one on the device
+                g2.act_host(0, state, a2, v2)
+            else:
+                plane = rng.randint(0, 256, (n_e, 84, 84), dtype=np.uint8)
+                restart = (rng.randint(0, 3, n_e) == 0).astype(np.uint8) if t % 2 else None
+                state = orc.stack_push(state, plane, restart)
+                g.act_host_newest(t, plane, restart, a if t < T else None, v)
+                g2.act_host(t, state, a2 if t < T else None, v2)
+            assert np.array_equal(v, v2)
+            if t < T:
+                assert np.array_equal(a, a2)
+                r = rng.randint(-1, 2, n_e).astype(np.int8)
+                term = (rng.randint(0, 5, n_e) == 0).astype(np.uint8)
+                g.observe_host(t, r, term)
+                g2.observe_host(t, r, term)
+        assert np.array_equal(g.debug_read(pb.DBG_FRAMES), g2.debug_read(pb.DBG_FRAMES))
+        assert np.array_equal(g.debug_read(pb.DBG_NEXT_FRAMES).reshape(n_e, 84, 84, 4), state)
+        g.update()
+        g2.update()
+        assert np.array_equal(g.params(), g2.params())
+    g.close()
+    g2.close()
+
+
 def test_bounded_wait_gives_up_and_the_update_is_skipped(orc):
     """A wait on a barrier nobody signals runs out after its poll limit: the kernel returns, the error word is set,
     the call reports ERR_TIMEOUT, and the context stays usable.  While the word is set an update changes neither

@@ -56,3 +56,30 @@ def test_bad_arguments():
     assert L.paac_preprocess(None, x.data_ptr(), None, x.data_ptr(), 1, None) == pb.ERR_ARG
     assert L.paac_preprocess(x.data_ptr(), x.data_ptr(), None, x.data_ptr(), 0, None) == pb.ERR_ARG
     assert L.paac_preprocess(x.data_ptr() + 1, x.data_ptr(), None, x.data_ptr(), 1, None) == pb.ERR_ARG
+
+
+def test_frame_stack_against_the_oracle(orc):
+    """paac_stack_push: the newest plane joins the state (or fills it where an episode restarts), bit for bit, for a
+    single environment, a ragged batch, 1024 environments, and in place."""
+    import torch
+    rng = np.random.RandomState(11)
+    for n in (1, 37, 1024):
+        prev = rng.randint(0, 256, (n, 84, 84, 4), dtype=np.uint8)
+        plane = rng.randint(0, 256, (n, 84, 84), dtype=np.uint8)
+        restart = (rng.randint(0, 4, n) == 0).astype(np.uint8)
+        for flags in (None, restart):
+            sin, pl = torch.from_numpy(prev).cuda(), torch.from_numpy(plane).cuda()
+            fl = torch.from_numpy(flags).cuda() if flags is not None else None
+            out = torch.zeros_like(sin)
+            assert pb.stack_push(sin, pl, fl, out, n, torch.cuda.current_stream().cuda_stream) == pb.OK
+            torch.cuda.synchronize()
+            want = orc.stack_push(prev, plane, flags)
+            assert np.array_equal(out.cpu().numpy(), want)
+            assert pb.stack_push(sin, pl, fl, sin, n, torch.cuda.current_stream().cuda_stream) == pb.OK      # in place
+            torch.cuda.synchronize()
+            assert np.array_equal(sin.cpu().numpy(), want)
+    x = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    L = pb.lib()
+    assert L.paac_stack_push(None, x.data_ptr(), None, x.data_ptr(), 1, None) == pb.ERR_ARG
+    assert L.paac_stack_push(x.data_ptr(), x.data_ptr(), None, x.data_ptr(), 0, None) == pb.ERR_ARG
+    assert L.paac_stack_push(x.data_ptr() + 4, x.data_ptr(), None, x.data_ptr(), 1, None) == pb.ERR_ARG
