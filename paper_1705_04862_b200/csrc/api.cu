@@ -33,9 +33,12 @@ struct paac_ctx {
   // second iteration (the two frame buffers alternate), so after two plain iterations each parity is captured
   // once into a CUDA graph and replayed from then on.  Anything that changes the sequence drops the graphs.
   bool graphs_on;          // option: allow recording
-  int plain_calls[2][2];   // [rollout / update][parity]: calls made with plain launches
-  cudaGraphExec_t graph[2][2];
-  uint64_t graph_launches[2][2];
+  // recorded launch sequences: kind 0 = rollout, 1 = update, 2 + 2 t + v = step t of the external-environment mode
+  // (v = 1: with the frame stack built on the device), each for both parities of the frame buffers
+  static constexpr int GRAPH_KINDS = 2 + 2 * 65;
+  int plain_calls[GRAPH_KINDS][2];   // calls made with plain launches
+  cudaGraphExec_t graph[GRAPH_KINDS][2];
+  uint64_t graph_launches[GRAPH_KINDS][2];
   bool simt_only;          // keep the bf16 network on the CUDA cores (cross-check of the tensor-core path)
 
   // device buffers (all inside the workspace)
@@ -193,7 +196,7 @@ bool forward_slot(paac_ctx* c, const uint8_t* frames, int slot, bool sample, Hea
 }
 
 void drop_graphs(paac_ctx* c) {
-  for (int k = 0; k < 2; ++k)
+  for (int k = 0; k < paac_ctx::GRAPH_KINDS; ++k)
     for (int par = 0; par < 2; ++par) {
       if (c->graph[k][par]) { cudaGraphExecDestroy(c->graph[k][par]); c->graph[k][par] = nullptr; }
       c->plain_calls[k][par] = 0;
@@ -534,10 +537,15 @@ int paac_profile_read(paac_ctx* c, int max_entries, const char** names, double* 
 }
 
 // ---- external-environment mode ------------------------------------------------------------------
-// the network on the state at `dst`, results to the host, bookkeeping of the external-environment rollout
-static int act_host_finish(paac_ctx* c, int t, uint8_t* dst, int32_t* actions, float* values) {
+// Step t of an external-environment rollout once the host's bytes are on their way: (the frame stack,) the network on
+// the state at `dst` -- a recorded sequence from the second time on --, results to the host, bookkeeping.
+static int act_host_finish(paac_ctx* c, int t, const uint8_t* prev, uint8_t* dst, int32_t* actions, float* values) {
   const bool sample = t < c->t_max;
-  forward_slot(c, dst, t, sample);
+  const size_t plane = (size_t)c->n_e * FRAME_H * FRAME_W;
+  run_recorded(c, 2 + 2 * t + (prev ? 1 : 0), c->cur, [&]() {
+    if (prev) launch_stack_push(c->lc, prev, c->newest, c->newest + plane, dst, c->n_e);
+    forward_slot(c, dst, t, sample);
+  });
   const size_t row = (size_t)t * c->n_e;
   if (sample) cudaMemcpyAsync(actions, c->actions + row, c->n_e * sizeof(int32_t), cudaMemcpyDeviceToHost, c->st);
   if (values) cudaMemcpyAsync(values, c->values + row, c->n_e * sizeof(float), cudaMemcpyDeviceToHost, c->st);
@@ -562,7 +570,7 @@ int paac_act_host(paac_ctx* c, int t, const uint8_t* frames, int32_t* actions, f
   if (frames && cudaMemcpyAsync(dst, frames, fstep, cudaMemcpyHostToDevice, c->st) != cudaSuccess) {
     cudaGetLastError(); return PAAC_ERR_CUDA;
   }
-  return act_host_finish(c, t, dst, actions, values);
+  return act_host_finish(c, t, nullptr, dst, actions, values);
 }
 
 int paac_act_host_newest(paac_ctx* c, int t, const uint8_t* newest, const uint8_t* restart, int32_t* actions, float* values) {
@@ -572,13 +580,13 @@ int paac_act_host_newest(paac_ctx* c, int t, const uint8_t* newest, const uint8_
   const size_t fstep = (size_t)c->n_e * FRAME_BYTES, plane = (size_t)c->n_e * FRAME_H * FRAME_W;
   const uint8_t* prev = c->frames[c->cur] + (size_t)(t - 1) * fstep;
   uint8_t* dst = t < c->t_max ? c->frames[c->cur] + t * fstep : c->frames[c->cur ^ 1];
-  uint8_t* flags = restart ? c->newest + plane : nullptr;
-  if (cudaMemcpyAsync(c->newest, newest, plane, cudaMemcpyHostToDevice, c->st) != cudaSuccess ||
-      (restart && cudaMemcpyAsync(flags, restart, c->n_e, cudaMemcpyHostToDevice, c->st) != cudaSuccess)) {
-    cudaGetLastError(); return PAAC_ERR_CUDA;
-  }
-  launch_stack_push(c->lc, prev, c->newest, flags, dst, c->n_e);
-  return act_host_finish(c, t, dst, actions, values);
+  // the restart flags always live on the device (all zero when the host has none), so that the recorded sequence
+  // is the same either way
+  const cudaError_t e1 = cudaMemcpyAsync(c->newest, newest, plane, cudaMemcpyHostToDevice, c->st);
+  const cudaError_t e2 = restart ? cudaMemcpyAsync(c->newest + plane, restart, c->n_e, cudaMemcpyHostToDevice, c->st)
+                                 : cudaMemsetAsync(c->newest + plane, 0, c->n_e, c->st);
+  if (e1 != cudaSuccess || e2 != cudaSuccess) { cudaGetLastError(); return PAAC_ERR_CUDA; }
+  return act_host_finish(c, t, prev, dst, actions, values);
 }
 
 int paac_observe_host(paac_ctx* c, int t, const int8_t* rewards, const uint8_t* terminals) {
