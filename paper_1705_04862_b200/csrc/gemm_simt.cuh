@@ -11,29 +11,30 @@ namespace paac {
 
 constexpr int SG_BM = 64, SG_BN = 64, SG_BK = 16, SG_THREADS = 256;
 
-// BM = rows of the output tile: 64, or 32 / 16 for contractions with at most that many rows (the weight gradients of
-// layers with 16 or 32 output channels, a batch of four states), where most of a 64-row tile's multiply-adds would be
+// BM x BN = the output tile: 64 x 64, or 32 / 16 rows for contractions with at most that many rows (the weight
+// gradients of layers with 16 or 32 output channels, a batch of four states), or 32 / 16 columns for contractions with
+// at most that many columns (the forward pass of those layers), where most of a 64 x 64 tile's multiply-adds would be
 // padding.
-template <int BM, class LA, class LB, class EP>
+template <int BM, int BN, class LA, class LB, class EP>
 __global__ void __launch_bounds__(SG_THREADS)
 gemm_simt_kernel(int M, int N, int K, int k_per_split, LA la, LB lb, EP ep) {
   pdl_entry();
-  constexpr int RM = BM / 16;                    // rows per thread
+  constexpr int RM = BM / 16, CN = BN / 16;      // rows and columns per thread
   __shared__ float As[SG_BK][BM + 4];
-  __shared__ float Bs[SG_BK][SG_BN + 4];
+  __shared__ float Bs[SG_BK][BN + 4];
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * SG_BN, split = blockIdx.z;
+  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN, split = blockIdx.z;
   const int k_begin = split * k_per_split;
   const int k_end = min(K, k_begin + k_per_split);
-  float acc[RM][4];
+  float acc[RM][CN];
 #pragma unroll
   for (int i = 0; i < RM; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int j = 0; j < CN; ++j) acc[i][j] = 0.f;
 
   // operand values of one k block, fetched into registers one block ahead of the multiply-adds that use them, so that
   // the loads' latency overlaps the arithmetic of the block before (the order of the additions does not change)
-  constexpr int NA = BM * SG_BK / SG_THREADS, NB = SG_BN * SG_BK / SG_THREADS;
+  constexpr int NA = BM * SG_BK / SG_THREADS, NB = BN * SG_BK / SG_THREADS;
   float ra[NA], rb[NB];
   auto fetch = [&](int k0) {
 #pragma unroll
@@ -48,7 +49,7 @@ gemm_simt_kernel(int M, int N, int K, int k_per_split, LA la, LB lb, EP ep) {
     for (int i = 0; i < NB; ++i) {
       const int idx = tid + i * SG_THREADS;
       int kk, nn;
-      if (LB::K_CONTIG) { kk = idx % SG_BK; nn = idx / SG_BK; } else { nn = idx % SG_BN; kk = idx / SG_BN; }
+      if (LB::K_CONTIG) { kk = idx % SG_BK; nn = idx / SG_BK; } else { nn = idx % BN; kk = idx / BN; }
       const int n = n0 + nn, k = k0 + kk;
       rb[i] = (n < N && k < k_end) ? lb(n, k) : 0.f;
     }
@@ -63,29 +64,29 @@ gemm_simt_kernel(int M, int N, int K, int k_per_split, LA la, LB lb, EP ep) {
 #pragma unroll
     for (int i = 0; i < NB; ++i) {
       const int idx = tid + i * SG_THREADS;
-      if (LB::K_CONTIG) Bs[idx % SG_BK][idx / SG_BK] = rb[i]; else Bs[idx / SG_BN][idx % SG_BN] = rb[i];
+      if (LB::K_CONTIG) Bs[idx % SG_BK][idx / SG_BK] = rb[i]; else Bs[idx / BN][idx % BN] = rb[i];
     }
     __syncthreads();
     if (k0 + SG_BK < k_end) fetch(k0 + SG_BK);
 #pragma unroll
     for (int kk = 0; kk < SG_BK; ++kk) {
-      float a[RM], b[4];
+      float a[RM], b[CN];
 #pragma unroll
       for (int i = 0; i < RM; ++i) a[i] = As[kk][ty * RM + i];
 #pragma unroll
-      for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+      for (int j = 0; j < CN; ++j) b[j] = Bs[kk][tx * CN + j];
 #pragma unroll
       for (int i = 0; i < RM; ++i)
 #pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        for (int j = 0; j < CN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
     }
     __syncthreads();
   }
 #pragma unroll
   for (int i = 0; i < RM; ++i)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int m = m0 + ty * RM + i, n = n0 + tx * 4 + j;
+    for (int j = 0; j < CN; ++j) {
+      const int m = m0 + ty * RM + i, n = n0 + tx * CN + j;
       if (m < M && n < N) ep(m, n, acc[i][j], split);
     }
 }
@@ -98,12 +99,18 @@ inline void gemm_simt(LaunchCtx& lc, int kid, int M, int N, int K, int splits, L
   kps = (kps + SG_BK - 1) / SG_BK * SG_BK;
   if (M <= 32) {
     dim3 grid(1, (N + SG_BN - 1) / SG_BN, (K + kps - 1) / kps);
-    if (M <= 16) launch_kernel(lc, gemm_simt_kernel<16, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
-    else launch_kernel(lc, gemm_simt_kernel<32, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
+    if (M <= 16) launch_kernel(lc, gemm_simt_kernel<16, SG_BN, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
+    else launch_kernel(lc, gemm_simt_kernel<32, SG_BN, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
+    return;
+  }
+  if (N <= 32) {
+    dim3 grid((M + SG_BM - 1) / SG_BM, 1, (K + kps - 1) / kps);
+    if (N <= 16) launch_kernel(lc, gemm_simt_kernel<SG_BM, 16, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
+    else launch_kernel(lc, gemm_simt_kernel<SG_BM, 32, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
     return;
   }
   dim3 grid((M + SG_BM - 1) / SG_BM, (N + SG_BN - 1) / SG_BN, (K + kps - 1) / kps);
-  launch_kernel(lc, gemm_simt_kernel<SG_BM, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
+  launch_kernel(lc, gemm_simt_kernel<SG_BM, SG_BN, LA, LB, EP>, grid, SG_THREADS, 0, M, N, K, kps, la, lb, ep);
 }
 // number of k-splits gemm_simt will really launch for a requested count
 inline int gemm_simt_splits(int K, int splits) {
