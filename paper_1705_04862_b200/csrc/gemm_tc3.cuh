@@ -1,8 +1,8 @@
 // The same generic contraction as gemm_simt.cuh on the tensor cores, accurate to float level:
 //   C(m, n) = sum_k A(m, k) * B(n, k)
 // with every float operand split into two TF32 pieces, x = hi + lo (hi = tf32(x), lo = tf32(x - hi), round to nearest,
-// together 22 significant bits), and three tcgen05 passes (kind::tf32) accumulated in one float accumulator in tensor
-// memory:
+// together 22 significant bits), and three tcgen05 passes (kind::tf32) per block of 32 k into a float accumulator in
+// tensor memory, the blocks' sums then added in registers:
 //   hi*hi + hi*lo + lo*hi      (the dropped lo*lo term and the rounding of lo are below 2^-21 of a product).
 // Two bfloat16 pieces (16 bits) are not enough here: errors of 1e-5 flip about one ReLU unit per update of the small
 // network and the free-running trajectories leave the float tolerance within three updates.
@@ -19,8 +19,8 @@
 // Only the twelve steps of one block are summed inside the tensor core, whose accumulation does not round to nearest;
 // summed there over a whole contraction (thousands of steps) the result was eight times further from the exact
 // one than the CUDA-core kernel's.
-// Every wait is bounded.  The tiles of the float configurations are small (4 to 160 rows), so most of a 128-row tile
-// is padding there: this path exists for its arithmetic, not for speed.
+// Every wait is bounded.  The contractions of the float configurations are small (4 to 160 rows in the fully connected
+// layers), so most of a 128-row tile is padding there: this path exists for its arithmetic, not for speed.
 #pragma once
 #include "gemm_simt.cuh"
 #include "tc_common.cuh"
