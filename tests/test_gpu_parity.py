@@ -492,6 +492,36 @@ def test_shape_sweep_two_implementations_agree():
         assert d <= 5e-2, (n_e, T, A, d)
 
 
+def test_shape_sweep_float_path_two_implementations_agree():
+    """Thirty ragged shapes through the float path, both networks, with the value-based variant and the learnable
+    environment mixed in: the CUDA-core contraction (whose tile shape follows the row and column counts) and the
+    three-pass tensor-core contraction finish without a device error and agree on the gradient (L2; single ReLU
+    flips between two float implementations show up at the 1e-3 level on large batches)."""
+    import random
+    rnd = random.Random(7)
+    combos = [(arch, n, t, a) for arch in ("nips", "nature") for n in (1, 2, 3, 5, 16, 37, 64, 100, 129, 255)
+              for t in (1, 2, 5, 7) for a in (2, 3, 5, 18, 19, 32)]
+    rnd.shuffle(combos)
+    for i, (arch, n_e, T, A) in enumerate(combos[:30]):
+        outs = []
+        for mode in (0, 1):
+            g = pb.Paac(arch, n_e, T, A, seed=5, precision=pb.FP32, lr=0.01, term_denom=50,
+                        algorithm=pb.ALGO_NSTEP_Q if i % 3 == 0 else pb.ALGO_A2C,
+                        environment=pb.ENV_PATTERN if i % 4 == 0 else pb.ENV_HASHED)
+            g.set_option(pb.OPT_FP32_TENSOR_CORES, mode)
+            if outs:
+                g.force_actions(outs[0][0])
+            g.rollout()
+            acts = g.debug_read(pb.DBG_ACTIONS).copy()
+            g.update()
+            grad = g.debug_read(pb.DBG_GRAD).copy()
+            assert g.error_word() == 0 and np.isfinite(grad).all(), (arch, n_e, T, A)
+            outs.append((acts, grad))
+            g.close()
+        d = np.linalg.norm(outs[0][1].astype(np.float64) - outs[1][1]) / max(np.linalg.norm(outs[1][1]), 1e-30)
+        assert d <= 2e-2, (arch, n_e, T, A, d)
+
+
 def test_odd_action_counts_on_the_tensor_core_path(orc):
     """Action counts and batch sizes whose product is odd: the heads' partial sums (policy rows, policy biases, value
     row, value bias, one behind the other per split) then start at odd float offsets unless padded; the value row is
