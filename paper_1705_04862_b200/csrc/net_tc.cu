@@ -1545,19 +1545,6 @@ tc_fc_cluster_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     fence_barrier_init();
   }
   if (warp == 8) tmem_alloc(&sh.tmem_base, FCC_BN);
-  // head weights of this column tile: row k = policy row k (k < A, 16-byte aligned) or the value row (k = A, which
-  // follows the policy biases in the parameter vector and is only 2-byte aligned), 256 bf16 each
-  for (int i = threadIdx.x; i < A * (FCC_BN / 8); i += FCC_THREADS) {
-    const int k = i / (FCC_BN / 8), c = i % (FCC_BN / 8);
-    const uint4 v = __ldg(reinterpret_cast<const uint4*>(wpi + (size_t)k * N + nt * FCC_BN) + c);
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(headw + (uint32_t)(k * FCC_BN + 8 * c) * 2u),
-                 "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-  }
-  for (int c = threadIdx.x; c < FCC_BN / 2; c += FCC_THREADS) {
-    const bf16* src = wv + nt * FCC_BN + 2 * c;
-    const uint32_t v = (uint32_t)__bfloat16_as_ushort(src[0]) | ((uint32_t)__bfloat16_as_ushort(src[1]) << 16);
-    asm volatile("st.shared.b32 [%0], %1;" ::"r"(headw + (uint32_t)(A * FCC_BN + 2 * c) * 2u), "r"(v) : "memory");
-  }
   tcgen05_fence_before();
   __syncthreads();
   tcgen05_fence_after();
@@ -1599,6 +1586,21 @@ tc_fc_cluster_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       if (ok) mma_commit(&sh.acc_full);
     }
   } else {
+    // While the K slice is being multiplied these four warps have nothing to wait for yet: they bring in the head
+    // weights of this column tile (row k = policy row k, k < A, 16-byte aligned, or the value row, k = A, which follows
+    // the policy biases in the parameter vector and is only 2-byte aligned; 256 bf16 each).  The weights are several
+    // kernels old; the block-wide barrier after the accumulator is parked makes them visible to the finishing phase.
+    for (int i = threadIdx.x; i < A * (FCC_BN / 8); i += 128) {
+      const int k = i / (FCC_BN / 8), c = i % (FCC_BN / 8);
+      const uint4 v = __ldg(reinterpret_cast<const uint4*>(wpi + (size_t)k * N + nt * FCC_BN) + c);
+      asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(headw + (uint32_t)(k * FCC_BN + 8 * c) * 2u),
+                   "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+    }
+    for (int c = threadIdx.x; c < FCC_BN / 2; c += 128) {
+      const bf16* src = wv + nt * FCC_BN + 2 * c;
+      const uint32_t v = (uint32_t)__bfloat16_as_ushort(src[0]) | ((uint32_t)__bfloat16_as_ushort(src[1]) << 16);
+      asm volatile("st.shared.b32 [%0], %1;" ::"r"(headw + (uint32_t)(A * FCC_BN + 2 * c) * 2u), "r"(v) : "memory");
+    }
     // ---------------- accumulator -> this CTA's shared memory (float, 16-byte chunks swizzled by row) ----------------
     const bool ok = mbar_wait(&sh.acc_full, 0, &sh.abort, error_word, ERR_WAIT_ACC);
     if (__all_sync(0xffffffffu, ok)) {
@@ -1652,16 +1654,31 @@ tc_fc_cluster_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
     for (int i = 0; i < 16; ++i) v[i] = 0.f;
     if (m < M) {
       const float4* src = reinterpret_cast<const float4*>(part + (size_t)m * N + nt * FCC_BN) + cg;
+      // the first six slices are asked for in one go (24 loads in flight per thread: the phase is a chain of L2
+      // latencies otherwise), a seventh and eighth, if any, after them; the additions keep the slice order
+      {
+        float4 t[6][4];
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        float4 t[4][4];
-#pragma unroll
-        for (int s = 0; s < 4; ++s)
+        for (int s = 0; s < 6; ++s)
 #pragma unroll
           for (int j = 0; j < 4; ++j)
-            t[s][j] = 4 * half + s < splits ? __ldcg(src + (size_t)(4 * half + s) * M * (N / 4) + 16 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+            t[s][j] = s < splits ? __ldcg(src + (size_t)s * M * (N / 4) + 16 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int s = 0; s < 4; ++s)
+        for (int s = 0; s < 6; ++s)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            v[4 * j] += t[s][j].x; v[4 * j + 1] += t[s][j].y; v[4 * j + 2] += t[s][j].z; v[4 * j + 3] += t[s][j].w;
+          }
+      }
+      if (splits > 6) {
+        float4 t[2][4];
+#pragma unroll
+        for (int s = 0; s < 2; ++s)
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            t[s][j] = 6 + s < splits ? __ldcg(src + (size_t)(6 + s) * M * (N / 4) + 16 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s = 0; s < 2; ++s)
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             v[4 * j] += t[s][j].x; v[4 * j + 1] += t[s][j].y; v[4 * j + 2] += t[s][j].z; v[4 * j + 3] += t[s][j].w;
