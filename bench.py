@@ -284,11 +284,16 @@ def run_ours(args, cfg):
                      "value": whole_job_value(n_e * T, world, sus_ms), "clocks": clk2}
 
     # ---- per-kernel CUDA-event breakdown over another K steps (same kernels, event pairs around each)
-    g.profile(True)
-    for _ in range(K):
-        step()
-    prof = g.profile_read()
-    g.profile(False)
+    # Two passes, and for every family the faster of the two: one stalled launch (seen once: 2.9 ms on a 9 us kernel)
+    # would otherwise decide which family counts as the dominant one.
+    passes = []
+    for _ in range(2):
+        g.profile(True)
+        for _ in range(K):
+            step()
+        passes.append(g.profile_read())
+        g.profile(False)
+    prof = {k: min((p[k] for p in passes if k in p), key=lambda v: v[0] / max(v[1], 1)) for k in passes[0]}
 
     # ---- the pre-processing kernel of Section 5.1 on n_e pairs of synthetic raw frames (bytes = two raw frames and the
     # previous state read, the new state written); the inputs (over 200 MB at n_e = 1024) exceed L2
@@ -375,8 +380,8 @@ def run_ours(args, cfg):
     work, P = kernel_work(cfg)
     tot = sum(ms for ms, _ in prof.values())
     shares = {k: {"ms_per_step": ms / K, "launches_per_step": n / K, "share": ms / tot} for k, (ms, n) in prof.items()}
-    dom = max(prof, key=lambda k: prof[k][0])
-    bound, amount, logical = work.get(dom, ("hbm", 0.0, 1))
+    dom = max((k for k in prof if k in work and work[k][1] > 0), key=lambda k: prof[k][0])
+    bound, amount, logical = work[dom]
     dom_ms = prof[dom][0] / K / logical                    # device time of one logical launch
     if bound == "tensor":
         ach, peak, unit = amount / (dom_ms * 1e-3) / 1e12, pk["bf16"], "TFLOP/s"
