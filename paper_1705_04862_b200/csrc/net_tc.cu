@@ -1498,8 +1498,10 @@ __global__ void __launch_bounds__(256) fc_finish_kernel(const float* __restrict_
 // and, from the rounded values, its share of the A + 1 head dot products (256 of the 512 hidden units) as
 // hp[column tile][m][k]; heads_sample_kernel adds the two shares.
 // Warps 0-3 move the accumulator, one thread of warp 4 streams the operands (tiled bulk copies), lane 0 of warp 8
-// issues the MMAs; warps 0-7 share the finishing phase.
-constexpr int FCC_BN = 256, FCC_STAGES = 4, FCC_MAX_SPLITS = 8, FCC_THREADS = 288, FCC_HP_LD = 32;
+// issues the MMAs; all twelve warps share the finishing phase (warps 9-11 are there only for it: with two rows per
+// warp a CTA's 21 or 22 rows then take one pass, and a pass costs a round trip to L2 however few rows it has).
+constexpr int FCC_BN = 256, FCC_STAGES = 4, FCC_MAX_SPLITS = 8, FCC_THREADS = 384, FCC_HP_LD = 32;
+constexpr int FCC_FIN_ROWS = 2 * (FCC_THREADS / 32);      // rows of the finishing phase per pass: 24 >= ceil(128 / 6)
 constexpr uint32_t FCC_STAGE_BYTES = TC_BM * 128 + FCC_BN * 128, FCC_ACC_BYTES = TC_BM * FCC_BN * 4;
 constexpr uint32_t FCC_HEADW_BYTES = 33 * FCC_BN * 2;
 static_assert(FCC_ACC_BYTES <= FCC_STAGES * FCC_STAGE_BYTES, "the parked accumulator reuses the operand stages");
@@ -1585,7 +1587,7 @@ tc_fc_cluster_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
       }
       if (ok) mma_commit(&sh.acc_full);
     }
-  } else {
+  } else if (warp < 4) {
     // While the K slice is being multiplied these four warps have nothing to wait for yet: they bring in the head
     // weights of this column tile (row k = policy row k, k < A, 16-byte aligned, or the value row, k = A, which follows
     // the policy biases in the parameter vector and is only 2-byte aligned; 256 bf16 each).  The weights are several
@@ -1640,11 +1642,11 @@ tc_fc_cluster_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_cons
   __syncwarp();
   cluster_sync_all();
   // ---------------- this CTA's share of the tile's rows: sum over the cluster, bias, ReLU, heads ----------------
-  // rows [128 rank / splits, 128 (rank + 1) / splits), sixteen at a time; thread (rl, cg) owns the 16-byte chunks
+  // rows [128 rank / splits, 128 (rank + 1) / splits), two per warp; thread (rl, cg) owns the 16-byte chunks
   // cg, cg + 16, cg + 32, cg + 48 of row rl, i.e. columns 4 (cg + 16 j) .. + 3: the sixteen threads of a row read
   // 256 contiguous bytes at a time
   const int row_lo = TC_BM * rank / splits, row_hi = TC_BM * (rank + 1) / splits;
-  for (int row0 = row_lo + 2 * warp; warp < 8 && row0 < row_hi; row0 += 16) {
+  for (int row0 = row_lo + 2 * warp; row0 < row_hi; row0 += FCC_FIN_ROWS) {
     const int cg = lane & 15;
     const uint32_t row = (uint32_t)(row0 + (lane >> 4));
     const bool live = (int)row < row_hi;
